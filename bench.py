@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the BMU-search hot path (som_norms + som_bmu) on synthetic MeSH-shaped batches.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch: som_norms (norm pass) followed by
+som_bmu (plan, fused search, combine/finalize).  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_24067_b200 import synth  # noqa: E402
+
+# Peak of the plain FP32 pipe that bounds the search: SMs x 128 lanes x max SM clock,
+# one add per lane per clock (the search executes adds, no multiplies).
+FP32_LANES_PER_SM = 128
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return FALLBACK_HBM_GBS, 1965.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        self.t0 = self.t1 = None
+
+    def begin(self):
+        self.t0 = time.time()
+
+    def end(self):
+        self.t1 = time.time()
+
+    def close(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.flush()
+        rows = []
+        import datetime
+        for line in open(self.f.name):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[3], parts[4:9]))
+            except Exception:
+                continue
+        os.unlink(self.f.name)
+        inside = [r for r in rows if self.t0 is not None and self.t0 - 0.05 <= r[0] <= self.t1 + 0.05]
+        use = inside if inside else rows
+        if not use:
+            return out
+        out["samples"] = len(inside)
+        out["sm_mhz"] = float(np.median([r[1] for r in use]))
+        out["sm_max_mhz"] = float(use[0][2])
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in use:
+            for nm, val in zip(names, r[4][1:]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def _dist_env():
+    ws = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    lr = int(os.environ.get("LOCAL_RANK", "0"))
+    return ws, rank, lr
+
+
+def _oracle_rate(w: synth.Workload, W_host_slab: np.ndarray, m_slab: int, indptr: np.ndarray,
+                 indices: np.ndarray, target_s: float):
+    """Time the CPU oracle on a bounded sample of the workload; returns (samples/s, description)."""
+    from oracle import som_oracle as orc
+    cores = orc.threads()
+    nn = orc.norms(W_host_slab, w.V, m_slab)  # norm pass not timed (GPU arm reports it separately)
+    n_probe = min(256, indptr.size - 1)
+    t = time.perf_counter()
+    orc.bmu(W_host_slab, w.V, m_slab, indptr[:n_probe + 1], indices, norms_=nn)
+    dt = max(time.perf_counter() - t, 1e-6)
+    n = int(max(n_probe, min(indptr.size - 1, n_probe * target_s / dt)))
+    t = time.perf_counter()
+    orc.bmu(W_host_slab, w.V, m_slab, indptr[:n + 1], indices, norms_=nn)
+    dt = time.perf_counter() - t
+    rate = n / dt * (m_slab / w.M)
+    desc = "first %d samples of the batch x %d of %d neurons (rate scaled by the neuron fraction), %d threads" % (
+        n, m_slab, w.M, cores)
+    return rate, cores, desc, dt
+
+
+def run_reference(args, w: synth.Workload):
+    """The CPU oracle as it stands, timed on host cores, on bounded samples of the workload."""
+    ws, rank, _ = _dist_env()
+    if rank != 0:
+        return
+    m_slab = min(w.M, 4096)
+    # the slab is the first m_slab neurons of the configured codebook
+    W_host = synth.codebook_slab(w.V, w.M, 0, m_slab, w.seed).numpy()
+    n_gen = min(w.batch, 200_000)
+    b = synth.sample_csr(n_gen, w.V, w.lam, w.seed)
+    indptr, indices = b.indptr.numpy(), b.indices.numpy()
+    per_step = max(1.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    rates, desc, cores = [], "", 1
+    for i in range(args.warmup + args.steps):
+        rate, cores, desc, dt = _oracle_rate(w, W_host, m_slab, indptr, indices, per_step)
+        if i >= args.warmup:
+            rates.append(rate)
+    value = float(np.mean(rates))
+    line = {
+        "impl": "reference", "metric": "bmu_samples_per_s", "value": value, "unit": "samples/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1000.0 * w.batch / value, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": 1 + w.lam},
+        "cpu_baseline": {"value": value, "unit": "samples/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w: synth.Workload):
+    ws, rank, lr = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
+    torch.cuda.set_device(lr)
+    dev = torch.device("cuda", lr)
+    dist = None
+    if ws > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2608_24067_b200 import som
+
+    hbm_gbs, sm_max_mhz, peak_src = _peaks()
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    add_peak = sm_count * FP32_LANES_PER_SM * sm_max_mhz * 1e6  # adds/s
+
+    # ---- inputs (synthetic, resident in HBM) -------------------------------------------------
+    W = torch.empty(w.V * w.M, dtype=torch.float32, device=dev)
+    synth.fill_codebook(w.V, w.M, w.seed, out=W)
+    n_batches = max(1, min(4, w.N // w.batch))
+    batches = []
+    for bi in range(n_batches):
+        first = (rank * n_batches + bi) * w.batch  # each rank (replica) gets its own samples
+        batches.append(synth.sample_csr(w.batch, w.V, w.lam, w.seed, zipf_s=w.zipf_s, device=dev,
+                                        first_sample=first))
+    nnz_mean = float(np.mean([b.nnz / b.n for b in batches]))
+    h = som.Som(w.V, w.M, W)
+    if args.variant is not None:
+        h.set_option(0, args.variant)
+    out_bmu = torch.empty(w.batch, dtype=torch.int32, device=dev)
+    out_dist = torch.empty(w.batch, dtype=torch.float32, device=dev)
+
+    def step(i):
+        b = batches[i % n_batches]
+        h.norms()
+        h.bmu(b.indptr, b.indices, out_bmu, out_dist)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------------------
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(lr) if rank == 0 else None
+    h.set_timing(True)
+    l0 = h.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    if sampler:
+        sampler.begin()
+    e0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record()
+    barrier()
+    if sampler:
+        sampler.end()
+    ms_total = e0.elapsed_time(e1)
+    launches = h.launch_count() - l0
+    phases = h.get_timing()
+    h.set_timing(False)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = ws * w.batch / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host entry point --------------------------------------------
+    hb = [(b.indptr.cpu().pin_memory(), b.indices.cpu().pin_memory()) for b in batches]
+    h_bmu = torch.empty(w.batch, dtype=torch.int32).pin_memory()
+    h_dist = torch.empty(w.batch, dtype=torch.float32).pin_memory()
+    e2e_steps = max(1, min(args.steps, 5))
+
+    def e2e_step(i):
+        ip, ix = hb[i % n_batches]
+        h.norms()
+        h.bmu_host(ip, ix, h_bmu, h_dist)
+
+    e2e_step(0)
+    barrier()
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i + 1)
+    e1.record()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1) / e2e_steps], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item())
+    e2e_value = ws * w.batch / (e2e_ms * 1e-3)
+    h2d = int(np.mean([ip.numel() * 4 + ix.numel() * 4 for ip, ix in hb]))
+    d2h = w.batch * 8
+
+    clocks = sampler.close() if sampler else None
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the fused search) -------------------------------------
+    adds = w.batch * nnz_mean * w.M  # nominal neuron-feature accumulations per launch
+    search_s = max(phases["search_ms"], 1e-6) * 1e-3
+    achieved = adds / search_s
+    alg_bytes = w.V * w.M * 4 + sum(b.nnz * 4 + (b.n + 1) * 4 for b in batches) / n_batches + w.batch * 8
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        traffic = json.load(open(tpath)).get(w.name)
+    roofline = {
+        "bound": "alu", "kernel": "fused BMU search", "achieved": achieved / 1e12, "peak": add_peak / 1e12,
+        "unit": "TFLOP/s", "frac": achieved / add_peak, "traffic": traffic,
+        "peak_source": "%d SMs x %d fp32 lanes x %.0f MHz (%s clock)" % (sm_count, FP32_LANES_PER_SM, sm_max_mhz, peak_src),
+        "search_ms": phases["search_ms"], "algorithmic_bytes": alg_bytes,
+        "hbm_time_at_peak_ms": alg_bytes / (hbm_gbs * 1e9) * 1e3, "hbm_peak_gbs": hbm_gbs,
+        "norms_ms": phases["norms_ms"],
+        "norms_hbm_frac": (w.V * w.M * 4 / max(phases["norms_ms"], 1e-6) / 1e6) / hbm_gbs,
+        "plan_ms": phases["plan_ms"], "finalize_ms": phases["finalize_ms"],
+        "step_frac_of_alu_roofline": (adds / add_peak) / (ms_per_step * 1e-3),
+    }
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ----------------------
+    cpu = None
+    if ws == 1 and not args.no_cpu_baseline:
+        m_slab = min(w.M, 4096)
+        Wh = W.view(w.V, w.M)[:, :m_slab].contiguous().cpu().numpy()
+        b = batches[0]
+        n_take = min(b.n, 100_000)
+        ip = b.indptr[:n_take + 1].cpu().numpy()
+        ix = b.indices[:int(b.indptr[n_take])].cpu().numpy()
+        rate, cores, desc, _ = _oracle_rate(w, Wh, m_slab, ip, ix, 12.0)
+        cpu = {"value": rate, "unit": "samples/s", "cores": cores, "kind": "oracle", "sample": desc}
+
+    line = {
+        "metric": "bmu_samples_per_s", "value": value, "unit": "samples/s", "n_gpus": ws,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": nnz_mean,
+                   "step": "som_norms + som_bmu on one batch", "replicas": ws,
+                   "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
+                       w.V * w.M * 4 / 1e6, batches[0].nnz * 4 / 1e6) if w.V * w.M * 4 > 126e6 else
+                   "inputs smaller than L2: steps rotate over %d distinct batches, no flush" % n_batches},
+        "accumulations_per_s": ws * adds / (ms_per_step * 1e-3),
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="index into the five workloads (default 1: 64x64)")
+    ap.add_argument("--variant", type=int, default=None, help="search kernel variant (library option 0)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

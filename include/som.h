@@ -1,0 +1,145 @@
+/*
+ * som.h - C ABI of the B200 best-matching-unit (BMU) search for sparse-binary
+ * self-organizing maps with a feature-major codebook.
+ *
+ * The operation (paper, Section 3.1, Eq. 1): for a binary sample x with active feature
+ * set S and M prototypes w_i,
+ *
+ *     BMU(x) = argmin_i ||x - w_i||^2 = argmin_i ( ||w_i||^2 - 2 * sum_{v in S} w_i[v] ),
+ *
+ * ties broken to the lowest neuron index (Section 3.1).  The codebook is stored
+ * feature-major (Section 3.2): weight (v, i) lives at W[v*M + i], so the M weights of one
+ * feature are contiguous.  Samples arrive as sparse-binary CSR (Section 4.2): a row-pointer
+ * array and one concatenated array of ascending column ids, values implicit 1.
+ *
+ * Conventions
+ *   - Every function returns an int status (SOM_OK == 0).  Nothing throws, prints or exits.
+ *   - "device pointer" = memory of the CUDA device that was current in som_create;
+ *     "host pointer" = ordinary process memory.  The library never takes ownership of a
+ *     caller's buffer.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     som_norms / som_bmu only enqueue work on it and return without synchronising,
+ *     except that growing the handle's workspace (first call, or a larger batch than any
+ *     before) allocates device memory, which may synchronise the device once.
+ *   - Thread safety: one handle must not be used from two host threads at once, and two
+ *     calls on the same handle must not overlap on the GPU (they share the workspace);
+ *     issue them on one stream or order the streams yourself.
+ */
+#ifndef SOM_B200_H
+#define SOM_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct som_handle som_handle; /* opaque */
+
+enum som_status {
+    SOM_OK = 0,
+    SOM_ERR_INVALID_ARG = 1, /* null pointer, V <= 0, M <= 0, n < 0, misaligned codebook */
+    SOM_ERR_NORMS_STALE = 2, /* som_bmu called before som_norms                           */
+    SOM_ERR_UNSUPPORTED = 3, /* size outside what the kernels index (see som_create)      */
+    SOM_ERR_CUDA = 4,        /* a CUDA call failed; see som_last_cuda_error               */
+    SOM_ERR_BAD_CSR = 5,     /* som_validate_csr found a malformed batch                  */
+    SOM_ERR_NO_DEVICE = 6    /* no CUDA device / device is not sm_100                     */
+};
+
+/*
+ * som_create - bind a handle to a codebook (Section 3.2, the feature-major codebook).
+ *   out         host pointer; receives the handle.
+ *   V           number of features, 1 <= V < 2^31.
+ *   M           number of neurons,  1 <= M < 2^31.
+ *   d_codebook  DEVICE pointer, fp32, V*M elements, element (v,i) at v*M + i, 16-byte
+ *               aligned.  BORROWED: the caller keeps ownership, must keep it alive while
+ *               the handle lives, and may rewrite it in place between calls; after any
+ *               rewrite som_norms must run again before the next som_bmu.
+ * M need not be a multiple of 4, but only then do the 128-bit vector paths apply; other
+ * M take a scalar-load kernel.  Allocates M*8 bytes of device memory for the norms.
+ */
+int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook);
+
+/*
+ * som_norms - recompute ||w_i||^2 for all M neurons (the norm term of Eq. 1; the paper's
+ * "negligible norm pass", Section 5.7).  One streaming read of the codebook; squares are
+ * accumulated in fp64 in a fixed order (deterministic) and stored as fp32.
+ * Must be called once after som_create and again after every codebook update.
+ */
+int som_norms(som_handle* h, void* stream);
+
+/*
+ * som_bmu - BMU search for one batch (Section 3.3; Algorithm 2, steps 4-7, best unit only).
+ *   d_indptr    DEVICE pointer, int32 [n_samples+1]; row s owns indices
+ *               [d_indptr[s], d_indptr[s+1]) of d_indices.  d_indptr[0] may be any offset.
+ *   d_indices   DEVICE pointer, int32; inside each row ascending, distinct, in [0, V).
+ *               These are preconditions (the paper sorts ascending, Section 3.1) and are
+ *               NOT checked here; som_validate_csr checks them.
+ *   n_samples   0 <= n_samples < 2^31; 0 is a successful no-op.
+ *   d_bmu       DEVICE pointer, int32 [n_samples]  out: index of the nearest neuron,
+ *               lowest index among exact fp32 ties.
+ *   d_min_dist  DEVICE pointer, fp32 [n_samples]   out: the full squared Euclidean distance
+ *               ||x - w_bmu||^2 = |S| - 2*sum_{v in S} w_bmu[v] + ||w_bmu||^2 (left side of
+ *               Eq. 1, no square root), recomputed for the winner in fp64 and rounded once.
+ * A sample with no active feature gets argmin ||w_i||^2 and that norm.
+ * Scores are accumulated in fp32 in a fixed order, so outputs are bit-identical from run
+ * to run for the same inputs.
+ */
+int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+            int32_t* d_bmu, float* d_min_dist, void* stream);
+
+/*
+ * som_bmu_host - the same search with HOST buffers: copies the CSR batch to device staging
+ * memory owned by the handle, runs som_bmu, copies both outputs back, all enqueued on
+ * `stream`, then synchronises that stream before returning.  h_* pointers are host memory
+ * (pinned memory makes the copies asynchronous and faster); h_indptr[0] must be 0.
+ * The paper has the corpus stream from host memory into the kernels (Section 4.2).
+ */
+int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,
+                 int32_t* h_bmu, float* h_min_dist, void* stream);
+
+/*
+ * som_validate_csr - check the preconditions of som_bmu on a device-resident batch:
+ * non-decreasing row pointers, ids in [0, V), strictly ascending inside each row
+ * (Section 4.2, the sparse-binary CSR container).  Synchronises `stream`.
+ * Returns SOM_OK or SOM_ERR_BAD_CSR.
+ */
+int som_validate_csr(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices,
+                     int64_t n_samples, void* stream);
+
+/*
+ * som_get_norms - copy the M fp32 norms computed by the last som_norms into a DEVICE buffer
+ * (enqueued on `stream`).  For tests and for callers that want ||w_i||^2 (Eq. 1).
+ */
+int som_get_norms(som_handle* h, float* d_out, void* stream);
+
+/* som_destroy - free the handle, its norms and workspace.  NULL is accepted. */
+int som_destroy(som_handle* h);
+
+/* Human-readable name of a status code (static storage). */
+const char* som_status_string(int status);
+
+/* cudaError_t value of the last failed CUDA call on this handle (0 if none). */
+int som_last_cuda_error(const som_handle* h);
+
+/*
+ * Instrumentation (no paper counterpart; used by the benchmark).
+ * som_set_timing(h, 1) makes each som_norms / som_bmu record CUDA events around its
+ * phases on the caller's stream (switching it on or off restarts the record).
+ * som_get_timing, called after the stream has been synchronised, returns the mean over the
+ * calls recorded since then (the most recent 32 of each kind at most):
+ *   out_ms[0] som_norms total, out_ms[1] som_bmu total, out_ms[2] som_bmu plan phase,
+ *   out_ms[3] som_bmu search kernel(s), out_ms[4] som_bmu finalize.
+ * som_launch_count returns how many kernels this handle has launched since creation.
+ * som_set_option tunes kernel selection: key 0 = search kernel variant
+ * (0 auto, 1 direct-load kernel, 2 shared-memory row-table kernel).
+ */
+int som_set_timing(som_handle* h, int enable);
+int som_get_timing(som_handle* h, float* out_ms, int n_out);
+int64_t som_launch_count(const som_handle* h);
+int som_set_option(som_handle* h, int key, int64_t value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOM_B200_H */

@@ -1,0 +1,285 @@
+// Host side of the C ABI declared in include/som.h: handle life cycle, argument checks,
+// workspace management, phase timing and kernel selection.  All compute is in the kernels.
+#include <new>
+
+#include "som_internal.cuh"
+
+namespace {
+
+struct DeviceGuard {
+    int prev;
+    bool switched;
+    explicit DeviceGuard(int dev) : prev(-1), switched(false)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
+            cudaSetDevice(dev);
+            switched = true;
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+int ensure_bytes(som_handle* h, void** buf, size_t* have, size_t need)
+{
+    if (need <= *have) return SOM_OK;
+    if (*buf) {
+        SOM_CK(h, cudaFree(*buf));  // synchronises: earlier work using the buffer is done
+        *buf = nullptr;
+        *have = 0;
+    }
+    need = som_align_up(need + need / 8, 1 << 20);
+    SOM_CK(h, cudaMalloc(buf, need));
+    *have = need;
+    return SOM_OK;
+}
+
+int ensure_events(som_handle* h)
+{
+    if (h->events_made) return SOM_OK;
+    for (int i = 0; i < SOM_N_EVENTS; ++i) SOM_CK(h, cudaEventCreate(&h->ev[i]));
+    h->events_made = 1;
+    return SOM_OK;
+}
+
+// Events live in a ring of SOM_EV_RING calls so that the mean over a timed region can be read
+// after one synchronisation at its end.
+inline int mark(som_handle* h, int64_t call, int slot, cudaStream_t st)
+{
+    if (!h->timing) return SOM_OK;
+    SOM_CK(h, cudaEventRecord(h->ev[(call % SOM_EV_RING) * SOM_EV_PER_CALL + slot], st));
+    return SOM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook)
+{
+    if (!out) return SOM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (V <= 0 || M <= 0 || !d_codebook) return SOM_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_codebook) & 15u) != 0) return SOM_ERR_INVALID_ARG;
+    if (M >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SOM_ERR_NO_DEVICE;
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return SOM_ERR_NO_DEVICE;
+    if (major != 10) return SOM_ERR_NO_DEVICE;  // the kernels are built for sm_100a only
+
+    som_handle* h = new (std::nothrow) som_handle();
+    if (!h) return SOM_ERR_INVALID_ARG;
+    h->device = dev;
+    h->sm_count = sms;
+    h->V = V;
+    h->M = M;
+    h->W = d_codebook;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->norm64), (size_t)M * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->norm32), (size_t)M * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->hnorm), (size_t)M * sizeof(float));
+    if (e != cudaSuccess) {
+        som_destroy(h);
+        return SOM_ERR_CUDA;
+    }
+    *out = h;
+    return SOM_OK;
+}
+
+int som_destroy(som_handle* h)
+{
+    if (!h) return SOM_OK;
+    DeviceGuard g(h->device);
+    cudaFree(h->norm64);
+    cudaFree(h->norm32);
+    cudaFree(h->hnorm);
+    cudaFree(h->ws);
+    cudaFree(h->stage);
+    if (h->events_made)
+        for (int i = 0; i < SOM_N_EVENTS; ++i) cudaEventDestroy(h->ev[i]);
+    delete h;
+    return SOM_OK;
+}
+
+int som_norms(som_handle* h, void* stream)
+{
+    if (!h) return SOM_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, som_norms_workspace_bytes(h));
+    if (rc) return rc;
+    if (h->timing && (rc = ensure_events(h))) return rc;
+    if ((rc = mark(h, h->ev_norms_calls, EV_NORMS_BEGIN, st))) return rc;
+    if ((rc = som_launch_norms(h, st))) return rc;
+    if ((rc = mark(h, h->ev_norms_calls, EV_NORMS_END, st))) return rc;
+    if (h->timing) h->ev_norms_calls += 1;
+    h->norms_valid = 1;
+    return SOM_OK;
+}
+
+int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+            int32_t* d_bmu, float* d_min_dist, void* stream)
+{
+    if (!h || n_samples < 0) return SOM_ERR_INVALID_ARG;
+    if (n_samples == 0) return SOM_OK;
+    if (!d_indptr || !d_bmu || !d_min_dist) return SOM_ERR_INVALID_ARG;
+    if (n_samples >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
+    if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+    const size_t key_bytes = som_align_up((size_t)n_samples * sizeof(unsigned long long), 256);
+    int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, key_bytes);
+    if (rc) return rc;
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(h->ws);
+
+    if (h->timing && (rc = ensure_events(h))) return rc;
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
+    SOM_CK(h, cudaMemsetAsync(keys, 0xFF, (size_t)n_samples * sizeof(unsigned long long), st));
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+    if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, st))) return rc;
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+    if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, st)))
+        return rc;
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
+    if (h->timing) h->ev_bmu_calls += 1;
+    return SOM_OK;
+}
+
+int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,
+                 int32_t* h_bmu, float* h_min_dist, void* stream)
+{
+    if (!h || n_samples < 0) return SOM_ERR_INVALID_ARG;
+    if (n_samples == 0) return SOM_OK;
+    if (!h_indptr || !h_bmu || !h_min_dist) return SOM_ERR_INVALID_ARG;
+    if (h_indptr[0] != 0 || h_indptr[n_samples] < 0) return SOM_ERR_INVALID_ARG;
+    const int64_t nnz = h_indptr[n_samples];
+    if (nnz > 0 && !h_indices) return SOM_ERR_INVALID_ARG;
+    if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+    const size_t b_ptr = som_align_up((size_t)(n_samples + 1) * 4, 256);
+    const size_t b_idx = som_align_up((size_t)(nnz > 0 ? nnz : 1) * 4, 256);
+    const size_t b_out = som_align_up((size_t)n_samples * 4, 256);
+    int rc = ensure_bytes(h, &h->stage, &h->stage_bytes, b_ptr + b_idx + 2 * b_out);
+    if (rc) return rc;
+    char* base = reinterpret_cast<char*>(h->stage);
+    int32_t* d_ptr = reinterpret_cast<int32_t*>(base);
+    int32_t* d_idx = reinterpret_cast<int32_t*>(base + b_ptr);
+    int32_t* d_bmu = reinterpret_cast<int32_t*>(base + b_ptr + b_idx);
+    float* d_dist = reinterpret_cast<float*>(base + b_ptr + b_idx + b_out);
+    SOM_CK(h, cudaMemcpyAsync(d_ptr, h_indptr, (size_t)(n_samples + 1) * 4, cudaMemcpyHostToDevice, st));
+    if (nnz > 0)
+        SOM_CK(h, cudaMemcpyAsync(d_idx, h_indices, (size_t)nnz * 4, cudaMemcpyHostToDevice, st));
+    rc = som_bmu(h, d_ptr, d_idx, n_samples, d_bmu, d_dist, stream);
+    if (rc) return rc;
+    SOM_CK(h, cudaMemcpyAsync(h_bmu, d_bmu, (size_t)n_samples * 4, cudaMemcpyDeviceToHost, st));
+    SOM_CK(h, cudaMemcpyAsync(h_min_dist, d_dist, (size_t)n_samples * 4, cudaMemcpyDeviceToHost, st));
+    SOM_CK(h, cudaStreamSynchronize(st));
+    return SOM_OK;
+}
+
+int som_validate_csr(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices,
+                     int64_t n_samples, void* stream)
+{
+    if (!h || n_samples < 0) return SOM_ERR_INVALID_ARG;
+    if (n_samples == 0) return SOM_OK;
+    if (!d_indptr) return SOM_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int rc = ensure_bytes(h, &h->stage, &h->stage_bytes, 256);
+    if (rc) return rc;
+    int* d_flag = reinterpret_cast<int*>(h->stage);
+    SOM_CK(h, cudaMemsetAsync(d_flag, 0, sizeof(int), st));
+    if ((rc = som_launch_validate(h, d_indptr, d_indices, n_samples, d_flag, st))) return rc;
+    int flag = 0;
+    SOM_CK(h, cudaMemcpyAsync(&flag, d_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
+    SOM_CK(h, cudaStreamSynchronize(st));
+    return flag ? SOM_ERR_BAD_CSR : SOM_OK;
+}
+
+int som_get_norms(som_handle* h, float* d_out, void* stream)
+{
+    if (!h || !d_out) return SOM_ERR_INVALID_ARG;
+    if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
+    DeviceGuard g(h->device);
+    SOM_CK(h, cudaMemcpyAsync(d_out, h->norm32, (size_t)h->M * sizeof(float), cudaMemcpyDeviceToDevice,
+                              reinterpret_cast<cudaStream_t>(stream)));
+    return SOM_OK;
+}
+
+const char* som_status_string(int status)
+{
+    switch (status) {
+        case SOM_OK: return "SOM_OK";
+        case SOM_ERR_INVALID_ARG: return "SOM_ERR_INVALID_ARG";
+        case SOM_ERR_NORMS_STALE: return "SOM_ERR_NORMS_STALE";
+        case SOM_ERR_UNSUPPORTED: return "SOM_ERR_UNSUPPORTED";
+        case SOM_ERR_CUDA: return "SOM_ERR_CUDA";
+        case SOM_ERR_BAD_CSR: return "SOM_ERR_BAD_CSR";
+        case SOM_ERR_NO_DEVICE: return "SOM_ERR_NO_DEVICE";
+        default: return "SOM_ERR_UNKNOWN";
+    }
+}
+
+int som_last_cuda_error(const som_handle* h) { return h ? h->last_cuda_error : 0; }
+
+int som_set_timing(som_handle* h, int enable)
+{
+    if (!h) return SOM_ERR_INVALID_ARG;
+    h->timing = enable ? 1 : 0;
+    h->ev_norms_calls = h->ev_bmu_calls = 0;
+    return SOM_OK;
+}
+
+int som_get_timing(som_handle* h, float* out_ms, int n_out)
+{
+    if (!h || !out_ms || n_out < 0) return SOM_ERR_INVALID_ARG;
+    float v[5] = {0, 0, 0, 0, 0};
+    DeviceGuard g(h->device);
+    auto ev = [&](int64_t call, int slot) { return h->ev[(call % SOM_EV_RING) * SOM_EV_PER_CALL + slot]; };
+    auto span = [&](int64_t call, int a, int b, float* acc) -> cudaError_t {
+        float ms = 0.f;
+        cudaError_t e = cudaEventElapsedTime(&ms, ev(call, a), ev(call, b));
+        *acc += ms;
+        return e;
+    };
+    {
+        const int64_t c1 = h->ev_norms_calls, c0 = c1 > SOM_EV_RING ? c1 - SOM_EV_RING : 0;
+        for (int64_t c = c0; c < c1; ++c) SOM_CK(h, span(c, EV_NORMS_BEGIN, EV_NORMS_END, &v[0]));
+        if (c1 > c0) v[0] /= (float)(c1 - c0);
+    }
+    {
+        const int64_t c1 = h->ev_bmu_calls, c0 = c1 > SOM_EV_RING ? c1 - SOM_EV_RING : 0;
+        for (int64_t c = c0; c < c1; ++c) {
+            SOM_CK(h, span(c, EV_BMU_BEGIN, EV_BMU_END, &v[1]));
+            SOM_CK(h, span(c, EV_BMU_BEGIN, EV_BMU_PLAN_END, &v[2]));
+            SOM_CK(h, span(c, EV_BMU_PLAN_END, EV_BMU_SEARCH_END, &v[3]));
+            SOM_CK(h, span(c, EV_BMU_SEARCH_END, EV_BMU_END, &v[4]));
+        }
+        if (c1 > c0)
+            for (int i = 1; i < 5; ++i) v[i] /= (float)(c1 - c0);
+    }
+    for (int i = 0; i < n_out && i < 5; ++i) out_ms[i] = v[i];
+    return SOM_OK;
+}
+
+int64_t som_launch_count(const som_handle* h) { return h ? h->launches : 0; }
+
+int som_set_option(som_handle* h, int key, int64_t value)
+{
+    if (!h) return SOM_ERR_INVALID_ARG;
+    if (key == 0) {
+        if (value < 0 || value > 2) return SOM_ERR_INVALID_ARG;
+        h->opt_variant = value;
+        return SOM_OK;
+    }
+    return SOM_ERR_INVALID_ARG;
+}
+
+}  // extern "C"

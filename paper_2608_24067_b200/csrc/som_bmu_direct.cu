@@ -1,0 +1,163 @@
+// Direct-load BMU search kernel, winner finalisation and CSR validation.
+//
+// k_bmu_direct is the simplest complete statement of the fused search (Section 3.3):
+// a warp owns one sample at a time and a block of 32*VEC neurons; every lane keeps VEC
+// score accumulators in registers, seeded with ||w_i||^2 / 2, and for each active feature v
+// subtracts the contiguous segment W[v*M + i0 .. i0+VEC) fetched with one 128-bit load
+// (feature-major layout: the warp's 32 loads cover 512 contiguous bytes).  The per-block
+// argmin is a warp-shuffle reduction on (score, index) with ties to the lower index, and
+// the cross-block combine is a 64-bit atomicMin on an order-preserving packed key, which is
+// commutative and associative and therefore deterministic.  No N x M score block is ever
+// written.  It serves every shape (any M, any row length) and is the fallback of the
+// faster row-table kernel.
+#include "som_internal.cuh"
+
+namespace {
+
+constexpr int DIRECT_THREADS = 256;
+constexpr int DIRECT_WARPS = DIRECT_THREADS / 32;
+constexpr int DIRECT_SAMPLES_PER_WARP = 16;
+
+template <int VEC>
+__global__ void __launch_bounds__(DIRECT_THREADS)
+k_bmu_direct(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
+             const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
+             unsigned long long* __restrict__ keys, int64_t neuron_off)
+{
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int64_t i0 = neuron_off + ((int64_t)blockIdx.y * 32 + lane) * VEC;
+    const float inf = __int_as_float(0x7f800000);
+
+    float seed[VEC];
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) seed[k] = (i0 + k < M) ? hnorm[i0 + k] : inf;
+    const bool live = i0 < M;  // with VEC == 4, M % 4 == 0: all four or none
+
+    const int64_t s0 = ((int64_t)blockIdx.x * DIRECT_WARPS + warp) * DIRECT_SAMPLES_PER_WARP;
+    const int64_t s1 = min(n, s0 + DIRECT_SAMPLES_PER_WARP);
+    for (int64_t s = s0; s < s1; ++s) {
+        const int beg = indptr[s];
+        const int end = indptr[s + 1];
+        float acc[VEC];
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) acc[k] = seed[k];
+        for (int base = beg; base < end; base += 32) {
+            const int mine = (base + lane < end) ? indices[base + lane] : 0;
+            const int cnt = min(32, end - base);
+            for (int j = 0; j < cnt; ++j) {
+                const int v = __shfl_sync(0xffffffffu, mine, j);
+                const float* p = W + (int64_t)v * M + i0;
+                if (VEC == 4) {
+                    if (live) {
+                        const float4 w = __ldg(reinterpret_cast<const float4*>(p));
+                        acc[0] -= w.x;
+                        acc[1 % VEC] -= w.y;
+                        acc[2 % VEC] -= w.z;
+                        acc[3 % VEC] -= w.w;
+                    }
+                } else {
+                    if (live) acc[0] -= __ldg(p);
+                }
+            }
+        }
+        float best = acc[0];
+        uint32_t bi = (uint32_t)i0;
+#pragma unroll
+        for (int k = 1; k < VEC; ++k)
+            if (acc[k] < best) { best = acc[k]; bi = (uint32_t)(i0 + k); }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ob = __shfl_down_sync(0xffffffffu, best, off);
+            const uint32_t oi = __shfl_down_sync(0xffffffffu, bi, off);
+            if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+        }
+        if (lane == 0) atomicMin(&keys[s], som_pack_key(best, bi));
+    }
+}
+
+// One thread per sample: unpack the winner and recompute its full squared distance
+// |S| - 2*dot + ||w||^2 (left side of Eq. 1) in fp64, ascending feature order.
+__global__ void k_finalize(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
+                           const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
+                           int64_t n, const unsigned long long* __restrict__ keys,
+                           int32_t* __restrict__ bmu, float* __restrict__ dist)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n) return;
+    const uint32_t idx = (uint32_t)(keys[s] & 0xffffffffull);
+    const int beg = indptr[s];
+    const int end = indptr[s + 1];
+    double dot = 0.0;
+    for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
+    bmu[s] = (int32_t)idx;
+    dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
+}
+
+__global__ void k_validate(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
+                           int64_t n, int V, int* __restrict__ flag)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n) return;
+    const int beg = indptr[s];
+    const int end = indptr[s + 1];
+    bool bad = end < beg || beg < 0;
+    if (!bad) {
+        int prev = -1;
+        for (int j = beg; j < end; ++j) {
+            const int v = indices[j];
+            if (v <= prev || v >= V) { bad = true; break; }
+            prev = v;
+        }
+    }
+    if (bad) atomicExch(flag, 1);
+}
+
+}  // namespace
+
+int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                          unsigned long long* keys, cudaStream_t st)
+{
+    const int vec = (h->M % 4 == 0) ? 4 : 1;
+    const int64_t per_block = (int64_t)DIRECT_WARPS * DIRECT_SAMPLES_PER_WARP;
+    const int64_t gx = (n + per_block - 1) / per_block;
+    const int64_t neurons_per_block = 32 * vec;
+    int64_t gy = (h->M + neurons_per_block - 1) / neurons_per_block;
+    // gridDim.y is limited to 65535: walk the neuron axis in slices
+    const int64_t max_gy = 65535;
+    for (int64_t y0 = 0; y0 < gy; y0 += max_gy) {
+        const int64_t ny = (gy - y0 < max_gy) ? gy - y0 : max_gy;
+        dim3 grid((unsigned)gx, (unsigned)ny);
+        const int64_t neuron_off = y0 * neurons_per_block;
+        if (vec == 4)
+            k_bmu_direct<4><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
+                                                             keys, neuron_off);
+        else
+            k_bmu_direct<1><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
+                                                             keys, neuron_off);
+        SOM_CK(h, cudaGetLastError());
+        h->launches += 1;
+    }
+    return SOM_OK;
+}
+
+int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                        const unsigned long long* keys, int32_t* bmu, float* dist, cudaStream_t st)
+{
+    const int64_t blocks = (n + 255) / 256;
+    k_finalize<<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, keys, bmu,
+                                                 dist);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
+    return SOM_OK;
+}
+
+int som_launch_validate(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                        int* d_flag, cudaStream_t st)
+{
+    const int64_t blocks = (n + 255) / 256;
+    k_validate<<<(unsigned)blocks, 256, 0, st>>>(indptr, indices, n, h->V, d_flag);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
+    return SOM_OK;
+}

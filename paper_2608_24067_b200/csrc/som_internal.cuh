@@ -1,0 +1,76 @@
+// Internal declarations shared by the translation units of the BMU library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/som.h"
+
+#define SOM_EV_PER_CALL 6
+#define SOM_EV_RING 32
+#define SOM_N_EVENTS (SOM_EV_PER_CALL * SOM_EV_RING)
+
+struct som_handle {
+    int device;
+    int sm_count;
+    int32_t V;
+    int64_t M;
+    const float* W;  // borrowed, feature-major
+
+    double* norm64;  // [M] ||w_i||^2 in fp64
+    float* norm32;   // [M] the same rounded to fp32
+    float* hnorm;    // [M] 0.5 * ||w_i||^2, the seed of every score accumulator
+    int norms_valid;
+
+    void* ws;  // grow-only device workspace shared by som_norms / som_bmu
+    size_t ws_bytes;
+    void* stage;  // grow-only device staging for som_bmu_host
+    size_t stage_bytes;
+
+    int last_cuda_error;
+    int timing;
+    int events_made;
+    cudaEvent_t ev[SOM_N_EVENTS];
+    int64_t ev_norms_calls;  // calls recorded since timing was switched on
+    int64_t ev_bmu_calls;
+    int64_t launches;
+    int64_t opt_variant;
+};
+
+// event slots
+enum { EV_NORMS_BEGIN = 0, EV_NORMS_END, EV_BMU_BEGIN, EV_BMU_PLAN_END, EV_BMU_SEARCH_END, EV_BMU_END };
+
+#define SOM_CK(h, call)                                   \
+    do {                                                  \
+        cudaError_t e__ = (call);                         \
+        if (e__ != cudaSuccess) {                         \
+            (h)->last_cuda_error = (int)e__;              \
+            return SOM_ERR_CUDA;                          \
+        }                                                 \
+    } while (0)
+
+static inline size_t som_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Order-preserving map of an fp32 value to uint32 (smaller float -> smaller uint).
+__device__ __forceinline__ uint32_t som_ordered_bits(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// (score, neuron) packed so that an unsigned 64-bit min is the lexicographic
+// (smallest score, then lowest neuron index) min.
+__device__ __forceinline__ unsigned long long som_pack_key(float score, uint32_t neuron)
+{
+    return ((unsigned long long)som_ordered_bits(score) << 32) | (unsigned long long)neuron;
+}
+
+// kernels' host launchers (each returns a som_status)
+int som_launch_norms(som_handle* h, cudaStream_t st);
+int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                          unsigned long long* keys, cudaStream_t st);
+int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                        const unsigned long long* keys, int32_t* bmu, float* dist, cudaStream_t st);
+int som_launch_validate(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                        int* d_flag, cudaStream_t st);
+size_t som_norms_workspace_bytes(const som_handle* h);

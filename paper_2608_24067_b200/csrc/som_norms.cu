@@ -1,0 +1,125 @@
+// Per-neuron squared norms ||w_i||^2 of a feature-major codebook (the norm term of Eq. 1).
+//
+// HBM-bound streaming pass: each thread owns VEC adjacent neurons and walks down the
+// feature rows with 128-bit loads (a warp reads 512 contiguous bytes of one row), several
+// rows in flight.  Squares are accumulated in fp64.  The V axis is split across blockIdx.y
+// so that small maps still fill 148 SMs; the per-split partial sums are combined in a second
+// kernel in ascending split order, which keeps the result independent of scheduling.
+#include "som_internal.cuh"
+
+namespace {
+
+constexpr int NORM_THREADS = 128;
+constexpr int NORM_UNROLL = 8;
+
+template <int VEC>
+__global__ void __launch_bounds__(NORM_THREADS)
+k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_split,
+                double* __restrict__ partial)
+{
+    const int64_t i = ((int64_t)blockIdx.x * NORM_THREADS + threadIdx.x) * VEC;
+    if (i >= M) return;
+    const int v0 = blockIdx.y * rows_per_split;
+    const int v1 = min(V, v0 + rows_per_split);
+    double acc[VEC];
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) acc[k] = 0.0;
+    const float* p = W + (int64_t)v0 * M + i;
+    int v = v0;
+    if (VEC == 4) {
+        for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
+            float4 w[NORM_UNROLL];
+#pragma unroll
+            for (int u = 0; u < NORM_UNROLL; ++u)
+                w[u] = __ldcs(reinterpret_cast<const float4*>(p + (int64_t)u * M));
+#pragma unroll
+            for (int u = 0; u < NORM_UNROLL; ++u) {
+                acc[0] = fma((double)w[u].x, (double)w[u].x, acc[0]);
+                acc[1 % VEC] = fma((double)w[u].y, (double)w[u].y, acc[1 % VEC]);
+                acc[2 % VEC] = fma((double)w[u].z, (double)w[u].z, acc[2 % VEC]);
+                acc[3 % VEC] = fma((double)w[u].w, (double)w[u].w, acc[3 % VEC]);
+            }
+            p += (int64_t)NORM_UNROLL * M;
+        }
+        for (; v < v1; ++v) {
+            float4 w = __ldcs(reinterpret_cast<const float4*>(p));
+            acc[0] = fma((double)w.x, (double)w.x, acc[0]);
+            acc[1 % VEC] = fma((double)w.y, (double)w.y, acc[1 % VEC]);
+            acc[2 % VEC] = fma((double)w.z, (double)w.z, acc[2 % VEC]);
+            acc[3 % VEC] = fma((double)w.w, (double)w.w, acc[3 % VEC]);
+            p += M;
+        }
+    } else {
+        for (; v < v1; ++v) {
+            float w = __ldcs(p);
+            acc[0] = fma((double)w, (double)w, acc[0]);
+            p += M;
+        }
+    }
+    double* out = partial + (int64_t)blockIdx.y * M + i;
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) out[k] = acc[k];
+}
+
+__global__ void k_norms_combine(const double* __restrict__ partial, int64_t M, int splits,
+                                double* __restrict__ norm64, float* __restrict__ norm32,
+                                float* __restrict__ hnorm)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    double s = 0.0;
+    for (int k = 0; k < splits; ++k) s += partial[(int64_t)k * M + i];
+    norm64[i] = s;
+    norm32[i] = (float)s;
+    hnorm[i] = (float)(0.5 * s);
+}
+
+struct NormPlan {
+    int vec;
+    int splits;
+    int rows_per_split;
+    int64_t col_blocks;
+};
+
+NormPlan plan_norms(const som_handle* h)
+{
+    NormPlan p;
+    p.vec = (h->M % 4 == 0) ? 4 : 1;
+    const int64_t col_threads = (h->M + p.vec - 1) / p.vec;
+    p.col_blocks = (col_threads + NORM_THREADS - 1) / NORM_THREADS;
+    // aim for ~16 resident blocks per SM worth of work, at least 16 rows per split
+    int64_t want = ((int64_t)h->sm_count * 16 + p.col_blocks - 1) / p.col_blocks;
+    int64_t max_splits = (h->V + 15) / 16;
+    if (want > max_splits) want = max_splits;
+    if (want < 1) want = 1;
+    if (want > 65535) want = 65535;
+    p.rows_per_split = (int)((h->V + want - 1) / want);
+    p.splits = (h->V + p.rows_per_split - 1) / p.rows_per_split;
+    return p;
+}
+
+}  // namespace
+
+size_t som_norms_workspace_bytes(const som_handle* h)
+{
+    NormPlan p = plan_norms(h);
+    return (size_t)p.splits * (size_t)h->M * sizeof(double);
+}
+
+int som_launch_norms(som_handle* h, cudaStream_t st)
+{
+    NormPlan p = plan_norms(h);
+    double* partial = reinterpret_cast<double*>(h->ws);
+    dim3 grid((unsigned)p.col_blocks, (unsigned)p.splits);
+    if (p.vec == 4)
+        k_norms_partial<4><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial);
+    else
+        k_norms_partial<1><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial);
+    SOM_CK(h, cudaGetLastError());
+    const int64_t blocks = (h->M + 255) / 256;
+    k_norms_combine<<<(unsigned)blocks, 256, 0, st>>>(partial, h->M, p.splits, h->norm64, h->norm32,
+                                                      h->hnorm);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 2;
+    return SOM_OK;
+}

@@ -1,0 +1,186 @@
+"""Thin Python binding over the C-ABI CUDA library (``include/som.h``).
+
+Argument marshalling only: every step of the search runs in the library's kernels.
+PyTorch supplies device memory and streams.  If ``libsom_b200.so`` is missing or cannot
+be loaded this module raises; there is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsom_b200.so")
+
+SOM_OK = 0
+STATUS_NAMES = {
+    0: "SOM_OK", 1: "SOM_ERR_INVALID_ARG", 2: "SOM_ERR_NORMS_STALE", 3: "SOM_ERR_UNSUPPORTED",
+    4: "SOM_ERR_CUDA", 5: "SOM_ERR_BAD_CSR", 6: "SOM_ERR_NO_DEVICE",
+}
+
+# every symbol include/som.h declares
+EXPORTS = [
+    "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
+    "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
+    "som_launch_count", "som_set_option",
+]
+
+_lib = None
+
+
+class SomError(RuntimeError):
+    def __init__(self, status: int, where: str, cuda_error: int = 0):
+        self.status = status
+        self.cuda_error = cuda_error
+        msg = "%s failed: %s" % (where, STATUS_NAMES.get(status, str(status)))
+        if cuda_error:
+            msg += " (cudaError %d)" % cuda_error
+        super().__init__(msg)
+
+
+def load_library():
+    """Load the compiled CUDA library; raise if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "CUDA library %s not found: build it with `python -m paper_2608_24067_b200.build` "
+            "(there is no CPU fallback)" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    P, I32, I64, INT = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int
+    lib.som_create.argtypes = [ctypes.POINTER(P), I32, I64, P]
+    lib.som_norms.argtypes = [P, P]
+    lib.som_bmu.argtypes = [P, P, P, I64, P, P, P]
+    lib.som_bmu_host.argtypes = [P, P, P, I64, P, P, P]
+    lib.som_validate_csr.argtypes = [P, P, P, I64, P]
+    lib.som_get_norms.argtypes = [P, P, P]
+    lib.som_destroy.argtypes = [P]
+    lib.som_status_string.argtypes = [INT]
+    lib.som_status_string.restype = ctypes.c_char_p
+    lib.som_last_cuda_error.argtypes = [P]
+    lib.som_set_timing.argtypes = [P, INT]
+    lib.som_get_timing.argtypes = [P, P, INT]
+    lib.som_launch_count.argtypes = [P]
+    lib.som_launch_count.restype = I64
+    lib.som_set_option.argtypes = [P, INT, I64]
+    for name in ("som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr",
+                 "som_get_norms", "som_destroy", "som_last_cuda_error", "som_set_timing",
+                 "som_get_timing", "som_set_option"):
+        getattr(lib, name).restype = INT
+    _lib = lib
+    return lib
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_ptr(t: torch.Tensor, dtype, name: str) -> int:
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous CUDA tensor of %s" % (name, dtype))
+    return t.data_ptr()
+
+
+def _host_ptr(t: torch.Tensor, dtype, name: str) -> int:
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous CPU tensor of %s" % (name, dtype))
+    return t.data_ptr()
+
+
+class Som:
+    """Handle over a feature-major fp32 codebook resident on the GPU (borrowed, not copied)."""
+
+    def __init__(self, V: int, M: int, codebook: torch.Tensor):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        if codebook.numel() != V * M:
+            raise ValueError("codebook must hold V*M elements")
+        ptr = _dev_ptr(codebook, torch.float32, "codebook")
+        self.V, self.M = int(V), int(M)
+        self.codebook = codebook  # keep the borrowed memory alive
+        with torch.cuda.device(codebook.device):
+            rc = self._lib.som_create(ctypes.byref(self._h), V, M, ptr)
+        if rc != SOM_OK:
+            self._h = ctypes.c_void_p()
+            raise SomError(rc, "som_create")
+
+    def _check(self, rc: int, where: str):
+        if rc != SOM_OK:
+            raise SomError(rc, where, self._lib.som_last_cuda_error(self._h))
+
+    def norms(self, stream=None):
+        """som_norms: recompute ||w_i||^2 (call after every codebook update)."""
+        self._check(self._lib.som_norms(self._h, _stream_ptr(stream)), "som_norms")
+
+    def bmu(self, indptr: torch.Tensor, indices: torch.Tensor, out_bmu: torch.Tensor | None = None,
+            out_dist: torch.Tensor | None = None, stream=None):
+        """som_bmu on device-resident CSR; returns (bmu int32 [n], min squared distance fp32 [n])."""
+        n = indptr.numel() - 1
+        dev = self.codebook.device
+        if out_bmu is None:
+            out_bmu = torch.empty(n, dtype=torch.int32, device=dev)
+        if out_dist is None:
+            out_dist = torch.empty(n, dtype=torch.float32, device=dev)
+        rc = self._lib.som_bmu(self._h, _dev_ptr(indptr, torch.int32, "indptr"),
+                               _dev_ptr(indices, torch.int32, "indices"), n,
+                               _dev_ptr(out_bmu, torch.int32, "out_bmu"),
+                               _dev_ptr(out_dist, torch.float32, "out_dist"), _stream_ptr(stream))
+        self._check(rc, "som_bmu")
+        return out_bmu, out_dist
+
+    def bmu_host(self, indptr: torch.Tensor, indices: torch.Tensor, out_bmu: torch.Tensor,
+                 out_dist: torch.Tensor, stream=None):
+        """som_bmu_host: CPU tensors in and out (pin them for speed); synchronises the stream."""
+        n = indptr.numel() - 1
+        rc = self._lib.som_bmu_host(self._h, _host_ptr(indptr, torch.int32, "indptr"),
+                                    _host_ptr(indices, torch.int32, "indices"), n,
+                                    _host_ptr(out_bmu, torch.int32, "out_bmu"),
+                                    _host_ptr(out_dist, torch.float32, "out_dist"), _stream_ptr(stream))
+        self._check(rc, "som_bmu_host")
+        return out_bmu, out_dist
+
+    def validate_csr(self, indptr: torch.Tensor, indices: torch.Tensor, stream=None) -> bool:
+        n = indptr.numel() - 1
+        rc = self._lib.som_validate_csr(self._h, _dev_ptr(indptr, torch.int32, "indptr"),
+                                        _dev_ptr(indices, torch.int32, "indices"), n,
+                                        _stream_ptr(stream))
+        if rc == 5:
+            return False
+        self._check(rc, "som_validate_csr")
+        return True
+
+    def get_norms(self, stream=None) -> torch.Tensor:
+        out = torch.empty(self.M, dtype=torch.float32, device=self.codebook.device)
+        self._check(self._lib.som_get_norms(self._h, out.data_ptr(), _stream_ptr(stream)), "som_get_norms")
+        return out
+
+    def set_timing(self, enable: bool):
+        self._check(self._lib.som_set_timing(self._h, int(enable)), "som_set_timing")
+
+    def get_timing(self) -> dict:
+        buf = (ctypes.c_float * 5)()
+        self._check(self._lib.som_get_timing(self._h, ctypes.cast(buf, ctypes.c_void_p), 5), "som_get_timing")
+        return {"norms_ms": buf[0], "bmu_ms": buf[1], "plan_ms": buf[2], "search_ms": buf[3],
+                "finalize_ms": buf[4]}
+
+    def launch_count(self) -> int:
+        return int(self._lib.som_launch_count(self._h))
+
+    def set_option(self, key: int, value: int):
+        self._check(self._lib.som_set_option(self._h, key, value), "som_set_option")
+
+    def destroy(self):
+        if self._h:
+            self._lib.som_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -125,6 +125,26 @@ def codebook_rows(V: int, M: int, rows: torch.Tensor, seed: int = 0,
     return out
 
 
+def codebook_slab(V: int, M: int, m0: int, m1: int, seed: int = 0, device="cpu",
+                  spikes_per_neuron: int = 20, chunk_elems: int = 1 << 24) -> torch.Tensor:
+    """Columns [m0, m1) of ``fill_codebook`` as a dense [V, m1-m0] fp32 tensor (same values)."""
+    dev = torch.device(device)
+    ms = m1 - m0
+    out = torch.empty(V, ms, dtype=torch.float32, device=dev)
+    i = torch.arange(m0, m1, dtype=torch.int64, device=dev)
+    rows_per_chunk = max(1, chunk_elems // max(1, ms))
+    for v0 in range(0, V, rows_per_chunk):
+        v1 = min(V, v0 + rows_per_chunk)
+        v = torch.arange(v0, v1, dtype=torch.int64, device=dev)
+        off = (v[:, None] * M + i[None, :]).reshape(-1)
+        out[v0:v1] = _u24_to_f32(hash32(seed, _STREAM_BASE, off, 0), 0.0, 0.05).view(v1 - v0, ms)
+    for k in range(spikes_per_neuron):
+        v = hash32(seed, _STREAM_SPIKE_POS, i, k) % V
+        val = _u24_to_f32(hash32(seed, _STREAM_SPIKE_VAL, v * M + i, 0), 0.3, 0.7)
+        out[v, i - m0] = val
+    return out
+
+
 def zipf_cdf(V: int, s: float) -> np.ndarray:
     """Cumulative distribution (float64, host) of p(v) ~ (v+1)^-s over v in [0,V)."""
     p = np.power(np.arange(1, V + 1, dtype=np.float64), -float(s))

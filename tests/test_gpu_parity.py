@@ -1,0 +1,245 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle.
+
+Index work must match exactly outside the stated near-tie band, distances within 1e-5
+relative, histograms of unambiguous winners bit-exact, outputs bit-identical run to run.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import parity
+from oracle import som_oracle as orc
+from paper_2608_24067_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "handbuilt_cases.txt")
+
+
+@pytest.fixture(scope="module")
+def som_mod():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_24067_b200 import som
+    som.load_library()  # fail loudly when the extension is missing
+    return som
+
+
+def _run_gpu(som_mod, W_dev, V, M, indptr_dev, indices_dev, variant=None):
+    h = som_mod.Som(V, M, W_dev)
+    if variant is not None:
+        h.set_option(0, variant)
+    h.norms()
+    bmu, dist = h.bmu(indptr_dev, indices_dev)
+    torch.cuda.synchronize()
+    return h, bmu.cpu().numpy(), dist.cpu().numpy()
+
+
+def _subset_csr(indptr, indices, rows):
+    """Host CSR of the chosen rows (numpy)."""
+    indptr = np.asarray(indptr, dtype=np.int64)
+    lens = indptr[rows + 1] - indptr[rows]
+    out_ptr = np.zeros(len(rows) + 1, np.int32)
+    out_ptr[1:] = np.cumsum(lens)
+    parts = [indices[indptr[r]:indptr[r + 1]] for r in rows]
+    out_idx = np.concatenate(parts).astype(np.int32) if len(parts) else np.zeros(0, np.int32)
+    return out_ptr, out_idx
+
+
+def _check_against_oracle(W_host, V, M, indptr, indices, g_bmu, g_dist, rows=None):
+    indptr = np.asarray(indptr)
+    indices = np.asarray(indices)
+    if rows is not None:
+        indptr, indices = _subset_csr(indptr, indices, rows)
+        g_bmu, g_dist = g_bmu[rows], g_dist[rows]
+    nn = orc.norms(W_host, V, M)
+    top2 = orc.bmu(W_host, V, M, indptr, indices, norms_=nn)
+    safe = np.clip(g_bmu.astype(np.int64), 0, M - 1)
+    d_at = orc.dist_at(W_host, V, M, indptr, indices, safe, norms_=nn)
+    rep = parity.check(g_bmu, g_dist, top2, d_at, M)
+    assert rep.ok, str(rep)
+    return rep
+
+
+@pytest.mark.parametrize("variant", [1, 0])
+@pytest.mark.parametrize("kind", ["zipf", "permuted", "uniform"])
+def test_config1_full(som_mod, kind, variant):
+    """Tiny 16x16 configuration, every sample checked."""
+    w = synth.CONFIGS[0]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(w.N, w.V, w.lam, w.seed, device="cuda",
+                         zipf_s=0.0 if kind == "uniform" else w.zipf_s,
+                         permute_ids=(kind == "permuted"))
+    h, g_bmu, g_dist = _run_gpu(som_mod, W, w.V, w.M, b.indptr, b.indices, variant)
+    assert h.validate_csr(b.indptr, b.indices)
+    rep = _check_against_oracle(W.cpu().numpy(), w.V, w.M, b.indptr.cpu().numpy(),
+                                b.indices.cpu().numpy(), g_bmu, g_dist)
+    assert rep.near_ties < 0.01 * w.N
+    # norms against the oracle's fp64 norms
+    nn = orc.norms(W.cpu().numpy(), w.V, w.M)
+    np.testing.assert_allclose(h.get_norms().cpu().numpy().astype(np.float64), nn, rtol=2e-7)
+
+
+@pytest.mark.parametrize("variant", [1, 0])
+def test_config2_sampled_rows(som_mod, variant):
+    """64x64 map, one million samples on the GPU; every 40th row against the oracle."""
+    w = synth.CONFIGS[1]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(w.N, w.V, w.lam, w.seed, device="cuda")
+    h, g_bmu, g_dist = _run_gpu(som_mod, W, w.V, w.M, b.indptr, b.indices, variant)
+    rows = np.arange(0, w.N, 40)
+    rows = np.concatenate([rows, [w.N - 1]])
+    rep = _check_against_oracle(W.cpu().numpy(), w.V, w.M, b.indptr.cpu().numpy(),
+                                b.indices.cpu().numpy(), g_bmu, g_dist, rows)
+    assert rep.near_ties < 0.05 * rows.size
+    # run-to-run determinism on the full batch
+    bmu2, dist2 = h.bmu(b.indptr, b.indices)
+    torch.cuda.synchronize()
+    assert np.array_equal(bmu2.cpu().numpy(), g_bmu)
+    assert np.array_equal(dist2.cpu().numpy().view(np.uint32), g_dist.view(np.uint32))
+
+
+def test_config3_full_size_sampled_rows(som_mod):
+    """128x128 map at its full size (4M samples, the benchmark's launch configuration);
+    a strided sample of rows against the oracle, plus properties that hold for all rows."""
+    w = synth.CONFIGS[2]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(w.N, w.V, w.lam, w.seed, device="cuda")
+    h, g_bmu, g_dist = _run_gpu(som_mod, W, w.V, w.M, b.indptr, b.indices)
+    assert g_bmu.min() >= 0 and g_bmu.max() < w.M
+    assert np.isfinite(g_dist).all() and g_dist.min() >= 0
+    rows = np.concatenate([np.arange(0, w.N, 2000), [w.N - 1]])
+    _check_against_oracle(W.cpu().numpy(), w.V, w.M, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
+                          g_bmu, g_dist, rows)
+
+
+def _parse_golden():
+    cases, cur = [], None
+    for line in open(GOLDEN):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        tok = line.split()
+        if tok[0] == "case":
+            cur = {"name": tok[1], "V": int(tok[2]), "M": int(tok[3]), "w": {}, "x": []}
+            cases.append(cur)
+        elif tok[0] == "w":
+            cur["w"][int(tok[1])] = [float(t) for t in tok[3:]]
+        elif tok[0] == "x":
+            left, right = line[1:].split("|")
+            ids = [int(t) for t in left.replace(":", " ").split()]
+            r = right.split()
+            cur["x"].append((ids, int(r[0]), float(r[1])))
+    return cases
+
+
+@pytest.mark.parametrize("variant", [1, 0])
+@pytest.mark.parametrize("case", _parse_golden(), ids=lambda c: c["name"])
+def test_handbuilt_cases_on_gpu(som_mod, case, variant):
+    """Exactly representable weights: winner and distance must be exact, ties to the lowest index."""
+    V, M = case["V"], case["M"]
+    Wn = np.array([case["w"][i] for i in range(M)], np.float32)
+    W = torch.from_numpy(np.ascontiguousarray(Wn.T)).cuda().reshape(-1)
+    rows = [np.array(x[0], np.int32) for x in case["x"]]
+    indptr = np.zeros(len(rows) + 1, np.int32)
+    indptr[1:] = np.cumsum([len(r) for r in rows])
+    indices = np.concatenate(rows) if rows else np.zeros(0, np.int32)
+    idx_dev = torch.from_numpy(indices).cuda() if indices.size else torch.zeros(1, dtype=torch.int32, device="cuda")
+    _, g_bmu, g_dist = _run_gpu(som_mod, W, V, M, torch.from_numpy(indptr).cuda(), idx_dev, variant)
+    for s, (_, b1, d1) in enumerate(case["x"]):
+        assert g_bmu[s] == b1 and g_dist[s] == np.float32(d1), (case["name"], s, g_bmu[s], g_dist[s])
+
+
+@pytest.mark.parametrize("variant", [1, 0])
+@pytest.mark.parametrize("V,M,n", [(50, 1, 30), (64, 37, 200), (97, 130, 300), (40, 4, 64),
+                                   (300, 260, 500), (1000, 1028, 700)])
+def test_ragged_shapes(som_mod, V, M, n, variant):
+    """Neuron counts that are not multiples of the vector width or of a block, tiny maps."""
+    rng = np.random.default_rng(V * 1000 + M)
+    W = rng.random((V, M)).astype(np.float32)
+    rows = []
+    for s in range(n):
+        k = int(rng.integers(0, min(V, 45) + 1))  # includes empty rows and rows longer than 32
+        rows.append(np.sort(rng.choice(V, size=k, replace=False)).astype(np.int32))
+    indptr = np.zeros(n + 1, np.int32)
+    indptr[1:] = np.cumsum([len(r) for r in rows])
+    indices = np.concatenate(rows).astype(np.int32)
+    _, g_bmu, g_dist = _run_gpu(som_mod, torch.from_numpy(W).cuda().reshape(-1), V, M,
+                                torch.from_numpy(indptr).cuda(), torch.from_numpy(indices).cuda(), variant)
+    _check_against_oracle(W, V, M, indptr, indices, g_bmu, g_dist)
+
+
+def test_indptr_with_base_offset(som_mod):
+    """d_indptr[0] may be any offset into d_indices (a batch cut out of a longer stream)."""
+    w = synth.CONFIGS[0]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(3000, w.V, w.lam, w.seed, device="cuda")
+    h = som_mod.Som(w.V, w.M, W)
+    h.norms()
+    full_bmu, full_dist = h.bmu(b.indptr, b.indices)
+    part_bmu, part_dist = h.bmu(b.indptr[1000:2001].contiguous(), b.indices)
+    torch.cuda.synchronize()
+    assert torch.equal(part_bmu, full_bmu[1000:2000])
+    assert torch.equal(part_dist, full_dist[1000:2000])
+
+
+def test_host_entry_point_matches_device_entry_point(som_mod):
+    w = synth.CONFIGS[0]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(5000, w.V, w.lam, w.seed, device="cpu")
+    h = som_mod.Som(w.V, w.M, W)
+    h.norms()
+    d_bmu, d_dist = h.bmu(b.indptr.cuda(), b.indices.cuda())
+    hb = torch.empty(b.n, dtype=torch.int32).pin_memory()
+    hd = torch.empty(b.n, dtype=torch.float32).pin_memory()
+    h.bmu_host(b.indptr.pin_memory(), b.indices.pin_memory(), hb, hd)
+    assert torch.equal(hb, d_bmu.cpu()) and torch.equal(hd, d_dist.cpu())
+
+
+def test_status_codes_and_noops(som_mod):
+    w = synth.CONFIGS[0]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(100, w.V, w.lam, w.seed, device="cuda")
+    h = som_mod.Som(w.V, w.M, W)
+    with pytest.raises(som_mod.SomError) as e:
+        h.bmu(b.indptr, b.indices)  # norms not computed yet
+    assert e.value.status == 2
+    h.norms()
+    # n = 0 is a successful no-op
+    out_b, out_d = h.bmu(b.indptr[:1].contiguous(), b.indices)
+    assert out_b.numel() == 0 and out_d.numel() == 0
+    # validator: unsorted row, out-of-range id
+    bad = b.indices.clone()
+    bad[0], bad[1] = b.indices[1], b.indices[0]
+    if int(b.indptr[1]) >= 2:
+        assert not h.validate_csr(b.indptr, bad)
+    bad = b.indices.clone()
+    bad[-1] = w.V
+    assert not h.validate_csr(b.indptr, bad)
+    assert h.validate_csr(b.indptr, b.indices)
+    # invalid arguments at creation
+    with pytest.raises(som_mod.SomError):
+        som_mod.Som(0, 0, W[:0])
+    lib = som_mod.load_library()
+    assert lib.som_status_string(5) == b"SOM_ERR_BAD_CSR"
+    assert lib.som_destroy(None) == 0
+
+
+def test_norms_follow_codebook_update(som_mod):
+    """After an in-place codebook update som_norms must be rerun; then results follow the new weights."""
+    V, M, n = 200, 64, 400
+    rng = np.random.default_rng(3)
+    W = torch.from_numpy(rng.random((V, M)).astype(np.float32)).cuda().reshape(-1)
+    b = synth.sample_csr(n, V, 7.0, seed=1, device="cuda")
+    h = som_mod.Som(V, M, W)
+    h.norms()
+    h.bmu(b.indptr, b.indices)
+    W.mul_(0.5)
+    W[5::M] += 0.25
+    h.norms()
+    g_bmu, g_dist = h.bmu(b.indptr, b.indices)
+    torch.cuda.synchronize()
+    _check_against_oracle(W.cpu().numpy(), V, M, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
+                          g_bmu.cpu().numpy(), g_dist.cpu().numpy())

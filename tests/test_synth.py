@@ -96,6 +96,8 @@ def test_codebook_reproducible_chunking_and_rows():
     rows = torch.tensor([0, 17, 299])
     assert torch.equal(synth.codebook_rows(V, M, rows, seed=5), a.view(V, M)[rows])
     assert not torch.equal(a, synth.fill_codebook(V, M, seed=6))
+    assert torch.equal(synth.codebook_slab(V, M, 8, 40, seed=5, chunk_elems=500), a.view(V, M)[:, 8:40])
+    assert torch.equal(synth.codebook_slab(V, M, 0, M, seed=5), a.view(V, M))
 
 
 def test_configs_table():
