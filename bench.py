@@ -193,6 +193,10 @@ def run_ours(args, w: synth.Workload):
     h = som.Som(w.V, w.M, W)
     if args.variant is not None:
         h.set_option(0, args.variant)
+    if args.hot_rows:
+        h.set_option(1, args.hot_rows)
+    if args.threads:
+        h.set_option(2, args.threads)
     out_bmu = torch.empty(w.batch, dtype=torch.int32, device=dev)
     out_dist = torch.empty(w.batch, dtype=torch.float32, device=dev)
 
@@ -332,6 +336,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, help="index into the five workloads (default 1: 64x64)")
     ap.add_argument("--variant", type=int, default=None, help="search kernel variant (library option 0)")
+    ap.add_argument("--hot-rows", type=int, default=0, help="row-table kernel: hot rows in shared memory")
+    ap.add_argument("--threads", type=int, default=0, help="row-table kernel: block size (512 or 1024)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]

@@ -18,9 +18,11 @@
  *     "host pointer" = ordinary process memory.  The library never takes ownership of a
  *     caller's buffer.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
- *     som_norms / som_bmu only enqueue work on it and return without synchronising,
- *     except that growing the handle's workspace (first call, or a larger batch than any
- *     before) allocates device memory, which may synchronise the device once.
+ *     som_norms / som_bmu only enqueue work on it, with two exceptions: growing the handle's
+ *     workspace (first call, or a larger batch than any before) allocates device memory,
+ *     which may synchronise the device once; and som_bmu, when it takes its row-table kernel,
+ *     first reads d_indptr[0] and d_indptr[n_samples] back to size its plan, which waits for
+ *     earlier work on `stream` (the search itself is then only enqueued).
  *   - Thread safety: one handle must not be used from two host threads at once, and two
  *     calls on the same handle must not overlap on the GPU (they share the workspace);
  *     issue them on one stream or order the streams yourself.
@@ -131,8 +133,9 @@ int som_last_cuda_error(const som_handle* h);
  *   out_ms[0] som_norms total, out_ms[1] som_bmu total, out_ms[2] som_bmu plan phase,
  *   out_ms[3] som_bmu search kernel(s), out_ms[4] som_bmu finalize.
  * som_launch_count returns how many kernels this handle has launched since creation.
- * som_set_option tunes kernel selection: key 0 = search kernel variant
- * (0 auto, 1 direct-load kernel, 2 shared-memory row-table kernel).
+ * som_set_option tunes kernel selection: key 0 = search kernel variant (0 auto, 1 direct-load
+ * kernel, 2 shared-memory row-table kernel where M % 4 == 0 and V <= 65536); key 1 = hot rows kept in shared
+ * memory by the row-table kernel (0 = default); key 2 = its block size (0 = default, 512, 768, 1024).
  */
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);

@@ -3,6 +3,7 @@
 #include <new>
 
 #include "som_internal.cuh"
+#include "som_plan.cuh"
 
 namespace {
 
@@ -99,6 +100,7 @@ int som_destroy(som_handle* h)
     cudaFree(h->hnorm);
     cudaFree(h->ws);
     cudaFree(h->stage);
+    if (h->host_pair) cudaFreeHost(h->host_pair);
     if (h->events_made)
         for (int i = 0; i < SOM_N_EVENTS; ++i) cudaEventDestroy(h->ev[i]);
     delete h;
@@ -132,19 +134,63 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
     DeviceGuard g(h->device);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
-    const size_t key_bytes = som_align_up((size_t)n_samples * sizeof(unsigned long long), 256);
-    int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, key_bytes);
-    if (rc) return rc;
-    unsigned long long* keys = reinterpret_cast<unsigned long long*>(h->ws);
-
+    int rc = SOM_OK;
     if (h->timing && (rc = ensure_events(h))) return rc;
-    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
-    SOM_CK(h, cudaMemsetAsync(keys, 0xFF, (size_t)n_samples * sizeof(unsigned long long), st));
-    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-    if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, st))) return rc;
-    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-    if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, st)))
-        return rc;
+
+    // Kernel selection.  The row-table kernel needs 128-bit aligned row segments (M % 4 == 0),
+    // feature ids that fit its 16-bit codes (V <= 65536) and enough (neuron range x sample part) units to occupy every SM; everything else goes
+    // to the direct-load kernel.
+    const SomTableGeom geom = som_table_geometry(h);
+    bool use_table = h->opt_variant != 1 && (h->M % 4 == 0) && h->V <= 65536 && h->M < ((int64_t)1 << 30);
+    if (use_table && h->opt_variant == 0) {
+        int64_t parts = n_samples / 8192;
+        parts = parts < 1 ? 1 : (parts > 16 ? 16 : parts);
+        const int64_t units = ((h->M + geom.T - 1) / geom.T) * parts;
+        if (units < 2 * (int64_t)h->sm_count) use_table = false;
+    }
+    int64_t nnz = 0;
+    if (use_table) {
+        // The plan's code buffer is sized from the batch's nnz, which lives on the device:
+        // read the two row pointers back (one short synchronisation of the stream per call).
+        if (!h->host_pair) SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 2 * sizeof(int32_t)));
+        SOM_CK(h, cudaMemcpyAsync(h->host_pair, d_indptr, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 1, d_indptr + n_samples, sizeof(int32_t),
+                                  cudaMemcpyDeviceToHost, st));
+        SOM_CK(h, cudaStreamSynchronize(st));
+        nnz = (int64_t)h->host_pair[1] - (int64_t)h->host_pair[0];
+        if (nnz < 0) return SOM_ERR_INVALID_ARG;
+        if (nnz + 6 * n_samples + 4 >= ((int64_t)1 << 31)) use_table = false;
+        if (nnz > 0 && !d_indices) return SOM_ERR_INVALID_ARG;
+    }
+
+    if (!use_table) {
+        const size_t key_bytes = som_align_up((size_t)n_samples * sizeof(unsigned long long), 256);
+        if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, key_bytes))) return rc;
+        unsigned long long* keys = reinterpret_cast<unsigned long long*>(h->ws);
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
+        SOM_CK(h, cudaMemsetAsync(keys, 0xFF, (size_t)n_samples * sizeof(unsigned long long), st));
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+        if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, st))) return rc;
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+        if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, st)))
+            return rc;
+    } else {
+        SomPlanBuffers pb;
+        const size_t need = som_plan_workspace_bytes(h->V, n_samples, nnz,
+                                                     SOM_PLAN_MASK_FEATURES + geom.n_hot, &pb);
+        if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
+        char* ws = reinterpret_cast<char*>(h->ws);
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
+        SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
+        if ((rc = som_launch_plan(h, d_indptr, d_indices, n_samples, ws, pb, SOM_PLAN_MASK_FEATURES,
+                                  geom.n_hot, (uint32_t)geom.T * 4u, st)))
+            return rc;
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, n_samples, ws, pb, geom.n_hot, st))) return rc;
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+        if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, d_bmu, d_min_dist, st)))
+            return rc;
+    }
     if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
     if (h->timing) h->ev_bmu_calls += 1;
     return SOM_OK;
@@ -277,6 +323,16 @@ int som_set_option(som_handle* h, int key, int64_t value)
     if (key == 0) {
         if (value < 0 || value > 2) return SOM_ERR_INVALID_ARG;
         h->opt_variant = value;
+        return SOM_OK;
+    }
+    if (key == 1) {
+        if (value < 0 || value > 65000) return SOM_ERR_INVALID_ARG;
+        h->opt_hot_rows = value;
+        return SOM_OK;
+    }
+    if (key == 2) {
+        if (value != 0 && value != 512 && value != 768 && value != 1024) return SOM_ERR_INVALID_ARG;
+        h->opt_threads = value;
         return SOM_OK;
     }
     return SOM_ERR_INVALID_ARG;

@@ -1,0 +1,364 @@
+// Row-table BMU search kernel (the fast path of som_bmu) and its finalisation.
+//
+// Decomposition (Section 3.3 of the paper, re-planned for B200): a work unit is a
+// neuron range of T = 32 neurons times a contiguous part of the mask-sorted sample list.
+// One persistent block per SM walks units in range-major order, so that at any time only a
+// few neuron ranges are live and their codebook slabs W[:, i0..i0+T) stay L2-resident while
+// HBM sees the codebook once per batch.  Inside a unit the warps pull chunks of samples from
+// a shared counter, which keeps them busy whatever the mix of row lengths.
+//
+// Inside a block the rows W[v*M + i0 .. i0+T) of the batch's hottest features (the row
+// table) are staged in shared memory once per unit.  Eight lanes form a team that owns one
+// sample at a time; a lane keeps 4 score accumulators in registers and subtracts, for every
+// code of the sample, a 128-bit slice of the row: a shared-memory read for hot features, a
+// coalesced 128-bit global read of the L2-resident slab for tail features.  The team's 8 loads
+// cover one contiguous 128-byte row segment.  Adds are issued as packed f32x2 operations,
+// which halves their issue slots.  The accumulators start from
+// ||w||^2/2 - sum(rows of the sample's mask features), which is held in registers across
+// consecutive samples that share the mask (they are adjacent after the plan's sort).
+//
+// Latency: a sample's 48-byte slot sits at a fixed address for its sorted position, so the
+// slot stream is prefetched into L1 several rounds ahead and the next slot and key are loaded
+// into registers while the current sample finishes.  A sample's first four tail rows go in
+// flight at the top of its round and are consumed after the hot rows; 32 resident warps cover
+// what latency remains, which is why the kernel is held to 64 registers per thread.
+// Instruction count: the hot loop is a jump table on the warp's longest hot list (shorter
+// lists are padded with a zero row), so a step costs extract + address + load + two packed
+// subtracts and no predicate.
+//
+// Argmin: each lane reduces its 4 scores, compares with the sample's packed key and only on a
+// (rare) improvement issues a 64-bit atomicMin on (ordered score bits, neuron).  The unsigned
+// minimum of that key is the lexicographic (score, lowest neuron) minimum, so the combine is
+// order-independent and ties break to the lowest neuron index (Section 3.1).
+#include "som_internal.cuh"
+#include "som_plan.cuh"
+
+namespace {
+
+constexpr int T = 32;       // neurons per range
+constexpr int ROWB = 128;   // bytes of one table row
+constexpr int CHUNK = 128;  // samples a warp takes at a time
+constexpr int SLOT_Q = SOM_SLOT_WORDS / 4;  // uint4 per slot
+
+typedef unsigned long long u64;
+
+struct Pair2 {  // four fp32 as two packed pairs
+    u64 lo, hi;
+};
+
+__device__ __forceinline__ u64 pack2(float a, float b)
+{
+    u64 r;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+
+__device__ __forceinline__ void unpack2(u64 v, float& a, float& b)
+{
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+
+__device__ __forceinline__ void sub_pair(Pair2& acc, const Pair2 w)
+{
+    asm("sub.rn.f32x2 %0, %0, %1;" : "+l"(acc.lo) : "l"(w.lo));
+    asm("sub.rn.f32x2 %0, %0, %1;" : "+l"(acc.hi) : "l"(w.hi));
+}
+
+__device__ __forceinline__ Pair2 lds_row(const unsigned char* p)
+{
+    const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
+    Pair2 r;
+    r.lo = v.x;
+    r.hi = v.y;
+    return r;
+}
+
+// 128-bit read of a tail row slice through the read-only path.  Normal eviction priority on
+// purpose: an L1::no_allocate hint also demotes the line to evict-first in L2, and the slab
+// rows are exactly what has to stay L2-resident.
+__device__ __forceinline__ Pair2 ldg_row(const float* p)
+{
+    Pair2 r;
+    asm("ld.global.nc.v2.b64 {%0,%1}, [%2];" : "=l"(r.lo), "=l"(r.hi) : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ void prefetch_l1(const void* p)
+{
+    asm volatile("prefetch.global.L1 [%0];" :: "l"(p));
+}
+
+__device__ __forceinline__ uint32_t lo16(uint32_t w) { return w & 0xffffu; }
+__device__ __forceinline__ uint32_t hi16(uint32_t w) { return w >> 16; }
+
+// address of row `code` in the codebook slab: base + code * row_stride_bytes, one mad.wide
+__device__ __forceinline__ const float* row_ptr(const float* base, uint32_t code, uint32_t stride_bytes)
+{
+    const float* p;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(p) : "r"(code), "r"(stride_bytes), "l"(base));
+    return p;
+}
+
+#define SOM_HOT(code) sub_pair(acc, lds_row(tab_q + ((code) << 7)))
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1)
+k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
+            const int32_t* __restrict__ slot_feat, int n_rows,
+            const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
+            u64* __restrict__ keys, int parts, int64_t part_len, int n_units)
+{
+    constexpr int WARPS = THREADS / 32;
+    extern __shared__ __align__(16) unsigned char tab[];
+    __shared__ int next_chunk;
+    __shared__ __align__(16) float hn_sh[T];  // ||w||^2/2 of the range's neurons (+inf past M)
+    float* tab_f = reinterpret_cast<float*>(tab);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int q = lane & 7;
+    const int sub = lane >> 3;
+    const float inf = __int_as_float(0x7f800000);
+    const unsigned char* tab_q = tab + q * 16;
+    const uint32_t stride_b = (uint32_t)M * 4u;  // the launcher guarantees M < 2^30
+
+    // row n_rows of the table is all zeros: the target of padded hot codes
+    if (threadIdx.x < T) tab_f[n_rows * T + threadIdx.x] = 0.f;
+
+    int cur_range = -1;
+    const float* w_q = W;
+    uint32_t i_first = 0;
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int range = unit / parts;
+        const int part = unit - range * parts;
+        const int64_t i0 = (int64_t)range * T;
+        __syncthreads();  // every warp has left the previous unit
+        if (threadIdx.x == 0) next_chunk = 0;
+        if (range != cur_range) {
+            for (int row0 = warp * 4; row0 < n_rows; row0 += WARPS * 4) {
+                float v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int row = row0 + u;
+                    const int f = row < n_rows ? slot_feat[row] : -1;
+                    v[u] = (f >= 0 && i0 + lane < M) ? __ldg(W + (int64_t)f * M + i0 + lane) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (row0 + u < n_rows) tab_f[(row0 + u) * T + lane] = v[u];
+            }
+            cur_range = range;
+            const int64_t i_lane = i0 + 4 * q;
+            i_first = (uint32_t)i_lane;
+            // lanes past the last neuron read a valid address and carry +inf scores, so they
+            // never beat a real neuron and need no predicate in the loop
+            w_q = W + (i_lane < M ? i_lane : 0);
+            if (threadIdx.x < T) hn_sh[threadIdx.x] = (i0 + threadIdx.x < M) ? hnorm[i0 + threadIdx.x] : inf;
+        }
+        __syncthreads();
+
+        const int64_t k_begin = (int64_t)part * part_len;
+        const int64_t k_end = min(n_pad, k_begin + part_len);  // a multiple of 4
+        const int n_chunks = (int)((k_end - k_begin + CHUNK - 1) / CHUNK);
+
+        uint32_t curmask = 0;
+        Pair2 base = lds_row(reinterpret_cast<const unsigned char*>(hn_sh) + q * 16);
+        for (;;) {
+            int chunk = 0;
+            if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
+            chunk = __shfl_sync(0xffffffffu, chunk, 0);
+            if (chunk >= n_chunks) break;
+            const int64_t w0 = k_begin + (int64_t)chunk * CHUNK;
+            const int rounds = (int)(min(k_end, w0 + CHUNK) - w0) >> 2;
+
+            const uint4* ps = slots + (w0 + sub) * SLOT_Q;  // this team's slot, 4 slots per round
+            u64* pk = keys + w0 + sub;
+            // L1 prefetch of the slot stream, six rounds ahead (the workspace behind the slot
+            // array is mapped, so running past its end is harmless)
+            const char* pf = reinterpret_cast<const char*>(slots + (w0 + 24) * SLOT_Q) + (lane & 1) * 128;
+            uint4 s0 = __ldg(ps), s1 = __ldg(ps + 1), s2 = __ldg(ps + 2);
+            u64 key = __ldcg(pk);
+            for (int r = 0; r < rounds; ++r) {
+                const uint32_t hdr = s0.x;
+                const uint32_t nt = hdr >> 24;  // SOM_SLOT_NT_OVERFLOW marks an overflow sample
+                const uint32_t nh = (hdr >> 16) & 0xffu;
+                const uint32_t mask = hdr & 0xffffu;
+                const bool p0 = nt > 0, p1 = nt > 1, p2 = nt > 2, p3 = nt > 3;
+
+                // ---- the first four tail rows of this sample go in flight first ---------------
+                Pair2 tr0, tr1, tr2, tr3;
+                if (p0) tr0 = ldg_row(row_ptr(w_q, lo16(s2.x), stride_b));
+                if (p1) tr1 = ldg_row(row_ptr(w_q, hi16(s2.x), stride_b));
+                if (p2) tr2 = ldg_row(row_ptr(w_q, lo16(s2.y), stride_b));
+                if (p3) tr3 = ldg_row(row_ptr(w_q, hi16(s2.y), stride_b));
+                if (lane < 2) prefetch_l1(pf);
+                pf += 4 * SOM_SLOT_WORDS * 4;
+
+                // ---- mask prefix ------------------------------------------------------------
+                if (mask != curmask) {
+                    base = lds_row(reinterpret_cast<const unsigned char*>(hn_sh) + q * 16);
+                    uint32_t mm = mask;
+                    while (mm) {
+                        const int b = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        sub_pair(base, lds_row(tab_q + b * ROWB));
+                    }
+                    curmask = mask;
+                }
+                Pair2 acc = base;
+
+                // ---- hot rows: exactly max(nh over the warp) steps; shorter lists are padded
+                //      with the zero row, so a step carries no predicate -------------------------
+                const uint32_t nh_max = __reduce_max_sync(0xffffffffu, nh);
+                switch (nh_max) {
+                    case 12: SOM_HOT(hi16(s1.w));
+                    case 11: SOM_HOT(lo16(s1.w));
+                    case 10: SOM_HOT(hi16(s1.z));
+                    case 9: SOM_HOT(lo16(s1.z));
+                    case 8: SOM_HOT(hi16(s1.y));
+                    case 7: SOM_HOT(lo16(s1.y));
+                    case 6: SOM_HOT(hi16(s1.x));
+                    case 5: SOM_HOT(lo16(s1.x));
+                    case 4: SOM_HOT(hi16(s0.w));
+                    case 3: SOM_HOT(lo16(s0.w));
+                    case 2: SOM_HOT(hi16(s0.z));
+                    case 1: SOM_HOT(lo16(s0.z));
+                    default: break;
+                }
+                const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7 / overflow fields
+
+                // ---- tail rows ------------------------------------------------------------------
+                if (p0) sub_pair(acc, tr0);
+                if (p1) sub_pair(acc, tr1);
+                if (p2) sub_pair(acc, tr2);
+                if (p3) sub_pair(acc, tr3);
+                if (nt > 4) {
+                    if (nt != SOM_SLOT_NT_OVERFLOW) {
+                        sub_pair(acc, ldg_row(row_ptr(w_q, lo16(t45), stride_b)));
+                        if (nt > 5) sub_pair(acc, ldg_row(row_ptr(w_q, hi16(t45), stride_b)));
+                        if (nt > 6) sub_pair(acc, ldg_row(row_ptr(w_q, lo16(t67), stride_b)));
+                        if (nt > 7) sub_pair(acc, ldg_row(row_ptr(w_q, hi16(t67), stride_b)));
+                    } else {
+                        // rare: a sample that does not fit its slot keeps 32-bit lists in the
+                        // overflow buffer (w10 = offset, w11 = hot count | tail count << 16).
+                        // Its inline tail codes are feature 0 four times; start over from base.
+                        acc = base;
+                        const uint32_t* ol = overflow + t45;
+                        const uint32_t onh = lo16(t67), ont = hi16(t67);
+                        const uint32_t nt_pad = (ont + 3u) & ~3u;
+                        for (uint32_t j = 0; j < ont; ++j)
+                            sub_pair(acc, ldg_row(row_ptr(w_q, __ldg(ol + j), stride_b)));
+                        for (uint32_t j = 0; j < onh; ++j) SOM_HOT(__ldg(ol + nt_pad + j));
+                    }
+                }
+
+                // ---- next round's slot and key (their lines were prefetched into L1); the slot
+                //      array is padded, so the load after the last round is in bounds -------------
+                const u64 key0 = key;
+                ps += 4 * SLOT_Q;
+                pk += 4;
+                s0 = __ldg(ps);
+                s1 = __ldg(ps + 1);
+                s2 = __ldg(ps + 2);
+                key = __ldcg(pk);
+
+                // ---- lane-local argmin, rare atomic combine ------------------------------------
+                float a0, a1, a2, a3;
+                unpack2(acc.lo, a0, a1);
+                unpack2(acc.hi, a2, a3);
+                const float mn = fminf(fminf(a0, a1), fminf(a2, a3));
+                const uint32_t cu = (uint32_t)(key0 >> 32);
+                const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
+                if (!(mn > cs)) {
+                    const int rr = (a0 == mn) ? 0 : ((a1 == mn) ? 1 : ((a2 == mn) ? 2 : 3));
+                    atomicMin(pk - 4, som_pack_key(mn, i_first + rr));
+                }
+            }
+        }
+    }
+}
+
+__global__ void k_finalize_sorted(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
+                                  const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
+                                  int64_t n, const uint4* __restrict__ slots,
+                                  const u64* __restrict__ keys, int32_t* __restrict__ bmu,
+                                  float* __restrict__ dist)
+{
+    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n) return;
+    const uint32_t s = slots[k * SLOT_Q].y;
+    const uint32_t idx = (uint32_t)(keys[k] & 0xffffffffull);
+    const int beg = indptr[s];
+    const int end = indptr[s + 1];
+    double dot = 0.0;
+    for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
+    bmu[s] = (int32_t)idx;
+    dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
+}
+
+template <int THREADS>
+int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& b, int n_hot, size_t smem,
+                 cudaStream_t st)
+{
+    const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
+    const int n_ranges = (int)((h->M + T - 1) / T);
+    int parts = (int)(n / 8192);
+    if (parts < 1) parts = 1;
+    if (parts > 16) parts = 16;
+    int64_t part_len = (n + parts - 1) / parts;
+    part_len = (part_len + CHUNK - 1) / CHUNK * CHUNK;
+    parts = (int)((n + part_len - 1) / part_len);
+    const int64_t n_units64 = (int64_t)n_ranges * parts;
+    if (n_units64 > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
+    const int n_units = (int)n_units64;
+    const int grid = n_units < h->sm_count ? n_units : h->sm_count;
+    auto kern = k_bmu_table<THREADS>;
+    SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<grid, THREADS, smem, st>>>(h->W, h->hnorm, h->M,
+                                      reinterpret_cast<const int32_t*>(ws + b.slot_feat),
+                                      SOM_PLAN_MASK_FEATURES + n_hot,
+                                      reinterpret_cast<const uint4*>(ws + b.slots),
+                                      reinterpret_cast<const uint32_t*>(ws + b.overflow), n,
+                                      reinterpret_cast<u64*>(ws + b.keys), parts, part_len, n_units);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
+    return SOM_OK;
+}
+
+}  // namespace
+
+SomTableGeom som_table_geometry(const som_handle* h)
+{
+    SomTableGeom g;
+    g.R = 4;
+    g.T = T;
+    g.threads = (h->opt_threads == 512) ? 512 : (h->opt_threads == 768 ? 768 : 1024);
+    int max_rows = (int)((227 * 1024 - 1024) / ROWB) - SOM_PLAN_MASK_FEATURES - 1;
+    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : 1536;
+    if (want > max_rows) want = max_rows;
+    g.n_hot = want;
+    g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * ROWB;  // + the zero row
+    return g;
+}
+
+int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
+                         cudaStream_t st)
+{
+    const SomTableGeom g = som_table_geometry(h);
+    if (g.threads == 1024) return launch_table<1024>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 768) return launch_table<768>(h, n, ws, b, n_hot, g.smem, st);
+    return launch_table<512>(h, n, ws, b, n_hot, g.smem, st);
+}
+
+int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                               char* ws, const SomPlanBuffers& b, int32_t* bmu, float* dist,
+                               cudaStream_t st)
+{
+    const int64_t blocks = (n + 255) / 256;
+    k_finalize_sorted<<<(unsigned)blocks, 256, 0, st>>>(
+        h->W, h->norm64, h->M, indptr, indices, n, reinterpret_cast<const uint4*>(ws + b.slots),
+        reinterpret_cast<const u64*>(ws + b.keys), bmu, dist);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
+    return SOM_OK;
+}

@@ -34,7 +34,11 @@ struct som_handle {
     int64_t ev_norms_calls;  // calls recorded since timing was switched on
     int64_t ev_bmu_calls;
     int64_t launches;
-    int64_t opt_variant;
+    int64_t opt_variant;   // 0 auto, 1 direct-load kernel, 2 row-table kernel
+    int64_t opt_hot_rows;  // 0 = default number of hot rows in shared memory
+    int64_t opt_threads;   // block size of the row-table kernel: 0 (default 512), 512 or 1024
+    int plan_attr_set;
+    int32_t* host_pair;    // pinned, 2 ints: read-back of indptr[0], indptr[n]
 };
 
 // event slots

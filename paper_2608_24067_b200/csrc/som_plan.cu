@@ -1,0 +1,380 @@
+// Per-batch plan of the row-table BMU kernel: the "merged feature lists" of a sample tile
+// (Section 3.3), pushed from one tile to the whole batch.
+//
+//   1. feature histogram of the batch                      (k_feat_hist)
+//   2. pick the 16 most frequent features ("mask" features) and the next H ("hot" features);
+//      give each a slot in the shared-memory row table      (k_select_hot, one block)
+//   3. classify each sample: 16-bit mask of mask features, number of hot / tail features,
+//      and count sort bins keyed on (mask, length class)    (k_classify)
+//   4. exclusive scan of the bins                           (k_scan_bins, one block)
+//   5. scatter every sample to its sorted position and write its fixed-size slot there:
+//      hot features as byte offsets of their table row, tail features as feature ids
+//      (k_scatter_slots); the rare sample that does not fit a slot gets an overflow list.
+//
+// Samples that share a mask end up adjacent, so the search kernel keeps
+// ||w||^2/2 - sum(mask rows) in registers across them ("clustering the corpus so that a
+// tile's feature union shrinks", Section 7 of the paper, taken to the register level).
+// Nothing here depends on the neuron range, so the plan is built once per batch.
+#include "som_internal.cuh"
+#include "som_plan.cuh"
+
+namespace {
+
+constexpr int PLAN_THREADS = 256;
+
+__device__ __forceinline__ int warp_incl_scan(int v, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// Exclusive scan of one int per thread over a 1024-thread block; returns the exclusive prefix,
+// *total receives the block sum.  warp_sums must hold 32 ints of shared memory.
+__device__ int block_excl_scan_1024(int v, int* warp_sums, int* total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int incl = warp_incl_scan(v, lane);
+    __syncthreads();
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int s = warp_sums[lane];
+        int si = warp_incl_scan(s, lane);
+        warp_sums[lane] = si - s;
+        if (lane == 31) *total = si;
+    }
+    __syncthreads();
+    return warp_sums[warp] + incl - v;
+}
+
+// ---- 1. feature histogram --------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+k_feat_hist(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n, int V,
+            int use_smem, uint32_t* __restrict__ feat_count)
+{
+    extern __shared__ uint32_t sh_hist[];
+    const int64_t beg = indptr[0], end = indptr[n];
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    if (use_smem) {
+        for (int v = threadIdx.x; v < V; v += blockDim.x) sh_hist[v] = 0;
+        __syncthreads();
+        for (int64_t p = beg + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < end; p += stride)
+            atomicAdd(&sh_hist[indices[p]], 1u);
+        __syncthreads();
+        for (int v = threadIdx.x; v < V; v += blockDim.x) {
+            const uint32_t c = sh_hist[v];
+            if (c) atomicAdd(&feat_count[v], c);
+        }
+    } else {
+        for (int64_t p = beg + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < end; p += stride)
+            atomicAdd(&feat_count[indices[p]], 1u);
+    }
+}
+
+// ---- 2. hot-set selection --------------------------------------------------------------------
+// K-th largest count by a 4-pass radix select.  thr = that count, n_greater = how many counts
+// are strictly larger.  All threads of the 1024-thread block call it.
+__device__ void kth_largest(const uint32_t* __restrict__ c, int V, int K, uint32_t* sh_hist,
+                            uint32_t* sh_state, uint32_t* thr, int* n_greater)
+{
+    if (threadIdx.x == 0) { sh_state[0] = 0; sh_state[1] = (uint32_t)K; sh_state[2] = 0; }
+    __syncthreads();
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        if (threadIdx.x < 256) sh_hist[threadIdx.x] = 0;
+        __syncthreads();
+        const uint32_t prefix = sh_state[0];
+        const uint32_t hi_mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
+        for (int v = threadIdx.x; v < V; v += blockDim.x) {
+            const uint32_t x = c[v];
+            if ((x & hi_mask) == prefix) atomicAdd(&sh_hist[(x >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t need = sh_state[1], cum = 0;
+            int d = 255;
+            while (d > 0 && cum + sh_hist[d] < need) { cum += sh_hist[d]; --d; }
+            sh_state[2] += cum;
+            sh_state[1] = need - cum;
+            sh_state[0] = prefix | ((uint32_t)d << shift);
+        }
+        __syncthreads();
+    }
+    *thr = sh_state[0];
+    *n_greater = (int)sh_state[2];
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(1024)
+k_select_hot(const uint32_t* __restrict__ feat_count, int V, int n_mask, int n_hot,
+             int32_t* __restrict__ feat_slot, int32_t* __restrict__ slot_feat, int32_t* __restrict__ n_slots)
+{
+    __shared__ uint32_t sh_hist[256];
+    __shared__ uint32_t sh_state[4];
+    __shared__ int warp_sums[32];
+    __shared__ int sh_total;
+    uint32_t thr_m, thr_a;
+    int gr_m, gr_a;
+    kth_largest(feat_count, V, n_mask, sh_hist, sh_state, &thr_m, &gr_m);
+    kth_largest(feat_count, V, n_mask + n_hot, sh_hist, sh_state, &thr_a, &gr_a);
+    const int need_m = n_mask - gr_m;            // ties at thr_m to take (lowest ids first)
+    const int need_a = n_mask + n_hot - gr_a;    // ties at thr_a to take
+    int tie_m_seen = 0, tie_a_seen = 0, mask_assigned = 0, hot_assigned = 0;
+    for (int v0 = 0; v0 < V; v0 += 1024) {
+        const int v = v0 + threadIdx.x;
+        const uint32_t c = (v < V) ? feat_count[v] : 0u;
+        const int e_m = (v < V && c == thr_m && c > 0) ? 1 : 0;
+        const int e_a = (v < V && c == thr_a && c > 0) ? 1 : 0;
+        int tot;
+        const int r_m = block_excl_scan_1024(e_m, warp_sums, &sh_total);
+        tot = sh_total;
+        const int is_mask = (v < V) && (c > thr_m || (e_m && tie_m_seen + r_m < need_m));
+        tie_m_seen += tot;
+        const int r_a = block_excl_scan_1024(e_a, warp_sums, &sh_total);
+        tot = sh_total;
+        const int is_sel = (v < V) && (c > thr_a || (e_a && tie_a_seen + r_a < need_a));
+        tie_a_seen += tot;
+        const int is_hot = is_sel && !is_mask;
+        const int s_m = block_excl_scan_1024(is_mask, warp_sums, &sh_total);
+        const int tot_m = sh_total;
+        const int s_h = block_excl_scan_1024(is_hot, warp_sums, &sh_total);
+        const int tot_h = sh_total;
+        if (v < V) {
+            int slot = -1;
+            if (is_mask) slot = mask_assigned + s_m;
+            else if (is_hot) slot = n_mask + hot_assigned + s_h;
+            feat_slot[v] = slot;
+            if (slot >= 0) slot_feat[slot] = v;
+        }
+        mask_assigned += tot_m;
+        hot_assigned += tot_h;
+    }
+    // unused slots (fewer distinct features than slots) point at no feature
+    for (int s = threadIdx.x; s < n_mask + n_hot; s += blockDim.x) {
+        const bool used = (s < n_mask) ? (s < mask_assigned) : (s - n_mask < hot_assigned);
+        if (!used) slot_feat[s] = -1;
+    }
+    if (threadIdx.x == 0) { n_slots[0] = mask_assigned; n_slots[1] = hot_assigned; }
+}
+
+// ---- 3. classify ----------------------------------------------------------------------------
+// Samples are grouped by mask, then by hot-list length, so that the four samples of a search
+// round share the register-resident prefix and the trip count of the hot loop.
+__device__ __forceinline__ uint32_t sort_bin(uint32_t mask, uint32_t n_hot)
+{
+    const uint32_t lc = n_hot > 15u ? 15u : n_hot;
+    return (mask << SOM_PLAN_LEN_BITS) | lc;
+}
+
+// Adds 1 to bins[bin] with one atomic per distinct bin in the warp; returns this thread's
+// rank inside the bin's increment (0-based) plus the old value.
+__device__ __forceinline__ uint32_t warp_agg_inc(uint32_t* bins, uint32_t bin, bool active)
+{
+    const unsigned act = __ballot_sync(0xffffffffu, active);
+    uint32_t res = 0;
+    if (active) {
+        const unsigned peers = __match_any_sync(act, bin);
+        const int lane = threadIdx.x & 31;
+        const int leader = __ffs(peers) - 1;
+        uint32_t old = 0;
+        if (lane == leader) old = atomicAdd(&bins[bin], (uint32_t)__popc(peers));
+        old = __shfl_sync(peers, old, leader);
+        res = old + (uint32_t)__popc(peers & ((1u << lane) - 1u));
+    }
+    return res;
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS)
+k_classify(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
+           const int32_t* __restrict__ feat_slot, int n_mask, uint32_t* __restrict__ pk,
+           uint32_t* __restrict__ ntail, uint32_t* __restrict__ bin_count)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool active = s < n;
+    uint32_t mask = 0, nh = 0, nt = 0;
+    if (active) {
+        const int beg = indptr[s], end = indptr[s + 1];
+        for (int j = beg; j < end; ++j) {
+            const int slot = feat_slot[indices[j]];
+            if (slot < 0) ++nt;
+            else if (slot < n_mask) mask |= 1u << slot;
+            else ++nh;
+        }
+        pk[s] = mask | (nh << 16);
+        ntail[s] = nt;
+    }
+    warp_agg_inc(bin_count, sort_bin(mask, nh), active);
+}
+
+// ---- 4. scan of the sort bins (one block of 1024 threads) --------------------------------------
+__global__ void __launch_bounds__(1024)
+k_scan_bins(const uint32_t* __restrict__ bin_count, uint32_t* __restrict__ bin_start, int n_bins)
+{
+    __shared__ int warp_sums[32];
+    __shared__ int sh_total;
+    const int per = (n_bins + 1023) / 1024;
+    const int b0 = threadIdx.x * per, b1 = min(n_bins, b0 + per);
+    int sum = 0;
+    for (int b = b0; b < b1; ++b) sum += (int)bin_count[b];
+    int run = block_excl_scan_1024(sum, warp_sums, &sh_total);
+    for (int b = b0; b < b1; ++b) {
+        bin_start[b] = (uint32_t)run;
+        run += (int)bin_count[b];
+    }
+}
+
+// ---- 5. scatter + slots ----------------------------------------------------------------------
+__global__ void __launch_bounds__(PLAN_THREADS)
+k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
+                const int32_t* __restrict__ feat_slot, int n_mask, int zero_row,
+                const uint32_t* __restrict__ pk, const uint32_t* __restrict__ ntail,
+                uint32_t* __restrict__ bin_cursor /* starts as bin_start */,
+                uint32_t* __restrict__ slots, uint32_t* __restrict__ overflow,
+                uint32_t* __restrict__ overflow_cursor)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool active = s < n;
+    uint32_t mask = 0, nh = 0, nt = 0, p = 0;
+    if (active) {
+        p = pk[s];
+        mask = p & 0xffffu;
+        nh = p >> 16;
+        nt = ntail[s];
+    }
+    const uint32_t pos = warp_agg_inc(bin_cursor, sort_bin(mask, nh), active);
+    if (!active) return;
+    uint32_t* slot = slots + (size_t)pos * SOM_SLOT_WORDS;
+    const bool fits = nh <= SOM_SLOT_MAX_HOT && nt <= SOM_SLOT_MAX_TAIL;
+    // (an overflow list holds at most 65535 hot and 65535 tail entries; the launcher checks V)
+    slot[0] = fits ? (mask | (nh << 16) | (nt << 24)) : (mask | (SOM_SLOT_NT_OVERFLOW << 24));
+    slot[1] = (uint32_t)s;
+    const int beg = indptr[s], end = indptr[s + 1];
+    if (fits) {
+        uint16_t* hot = reinterpret_cast<uint16_t*>(slot + 2);
+        uint16_t* tail = reinterpret_cast<uint16_t*>(slot + 8);
+        for (int j = beg; j < end; ++j) {
+            const int v = indices[j];
+            const int fs = feat_slot[v];
+            if (fs < 0) *tail++ = (uint16_t)v;
+            else if (fs >= n_mask) *hot++ = (uint16_t)fs;
+        }
+        // unused hot codes point at the all-zero row that follows the table
+        for (uint16_t* e = reinterpret_cast<uint16_t*>(slot + 8); hot < e; ++hot) *hot = (uint16_t)zero_row;
+    } else {
+        const uint32_t nt_pad = (nt + 3u) & ~3u, nh_pad = (nh + 3u) & ~3u;
+        const uint32_t off = atomicAdd(overflow_cursor, nt_pad + nh_pad);
+        // hot-code words all point at the zero row; the list offset and the true counts
+        // (which may not fit the header fields) go where the tail codes would be
+        const uint32_t zz = (uint32_t)zero_row | ((uint32_t)zero_row << 16);
+        for (int w = 2; w < 8; ++w) slot[w] = zz;
+        slot[8] = 0u;  // inline tail codes of an overflow sample: feature 0, a valid row
+        slot[9] = 0u;
+        slot[10] = off;
+        slot[11] = nh | (nt << 16);
+        uint32_t* tail = overflow + off;
+        uint32_t* hot = tail + nt_pad;
+        for (int j = beg; j < end; ++j) {
+            const int v = indices[j];
+            const int fs = feat_slot[v];
+            if (fs < 0) *tail++ = (uint32_t)v;
+            else if (fs >= n_mask) *hot++ = (uint32_t)fs;
+        }
+    }
+}
+
+// The slot array is padded to whole rounds with copies of the last slot.
+__global__ void k_pad_slots(uint4* __restrict__ slots, int64_t n, int64_t n_pad)
+{
+    const int64_t extra = (n_pad - n) * (SOM_SLOT_WORDS / 4);
+    if (threadIdx.x < extra) {
+        const int64_t dst = n * (SOM_SLOT_WORDS / 4) + threadIdx.x;
+        slots[dst] = slots[(n - 1) * (SOM_SLOT_WORDS / 4) + threadIdx.x % (SOM_SLOT_WORDS / 4)];
+    }
+}
+
+}  // namespace
+
+size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_max, SomPlanBuffers* b)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t o = off;
+        off = som_align_up(off + bytes, 256);
+        return o;
+    };
+    b->keys = take((size_t)(n + 16) * 8);
+    b->feat_count = take((size_t)V * 4);
+    b->feat_slot = take((size_t)V * 4);
+    b->slot_feat = take((size_t)n_slots_max * 4);
+    b->n_slots = take(16);
+    b->pk = take((size_t)n * 4);
+    b->ntail = take((size_t)n * 4);
+    b->bin_count = take((size_t)SOM_PLAN_BINS * 4);
+    b->bin_start = take((size_t)SOM_PLAN_BINS * 4);
+    b->slots = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
+    b->overflow = take((size_t)(nnz + 6 * n + 4) * 4);
+    return off;
+}
+
+int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                    char* ws, const SomPlanBuffers& b, int n_mask, int n_hot, uint32_t row_bytes,
+                    cudaStream_t st)
+{
+    uint32_t* feat_count = reinterpret_cast<uint32_t*>(ws + b.feat_count);
+    int32_t* feat_slot = reinterpret_cast<int32_t*>(ws + b.feat_slot);
+    int32_t* slot_feat = reinterpret_cast<int32_t*>(ws + b.slot_feat);
+    int32_t* n_slots = reinterpret_cast<int32_t*>(ws + b.n_slots);
+    uint32_t* pk = reinterpret_cast<uint32_t*>(ws + b.pk);
+    uint32_t* ntail = reinterpret_cast<uint32_t*>(ws + b.ntail);
+    uint32_t* bin_count = reinterpret_cast<uint32_t*>(ws + b.bin_count);
+    uint32_t* bin_start = reinterpret_cast<uint32_t*>(ws + b.bin_start);
+    uint32_t* slots = reinterpret_cast<uint32_t*>(ws + b.slots);
+    uint32_t* overflow = reinterpret_cast<uint32_t*>(ws + b.overflow);
+
+    SOM_CK(h, cudaMemsetAsync(feat_count, 0, (size_t)h->V * 4, st));
+    SOM_CK(h, cudaMemsetAsync(bin_count, 0, (size_t)SOM_PLAN_BINS * 4, st));
+    SOM_CK(h, cudaMemsetAsync(n_slots, 0, 16, st));
+
+    // 1. histogram
+    {
+        const size_t sh = (size_t)h->V * 4;
+        const int use_smem = sh <= (size_t)160 * 1024;
+        int blocks = h->sm_count;
+        if (use_smem) {
+            if (!h->plan_attr_set) {
+                SOM_CK(h, cudaFuncSetAttribute(k_feat_hist, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+                h->plan_attr_set = 1;
+            }
+        } else {
+            blocks = h->sm_count * 2;
+        }
+        k_feat_hist<<<blocks, 1024, use_smem ? sh : 0, st>>>(indptr, indices, n, h->V, use_smem, feat_count);
+        SOM_CK(h, cudaGetLastError());
+    }
+    // 2. select
+    k_select_hot<<<1, 1024, 0, st>>>(feat_count, h->V, n_mask, n_hot, feat_slot, slot_feat, n_slots);
+    SOM_CK(h, cudaGetLastError());
+    // 3. classify
+    const unsigned sblocks = (unsigned)((n + PLAN_THREADS - 1) / PLAN_THREADS);
+    k_classify<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, feat_slot, n_mask, pk, ntail, bin_count);
+    SOM_CK(h, cudaGetLastError());
+    // 4. scan bins
+    k_scan_bins<<<1, 1024, 0, st>>>(bin_count, bin_start, SOM_PLAN_BINS);
+    SOM_CK(h, cudaGetLastError());
+    // 5. scatter + slots (bin_start doubles as the running cursor)
+    k_scatter_slots<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, feat_slot, n_mask, n_mask + n_hot, pk, ntail,
+                                                      bin_start, slots, overflow,
+                                                      reinterpret_cast<uint32_t*>(n_slots) + 2);
+    SOM_CK(h, cudaGetLastError());
+    const int64_t n_pad = (n + 3) / 4 * 4;
+    if (n_pad > n) {
+        k_pad_slots<<<1, 32, 0, st>>>(reinterpret_cast<uint4*>(slots), n, n_pad);
+        SOM_CK(h, cudaGetLastError());
+        h->launches += 1;
+    }
+    h->launches += 5;
+    return SOM_OK;
+}

@@ -1,0 +1,70 @@
+// Layout of the per-batch plan in the handle's workspace, shared by the plan kernels and the
+// row-table search kernel.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+struct som_handle;
+
+#define SOM_PLAN_MASK_FEATURES 16
+#define SOM_PLAN_LEN_BITS 4
+#define SOM_PLAN_BINS (1 << (SOM_PLAN_MASK_FEATURES + SOM_PLAN_LEN_BITS))
+
+// One 48-byte slot per sample, at a fixed address for its sorted position k (slots[k]), so
+// that the search kernel can load it one round ahead without chasing an offset.  As 12 words:
+//   w0        mask of mask features (bits 0-15) | hot codes (16-23) | tail codes (24-31);
+//             a tail count of SOM_SLOT_NT_OVERFLOW marks a sample kept in the overflow buffer
+//   w1        sample index
+//   w2..w7    hot codes 0..11, 16 bits each: row of the feature in the shared-memory table;
+//             unused ones hold the index of the all-zero row that follows the table
+//   w8..w11   tail codes 0..7, 16 bits each: feature id
+//             (overflow sample: w8 = w9 = 0, w10 = offset of its lists in the overflow
+//             buffer, w11 = hot count | tail count << 16)
+// A sample fits when it has at most 12 hot and 8 tail features; the rare others keep 32-bit
+// lists in the overflow buffer: tail ids padded to a multiple of 4, then hot rows likewise
+// (at most 65535 of each).  16-bit codes require V <= 65536 and at most 65536 table rows.
+// The slot array is padded to a multiple of 4 samples with copies of the last slot, so the
+// search kernel always runs whole rounds; the duplicates redo the same idempotent atomicMin.
+#define SOM_SLOT_WORDS 12
+#define SOM_SLOT_MAX_HOT 12
+#define SOM_SLOT_MAX_TAIL 8
+#define SOM_SLOT_NT_OVERFLOW 255u
+
+// byte offsets into the workspace
+struct SomPlanBuffers {
+    size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
+    size_t feat_count;  // u32 [V]
+    size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
+    size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
+    size_t n_slots;     // i32 [4]      mask slots used, hot slots used, overflow cursor
+    size_t pk;          // u32 [n]      mask | n_hot << 16, by sample
+    size_t ntail;       // u32 [n]
+    size_t bin_count;   // u32 [bins]
+    size_t bin_start;   // u32 [bins]
+    size_t slots;       // 48 B [n + 16]
+    size_t overflow;    // u32 [nnz + 6n]
+};
+
+size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_max, SomPlanBuffers* b);
+
+int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
+                    const SomPlanBuffers& b, int n_mask, int n_hot, uint32_t row_bytes, cudaStream_t st);
+
+int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
+                         cudaStream_t st);
+
+int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                               char* ws, const SomPlanBuffers& b, int32_t* bmu, float* dist,
+                               cudaStream_t st);
+
+// Geometry of the row-table kernel for this handle: neurons per range, hot rows that fit.
+struct SomTableGeom {
+    int R;        // neurons per lane (4)
+    int T;        // neurons per range = 8 * R
+    int n_hot;    // hot rows held in shared memory
+    int threads;  // block size
+    size_t smem;  // dynamic shared memory bytes
+};
+SomTableGeom som_table_geometry(const som_handle* h);

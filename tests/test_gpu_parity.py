@@ -63,7 +63,7 @@ def _check_against_oracle(W_host, V, M, indptr, indices, g_bmu, g_dist, rows=Non
     return rep
 
 
-@pytest.mark.parametrize("variant", [1, 0])
+@pytest.mark.parametrize("variant", [1, 2, 0])
 @pytest.mark.parametrize("kind", ["zipf", "permuted", "uniform"])
 def test_config1_full(som_mod, kind, variant):
     """Tiny 16x16 configuration, every sample checked."""
@@ -82,7 +82,7 @@ def test_config1_full(som_mod, kind, variant):
     np.testing.assert_allclose(h.get_norms().cpu().numpy().astype(np.float64), nn, rtol=2e-7)
 
 
-@pytest.mark.parametrize("variant", [1, 0])
+@pytest.mark.parametrize("variant", [1, 2, 0])
 def test_config2_sampled_rows(som_mod, variant):
     """64x64 map, one million samples on the GPU; every 40th row against the oracle."""
     w = synth.CONFIGS[1]
@@ -135,7 +135,7 @@ def _parse_golden():
     return cases
 
 
-@pytest.mark.parametrize("variant", [1, 0])
+@pytest.mark.parametrize("variant", [1, 2, 0])
 @pytest.mark.parametrize("case", _parse_golden(), ids=lambda c: c["name"])
 def test_handbuilt_cases_on_gpu(som_mod, case, variant):
     """Exactly representable weights: winner and distance must be exact, ties to the lowest index."""
@@ -152,7 +152,7 @@ def test_handbuilt_cases_on_gpu(som_mod, case, variant):
         assert g_bmu[s] == b1 and g_dist[s] == np.float32(d1), (case["name"], s, g_bmu[s], g_dist[s])
 
 
-@pytest.mark.parametrize("variant", [1, 0])
+@pytest.mark.parametrize("variant", [1, 2, 0])
 @pytest.mark.parametrize("V,M,n", [(50, 1, 30), (64, 37, 200), (97, 130, 300), (40, 4, 64),
                                    (300, 260, 500), (1000, 1028, 700)])
 def test_ragged_shapes(som_mod, V, M, n, variant):
