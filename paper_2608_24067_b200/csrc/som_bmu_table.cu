@@ -46,13 +46,6 @@ struct Pair2 {  // four fp32 as two packed pairs
     u64 lo, hi;
 };
 
-__device__ __forceinline__ u64 pack2(float a, float b)
-{
-    u64 r;
-    asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(a), "f"(b));
-    return r;
-}
-
 __device__ __forceinline__ void unpack2(u64 v, float& a, float& b)
 {
     asm("mov.b64 {%0,%1}, %2;" : "=f"(a), "=f"(b) : "l"(v));

@@ -6,7 +6,7 @@
 //      give each a slot in the shared-memory row table      (k_select_hot, one block)
 //   3. classify each sample: 16-bit mask of mask features, number of hot / tail features,
 //      and count sort bins keyed on (mask, length class)    (k_classify)
-//   4. exclusive scan of the bins                           (k_scan_bins, one block)
+//   4. exclusive scan of the bins                           (k_scan_*)
 //   5. scatter every sample to its sorted position and write its fixed-size slot there:
 //      hot features as byte offsets of their table row, tail features as feature ids
 //      (k_scatter_slots); the rare sample that does not fit a slot gets an overflow list.
@@ -209,20 +209,63 @@ k_classify(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indic
     warp_agg_inc(bin_count, sort_bin(mask, nh), active);
 }
 
-// ---- 4. scan of the sort bins (one block of 1024 threads) --------------------------------------
+// ---- 4. exclusive scan of the sort bins (three kernels) ----------------------------------------
+constexpr int SCAN_ITEMS = 4;
+constexpr int SCAN_BLOCK = 1024 * SCAN_ITEMS;
+
 __global__ void __launch_bounds__(1024)
-k_scan_bins(const uint32_t* __restrict__ bin_count, uint32_t* __restrict__ bin_start, int n_bins)
+k_scan_reduce(const uint32_t* __restrict__ in, int n, uint32_t* __restrict__ block_sums)
 {
     __shared__ int warp_sums[32];
     __shared__ int sh_total;
-    const int per = (n_bins + 1023) / 1024;
-    const int b0 = threadIdx.x * per, b1 = min(n_bins, b0 + per);
+    const int base = blockIdx.x * SCAN_BLOCK + threadIdx.x * SCAN_ITEMS;
     int sum = 0;
-    for (int b = b0; b < b1; ++b) sum += (int)bin_count[b];
-    int run = block_excl_scan_1024(sum, warp_sums, &sh_total);
-    for (int b = b0; b < b1; ++b) {
-        bin_start[b] = (uint32_t)run;
-        run += (int)bin_count[b];
+    if (base + SCAN_ITEMS <= n) {
+        const uint4 v = *reinterpret_cast<const uint4*>(in + base);
+        sum = (int)(v.x + v.y + v.z + v.w);
+    } else {
+        for (int u = 0; u < SCAN_ITEMS; ++u)
+            if (base + u < n) sum += (int)in[base + u];
+    }
+    block_excl_scan_1024(sum, warp_sums, &sh_total);
+    if (threadIdx.x == 0) block_sums[blockIdx.x] = (uint32_t)sh_total;
+}
+
+__global__ void __launch_bounds__(1024)
+k_scan_block_sums(uint32_t* __restrict__ block_sums, int n_blocks)
+{
+    __shared__ int warp_sums[32];
+    __shared__ int sh_total;
+    int carry = 0;
+    for (int b0 = 0; b0 < n_blocks; b0 += 1024) {
+        const int b = b0 + threadIdx.x;
+        const int v = (b < n_blocks) ? (int)block_sums[b] : 0;
+        const int ex = block_excl_scan_1024(v, warp_sums, &sh_total);
+        if (b < n_blocks) block_sums[b] = (uint32_t)(carry + ex);
+        carry += sh_total;
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+k_scan_apply(const uint32_t* __restrict__ in, int n, const uint32_t* __restrict__ block_sums,
+             uint32_t* __restrict__ out)
+{
+    __shared__ int warp_sums[32];
+    __shared__ int sh_total;
+    const int base = blockIdx.x * SCAN_BLOCK + threadIdx.x * SCAN_ITEMS;
+    int v[SCAN_ITEMS];
+    int sum = 0;
+#pragma unroll
+    for (int u = 0; u < SCAN_ITEMS; ++u) {
+        v[u] = (base + u < n) ? (int)in[base + u] : 0;
+        sum += v[u];
+    }
+    int run = block_excl_scan_1024(sum, warp_sums, &sh_total) + (int)block_sums[blockIdx.x];
+#pragma unroll
+    for (int u = 0; u < SCAN_ITEMS; ++u) {
+        if (base + u < n) out[base + u] = (uint32_t)run;
+        run += v[u];
     }
 }
 
@@ -314,6 +357,7 @@ size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_m
     b->ntail = take((size_t)n * 4);
     b->bin_count = take((size_t)SOM_PLAN_BINS * 4);
     b->bin_start = take((size_t)SOM_PLAN_BINS * 4);
+    b->block_sums = take((size_t)(SOM_PLAN_BINS / SCAN_BLOCK + 2) * 4);
     b->slots = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
     b->overflow = take((size_t)(nnz + 6 * n + 4) * 4);
     return off;
@@ -362,8 +406,16 @@ int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices
     k_classify<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, feat_slot, n_mask, pk, ntail, bin_count);
     SOM_CK(h, cudaGetLastError());
     // 4. scan bins
-    k_scan_bins<<<1, 1024, 0, st>>>(bin_count, bin_start, SOM_PLAN_BINS);
-    SOM_CK(h, cudaGetLastError());
+    {
+        uint32_t* block_sums = reinterpret_cast<uint32_t*>(ws + b.block_sums);
+        const int scan_blocks = (SOM_PLAN_BINS + SCAN_BLOCK - 1) / SCAN_BLOCK;
+        k_scan_reduce<<<scan_blocks, 1024, 0, st>>>(bin_count, SOM_PLAN_BINS, block_sums);
+        SOM_CK(h, cudaGetLastError());
+        k_scan_block_sums<<<1, 1024, 0, st>>>(block_sums, scan_blocks);
+        SOM_CK(h, cudaGetLastError());
+        k_scan_apply<<<scan_blocks, 1024, 0, st>>>(bin_count, SOM_PLAN_BINS, block_sums, bin_start);
+        SOM_CK(h, cudaGetLastError());
+    }
     // 5. scatter + slots (bin_start doubles as the running cursor)
     k_scatter_slots<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, feat_slot, n_mask, n_mask + n_hot, pk, ntail,
                                                       bin_start, slots, overflow,
@@ -375,6 +427,6 @@ int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices
         SOM_CK(h, cudaGetLastError());
         h->launches += 1;
     }
-    h->launches += 5;
+    h->launches += 7;
     return SOM_OK;
 }

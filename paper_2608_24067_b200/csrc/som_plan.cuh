@@ -43,6 +43,7 @@ struct SomPlanBuffers {
     size_t ntail;       // u32 [n]
     size_t bin_count;   // u32 [bins]
     size_t bin_start;   // u32 [bins]
+    size_t block_sums;  // u32 [scan blocks]
     size_t slots;       // 48 B [n + 16]
     size_t overflow;    // u32 [nnz + 6n]
 };
