@@ -115,6 +115,30 @@ int som_validate_csr(som_handle* h, const int32_t* d_indptr, const int32_t* d_in
  */
 int som_get_norms(som_handle* h, float* d_out, void* stream);
 
+/*
+ * som_norms_noalloc - ||w_i||^2 for all M neurons without a handle and without allocating.
+ * (No counterpart in the paper: an integration convenience of this library.)
+ *
+ * For callers that must not call cudaMalloc: a process whose device memory already belongs
+ * to its own pool, where a raw allocation can fail or fragment that pool, or a
+ * latency-critical loop that cannot take the device-wide synchronisation an allocation may
+ * imply.  som_norms keeps per-split partial sums in an allocated workspace; this variant
+ * keeps them in a fixed 4 MiB array built into the library, which every GPU that loads the
+ * library holds until the process exits.
+ *   V, M        as in som_create, with M <= SOM_NOALLOC_MAX_M; a larger M returns
+ *               SOM_ERR_UNSUPPORTED and nothing runs.
+ *   d_codebook  DEVICE pointer, fp32, feature-major, V*M elements (borrowed, read only).
+ *   d_norms     DEVICE pointer, fp32 [M], out: squared norms, fp64 accumulation rounded once.
+ *   stream      the two kernels are enqueued on it; the call does not synchronise.
+ * The first call on each device looks up the array's device address; make that first call
+ * outside any stream capture.  All calls on a device share the array, which keeps the last
+ * call's contents (nothing in it needs clearing: each call overwrites what it reads), so two
+ * calls that may overlap on the GPU must be ordered by the caller or they race.
+ * The device must be the current one; allocates nothing on host or device.
+ */
+#define SOM_NOALLOC_MAX_M 524288
+int som_norms_noalloc(int32_t V, int64_t M, const float* d_codebook, float* d_norms, void* stream);
+
 /* som_destroy - free the handle, its norms and workspace.  NULL is accepted. */
 int som_destroy(som_handle* h);
 

@@ -24,8 +24,10 @@ STATUS_NAMES = {
 EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
-    "som_launch_count", "som_set_option",
+    "som_launch_count", "som_set_option", "som_norms_noalloc",
 ]
+
+NOALLOC_MAX_M = 524288
 
 _lib = None
 
@@ -66,6 +68,8 @@ def load_library():
     lib.som_launch_count.argtypes = [P]
     lib.som_launch_count.restype = I64
     lib.som_set_option.argtypes = [P, INT, I64]
+    lib.som_norms_noalloc.argtypes = [I32, I64, P, P, P]
+    lib.som_norms_noalloc.restype = INT
     for name in ("som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr",
                  "som_get_norms", "som_destroy", "som_last_cuda_error", "som_set_timing",
                  "som_get_timing", "som_set_option"):
@@ -90,6 +94,21 @@ def _host_ptr(t: torch.Tensor, dtype, name: str) -> int:
     if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
         raise TypeError("%s must be a contiguous CPU tensor of %s" % (name, dtype))
     return t.data_ptr()
+
+
+def norms_noalloc(V: int, M: int, codebook: torch.Tensor, out: torch.Tensor, stream=None) -> torch.Tensor:
+    """som_norms_noalloc: squared norms into a caller-provided fp32 CUDA tensor, for callers that
+    must not allocate device memory (no handle, scratch lives inside the library; M is limited
+    to NOALLOC_MAX_M).  ``out`` is written on ``stream``; nothing is allocated here either."""
+    lib = load_library()
+    if codebook.numel() != V * M or out.numel() != M:
+        raise ValueError("codebook must hold V*M elements and out M elements")
+    with torch.cuda.device(codebook.device):
+        rc = lib.som_norms_noalloc(V, M, _dev_ptr(codebook, torch.float32, "codebook"),
+                                   _dev_ptr(out, torch.float32, "out"), _stream_ptr(stream))
+    if rc != SOM_OK:
+        raise SomError(rc, "som_norms_noalloc")
+    return out
 
 
 class Som:
