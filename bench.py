@@ -112,6 +112,25 @@ def _dist_env():
     return ws, rank, lr
 
 
+def replica_first_samples(rank: int, n_batches: int, batch: int):
+    """First sample id of each batch of a rank: replicas draw disjoint parts of one sample stream."""
+    return [(rank * n_batches + bi) * batch for bi in range(n_batches)]
+
+
+def max_over_ranks(ms_local: float, dist, dev) -> float:
+    """Timed region of the job = the slowest rank's (no-op without a process group)."""
+    if dist is None:
+        return float(ms_local)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_samples_per_s(world: int, batch: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every replica processed one batch per step."""
+    return world * batch / (ms_per_step * 1e-3)
+
+
 def _oracle_rate(w: synth.Workload, W_host_slab: np.ndarray, m_slab: int, indptr: np.ndarray,
                  indices: np.ndarray, target_s: float):
     """Time the CPU oracle on a bounded sample of the workload; returns (samples/s, description)."""
@@ -185,8 +204,7 @@ def run_ours(args, w: synth.Workload):
     synth.fill_codebook(w.V, w.M, w.seed, out=W)
     n_batches = max(1, min(4, w.N // w.batch))
     batches = []
-    for bi in range(n_batches):
-        first = (rank * n_batches + bi) * w.batch  # each rank (replica) gets its own samples
+    for first in replica_first_samples(rank, n_batches, w.batch):  # each replica gets its own samples
         batches.append(synth.sample_csr(w.batch, w.V, w.lam, w.seed, zipf_s=w.zipf_s, device=dev,
                                         first_sample=first))
     nnz_mean = float(np.mean([b.nnz / b.n for b in batches]))
@@ -232,12 +250,9 @@ def run_ours(args, w: synth.Workload):
     launches = h.launch_count() - l0
     phases = h.get_timing()
     h.set_timing(False)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, dev)
     ms_per_step = ms_total / args.steps
-    value = ws * w.batch / (ms_per_step * 1e-3)
+    value = aggregate_samples_per_s(ws, w.batch, ms_per_step)
 
     # ---- end to end through the host entry point --------------------------------------------
     hb = [(b.indptr.cpu().pin_memory(), b.indices.cpu().pin_memory()) for b in batches]
@@ -257,11 +272,8 @@ def run_ours(args, w: synth.Workload):
         e2e_step(i + 1)
     e1.record()
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1) / e2e_steps], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item())
-    e2e_value = ws * w.batch / (e2e_ms * 1e-3)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps, dist, dev)
+    e2e_value = aggregate_samples_per_s(ws, w.batch, e2e_ms)
     h2d = int(np.mean([ip.numel() * 4 + ix.numel() * 4 for ip, ix in hb]))
     d2h = w.batch * 8
 
