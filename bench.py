@@ -215,6 +215,8 @@ def run_ours(args, w: synth.Workload):
         h.set_option(1, args.hot_rows)
     if args.threads:
         h.set_option(2, args.threads)
+    if args.lane_neurons:
+        h.set_option(3, args.lane_neurons)
     out_bmu = torch.empty(w.batch, dtype=torch.int32, device=dev)
     out_dist = torch.empty(w.batch, dtype=torch.float32, device=dev)
 
@@ -350,6 +352,7 @@ def main():
     ap.add_argument("--variant", type=int, default=None, help="search kernel variant (library option 0)")
     ap.add_argument("--hot-rows", type=int, default=0, help="row-table kernel: hot rows in shared memory")
     ap.add_argument("--threads", type=int, default=0, help="row-table kernel: block size (512 or 1024)")
+    ap.add_argument("--lane-neurons", type=int, default=0, help="row-table kernel: neurons per lane (4 or 8)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]

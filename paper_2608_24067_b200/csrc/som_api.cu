@@ -330,6 +330,11 @@ int som_set_option(som_handle* h, int key, int64_t value)
         h->opt_hot_rows = value;
         return SOM_OK;
     }
+    if (key == 3) {
+        if (value != 0 && value != 4 && value != 8) return SOM_ERR_INVALID_ARG;
+        h->opt_r = value;
+        return SOM_OK;
+    }
     if (key == 2) {
         if (value != 0 && value != 512 && value != 768 && value != 1024) return SOM_ERR_INVALID_ARG;
         h->opt_threads = value;

@@ -33,17 +33,26 @@
 #include "som_internal.cuh"
 #include "som_plan.cuh"
 
+#ifndef SOM_TAIL_LOAD_CG
+#define SOM_TAIL_LOAD_CG 1
+#endif
+
 namespace {
 
-constexpr int T = 32;       // neurons per range
-constexpr int ROWB = 128;   // bytes of one table row
 constexpr int CHUNK = 128;  // samples a warp takes at a time
+constexpr int RING_STAGE = 224;  // bytes of one ring stage: 4 slots + 4 keys
 constexpr int SLOT_Q = SOM_SLOT_WORDS / 4;  // uint4 per slot
 
 typedef unsigned long long u64;
 
 struct Pair2 {  // four fp32 as two packed pairs
     u64 lo, hi;
+};
+
+// R neurons of one lane: H = R / 4 groups of four consecutive neurons, 32 neurons apart
+template <int H>
+struct Acc {
+    Pair2 g[H];
 };
 
 __device__ __forceinline__ void unpack2(u64 v, float& a, float& b)
@@ -66,19 +75,46 @@ __device__ __forceinline__ Pair2 lds_row(const unsigned char* p)
     return r;
 }
 
-// 128-bit read of a tail row slice through the read-only path.  Normal eviction priority on
-// purpose: an L1::no_allocate hint also demotes the line to evict-first in L2, and the slab
-// rows are exactly what has to stay L2-resident.
+// 128-bit read of a tail row slice, cached in L2 only.  Two things matter here: an
+// L1::no_allocate hint would also demote the line to evict-first in L2, and the slab rows are
+// exactly what has to stay L2-resident; and a load that allocates in L1 would push the
+// prefetched slot stream out of the small L1 left beside the shared-memory table.
 __device__ __forceinline__ Pair2 ldg_row(const float* p)
 {
     Pair2 r;
+#if SOM_TAIL_LOAD_CG
+    asm("ld.global.cg.v2.b64 {%0,%1}, [%2];" : "=l"(r.lo), "=l"(r.hi) : "l"(p));
+#else
     asm("ld.global.nc.v2.b64 {%0,%1}, [%2];" : "=l"(r.lo), "=l"(r.hi) : "l"(p));
+#endif
     return r;
 }
 
-__device__ __forceinline__ void prefetch_l1(const void* p)
+template <int H>
+__device__ __forceinline__ void sub_acc(Acc<H>& a, const Acc<H>& w)
 {
-    asm volatile("prefetch.global.L1 [%0];" :: "l"(p));
+#pragma unroll
+    for (int x = 0; x < H; ++x) sub_pair(a.g[x], w.g[x]);
+}
+
+// a lane's slice of a shared-memory row: 16 bytes per group, groups 128 bytes apart
+template <int H>
+__device__ __forceinline__ Acc<H> lds_acc(const unsigned char* p)
+{
+    Acc<H> r;
+#pragma unroll
+    for (int x = 0; x < H; ++x) r.g[x] = lds_row(p + 128 * x);
+    return r;
+}
+
+// a lane's slice of a codebook row in global memory
+template <int H>
+__device__ __forceinline__ Acc<H> ldg_acc(const float* p)
+{
+    Acc<H> r;
+#pragma unroll
+    for (int x = 0; x < H; ++x) r.g[x] = ldg_row(p + 32 * x);
+    return r;
 }
 
 __device__ __forceinline__ uint32_t lo16(uint32_t w) { return w & 0xffffu; }
@@ -92,19 +128,28 @@ __device__ __forceinline__ const float* row_ptr(const float* base, uint32_t code
     return p;
 }
 
-#define SOM_HOT(code) sub_pair(acc, lds_row(tab_q + ((code) << 7)))
+#define SOM_HOT(code) sub_acc<H>(acc, lds_acc<H>(tab_q + (code) * ROWB))
+#define SOM_TAIL(code) ldg_acc<H>(row_ptr(w_q, (code), stride_b))
 
-template <int THREADS>
+// R = neurons per lane (4 or 8); a team of 8 lanes covers T = 8*R neurons of one sample.
+template <int R, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1)
 k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
             const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
             u64* __restrict__ keys, int parts, int64_t part_len, int n_units)
 {
+    constexpr int H = R / 4;
+    constexpr int T = 8 * R;
+    constexpr int ROWB = T * 4;
     constexpr int WARPS = THREADS / 32;
     extern __shared__ __align__(16) unsigned char tab[];
     __shared__ int next_chunk;
     __shared__ __align__(16) float hn_sh[T];  // ||w||^2/2 of the range's neurons (+inf past M)
+    // Warp-private ring of two stages; a stage holds the four slots (192 B) and four keys (32 B)
+    // of one round.  The bytes of round r+2 are in flight in registers, round r+1 is being
+    // stored, round r is being read: slot and key latency never sits on the critical path.
+    __shared__ __align__(16) unsigned char ring_sh[WARPS * 2 * RING_STAGE];
     float* tab_f = reinterpret_cast<float*>(tab);
 
     const int lane = threadIdx.x & 31;
@@ -113,10 +158,11 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
     const int sub = lane >> 3;
     const float inf = __int_as_float(0x7f800000);
     const unsigned char* tab_q = tab + q * 16;
+    const unsigned char* hn_q = reinterpret_cast<const unsigned char*>(hn_sh) + q * 16;
     const uint32_t stride_b = (uint32_t)M * 4u;  // the launcher guarantees M < 2^30
 
     // row n_rows of the table is all zeros: the target of padded hot codes
-    if (threadIdx.x < T) tab_f[n_rows * T + threadIdx.x] = 0.f;
+    for (int c = threadIdx.x; c < T; c += THREADS) tab_f[n_rows * T + c] = 0.f;
 
     int cur_range = -1;
     const float* w_q = W;
@@ -129,24 +175,32 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
         if (threadIdx.x == 0) next_chunk = 0;
         if (range != cur_range) {
             for (int row0 = warp * 4; row0 < n_rows; row0 += WARPS * 4) {
-                float v[4];
+                float v[4][H];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int row = row0 + u;
                     const int f = row < n_rows ? slot_feat[row] : -1;
-                    v[u] = (f >= 0 && i0 + lane < M) ? __ldg(W + (int64_t)f * M + i0 + lane) : 0.f;
+#pragma unroll
+                    for (int x = 0; x < H; ++x) {
+                        const int64_t i = i0 + 32 * x + lane;
+                        v[u][x] = (f >= 0 && i < M) ? __ldg(W + (int64_t)f * M + i) : 0.f;
+                    }
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (row0 + u < n_rows) tab_f[(row0 + u) * T + lane] = v[u];
+                    if (row0 + u < n_rows) {
+#pragma unroll
+                        for (int x = 0; x < H; ++x) tab_f[(row0 + u) * T + 32 * x + lane] = v[u][x];
+                    }
             }
             cur_range = range;
+            // Lanes (or their upper group) past the last neuron still read valid addresses and
+            // carry +inf scores, so they never beat a real neuron and need no predicate below.
+            // With R = 8 the launcher guarantees M % 64 == 0, so a lane is all in or all out.
             const int64_t i_lane = i0 + 4 * q;
             i_first = (uint32_t)i_lane;
-            // lanes past the last neuron read a valid address and carry +inf scores, so they
-            // never beat a real neuron and need no predicate in the loop
             w_q = W + (i_lane < M ? i_lane : 0);
-            if (threadIdx.x < T) hn_sh[threadIdx.x] = (i0 + threadIdx.x < M) ? hnorm[i0 + threadIdx.x] : inf;
+            for (int c = threadIdx.x; c < T; c += THREADS) hn_sh[c] = (i0 + c < M) ? hnorm[i0 + c] : inf;
         }
         __syncthreads();
 
@@ -155,7 +209,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
         const int n_chunks = (int)((k_end - k_begin + CHUNK - 1) / CHUNK);
 
         uint32_t curmask = 0;
-        Pair2 base = lds_row(reinterpret_cast<const unsigned char*>(hn_sh) + q * 16);
+        Acc<H> base = lds_acc<H>(hn_q);
         for (;;) {
             int chunk = 0;
             if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
@@ -164,14 +218,40 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
             const int64_t w0 = k_begin + (int64_t)chunk * CHUNK;
             const int rounds = (int)(min(k_end, w0 + CHUNK) - w0) >> 2;
 
-            const uint4* ps = slots + (w0 + sub) * SLOT_Q;  // this team's slot, 4 slots per round
+            // Ring feed: lanes 0..11 carry the twelve 16-byte pieces of a round's four slots,
+            // lanes 12..13 the two 16-byte pieces of its four keys.
+            unsigned char* ring = ring_sh + warp * 2 * RING_STAGE;
+            const uint4* feed = (lane < 12) ? slots + w0 * SLOT_Q + lane
+                                            : reinterpret_cast<const uint4*>(keys + w0) + (lane - 12);
+            const int feed_step = (lane < 12) ? 4 * SLOT_Q : 2;  // uint4 per round
+            const bool feeder = lane < 14;
+            unsigned char* my_store = ring + (lane < 12 ? lane * 16 : 192 + (lane - 12) * 16);
+            const unsigned char* my_slot = ring + sub * 48;
+            const unsigned char* my_key = ring + 192 + sub * 8;
+            uint4 g = make_uint4(0u, 0u, 0u, 0u);
+            __syncwarp();  // the previous chunk's last reads of the ring are done
+            if (feeder) {
+                *reinterpret_cast<uint4*>(my_store) = __ldcg(feed);  // round 0 -> stage 0
+                g = __ldcg(feed + feed_step);                        // round 1, in flight
+            }
+            feed += 2 * feed_step;
+            __syncwarp();
             u64* pk = keys + w0 + sub;
-            // L1 prefetch of the slot stream, six rounds ahead (the workspace behind the slot
-            // array is mapped, so running past its end is harmless)
-            const char* pf = reinterpret_cast<const char*>(slots + (w0 + 24) * SLOT_Q) + (lane & 1) * 128;
-            uint4 s0 = __ldg(ps), s1 = __ldg(ps + 1), s2 = __ldg(ps + 2);
-            u64 key = __ldcg(pk);
             for (int r = 0; r < rounds; ++r) {
+                const int st = (r & 1) * RING_STAGE;
+                const uint4 s0 = *reinterpret_cast<const uint4*>(my_slot + st);
+                const uint4 s1 = *reinterpret_cast<const uint4*>(my_slot + st + 16);
+                const uint4 s2 = *reinterpret_cast<const uint4*>(my_slot + st + 32);
+                const u64 key0 = *reinterpret_cast<const u64*>(my_key + st);
+                // round r+1 goes into the other stage (its previous content, round r-1, was
+                // consumed a round ago); round r+2 goes in flight.  The slot and key arrays
+                // are padded, so the loads past the chunk's end stay in bounds.
+                if (feeder) {
+                    *reinterpret_cast<uint4*>(my_store + (RING_STAGE - st)) = g;
+                    g = __ldcg(feed);
+                }
+                feed += feed_step;
+                __syncwarp();
                 const uint32_t hdr = s0.x;
                 const uint32_t nt = hdr >> 24;  // SOM_SLOT_NT_OVERFLOW marks an overflow sample
                 const uint32_t nh = (hdr >> 16) & 0xffu;
@@ -179,26 +259,24 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                 const bool p0 = nt > 0, p1 = nt > 1, p2 = nt > 2, p3 = nt > 3;
 
                 // ---- the first four tail rows of this sample go in flight first ---------------
-                Pair2 tr0, tr1, tr2, tr3;
-                if (p0) tr0 = ldg_row(row_ptr(w_q, lo16(s2.x), stride_b));
-                if (p1) tr1 = ldg_row(row_ptr(w_q, hi16(s2.x), stride_b));
-                if (p2) tr2 = ldg_row(row_ptr(w_q, lo16(s2.y), stride_b));
-                if (p3) tr3 = ldg_row(row_ptr(w_q, hi16(s2.y), stride_b));
-                if (lane < 2) prefetch_l1(pf);
-                pf += 4 * SOM_SLOT_WORDS * 4;
+                Acc<H> tr0, tr1, tr2, tr3;
+                if (p0) tr0 = SOM_TAIL(lo16(s2.x));
+                if (p1) tr1 = SOM_TAIL(hi16(s2.x));
+                if (p2) tr2 = SOM_TAIL(lo16(s2.y));
+                if (p3) tr3 = SOM_TAIL(hi16(s2.y));
 
                 // ---- mask prefix ------------------------------------------------------------
                 if (mask != curmask) {
-                    base = lds_row(reinterpret_cast<const unsigned char*>(hn_sh) + q * 16);
+                    base = lds_acc<H>(hn_q);
                     uint32_t mm = mask;
                     while (mm) {
                         const int b = __ffs(mm) - 1;
                         mm &= mm - 1;
-                        sub_pair(base, lds_row(tab_q + b * ROWB));
+                        sub_acc<H>(base, lds_acc<H>(tab_q + b * ROWB));
                     }
                     curmask = mask;
                 }
-                Pair2 acc = base;
+                Acc<H> acc = base;
 
                 // ---- hot rows: exactly max(nh over the warp) steps; shorter lists are padded
                 //      with the zero row, so a step carries no predicate -------------------------
@@ -221,16 +299,16 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7 / overflow fields
 
                 // ---- tail rows ------------------------------------------------------------------
-                if (p0) sub_pair(acc, tr0);
-                if (p1) sub_pair(acc, tr1);
-                if (p2) sub_pair(acc, tr2);
-                if (p3) sub_pair(acc, tr3);
+                if (p0) sub_acc<H>(acc, tr0);
+                if (p1) sub_acc<H>(acc, tr1);
+                if (p2) sub_acc<H>(acc, tr2);
+                if (p3) sub_acc<H>(acc, tr3);
                 if (nt > 4) {
                     if (nt != SOM_SLOT_NT_OVERFLOW) {
-                        sub_pair(acc, ldg_row(row_ptr(w_q, lo16(t45), stride_b)));
-                        if (nt > 5) sub_pair(acc, ldg_row(row_ptr(w_q, hi16(t45), stride_b)));
-                        if (nt > 6) sub_pair(acc, ldg_row(row_ptr(w_q, lo16(t67), stride_b)));
-                        if (nt > 7) sub_pair(acc, ldg_row(row_ptr(w_q, hi16(t67), stride_b)));
+                        sub_acc<H>(acc, SOM_TAIL(lo16(t45)));
+                        if (nt > 5) sub_acc<H>(acc, SOM_TAIL(hi16(t45)));
+                        if (nt > 6) sub_acc<H>(acc, SOM_TAIL(lo16(t67)));
+                        if (nt > 7) sub_acc<H>(acc, SOM_TAIL(hi16(t67)));
                     } else {
                         // rare: a sample that does not fit its slot keeps 32-bit lists in the
                         // overflow buffer (w10 = offset, w11 = hot count | tail count << 16).
@@ -239,32 +317,31 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                         const uint32_t* ol = overflow + t45;
                         const uint32_t onh = lo16(t67), ont = hi16(t67);
                         const uint32_t nt_pad = (ont + 3u) & ~3u;
-                        for (uint32_t j = 0; j < ont; ++j)
-                            sub_pair(acc, ldg_row(row_ptr(w_q, __ldg(ol + j), stride_b)));
+                        for (uint32_t j = 0; j < ont; ++j) sub_acc<H>(acc, SOM_TAIL(__ldg(ol + j)));
                         for (uint32_t j = 0; j < onh; ++j) SOM_HOT(__ldg(ol + nt_pad + j));
                     }
                 }
 
-                // ---- next round's slot and key (their lines were prefetched into L1); the slot
-                //      array is padded, so the load after the last round is in bounds -------------
-                const u64 key0 = key;
-                ps += 4 * SLOT_Q;
                 pk += 4;
-                s0 = __ldg(ps);
-                s1 = __ldg(ps + 1);
-                s2 = __ldg(ps + 2);
-                key = __ldcg(pk);
 
                 // ---- lane-local argmin, rare atomic combine ------------------------------------
-                float a0, a1, a2, a3;
-                unpack2(acc.lo, a0, a1);
-                unpack2(acc.hi, a2, a3);
-                const float mn = fminf(fminf(a0, a1), fminf(a2, a3));
+                float a[R];
+#pragma unroll
+                for (int x = 0; x < H; ++x) {
+                    unpack2(acc.g[x].lo, a[4 * x], a[4 * x + 1]);
+                    unpack2(acc.g[x].hi, a[4 * x + 2], a[4 * x + 3]);
+                }
+                float mn = fminf(fminf(a[0], a[1]), fminf(a[2], a[3]));
+                if (R == 8) mn = fminf(mn, fminf(fminf(a[4 % R], a[5 % R]), fminf(a[6 % R], a[7 % R])));
                 const uint32_t cu = (uint32_t)(key0 >> 32);
                 const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
                 if (!(mn > cs)) {
-                    const int rr = (a0 == mn) ? 0 : ((a1 == mn) ? 1 : ((a2 == mn) ? 2 : 3));
-                    atomicMin(pk - 4, som_pack_key(mn, i_first + rr));
+                    int rr = R - 1;
+#pragma unroll
+                    for (int j = R - 2; j >= 0; --j)
+                        if (a[j] == mn) rr = j;  // lowest neuron among the lane's minima
+                    const uint32_t neuron = i_first + (uint32_t)((rr >> 2) * 32 + (rr & 3));
+                    atomicMin(pk - 4, som_pack_key(mn, neuron));
                 }
             }
         }
@@ -289,10 +366,11 @@ __global__ void k_finalize_sorted(const float* __restrict__ W, const double* __r
     dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
 }
 
-template <int THREADS>
+template <int R, int THREADS>
 int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& b, int n_hot, size_t smem,
                  cudaStream_t st)
 {
+    constexpr int T = 8 * R;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
     const int n_ranges = (int)((h->M + T - 1) / T);
     int parts = (int)(n / 8192);
@@ -305,7 +383,7 @@ int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& 
     if (n_units64 > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
     const int n_units = (int)n_units64;
     const int grid = n_units < h->sm_count ? n_units : h->sm_count;
-    auto kern = k_bmu_table<THREADS>;
+    auto kern = k_bmu_table<R, THREADS>;
     SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<grid, THREADS, smem, st>>>(h->W, h->hnorm, h->M,
                                       reinterpret_cast<const int32_t*>(ws + b.slot_feat),
@@ -323,14 +401,20 @@ int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& 
 SomTableGeom som_table_geometry(const som_handle* h)
 {
     SomTableGeom g;
-    g.R = 4;
-    g.T = T;
-    g.threads = (h->opt_threads == 512) ? 512 : (h->opt_threads == 768 ? 768 : 1024);
-    int max_rows = (int)((227 * 1024 - 1024) / ROWB) - SOM_PLAN_MASK_FEATURES - 1;
-    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : 1536;
+    // 8 neurons per lane (half as many rounds for the same work) whenever the neuron count is
+    // a multiple of the 64-neuron range it needs; it wants 128 registers, hence 512 threads
+    g.R = (h->opt_r != 4 && h->M % 64 == 0) ? 8 : 4;
+    g.T = 8 * g.R;
+    const int row_bytes = g.T * 4;
+    const int def_threads = g.R == 8 ? 512 : 1024;
+    g.threads = (h->opt_threads == 512 || h->opt_threads == 768 || h->opt_threads == 1024)
+                    ? (int)h->opt_threads : def_threads;
+    // 227 KB per block, minus the static shared memory (slot rings, norms) of the kernel
+    int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
+    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (g.R == 8 ? 760 : 1536);
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
-    g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * ROWB;  // + the zero row
+    g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * row_bytes;  // + the zero row
     return g;
 }
 
@@ -338,9 +422,14 @@ int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffer
                          cudaStream_t st)
 {
     const SomTableGeom g = som_table_geometry(h);
-    if (g.threads == 1024) return launch_table<1024>(h, n, ws, b, n_hot, g.smem, st);
-    if (g.threads == 768) return launch_table<768>(h, n, ws, b, n_hot, g.smem, st);
-    return launch_table<512>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.R == 8) {
+        if (g.threads == 1024) return launch_table<8, 1024>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 768) return launch_table<8, 768>(h, n, ws, b, n_hot, g.smem, st);
+        return launch_table<8, 512>(h, n, ws, b, n_hot, g.smem, st);
+    }
+    if (g.threads == 1024) return launch_table<4, 1024>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 768) return launch_table<4, 768>(h, n, ws, b, n_hot, g.smem, st);
+    return launch_table<4, 512>(h, n, ws, b, n_hot, g.smem, st);
 }
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,

@@ -37,6 +37,7 @@ struct som_handle {
     int64_t opt_variant;   // 0 auto, 1 direct-load kernel, 2 row-table kernel
     int64_t opt_hot_rows;  // 0 = default number of hot rows in shared memory
     int64_t opt_threads;   // block size of the row-table kernel: 0 (default 512), 512 or 1024
+    int64_t opt_r;         // neurons per lane of the row-table kernel: 0/4 or 8
     int plan_attr_set;
     int32_t* host_pair;    // pinned, 2 ints: read-back of indptr[0], indptr[n]
 };

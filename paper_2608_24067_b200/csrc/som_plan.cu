@@ -161,12 +161,13 @@ k_select_hot(const uint32_t* __restrict__ feat_count, int V, int n_mask, int n_h
 }
 
 // ---- 3. classify ----------------------------------------------------------------------------
-// Samples are grouped by mask, then by hot-list length, so that the four samples of a search
-// round share the register-resident prefix and the trip count of the hot loop.
-__device__ __forceinline__ uint32_t sort_bin(uint32_t mask, uint32_t n_hot)
+// Samples are grouped by mask, then by hot count, then by tail count, so that the four samples
+// of a search round share the register-resident prefix and the trip counts of both row loops.
+__device__ __forceinline__ uint32_t sort_bin(uint32_t mask, uint32_t n_hot, uint32_t n_tail)
 {
-    const uint32_t lc = n_hot > 15u ? 15u : n_hot;
-    return (mask << SOM_PLAN_LEN_BITS) | lc;
+    const uint32_t ch = n_hot > 15u ? 15u : n_hot;
+    const uint32_t ct = n_tail > 7u ? 7u : n_tail;
+    return (mask << SOM_PLAN_LEN_BITS) | (ch << 3) | ct;
 }
 
 // Adds 1 to bins[bin] with one atomic per distinct bin in the warp; returns this thread's
@@ -206,7 +207,7 @@ k_classify(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indic
         pk[s] = mask | (nh << 16);
         ntail[s] = nt;
     }
-    warp_agg_inc(bin_count, sort_bin(mask, nh), active);
+    warp_agg_inc(bin_count, sort_bin(mask, nh, nt), active);
 }
 
 // ---- 4. exclusive scan of the sort bins (three kernels) ----------------------------------------
@@ -287,7 +288,7 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
         nh = p >> 16;
         nt = ntail[s];
     }
-    const uint32_t pos = warp_agg_inc(bin_cursor, sort_bin(mask, nh), active);
+    const uint32_t pos = warp_agg_inc(bin_cursor, sort_bin(mask, nh, nt), active);
     if (!active) return;
     uint32_t* slot = slots + (size_t)pos * SOM_SLOT_WORDS;
     const bool fits = nh <= SOM_SLOT_MAX_HOT && nt <= SOM_SLOT_MAX_TAIL;

@@ -9,7 +9,7 @@
 struct som_handle;
 
 #define SOM_PLAN_MASK_FEATURES 16
-#define SOM_PLAN_LEN_BITS 4
+#define SOM_PLAN_LEN_BITS 7 /* hot count (4 bits) and tail count (3 bits) */
 #define SOM_PLAN_BINS (1 << (SOM_PLAN_MASK_FEATURES + SOM_PLAN_LEN_BITS))
 
 // One 48-byte slot per sample, at a fixed address for its sorted position k (slots[k]), so

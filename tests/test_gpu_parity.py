@@ -101,6 +101,25 @@ def test_config2_sampled_rows(som_mod, variant):
     assert np.array_equal(dist2.cpu().numpy().view(np.uint32), g_dist.view(np.uint32))
 
 
+@pytest.mark.parametrize("lane_neurons,threads", [(4, 1024), (4, 768), (8, 512), (8, 768)])
+def test_row_table_geometries(som_mod, lane_neurons, threads):
+    """Both lane widths of the row-table kernel (32- and 64-neuron ranges) and block sizes,
+    with permuted feature ids so that the hot features are not the low ids."""
+    V, M, n = 30_000, 1_024, 60_000
+    W = synth.fill_codebook(V, M, 3, device="cuda")
+    b = synth.sample_csr(n, V, 11.0, 3, device="cuda", permute_ids=True)
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, 2)
+    h.set_option(3, lane_neurons)
+    h.set_option(2, threads)
+    h.norms()
+    bmu, dist = h.bmu(b.indptr, b.indices)
+    torch.cuda.synchronize()
+    rows = np.arange(0, n, 7)
+    _check_against_oracle(W.cpu().numpy(), V, M, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
+                          bmu.cpu().numpy(), dist.cpu().numpy(), rows)
+
+
 def test_config3_full_size_sampled_rows(som_mod):
     """128x128 map at its full size (4M samples, the benchmark's launch configuration);
     a strided sample of rows against the oracle, plus properties that hold for all rows."""
