@@ -159,7 +159,7 @@ int som_last_cuda_error(const som_handle* h);
  * som_launch_count returns how many kernels this handle has launched since creation.
  * som_set_option tunes kernel selection: key 0 = search kernel variant (0 auto, 1 direct-load
  * kernel, 2 shared-memory row-table kernel where M % 4 == 0 and V <= 65536); key 1 = hot rows kept in shared
- * memory by the row-table kernel (0 = default); key 2 = its block size (0 = default, 512, 768, 1024);
+ * memory by the row-table kernel (0 = default); key 2 = its block size (0 = default, 512, 640, 768, 896, 1024);
  * key 3 = neurons per lane there (0 = default, 4, 8; 8 needs M % 64 == 0).
  */
 int som_set_timing(som_handle* h, int enable);

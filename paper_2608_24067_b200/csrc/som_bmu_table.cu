@@ -402,12 +402,14 @@ SomTableGeom som_table_geometry(const som_handle* h)
 {
     SomTableGeom g;
     // 8 neurons per lane (half as many rounds for the same work) whenever the neuron count is
-    // a multiple of the 64-neuron range it needs; it wants 128 registers, hence 512 threads
+    // a multiple of the 64-neuron range it needs; 640 threads leave it 96 registers, the
+    // measured optimum between resident warps and spills
     g.R = (h->opt_r != 4 && h->M % 64 == 0) ? 8 : 4;
     g.T = 8 * g.R;
     const int row_bytes = g.T * 4;
-    const int def_threads = g.R == 8 ? 512 : 1024;
-    g.threads = (h->opt_threads == 512 || h->opt_threads == 768 || h->opt_threads == 1024)
+    const int def_threads = g.R == 8 ? 640 : 1024;
+    g.threads = (h->opt_threads == 512 || h->opt_threads == 640 || h->opt_threads == 768 ||
+                 h->opt_threads == 896 || h->opt_threads == 1024)
                     ? (int)h->opt_threads : def_threads;
     // 227 KB per block, minus the static shared memory (slot rings, norms) of the kernel
     int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
@@ -424,11 +426,15 @@ int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffer
     const SomTableGeom g = som_table_geometry(h);
     if (g.R == 8) {
         if (g.threads == 1024) return launch_table<8, 1024>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 896) return launch_table<8, 896>(h, n, ws, b, n_hot, g.smem, st);
         if (g.threads == 768) return launch_table<8, 768>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 640) return launch_table<8, 640>(h, n, ws, b, n_hot, g.smem, st);
         return launch_table<8, 512>(h, n, ws, b, n_hot, g.smem, st);
     }
     if (g.threads == 1024) return launch_table<4, 1024>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 896) return launch_table<4, 896>(h, n, ws, b, n_hot, g.smem, st);
     if (g.threads == 768) return launch_table<4, 768>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 640) return launch_table<4, 640>(h, n, ws, b, n_hot, g.smem, st);
     return launch_table<4, 512>(h, n, ws, b, n_hot, g.smem, st);
 }
 
