@@ -291,10 +291,13 @@ def run_ours(args, w: synth.Workload):
     search_s = max(phases["search_ms"], 1e-6) * 1e-3
     achieved = adds / search_s
     alg_bytes = w.V * w.M * 4 + sum(b.nnz * 4 + (b.n + 1) * 4 for b in batches) / n_batches + w.batch * 8
+    # DRAM bytes per launch of the search kernel from the committed ncu summary of this workload
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    tpath = os.path.join(ROOT, "profiles", "k_bmu_table_%s.md" % w.name)
     if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get(w.name)
+        for tl in open(tpath):
+            if tl.startswith("traffic_bytes_per_launch"):
+                traffic = float(tl.split("=")[1])
     roofline = {
         "bound": "alu", "kernel": "fused BMU search", "achieved": achieved / 1e12, "peak": add_peak / 1e12,
         "unit": "TFLOP/s", "frac": achieved / add_peak, "traffic": traffic,
