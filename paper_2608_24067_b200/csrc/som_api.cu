@@ -183,7 +183,7 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
         SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
         if ((rc = som_launch_plan(h, d_indptr, d_indices, n_samples, ws, pb, SOM_PLAN_MASK_FEATURES,
-                                  geom.n_hot, (uint32_t)geom.T * 4u, st)))
+                                  geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
         if ((rc = som_launch_bmu_table(h, n_samples, ws, pb, geom.n_hot, st))) return rc;

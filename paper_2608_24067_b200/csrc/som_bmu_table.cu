@@ -1,32 +1,34 @@
 // Row-table BMU search kernel (the fast path of som_bmu) and its finalisation.
 //
-// Decomposition (Section 3.3 of the paper, re-planned for B200): a work unit is a
-// neuron range of T = 32 neurons times a contiguous part of the mask-sorted sample list.
-// One persistent block per SM walks units in range-major order, so that at any time only a
-// few neuron ranges are live and their codebook slabs W[:, i0..i0+T) stay L2-resident while
-// HBM sees the codebook once per batch.  Inside a unit the warps pull chunks of samples from
-// a shared counter, which keeps them busy whatever the mix of row lengths.
+// Decomposition (Section 3.3 of the paper, re-planned for B200): a work unit is a neuron
+// range of T = 8*R neurons (R = 8 or 4 per lane) times a contiguous part of the mask-sorted
+// sample list.  One persistent block per SM walks units in range-major order, so that at any
+// time only a few neuron ranges are live and their codebook slabs W[:, i0..i0+T) stay
+// L2-resident while HBM sees the codebook about once per batch.  Inside a unit the warps pull
+// chunks of samples from a shared counter, which keeps them busy whatever the mix of row
+// lengths.
 //
 // Inside a block the rows W[v*M + i0 .. i0+T) of the batch's hottest features (the row
 // table) are staged in shared memory once per unit.  Eight lanes form a team that owns one
-// sample at a time; a lane keeps 4 score accumulators in registers and subtracts, for every
-// code of the sample, a 128-bit slice of the row: a shared-memory read for hot features, a
-// coalesced 128-bit global read of the L2-resident slab for tail features.  The team's 8 loads
-// cover one contiguous 128-byte row segment.  Adds are issued as packed f32x2 operations,
-// which halves their issue slots.  The accumulators start from
-// ||w||^2/2 - sum(rows of the sample's mask features), which is held in registers across
-// consecutive samples that share the mask (they are adjacent after the plan's sort).
+// sample at a time; a lane keeps R score accumulators in registers (R/4 groups of four
+// neurons, 32 neurons apart) and subtracts, for every code of the sample, one 128-bit slice of
+// the row per group: a shared-memory read for hot features, a coalesced 128-bit L2-only read
+// of the L2-resident slab for tail features.  The team's 8 loads of a group cover one
+// contiguous 128-byte row segment.  Subtractions are packed f32x2 operations, which halves
+// their issue slots.  The accumulators start from ||w||^2/2 - sum(rows of the sample's mask
+// features), which is held in registers across consecutive samples that share the mask (they
+// are adjacent after the plan's sort).
 //
-// Latency: a sample's 48-byte slot sits at a fixed address for its sorted position, so the
-// slot stream is prefetched into L1 several rounds ahead and the next slot and key are loaded
-// into registers while the current sample finishes.  A sample's first four tail rows go in
-// flight at the top of its round and are consumed after the hot rows; 32 resident warps cover
-// what latency remains, which is why the kernel is held to 64 registers per thread.
-// Instruction count: the hot loop is a jump table on the warp's longest hot list (shorter
-// lists are padded with a zero row), so a step costs extract + address + load + two packed
-// subtracts and no predicate.
+// Feeding the teams: a sample's 48-byte slot sits at a fixed address for its sorted position.
+// Each warp owns a two-stage ring in shared memory; 14 of its lanes fetch the slot and key
+// bytes of round r+2 into registers, store those of round r+1, and every team reads round r
+// from the ring, so slot and key latency is never on the critical path.  A sample's first
+// four tail rows go in flight at the top of its round and are consumed after its hot rows.
+// The hot loop is a jump table on the longest hot list of the warp's four samples (shorter
+// lists are padded with an all-zero row), the slot array is padded to whole rounds and all
+// addressing is by pointer increment, so the inner steps carry no predicate.
 //
-// Argmin: each lane reduces its 4 scores, compares with the sample's packed key and only on a
+// Argmin: each lane reduces its R scores, compares with the sample's packed key and only on a
 // (rare) improvement issues a 64-bit atomicMin on (ordered score bits, neuron).  The unsigned
 // minimum of that key is the lexicographic (score, lowest neuron) minimum, so the combine is
 // order-independent and ties break to the lowest neuron index (Section 3.1).
@@ -413,7 +415,9 @@ SomTableGeom som_table_geometry(const som_handle* h)
                     ? (int)h->opt_threads : def_threads;
     // 227 KB per block, minus the static shared memory (slot rings, norms) of the kernel
     int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
-    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (g.R == 8 ? 760 : 1536);
+    // Defaults keep dynamic + static shared memory under 196 KB: one step more and the SM's
+    // carve-out leaves 28 KB instead of 60 KB of L1, which costs 12 % at 128x128 (measured).
+    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (g.R == 8 ? 720 : 1376);
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
     g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * row_bytes;  // + the zero row

@@ -365,8 +365,7 @@ size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_m
 }
 
 int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                    char* ws, const SomPlanBuffers& b, int n_mask, int n_hot, uint32_t row_bytes,
-                    cudaStream_t st)
+                    char* ws, const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st)
 {
     uint32_t* feat_count = reinterpret_cast<uint32_t*>(ws + b.feat_count);
     int32_t* feat_slot = reinterpret_cast<int32_t*>(ws + b.feat_slot);

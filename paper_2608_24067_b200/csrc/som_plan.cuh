@@ -51,7 +51,7 @@ struct SomPlanBuffers {
 size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_max, SomPlanBuffers* b);
 
 int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
-                    const SomPlanBuffers& b, int n_mask, int n_hot, uint32_t row_bytes, cudaStream_t st);
+                    const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st);
 
 int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
                          cudaStream_t st);
