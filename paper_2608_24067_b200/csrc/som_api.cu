@@ -336,7 +336,8 @@ int som_set_option(som_handle* h, int key, int64_t value)
         return SOM_OK;
     }
     if (key == 2) {
-        if (value != 0 && value != 512 && value != 640 && value != 768 && value != 896 && value != 1024)
+        if (value != 0 && value != 512 && value != 640 && value != 768 &&
+            value != 896 && value != 1024)
             return SOM_ERR_INVALID_ARG;
         h->opt_threads = value;
         return SOM_OK;
