@@ -217,6 +217,8 @@ def run_ours(args, w: synth.Workload):
         h.set_option(2, args.threads)
     if args.lane_neurons:
         h.set_option(3, args.lane_neurons)
+    if args.parts:
+        h.set_option(4, args.parts)
     out_bmu = torch.empty(w.batch, dtype=torch.int32, device=dev)
     out_dist = torch.empty(w.batch, dtype=torch.float32, device=dev)
 
@@ -356,6 +358,7 @@ def main():
     ap.add_argument("--hot-rows", type=int, default=0, help="row-table kernel: hot rows in shared memory")
     ap.add_argument("--threads", type=int, default=0, help="row-table kernel: block size (512 or 1024)")
     ap.add_argument("--lane-neurons", type=int, default=0, help="row-table kernel: neurons per lane (4 or 8)")
+    ap.add_argument("--parts", type=int, default=0, help="row-table kernel: most sample parts per neuron range")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]

@@ -143,8 +143,8 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
     const SomTableGeom geom = som_table_geometry(h);
     bool use_table = h->opt_variant != 1 && (h->M % 4 == 0) && h->V <= 65536 && h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
-        int64_t parts = n_samples / 8192;
-        parts = parts < 1 ? 1 : (parts > 16 ? 16 : parts);
+        int64_t parts = n_samples / 31250;
+        parts = parts < 1 ? 1 : (parts > 32 ? 32 : parts);
         const int64_t units = ((h->M + geom.T - 1) / geom.T) * parts;
         if (units < 2 * (int64_t)h->sm_count) use_table = false;
     }
@@ -328,6 +328,11 @@ int som_set_option(som_handle* h, int key, int64_t value)
     if (key == 1) {
         if (value < 0 || value > 65000) return SOM_ERR_INVALID_ARG;
         h->opt_hot_rows = value;
+        return SOM_OK;
+    }
+    if (key == 4) {
+        if (value < 0 || value > 1024) return SOM_ERR_INVALID_ARG;
+        h->opt_parts = value;
         return SOM_OK;
     }
     if (key == 3) {

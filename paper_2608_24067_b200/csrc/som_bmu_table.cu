@@ -376,9 +376,15 @@ int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& 
     constexpr int T = 8 * R;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
     const int n_ranges = (int)((h->M + T - 1) / T);
-    int parts = (int)(n / 8192);
+    // Parts per neuron range: more parts mean fewer ranges live at once (their slabs must share
+    // L2 with the slot stream) but smaller units, each of which rebuilds the row table.  About
+    // 31,000 samples per unit and at most 32 parts measured best; 42,000 when a codebook row is
+    // longer than a 2 MB page, where every row of the table build is a TLB miss.
+    const int64_t unit_samples = (h->M * 4 >= (2 << 20)) ? 41666 : 31250;
+    int parts = h->opt_parts > 0 ? (int)h->opt_parts : (int)(n / unit_samples);
+    if (parts > 32 && h->opt_parts <= 0) parts = 32;
+    if ((int64_t)parts * 1024 > n) parts = (int)(n / 1024);
     if (parts < 1) parts = 1;
-    if (parts > 16) parts = 16;
     int64_t part_len = (n + parts - 1) / parts;
     part_len = (part_len + CHUNK - 1) / CHUNK * CHUNK;
     parts = (int)((n + part_len - 1) / part_len);

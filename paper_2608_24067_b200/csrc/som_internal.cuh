@@ -38,6 +38,7 @@ struct som_handle {
     int64_t opt_hot_rows;  // 0 = default number of hot rows in shared memory
     int64_t opt_threads;   // block size of the row-table kernel: 0 (default 512), 512 or 1024
     int64_t opt_r;         // neurons per lane of the row-table kernel: 0/4 or 8
+    int64_t opt_parts;     // row-table kernel: most sample parts per neuron range (0 = 16)
     int plan_attr_set;
     int32_t* host_pair;    // pinned, 2 ints: read-back of indptr[0], indptr[n]
 };
