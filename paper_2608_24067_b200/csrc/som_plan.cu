@@ -290,34 +290,46 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
     }
     const uint32_t pos = warp_agg_inc(bin_cursor, sort_bin(mask, nh, nt), active);
     if (!active) return;
-    uint32_t* slot = slots + (size_t)pos * SOM_SLOT_WORDS;
     const bool fits = nh <= SOM_SLOT_MAX_HOT && nt <= SOM_SLOT_MAX_TAIL;
     // (an overflow list holds at most 65535 hot and 65535 tail entries; the launcher checks V)
-    slot[0] = fits ? (mask | (nh << 16) | (nt << 24)) : (mask | (SOM_SLOT_NT_OVERFLOW << 24));
-    slot[1] = (uint32_t)s;
+    // The slot is assembled in registers and written with three 128-bit stores.  Unused hot
+    // codes point at the all-zero row that follows the table; unused tail codes are feature 0.
+    const uint32_t zz = (uint32_t)zero_row | ((uint32_t)zero_row << 16);
+    uint32_t w[SOM_SLOT_WORDS];
+    w[0] = fits ? (mask | (nh << 16) | (nt << 24)) : (mask | (SOM_SLOT_NT_OVERFLOW << 24));
+    w[1] = (uint32_t)s;
+#pragma unroll
+    for (int i = 2; i < 8; ++i) w[i] = zz;
+#pragma unroll
+    for (int i = 8; i < 12; ++i) w[i] = 0u;
     const int beg = indptr[s], end = indptr[s + 1];
     if (fits) {
-        uint16_t* hot = reinterpret_cast<uint16_t*>(slot + 2);
-        uint16_t* tail = reinterpret_cast<uint16_t*>(slot + 8);
+        uint32_t ih = 0, it = 0;
         for (int j = beg; j < end; ++j) {
             const int v = indices[j];
             const int fs = feat_slot[v];
-            if (fs < 0) *tail++ = (uint16_t)v;
-            else if (fs >= n_mask) *hot++ = (uint16_t)fs;
+            if (fs < 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if ((it >> 1) == (uint32_t)i)
+                        w[8 + i] = (it & 1u) ? (w[8 + i] | ((uint32_t)v << 16)) : (uint32_t)v;
+                ++it;
+            } else if (fs >= n_mask) {
+#pragma unroll
+                for (int i = 0; i < 6; ++i)
+                    if ((ih >> 1) == (uint32_t)i)
+                        w[2 + i] = (ih & 1u) ? ((w[2 + i] & 0xffffu) | ((uint32_t)fs << 16))
+                                             : ((w[2 + i] & 0xffff0000u) | (uint32_t)fs);
+                ++ih;
+            }
         }
-        // unused hot codes point at the all-zero row that follows the table
-        for (uint16_t* e = reinterpret_cast<uint16_t*>(slot + 8); hot < e; ++hot) *hot = (uint16_t)zero_row;
     } else {
         const uint32_t nt_pad = (nt + 3u) & ~3u, nh_pad = (nh + 3u) & ~3u;
         const uint32_t off = atomicAdd(overflow_cursor, nt_pad + nh_pad);
-        // hot-code words all point at the zero row; the list offset and the true counts
-        // (which may not fit the header fields) go where the tail codes would be
-        const uint32_t zz = (uint32_t)zero_row | ((uint32_t)zero_row << 16);
-        for (int w = 2; w < 8; ++w) slot[w] = zz;
-        slot[8] = 0u;  // inline tail codes of an overflow sample: feature 0, a valid row
-        slot[9] = 0u;
-        slot[10] = off;
-        slot[11] = nh | (nt << 16);
+        // the list offset and the true counts (which may not fit the header fields) go where
+        // the last tail codes would be; the inline tail codes stay feature 0, a valid row
+        w[10] = off;
+        w[11] = nh | (nt << 16);
         uint32_t* tail = overflow + off;
         uint32_t* hot = tail + nt_pad;
         for (int j = beg; j < end; ++j) {
@@ -327,6 +339,10 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
             else if (fs >= n_mask) *hot++ = (uint32_t)fs;
         }
     }
+    uint4* slot = reinterpret_cast<uint4*>(slots + (size_t)pos * SOM_SLOT_WORDS);
+    slot[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    slot[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    slot[2] = make_uint4(w[8], w[9], w[10], w[11]);
 }
 
 // The slot array is padded to whole rounds with copies of the last slot.
