@@ -359,9 +359,15 @@ def main():
     ap.add_argument("--threads", type=int, default=0, help="row-table kernel: block size (512 or 1024)")
     ap.add_argument("--lane-neurons", type=int, default=0, help="row-table kernel: neurons per lane (4 or 8)")
     ap.add_argument("--parts", type=int, default=0, help="row-table kernel: most sample parts per neuron range")
+    ap.add_argument("--features", default="zipf", choices=["zipf", "uniform"],
+                    help="feature popularity of the samples: the workload's Zipf law, or the stress variant "
+                         "with features uniform over V (no sharing between samples)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]
+    if args.features == "uniform":
+        import dataclasses
+        w = dataclasses.replace(w, name=w.name + "-uniform", zipf_s=0.0)
     if args.impl == "reference":
         run_reference(args, w)
     else:

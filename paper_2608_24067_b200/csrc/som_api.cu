@@ -143,8 +143,7 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
     const SomTableGeom geom = som_table_geometry(h);
     bool use_table = h->opt_variant != 1 && (h->M % 4 == 0) && h->V <= 65536 && h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
-        int64_t parts = n_samples / 31250;
-        parts = parts < 1 ? 1 : (parts > 32 ? 32 : parts);
+        const int64_t parts = som_table_default_parts(n_samples);
         const int64_t units = ((h->M + geom.T - 1) / geom.T) * parts;
         if (units < 2 * (int64_t)h->sm_count) use_table = false;
     }

@@ -2,7 +2,7 @@
 //
 // Decomposition (Section 3.3 of the paper, re-planned for B200): a work unit is a neuron
 // range of T = 8*R neurons (R = 8 or 4 per lane) times a contiguous part of the mask-sorted
-// sample list.  One persistent block per SM walks units in range-major order, so that at any
+// sample list.  One persistent block per SM claims units in range-major order, so that at any
 // time only a few neuron ranges are live and their codebook slabs W[:, i0..i0+T) stay
 // L2-resident while HBM sees the codebook about once per batch.  Inside a unit the warps pull
 // chunks of samples from a shared counter, which keeps them busy whatever the mix of row
@@ -140,7 +140,8 @@ __global__ void __launch_bounds__(THREADS, 1)
 k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
             const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
-            u64* __restrict__ keys, int parts, int64_t part_len, int n_units)
+            u64* __restrict__ keys, int parts, int64_t part_len, int n_units,
+            int* __restrict__ unit_counter)
 {
     constexpr int H = R / 4;
     constexpr int T = 8 * R;
@@ -148,6 +149,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
     constexpr int WARPS = THREADS / 32;
     extern __shared__ __align__(16) unsigned char tab[];
     __shared__ int next_chunk;
+    __shared__ int unit_sh;
     __shared__ __align__(16) float hn_sh[T];  // ||w||^2/2 of the range's neurons (+inf past M)
     // Warp-private ring of two stages; a stage holds the four slots (192 B) and four keys (32 B)
     // of one round.  The bytes of round r+2 are in flight in registers, round r+1 is being
@@ -170,12 +172,22 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
     int cur_range = -1;
     const float* w_q = W;
     uint32_t i_first = 0;
-    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+    for (;;) {
+        // Units are claimed from a global counter in range-major order, so the blocks always
+        // work on neighbouring units: the window of live neuron ranges (whose slabs must share
+        // L2 with the slot stream) stays a few ranges wide however long the launch runs, and no
+        // block is left with a queue of its own at the end.
+        __syncthreads();  // every warp has left the previous unit
+        if (threadIdx.x == 0) {
+            unit_sh = atomicAdd(unit_counter, 1);
+            next_chunk = 0;
+        }
+        __syncthreads();
+        const int unit = unit_sh;
+        if (unit >= n_units) break;
         const int range = unit / parts;
         const int part = unit - range * parts;
         const int64_t i0 = (int64_t)range * T;
-        __syncthreads();  // every warp has left the previous unit
-        if (threadIdx.x == 0) next_chunk = 0;
         if (range != cur_range) {
             for (int row0 = warp * 4; row0 < n_rows; row0 += WARPS * 4) {
                 float v[4][H];
@@ -376,13 +388,7 @@ int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& 
     constexpr int T = 8 * R;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
     const int n_ranges = (int)((h->M + T - 1) / T);
-    // Parts per neuron range: more parts mean fewer ranges live at once (their slabs must share
-    // L2 with the slot stream) but smaller units, each of which rebuilds the row table.  About
-    // 31,000 samples per unit and at most 32 parts measured best; 42,000 when a codebook row is
-    // longer than a 2 MB page, where every row of the table build is a TLB miss.
-    const int64_t unit_samples = (h->M * 4 >= (2 << 20)) ? 41666 : 31250;
-    int parts = h->opt_parts > 0 ? (int)h->opt_parts : (int)(n / unit_samples);
-    if (parts > 32 && h->opt_parts <= 0) parts = 32;
+    int parts = h->opt_parts > 0 ? (int)h->opt_parts : som_table_default_parts(n);
     if ((int64_t)parts * 1024 > n) parts = (int)(n / 1024);
     if (parts < 1) parts = 1;
     int64_t part_len = (n + parts - 1) / parts;
@@ -399,7 +405,8 @@ int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& 
                                       SOM_PLAN_MASK_FEATURES + n_hot,
                                       reinterpret_cast<const uint4*>(ws + b.slots),
                                       reinterpret_cast<const uint32_t*>(ws + b.overflow), n,
-                                      reinterpret_cast<u64*>(ws + b.keys), parts, part_len, n_units);
+                                      reinterpret_cast<u64*>(ws + b.keys), parts, part_len, n_units,
+                                      reinterpret_cast<int*>(ws + b.n_slots) + 3);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -38,7 +38,7 @@ struct SomPlanBuffers {
     size_t feat_count;  // u32 [V]
     size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
     size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
-    size_t n_slots;     // i32 [4]      mask slots used, hot slots used, overflow cursor
+    size_t n_slots;     // i32 [4]      mask slots used, hot slots used, overflow cursor, search unit counter
     size_t pk;          // u32 [n]      mask | n_hot << 16, by sample
     size_t ntail;       // u32 [n]
     size_t bin_count;   // u32 [bins]
@@ -47,6 +47,16 @@ struct SomPlanBuffers {
     size_t slots;       // 48 B [n + 16]
     size_t overflow;    // u32 [nnz + 6n]
 };
+
+// Sample parts per neuron range of the row-table kernel.  More parts mean fewer ranges live at
+// once (their slabs must share L2 with the slot stream) but smaller units, each of which
+// rebuilds the row table; with units claimed in order the optimum is flat: about 20,000
+// samples per unit, at most 32 parts (measured on 250k to 4M-sample batches).
+static inline int som_table_default_parts(int64_t n)
+{
+    const int64_t parts = n / 20000;
+    return parts < 1 ? 1 : (parts > 32 ? 32 : (int)parts);
+}
 
 size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_max, SomPlanBuffers* b);
 
