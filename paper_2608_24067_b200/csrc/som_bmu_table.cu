@@ -100,6 +100,19 @@ __device__ __forceinline__ void sub_acc(Acc<H>& a, const Acc<H>& w)
     for (int x = 0; x < H; ++x) sub_pair(a.g[x], w.g[x]);
 }
 
+// out = a - w (three-operand form: no copy of `a` is needed when it must survive)
+template <int H>
+__device__ __forceinline__ Acc<H> sub_acc3(const Acc<H>& a, const Acc<H>& w)
+{
+    Acc<H> r;
+#pragma unroll
+    for (int x = 0; x < H; ++x) {
+        asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r.g[x].lo) : "l"(a.g[x].lo), "l"(w.g[x].lo));
+        asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r.g[x].hi) : "l"(a.g[x].hi), "l"(w.g[x].hi));
+    }
+    return r;
+}
+
 // a lane's slice of a shared-memory row: 16 bytes per group, groups 128 bytes apart
 template <int H>
 __device__ __forceinline__ Acc<H> lds_acc(const unsigned char* p)
@@ -291,11 +304,12 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                     }
                     curmask = mask;
                 }
-                Acc<H> acc = base;
 
-                // ---- hot rows: exactly max(nh over the warp) steps; shorter lists are padded
-                //      with the zero row, so a step carries no predicate -------------------------
+                // ---- hot rows: exactly max(nh over the warp, 1) steps; shorter lists are padded
+                //      with the zero row, so a step carries no predicate.  The first step also
+                //      moves the running score out of `base` (which the next sample may reuse).
                 const uint32_t nh_max = __reduce_max_sync(0xffffffffu, nh);
+                Acc<H> acc = sub_acc3<H>(base, lds_acc<H>(tab_q + lo16(s0.z) * ROWB));
                 switch (nh_max) {
                     case 12: SOM_HOT(hi16(s1.w));
                     case 11: SOM_HOT(lo16(s1.w));
@@ -308,7 +322,6 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                     case 4: SOM_HOT(hi16(s0.w));
                     case 3: SOM_HOT(lo16(s0.w));
                     case 2: SOM_HOT(hi16(s0.z));
-                    case 1: SOM_HOT(lo16(s0.z));
                     default: break;
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7 / overflow fields
