@@ -225,7 +225,10 @@ def run_ours(args, w: synth.Workload):
     def step(i):
         b = batches[i % n_batches]
         h.norms()
-        h.bmu(b.indptr, b.indices, out_bmu, out_dist)
+        if args.top2:
+            h.bmu2(b.indptr, b.indices)
+        else:
+            h.bmu(b.indptr, b.indices, out_bmu, out_dist)
 
     def barrier():
         if dist is not None:
@@ -330,7 +333,8 @@ def run_ours(args, w: synth.Workload):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": nnz_mean,
-                   "step": "som_norms + som_bmu on one batch", "replicas": ws,
+                   "step": "som_norms + %s on one batch" % ("som_bmu2" if args.top2 else "som_bmu"),
+                   "replicas": ws,
                    "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
                        w.V * w.M * 4 / 1e6, batches[0].nnz * 4 / 1e6) if w.V * w.M * 4 > 126e6 else
                    "inputs smaller than L2: steps rotate over %d distinct batches, no flush" % n_batches},
@@ -362,6 +366,8 @@ def main():
     ap.add_argument("--features", default="zipf", choices=["zipf", "uniform"],
                     help="feature popularity of the samples: the workload's Zipf law, or the stress variant "
                          "with features uniform over V (no sharing between samples)")
+    ap.add_argument("--top2", action="store_true",
+                    help="time som_bmu2 (best and second-best unit) instead of som_bmu")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]

@@ -91,6 +91,22 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
             int32_t* d_bmu, float* d_min_dist, void* stream);
 
 /*
+ * som_bmu2 - som_bmu that also returns the second-best unit, found in the same sweep (the
+ * paper's search kernel keeps the two best units of every sample: Section 3.3; Algorithm 2,
+ * step 7; the second one feeds the topographic error, Section 3.5).
+ *   d_bmu, d_min_dist   as in som_bmu.
+ *   d_bmu2     DEVICE pointer, int32 [n_samples]  out: the neuron that comes second in the order
+ *              (fp32 score, neuron index), i.e. the nearest neuron other than d_bmu, lowest
+ *              index among exact fp32 ties; -1 when the map has a single neuron.
+ *   d_dist2    DEVICE pointer, fp32 [n_samples]   out: its full squared distance, recomputed in
+ *              fp64 and rounded once like d_min_dist; +inf when d_bmu2 is -1.
+ * Same preconditions, asynchrony and determinism as som_bmu; d_bmu/d_min_dist are bit-identical
+ * to som_bmu's for the same inputs.
+ */
+int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+             int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream);
+
+/*
  * som_bmu_host - the same search with HOST buffers: copies the CSR batch to device staging
  * memory owned by the handle, runs som_bmu, copies both outputs back, all enqueued on
  * `stream`, then synchronises that stream before returning.  h_* pointers are host memory

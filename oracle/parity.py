@@ -14,6 +14,13 @@ flips a few assignments between near-tied neurons, and that fp64 removes them):
   neuron* within ``DIST_REL`` (1e-5) relative (``DIST_ABS`` 1e-6 absolute floor for
   distances that are exactly or nearly zero);
 * the hit-count histogram built from unambiguous samples must be identical.
+
+Second-best unit (the search of Algorithm 2 keeps the two best units): the reported second
+unit g2 must differ from the reported best unit, and its fp64 distance may exceed the oracle's
+second-best distance d2 by at most the same relative band (it may be lower: when the two best
+are near-tied and the implementation ranks them the other way round, g2 is the oracle's best).
+Where the oracle's second and third are further apart than the band this forces g2 == b2, so no
+third-best distance is needed.  Its reported distance follows the same ``DIST_REL`` rule.
 """
 from __future__ import annotations
 
@@ -70,3 +77,40 @@ def check(g_bmu, g_dist, top2, d_at_g, M: int) -> ParityReport:
     ho = np.bincount(b1[unamb], minlength=M)
     return ParityReport(n, int(unamb.sum()), int((~unamb).sum()), idx_bad, band_bad, rel, viol,
                         bool(np.array_equal(hg, ho)))
+
+
+@dataclass
+class SecondReport:
+    n: int
+    differs_from_oracle: int   # g2 != b2 (allowed only inside the band)
+    same_as_best: int          # g2 == g1: never allowed
+    outside_band: int
+    dist_violations: int
+    max_dist_rel_err: float
+
+    @property
+    def ok(self) -> bool:
+        return self.same_as_best == 0 and self.outside_band == 0 and self.dist_violations == 0
+
+    def __str__(self):
+        return ("n=%d second_differs=%d same_as_best=%d outside_band=%d dist_violations=%d "
+                "max_dist_rel_err=%.3g" % (self.n, self.differs_from_oracle, self.same_as_best,
+                                           self.outside_band, self.dist_violations, self.max_dist_rel_err))
+
+
+def check_second(g_bmu, g_bmu2, g_dist2, top2, d_at_g2, M: int) -> SecondReport:
+    """g_bmu/g_bmu2/g_dist2: implementation outputs; top2: oracle Top2; d_at_g2: oracle fp64
+    distance of each sample to g_bmu2.  Requires M >= 2 (with one neuron there is no second)."""
+    g1 = np.asarray(g_bmu).astype(np.int64)
+    g2 = np.asarray(g_bmu2).astype(np.int64)
+    gd = np.asarray(g_dist2).astype(np.float64)
+    d2 = top2.d2
+    in_range = (g2 >= 0) & (g2 < M)
+    scale = np.where(np.abs(d2) > 1e-30, np.abs(d2), 1.0)
+    same = int(np.sum(g2 == g1))
+    band_bad = int(np.sum(~in_range | ((d_at_g2 - d2) > GAP_REL * scale)))
+    tol = DIST_REL * np.abs(d_at_g2) + DIST_ABS
+    err = np.abs(gd - d_at_g2)
+    viol = int(np.sum(~(err <= tol)))
+    rel = float(np.max(err / np.maximum(np.abs(d_at_g2), 1e-30), initial=0.0, where=np.abs(d_at_g2) > 1e-3))
+    return SecondReport(g1.size, int(np.sum(g2 != top2.b2)), same, band_bad, viol, rel)

@@ -123,12 +123,14 @@ int som_norms(som_handle* h, void* stream)
     return SOM_OK;
 }
 
-int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
-            int32_t* d_bmu, float* d_min_dist, void* stream)
+// The search behind som_bmu (d_bmu2 == nullptr) and som_bmu2 (both second-best outputs given).
+static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+                    int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream)
 {
     if (!h || n_samples < 0) return SOM_ERR_INVALID_ARG;
     if (n_samples == 0) return SOM_OK;
     if (!d_indptr || !d_bmu || !d_min_dist) return SOM_ERR_INVALID_ARG;
+    const bool top2 = d_bmu2 != nullptr;
     if (n_samples >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
     if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
     DeviceGuard g(h->device);
@@ -164,14 +166,17 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
 
     if (!use_table) {
         const size_t key_bytes = som_align_up((size_t)n_samples * sizeof(unsigned long long), 256);
-        if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, key_bytes))) return rc;
+        if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, 2 * key_bytes))) return rc;
         unsigned long long* keys = reinterpret_cast<unsigned long long*>(h->ws);
+        unsigned long long* keys2 = top2 ? keys + key_bytes / sizeof(unsigned long long) : nullptr;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
-        SOM_CK(h, cudaMemsetAsync(keys, 0xFF, (size_t)n_samples * sizeof(unsigned long long), st));
+        SOM_CK(h, cudaMemsetAsync(keys, 0xFF, top2 ? 2 * key_bytes : key_bytes, st));
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, st))) return rc;
+        if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, st))) return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, st)))
+            return rc;
+        if (top2 && (rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys2, d_bmu2, d_dist2, st)))
             return rc;
     } else {
         SomPlanBuffers pb;
@@ -181,18 +186,37 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
         char* ws = reinterpret_cast<char*>(h->ws);
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
         SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
+        if (top2)
+            SOM_CK(h, cudaMemsetAsync(ws + pb.keys2, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
         if ((rc = som_launch_plan(h, d_indptr, d_indices, n_samples, ws, pb, SOM_PLAN_MASK_FEATURES,
                                   geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_table(h, n_samples, ws, pb, geom.n_hot, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, n_samples, ws, pb, geom.n_hot, top2, st))) return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-        if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, d_bmu, d_min_dist, st)))
+        if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, false, d_bmu,
+                                             d_min_dist, st)))
+            return rc;
+        if (top2 && (rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, true, d_bmu2,
+                                                     d_dist2, st)))
             return rc;
     }
     if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
     if (h->timing) h->ev_bmu_calls += 1;
     return SOM_OK;
+}
+
+int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+            int32_t* d_bmu, float* d_min_dist, void* stream)
+{
+    return bmu_impl(h, d_indptr, d_indices, n_samples, d_bmu, d_min_dist, nullptr, nullptr, stream);
+}
+
+int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+             int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream)
+{
+    if (n_samples > 0 && (!d_bmu2 || !d_dist2)) return SOM_ERR_INVALID_ARG;
+    return bmu_impl(h, d_indptr, d_indices, n_samples, d_bmu, d_min_dist, d_bmu2, d_dist2, stream);
 }
 
 int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,

@@ -18,11 +18,19 @@ constexpr int DIRECT_THREADS = 256;
 constexpr int DIRECT_WARPS = DIRECT_THREADS / 32;
 constexpr int DIRECT_SAMPLES_PER_WARP = 16;
 
-template <int VEC>
+// (score, index) order: smaller score first, then lower index
+__device__ __forceinline__ bool before(float a, uint32_t ai, float b, uint32_t bi)
+{
+    return a < b || (a == b && ai < bi);
+}
+
+// TOP2 also keeps the second-best unit in keys2 (Algorithm 2 keeps the two best units).
+template <int VEC, bool TOP2>
 __global__ void __launch_bounds__(DIRECT_THREADS)
 k_bmu_direct(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
              const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
-             unsigned long long* __restrict__ keys, int64_t neuron_off)
+             unsigned long long* __restrict__ keys, unsigned long long* __restrict__ keys2,
+             int64_t neuron_off)
 {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -63,16 +71,53 @@ k_bmu_direct(const float* __restrict__ W, const float* __restrict__ hnorm, int64
         }
         float best = acc[0];
         uint32_t bi = (uint32_t)i0;
+        float second = inf;            // TOP2: the lane's, then the warp's, second best
+        uint32_t si = 0xffffffffu;
 #pragma unroll
-        for (int k = 1; k < VEC; ++k)
-            if (acc[k] < best) { best = acc[k]; bi = (uint32_t)(i0 + k); }
+        for (int k = 1; k < VEC; ++k) {
+            const uint32_t ik = (uint32_t)(i0 + k);
+            if (acc[k] < best) {
+                if (TOP2) { second = best; si = bi; }
+                best = acc[k];
+                bi = ik;
+            } else if (TOP2 && before(acc[k], ik, second, si)) {
+                second = acc[k];
+                si = ik;
+            }
+        }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             const float ob = __shfl_down_sync(0xffffffffu, best, off);
             const uint32_t oi = __shfl_down_sync(0xffffffffu, bi, off);
-            if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+            if (TOP2) {
+                // merge two sorted pairs into the best two of the four
+                const float os = __shfl_down_sync(0xffffffffu, second, off);
+                const uint32_t osi = __shfl_down_sync(0xffffffffu, si, off);
+                if (before(ob, oi, best, bi)) {
+                    if (before(best, bi, os, osi)) { second = best; si = bi; }
+                    else { second = os; si = osi; }
+                    best = ob;
+                    bi = oi;
+                } else if (before(ob, oi, second, si)) {
+                    second = ob;
+                    si = oi;
+                }
+            } else {
+                if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+            }
         }
-        if (lane == 0) atomicMin(&keys[s], som_pack_key(best, bi));
+        if (lane == 0) {
+            const unsigned long long c1 = som_pack_key(best, bi);
+            if (!TOP2) {
+                atomicMin(&keys[s], c1);
+            } else {
+                // keys ends as the minimum of all candidates; each other candidate reaches
+                // keys2 exactly once (directly, or when a smaller one displaces it from keys)
+                const unsigned long long old = atomicMin(&keys[s], c1);
+                atomicMin(&keys2[s], old > c1 ? old : c1);
+                if (si != 0xffffffffu) atomicMin(&keys2[s], som_pack_key(second, si));
+            }
+        }
     }
 }
 
@@ -86,6 +131,11 @@ __global__ void k_finalize(const float* __restrict__ W, const double* __restrict
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n) return;
     const uint32_t idx = (uint32_t)(keys[s] & 0xffffffffull);
+    if (idx >= M) {  // only a second-best key can be empty: fewer than two neurons
+        bmu[s] = -1;
+        dist[s] = __int_as_float(0x7f800000);
+        return;
+    }
     const int beg = indptr[s];
     const int end = indptr[s + 1];
     double dot = 0.0;
@@ -116,7 +166,7 @@ __global__ void k_validate(const int32_t* __restrict__ indptr, const int32_t* __
 }  // namespace
 
 int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                          unsigned long long* keys, cudaStream_t st)
+                          unsigned long long* keys, unsigned long long* keys2, cudaStream_t st)
 {
     const int vec = (h->M % 4 == 0) ? 4 : 1;
     const int64_t per_block = (int64_t)DIRECT_WARPS * DIRECT_SAMPLES_PER_WARP;
@@ -129,12 +179,18 @@ int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* i
         const int64_t ny = (gy - y0 < max_gy) ? gy - y0 : max_gy;
         dim3 grid((unsigned)gx, (unsigned)ny);
         const int64_t neuron_off = y0 * neurons_per_block;
-        if (vec == 4)
-            k_bmu_direct<4><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
-                                                             keys, neuron_off);
+        if (vec == 4 && !keys2)
+            k_bmu_direct<4, false><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
+                                                                    keys, keys2, neuron_off);
+        else if (vec == 4)
+            k_bmu_direct<4, true><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
+                                                                   keys, keys2, neuron_off);
+        else if (!keys2)
+            k_bmu_direct<1, false><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
+                                                                    keys, keys2, neuron_off);
         else
-            k_bmu_direct<1><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
-                                                             keys, neuron_off);
+            k_bmu_direct<1, true><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
+                                                                   keys, keys2, neuron_off);
         SOM_CK(h, cudaGetLastError());
         h->launches += 1;
     }

@@ -148,12 +148,14 @@ __device__ __forceinline__ const float* row_ptr(const float* base, uint32_t code
 #define SOM_TAIL(code) ldg_acc<H>(row_ptr(w_q, (code), stride_b))
 
 // R = neurons per lane (4 or 8); a team of 8 lanes covers T = 8*R neurons of one sample.
-template <int R, int THREADS>
+// TOP2 also keeps the second-best unit of every sample in keys2 (Algorithm 2 keeps the two
+// best units); the candidate filter then tests against the second-best score.
+template <int R, int THREADS, bool TOP2>
 __global__ void __launch_bounds__(THREADS, 1)
 k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
             const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
-            u64* __restrict__ keys, int parts, int64_t part_len, int n_units,
+            u64* __restrict__ keys, u64* __restrict__ keys2, int parts, int64_t part_len, int n_units,
             int* __restrict__ unit_counter)
 {
     constexpr int H = R / 4;
@@ -249,8 +251,11 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
             // Ring feed: lanes 0..11 carry the twelve 16-byte pieces of a round's four slots,
             // lanes 12..13 the two 16-byte pieces of its four keys.
             unsigned char* ring = ring_sh + warp * 2 * RING_STAGE;
+            // the keys a round tests its candidates against: the best so far, or with TOP2 the
+            // second best so far (a stale, larger value only lets more candidates through)
+            const u64* filter_keys = TOP2 ? keys2 : keys;
             const uint4* feed = (lane < 12) ? slots + w0 * SLOT_Q + lane
-                                            : reinterpret_cast<const uint4*>(keys + w0) + (lane - 12);
+                                            : reinterpret_cast<const uint4*>(filter_keys + w0) + (lane - 12);
             const int feed_step = (lane < 12) ? 4 * SLOT_Q : 2;  // uint4 per round
             const bool feeder = lane < 14;
             unsigned char* my_store = ring + (lane < 12 ? lane * 16 : 192 + (lane - 12) * 16);
@@ -369,7 +374,27 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                     for (int j = R - 2; j >= 0; --j)
                         if (a[j] == mn) rr = j;  // lowest neuron among the lane's minima
                     const uint32_t neuron = i_first + (uint32_t)((rr >> 2) * 32 + (rr & 3));
-                    atomicMin(pk - 4, som_pack_key(mn, neuron));
+                    const u64 c1 = som_pack_key(mn, neuron);
+                    if (!TOP2) {
+                        atomicMin(pk - 4, c1);
+                    } else {
+                        // Two-key combine.  keys ends as the minimum of all candidates; every
+                        // other candidate reaches keys2 exactly once, either directly (it did
+                        // not beat the best of its time) or when a later, smaller candidate
+                        // displaces it from keys, so keys2 ends as the second smallest.  Both
+                        // are minima of fixed sets: order-independent, ties to the lower index.
+                        u64* k1 = pk - 4;
+                        u64* k2 = keys2 + (k1 - keys);
+                        const u64 old = atomicMin(k1, c1);
+                        atomicMin(k2, old > c1 ? old : c1);
+                        float m2 = inf;
+                        int r2 = 0;
+#pragma unroll
+                        for (int j = R - 1; j >= 0; --j)
+                            if (j != rr && a[j] <= m2) { m2 = a[j]; r2 = j; }
+                        if (!(m2 > cs))
+                            atomicMin(k2, som_pack_key(m2, i_first + (uint32_t)((r2 >> 2) * 32 + (r2 & 3))));
+                    }
                 }
             }
         }
@@ -386,6 +411,11 @@ __global__ void k_finalize_sorted(const float* __restrict__ W, const double* __r
     if (k >= n) return;
     const uint32_t s = slots[k * SLOT_Q].y;
     const uint32_t idx = (uint32_t)(keys[k] & 0xffffffffull);
+    if (idx >= M) {  // only a second-best key can be empty: fewer than two neurons
+        bmu[s] = -1;
+        dist[s] = __int_as_float(0x7f800000);
+        return;
+    }
     const int beg = indptr[s];
     const int end = indptr[s + 1];
     double dot = 0.0;
@@ -394,7 +424,7 @@ __global__ void k_finalize_sorted(const float* __restrict__ W, const double* __r
     dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
 }
 
-template <int R, int THREADS>
+template <int R, int THREADS, bool TOP2>
 int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& b, int n_hot, size_t smem,
                  cudaStream_t st)
 {
@@ -411,14 +441,15 @@ int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& 
     if (n_units64 > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
     const int n_units = (int)n_units64;
     const int grid = n_units < h->sm_count ? n_units : h->sm_count;
-    auto kern = k_bmu_table<R, THREADS>;
+    auto kern = k_bmu_table<R, THREADS, TOP2>;
     SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<grid, THREADS, smem, st>>>(h->W, h->hnorm, h->M,
                                       reinterpret_cast<const int32_t*>(ws + b.slot_feat),
                                       SOM_PLAN_MASK_FEATURES + n_hot,
                                       reinterpret_cast<const uint4*>(ws + b.slots),
                                       reinterpret_cast<const uint32_t*>(ws + b.overflow), n,
-                                      reinterpret_cast<u64*>(ws + b.keys), parts, part_len, n_units,
+                                      reinterpret_cast<u64*>(ws + b.keys),
+                                      TOP2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr, parts, part_len, n_units,
                                       reinterpret_cast<int*>(ws + b.n_slots) + 3);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
@@ -451,32 +482,40 @@ SomTableGeom som_table_geometry(const som_handle* h)
     return g;
 }
 
-int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
-                         cudaStream_t st)
+template <bool TOP2>
+static int launch_table_any(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
+                            cudaStream_t st)
 {
     const SomTableGeom g = som_table_geometry(h);
     if (g.R == 8) {
-        if (g.threads == 1024) return launch_table<8, 1024>(h, n, ws, b, n_hot, g.smem, st);
-        if (g.threads == 896) return launch_table<8, 896>(h, n, ws, b, n_hot, g.smem, st);
-        if (g.threads == 768) return launch_table<8, 768>(h, n, ws, b, n_hot, g.smem, st);
-        if (g.threads == 640) return launch_table<8, 640>(h, n, ws, b, n_hot, g.smem, st);
-        return launch_table<8, 512>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 1024) return launch_table<8, 1024, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 896) return launch_table<8, 896, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 768) return launch_table<8, 768, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 640) return launch_table<8, 640, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+        return launch_table<8, 512, TOP2>(h, n, ws, b, n_hot, g.smem, st);
     }
-    if (g.threads == 1024) return launch_table<4, 1024>(h, n, ws, b, n_hot, g.smem, st);
-    if (g.threads == 896) return launch_table<4, 896>(h, n, ws, b, n_hot, g.smem, st);
-    if (g.threads == 768) return launch_table<4, 768>(h, n, ws, b, n_hot, g.smem, st);
-    if (g.threads == 640) return launch_table<4, 640>(h, n, ws, b, n_hot, g.smem, st);
-    return launch_table<4, 512>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 1024) return launch_table<4, 1024, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 896) return launch_table<4, 896, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 768) return launch_table<4, 768, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 640) return launch_table<4, 640, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+    return launch_table<4, 512, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+}
+
+int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
+                         bool top2, cudaStream_t st)
+{
+    return top2 ? launch_table_any<true>(h, n, ws, b, n_hot, st)
+                : launch_table_any<false>(h, n, ws, b, n_hot, st);
 }
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                               char* ws, const SomPlanBuffers& b, int32_t* bmu, float* dist,
+                               char* ws, const SomPlanBuffers& b, bool second, int32_t* bmu, float* dist,
                                cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
     k_finalize_sorted<<<(unsigned)blocks, 256, 0, st>>>(
         h->W, h->norm64, h->M, indptr, indices, n, reinterpret_cast<const uint4*>(ws + b.slots),
-        reinterpret_cast<const u64*>(ws + b.keys), bmu, dist);
+        reinterpret_cast<const u64*>(ws + (second ? b.keys2 : b.keys)), bmu, dist);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -74,7 +74,7 @@ __device__ __forceinline__ unsigned long long som_pack_key(float score, uint32_t
 // kernels' host launchers (each returns a som_status)
 int som_launch_norms(som_handle* h, cudaStream_t st);
 int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                          unsigned long long* keys, cudaStream_t st);
+                          unsigned long long* keys, unsigned long long* keys2, cudaStream_t st);
 int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                         const unsigned long long* keys, int32_t* bmu, float* dist, cudaStream_t st);
 int som_launch_validate(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,

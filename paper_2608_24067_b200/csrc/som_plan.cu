@@ -366,6 +366,7 @@ size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_m
         return o;
     };
     b->keys = take((size_t)(n + 16) * 8);
+    b->keys2 = take((size_t)(n + 16) * 8);
     b->feat_count = take((size_t)V * 4);
     b->feat_slot = take((size_t)V * 4);
     b->slot_feat = take((size_t)n_slots_max * 4);

@@ -35,6 +35,7 @@ struct som_handle;
 // byte offsets into the workspace
 struct SomPlanBuffers {
     size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
+    size_t keys2;       // u64 [n]      the same for the second-best unit (two-best search only)
     size_t feat_count;  // u32 [V]
     size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
     size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
@@ -64,10 +65,10 @@ int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices
                     const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st);
 
 int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
-                         cudaStream_t st);
+                         bool top2, cudaStream_t st);
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                               char* ws, const SomPlanBuffers& b, int32_t* bmu, float* dist,
+                               char* ws, const SomPlanBuffers& b, bool second, int32_t* bmu, float* dist,
                                cudaStream_t st);
 
 // Geometry of the row-table kernel for this handle: neurons per range, hot rows that fit.

@@ -24,7 +24,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
-    "som_launch_count", "som_set_option", "som_norms_noalloc",
+    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -57,6 +57,8 @@ def load_library():
     lib.som_norms.argtypes = [P, P]
     lib.som_bmu.argtypes = [P, P, P, I64, P, P, P]
     lib.som_bmu_host.argtypes = [P, P, P, I64, P, P, P]
+    lib.som_bmu2.argtypes = [P, P, P, I64, P, P, P, P, P]
+    lib.som_bmu2.restype = INT
     lib.som_validate_csr.argtypes = [P, P, P, I64, P]
     lib.som_get_norms.argtypes = [P, P, P]
     lib.som_destroy.argtypes = [P]
@@ -151,6 +153,19 @@ class Som:
                                _dev_ptr(out_dist, torch.float32, "out_dist"), _stream_ptr(stream))
         self._check(rc, "som_bmu")
         return out_bmu, out_dist
+
+    def bmu2(self, indptr: torch.Tensor, indices: torch.Tensor, stream=None):
+        """som_bmu2: best and second-best unit per sample; returns (bmu, dist, bmu2, dist2)."""
+        n = indptr.numel() - 1
+        dev = self.codebook.device
+        out = [torch.empty(n, dtype=dt, device=dev)
+               for dt in (torch.int32, torch.float32, torch.int32, torch.float32)]
+        rc = self._lib.som_bmu2(self._h, _dev_ptr(indptr, torch.int32, "indptr"),
+                                _dev_ptr(indices, torch.int32, "indices"), n,
+                                out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), out[3].data_ptr(),
+                                _stream_ptr(stream))
+        self._check(rc, "som_bmu2")
+        return tuple(out)
 
     def bmu_host(self, indptr: torch.Tensor, indices: torch.Tensor, out_bmu: torch.Tensor,
                  out_dist: torch.Tensor, stream=None):

@@ -212,3 +212,36 @@ def test_argmin_invariant_to_common_shift_of_sample():
         score = nn - 2.0 * Wd[r].sum(axis=0)
         assert score.argmin() == D[s].argmin()
         np.testing.assert_allclose(score + len(r), D[s], rtol=1e-12, atol=1e-12)
+
+
+def test_second_best_parity_rule_on_brute_force():
+    """The band rule for the second-best unit, against an explicit ranking of all fp64 distances:
+    the true second passes, the third-best fails wherever it lies outside the band, a repeat of
+    the best unit always fails, and swapped near-tied leaders pass."""
+    from oracle import parity
+    rng = np.random.default_rng(11)
+    V, M, n = 40, 12, 300
+    W = rng.random((V, M)).astype(np.float32)
+    rows = [np.sort(rng.choice(V, size=int(rng.integers(1, 9)), replace=False)).astype(np.int32) for _ in range(n)]
+    indptr = np.zeros(n + 1, np.int32)
+    indptr[1:] = np.cumsum([len(r) for r in rows])
+    indices = np.concatenate(rows)
+    D = orc.all_distances(W.reshape(-1), V, M, indptr, indices)
+    order = np.argsort(D, axis=1, kind="stable")
+    t = orc.bmu(W.reshape(-1), V, M, indptr, indices)
+    ar = np.arange(n)
+    np.testing.assert_array_equal(order[:, 0], t.b1)
+    np.testing.assert_array_equal(order[:, 1], t.b2)
+    good = parity.check_second(t.b1, t.b2, D[ar, t.b2], t, D[ar, t.b2], M)
+    assert good.ok and good.differs_from_oracle == 0
+    third = order[:, 2]
+    far = (D[ar, third] - t.d2) > parity.GAP_REL * t.d2
+    assert far.sum() > n // 2
+    bad = parity.check_second(t.b1, third, D[ar, third], t, D[ar, third], M)
+    assert not bad.ok and bad.outside_band == int(far.sum())
+    rep = parity.check_second(t.b1, t.b1, t.d1, t, t.d1, M)
+    assert not rep.ok and rep.same_as_best == n
+    swapped = parity.check_second(t.b2, t.b1, t.d1, t, t.d1, M)  # leaders the other way round
+    assert swapped.ok
+    wrong_dist = parity.check_second(t.b1, t.b2, D[ar, t.b2] * (1 + 1e-4), t, D[ar, t.b2], M)
+    assert wrong_dist.dist_violations == n
