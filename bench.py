@@ -366,6 +366,8 @@ def main():
     ap.add_argument("--features", default="zipf", choices=["zipf", "uniform"],
                     help="feature popularity of the samples: the workload's Zipf law, or the stress variant "
                          "with features uniform over V (no sharing between samples)")
+    ap.add_argument("--zipf-s", type=float, default=None,
+                    help="override the Zipf exponent of the feature popularity (0 = uniform)")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -374,6 +376,9 @@ def main():
     if args.features == "uniform":
         import dataclasses
         w = dataclasses.replace(w, name=w.name + "-uniform", zipf_s=0.0)
+    if args.zipf_s is not None:
+        import dataclasses
+        w = dataclasses.replace(w, name="%s-zipf%g" % (w.name, args.zipf_s), zipf_s=args.zipf_s)
     if args.impl == "reference":
         run_reference(args, w)
     else:

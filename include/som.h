@@ -20,9 +20,11 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     som_norms / som_bmu only enqueue work on it, with two exceptions: growing the handle's
  *     workspace (first call, or a larger batch than any before) allocates device memory,
- *     which may synchronise the device once; and som_bmu, when it takes its row-table kernel,
- *     first reads d_indptr[0] and d_indptr[n_samples] back to size its plan, which waits for
- *     earlier work on `stream` (the search itself is then only enqueued).
+ *     which may synchronise the device once; and som_bmu, when its row-table kernel is a
+ *     candidate, first runs the feature-selection step of its plan and reads three integers back
+ *     (d_indptr[0], d_indptr[n_samples] and the number of feature instances its table would
+ *     serve) to size the plan and pick the kernel, which waits for earlier work on `stream`
+ *     (the search itself is then only enqueued).
  *   - Thread safety: one handle must not be used from two host threads at once, and two
  *     calls on the same handle must not overlap on the GPU (they share the workspace);
  *     issue them on one stream or order the streams yourself.
@@ -176,7 +178,10 @@ int som_last_cuda_error(const som_handle* h);
  * som_set_option tunes kernel selection: key 0 = search kernel variant (0 auto, 1 direct-load
  * kernel, 2 shared-memory row-table kernel where M % 4 == 0 and V <= 65536); key 1 = hot rows kept in shared
  * memory by the row-table kernel (0 = default); key 2 = its block size (0 = default, 512, 640, 768, 896, 1024);
- * key 3 = neurons per lane there (0 = default, 4, 8; 8 needs M % 64 == 0).
+ * key 3 = neurons per lane there (0 = default, 4, 8; 8 needs M % 64 == 0); key 4 = sample parts per
+ * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
+ * feature instances that the row table's features must cover for the row-table kernel to be taken
+ * (0 = default 50; batches below it go to the direct-load kernel).
  */
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);

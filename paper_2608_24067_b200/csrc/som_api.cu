@@ -100,6 +100,7 @@ int som_destroy(som_handle* h)
     cudaFree(h->hnorm);
     cudaFree(h->ws);
     cudaFree(h->stage);
+    cudaFree(h->head);
     if (h->host_pair) cudaFreeHost(h->host_pair);
     if (h->events_made)
         for (int i = 0; i < SOM_N_EVENTS; ++i) cudaEventDestroy(h->ev[i]);
@@ -140,8 +141,11 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     if (h->timing && (rc = ensure_events(h))) return rc;
 
     // Kernel selection.  The row-table kernel needs 128-bit aligned row segments (M % 4 == 0),
-    // feature ids that fit its 16-bit codes (V <= 65536) and enough (neuron range x sample part) units to occupy every SM; everything else goes
-    // to the direct-load kernel.
+    // feature ids that fit its 16-bit codes (V <= 65536) and enough (neuron range x sample
+    // part) units to occupy every SM; everything else goes to the direct-load kernel.  So do,
+    // in automatic mode, batches whose most frequent features cover too few feature instances
+    // for a shared-memory table to pay: there the direct-load kernel, bound by L2 bandwidth
+    // alone, is faster (measured cross-over: about half of the instances).
     const SomTableGeom geom = som_table_geometry(h);
     bool use_table = h->opt_variant != 1 && (h->M % 4 == 0) && h->V <= 65536 && h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
@@ -150,18 +154,35 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (units < 2 * (int64_t)h->sm_count) use_table = false;
     }
     int64_t nnz = 0;
+    SomPlanBuffers pb;
+    char* head = nullptr;
+    bool begun = false;
     if (use_table) {
-        // The plan's code buffer is sized from the batch's nnz, which lives on the device:
-        // read the two row pointers back (one short synchronisation of the stream per call).
-        if (!h->host_pair) SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 2 * sizeof(int32_t)));
+        // The selection phase of the plan runs first; then the two row pointers (the workspace
+        // is sized from the batch's nnz, which lives on the device) and the number of instances
+        // the chosen features cover come back in one short synchronisation of the stream.
+        const size_t head_need = som_plan_head_bytes(h->V, SOM_PLAN_MASK_FEATURES + geom.n_hot, &pb);
+        if ((rc = ensure_bytes(h, &h->head, &h->head_bytes, head_need))) return rc;
+        head = reinterpret_cast<char*>(h->head);
+        if (!h->host_pair) SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
+        begun = true;
+        if ((rc = som_launch_plan_select(h, d_indptr, d_indices, n_samples, head, pb, SOM_PLAN_MASK_FEATURES,
+                                         geom.n_hot, st)))
+            return rc;
         SOM_CK(h, cudaMemcpyAsync(h->host_pair, d_indptr, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
         SOM_CK(h, cudaMemcpyAsync(h->host_pair + 1, d_indptr + n_samples, sizeof(int32_t),
                                   cudaMemcpyDeviceToHost, st));
+        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 2,
+                                  reinterpret_cast<const int32_t*>(head + pb.n_slots) + SOM_PLAN_COVERED,
+                                  sizeof(int32_t), cudaMemcpyDeviceToHost, st));
         SOM_CK(h, cudaStreamSynchronize(st));
         nnz = (int64_t)h->host_pair[1] - (int64_t)h->host_pair[0];
         if (nnz < 0) return SOM_ERR_INVALID_ARG;
         if (nnz + 6 * n_samples + 4 >= ((int64_t)1 << 31)) use_table = false;
         if (nnz > 0 && !d_indices) return SOM_ERR_INVALID_ARG;
+        const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 50;
+        if (h->opt_variant == 0 && (int64_t)h->host_pair[2] * 100 < cover_pct * nnz) use_table = false;
     }
 
     if (!use_table) {
@@ -169,7 +190,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, 2 * key_bytes))) return rc;
         unsigned long long* keys = reinterpret_cast<unsigned long long*>(h->ws);
         unsigned long long* keys2 = top2 ? keys + key_bytes / sizeof(unsigned long long) : nullptr;
-        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
+        if (!begun && (rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
         SOM_CK(h, cudaMemsetAsync(keys, 0xFF, top2 ? 2 * key_bytes : key_bytes, st));
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
         if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, st))) return rc;
@@ -179,20 +200,17 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (top2 && (rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys2, d_bmu2, d_dist2, st)))
             return rc;
     } else {
-        SomPlanBuffers pb;
-        const size_t need = som_plan_workspace_bytes(h->V, n_samples, nnz,
-                                                     SOM_PLAN_MASK_FEATURES + geom.n_hot, &pb);
+        const size_t need = som_plan_workspace_bytes(n_samples, nnz, &pb);
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
         char* ws = reinterpret_cast<char*>(h->ws);
-        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
         SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
         if (top2)
             SOM_CK(h, cudaMemsetAsync(ws + pb.keys2, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
-        if ((rc = som_launch_plan(h, d_indptr, d_indices, n_samples, ws, pb, SOM_PLAN_MASK_FEATURES,
-                                  geom.n_hot, st)))
+        if ((rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, head, ws, pb, SOM_PLAN_MASK_FEATURES,
+                                       geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_table(h, n_samples, ws, pb, geom.n_hot, top2, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, n_samples, head, ws, pb, geom.n_hot, top2, st))) return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, false, d_bmu,
                                              d_min_dist, st)))
@@ -356,6 +374,11 @@ int som_set_option(som_handle* h, int key, int64_t value)
     if (key == 4) {
         if (value < 0 || value > 1024) return SOM_ERR_INVALID_ARG;
         h->opt_parts = value;
+        return SOM_OK;
+    }
+    if (key == 5) {
+        if (value < 0 || value > 100) return SOM_ERR_INVALID_ARG;
+        h->opt_cover = value;
         return SOM_OK;
     }
     if (key == 3) {

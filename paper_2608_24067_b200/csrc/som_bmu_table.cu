@@ -425,8 +425,8 @@ __global__ void k_finalize_sorted(const float* __restrict__ W, const double* __r
 }
 
 template <int R, int THREADS, bool TOP2>
-int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& b, int n_hot, size_t smem,
-                 cudaStream_t st)
+int launch_table(som_handle* h, int64_t n_real, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
+                 size_t smem, cudaStream_t st)
 {
     constexpr int T = 8 * R;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
@@ -444,13 +444,13 @@ int launch_table(som_handle* h, int64_t n_real, char* ws, const SomPlanBuffers& 
     auto kern = k_bmu_table<R, THREADS, TOP2>;
     SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<grid, THREADS, smem, st>>>(h->W, h->hnorm, h->M,
-                                      reinterpret_cast<const int32_t*>(ws + b.slot_feat),
+                                      reinterpret_cast<const int32_t*>(head + b.slot_feat),
                                       SOM_PLAN_MASK_FEATURES + n_hot,
                                       reinterpret_cast<const uint4*>(ws + b.slots),
                                       reinterpret_cast<const uint32_t*>(ws + b.overflow), n,
                                       reinterpret_cast<u64*>(ws + b.keys),
                                       TOP2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr, parts, part_len, n_units,
-                                      reinterpret_cast<int*>(ws + b.n_slots) + 3);
+                                      reinterpret_cast<int*>(head + b.n_slots) + 3);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;
@@ -483,29 +483,29 @@ SomTableGeom som_table_geometry(const som_handle* h)
 }
 
 template <bool TOP2>
-static int launch_table_any(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
-                            cudaStream_t st)
+static int launch_table_any(som_handle* h, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
+                            int n_hot, cudaStream_t st)
 {
     const SomTableGeom g = som_table_geometry(h);
     if (g.R == 8) {
-        if (g.threads == 1024) return launch_table<8, 1024, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-        if (g.threads == 896) return launch_table<8, 896, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-        if (g.threads == 768) return launch_table<8, 768, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-        if (g.threads == 640) return launch_table<8, 640, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-        return launch_table<8, 512, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+        if (g.threads == 1024) return launch_table<8, 1024, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+        if (g.threads == 896) return launch_table<8, 896, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+        if (g.threads == 768) return launch_table<8, 768, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+        if (g.threads == 640) return launch_table<8, 640, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+        return launch_table<8, 512, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
     }
-    if (g.threads == 1024) return launch_table<4, 1024, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-    if (g.threads == 896) return launch_table<4, 896, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-    if (g.threads == 768) return launch_table<4, 768, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-    if (g.threads == 640) return launch_table<4, 640, TOP2>(h, n, ws, b, n_hot, g.smem, st);
-    return launch_table<4, 512, TOP2>(h, n, ws, b, n_hot, g.smem, st);
+    if (g.threads == 1024) return launch_table<4, 1024, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+    if (g.threads == 896) return launch_table<4, 896, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+    if (g.threads == 768) return launch_table<4, 768, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+    if (g.threads == 640) return launch_table<4, 640, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+    return launch_table<4, 512, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
 }
 
-int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
+int som_launch_bmu_table(som_handle* h, int64_t n, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
                          bool top2, cudaStream_t st)
 {
-    return top2 ? launch_table_any<true>(h, n, ws, b, n_hot, st)
-                : launch_table_any<false>(h, n, ws, b, n_hot, st);
+    return top2 ? launch_table_any<true>(h, n, head, ws, b, n_hot, st)
+                : launch_table_any<false>(h, n, head, ws, b, n_hot, st);
 }
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,

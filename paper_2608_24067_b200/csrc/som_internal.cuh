@@ -26,6 +26,8 @@ struct som_handle {
     size_t ws_bytes;
     void* stage;  // grow-only device staging for som_bmu_host
     size_t stage_bytes;
+    void* head;  // small plan arrays that the selection phase fills before nnz is known
+    size_t head_bytes;
 
     int last_cuda_error;
     int timing;
@@ -38,9 +40,10 @@ struct som_handle {
     int64_t opt_hot_rows;  // 0 = default number of hot rows in shared memory
     int64_t opt_threads;   // block size of the row-table kernel: 0 (default 512), 512 or 1024
     int64_t opt_r;         // neurons per lane of the row-table kernel: 0/4 or 8
-    int64_t opt_parts;     // row-table kernel: most sample parts per neuron range (0 = 16)
+    int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
     int plan_attr_set;
-    int32_t* host_pair;    // pinned, 2 ints: read-back of indptr[0], indptr[n]
+    int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 50)
+    int32_t* host_pair;    // pinned, 3 ints: read-back of indptr[0], indptr[n], covered instances
 };
 
 // event slots

@@ -147,7 +147,10 @@ k_select_hot(const uint32_t* __restrict__ feat_count, int V, int n_mask, int n_h
             if (is_mask) slot = mask_assigned + s_m;
             else if (is_hot) slot = n_mask + hot_assigned + s_h;
             feat_slot[v] = slot;
-            if (slot >= 0) slot_feat[slot] = v;
+            if (slot >= 0) {
+                slot_feat[slot] = v;
+                atomicAdd(&n_slots[SOM_PLAN_COVERED], (int)c);  // instances the table will serve
+            }
         }
         mask_assigned += tot_m;
         hot_assigned += tot_h;
@@ -357,7 +360,22 @@ __global__ void k_pad_slots(uint4* __restrict__ slots, int64_t n, int64_t n_pad)
 
 }  // namespace
 
-size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_max, SomPlanBuffers* b)
+size_t som_plan_head_bytes(int32_t V, int n_slots_max, SomPlanBuffers* b)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t o = off;
+        off = som_align_up(off + bytes, 256);
+        return o;
+    };
+    b->feat_count = take((size_t)V * 4);
+    b->feat_slot = take((size_t)V * 4);
+    b->slot_feat = take((size_t)n_slots_max * 4);
+    b->n_slots = take(SOM_PLAN_N_SLOTS_INTS * 4);
+    return off;
+}
+
+size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b)
 {
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -367,10 +385,6 @@ size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_m
     };
     b->keys = take((size_t)(n + 16) * 8);
     b->keys2 = take((size_t)(n + 16) * 8);
-    b->feat_count = take((size_t)V * 4);
-    b->feat_slot = take((size_t)V * 4);
-    b->slot_feat = take((size_t)n_slots_max * 4);
-    b->n_slots = take(16);
     b->pk = take((size_t)n * 4);
     b->ntail = take((size_t)n * 4);
     b->bin_count = take((size_t)SOM_PLAN_BINS * 4);
@@ -381,23 +395,16 @@ size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_m
     return off;
 }
 
-int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                    char* ws, const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st)
+int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                           char* head, const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st)
 {
-    uint32_t* feat_count = reinterpret_cast<uint32_t*>(ws + b.feat_count);
-    int32_t* feat_slot = reinterpret_cast<int32_t*>(ws + b.feat_slot);
-    int32_t* slot_feat = reinterpret_cast<int32_t*>(ws + b.slot_feat);
-    int32_t* n_slots = reinterpret_cast<int32_t*>(ws + b.n_slots);
-    uint32_t* pk = reinterpret_cast<uint32_t*>(ws + b.pk);
-    uint32_t* ntail = reinterpret_cast<uint32_t*>(ws + b.ntail);
-    uint32_t* bin_count = reinterpret_cast<uint32_t*>(ws + b.bin_count);
-    uint32_t* bin_start = reinterpret_cast<uint32_t*>(ws + b.bin_start);
-    uint32_t* slots = reinterpret_cast<uint32_t*>(ws + b.slots);
-    uint32_t* overflow = reinterpret_cast<uint32_t*>(ws + b.overflow);
+    uint32_t* feat_count = reinterpret_cast<uint32_t*>(head + b.feat_count);
+    int32_t* feat_slot = reinterpret_cast<int32_t*>(head + b.feat_slot);
+    int32_t* slot_feat = reinterpret_cast<int32_t*>(head + b.slot_feat);
+    int32_t* n_slots = reinterpret_cast<int32_t*>(head + b.n_slots);
 
     SOM_CK(h, cudaMemsetAsync(feat_count, 0, (size_t)h->V * 4, st));
-    SOM_CK(h, cudaMemsetAsync(bin_count, 0, (size_t)SOM_PLAN_BINS * 4, st));
-    SOM_CK(h, cudaMemsetAsync(n_slots, 0, 16, st));
+    SOM_CK(h, cudaMemsetAsync(n_slots, 0, SOM_PLAN_N_SLOTS_INTS * 4, st));
 
     // 1. histogram
     {
@@ -418,6 +425,24 @@ int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices
     // 2. select
     k_select_hot<<<1, 1024, 0, st>>>(feat_count, h->V, n_mask, n_hot, feat_slot, slot_feat, n_slots);
     SOM_CK(h, cudaGetLastError());
+    h->launches += 2;
+    return SOM_OK;
+}
+
+int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                         char* head, char* ws, const SomPlanBuffers& b, int n_mask, int n_hot,
+                         cudaStream_t st)
+{
+    int32_t* feat_slot = reinterpret_cast<int32_t*>(head + b.feat_slot);
+    int32_t* n_slots = reinterpret_cast<int32_t*>(head + b.n_slots);
+    uint32_t* pk = reinterpret_cast<uint32_t*>(ws + b.pk);
+    uint32_t* ntail = reinterpret_cast<uint32_t*>(ws + b.ntail);
+    uint32_t* bin_count = reinterpret_cast<uint32_t*>(ws + b.bin_count);
+    uint32_t* bin_start = reinterpret_cast<uint32_t*>(ws + b.bin_start);
+    uint32_t* slots = reinterpret_cast<uint32_t*>(ws + b.slots);
+    uint32_t* overflow = reinterpret_cast<uint32_t*>(ws + b.overflow);
+
+    SOM_CK(h, cudaMemsetAsync(bin_count, 0, (size_t)SOM_PLAN_BINS * 4, st));
     // 3. classify
     const unsigned sblocks = (unsigned)((n + PLAN_THREADS - 1) / PLAN_THREADS);
     k_classify<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, feat_slot, n_mask, pk, ntail, bin_count);
@@ -444,6 +469,6 @@ int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices
         SOM_CK(h, cudaGetLastError());
         h->launches += 1;
     }
-    h->launches += 7;
+    h->launches += 5;
     return SOM_OK;
 }

@@ -32,14 +32,19 @@ struct som_handle;
 #define SOM_SLOT_MAX_TAIL 8
 #define SOM_SLOT_NT_OVERFLOW 255u
 
-// byte offsets into the workspace
+// Byte offsets of the plan's arrays.  The first four live in the small "head" buffer, which
+// the selection phase fills before the batch's nnz is known on the host; the others live in
+// the handle's workspace, sized from nnz.
 struct SomPlanBuffers {
-    size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
-    size_t keys2;       // u64 [n]      the same for the second-best unit (two-best search only)
+    // head buffer
     size_t feat_count;  // u32 [V]
     size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
     size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
-    size_t n_slots;     // i32 [4]      mask slots used, hot slots used, overflow cursor, search unit counter
+    size_t n_slots;     // i32 [8]      mask slots used, hot slots used, overflow cursor, search unit
+                        //              counter, feature instances covered by the table
+    // workspace
+    size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
+    size_t keys2;       // u64 [n]      the same for the second-best unit (two-best search only)
     size_t pk;          // u32 [n]      mask | n_hot << 16, by sample
     size_t ntail;       // u32 [n]
     size_t bin_count;   // u32 [bins]
@@ -48,6 +53,8 @@ struct SomPlanBuffers {
     size_t slots;       // 48 B [n + 16]
     size_t overflow;    // u32 [nnz + 6n]
 };
+#define SOM_PLAN_N_SLOTS_INTS 8
+#define SOM_PLAN_COVERED 4 /* index into n_slots */
 
 // Sample parts per neuron range of the row-table kernel.  More parts mean fewer ranges live at
 // once (their slabs must share L2 with the slot stream) but smaller units, each of which
@@ -59,12 +66,19 @@ static inline int som_table_default_parts(int64_t n)
     return parts < 1 ? 1 : (parts > 32 ? 32 : (int)parts);
 }
 
-size_t som_plan_workspace_bytes(int32_t V, int64_t n, int64_t nnz, int n_slots_max, SomPlanBuffers* b);
+size_t som_plan_head_bytes(int32_t V, int n_slots_max, SomPlanBuffers* b);
+size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b);
 
-int som_launch_plan(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
-                    const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st);
+// Phase 1 (needs no workspace): feature histogram and choice of the mask and hot features;
+// leaves the number of feature instances they cover in n_slots[SOM_PLAN_COVERED].
+int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                           char* head, const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st);
+// Phase 2: classify, sort and re-encode the samples into slots.
+int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
+                         char* head, char* ws, const SomPlanBuffers& b, int n_mask, int n_hot,
+                         cudaStream_t st);
 
-int som_launch_bmu_table(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, int n_hot,
+int som_launch_bmu_table(som_handle* h, int64_t n, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
                          bool top2, cudaStream_t st);
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
