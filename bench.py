@@ -200,7 +200,8 @@ def run_ours(args, w: synth.Workload):
     add_peak = sm_count * FP32_LANES_PER_SM * sm_max_mhz * 1e6  # adds/s
 
     # ---- inputs (synthetic, resident in HBM) -------------------------------------------------
-    W = torch.empty(w.V * w.M, dtype=torch.float32, device=dev)
+    store_bytes = 2 if args.store == "f16" else 4
+    W = torch.empty(w.V * w.M, dtype=torch.float16 if args.store == "f16" else torch.float32, device=dev)
     synth.fill_codebook(w.V, w.M, w.seed, out=W)
     n_batches = max(1, min(4, w.N // w.batch))
     batches = []
@@ -295,11 +296,11 @@ def run_ours(args, w: synth.Workload):
     adds = w.batch * nnz_mean * w.M  # nominal neuron-feature accumulations per launch
     search_s = max(phases["search_ms"], 1e-6) * 1e-3
     achieved = adds / search_s
-    alg_bytes = w.V * w.M * 4 + sum(b.nnz * 4 + (b.n + 1) * 4 for b in batches) / n_batches + w.batch * 8
+    alg_bytes = w.V * w.M * store_bytes + sum(b.nnz * 4 + (b.n + 1) * 4 for b in batches) / n_batches + w.batch * 8
     # DRAM bytes per launch of the search kernel from the committed ncu summary of this workload
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "k_bmu_table_%s.md" % w.name)
-    if os.path.exists(tpath):
+    if os.path.exists(tpath) and args.store == "f32":  # the committed capture is of the fp32 path
         for tl in open(tpath):
             if tl.startswith("traffic_bytes_per_launch"):
                 traffic = float(tl.split("=")[1])
@@ -310,7 +311,7 @@ def run_ours(args, w: synth.Workload):
         "search_ms": phases["search_ms"], "algorithmic_bytes": alg_bytes,
         "hbm_time_at_peak_ms": alg_bytes / (hbm_gbs * 1e9) * 1e3, "hbm_peak_gbs": hbm_gbs,
         "norms_ms": phases["norms_ms"],
-        "norms_hbm_frac": (w.V * w.M * 4 / max(phases["norms_ms"], 1e-6) / 1e6) / hbm_gbs,
+        "norms_hbm_frac": (w.V * w.M * store_bytes / max(phases["norms_ms"], 1e-6) / 1e6) / hbm_gbs,
         "plan_ms": phases["plan_ms"], "finalize_ms": phases["finalize_ms"],
         "step_frac_of_alu_roofline": (adds / add_peak) / (ms_per_step * 1e-3),
     }
@@ -319,7 +320,7 @@ def run_ours(args, w: synth.Workload):
     cpu = None
     if ws == 1 and not args.no_cpu_baseline:
         m_slab = min(w.M, 4096)
-        Wh = W.view(w.V, w.M)[:, :m_slab].contiguous().cpu().numpy()
+        Wh = W.view(w.V, w.M)[:, :m_slab].float().contiguous().cpu().numpy()
         b = batches[0]
         n_take = min(b.n, 100_000)
         ip = b.indptr[:n_take + 1].cpu().numpy()
@@ -330,13 +331,14 @@ def run_ours(args, w: synth.Workload):
     line = {
         "metric": "bmu_samples_per_s", "value": value, "unit": "samples/s", "n_gpus": ws,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if args.store == "f32" else "f32 accumulate, f16-stored codebook",
         "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": nnz_mean,
                    "step": "som_norms + %s on one batch" % ("som_bmu2" if args.top2 else "som_bmu"),
                    "replicas": ws,
                    "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
-                       w.V * w.M * 4 / 1e6, batches[0].nnz * 4 / 1e6) if w.V * w.M * 4 > 126e6 else
+                       w.V * w.M * store_bytes / 1e6, batches[0].nnz * 4 / 1e6) if w.V * w.M * store_bytes > 126e6 else
                    "inputs smaller than L2: steps rotate over %d distinct batches, no flush" % n_batches},
         "accumulations_per_s": ws * adds / (ms_per_step * 1e-3),
         "roofline": roofline,
@@ -368,6 +370,8 @@ def main():
                          "with features uniform over V (no sharing between samples)")
     ap.add_argument("--zipf-s", type=float, default=None,
                     help="override the Zipf exponent of the feature popularity (0 = uniform)")
+    ap.add_argument("--store", default="f32", choices=["f32", "f16"],
+                    help="codebook storage: fp32 (the configurations) or fp16 with fp32 accumulation")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -379,6 +383,9 @@ def main():
     if args.zipf_s is not None:
         import dataclasses
         w = dataclasses.replace(w, name="%s-zipf%g" % (w.name, args.zipf_s), zipf_s=args.zipf_s)
+    if args.store == "f16":
+        import dataclasses
+        w = dataclasses.replace(w, name=w.name + "-f16")
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -65,6 +65,20 @@ enum som_status {
 int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook);
 
 /*
+ * som_create_f16 - som_create for a codebook STORED in fp16 and accumulated in fp32, the paper's
+ * production precision (Section 3.2): half the codebook bytes in HBM, L2 and shared memory
+ * (the 1024x1024 map takes 63 GB instead of 126 GB).
+ *   d_codebook_f16  DEVICE pointer, IEEE binary16, V*M elements, element (v,i) at v*M + i, 16-byte
+ *                   aligned, borrowed like som_create's.
+ * Every later call behaves as with som_create: each stored weight is widened exactly to fp32
+ * before it is used, scores are accumulated in fp32, norms and reported distances in fp64, so the
+ * results are those of som_create on the same values held as fp32.  The vector paths need
+ * M % 8 == 0 (norms), M % 4 == 0 (direct-load kernel) and M % 64 == 0 (row-table kernel); other M
+ * take the scalar-load kernels.
+ */
+int som_create_f16(som_handle** out, int32_t V, int64_t M, const void* d_codebook_f16);
+
+/*
  * som_norms - recompute ||w_i||^2 for all M neurons (the norm term of Eq. 1; the paper's
  * "negligible norm pass", Section 5.7).  One streaming read of the codebook; squares are
  * accumulated in fp64 in a fixed order (deterministic) and stored as fp32.

@@ -58,7 +58,7 @@ inline int mark(som_handle* h, int64_t call, int slot, cudaStream_t st)
 
 extern "C" {
 
-int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook)
+static int create_impl(som_handle** out, int32_t V, int64_t M, const void* d_codebook, bool f16)
 {
     if (!out) return SOM_ERR_INVALID_ARG;
     *out = nullptr;
@@ -79,7 +79,8 @@ int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook)
     h->sm_count = sms;
     h->V = V;
     h->M = M;
-    h->W = d_codebook;
+    h->W = f16 ? nullptr : static_cast<const float*>(d_codebook);
+    h->Wh = f16 ? static_cast<const __half*>(d_codebook) : nullptr;
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->norm64), (size_t)M * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->norm32), (size_t)M * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->hnorm), (size_t)M * sizeof(float));
@@ -89,6 +90,16 @@ int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook)
     }
     *out = h;
     return SOM_OK;
+}
+
+int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook)
+{
+    return create_impl(out, V, M, d_codebook, false);
+}
+
+int som_create_f16(som_handle** out, int32_t V, int64_t M, const void* d_codebook_f16)
+{
+    return create_impl(out, V, M, d_codebook_f16, true);
 }
 
 int som_destroy(som_handle* h)
@@ -147,7 +158,8 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     // for a shared-memory table to pay: there the direct-load kernel, bound by L2 bandwidth
     // alone, is faster (measured cross-over: about half of the instances).
     const SomTableGeom geom = som_table_geometry(h);
-    bool use_table = h->opt_variant != 1 && (h->M % 4 == 0) && h->V <= 65536 && h->M < ((int64_t)1 << 30);
+    bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
+                     h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
         const int64_t parts = som_table_default_parts(n_samples);
         const int64_t units = ((h->M + geom.T - 1) / geom.T) * parts;

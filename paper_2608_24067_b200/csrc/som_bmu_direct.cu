@@ -24,10 +24,25 @@ __device__ __forceinline__ bool before(float a, uint32_t ai, float b, uint32_t b
     return a < b || (a == b && ai < bi);
 }
 
+// four adjacent weights of one feature row with one vector load (16 bytes of fp32, 8 of fp16)
+__device__ __forceinline__ void load4(const float* p, float (&w)[4])
+{
+    const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+    w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+}
+__device__ __forceinline__ void load4(const __half* p, float (&w)[4])
+{
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+    w[0] = a.x; w[1] = a.y; w[2] = b.x; w[3] = b.y;
+}
+
 // TOP2 also keeps the second-best unit in keys2 (Algorithm 2 keeps the two best units).
-template <int VEC, bool TOP2>
+// ST is the storage type of the codebook (float, or __half widened exactly before the fp32 add).
+template <int VEC, bool TOP2, typename ST>
 __global__ void __launch_bounds__(DIRECT_THREADS)
-k_bmu_direct(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
+k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
              const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
              unsigned long long* __restrict__ keys, unsigned long long* __restrict__ keys2,
              int64_t neuron_off)
@@ -55,17 +70,18 @@ k_bmu_direct(const float* __restrict__ W, const float* __restrict__ hnorm, int64
             const int cnt = min(32, end - base);
             for (int j = 0; j < cnt; ++j) {
                 const int v = __shfl_sync(0xffffffffu, mine, j);
-                const float* p = W + (int64_t)v * M + i0;
+                const ST* p = W + (int64_t)v * M + i0;
                 if (VEC == 4) {
                     if (live) {
-                        const float4 w = __ldg(reinterpret_cast<const float4*>(p));
-                        acc[0] -= w.x;
-                        acc[1 % VEC] -= w.y;
-                        acc[2 % VEC] -= w.z;
-                        acc[3 % VEC] -= w.w;
+                        float w[4];
+                        load4(p, w);
+                        acc[0] -= w[0];
+                        acc[1 % VEC] -= w[1];
+                        acc[2 % VEC] -= w[2];
+                        acc[3 % VEC] -= w[3];
                     }
                 } else {
-                    if (live) acc[0] -= __ldg(p);
+                    if (live) acc[0] -= som_weight(p);
                 }
             }
         }
@@ -123,7 +139,8 @@ k_bmu_direct(const float* __restrict__ W, const float* __restrict__ hnorm, int64
 
 // One thread per sample: unpack the winner and recompute its full squared distance
 // |S| - 2*dot + ||w||^2 (left side of Eq. 1) in fp64, ascending feature order.
-__global__ void k_finalize(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
+template <typename ST>
+__global__ void k_finalize(const ST* __restrict__ W, const double* __restrict__ norm64, int64_t M,
                            const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                            int64_t n, const unsigned long long* __restrict__ keys,
                            int32_t* __restrict__ bmu, float* __restrict__ dist)
@@ -139,7 +156,7 @@ __global__ void k_finalize(const float* __restrict__ W, const double* __restrict
     const int beg = indptr[s];
     const int end = indptr[s + 1];
     double dot = 0.0;
-    for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
+    for (int j = beg; j < end; ++j) dot += (double)som_weight(W + (int64_t)indices[j] * M + idx);
     bmu[s] = (int32_t)idx;
     dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
 }
@@ -179,18 +196,21 @@ int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* i
         const int64_t ny = (gy - y0 < max_gy) ? gy - y0 : max_gy;
         dim3 grid((unsigned)gx, (unsigned)ny);
         const int64_t neuron_off = y0 * neurons_per_block;
-        if (vec == 4 && !keys2)
-            k_bmu_direct<4, false><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
-                                                                    keys, keys2, neuron_off);
-        else if (vec == 4)
-            k_bmu_direct<4, true><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
-                                                                   keys, keys2, neuron_off);
-        else if (!keys2)
-            k_bmu_direct<1, false><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
-                                                                    keys, keys2, neuron_off);
-        else
-            k_bmu_direct<1, true><<<grid, DIRECT_THREADS, 0, st>>>(h->W, h->hnorm, h->M, indptr, indices, n,
-                                                                   keys, keys2, neuron_off);
+#define SOM_DIRECT(VEC_, TOP2_, ST_, W_)                                                          \
+    k_bmu_direct<VEC_, TOP2_, ST_><<<grid, DIRECT_THREADS, 0, st>>>(W_, h->hnorm, h->M, indptr, indices, n, \
+                                                                    keys, keys2, neuron_off)
+        if (h->Wh) {
+            if (vec == 4 && !keys2) SOM_DIRECT(4, false, __half, h->Wh);
+            else if (vec == 4) SOM_DIRECT(4, true, __half, h->Wh);
+            else if (!keys2) SOM_DIRECT(1, false, __half, h->Wh);
+            else SOM_DIRECT(1, true, __half, h->Wh);
+        } else {
+            if (vec == 4 && !keys2) SOM_DIRECT(4, false, float, h->W);
+            else if (vec == 4) SOM_DIRECT(4, true, float, h->W);
+            else if (!keys2) SOM_DIRECT(1, false, float, h->W);
+            else SOM_DIRECT(1, true, float, h->W);
+        }
+#undef SOM_DIRECT
         SOM_CK(h, cudaGetLastError());
         h->launches += 1;
     }
@@ -201,8 +221,12 @@ int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* ind
                         const unsigned long long* keys, int32_t* bmu, float* dist, cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
-    k_finalize<<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, keys, bmu,
-                                                 dist);
+    if (h->Wh)
+        k_finalize<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, indptr, indices, n, keys,
+                                                             bmu, dist);
+    else
+        k_finalize<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, keys,
+                                                            bmu, dist);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -137,31 +137,164 @@ __device__ __forceinline__ uint32_t lo16(uint32_t w) { return w & 0xffffu; }
 __device__ __forceinline__ uint32_t hi16(uint32_t w) { return w >> 16; }
 
 // address of row `code` in the codebook slab: base + code * row_stride_bytes, one mad.wide
-__device__ __forceinline__ const float* row_ptr(const float* base, uint32_t code, uint32_t stride_bytes)
+__device__ __forceinline__ const unsigned char* row_ptr(const unsigned char* base, uint32_t code,
+                                                        uint32_t stride_bytes)
 {
-    const float* p;
+    const unsigned char* p;
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(p) : "r"(code), "r"(stride_bytes), "l"(base));
     return p;
 }
 
-#define SOM_HOT(code) sub_acc<H>(acc, lds_acc<H>(tab_q + (code) * ROWB))
-#define SOM_TAIL(code) ldg_acc<H>(row_ptr(w_q, (code), stride_b))
+// ---- storage layouts of the row table -------------------------------------------------------
+// A layout says how a lane's R neurons map onto a T-neuron row, how the lane reads its slice of
+// a row from shared or global memory, and how a slice is subtracted from the lane's scores.
+// In both layouts lane q of a team starts 16 bytes * q into a row.
 
-// R = neurons per lane (4 or 8); a team of 8 lanes covers T = 8*R neurons of one sample.
-// TOP2 also keeps the second-best unit of every sample in keys2 (Algorithm 2 keeps the two
+// fp32 storage: R/4 groups of four neurons, 32 neurons apart; scores as packed f32x2 pairs.
+template <int R_>
+struct LayF32 {
+    typedef float Store;
+    static constexpr int R = R_, H = R_ / 4, T = 8 * R_, ROWB = T * 4;
+    typedef Acc<H> Scores;
+    typedef Acc<H> Slice;
+    static __device__ __forceinline__ Slice lds(const unsigned char* p) { return lds_acc<H>(p); }
+    static __device__ __forceinline__ Slice ldg(const unsigned char* p)
+    {
+        return ldg_acc<H>(reinterpret_cast<const float*>(p));
+    }
+    static __device__ __forceinline__ void sub(Scores& a, const Slice& w) { sub_acc<H>(a, w); }
+    static __device__ __forceinline__ Scores sub3(const Scores& a, const Slice& w) { return sub_acc3<H>(a, w); }
+    static __device__ __forceinline__ Scores seed(const float* hn, int q)
+    {
+        return lds_acc<H>(reinterpret_cast<const unsigned char*>(hn) + q * 16);
+    }
+    static __device__ __forceinline__ void unpack(const Scores& s, float (&a)[R_])
+    {
+#pragma unroll
+        for (int x = 0; x < H; ++x) {
+            unpack2(s.g[x].lo, a[4 * x], a[4 * x + 1]);
+            unpack2(s.g[x].hi, a[4 * x + 2], a[4 * x + 3]);
+        }
+    }
+    static __device__ __forceinline__ int lane_first(int q) { return 4 * q; }
+    static __device__ __forceinline__ uint32_t neuron_of(int rr) { return (uint32_t)((rr >> 2) * 32 + (rr & 3)); }
+    // stage table rows row0.. of this warp: a lane moves element `lane` of each 32-neuron group
+    static __device__ __forceinline__ void stage(unsigned char* tab, const float* __restrict__ W, int64_t M,
+                                                 int64_t i0, const int32_t* __restrict__ slot_feat,
+                                                 int n_rows, int warp, int lane, int warps)
+    {
+        float* tab_f = reinterpret_cast<float*>(tab);
+        for (int row0 = warp * 4; row0 < n_rows; row0 += warps * 4) {
+            float v[4][H];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int row = row0 + u;
+                const int f = row < n_rows ? slot_feat[row] : -1;
+#pragma unroll
+                for (int x = 0; x < H; ++x) {
+                    const int64_t i = i0 + 32 * x + lane;
+                    v[u][x] = (f >= 0 && i < M) ? __ldg(W + (int64_t)f * M + i) : 0.f;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (row0 + u < n_rows) {
+#pragma unroll
+                    for (int x = 0; x < H; ++x) tab_f[(row0 + u) * T + 32 * x + lane] = v[u][x];
+                }
+        }
+    }
+};
+
+// fp16 storage, fp32 scores (the paper's production precision, Section 3.2): a lane owns eight
+// consecutive neurons, i.e. one 128-bit slice of a 128-byte row, so a row costs half the
+// shared-memory and L2 wavefronts of the fp32 layout.  Every weight is widened exactly inside
+// the subtraction (fma.rn.f32.f16 with the multiplier -1: one rounding, that of the fp32 sum).
+struct LayF16 {
+    typedef __half Store;
+    static constexpr int R = 8, T = 64, ROWB = T * 2;
+    struct Scores { float v[8]; };
+    typedef uint4 Slice;
+    static __device__ __forceinline__ Slice lds(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
+    static __device__ __forceinline__ Slice ldg(const unsigned char* p)
+    {
+        Slice r;
+        asm("ld.global.nc.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+        return r;
+    }
+    static __device__ __forceinline__ void sub2(float& d0, float& d1, float a0, float a1, uint32_t w)
+    {
+        asm("{\n\t.reg .b16 l, h, m;\n\tmov.b16 m, 0xBC00;\n\tmov.b32 {l, h}, %4;\n\t"
+            "fma.rn.f32.f16 %0, l, m, %2;\n\tfma.rn.f32.f16 %1, h, m, %3;\n\t}"
+            : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "r"(w));
+    }
+    static __device__ __forceinline__ Scores sub3(const Scores& a, const Slice& w)
+    {
+        Scores r;
+        sub2(r.v[0], r.v[1], a.v[0], a.v[1], w.x);
+        sub2(r.v[2], r.v[3], a.v[2], a.v[3], w.y);
+        sub2(r.v[4], r.v[5], a.v[4], a.v[5], w.z);
+        sub2(r.v[6], r.v[7], a.v[6], a.v[7], w.w);
+        return r;
+    }
+    static __device__ __forceinline__ void sub(Scores& a, const Slice& w) { a = sub3(a, w); }
+    static __device__ __forceinline__ Scores seed(const float* hn, int q)
+    {
+        const float4 lo = *reinterpret_cast<const float4*>(hn + 8 * q);
+        const float4 hi = *reinterpret_cast<const float4*>(hn + 8 * q + 4);
+        Scores r;
+        r.v[0] = lo.x; r.v[1] = lo.y; r.v[2] = lo.z; r.v[3] = lo.w;
+        r.v[4] = hi.x; r.v[5] = hi.y; r.v[6] = hi.z; r.v[7] = hi.w;
+        return r;
+    }
+    static __device__ __forceinline__ void unpack(const Scores& s, float (&a)[8])
+    {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) a[j] = s.v[j];
+    }
+    static __device__ __forceinline__ int lane_first(int q) { return 8 * q; }
+    static __device__ __forceinline__ uint32_t neuron_of(int rr) { return (uint32_t)rr; }
+    // a lane moves one 32-bit word (two neurons) of each row; M % 64 == 0 is guaranteed
+    static __device__ __forceinline__ void stage(unsigned char* tab, const __half* __restrict__ W, int64_t M,
+                                                 int64_t i0, const int32_t* __restrict__ slot_feat,
+                                                 int n_rows, int warp, int lane, int warps)
+    {
+        uint32_t* tab_w = reinterpret_cast<uint32_t*>(tab);
+        for (int row0 = warp * 8; row0 < n_rows; row0 += warps * 8) {
+            uint32_t v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int row = row0 + u;
+                const int f = row < n_rows ? slot_feat[row] : -1;
+                v[u] = (f >= 0) ? __ldg(reinterpret_cast<const uint32_t*>(W + (int64_t)f * M + i0) + lane) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (row0 + u < n_rows) tab_w[(row0 + u) * 32 + lane] = v[u];
+        }
+    }
+};
+
+#define SOM_HOT(code) L::sub(acc, L::lds(tab_q + (code) * ROWB))
+#define SOM_TAIL(code) L::ldg(row_ptr(w_q, (code), stride_b))
+
+// L = storage layout (R = neurons per lane, 4 or 8; a team of 8 lanes covers T = 8*R neurons of
+// one sample).  TOP2 also keeps the second-best unit of every sample in keys2 (Algorithm 2 keeps the two
 // best units); the candidate filter then tests against the second-best score.
-template <int R, int THREADS, bool TOP2>
+template <typename L, int THREADS, bool TOP2>
 __global__ void __launch_bounds__(THREADS, 1)
-k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
+k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
             const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
             u64* __restrict__ keys, u64* __restrict__ keys2, int parts, int64_t part_len, int n_units,
             int* __restrict__ unit_counter)
 {
-    constexpr int H = R / 4;
-    constexpr int T = 8 * R;
-    constexpr int ROWB = T * 4;
+    constexpr int R = L::R;
+    constexpr int T = L::T;
+    constexpr int ROWB = L::ROWB;
     constexpr int WARPS = THREADS / 32;
+    typedef typename L::Scores Scores;
+    typedef typename L::Slice Slice;
     extern __shared__ __align__(16) unsigned char tab[];
     __shared__ int next_chunk;
     __shared__ int unit_sh;
@@ -170,22 +303,20 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
     // of one round.  The bytes of round r+2 are in flight in registers, round r+1 is being
     // stored, round r is being read: slot and key latency never sits on the critical path.
     __shared__ __align__(16) unsigned char ring_sh[WARPS * 2 * RING_STAGE];
-    float* tab_f = reinterpret_cast<float*>(tab);
-
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int q = lane & 7;
     const int sub = lane >> 3;
     const float inf = __int_as_float(0x7f800000);
     const unsigned char* tab_q = tab + q * 16;
-    const unsigned char* hn_q = reinterpret_cast<const unsigned char*>(hn_sh) + q * 16;
-    const uint32_t stride_b = (uint32_t)M * 4u;  // the launcher guarantees M < 2^30
+    const uint32_t stride_b = (uint32_t)M * (uint32_t)sizeof(typename L::Store);  // launcher: M < 2^30
 
     // row n_rows of the table is all zeros: the target of padded hot codes
-    for (int c = threadIdx.x; c < T; c += THREADS) tab_f[n_rows * T + c] = 0.f;
+    for (int c = threadIdx.x; c < ROWB / 4; c += THREADS)
+        reinterpret_cast<uint32_t*>(tab)[n_rows * (ROWB / 4) + c] = 0u;
 
     int cur_range = -1;
-    const float* w_q = W;
+    const unsigned char* w_q = reinterpret_cast<const unsigned char*>(W);
     uint32_t i_first = 0;
     for (;;) {
         // Units are claimed from a global counter in range-major order, so the blocks always
@@ -204,32 +335,14 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
         const int part = unit - range * parts;
         const int64_t i0 = (int64_t)range * T;
         if (range != cur_range) {
-            for (int row0 = warp * 4; row0 < n_rows; row0 += WARPS * 4) {
-                float v[4][H];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int row = row0 + u;
-                    const int f = row < n_rows ? slot_feat[row] : -1;
-#pragma unroll
-                    for (int x = 0; x < H; ++x) {
-                        const int64_t i = i0 + 32 * x + lane;
-                        v[u][x] = (f >= 0 && i < M) ? __ldg(W + (int64_t)f * M + i) : 0.f;
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (row0 + u < n_rows) {
-#pragma unroll
-                        for (int x = 0; x < H; ++x) tab_f[(row0 + u) * T + 32 * x + lane] = v[u][x];
-                    }
-            }
+            L::stage(tab, W, M, i0, slot_feat, n_rows, warp, lane, WARPS);
             cur_range = range;
             // Lanes (or their upper group) past the last neuron still read valid addresses and
             // carry +inf scores, so they never beat a real neuron and need no predicate below.
             // With R = 8 the launcher guarantees M % 64 == 0, so a lane is all in or all out.
-            const int64_t i_lane = i0 + 4 * q;
+            const int64_t i_lane = i0 + L::lane_first(q);
             i_first = (uint32_t)i_lane;
-            w_q = W + (i_lane < M ? i_lane : 0);
+            w_q = reinterpret_cast<const unsigned char*>(W + (i_lane < M ? i_lane : 0));
             for (int c = threadIdx.x; c < T; c += THREADS) hn_sh[c] = (i0 + c < M) ? hnorm[i0 + c] : inf;
         }
         __syncthreads();
@@ -239,7 +352,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
         const int n_chunks = (int)((k_end - k_begin + CHUNK - 1) / CHUNK);
 
         uint32_t curmask = 0;
-        Acc<H> base = lds_acc<H>(hn_q);
+        Scores base = L::seed(hn_sh, q);
         for (;;) {
             int chunk = 0;
             if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
@@ -292,7 +405,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                 const bool p0 = nt > 0, p1 = nt > 1, p2 = nt > 2, p3 = nt > 3;
 
                 // ---- the first four tail rows of this sample go in flight first ---------------
-                Acc<H> tr0, tr1, tr2, tr3;
+                Slice tr0, tr1, tr2, tr3;
                 if (p0) tr0 = SOM_TAIL(lo16(s2.x));
                 if (p1) tr1 = SOM_TAIL(hi16(s2.x));
                 if (p2) tr2 = SOM_TAIL(lo16(s2.y));
@@ -300,12 +413,12 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
 
                 // ---- mask prefix ------------------------------------------------------------
                 if (mask != curmask) {
-                    base = lds_acc<H>(hn_q);
+                    base = L::seed(hn_sh, q);
                     uint32_t mm = mask;
                     while (mm) {
                         const int b = __ffs(mm) - 1;
                         mm &= mm - 1;
-                        sub_acc<H>(base, lds_acc<H>(tab_q + b * ROWB));
+                        L::sub(base, L::lds(tab_q + b * ROWB));
                     }
                     curmask = mask;
                 }
@@ -314,7 +427,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                 //      with the zero row, so a step carries no predicate.  The first step also
                 //      moves the running score out of `base` (which the next sample may reuse).
                 const uint32_t nh_max = __reduce_max_sync(0xffffffffu, nh);
-                Acc<H> acc = sub_acc3<H>(base, lds_acc<H>(tab_q + lo16(s0.z) * ROWB));
+                Scores acc = L::sub3(base, L::lds(tab_q + lo16(s0.z) * ROWB));
                 switch (nh_max) {
                     case 12: SOM_HOT(hi16(s1.w));
                     case 11: SOM_HOT(lo16(s1.w));
@@ -332,16 +445,16 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7 / overflow fields
 
                 // ---- tail rows ------------------------------------------------------------------
-                if (p0) sub_acc<H>(acc, tr0);
-                if (p1) sub_acc<H>(acc, tr1);
-                if (p2) sub_acc<H>(acc, tr2);
-                if (p3) sub_acc<H>(acc, tr3);
+                if (p0) L::sub(acc, tr0);
+                if (p1) L::sub(acc, tr1);
+                if (p2) L::sub(acc, tr2);
+                if (p3) L::sub(acc, tr3);
                 if (nt > 4) {
                     if (nt != SOM_SLOT_NT_OVERFLOW) {
-                        sub_acc<H>(acc, SOM_TAIL(lo16(t45)));
-                        if (nt > 5) sub_acc<H>(acc, SOM_TAIL(hi16(t45)));
-                        if (nt > 6) sub_acc<H>(acc, SOM_TAIL(lo16(t67)));
-                        if (nt > 7) sub_acc<H>(acc, SOM_TAIL(hi16(t67)));
+                        L::sub(acc, SOM_TAIL(lo16(t45)));
+                        if (nt > 5) L::sub(acc, SOM_TAIL(hi16(t45)));
+                        if (nt > 6) L::sub(acc, SOM_TAIL(lo16(t67)));
+                        if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
                     } else {
                         // rare: a sample that does not fit its slot keeps 32-bit lists in the
                         // overflow buffer (w10 = offset, w11 = hot count | tail count << 16).
@@ -350,7 +463,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                         const uint32_t* ol = overflow + t45;
                         const uint32_t onh = lo16(t67), ont = hi16(t67);
                         const uint32_t nt_pad = (ont + 3u) & ~3u;
-                        for (uint32_t j = 0; j < ont; ++j) sub_acc<H>(acc, SOM_TAIL(__ldg(ol + j)));
+                        for (uint32_t j = 0; j < ont; ++j) L::sub(acc, SOM_TAIL(__ldg(ol + j)));
                         for (uint32_t j = 0; j < onh; ++j) SOM_HOT(__ldg(ol + nt_pad + j));
                     }
                 }
@@ -359,11 +472,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
 
                 // ---- lane-local argmin, rare atomic combine ------------------------------------
                 float a[R];
-#pragma unroll
-                for (int x = 0; x < H; ++x) {
-                    unpack2(acc.g[x].lo, a[4 * x], a[4 * x + 1]);
-                    unpack2(acc.g[x].hi, a[4 * x + 2], a[4 * x + 3]);
-                }
+                L::unpack(acc, a);
                 float mn = fminf(fminf(a[0], a[1]), fminf(a[2], a[3]));
                 if (R == 8) mn = fminf(mn, fminf(fminf(a[4 % R], a[5 % R]), fminf(a[6 % R], a[7 % R])));
                 const uint32_t cu = (uint32_t)(key0 >> 32);
@@ -373,7 +482,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
 #pragma unroll
                     for (int j = R - 2; j >= 0; --j)
                         if (a[j] == mn) rr = j;  // lowest neuron among the lane's minima
-                    const uint32_t neuron = i_first + (uint32_t)((rr >> 2) * 32 + (rr & 3));
+                    const uint32_t neuron = i_first + L::neuron_of(rr);
                     const u64 c1 = som_pack_key(mn, neuron);
                     if (!TOP2) {
                         atomicMin(pk - 4, c1);
@@ -393,7 +502,7 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
                         for (int j = R - 1; j >= 0; --j)
                             if (j != rr && a[j] <= m2) { m2 = a[j]; r2 = j; }
                         if (!(m2 > cs))
-                            atomicMin(k2, som_pack_key(m2, i_first + (uint32_t)((r2 >> 2) * 32 + (r2 & 3))));
+                            atomicMin(k2, som_pack_key(m2, i_first + L::neuron_of(r2)));
                     }
                 }
             }
@@ -401,7 +510,8 @@ k_bmu_table(const float* __restrict__ W, const float* __restrict__ hnorm, int64_
     }
 }
 
-__global__ void k_finalize_sorted(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
+template <typename ST>
+__global__ void k_finalize_sorted(const ST* __restrict__ W, const double* __restrict__ norm64, int64_t M,
                                   const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                                   int64_t n, const uint4* __restrict__ slots,
                                   const u64* __restrict__ keys, int32_t* __restrict__ bmu,
@@ -419,16 +529,16 @@ __global__ void k_finalize_sorted(const float* __restrict__ W, const double* __r
     const int beg = indptr[s];
     const int end = indptr[s + 1];
     double dot = 0.0;
-    for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
+    for (int j = beg; j < end; ++j) dot += (double)som_weight(W + (int64_t)indices[j] * M + idx);
     bmu[s] = (int32_t)idx;
     dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
 }
 
-template <int R, int THREADS, bool TOP2>
+template <typename L, int THREADS, bool TOP2>
 int launch_table(som_handle* h, int64_t n_real, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
                  size_t smem, cudaStream_t st)
 {
-    constexpr int T = 8 * R;
+    constexpr int T = L::T;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
     const int n_ranges = (int)((h->M + T - 1) / T);
     int parts = h->opt_parts > 0 ? (int)h->opt_parts : som_table_default_parts(n);
@@ -441,9 +551,10 @@ int launch_table(som_handle* h, int64_t n_real, char* head, char* ws, const SomP
     if (n_units64 > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
     const int n_units = (int)n_units64;
     const int grid = n_units < h->sm_count ? n_units : h->sm_count;
-    auto kern = k_bmu_table<R, THREADS, TOP2>;
+    auto kern = k_bmu_table<L, THREADS, TOP2>;
+    const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(h->Wh ? (const void*)h->Wh : (const void*)h->W);
     SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<grid, THREADS, smem, st>>>(h->W, h->hnorm, h->M,
+    kern<<<grid, THREADS, smem, st>>>(codebook, h->hnorm, h->M,
                                       reinterpret_cast<const int32_t*>(head + b.slot_feat),
                                       SOM_PLAN_MASK_FEATURES + n_hot,
                                       reinterpret_cast<const uint4*>(ws + b.slots),
@@ -464,9 +575,10 @@ SomTableGeom som_table_geometry(const som_handle* h)
     // 8 neurons per lane (half as many rounds for the same work) whenever the neuron count is
     // a multiple of the 64-neuron range it needs; 640 threads leave it 96 registers, the
     // measured optimum between resident warps and spills
-    g.R = (h->opt_r != 4 && h->M % 64 == 0) ? 8 : 4;
+    // (an fp16-stored codebook has the 8-neuron layout only; som_table_usable checks M % 64)
+    g.R = (h->Wh || (h->opt_r != 4 && h->M % 64 == 0)) ? 8 : 4;
     g.T = 8 * g.R;
-    const int row_bytes = g.T * 4;
+    const int row_bytes = g.T * (h->Wh ? 2 : 4);
     const int def_threads = g.R == 8 ? 640 : 1024;
     g.threads = (h->opt_threads == 512 || h->opt_threads == 640 || h->opt_threads == 768 ||
                  h->opt_threads == 896 || h->opt_threads == 1024)
@@ -475,7 +587,7 @@ SomTableGeom som_table_geometry(const som_handle* h)
     int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
     // Defaults keep dynamic + static shared memory under 196 KB: one step more and the SM's
     // carve-out leaves 28 KB instead of 60 KB of L1, which costs 12 % at 128x128 (measured).
-    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (g.R == 8 ? 720 : 1376);
+    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (h->Wh ? 1456 : (g.R == 8 ? 720 : 1376));
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
     g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * row_bytes;  // + the zero row
@@ -487,18 +599,27 @@ static int launch_table_any(som_handle* h, int64_t n, char* head, char* ws, cons
                             int n_hot, cudaStream_t st)
 {
     const SomTableGeom g = som_table_geometry(h);
-    if (g.R == 8) {
-        if (g.threads == 1024) return launch_table<8, 1024, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-        if (g.threads == 896) return launch_table<8, 896, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-        if (g.threads == 768) return launch_table<8, 768, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-        if (g.threads == 640) return launch_table<8, 640, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-        return launch_table<8, 512, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+#define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, TOP2>(h, n, head, ws, b, n_hot, g.smem, st)
+    if (h->Wh) {
+        if (g.threads == 1024) SOM_TABLE(LayF16, 1024);
+        if (g.threads == 896) SOM_TABLE(LayF16, 896);
+        if (g.threads == 768) SOM_TABLE(LayF16, 768);
+        if (g.threads == 640) SOM_TABLE(LayF16, 640);
+        SOM_TABLE(LayF16, 512);
     }
-    if (g.threads == 1024) return launch_table<4, 1024, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-    if (g.threads == 896) return launch_table<4, 896, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-    if (g.threads == 768) return launch_table<4, 768, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-    if (g.threads == 640) return launch_table<4, 640, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
-    return launch_table<4, 512, TOP2>(h, n, head, ws, b, n_hot, g.smem, st);
+    if (g.R == 8) {
+        if (g.threads == 1024) SOM_TABLE(LayF32<8>, 1024);
+        if (g.threads == 896) SOM_TABLE(LayF32<8>, 896);
+        if (g.threads == 768) SOM_TABLE(LayF32<8>, 768);
+        if (g.threads == 640) SOM_TABLE(LayF32<8>, 640);
+        SOM_TABLE(LayF32<8>, 512);
+    }
+    if (g.threads == 1024) SOM_TABLE(LayF32<4>, 1024);
+    if (g.threads == 896) SOM_TABLE(LayF32<4>, 896);
+    if (g.threads == 768) SOM_TABLE(LayF32<4>, 768);
+    if (g.threads == 640) SOM_TABLE(LayF32<4>, 640);
+    SOM_TABLE(LayF32<4>, 512);
+#undef SOM_TABLE
 }
 
 int som_launch_bmu_table(som_handle* h, int64_t n, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
@@ -513,9 +634,14 @@ int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32
                                cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
-    k_finalize_sorted<<<(unsigned)blocks, 256, 0, st>>>(
-        h->W, h->norm64, h->M, indptr, indices, n, reinterpret_cast<const uint4*>(ws + b.slots),
-        reinterpret_cast<const u64*>(ws + (second ? b.keys2 : b.keys)), bmu, dist);
+    const uint4* slots = reinterpret_cast<const uint4*>(ws + b.slots);
+    const u64* keys = reinterpret_cast<const u64*>(ws + (second ? b.keys2 : b.keys));
+    if (h->Wh)
+        k_finalize_sorted<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, indptr, indices, n,
+                                                                    slots, keys, bmu, dist);
+    else
+        k_finalize_sorted<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n,
+                                                                   slots, keys, bmu, dist);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

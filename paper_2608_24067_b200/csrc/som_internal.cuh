@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of the BMU library (sm_100a).
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -15,7 +16,8 @@ struct som_handle {
     int sm_count;
     int32_t V;
     int64_t M;
-    const float* W;  // borrowed, feature-major
+    const float* W;    // borrowed, feature-major fp32 codebook (nullptr when stored as fp16)
+    const __half* Wh;  // borrowed, feature-major fp16 codebook (som_create_f16), else nullptr
 
     double* norm64;  // [M] ||w_i||^2 in fp64
     float* norm32;   // [M] the same rounded to fp32
@@ -73,6 +75,10 @@ __device__ __forceinline__ unsigned long long som_pack_key(float score, uint32_t
 {
     return ((unsigned long long)som_ordered_bits(score) << 32) | (unsigned long long)neuron;
 }
+
+// One stored weight as fp32 (exact for both storage types).
+__device__ __forceinline__ float som_weight(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float som_weight(const __half* p) { return __half2float(__ldg(p)); }
 
 // kernels' host launchers (each returns a som_status)
 int som_launch_norms(som_handle* h, cudaStream_t st);

@@ -61,6 +61,63 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
     for (int k = 0; k < VEC; ++k) out[k] = acc[k];
 }
 
+// The same pass over an fp16-stored codebook: VEC = 8 neurons per thread (one 128-bit load of
+// eight halves per row) or 1; every weight is widened exactly and squared in fp64.
+template <int VEC>
+__global__ void __launch_bounds__(NORM_THREADS)
+k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_split,
+                  double* __restrict__ partial)
+{
+    const int64_t i = ((int64_t)blockIdx.x * NORM_THREADS + threadIdx.x) * VEC;
+    if (i >= M) return;
+    const int v0 = blockIdx.y * rows_per_split;
+    const int v1 = min(V, v0 + rows_per_split);
+    double acc[VEC];
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) acc[k] = 0.0;
+    const __half* p = W + (int64_t)v0 * M + i;
+    int v = v0;
+    if (VEC == 8) {
+        for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
+            uint4 w[NORM_UNROLL];
+#pragma unroll
+            for (int u = 0; u < NORM_UNROLL; ++u)
+                w[u] = __ldcs(reinterpret_cast<const uint4*>(p + (int64_t)u * M));
+#pragma unroll
+            for (int u = 0; u < NORM_UNROLL; ++u) {
+                const uint32_t word[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&word[k]));
+                    acc[(2 * k) % VEC] = fma((double)f.x, (double)f.x, acc[(2 * k) % VEC]);
+                    acc[(2 * k + 1) % VEC] = fma((double)f.y, (double)f.y, acc[(2 * k + 1) % VEC]);
+                }
+            }
+            p += (int64_t)NORM_UNROLL * M;
+        }
+        for (; v < v1; ++v) {
+            const uint4 w = __ldcs(reinterpret_cast<const uint4*>(p));
+            const uint32_t word[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&word[k]));
+                acc[(2 * k) % VEC] = fma((double)f.x, (double)f.x, acc[(2 * k) % VEC]);
+                acc[(2 * k + 1) % VEC] = fma((double)f.y, (double)f.y, acc[(2 * k + 1) % VEC]);
+            }
+            p += M;
+        }
+    } else {
+        for (; v < v1; ++v) {
+            const float w = __half2float(__ldcs(p));
+            acc[0] = fma((double)w, (double)w, acc[0]);
+            p += M;
+        }
+    }
+    double* out = partial + (int64_t)blockIdx.y * M + i;
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) out[k] = acc[k];
+}
+
 __global__ void k_norms_combine(const double* __restrict__ partial, int64_t M, int splits,
                                 double* __restrict__ norm64, float* __restrict__ norm32,
                                 float* __restrict__ hnorm)
@@ -84,7 +141,7 @@ struct NormPlan {
 NormPlan plan_norms(const som_handle* h)
 {
     NormPlan p;
-    p.vec = (h->M % 4 == 0) ? 4 : 1;
+    p.vec = h->Wh ? ((h->M % 8 == 0) ? 8 : 1) : ((h->M % 4 == 0) ? 4 : 1);
     const int64_t col_threads = (h->M + p.vec - 1) / p.vec;
     p.col_blocks = (col_threads + NORM_THREADS - 1) / NORM_THREADS;
     // aim for ~16 resident blocks per SM worth of work, at least 16 rows per split
@@ -111,7 +168,11 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
     NormPlan p = plan_norms(h);
     double* partial = reinterpret_cast<double*>(h->ws);
     dim3 grid((unsigned)p.col_blocks, (unsigned)p.splits);
-    if (p.vec == 4)
+    if (h->Wh && p.vec == 8)
+        k_norms_partial_h<8><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
+    else if (h->Wh)
+        k_norms_partial_h<1><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
+    else if (p.vec == 4)
         k_norms_partial<4><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial);
     else
         k_norms_partial<1><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial);

@@ -24,7 +24,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
-    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2",
+    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -54,6 +54,8 @@ def load_library():
     lib = ctypes.CDLL(LIB_PATH)
     P, I32, I64, INT = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int
     lib.som_create.argtypes = [ctypes.POINTER(P), I32, I64, P]
+    lib.som_create_f16.argtypes = [ctypes.POINTER(P), I32, I64, P]
+    lib.som_create_f16.restype = INT
     lib.som_norms.argtypes = [P, P]
     lib.som_bmu.argtypes = [P, P, P, I64, P, P, P]
     lib.som_bmu_host.argtypes = [P, P, P, I64, P, P, P]
@@ -114,18 +116,22 @@ def norms_noalloc(V: int, M: int, codebook: torch.Tensor, out: torch.Tensor, str
 
 
 class Som:
-    """Handle over a feature-major fp32 codebook resident on the GPU (borrowed, not copied)."""
+    """Handle over a feature-major codebook resident on the GPU (borrowed, not copied): an fp32
+    tensor (som_create) or an fp16 tensor (som_create_f16: fp16 storage, fp32 accumulation)."""
 
     def __init__(self, V: int, M: int, codebook: torch.Tensor):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         if codebook.numel() != V * M:
             raise ValueError("codebook must hold V*M elements")
-        ptr = _dev_ptr(codebook, torch.float32, "codebook")
+        if codebook.dtype not in (torch.float32, torch.float16):
+            raise TypeError("codebook must be a float32 or float16 CUDA tensor")
+        ptr = _dev_ptr(codebook, codebook.dtype, "codebook")
         self.V, self.M = int(V), int(M)
         self.codebook = codebook  # keep the borrowed memory alive
+        create = self._lib.som_create if codebook.dtype == torch.float32 else self._lib.som_create_f16
         with torch.cuda.device(codebook.device):
-            rc = self._lib.som_create(ctypes.byref(self._h), V, M, ptr)
+            rc = create(ctypes.byref(self._h), V, M, ptr)
         if rc != SOM_OK:
             self._h = ctypes.c_void_p()
             raise SomError(rc, "som_create")

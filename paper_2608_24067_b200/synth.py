@@ -78,12 +78,13 @@ def fill_codebook(V: int, M: int, seed: int = 0, device="cpu", out: torch.Tensor
     Base fill U[0,0.05) keyed on the flat offset; then ``spikes_per_neuron`` feature
     ids per neuron, uniform over V, are overwritten with U[0.3,1).  A spike's value is
     keyed on (v,i) and not on the draw number, so a repeated pick writes the same value
-    twice and the result does not depend on write order.
+    twice and the result does not depend on write order.  ``out`` may be a float16 tensor: each
+    fp32 value is then rounded to the nearest fp16 on store (the fp16-stored codebook).
     """
     total = V * M
     if out is None:
         out = torch.empty(total, dtype=torch.float32, device=device)
-    assert out.numel() == total and out.dtype == torch.float32
+    assert out.numel() == total and out.dtype in (torch.float32, torch.float16)
     dev = out.device
     rows_per_chunk = max(1, chunk_elems // M)
     for v0 in range(0, V, rows_per_chunk):
@@ -100,7 +101,7 @@ def fill_codebook(V: int, M: int, seed: int = 0, device="cpu", out: torch.Tensor
             v = hash32(seed, _STREAM_SPIKE_POS, i, k) % V
             flat = v * M + i
             val = _u24_to_f32(hash32(seed, _STREAM_SPIKE_VAL, flat, 0), 0.3, 0.7)
-            out[flat] = val
+            out[flat] = val.to(out.dtype)
     return out
 
 
