@@ -155,6 +155,7 @@ template <int R_>
 struct LayF32 {
     typedef float Store;
     static constexpr int R = R_, H = R_ / 4, T = 8 * R_, ROWB = T * 4;
+    static constexpr float SEED_SIGN = 1.f;     // scores are held as they are
     typedef Acc<H> Scores;
     typedef Acc<H> Slice;
     static __device__ __forceinline__ Slice lds(const unsigned char* p) { return lds_acc<H>(p); }
@@ -209,10 +210,14 @@ struct LayF32 {
 // fp16 storage, fp32 scores (the paper's production precision, Section 3.2): a lane owns eight
 // consecutive neurons, i.e. one 128-bit slice of a 128-byte row, so a row costs half the
 // shared-memory and L2 wavefronts of the fp32 layout.  Every weight is widened exactly inside
-// the subtraction (fma.rn.f32.f16 with the multiplier -1: one rounding, that of the fp32 sum).
+// the mixed-precision add (add.rn.f32.f16: one rounding, that of the fp32 sum).  That
+// instruction only adds, so the lane holds NEGATED scores, sum(rows) - ||w||^2/2, and flips
+// the sign when it hands them to the argmin; (-a) - w and -(a + w) round identically, so the
+// scores are those of the subtracting form.
 struct LayF16 {
     typedef __half Store;
     static constexpr int R = 8, T = 64, ROWB = T * 2;
+    static constexpr float SEED_SIGN = -1.f;  // the seed array holds -||w||^2/2
     struct Scores { float v[8]; };
     typedef uint4 Slice;
     static __device__ __forceinline__ Slice lds(const unsigned char* p) { return *reinterpret_cast<const uint4*>(p); }
@@ -222,19 +227,19 @@ struct LayF16 {
         asm("ld.global.nc.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
         return r;
     }
-    static __device__ __forceinline__ void sub2(float& d0, float& d1, float a0, float a1, uint32_t w)
+    static __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, uint32_t w)
     {
-        asm("{\n\t.reg .b16 l, h, m;\n\tmov.b16 m, 0xBC00;\n\tmov.b32 {l, h}, %4;\n\t"
-            "fma.rn.f32.f16 %0, l, m, %2;\n\tfma.rn.f32.f16 %1, h, m, %3;\n\t}"
+        asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %4;\n\t"
+            "add.rn.f32.f16 %0, l, %2;\n\tadd.rn.f32.f16 %1, h, %3;\n\t}"
             : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "r"(w));
     }
     static __device__ __forceinline__ Scores sub3(const Scores& a, const Slice& w)
     {
         Scores r;
-        sub2(r.v[0], r.v[1], a.v[0], a.v[1], w.x);
-        sub2(r.v[2], r.v[3], a.v[2], a.v[3], w.y);
-        sub2(r.v[4], r.v[5], a.v[4], a.v[5], w.z);
-        sub2(r.v[6], r.v[7], a.v[6], a.v[7], w.w);
+        add2(r.v[0], r.v[1], a.v[0], a.v[1], w.x);
+        add2(r.v[2], r.v[3], a.v[2], a.v[3], w.y);
+        add2(r.v[4], r.v[5], a.v[4], a.v[5], w.z);
+        add2(r.v[6], r.v[7], a.v[6], a.v[7], w.w);
         return r;
     }
     static __device__ __forceinline__ void sub(Scores& a, const Slice& w) { a = sub3(a, w); }
@@ -250,7 +255,7 @@ struct LayF16 {
     static __device__ __forceinline__ void unpack(const Scores& s, float (&a)[8])
     {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) a[j] = s.v[j];
+        for (int j = 0; j < 8; ++j) a[j] = -s.v[j];
     }
     static __device__ __forceinline__ int lane_first(int q) { return 8 * q; }
     static __device__ __forceinline__ uint32_t neuron_of(int rr) { return (uint32_t)rr; }
@@ -343,7 +348,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const int64_t i_lane = i0 + L::lane_first(q);
             i_first = (uint32_t)i_lane;
             w_q = reinterpret_cast<const unsigned char*>(W + (i_lane < M ? i_lane : 0));
-            for (int c = threadIdx.x; c < T; c += THREADS) hn_sh[c] = (i0 + c < M) ? hnorm[i0 + c] : inf;
+            for (int c = threadIdx.x; c < T; c += THREADS)
+                hn_sh[c] = L::SEED_SIGN * ((i0 + c < M) ? hnorm[i0 + c] : inf);
         }
         __syncthreads();
 
@@ -579,7 +585,8 @@ SomTableGeom som_table_geometry(const som_handle* h)
     g.R = (h->Wh || (h->opt_r != 4 && h->M % 64 == 0)) ? 8 : 4;
     g.T = 8 * g.R;
     const int row_bytes = g.T * (h->Wh ? 2 : 4);
-    const int def_threads = g.R == 8 ? 640 : 1024;
+    // (the fp16 layout holds half as many row registers: 896 threads at 72 registers measured best)
+    const int def_threads = h->Wh ? 896 : (g.R == 8 ? 640 : 1024);
     g.threads = (h->opt_threads == 512 || h->opt_threads == 640 || h->opt_threads == 768 ||
                  h->opt_threads == 896 || h->opt_threads == 1024)
                     ? (int)h->opt_threads : def_threads;
