@@ -192,7 +192,8 @@ int som_last_cuda_error(const som_handle* h);
  * som_set_option tunes kernel selection: key 0 = search kernel variant (0 auto, 1 direct-load
  * kernel, 2 shared-memory row-table kernel where M % 4 == 0 and V <= 65536); key 1 = hot rows kept in shared
  * memory by the row-table kernel (0 = default); key 2 = its block size (0 = default, 512, 640, 768, 896, 1024);
- * key 3 = neurons per lane there (0 = default, 4, 8; 8 needs M % 64 == 0); key 4 = sample parts per
+ * key 3 = neurons per lane there (0 = default; fp32 storage: 4, 8, where 8 needs M % 64 == 0; fp16 storage:
+ * 8, 16, where 16 needs M % 128 == 0); key 4 = sample parts per
  * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
  * feature instances that the row table's features must cover for the row-table kernel to be taken
  * (0 = default 50; batches below it go to the direct-load kernel).

@@ -161,7 +161,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
                      h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
-        const int64_t parts = som_table_default_parts(n_samples);
+        const int64_t parts = som_table_default_parts(n_samples, geom.T);
         const int64_t units = ((h->M + geom.T - 1) / geom.T) * parts;
         if (units < 2 * (int64_t)h->sm_count) use_table = false;
     }
@@ -394,7 +394,7 @@ int som_set_option(som_handle* h, int key, int64_t value)
         return SOM_OK;
     }
     if (key == 3) {
-        if (value != 0 && value != 4 && value != 8) return SOM_ERR_INVALID_ARG;
+        if (value != 0 && value != 4 && value != 8 && value != 16) return SOM_ERR_INVALID_ARG;
         h->opt_r = value;
         return SOM_OK;
     }

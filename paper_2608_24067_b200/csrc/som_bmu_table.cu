@@ -280,6 +280,86 @@ struct LayF16 {
     }
 };
 
+// The same with 16 neurons per lane: two groups of eight, 64 neurons apart (two 128-bit slices
+// of a 256-byte row).  Twice the work per round for the same per-round bookkeeping.
+struct LayF16W {
+    typedef __half Store;
+    static constexpr int R = 16, T = 128, ROWB = T * 2;
+    static constexpr float SEED_SIGN = -1.f;
+    struct Scores { float v[16]; };
+    struct Slice { uint4 g[2]; };
+    static __device__ __forceinline__ Slice lds(const unsigned char* p)
+    {
+        Slice r;
+        r.g[0] = *reinterpret_cast<const uint4*>(p);
+        r.g[1] = *reinterpret_cast<const uint4*>(p + 128);
+        return r;
+    }
+    static __device__ __forceinline__ Slice ldg(const unsigned char* p)
+    {
+        Slice r;
+        r.g[0] = LayF16::ldg(p);
+        r.g[1] = LayF16::ldg(p + 128);
+        return r;
+    }
+    static __device__ __forceinline__ Scores sub3(const Scores& a, const Slice& w)
+    {
+        Scores r;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            LayF16::add2(r.v[8 * x + 0], r.v[8 * x + 1], a.v[8 * x + 0], a.v[8 * x + 1], w.g[x].x);
+            LayF16::add2(r.v[8 * x + 2], r.v[8 * x + 3], a.v[8 * x + 2], a.v[8 * x + 3], w.g[x].y);
+            LayF16::add2(r.v[8 * x + 4], r.v[8 * x + 5], a.v[8 * x + 4], a.v[8 * x + 5], w.g[x].z);
+            LayF16::add2(r.v[8 * x + 6], r.v[8 * x + 7], a.v[8 * x + 6], a.v[8 * x + 7], w.g[x].w);
+        }
+        return r;
+    }
+    static __device__ __forceinline__ void sub(Scores& a, const Slice& w) { a = sub3(a, w); }
+    static __device__ __forceinline__ Scores seed(const float* hn, int q)
+    {
+        Scores r;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const float4 lo = *reinterpret_cast<const float4*>(hn + 64 * x + 8 * q);
+            const float4 hi = *reinterpret_cast<const float4*>(hn + 64 * x + 8 * q + 4);
+            r.v[8 * x + 0] = lo.x; r.v[8 * x + 1] = lo.y; r.v[8 * x + 2] = lo.z; r.v[8 * x + 3] = lo.w;
+            r.v[8 * x + 4] = hi.x; r.v[8 * x + 5] = hi.y; r.v[8 * x + 6] = hi.z; r.v[8 * x + 7] = hi.w;
+        }
+        return r;
+    }
+    static __device__ __forceinline__ void unpack(const Scores& s, float (&a)[16])
+    {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) a[j] = -s.v[j];
+    }
+    static __device__ __forceinline__ int lane_first(int q) { return 8 * q; }
+    static __device__ __forceinline__ uint32_t neuron_of(int rr) { return (uint32_t)((rr >> 3) * 64 + (rr & 7)); }
+    // a lane moves two 32-bit words (four neurons) of each row; M % 128 == 0 is guaranteed
+    static __device__ __forceinline__ void stage(unsigned char* tab, const __half* __restrict__ W, int64_t M,
+                                                 int64_t i0, const int32_t* __restrict__ slot_feat,
+                                                 int n_rows, int warp, int lane, int warps)
+    {
+        uint32_t* tab_w = reinterpret_cast<uint32_t*>(tab);
+        for (int row0 = warp * 4; row0 < n_rows; row0 += warps * 4) {
+            uint32_t v[4][2];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int row = row0 + u;
+                const int f = row < n_rows ? slot_feat[row] : -1;
+                const uint32_t* src = reinterpret_cast<const uint32_t*>(W + (int64_t)(f >= 0 ? f : 0) * M + i0);
+                v[u][0] = (f >= 0) ? __ldg(src + lane) : 0u;
+                v[u][1] = (f >= 0) ? __ldg(src + 32 + lane) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (row0 + u < n_rows) {
+                    tab_w[(row0 + u) * 64 + lane] = v[u][0];
+                    tab_w[(row0 + u) * 64 + 32 + lane] = v[u][1];
+                }
+        }
+    }
+};
+
 #define SOM_HOT(code) L::sub(acc, L::lds(tab_q + (code) * ROWB))
 #define SOM_TAIL(code) L::ldg(row_ptr(w_q, (code), stride_b))
 
@@ -480,7 +560,11 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 float a[R];
                 L::unpack(acc, a);
                 float mn = fminf(fminf(a[0], a[1]), fminf(a[2], a[3]));
-                if (R == 8) mn = fminf(mn, fminf(fminf(a[4 % R], a[5 % R]), fminf(a[6 % R], a[7 % R])));
+                if (R >= 8) mn = fminf(mn, fminf(fminf(a[4 % R], a[5 % R]), fminf(a[6 % R], a[7 % R])));
+                if (R == 16) {
+                    mn = fminf(mn, fminf(fminf(a[8 % R], a[9 % R]), fminf(a[10 % R], a[11 % R])));
+                    mn = fminf(mn, fminf(fminf(a[12 % R], a[13 % R]), fminf(a[14 % R], a[15 % R])));
+                }
                 const uint32_t cu = (uint32_t)(key0 >> 32);
                 const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
                 if (!(mn > cs)) {
@@ -547,7 +631,7 @@ int launch_table(som_handle* h, int64_t n_real, char* head, char* ws, const SomP
     constexpr int T = L::T;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
     const int n_ranges = (int)((h->M + T - 1) / T);
-    int parts = h->opt_parts > 0 ? (int)h->opt_parts : som_table_default_parts(n);
+    int parts = h->opt_parts > 0 ? (int)h->opt_parts : som_table_default_parts(n, T);
     if ((int64_t)parts * 1024 > n) parts = (int)(n / 1024);
     if (parts < 1) parts = 1;
     int64_t part_len = (n + parts - 1) / parts;
@@ -583,10 +667,11 @@ SomTableGeom som_table_geometry(const som_handle* h)
     // measured optimum between resident warps and spills
     // (an fp16-stored codebook has the 8-neuron layout only; som_table_usable checks M % 64)
     g.R = (h->Wh || (h->opt_r != 4 && h->M % 64 == 0)) ? 8 : 4;
+    if (h->Wh && h->opt_r != 8 && h->M % 128 == 0) g.R = 16;  // wide fp16 layout wherever it divides M
     g.T = 8 * g.R;
     const int row_bytes = g.T * (h->Wh ? 2 : 4);
     // (the fp16 layout holds half as many row registers: 896 threads at 72 registers measured best)
-    const int def_threads = h->Wh ? 896 : (g.R == 8 ? 640 : 1024);
+    const int def_threads = h->Wh ? (g.R == 16 ? 512 : 896) : (g.R == 8 ? 640 : 1024);
     g.threads = (h->opt_threads == 512 || h->opt_threads == 640 || h->opt_threads == 768 ||
                  h->opt_threads == 896 || h->opt_threads == 1024)
                     ? (int)h->opt_threads : def_threads;
@@ -594,7 +679,7 @@ SomTableGeom som_table_geometry(const som_handle* h)
     int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
     // Defaults keep dynamic + static shared memory under 196 KB: one step more and the SM's
     // carve-out leaves 28 KB instead of 60 KB of L1, which costs 12 % at 128x128 (measured).
-    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (h->Wh ? 1456 : (g.R == 8 ? 720 : 1376));
+    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (row_bytes == 128 ? (h->Wh ? 1456 : 1376) : 720);
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
     g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * row_bytes;  // + the zero row
@@ -607,6 +692,11 @@ static int launch_table_any(som_handle* h, int64_t n, char* head, char* ws, cons
 {
     const SomTableGeom g = som_table_geometry(h);
 #define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, TOP2>(h, n, head, ws, b, n_hot, g.smem, st)
+    if (h->Wh && g.R == 16) {
+        if (g.threads == 768) SOM_TABLE(LayF16W, 768);
+        if (g.threads == 640) SOM_TABLE(LayF16W, 640);
+        SOM_TABLE(LayF16W, 512);
+    }
     if (h->Wh) {
         if (g.threads == 1024) SOM_TABLE(LayF16, 1024);
         if (g.threads == 896) SOM_TABLE(LayF16, 896);

@@ -41,7 +41,7 @@ struct som_handle {
     int64_t opt_variant;   // 0 auto, 1 direct-load kernel, 2 row-table kernel
     int64_t opt_hot_rows;  // 0 = default number of hot rows in shared memory
     int64_t opt_threads;   // block size of the row-table kernel: 0 (default 512), 512 or 1024
-    int64_t opt_r;         // neurons per lane of the row-table kernel: 0/4 or 8
+    int64_t opt_r;         // neurons per lane of the row-table kernel: 0 = default, 4, 8 or 16
     int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
     int plan_attr_set;
     int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 50)

@@ -59,11 +59,14 @@ struct SomPlanBuffers {
 // Sample parts per neuron range of the row-table kernel.  More parts mean fewer ranges live at
 // once (their slabs must share L2 with the slot stream) but smaller units, each of which
 // rebuilds the row table; with units claimed in order the optimum is flat: about 20,000
-// samples per unit, at most 32 parts (measured on 250k to 4M-sample batches).
-static inline int som_table_default_parts(int64_t n)
+// samples per unit, at most 32 parts (measured on 250k to 4M-sample batches).  The 128-neuron
+// ranges of the wide fp16 layout are half as many, so their units are made smaller.
+static inline int som_table_default_parts(int64_t n, int range_neurons)
 {
-    const int64_t parts = n / 20000;
-    return parts < 1 ? 1 : (parts > 32 ? 32 : (int)parts);
+    const bool wide = range_neurons >= 128;
+    const int64_t parts = n / (wide ? 15000 : 20000);
+    const int64_t cap = wide ? 64 : 32;
+    return parts < 1 ? 1 : (parts > cap ? (int)cap : (int)parts);
 }
 
 size_t som_plan_head_bytes(int32_t V, int n_slots_max, SomPlanBuffers* b);

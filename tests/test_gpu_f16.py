@@ -89,12 +89,14 @@ def test_f16_config2_sampled_rows(som_mod, variant):
     assert rep.near_ties < 0.05 * rows.size
 
 
-@pytest.mark.parametrize("threads", [512, 640, 768, 1024])
-def test_f16_row_table_block_sizes(som_mod, threads):
+@pytest.mark.parametrize("lane_neurons,threads", [(8, 640), (8, 896), (8, 1024), (16, 512), (16, 640)])
+def test_f16_row_table_geometries(som_mod, lane_neurons, threads):
+    """Both fp16 layouts of the row-table kernel (64- and 128-neuron ranges) and block sizes."""
     V, M, n = 30_000, 1_024, 60_000
     W16 = synth.fill_codebook(V, M, 3, device="cuda").half()
     b = synth.sample_csr(n, V, 11.0, 3, device="cuda", permute_ids=True)
-    _run_and_check(som_mod, W16, V, M, b.indptr, b.indices, 2, options=((2, threads),), rows=np.arange(0, n, 7))
+    _run_and_check(som_mod, W16, V, M, b.indptr, b.indices, 2, options=((3, lane_neurons), (2, threads)),
+                   rows=np.arange(0, n, 7))
 
 
 @pytest.mark.parametrize("variant", [1, 2, 0])
