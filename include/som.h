@@ -123,6 +123,30 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
              int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream);
 
 /*
+ * som_update - the batch update that follows the search in an epoch (Section 3.4; Algorithm 2,
+ * steps 8-9): scatter the samples onto the lattice (per cell the sum of its assigned samples
+ * and their count), blur both fields with three unnormalised box passes per lattice axis of
+ * half-width `radius` whose window is truncated at the lattice edge, and REPLACE every prototype
+ * by the ratio; a neuron whose blurred count is zero keeps its prototype.  No learning rate.
+ *   rows, cols   lattice shape, rows * cols == M; neuron i sits at row i / cols, column i % cols.
+ *   d_indptr, d_indices, n_samples   the epoch's samples as in som_bmu (DEVICE CSR); an epoch
+ *                searched in several batches passes their concatenation.
+ *   d_bmu        DEVICE pointer, int32 [n_samples]: the best unit of every sample (som_bmu's output).
+ *   radius       box half-width in cells, >= 0; the paper uses the schedule's sigma rounded to whole
+ *                cells and never smaller than one (the caller applies the schedule).
+ * WRITES the codebook the handle borrows, in place (fp32, or fp16 for som_create_f16: sums and the
+ * blur are carried in fp32/fp64 and rounded to the storage type only at this final write), so
+ * som_norms must run again before the next search.  Work is enqueued on `stream`; the features are
+ * processed in slabs through the handle's workspace (option 6 bounds it), so no second V x M array
+ * is needed.  The window sums are running sums (add the entering cell, subtract the leaving one):
+ * constant work per cell whatever the radius, but a cell whose exact sum is many orders of
+ * magnitude below the largest sum of its line inherits that line's rounding error (2^-53 relative
+ * to the largest; the sums are carried in fp64).
+ */
+int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indptr, const int32_t* d_indices,
+               int64_t n_samples, const int32_t* d_bmu, int32_t radius, void* stream);
+
+/*
  * som_bmu_host - the same search with HOST buffers: copies the CSR batch to device staging
  * memory owned by the handle, runs som_bmu, copies both outputs back, all enqueued on
  * `stream`, then synchronises that stream before returning.  h_* pointers are host memory
@@ -196,7 +220,8 @@ int som_last_cuda_error(const som_handle* h);
  * 8, 16, where 16 needs M % 128 == 0); key 4 = sample parts per
  * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
  * feature instances that the row table's features must cover for the row-table kernel to be taken
- * (0 = default 50; batches below it go to the direct-load kernel).
+ * (0 = default 50; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
+ * slab buffers in MiB (0 = default 1024).
  */
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);

@@ -249,6 +249,24 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
     return bmu_impl(h, d_indptr, d_indices, n_samples, d_bmu, d_min_dist, d_bmu2, d_dist2, stream);
 }
 
+int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indptr, const int32_t* d_indices,
+               int64_t n_samples, const int32_t* d_bmu, int32_t radius, void* stream)
+{
+    if (!h || n_samples < 0 || rows <= 0 || cols <= 0 || radius < 0) return SOM_ERR_INVALID_ARG;
+    if ((int64_t)rows * cols != h->M) return SOM_ERR_INVALID_ARG;
+    if (n_samples > 0 && (!d_indptr || !d_bmu)) return SOM_ERR_INVALID_ARG;
+    if (n_samples >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int planes = 1;
+    const int64_t budget = (h->opt_update_mib > 0 ? h->opt_update_mib : 1024) << 20;
+    const size_t need = som_update_workspace_bytes(h, budget, &planes);
+    int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need);
+    if (rc) return rc;
+    h->norms_valid = 0;  // the codebook changes: som_norms must run before the next search
+    return som_launch_update(h, rows, cols, d_indptr, d_indices, n_samples, d_bmu, radius, planes, st);
+}
+
 int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,
                  int32_t* h_bmu, float* h_min_dist, void* stream)
 {
@@ -386,6 +404,11 @@ int som_set_option(som_handle* h, int key, int64_t value)
     if (key == 4) {
         if (value < 0 || value > 1024) return SOM_ERR_INVALID_ARG;
         h->opt_parts = value;
+        return SOM_OK;
+    }
+    if (key == 6) {
+        if (value < 0 || value > (1 << 20)) return SOM_ERR_INVALID_ARG;
+        h->opt_update_mib = value;
         return SOM_OK;
     }
     if (key == 5) {

@@ -44,6 +44,7 @@ struct som_handle {
     int64_t opt_r;         // neurons per lane of the row-table kernel: 0 = default, 4, 8 or 16
     int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
     int plan_attr_set;
+    int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 1024)
     int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 50)
     int32_t* host_pair;    // pinned, 3 ints: read-back of indptr[0], indptr[n], covered instances
 };
@@ -89,3 +90,6 @@ int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* ind
 int som_launch_validate(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                         int* d_flag, cudaStream_t st);
 size_t som_norms_workspace_bytes(const som_handle* h);
+size_t som_update_workspace_bytes(const som_handle* h, int64_t budget_bytes, int* planes_per_slab);
+int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, const int32_t* indices,
+                      int64_t n, const int32_t* bmu, int radius, int planes_per_slab, cudaStream_t st);

@@ -1,0 +1,234 @@
+// Batch update of the codebook (Section 3.4 of the paper; Algorithm 2, steps 8-9): scatter the
+// batch onto the lattice (per cell the sum of the assigned binary samples, num, and their count,
+// den), blur both fields with three unnormalised box passes per lattice axis whose window is
+// truncated at the edge, and replace every prototype by num / den where den > 0.
+//
+// Layout and order of work.  The codebook is feature-major, so the field of one feature (a
+// "plane": rows x cols cells, neuron i at row i / cols, column i % cols) is contiguous, and the
+// planes are independent.  They are processed in slabs of as many planes as fit a bounded
+// workspace (two buffers), so the update needs no second V x M array beside the codebook:
+//   1. scatter the slab's features into buffer A in TRANSPOSED cell order (col-major), so that
+//   2. three box passes along the slow index, one thread per (plane, fast index) walking a line
+//      with coalesced loads and a running window sum (add the entering element, subtract the
+//      leaving one: O(1) per cell whatever the radius), are the passes along the lattice rows;
+//   3. a tiled transpose back to neuron order;
+//   4. three more such passes, now along the lattice columns, the last one fused with the
+//      division and the write of the new weights (fp32 or fp16 storage; rounding happens only at
+//      this final write).
+// Box passes along different axes commute, so three per axis in this order equal the paper's
+// (row, column) x 3.  The running sums are carried in fp64 (the paper carries fp32); the fields
+// between passes are fp32.  Whether a neuron's blurred denominator is zero is decided exactly,
+// from an integer box count of the occupied cells over the reach of three passes (3 * radius):
+// a running sum that subtracts can leave a rounding residue where the exact sum is zero.
+#include "som_internal.cuh"
+
+namespace {
+
+constexpr int UPD_THREADS = 256;
+
+__global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows, int cols,
+                            float* __restrict__ den_t, int32_t* __restrict__ occ)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n) return;
+    const int c = bmu[s];
+    const int r = c / cols, q = c - r * cols;
+    atomicAdd(&den_t[(int64_t)q * rows + r], 1.0f);  // transposed cell order
+    occ[c] = 1;
+}
+
+// one thread per sample: its features inside [v0, v1) add 1 to the cell of its best unit
+__global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
+                              int64_t n, const int32_t* __restrict__ bmu, int v0, int v1, int rows, int cols,
+                              float* __restrict__ num_t)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n) return;
+    const int c = bmu[s];
+    const int r = c / cols, q = c - r * cols;
+    const int64_t cell_t = (int64_t)q * rows + r;
+    const int64_t M = (int64_t)rows * cols;
+    const int beg = indptr[s], end = indptr[s + 1];
+    for (int j = beg; j < end; ++j) {
+        const int v = indices[j];
+        if (v >= v1) break;  // ids ascend inside a row
+        if (v >= v0) atomicAdd(&num_t[(int64_t)(v - v0) * M + cell_t], 1.0f);
+    }
+}
+
+// Box pass along the slow index of planes laid out [plane][len][width]: thread (plane, f) walks
+// i = 0..len-1 at fixed fast index f.  out = sum of in over [i - radius, i + radius] clipped to
+// the line.  T = float (fields) or int32 (the occupancy count).
+template <typename T, typename ACC>
+__global__ void k_box_pass(const T* __restrict__ in, T* __restrict__ out, int64_t planes, int len, int width,
+                           int radius)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= planes * width) return;
+    const int64_t p = t / width;
+    const int f = (int)(t - p * width);
+    const T* src = in + p * (int64_t)len * width + f;
+    T* dst = out + p * (int64_t)len * width + f;
+    ACC sum = 0;
+    const int first = radius < len - 1 ? radius : len - 1;
+    for (int j = 0; j <= first; ++j) sum += (ACC)src[(int64_t)j * width];
+    dst[0] = (T)sum;
+    for (int i = 1; i < len; ++i) {
+        if (i + radius < len) sum += (ACC)src[(int64_t)(i + radius) * width];
+        if (i - radius - 1 >= 0) sum -= (ACC)src[(int64_t)(i - radius - 1) * width];
+        dst[(int64_t)i * width] = (T)sum;
+    }
+}
+
+// The last pass, along the lattice columns of planes in neuron order, fused with the division
+// and the write of the new weights of features v0 + plane.  den_b is the blurred denominator
+// and reach the exact count of occupied cells within reach; where it is zero the prototype stays.
+template <typename ST>
+__global__ void k_box_pass_divide(const float* __restrict__ in, int64_t planes, int rows, int cols, int radius,
+                                  const float* __restrict__ den_b, const int32_t* __restrict__ reach,
+                                  ST* __restrict__ W, int v0)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= planes * cols) return;
+    const int64_t p = t / cols;
+    const int f = (int)(t - p * cols);
+    const int64_t M = (int64_t)rows * cols;
+    const float* src = in + p * M + f;
+    ST* dst = W + (int64_t)(v0 + p) * M + f;
+    double sum = 0.0;
+    const int first = radius < rows - 1 ? radius : rows - 1;
+    for (int j = 0; j <= first; ++j) sum += (double)src[(int64_t)j * cols];
+    for (int i = 0; i < rows; ++i) {
+        if (i > 0) {
+            if (i + radius < rows) sum += (double)src[(int64_t)(i + radius) * cols];
+            if (i - radius - 1 >= 0) sum -= (double)src[(int64_t)(i - radius - 1) * cols];
+        }
+        const int64_t cell = (int64_t)i * cols + f;
+        if (reach[cell] > 0) {
+            const float w = (float)(sum / (double)den_b[cell]);
+            dst[(int64_t)i * cols] = (ST)w;
+        }
+    }
+}
+
+// [plane][a][b] -> [plane][b][a] through 32 x 32 shared-memory tiles
+template <typename T>
+__global__ void k_transpose(const T* __restrict__ in, T* __restrict__ out, int a, int b)
+{
+    __shared__ T tile[32][33];
+    const int64_t plane = blockIdx.z;
+    const T* src = in + plane * (int64_t)a * b;
+    T* dst = out + plane * (int64_t)a * b;
+    const int b0 = blockIdx.x * 32, a0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+        const int ia = a0 + j, ib = b0 + threadIdx.x;
+        if (ia < a && ib < b) tile[j][threadIdx.x] = src[(int64_t)ia * b + ib];
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+        const int ib = b0 + j, ia = a0 + threadIdx.x;
+        if (ia < a && ib < b) dst[(int64_t)ib * a + ia] = tile[threadIdx.x][j];
+    }
+}
+
+inline unsigned blocks_for(int64_t threads) { return (unsigned)((threads + UPD_THREADS - 1) / UPD_THREADS); }
+
+// three passes along the slow index, ping-ponging between x and y; returns where the result is
+template <typename T, typename ACC>
+T* three_passes(som_handle* h, T* x, T* y, int64_t planes, int len, int width, int radius, cudaStream_t st)
+{
+    for (int pass = 0; pass < 3; ++pass) {
+        k_box_pass<T, ACC><<<blocks_for(planes * width), UPD_THREADS, 0, st>>>(x, y, planes, len, width, radius);
+        h->launches += 1;
+        T* t = x; x = y; y = t;
+    }
+    return x;
+}
+
+template <typename T>
+void transpose(som_handle* h, const T* in, T* out, int64_t planes, int a, int b, cudaStream_t st)
+{
+    for (int64_t p0 = 0; p0 < planes; p0 += 65535) {
+        const int64_t np = planes - p0 < 65535 ? planes - p0 : 65535;
+        dim3 grid((unsigned)((b + 31) / 32), (unsigned)((a + 31) / 32), (unsigned)np);
+        k_transpose<T><<<grid, dim3(32, 8), 0, st>>>(in + p0 * (int64_t)a * b, out + p0 * (int64_t)a * b, a, b);
+        h->launches += 1;
+    }
+}
+
+}  // namespace
+
+size_t som_update_workspace_bytes(const som_handle* h, int64_t budget_bytes, int* planes_per_slab)
+{
+    const int64_t M = h->M;
+    int64_t planes = budget_bytes / (2 * M * 4);
+    if (planes < 1) planes = 1;
+    if (planes > h->V) planes = h->V;
+    *planes_per_slab = (int)planes;
+    // den (2 buffers), occupancy and reach (2 + 2 int buffers), then the two slab buffers
+    return som_align_up((size_t)M * 4, 256) * 6 + 2 * som_align_up((size_t)planes * M * 4, 256);
+}
+
+int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, const int32_t* indices,
+                      int64_t n, const int32_t* bmu, int radius, int planes_per_slab, cudaStream_t st)
+{
+    const int64_t M = h->M;
+    const size_t mb = som_align_up((size_t)M * 4, 256);
+    char* ws = reinterpret_cast<char*>(h->ws);
+    float* den_a = reinterpret_cast<float*>(ws);
+    float* den_b = reinterpret_cast<float*>(ws + mb);
+    int32_t* occ_a = reinterpret_cast<int32_t*>(ws + 2 * mb);
+    int32_t* occ_b = reinterpret_cast<int32_t*>(ws + 3 * mb);
+    int32_t* occ_c = reinterpret_cast<int32_t*>(ws + 4 * mb);
+    float* slab_a = reinterpret_cast<float*>(ws + 6 * mb);
+    float* slab_b = reinterpret_cast<float*>(ws + 6 * mb + som_align_up((size_t)planes_per_slab * M * 4, 256));
+
+    // ---- denominator and the exact reach of the blur --------------------------------------------
+    SOM_CK(h, cudaMemsetAsync(den_a, 0, (size_t)M * 4, st));
+    SOM_CK(h, cudaMemsetAsync(occ_a, 0, (size_t)M * 4, st));
+    if (n > 0) {
+        k_upd_count<<<blocks_for(n), UPD_THREADS, 0, st>>>(bmu, n, rows, cols, den_a, occ_a);
+        h->launches += 1;
+    }
+    float* d = three_passes<float, double>(h, den_a, den_b, 1, cols, rows, radius, st);  // along the lattice rows
+    float* d_other = (d == den_a) ? den_b : den_a;
+    transpose<float>(h, d, d_other, 1, cols, rows, st);
+    float* den_blurred = three_passes<float, double>(h, d_other, d, 1, rows, cols, radius, st);
+    // occupied cells within 3 * radius along each axis (exact integer counts; the count of a cell
+    // is at most M, so int32 suffices)
+    const int reach_r = 3 * radius;
+    k_box_pass<int32_t, int32_t><<<blocks_for(cols), UPD_THREADS, 0, st>>>(occ_a, occ_b, 1, rows, cols, reach_r);
+    transpose<int32_t>(h, occ_b, occ_c, 1, rows, cols, st);
+    k_box_pass<int32_t, int32_t><<<blocks_for(rows), UPD_THREADS, 0, st>>>(occ_c, occ_b, 1, cols, rows, reach_r);
+    transpose<int32_t>(h, occ_b, occ_c, 1, cols, rows, st);  // occ_c: reach count in neuron order
+    h->launches += 2;
+    SOM_CK(h, cudaGetLastError());
+
+    // ---- numerator, slab by slab ------------------------------------------------------------------
+    for (int v0 = 0; v0 < h->V; v0 += planes_per_slab) {
+        const int v1 = (v0 + planes_per_slab < h->V) ? v0 + planes_per_slab : h->V;
+        const int64_t planes = v1 - v0;
+        SOM_CK(h, cudaMemsetAsync(slab_a, 0, (size_t)planes * M * 4, st));
+        if (n > 0) {
+            k_upd_scatter<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols, slab_a);
+            h->launches += 1;
+        }
+        float* x = three_passes<float, double>(h, slab_a, slab_b, planes, cols, rows, radius, st);
+        float* y = (x == slab_a) ? slab_b : slab_a;
+        transpose<float>(h, x, y, planes, cols, rows, st);  // y: neuron order
+        for (int pass = 0; pass < 2; ++pass) {
+            k_box_pass<float, double><<<blocks_for(planes * cols), UPD_THREADS, 0, st>>>(y, x, planes, rows, cols, radius);
+            h->launches += 1;
+            float* t = x; x = y; y = t;
+        }
+        if (h->Wh)
+            k_box_pass_divide<__half><<<blocks_for(planes * cols), UPD_THREADS, 0, st>>>(
+                y, planes, rows, cols, radius, den_blurred, occ_c, const_cast<__half*>(h->Wh), v0);
+        else
+            k_box_pass_divide<float><<<blocks_for(planes * cols), UPD_THREADS, 0, st>>>(
+                y, planes, rows, cols, radius, den_blurred, occ_c, const_cast<float*>(h->W), v0);
+        h->launches += 1;
+        SOM_CK(h, cudaGetLastError());
+    }
+    return SOM_OK;
+}

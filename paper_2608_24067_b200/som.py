@@ -24,7 +24,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
-    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16",
+    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -61,6 +61,8 @@ def load_library():
     lib.som_bmu_host.argtypes = [P, P, P, I64, P, P, P]
     lib.som_bmu2.argtypes = [P, P, P, I64, P, P, P, P, P]
     lib.som_bmu2.restype = INT
+    lib.som_update.argtypes = [P, I32, I32, P, P, I64, P, I32, P]
+    lib.som_update.restype = INT
     lib.som_validate_csr.argtypes = [P, P, P, I64, P]
     lib.som_get_norms.argtypes = [P, P, P]
     lib.som_destroy.argtypes = [P]
@@ -172,6 +174,15 @@ class Som:
                                 _stream_ptr(stream))
         self._check(rc, "som_bmu2")
         return tuple(out)
+
+    def update(self, rows: int, cols: int, indptr: torch.Tensor, indices: torch.Tensor, bmu: torch.Tensor,
+               radius: int, stream=None):
+        """som_update: batch update of the borrowed codebook in place (call norms() afterwards)."""
+        n = indptr.numel() - 1
+        rc = self._lib.som_update(self._h, rows, cols, _dev_ptr(indptr, torch.int32, "indptr"),
+                                  _dev_ptr(indices, torch.int32, "indices"), n,
+                                  _dev_ptr(bmu, torch.int32, "bmu"), radius, _stream_ptr(stream))
+        self._check(rc, "som_update")
 
     def bmu_host(self, indptr: torch.Tensor, indices: torch.Tensor, out_bmu: torch.Tensor,
                  out_dist: torch.Tensor, stream=None):
