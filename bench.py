@@ -220,6 +220,8 @@ def run_ours(args, w: synth.Workload):
         h.set_option(3, args.lane_neurons)
     if args.parts:
         h.set_option(4, args.parts)
+    if args.update_mib:
+        h.set_option(6, args.update_mib)
     out_bmu = torch.empty(w.batch, dtype=torch.int32, device=dev)
     out_dist = torch.empty(w.batch, dtype=torch.float32, device=dev)
 
@@ -287,6 +289,29 @@ def run_ours(args, w: synth.Workload):
 
     clocks = sampler.close() if sampler else None
 
+    # ---- optional: the update phase of an epoch, timed on its own -----------------------------
+    update = None
+    edge = int(round(w.M ** 0.5))
+    if args.with_update and edge * edge == w.M:
+        b0 = batches[0]
+        h.norms()
+        bm, _ = h.bmu(b0.indptr, b0.indices)
+        radius = max(1, edge // 4)
+        h.update(edge, edge, b0.indptr, b0.indices, bm, radius)  # warm-up (allocates the workspace)
+        barrier()
+        u_steps = max(1, min(args.steps, 5))
+        e0.record()
+        for _ in range(u_steps):
+            h.update(edge, edge, b0.indptr, b0.indices, bm, radius)
+        e1.record()
+        barrier()
+        u_ms = max_over_ranks(e0.elapsed_time(e1) / u_steps, dist, dev)
+        u_bytes = w.V * w.M * store_bytes + b0.nnz * 4 + (b0.n + 1) * 4 + b0.n * 4  # write W, read CSR + bmu
+        update = {"ms": u_ms, "lattice": [edge, edge], "radius": radius, "algorithmic_bytes": u_bytes,
+                  "hbm_frac": u_bytes / (u_ms * 1e-3) / (hbm_gbs * 1e9),
+                  "share_of_epoch": u_ms / (u_ms + ms_per_step)}
+        h.norms()
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -348,6 +373,8 @@ def run_ours(args, w: synth.Workload):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if update is not None:
+        line["update"] = update
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -372,6 +399,10 @@ def main():
                     help="override the Zipf exponent of the feature popularity (0 = uniform)")
     ap.add_argument("--store", default="f32", choices=["f32", "f16"],
                     help="codebook storage: fp32 (the configurations) or fp16 with fp32 accumulation")
+    ap.add_argument("--with-update", action="store_true",
+                    help="also time som_update (the batch update that follows the search in an epoch) "
+                         "on a square lattice and report it under \"update\"")
+    ap.add_argument("--update-mib", type=int, default=0, help="som_update: workspace budget in MiB (library option 6)")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -221,7 +221,7 @@ int som_last_cuda_error(const som_handle* h);
  * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
  * feature instances that the row table's features must cover for the row-table kernel to be taken
  * (0 = default 50; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
- * slab buffers in MiB (0 = default 1024).
+ * slab buffers in MiB (0 = default 4096).
  */
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);

@@ -259,7 +259,7 @@ int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indpt
     DeviceGuard g(h->device);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int planes = 1;
-    const int64_t budget = (h->opt_update_mib > 0 ? h->opt_update_mib : 1024) << 20;
+    const int64_t budget = (h->opt_update_mib > 0 ? h->opt_update_mib : 4096) << 20;
     const size_t need = som_update_workspace_bytes(h, budget, &planes);
     int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need);
     if (rc) return rc;

@@ -44,7 +44,7 @@ struct som_handle {
     int64_t opt_r;         // neurons per lane of the row-table kernel: 0 = default, 4, 8 or 16
     int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
     int plan_attr_set;
-    int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 1024)
+    int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)
     int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 50)
     int32_t* host_pair;    // pinned, 3 ints: read-back of indptr[0], indptr[n], covered instances
 };

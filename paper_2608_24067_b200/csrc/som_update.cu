@@ -26,15 +26,37 @@ namespace {
 
 constexpr int UPD_THREADS = 256;
 
-__global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows, int cols,
+// Count of samples per cell into den_t (TRANSPOSED cell order) and the occupancy flags.  Small
+// lattices take a per-block histogram in shared memory first (a million samples on a few
+// thousand cells would otherwise queue on a handful of L2 atomic units); counts are exact in fp32.
+__global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows, int cols, int use_smem,
                             float* __restrict__ den_t, int32_t* __restrict__ occ)
 {
-    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= n) return;
-    const int c = bmu[s];
-    const int r = c / cols, q = c - r * cols;
-    atomicAdd(&den_t[(int64_t)q * rows + r], 1.0f);  // transposed cell order
-    occ[c] = 1;
+    extern __shared__ unsigned int hist[];
+    const int M = rows * cols;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    if (use_smem) {
+        for (int c = threadIdx.x; c < M; c += blockDim.x) hist[c] = 0u;
+        __syncthreads();
+        for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < n; s += stride)
+            atomicAdd(&hist[bmu[s]], 1u);
+        __syncthreads();
+        for (int c = threadIdx.x; c < M; c += blockDim.x) {
+            const unsigned int k = hist[c];
+            if (k) {
+                const int r = c / cols, q = c - r * cols;
+                atomicAdd(&den_t[(int64_t)q * rows + r], (float)k);
+                occ[c] = 1;
+            }
+        }
+    } else {
+        for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < n; s += stride) {
+            const int c = bmu[s];
+            const int r = c / cols, q = c - r * cols;
+            atomicAdd(&den_t[(int64_t)q * rows + r], 1.0f);
+            occ[c] = 1;
+        }
+    }
 }
 
 // one thread per sample: its features inside [v0, v1) add 1 to the cell of its best unit
@@ -46,7 +68,7 @@ __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t*
     if (s >= n) return;
     const int c = bmu[s];
     const int r = c / cols, q = c - r * cols;
-    const int64_t cell_t = (int64_t)q * rows + r;
+    const int64_t cell_t = (int64_t)q * rows + r;  // transposed cell order
     const int64_t M = (int64_t)rows * cols;
     const int beg = indptr[s], end = indptr[s + 1];
     for (int j = beg; j < end; ++j) {
@@ -81,12 +103,20 @@ __global__ void k_box_pass(const T* __restrict__ in, T* __restrict__ out, int64_
 }
 
 // The last pass, along the lattice columns of planes in neuron order, fused with the division
-// and the write of the new weights of features v0 + plane.  den_b is the blurred denominator
-// and reach the exact count of occupied cells within reach; where it is zero the prototype stays.
+// (a multiplication by the reciprocal of the blurred denominator, both in fp64) and the write of
+// the new weights of features v0 + plane.  A zero reciprocal marks a neuron out of every
+// sample's reach: its prototype stays.
+// 1 / blurred denominator in fp64 where the cell is within reach of a sample, else 0 (= keep)
+__global__ void k_upd_reciprocal(const float* __restrict__ den_b, const int32_t* __restrict__ reach, int64_t M,
+                                 double* __restrict__ rden)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < M) rden[i] = reach[i] > 0 ? 1.0 / (double)den_b[i] : 0.0;
+}
+
 template <typename ST>
 __global__ void k_box_pass_divide(const float* __restrict__ in, int64_t planes, int rows, int cols, int radius,
-                                  const float* __restrict__ den_b, const int32_t* __restrict__ reach,
-                                  ST* __restrict__ W, int v0)
+                                  const double* __restrict__ rden, ST* __restrict__ W, int v0)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= planes * cols) return;
@@ -103,11 +133,8 @@ __global__ void k_box_pass_divide(const float* __restrict__ in, int64_t planes, 
             if (i + radius < rows) sum += (double)src[(int64_t)(i + radius) * cols];
             if (i - radius - 1 >= 0) sum -= (double)src[(int64_t)(i - radius - 1) * cols];
         }
-        const int64_t cell = (int64_t)i * cols + f;
-        if (reach[cell] > 0) {
-            const float w = (float)(sum / (double)den_b[cell]);
-            dst[(int64_t)i * cols] = (ST)w;
-        }
+        const double rd = rden[(int64_t)i * cols + f];
+        if (rd != 0.0) dst[(int64_t)i * cols] = (ST)(float)(sum * rd);
     }
 }
 
@@ -165,8 +192,8 @@ size_t som_update_workspace_bytes(const som_handle* h, int64_t budget_bytes, int
     if (planes < 1) planes = 1;
     if (planes > h->V) planes = h->V;
     *planes_per_slab = (int)planes;
-    // den (2 buffers), occupancy and reach (2 + 2 int buffers), then the two slab buffers
-    return som_align_up((size_t)M * 4, 256) * 6 + 2 * som_align_up((size_t)planes * M * 4, 256);
+    // den (2 buffers), occupancy and reach (3 int buffers, 1 spare), reciprocal (fp64), then the two slab buffers
+    return som_align_up((size_t)M * 4, 256) * 8 + 2 * som_align_up((size_t)planes * M * 4, 256);
 }
 
 int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, const int32_t* indices,
@@ -180,14 +207,20 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
     int32_t* occ_a = reinterpret_cast<int32_t*>(ws + 2 * mb);
     int32_t* occ_b = reinterpret_cast<int32_t*>(ws + 3 * mb);
     int32_t* occ_c = reinterpret_cast<int32_t*>(ws + 4 * mb);
-    float* slab_a = reinterpret_cast<float*>(ws + 6 * mb);
-    float* slab_b = reinterpret_cast<float*>(ws + 6 * mb + som_align_up((size_t)planes_per_slab * M * 4, 256));
+    float* slab_a = reinterpret_cast<float*>(ws + 8 * mb);
+    float* slab_b = reinterpret_cast<float*>(ws + 8 * mb + som_align_up((size_t)planes_per_slab * M * 4, 256));
 
     // ---- denominator and the exact reach of the blur --------------------------------------------
     SOM_CK(h, cudaMemsetAsync(den_a, 0, (size_t)M * 4, st));
     SOM_CK(h, cudaMemsetAsync(occ_a, 0, (size_t)M * 4, st));
     if (n > 0) {
-        k_upd_count<<<blocks_for(n), UPD_THREADS, 0, st>>>(bmu, n, rows, cols, den_a, occ_a);
+        const int use_smem = M * 4 <= 96 * 1024;
+        if (use_smem) {
+            SOM_CK(h, cudaFuncSetAttribute(k_upd_count, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
+            k_upd_count<<<h->sm_count * 2, 1024, (size_t)M * 4, st>>>(bmu, n, rows, cols, 1, den_a, occ_a);
+        } else {
+            k_upd_count<<<h->sm_count * 8, UPD_THREADS, 0, st>>>(bmu, n, rows, cols, 0, den_a, occ_a);
+        }
         h->launches += 1;
     }
     float* d = three_passes<float, double>(h, den_a, den_b, 1, cols, rows, radius, st);  // along the lattice rows
@@ -201,7 +234,9 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
     transpose<int32_t>(h, occ_b, occ_c, 1, rows, cols, st);
     k_box_pass<int32_t, int32_t><<<blocks_for(rows), UPD_THREADS, 0, st>>>(occ_c, occ_b, 1, cols, rows, reach_r);
     transpose<int32_t>(h, occ_b, occ_c, 1, cols, rows, st);  // occ_c: reach count in neuron order
-    h->launches += 2;
+    double* rden = reinterpret_cast<double*>(ws + 6 * mb);
+    k_upd_reciprocal<<<blocks_for(M), UPD_THREADS, 0, st>>>(den_blurred, occ_c, M, rden);
+    h->launches += 3;
     SOM_CK(h, cudaGetLastError());
 
     // ---- numerator, slab by slab ------------------------------------------------------------------
@@ -223,10 +258,10 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         }
         if (h->Wh)
             k_box_pass_divide<__half><<<blocks_for(planes * cols), UPD_THREADS, 0, st>>>(
-                y, planes, rows, cols, radius, den_blurred, occ_c, const_cast<__half*>(h->Wh), v0);
+                y, planes, rows, cols, radius, rden, const_cast<__half*>(h->Wh), v0);
         else
             k_box_pass_divide<float><<<blocks_for(planes * cols), UPD_THREADS, 0, st>>>(
-                y, planes, rows, cols, radius, den_blurred, occ_c, const_cast<float*>(h->W), v0);
+                y, planes, rows, cols, radius, rden, const_cast<float*>(h->W), v0);
         h->launches += 1;
         SOM_CK(h, cudaGetLastError());
     }
