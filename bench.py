@@ -222,6 +222,8 @@ def run_ours(args, w: synth.Workload):
         h.set_option(4, args.parts)
     if args.update_mib:
         h.set_option(6, args.update_mib)
+    if args.two_stage:
+        h.set_option(7, 1)
     out_bmu = torch.empty(w.batch, dtype=torch.int32, device=dev)
     out_dist = torch.empty(w.batch, dtype=torch.float32, device=dev)
 
@@ -375,6 +377,8 @@ def run_ours(args, w: synth.Workload):
     }
     if update is not None:
         line["update"] = update
+    if args.two_stage:
+        line["two_stage"] = {"uncertain_samples_last_call": h.last_uncertain(), "batch": w.batch}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -403,6 +407,8 @@ def main():
                     help="also time som_update (the batch update that follows the search in an epoch) "
                          "on a square lattice and report it under \"update\"")
     ap.add_argument("--update-mib", type=int, default=0, help="som_update: workspace budget in MiB (library option 6)")
+    ap.add_argument("--two-stage", action="store_true",
+                    help="fp32 storage: certified first pass over an fp16 copy, exact second pass (library option 7)")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
     ap.add_argument("--no-cpu-baseline", action="store_true")

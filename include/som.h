@@ -221,11 +221,20 @@ int som_last_cuda_error(const som_handle* h);
  * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
  * feature instances that the row table's features must cover for the row-table kernel to be taken
  * (0 = default 50; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
- * slab buffers in MiB (0 = default 4096).
+ * slab buffers in MiB (0 = default 4096); key 7 = two-stage search for fp32 storage (0 = off, the default;
+ * 1 = on): som_norms then also keeps an fp16 copy of the codebook (V*M*2 more bytes of device memory,
+ * allocated by this call, which fails with SOM_ERR_CUDA if they cannot be had) and the largest |weight|;
+ * som_bmu ranks the neurons by a first pass over that copy, keeps the result for every sample whose two
+ * best first-pass scores are further apart than twice a bound on what the fp16 rounding and the fp32
+ * summation can change (then the best unit of the exact weights is provably the same one), and searches
+ * the other samples again with the fp32 weights.  Reported distances always come from the fp32 weights.
+ * Needs M % 128 == 0 and the row-table kernel; som_bmu2 never uses it.  som_last_uncertain returns how many
+ * samples the last two-stage search sent to its second pass.
  */
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);
 int64_t som_launch_count(const som_handle* h);
+int64_t som_last_uncertain(const som_handle* h);
 int som_set_option(som_handle* h, int key, int64_t value);
 
 #ifdef __cplusplus

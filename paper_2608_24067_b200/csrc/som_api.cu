@@ -112,6 +112,8 @@ int som_destroy(som_handle* h)
     cudaFree(h->ws);
     cudaFree(h->stage);
     cudaFree(h->head);
+    cudaFree(h->shadow);
+    cudaFree(h->wmax_bits);
     if (h->host_pair) cudaFreeHost(h->host_pair);
     if (h->events_made)
         for (int i = 0; i < SOM_N_EVENTS; ++i) cudaEventDestroy(h->ev[i]);
@@ -129,6 +131,7 @@ int som_norms(som_handle* h, void* stream)
     if (h->timing && (rc = ensure_events(h))) return rc;
     if ((rc = mark(h, h->ev_norms_calls, EV_NORMS_BEGIN, st))) return rc;
     if ((rc = som_launch_norms(h, st))) return rc;
+    h->shadow_valid = h->shadow != nullptr && h->M % 4 == 0;
     if ((rc = mark(h, h->ev_norms_calls, EV_NORMS_END, st))) return rc;
     if (h->timing) h->ev_norms_calls += 1;
     h->norms_valid = 1;
@@ -157,7 +160,14 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     // in automatic mode, batches whose most frequent features cover too few feature instances
     // for a shared-memory table to pay: there the direct-load kernel, bound by L2 bandwidth
     // alone, is faster (measured cross-over: about half of the instances).
-    const SomTableGeom geom = som_table_geometry(h);
+    // Two-stage search (option 7, fp32 storage): a first pass over the fp16 shadow of the
+    // codebook with the wide fp16 layout, a certificate per sample, an exact fp32 pass for the
+    // samples that fail it.  It needs the shadow written by the last som_norms and the row-table
+    // kernel; the two-best search does not use it (a certificate for the second unit would need
+    // the third).
+    const bool two_stage_ok = h->opt_two_stage == 1 && h->shadow && h->shadow_valid && !h->Wh && !top2 &&
+                              h->M % 128 == 0;
+    const SomTableGeom geom = som_table_geometry(h, two_stage_ok);
     bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
                      h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
@@ -205,12 +215,47 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (!begun && (rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
         SOM_CK(h, cudaMemsetAsync(keys, 0xFF, top2 ? 2 * key_bytes : key_bytes, st));
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, st))) return rc;
+        if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, nullptr, st))) return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-        if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, st)))
+        if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, nullptr, st)))
             return rc;
-        if (top2 && (rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys2, d_bmu2, d_dist2, st)))
+        if (top2 &&
+            (rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys2, d_bmu2, d_dist2, nullptr, st)))
             return rc;
+    } else if (two_stage_ok) {
+        const size_t need = som_plan_workspace_bytes(n_samples, nnz, &pb);
+        if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
+        char* ws = reinterpret_cast<char*>(h->ws);
+        const size_t kb = (size_t)(n_samples + 16) * sizeof(unsigned long long);
+        SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, kb, st));
+        SOM_CK(h, cudaMemsetAsync(ws + pb.keys2, 0xFF, kb, st));
+        if ((rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, head, ws, pb, SOM_PLAN_MASK_FEATURES,
+                                       geom.n_hot, st)))
+            return rc;
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+        // first pass: two best units by the fp16-rounded weights
+        if ((rc = som_launch_bmu_table(h, true, n_samples, head, ws, pb, geom.n_hot, true, st))) return rc;
+        // certificate; certain samples are finalised, the others listed
+        int32_t* uncertain = reinterpret_cast<int32_t*>(ws + pb.uncertain);
+        int* n_unc_dev = reinterpret_cast<int*>(head + pb.n_slots) + SOM_PLAN_UNCERTAIN;
+        if ((rc = som_launch_certify(h, d_indptr, d_indices, n_samples, ws, pb, d_bmu, d_min_dist, uncertain,
+                                     n_unc_dev, st)))
+            return rc;
+        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        SOM_CK(h, cudaStreamSynchronize(st));
+        const int64_t n_unc = h->host_pair[3];
+        h->last_uncertain = n_unc;
+        if (n_unc > 0) {
+            // exact pass over the listed samples: fp32 weights, all neurons
+            unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
+            SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, (size_t)n_unc * sizeof(unsigned long long), st));
+            if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_unc, ukeys, nullptr, uncertain, st))) return rc;
+            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+            if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_unc, ukeys, d_bmu, d_min_dist, uncertain, st)))
+                return rc;
+        } else if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) {
+            return rc;
+        }
     } else {
         const size_t need = som_plan_workspace_bytes(n_samples, nnz, &pb);
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
@@ -222,7 +267,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
                                        geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_table(h, n_samples, head, ws, pb, geom.n_hot, top2, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, false, n_samples, head, ws, pb, geom.n_hot, top2, st))) return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, false, d_bmu,
                                              d_min_dist, st)))
@@ -386,6 +431,8 @@ int som_get_timing(som_handle* h, float* out_ms, int n_out)
     return SOM_OK;
 }
 
+int64_t som_last_uncertain(const som_handle* h) { return h ? h->last_uncertain : 0; }
+
 int64_t som_launch_count(const som_handle* h) { return h ? h->launches : 0; }
 
 int som_set_option(som_handle* h, int key, int64_t value)
@@ -404,6 +451,19 @@ int som_set_option(som_handle* h, int key, int64_t value)
     if (key == 4) {
         if (value < 0 || value > 1024) return SOM_ERR_INVALID_ARG;
         h->opt_parts = value;
+        return SOM_OK;
+    }
+    if (key == 7) {
+        if (value != 0 && value != 1) return SOM_ERR_INVALID_ARG;
+        if (value == 1 && !h->shadow && !h->Wh) {
+            DeviceGuard g(h->device);
+            // the fp16 shadow of the codebook: half its size again in device memory
+            SOM_CK(h, cudaMalloc(reinterpret_cast<void**>(&h->shadow), (size_t)h->V * (size_t)h->M * sizeof(__half)));
+            SOM_CK(h, cudaMalloc(reinterpret_cast<void**>(&h->wmax_bits), 256));
+            h->shadow_valid = 0;
+            h->norms_valid = 0;  // the next som_norms writes the shadow
+        }
+        h->opt_two_stage = value;
         return SOM_OK;
     }
     if (key == 6) {

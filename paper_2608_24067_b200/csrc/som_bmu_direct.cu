@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(DIRECT_THREADS)
 k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
              const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
              unsigned long long* __restrict__ keys, unsigned long long* __restrict__ keys2,
-             int64_t neuron_off)
+             int64_t neuron_off, const int32_t* __restrict__ sample_list)
 {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -60,8 +60,10 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
     const int64_t s0 = ((int64_t)blockIdx.x * DIRECT_WARPS + warp) * DIRECT_SAMPLES_PER_WARP;
     const int64_t s1 = min(n, s0 + DIRECT_SAMPLES_PER_WARP);
     for (int64_t s = s0; s < s1; ++s) {
-        const int beg = indptr[s];
-        const int end = indptr[s + 1];
+        // with a sample list, position s of the list (and of the key arrays) is sample list[s]
+        const int64_t sid = sample_list ? (int64_t)sample_list[s] : s;
+        const int beg = indptr[sid];
+        const int end = indptr[sid + 1];
         float acc[VEC];
 #pragma unroll
         for (int k = 0; k < VEC; ++k) acc[k] = seed[k];
@@ -143,11 +145,13 @@ template <typename ST>
 __global__ void k_finalize(const ST* __restrict__ W, const double* __restrict__ norm64, int64_t M,
                            const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                            int64_t n, const unsigned long long* __restrict__ keys,
-                           int32_t* __restrict__ bmu, float* __restrict__ dist)
+                           int32_t* __restrict__ bmu, float* __restrict__ dist,
+                           const int32_t* __restrict__ sample_list)
 {
-    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= n) return;
-    const uint32_t idx = (uint32_t)(keys[s] & 0xffffffffull);
+    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n) return;
+    const int64_t s = sample_list ? (int64_t)sample_list[k] : k;
+    const uint32_t idx = (uint32_t)(keys[k] & 0xffffffffull);
     if (idx >= M) {  // only a second-best key can be empty: fewer than two neurons
         bmu[s] = -1;
         dist[s] = __int_as_float(0x7f800000);
@@ -183,7 +187,8 @@ __global__ void k_validate(const int32_t* __restrict__ indptr, const int32_t* __
 }  // namespace
 
 int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                          unsigned long long* keys, unsigned long long* keys2, cudaStream_t st)
+                          unsigned long long* keys, unsigned long long* keys2, const int32_t* sample_list,
+                          cudaStream_t st)
 {
     const int vec = (h->M % 4 == 0) ? 4 : 1;
     const int64_t per_block = (int64_t)DIRECT_WARPS * DIRECT_SAMPLES_PER_WARP;
@@ -198,7 +203,7 @@ int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* i
         const int64_t neuron_off = y0 * neurons_per_block;
 #define SOM_DIRECT(VEC_, TOP2_, ST_, W_)                                                          \
     k_bmu_direct<VEC_, TOP2_, ST_><<<grid, DIRECT_THREADS, 0, st>>>(W_, h->hnorm, h->M, indptr, indices, n, \
-                                                                    keys, keys2, neuron_off)
+                                                                    keys, keys2, neuron_off, sample_list)
         if (h->Wh) {
             if (vec == 4 && !keys2) SOM_DIRECT(4, false, __half, h->Wh);
             else if (vec == 4) SOM_DIRECT(4, true, __half, h->Wh);
@@ -218,15 +223,16 @@ int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* i
 }
 
 int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                        const unsigned long long* keys, int32_t* bmu, float* dist, cudaStream_t st)
+                        const unsigned long long* keys, int32_t* bmu, float* dist, const int32_t* sample_list,
+                        cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
     if (h->Wh)
         k_finalize<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, indptr, indices, n, keys,
-                                                             bmu, dist);
+                                                             bmu, dist, sample_list);
     else
         k_finalize<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, keys,
-                                                            bmu, dist);
+                                                            bmu, dist, sample_list);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

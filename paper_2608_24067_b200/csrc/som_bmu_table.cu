@@ -625,8 +625,8 @@ __global__ void k_finalize_sorted(const ST* __restrict__ W, const double* __rest
 }
 
 template <typename L, int THREADS, bool TOP2>
-int launch_table(som_handle* h, int64_t n_real, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
-                 size_t smem, cudaStream_t st)
+int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* head, char* ws,
+                 const SomPlanBuffers& b, int n_hot, size_t smem, cudaStream_t st)
 {
     constexpr int T = L::T;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
@@ -642,7 +642,7 @@ int launch_table(som_handle* h, int64_t n_real, char* head, char* ws, const SomP
     const int n_units = (int)n_units64;
     const int grid = n_units < h->sm_count ? n_units : h->sm_count;
     auto kern = k_bmu_table<L, THREADS, TOP2>;
-    const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(h->Wh ? (const void*)h->Wh : (const void*)h->W);
+    const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
     SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<grid, THREADS, smem, st>>>(codebook, h->hnorm, h->M,
                                       reinterpret_cast<const int32_t*>(head + b.slot_feat),
@@ -659,19 +659,20 @@ int launch_table(som_handle* h, int64_t n_real, char* head, char* ws, const SomP
 
 }  // namespace
 
-SomTableGeom som_table_geometry(const som_handle* h)
+SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
 {
+    const bool f16 = h->Wh != nullptr || shadow;  // the layout of the codebook this launch reads
     SomTableGeom g;
     // 8 neurons per lane (half as many rounds for the same work) whenever the neuron count is
     // a multiple of the 64-neuron range it needs; 640 threads leave it 96 registers, the
     // measured optimum between resident warps and spills
     // (an fp16-stored codebook has the 8-neuron layout only; som_table_usable checks M % 64)
-    g.R = (h->Wh || (h->opt_r != 4 && h->M % 64 == 0)) ? 8 : 4;
-    if (h->Wh && h->opt_r != 8 && h->M % 128 == 0) g.R = 16;  // wide fp16 layout wherever it divides M
+    g.R = (f16 || (h->opt_r != 4 && h->M % 64 == 0)) ? 8 : 4;
+    if (f16 && h->opt_r != 8 && h->M % 128 == 0) g.R = 16;  // wide fp16 layout wherever it divides M
     g.T = 8 * g.R;
-    const int row_bytes = g.T * (h->Wh ? 2 : 4);
+    const int row_bytes = g.T * (f16 ? 2 : 4);
     // (the fp16 layout holds half as many row registers: 896 threads at 72 registers measured best)
-    const int def_threads = h->Wh ? (g.R == 16 ? 512 : 896) : (g.R == 8 ? 640 : 1024);
+    const int def_threads = f16 ? (g.R == 16 ? 512 : 896) : (g.R == 8 ? 640 : 1024);
     g.threads = (h->opt_threads == 512 || h->opt_threads == 640 || h->opt_threads == 768 ||
                  h->opt_threads == 896 || h->opt_threads == 1024)
                     ? (int)h->opt_threads : def_threads;
@@ -679,7 +680,7 @@ SomTableGeom som_table_geometry(const som_handle* h)
     int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
     // Defaults keep dynamic + static shared memory under 196 KB: one step more and the SM's
     // carve-out leaves 28 KB instead of 60 KB of L1, which costs 12 % at 128x128 (measured).
-    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (row_bytes == 128 ? (h->Wh ? 1456 : 1376) : 720);
+    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (row_bytes == 128 ? (f16 ? 1456 : 1376) : 720);
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
     g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * row_bytes;  // + the zero row
@@ -687,17 +688,19 @@ SomTableGeom som_table_geometry(const som_handle* h)
 }
 
 template <bool TOP2>
-static int launch_table_any(som_handle* h, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
-                            int n_hot, cudaStream_t st)
+static int launch_table_any(som_handle* h, bool shadow, int64_t n, char* head, char* ws,
+                            const SomPlanBuffers& b, int n_hot, cudaStream_t st)
 {
-    const SomTableGeom g = som_table_geometry(h);
-#define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, TOP2>(h, n, head, ws, b, n_hot, g.smem, st)
-    if (h->Wh && g.R == 16) {
+    const SomTableGeom g = som_table_geometry(h, shadow);
+    const bool f16 = h->Wh != nullptr || shadow;
+    const void* cb = shadow ? (const void*)h->shadow : (h->Wh ? (const void*)h->Wh : (const void*)h->W);
+#define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, TOP2>(h, cb, n, head, ws, b, n_hot, g.smem, st)
+    if (f16 && g.R == 16) {
         if (g.threads == 768) SOM_TABLE(LayF16W, 768);
         if (g.threads == 640) SOM_TABLE(LayF16W, 640);
         SOM_TABLE(LayF16W, 512);
     }
-    if (h->Wh) {
+    if (f16) {
         if (g.threads == 1024) SOM_TABLE(LayF16, 1024);
         if (g.threads == 896) SOM_TABLE(LayF16, 896);
         if (g.threads == 768) SOM_TABLE(LayF16, 768);
@@ -719,11 +722,72 @@ static int launch_table_any(som_handle* h, int64_t n, char* head, char* ws, cons
 #undef SOM_TABLE
 }
 
-int som_launch_bmu_table(som_handle* h, int64_t n, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
-                         bool top2, cudaStream_t st)
+int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
+                         int n_hot, bool top2, cudaStream_t st)
 {
-    return top2 ? launch_table_any<true>(h, n, head, ws, b, n_hot, st)
-                : launch_table_any<false>(h, n, head, ws, b, n_hot, st);
+    return top2 ? launch_table_any<true>(h, shadow, n, head, ws, b, n_hot, st)
+                : launch_table_any<false>(h, shadow, n, head, ws, b, n_hot, st);
+}
+
+// ---- two-stage search: certification of the first pass ----------------------------------------
+// The first pass ranked the neurons by fp32 sums of the fp16-rounded weights.  For a sample with
+// k active features every such score differs from the fp32 score of the exact weights by at most
+//   eps = k * wmax * 2^-11  (rounding of each weight to fp16, round to nearest)
+//       + 2 * (k + 2) * 2^-24 * B  (fp32 summation, either path; B bounds every partial sum),
+// so when the two best first-pass scores are more than 2 * eps apart the best unit of the exact
+// weights is the first pass's best unit.  Such samples are finalised here (distance recomputed in
+// fp64 from the fp32 weights, as always); the others are listed for an exact fp32 search.
+namespace {
+__device__ __forceinline__ float score_of_key(u64 key)
+{
+    const uint32_t cu = (uint32_t)(key >> 32);
+    return __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
+}
+
+__global__ void k_certify(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
+                          const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
+                          const uint4* __restrict__ slots, const u64* __restrict__ keys,
+                          const u64* __restrict__ keys2, const unsigned int* __restrict__ wmax_bits,
+                          int32_t* __restrict__ bmu, float* __restrict__ dist,
+                          int32_t* __restrict__ uncertain, int* __restrict__ n_uncertain)
+{
+    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n) return;
+    const uint32_t s = slots[k * SLOT_Q].y;
+    const u64 k1 = keys[k], k2 = keys2[k];
+    const int beg = indptr[s];
+    const int end = indptr[s + 1];
+    const float wmax = __uint_as_float(*wmax_bits);
+    const float s1 = score_of_key(k1), s2 = score_of_key(k2);
+    const float cnt = (float)(end - beg);
+    const float bound = fmaxf(fabsf(s1), fabsf(s2)) + 2.f * cnt * wmax;
+    const float eps = cnt * wmax * 4.8828125e-4f * 1.0001f + 2.f * (cnt + 2.f) * 5.9604645e-8f * bound;
+    const bool certain = (s2 - s1) > 2.f * eps;  // false for NaN or an empty second key
+    if (!certain) {
+        uncertain[atomicAdd(n_uncertain, 1)] = (int32_t)s;
+        return;
+    }
+    const uint32_t idx = (uint32_t)(k1 & 0xffffffffull);
+    double dot = 0.0;
+    for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
+    bmu[s] = (int32_t)idx;
+    dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
+}
+}  // namespace
+
+int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
+                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* uncertain,
+                       int* n_uncertain, cudaStream_t st)
+{
+    const int64_t blocks = (n + 255) / 256;
+    k_certify<<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n,
+                                                reinterpret_cast<const uint4*>(ws + b.slots),
+                                                reinterpret_cast<const u64*>(ws + b.keys),
+                                                reinterpret_cast<const u64*>(ws + b.keys2), h->wmax_bits, bmu,
+                                                dist, uncertain, n_uncertain);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
+    return SOM_OK;
 }
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,

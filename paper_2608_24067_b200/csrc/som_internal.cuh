@@ -18,6 +18,10 @@ struct som_handle {
     int64_t M;
     const float* W;    // borrowed, feature-major fp32 codebook (nullptr when stored as fp16)
     const __half* Wh;  // borrowed, feature-major fp16 codebook (som_create_f16), else nullptr
+    __half* shadow;    // owned fp16 copy of an fp32 codebook for the two-stage search (nullptr = none)
+    unsigned int* wmax_bits;  // device: float bits of max |weight|, written by som_norms with the shadow
+    int shadow_valid;         // the last som_norms wrote the shadow
+    int64_t last_uncertain;   // samples the last two-stage search sent to its exact pass
 
     double* norm64;  // [M] ||w_i||^2 in fp64
     float* norm32;   // [M] the same rounded to fp32
@@ -45,8 +49,9 @@ struct som_handle {
     int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
     int plan_attr_set;
     int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)
+    int64_t opt_two_stage;  // 0 = off, 1 = on where it applies (fp32 storage, M % 128 == 0, memory for the shadow)
     int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 50)
-    int32_t* host_pair;    // pinned, 3 ints: read-back of indptr[0], indptr[n], covered instances
+    int32_t* host_pair;    // pinned, 4 ints: read-back of indptr[0], indptr[n], covered instances, uncertain samples
 };
 
 // event slots
@@ -84,9 +89,11 @@ __device__ __forceinline__ float som_weight(const __half* p) { return __half2flo
 // kernels' host launchers (each returns a som_status)
 int som_launch_norms(som_handle* h, cudaStream_t st);
 int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                          unsigned long long* keys, unsigned long long* keys2, cudaStream_t st);
+                          unsigned long long* keys, unsigned long long* keys2, const int32_t* sample_list,
+                          cudaStream_t st);
 int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
-                        const unsigned long long* keys, int32_t* bmu, float* dist, cudaStream_t st);
+                        const unsigned long long* keys, int32_t* bmu, float* dist, const int32_t* sample_list,
+                        cudaStream_t st);
 int som_launch_validate(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                         int* d_flag, cudaStream_t st);
 size_t som_norms_workspace_bytes(const som_handle* h);

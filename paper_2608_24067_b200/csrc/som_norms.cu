@@ -12,10 +12,24 @@ namespace {
 constexpr int NORM_THREADS = 128;
 constexpr int NORM_UNROLL = 8;
 
-template <int VEC>
+// four floats -> four halves (round to nearest even), one 64-bit store
+__device__ __forceinline__ void store_half4(__half* dst, const float4 w)
+{
+    const __half2 a = __floats2half2_rn(w.x, w.y);
+    const __half2 b = __floats2half2_rn(w.z, w.w);
+    uint2 v;
+    v.x = *reinterpret_cast<const uint32_t*>(&a);
+    v.y = *reinterpret_cast<const uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(dst) = v;
+}
+
+// SHADOW (VEC == 4 only): the pass also writes an fp16 copy of the codebook and the largest
+// |weight| (as float bits, through atomicMax: non-negative floats order like their bits), which
+// the two-stage search uses for its first pass and its error bound.
+template <int VEC, bool SHADOW>
 __global__ void __launch_bounds__(NORM_THREADS)
 k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_split,
-                double* __restrict__ partial)
+                double* __restrict__ partial, __half* __restrict__ shadow, unsigned int* __restrict__ wmax_bits)
 {
     const int64_t i = ((int64_t)blockIdx.x * NORM_THREADS + threadIdx.x) * VEC;
     if (i >= M) return;
@@ -25,6 +39,8 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
 #pragma unroll
     for (int k = 0; k < VEC; ++k) acc[k] = 0.0;
     const float* p = W + (int64_t)v0 * M + i;
+    __half* ps = SHADOW ? shadow + (int64_t)v0 * M + i : nullptr;
+    float wmax = 0.f;
     int v = v0;
     if (VEC == 4) {
         for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
@@ -34,15 +50,25 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
                 w[u] = __ldcs(reinterpret_cast<const float4*>(p + (int64_t)u * M));
 #pragma unroll
             for (int u = 0; u < NORM_UNROLL; ++u) {
+                if (SHADOW) {
+                    store_half4(ps + (int64_t)u * M, w[u]);
+                    wmax = fmaxf(wmax, fmaxf(fmaxf(fabsf(w[u].x), fabsf(w[u].y)), fmaxf(fabsf(w[u].z), fabsf(w[u].w))));
+                }
                 acc[0] = fma((double)w[u].x, (double)w[u].x, acc[0]);
                 acc[1 % VEC] = fma((double)w[u].y, (double)w[u].y, acc[1 % VEC]);
                 acc[2 % VEC] = fma((double)w[u].z, (double)w[u].z, acc[2 % VEC]);
                 acc[3 % VEC] = fma((double)w[u].w, (double)w[u].w, acc[3 % VEC]);
             }
             p += (int64_t)NORM_UNROLL * M;
+            if (SHADOW) ps += (int64_t)NORM_UNROLL * M;
         }
         for (; v < v1; ++v) {
             float4 w = __ldcs(reinterpret_cast<const float4*>(p));
+            if (SHADOW) {
+                store_half4(ps, w);
+                wmax = fmaxf(wmax, fmaxf(fmaxf(fabsf(w.x), fabsf(w.y)), fmaxf(fabsf(w.z), fabsf(w.w))));
+                ps += M;
+            }
             acc[0] = fma((double)w.x, (double)w.x, acc[0]);
             acc[1 % VEC] = fma((double)w.y, (double)w.y, acc[1 % VEC]);
             acc[2 % VEC] = fma((double)w.z, (double)w.z, acc[2 % VEC]);
@@ -59,6 +85,13 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
     double* out = partial + (int64_t)blockIdx.y * M + i;
 #pragma unroll
     for (int k = 0; k < VEC; ++k) out[k] = acc[k];
+    if (SHADOW) {
+        // one atomic per warp (lanes past the last neuron have left: reduce over the active ones);
+        // NaN weights are outside the preconditions, fmaxf drops them
+        const unsigned int active = __activemask();
+        const unsigned int best = __reduce_max_sync(active, __float_as_uint(wmax));
+        if ((threadIdx.x & 31) == (__ffs(active) - 1)) atomicMax(wmax_bits, best);
+    }
 }
 
 // The same pass over an fp16-stored codebook: VEC = 8 neurons per thread (one 128-bit load of
@@ -172,10 +205,16 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
         k_norms_partial_h<8><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
     else if (h->Wh)
         k_norms_partial_h<1><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
-    else if (p.vec == 4)
-        k_norms_partial<4><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial);
+    else if (p.vec == 4 && h->shadow) {
+        SOM_CK(h, cudaMemsetAsync(h->wmax_bits, 0, sizeof(unsigned int), st));
+        k_norms_partial<4, true><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                h->shadow, h->wmax_bits);
+    } else if (p.vec == 4)
+        k_norms_partial<4, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                 nullptr, nullptr);
     else
-        k_norms_partial<1><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial);
+        k_norms_partial<1, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                 nullptr, nullptr);
     SOM_CK(h, cudaGetLastError());
     const int64_t blocks = (h->M + 255) / 256;
     k_norms_combine<<<(unsigned)blocks, 256, 0, st>>>(partial, h->M, p.splits, h->norm64, h->norm32,

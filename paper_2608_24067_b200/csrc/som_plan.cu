@@ -392,6 +392,8 @@ size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b)
     b->block_sums = take((size_t)(SOM_PLAN_BINS / SCAN_BLOCK + 2) * 4);
     b->slots = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
     b->overflow = take((size_t)(nnz + 6 * n + 4) * 4);
+    b->uncertain = take((size_t)n * 4);
+    b->ukeys = take((size_t)n * 8);
     return off;
 }
 

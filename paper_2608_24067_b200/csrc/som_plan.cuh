@@ -41,7 +41,7 @@ struct SomPlanBuffers {
     size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
     size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
     size_t n_slots;     // i32 [8]      mask slots used, hot slots used, overflow cursor, search unit
-                        //              counter, feature instances covered by the table
+                        //              counter, feature instances covered by the table, uncertain samples
     // workspace
     size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
     size_t keys2;       // u64 [n]      the same for the second-best unit (two-best search only)
@@ -52,9 +52,12 @@ struct SomPlanBuffers {
     size_t block_sums;  // u32 [scan blocks]
     size_t slots;       // 48 B [n + 16]
     size_t overflow;    // u32 [nnz + 6n]
+    size_t uncertain;   // i32 [n]      samples the two-stage search sends to its exact pass
+    size_t ukeys;       // u64 [n]      their packed keys, by position in that list
 };
 #define SOM_PLAN_N_SLOTS_INTS 8
 #define SOM_PLAN_COVERED 4 /* index into n_slots */
+#define SOM_PLAN_UNCERTAIN 5 /* index into n_slots: length of the two-stage search's uncertain list */
 
 // Sample parts per neuron range of the row-table kernel.  More parts mean fewer ranges live at
 // once (their slabs must share L2 with the slot stream) but smaller units, each of which
@@ -81,8 +84,13 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
                          char* head, char* ws, const SomPlanBuffers& b, int n_mask, int n_hot,
                          cudaStream_t st);
 
-int som_launch_bmu_table(som_handle* h, int64_t n, char* head, char* ws, const SomPlanBuffers& b, int n_hot,
-                         bool top2, cudaStream_t st);
+// shadow = read the handle's fp16 shadow of an fp32 codebook (first pass of the two-stage search)
+int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
+                         int n_hot, bool top2, cudaStream_t st);
+
+int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
+                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* uncertain,
+                       int* n_uncertain, cudaStream_t st);
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                                char* ws, const SomPlanBuffers& b, bool second, int32_t* bmu, float* dist,
@@ -96,4 +104,4 @@ struct SomTableGeom {
     int threads;  // block size
     size_t smem;  // dynamic shared memory bytes
 };
-SomTableGeom som_table_geometry(const som_handle* h);
+SomTableGeom som_table_geometry(const som_handle* h, bool shadow = false);

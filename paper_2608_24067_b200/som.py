@@ -24,7 +24,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
-    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update",
+    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -73,6 +73,8 @@ def load_library():
     lib.som_get_timing.argtypes = [P, P, INT]
     lib.som_launch_count.argtypes = [P]
     lib.som_launch_count.restype = I64
+    lib.som_last_uncertain.argtypes = [P]
+    lib.som_last_uncertain.restype = I64
     lib.som_set_option.argtypes = [P, INT, I64]
     lib.som_norms_noalloc.argtypes = [I32, I64, P, P, P]
     lib.som_norms_noalloc.restype = INT
@@ -221,6 +223,9 @@ class Som:
 
     def launch_count(self) -> int:
         return int(self._lib.som_launch_count(self._h))
+
+    def last_uncertain(self) -> int:
+        return int(self._lib.som_last_uncertain(self._h))
 
     def set_option(self, key: int, value: int):
         self._check(self._lib.som_set_option(self._h, key, value), "som_set_option")

@@ -170,6 +170,9 @@ def test_f16_largest_map_full_size_sampled_rows(som_mod):
     uses, through som_bmu2; a strided sample of rows is checked against the oracle, which reads
     the device codebook slab by slab, and range properties are checked for every row."""
     w = synth.CONFIGS[4]
+    import gc
+    gc.collect()  # handles and tensors of earlier tests
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     need = w.V * w.M * 2 + (6 << 30)
     if free < need:

@@ -300,6 +300,9 @@ def test_large_configs_full_size_sampled_rows(som_mod, cfg, n_rows):
     the benchmark uses; a strided sample of rows is checked against the oracle, which reads the
     device codebook slab by slab, and range / finiteness properties are checked for every row."""
     w = synth.CONFIGS[cfg]
+    import gc
+    gc.collect()  # handles and tensors of earlier tests
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     need = w.V * w.M * 4 + (6 << 30)
     if free < need:

@@ -1,0 +1,114 @@
+"""GPU parity tests of the two-stage search (option 7): certified first pass over an fp16 copy of
+an fp32 codebook, exact fp32 second pass for the uncertain samples.  The result must satisfy the
+same parity rule as the plain fp32 search, and certified samples must have the plain search's unit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import parity
+from oracle import som_oracle as orc
+from paper_2608_24067_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def som_mod():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_24067_b200 import som
+    som.load_library()  # fail loudly when the extension is missing
+    return som
+
+
+def _subset(indptr, indices, rows):
+    indptr = np.asarray(indptr, dtype=np.int64)
+    lens = indptr[rows + 1] - indptr[rows]
+    out_ptr = np.zeros(len(rows) + 1, np.int32)
+    out_ptr[1:] = np.cumsum(lens)
+    out_idx = np.concatenate([indices[indptr[r]:indptr[r + 1]] for r in rows]).astype(np.int32)
+    return out_ptr, out_idx
+
+
+def _run(som_mod, W, V, M, b, two_stage, variant=2):
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, variant)
+    if two_stage:
+        h.set_option(7, 1)
+    h.norms()
+    bmu, dist = h.bmu(b.indptr, b.indices)
+    again = h.bmu(b.indptr, b.indices)
+    torch.cuda.synchronize()
+    assert torch.equal(bmu, again[0]) and torch.equal(dist.view(torch.int32), again[1].view(torch.int32))
+    return h, bmu.cpu().numpy(), dist.cpu().numpy()
+
+
+def _check(W_host, V, M, b, g_bmu, g_dist, rows):
+    ip, ix = _subset(b.indptr.cpu().numpy(), b.indices.cpu().numpy(), rows)
+    nn = orc.norms(W_host, V, M)
+    top2 = orc.bmu(W_host, V, M, ip, ix, norms_=nn)
+    d_at = orc.dist_at(W_host, V, M, ip, ix, np.clip(g_bmu[rows].astype(np.int64), 0, M - 1), norms_=nn)
+    rep = parity.check(g_bmu[rows], g_dist[rows], top2, d_at, M)
+    assert rep.ok, str(rep)
+    return rep
+
+
+@pytest.mark.parametrize("scale", [1.0, 37.0, 1.0 / 64.0])
+def test_two_stage_matches_oracle_and_plain_search(som_mod, scale):
+    """The error bound scales with the largest weight, so the certificate must hold for scaled codebooks."""
+    V, M, n = 30_000, 1_024, 80_000
+    W = synth.fill_codebook(V, M, 5, device="cuda") * scale
+    b = synth.sample_csr(n, V, 11.0, 5, device="cuda")
+    h2, bmu2, dist2 = _run(som_mod, W, V, M, b, True)
+    h1, bmu1, dist1 = _run(som_mod, W, V, M, b, False)
+    unc = h2.last_uncertain()
+    assert 0 < unc < n // 2  # most samples are certified, some are not
+    differ = np.flatnonzero(bmu1 != bmu2)
+    assert differ.size <= unc  # only samples of the exact pass can differ (near ties, other summation order)
+    same = bmu1 == bmu2
+    assert np.array_equal(dist1[same].view(np.uint32), dist2[same].view(np.uint32))
+    rows = np.unique(np.concatenate([np.arange(0, n, 9), differ]))
+    _check(W.cpu().numpy(), V, M, b, bmu2, dist2, rows)
+
+
+def test_two_stage_config2_sampled_rows(som_mod):
+    w = synth.CONFIGS[1]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(w.N, w.V, w.lam, w.seed, device="cuda")
+    h, bmu, dist = _run(som_mod, W, w.V, w.M, b, True, variant=0)
+    assert 0 < h.last_uncertain() < w.N // 4
+    rows = np.concatenate([np.arange(0, w.N, 40), [w.N - 1]])
+    _check(W.cpu().numpy(), w.V, w.M, b, bmu, dist, rows)
+
+
+def test_two_stage_with_duplicate_neurons_sends_everything_to_the_exact_pass(som_mod):
+    """Two identical halves of the map: every best unit has an exact twin, no sample can be certified,
+    and the lowest index must win."""
+    V, half, n = 2_000, 1_024, 40_000
+    Wh = synth.fill_codebook(V, half, 2, device="cuda").view(V, half)
+    W = torch.cat([Wh, Wh], dim=1).contiguous().view(-1)
+    M = 2 * half
+    b = synth.sample_csr(n, V, 7.0, 2, device="cuda")
+    h, bmu, dist = _run(som_mod, W, V, M, b, True)
+    assert h.last_uncertain() == n
+    assert bmu.max() < half
+    _check(W.cpu().numpy(), V, M, b, bmu, dist, np.arange(0, n, 11))
+
+
+def test_two_stage_needs_its_shadow_from_norms(som_mod):
+    """Switching the option on invalidates the norms: the next som_norms has to write the copy."""
+    V, M, n = 2_000, 1_024, 30_000
+    W = synth.fill_codebook(V, M, 1, device="cuda")
+    b = synth.sample_csr(n, V, 7.0, 1, device="cuda")
+    h = som_mod.Som(V, M, W)
+    h.norms()
+    h.set_option(7, 1)
+    with pytest.raises(som_mod.SomError):
+        h.bmu(b.indptr, b.indices)
+    h.norms()
+    # after an in-place change of the codebook the copy follows at the next som_norms
+    W.mul_(0.5)
+    h.norms()
+    bmu, dist = h.bmu(b.indptr, b.indices)
+    torch.cuda.synchronize()
+    _check(W.cpu().numpy(), V, M, b, bmu.cpu().numpy(), dist.cpu().numpy(), np.arange(0, n, 13))
