@@ -246,13 +246,33 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         const int64_t n_unc = h->host_pair[3];
         h->last_uncertain = n_unc;
         if (n_unc > 0) {
-            // exact pass over the listed samples: fp32 weights, all neurons
+            // exact pass over the listed samples: fp32 weights, all neurons.  With enough of
+            // them the row-table kernel runs again on their compacted slots (same plan: both
+            // layouts hold the same number of hot rows), else the direct-load kernel.
             unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
-            SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, (size_t)n_unc * sizeof(unsigned long long), st));
-            if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_unc, ukeys, nullptr, uncertain, st))) return rc;
-            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-            if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_unc, ukeys, d_bmu, d_min_dist, uncertain, st)))
-                return rc;
+            const SomTableGeom exact = som_table_geometry(h, false);
+            const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T);
+            if (exact.n_hot == geom.n_hot && units >= 2 * (int64_t)h->sm_count) {
+                SomPlanBuffers pe = pb;
+                pe.slots = pb.slots2;
+                pe.keys = pb.ukeys;
+                SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, (size_t)(n_unc + 16) * sizeof(unsigned long long), st));
+                SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(head + pb.n_slots) + 3, 0, sizeof(int), st));
+                if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_unc, st))) return rc;
+                if ((rc = som_launch_bmu_table(h, false, n_unc, head, ws, pe, exact.n_hot, false, st))) return rc;
+                if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+                if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_unc, ws, pe, false, d_bmu,
+                                                     d_min_dist, st)))
+                    return rc;
+            } else {
+                SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, (size_t)n_unc * sizeof(unsigned long long), st));
+                if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_unc, ukeys, nullptr, uncertain, st)))
+                    return rc;
+                if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+                if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_unc, ukeys, d_bmu, d_min_dist, uncertain,
+                                              st)))
+                    return rc;
+            }
         } else if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) {
             return rc;
         }

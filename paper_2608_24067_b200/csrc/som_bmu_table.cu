@@ -749,29 +749,53 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
                           const uint4* __restrict__ slots, const u64* __restrict__ keys,
                           const u64* __restrict__ keys2, const unsigned int* __restrict__ wmax_bits,
                           int32_t* __restrict__ bmu, float* __restrict__ dist,
-                          int32_t* __restrict__ uncertain, int* __restrict__ n_uncertain)
+                          int32_t* __restrict__ uncertain, uint4* __restrict__ slots2,
+                          int* __restrict__ n_uncertain)
 {
+    __shared__ int warp_count[8];
+    __shared__ int block_base;
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= n) return;
-    const uint32_t s = slots[k * SLOT_Q].y;
-    const u64 k1 = keys[k], k2 = keys2[k];
-    const int beg = indptr[s];
-    const int end = indptr[s + 1];
-    const float wmax = __uint_as_float(*wmax_bits);
-    const float s1 = score_of_key(k1), s2 = score_of_key(k2);
-    const float cnt = (float)(end - beg);
-    const float bound = fmaxf(fabsf(s1), fabsf(s2)) + 2.f * cnt * wmax;
-    const float eps = cnt * wmax * 4.8828125e-4f * 1.0001f + 2.f * (cnt + 2.f) * 5.9604645e-8f * bound;
-    const bool certain = (s2 - s1) > 2.f * eps;  // false for NaN or an empty second key
-    if (!certain) {
-        uncertain[atomicAdd(n_uncertain, 1)] = (int32_t)s;
-        return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    bool flag = false;
+    uint32_t s = 0;
+    if (k < n) {
+        s = slots[k * SLOT_Q].y;
+        const u64 k1 = keys[k], k2 = keys2[k];
+        const int beg = indptr[s];
+        const int end = indptr[s + 1];
+        const float wmax = __uint_as_float(*wmax_bits);
+        const float s1 = score_of_key(k1), s2 = score_of_key(k2);
+        const float cnt = (float)(end - beg);
+        const float bound = fmaxf(fabsf(s1), fabsf(s2)) + 2.f * cnt * wmax;
+        const float eps = cnt * wmax * 4.8828125e-4f * 1.0001f + 2.f * (cnt + 2.f) * 5.9604645e-8f * bound;
+        const bool certain = (s2 - s1) > 2.f * eps;  // false for NaN or an empty second key
+        flag = !certain;
+        if (certain) {
+            const uint32_t idx = (uint32_t)(k1 & 0xffffffffull);
+            double dot = 0.0;
+            for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
+            bmu[s] = (int32_t)idx;
+            dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
+        }
     }
-    const uint32_t idx = (uint32_t)(k1 & 0xffffffffull);
-    double dot = 0.0;
-    for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
-    bmu[s] = (int32_t)idx;
-    dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
+    // The uncertain samples of a block keep their (mask-sorted) order: their ids and their
+    // slots are compacted to one contiguous run of the lists, so that the exact pass can run
+    // the row-table kernel on the same plan.
+    const unsigned int votes = __ballot_sync(0xffffffffu, flag);
+    if (lane == 0) warp_count[warp] = __popc(votes);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int total = 0;
+        for (int w = 0; w < 8; ++w) { const int c = warp_count[w]; warp_count[w] = total; total += c; }
+        block_base = total ? atomicAdd(n_uncertain, total) : 0;
+    }
+    __syncthreads();
+    if (flag) {
+        const int pos = block_base + warp_count[warp] + __popc(votes & ((1u << lane) - 1u));
+        uncertain[pos] = (int32_t)s;
+#pragma unroll
+        for (int x = 0; x < SLOT_Q; ++x) slots2[(int64_t)pos * SLOT_Q + x] = slots[k * SLOT_Q + x];
+    }
 }
 }  // namespace
 
@@ -784,7 +808,8 @@ int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indi
                                                 reinterpret_cast<const uint4*>(ws + b.slots),
                                                 reinterpret_cast<const u64*>(ws + b.keys),
                                                 reinterpret_cast<const u64*>(ws + b.keys2), h->wmax_bits, bmu,
-                                                dist, uncertain, n_uncertain);
+                                                dist, uncertain, reinterpret_cast<uint4*>(ws + b.slots2),
+                                                n_uncertain);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

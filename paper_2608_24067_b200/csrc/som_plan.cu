@@ -393,8 +393,20 @@ size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b)
     b->slots = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
     b->overflow = take((size_t)(nnz + 6 * n + 4) * 4);
     b->uncertain = take((size_t)n * 4);
-    b->ukeys = take((size_t)n * 8);
+    b->ukeys = take((size_t)(n + 16) * 8);
+    b->slots2 = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
     return off;
+}
+
+int som_launch_pad_slots(som_handle* h, char* ws, size_t slots_offset, int64_t n, cudaStream_t st)
+{
+    const int64_t n_pad = (n + 3) / 4 * 4;
+    if (n_pad > n && n > 0) {
+        k_pad_slots<<<1, 32, 0, st>>>(reinterpret_cast<uint4*>(ws + slots_offset), n, n_pad);
+        SOM_CK(h, cudaGetLastError());
+        h->launches += 1;
+    }
+    return SOM_OK;
 }
 
 int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,

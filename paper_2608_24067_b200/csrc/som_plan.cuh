@@ -53,7 +53,8 @@ struct SomPlanBuffers {
     size_t slots;       // 48 B [n + 16]
     size_t overflow;    // u32 [nnz + 6n]
     size_t uncertain;   // i32 [n]      samples the two-stage search sends to its exact pass
-    size_t ukeys;       // u64 [n]      their packed keys, by position in that list
+    size_t ukeys;       // u64 [n + 16] their packed keys, by position in that list
+    size_t slots2;      // 48 B [n + 16] their slots, compacted in list order
 };
 #define SOM_PLAN_N_SLOTS_INTS 8
 #define SOM_PLAN_COVERED 4 /* index into n_slots */
@@ -87,6 +88,9 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
 // shadow = read the handle's fp16 shadow of an fp32 codebook (first pass of the two-stage search)
 int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
                          int n_hot, bool top2, cudaStream_t st);
+
+// pads a slot array of n slots to a multiple of four with copies of the last one
+int som_launch_pad_slots(som_handle* h, char* ws, size_t slots_offset, int64_t n, cudaStream_t st);
 
 int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
                        const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* uncertain,
