@@ -732,7 +732,8 @@ int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char
 // ---- two-stage search: certification of the first pass ----------------------------------------
 // The first pass ranked the neurons by fp32 sums of the fp16-rounded weights.  For a sample with
 // k active features every such score differs from the fp32 score of the exact weights by at most
-//   eps = k * wmax * 2^-11  (rounding of each weight to fp16, round to nearest)
+//   eps = k * max(wmax * 2^-11, 2^-25)  (rounding of each weight to fp16, round to nearest;
+//                                        the second term covers fp16's subnormal range)
 //       + 2 * (k + 2) * 2^-24 * B  (fp32 summation, either path; B bounds every partial sum),
 // so when the two best first-pass scores are more than 2 * eps apart the best unit of the exact
 // weights is the first pass's best unit.  Such samples are finalised here (distance recomputed in
@@ -767,7 +768,9 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
         const float s1 = score_of_key(k1), s2 = score_of_key(k2);
         const float cnt = (float)(end - beg);
         const float bound = fmaxf(fabsf(s1), fabsf(s2)) + 2.f * cnt * wmax;
-        const float eps = cnt * wmax * 4.8828125e-4f * 1.0001f + 2.f * (cnt + 2.f) * 5.9604645e-8f * bound;
+        // per weight: 2^-11 relative in fp16's normal range, at most 2^-25 absolute below it
+        const float per_weight = fmaxf(wmax * 4.8828125e-4f, 2.9802322e-8f) * 1.0001f;
+        const float eps = cnt * per_weight + 2.f * (cnt + 2.f) * 5.9604645e-8f * bound;
         const bool certain = (s2 - s1) > 2.f * eps;  // false for NaN or an empty second key
         flag = !certain;
         if (certain) {

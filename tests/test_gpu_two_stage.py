@@ -53,7 +53,7 @@ def _check(W_host, V, M, b, g_bmu, g_dist, rows):
     return rep
 
 
-@pytest.mark.parametrize("scale", [1.0, 37.0, 1.0 / 64.0])
+@pytest.mark.parametrize("scale", [1.0, 37.0, 1.0 / 64.0, 1e-6, 1e5])
 def test_two_stage_matches_oracle_and_plain_search(som_mod, scale):
     """The error bound scales with the largest weight, so the certificate must hold for scaled codebooks."""
     V, M, n = 30_000, 1_024, 80_000
@@ -62,7 +62,10 @@ def test_two_stage_matches_oracle_and_plain_search(som_mod, scale):
     h2, bmu2, dist2 = _run(som_mod, W, V, M, b, True)
     h1, bmu1, dist1 = _run(som_mod, W, V, M, b, False)
     unc = h2.last_uncertain()
-    assert 0 < unc < n // 2  # most samples are certified, some are not
+    if 1e-3 < scale < 1e3:
+        assert 0 < unc < n // 2  # most samples are certified, some are not
+    # (weights of 1e-6 fall into fp16's subnormal range, weights of 1e5 overflow it: the bound
+    # then certifies little or nothing and the exact pass does the work)
     differ = np.flatnonzero(bmu1 != bmu2)
     assert differ.size <= unc  # only samples of the exact pass can differ (near ties, other summation order)
     same = bmu1 == bmu2
