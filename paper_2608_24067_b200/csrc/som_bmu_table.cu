@@ -1,30 +1,32 @@
-// Row-table BMU search kernel (the fast path of som_bmu) and its finalisation.
+// Row-table BMU search kernel (the fast path of som_bmu), the certificate of the two-stage
+// search and the finalisation.
 //
 // Decomposition (Section 3.3 of the paper, re-planned for B200): a work unit is a neuron
-// range of T = 8*R neurons (R = 8 or 4 per lane) times a contiguous part of the mask-sorted
-// sample list.  One persistent block per SM claims units in range-major order, so that at any
-// time only a few neuron ranges are live and their codebook slabs W[:, i0..i0+T) stay
-// L2-resident while HBM sees the codebook about once per batch.  Inside a unit the warps pull
-// chunks of samples from a shared counter, which keeps them busy whatever the mix of row
-// lengths.
+// range of T = 8*R neurons (R neurons per lane) times a contiguous part of the mask-sorted
+// sample list.  One persistent block per SM claims units from a global counter in range-major
+// order, so that at any time only a few neuron ranges are live and their codebook slabs
+// W[:, i0..i0+T) stay L2-resident while HBM sees the codebook about once per batch.  Inside a
+// unit the warps pull chunks of samples from a shared counter, which keeps them busy whatever
+// the mix of row lengths.
 //
 // Inside a block the rows W[v*M + i0 .. i0+T) of the batch's hottest features (the row
 // table) are staged in shared memory once per unit.  Eight lanes form a team that owns one
-// sample at a time; a lane keeps R score accumulators in registers (R/4 groups of four
-// neurons, 32 neurons apart) and subtracts, for every code of the sample, one 128-bit slice of
-// the row per group: a shared-memory read for hot features, a coalesced 128-bit L2-only read
-// of the L2-resident slab for tail features.  The team's 8 loads of a group cover one
-// contiguous 128-byte row segment.  Subtractions are packed f32x2 operations, which halves
-// their issue slots.  The accumulators start from ||w||^2/2 - sum(rows of the sample's mask
-// features), which is held in registers across consecutive samples that share the mask (they
-// are adjacent after the plan's sort).
+// sample at a time; a lane keeps R score accumulators in registers and subtracts, for every
+// code of the sample, its 128-bit slices of the row: a shared-memory read for hot features, a
+// coalesced 128-bit read-only load of the L2-resident slab for tail features (the team's eight
+// loads cover one contiguous 128-byte segment).  How the R neurons map onto a row, and how a
+// slice is consumed, is the storage layout's business (fp32: packed f32x2 subtractions;
+// fp16: mixed-precision adds; see the Lay* structs).  The accumulators start from ||w||^2/2
+// minus the rows of the sample's mask features, which is held in registers across consecutive
+// samples that share the mask (they are adjacent after the plan's sort).
 //
 // Feeding the teams: a sample's 48-byte slot sits at a fixed address for its sorted position.
 // Each warp owns a two-stage ring in shared memory; 14 of its lanes fetch the slot and key
 // bytes of round r+2 into registers, store those of round r+1, and every team reads round r
 // from the ring, so slot and key latency is never on the critical path.  A sample's first
 // four tail rows go in flight at the top of its round and are consumed after its hot rows.
-// The hot loop is a jump table on the longest hot list of the warp's four samples (shorter
+// The first hot row is subtracted in three-operand form (score = prefix - row), the rest of
+// the hot loop is a jump table on the longest hot list of the warp's four samples (shorter
 // lists are padded with an all-zero row), the slot array is padded to whole rounds and all
 // addressing is by pointer increment, so the inner steps carry no predicate.
 //
@@ -34,10 +36,6 @@
 // order-independent and ties break to the lowest neuron index (Section 3.1).
 #include "som_internal.cuh"
 #include "som_plan.cuh"
-
-#ifndef SOM_TAIL_LOAD_CG
-#define SOM_TAIL_LOAD_CG 0
-#endif
 
 namespace {
 
@@ -85,11 +83,7 @@ __device__ __forceinline__ Pair2 lds_row(const unsigned char* p)
 __device__ __forceinline__ Pair2 ldg_row(const float* p)
 {
     Pair2 r;
-#if SOM_TAIL_LOAD_CG
-    asm("ld.global.cg.v2.b64 {%0,%1}, [%2];" : "=l"(r.lo), "=l"(r.hi) : "l"(p));
-#else
     asm("ld.global.nc.v2.b64 {%0,%1}, [%2];" : "=l"(r.lo), "=l"(r.hi) : "l"(p));
-#endif
     return r;
 }
 

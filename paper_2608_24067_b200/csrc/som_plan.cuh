@@ -102,7 +102,7 @@ int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32
 
 // Geometry of the row-table kernel for this handle: neurons per range, hot rows that fit.
 struct SomTableGeom {
-    int R;        // neurons per lane (4)
+    int R;        // neurons per lane (4, 8 or 16)
     int T;        // neurons per range = 8 * R
     int n_hot;    // hot rows held in shared memory
     int threads;  // block size

@@ -324,3 +324,21 @@ def test_large_configs_full_size_sampled_rows(som_mod, cfg, n_rows):
     h.destroy()
     del W
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("variant", [1, 2, 0])
+def test_batch_of_empty_samples(som_mod, variant):
+    """Every sample empty (nnz = 0, no index array needed): each gets argmin ||w_i||^2 and that norm."""
+    V, M, n = 500, 1_024, 100_000
+    W = synth.fill_codebook(V, M, 8, device="cuda")
+    indptr = torch.zeros(n + 1, dtype=torch.int32, device="cuda")
+    indices = torch.zeros(1, dtype=torch.int32, device="cuda")
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, variant)
+    h.norms()
+    bmu, dist = h.bmu(indptr, indices)
+    torch.cuda.synchronize()
+    nn = orc.norms(W.cpu().numpy(), V, M)
+    best = int(np.argmin(nn.astype(np.float32)))
+    assert np.all(bmu.cpu().numpy() == best)
+    np.testing.assert_allclose(dist.cpu().numpy(), np.float32(nn[best]), rtol=1e-6)
