@@ -113,6 +113,54 @@ void som_oracle_dist_at(const float* W, int layout, int64_t V, int64_t M, const 
     }
 }
 
+/*
+ * Sparse real-valued samples (the paper's outlook, Section 7: "carrying ||x||^2 and a values array
+ * alongside the feature indices"): x has value val[k] at feature idx[k] and 0 elsewhere, and
+ *   d(x, w_i) = ||x - w_i||^2 = sum_k val[k]^2 - 2 * sum_k val[k] * w_i[idx[k]] + ||w_i||^2.
+ */
+static double distance_values(const float* W, int layout, int64_t V, int64_t M, const double* norms,
+                              const int32_t* idx, const float* val, int64_t nnz, int64_t i)
+{
+    double xx = 0.0, dot = 0.0;
+    for (int64_t k = 0; k < nnz; ++k) {
+        const double x = (double)val[k];
+        xx += x * x;
+        dot += x * weight(W, layout, V, M, (int64_t)idx[k], i);
+    }
+    return xx - 2.0 * dot + norms[i];
+}
+
+/* som_oracle_bmu for sparse real-valued samples (values[] runs parallel to indices[]). */
+void som_oracle_bmu_values(const float* W, int layout, int64_t V, int64_t M, const double* norms,
+                           const int32_t* indptr, const int32_t* indices, const float* values, int64_t n,
+                           int64_t* b1, double* d1, int64_t* b2, double* d2)
+{
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t s = 0; s < n; ++s) {
+        const int32_t* idx = indices + indptr[s];
+        const float* val = values + indptr[s];
+        int64_t nnz = (int64_t)indptr[s + 1] - (int64_t)indptr[s];
+        int64_t bb1 = -1, bb2 = -1;
+        double dd1 = INFINITY, dd2 = INFINITY;
+        for (int64_t i = 0; i < M; ++i) {
+            double d = distance_values(W, layout, V, M, norms, idx, val, nnz, i);
+            if (d < dd1) { dd2 = dd1; bb2 = bb1; dd1 = d; bb1 = i; }
+            else if (d < dd2) { dd2 = d; bb2 = i; }
+        }
+        b1[s] = bb1; d1[s] = dd1; b2[s] = bb2; d2[s] = dd2;
+    }
+}
+
+void som_oracle_dist_at_values(const float* W, int layout, int64_t V, int64_t M, const double* norms,
+                               const int32_t* indptr, const int32_t* indices, const float* values,
+                               int64_t n, const int64_t* neuron, double* d)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < n; ++s)
+        d[s] = distance_values(W, layout, V, M, norms, indices + indptr[s], values + indptr[s],
+                               (int64_t)indptr[s + 1] - (int64_t)indptr[s], neuron[s]);
+}
+
 /* Full n x M distance matrix (row-major), for tiny inputs only. */
 void som_oracle_all_distances(const float* W, int layout, int64_t V, int64_t M, const double* norms,
                               const int32_t* indptr, const int32_t* indices, int64_t n, double* out)

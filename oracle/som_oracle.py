@@ -48,8 +48,10 @@ def _load():
                                        P, P, P, P]
         lib.som_oracle_dist_at.argtypes = [P, ctypes.c_int, I64, I64, P, P, P, I64, P, P]
         lib.som_oracle_all_distances.argtypes = [P, ctypes.c_int, I64, I64, P, P, P, I64, P]
+        lib.som_oracle_bmu_values.argtypes = [P, ctypes.c_int, I64, I64, P, P, P, P, I64, P, P, P, P]
+        lib.som_oracle_dist_at_values.argtypes = [P, ctypes.c_int, I64, I64, P, P, P, P, I64, P, P]
         for f in (lib.som_oracle_norms, lib.som_oracle_bmu, lib.som_oracle_dist_at,
-                  lib.som_oracle_all_distances):
+                  lib.som_oracle_all_distances, lib.som_oracle_bmu_values, lib.som_oracle_dist_at_values):
             f.restype = None
         _lib = lib
     return _lib
@@ -112,6 +114,38 @@ def bmu(W, V: int, M: int, indptr, indices, layout: int = FEATURE_MAJOR, norms_=
         merge = 1
     _load().som_oracle_bmu(_p(W), layout, V, M, _p(norms_), _p(indptr), _p(indices), n,
                            m_offset, merge, _p(out.b1), _p(out.d1), _p(out.b2), _p(out.d2))
+    return out
+
+
+def bmu_values(W, V: int, M: int, indptr, indices, values, layout: int = FEATURE_MAJOR, norms_=None) -> Top2:
+    """Best and second-best unit per sparse real-valued sample (``values`` parallel to ``indices``)."""
+    W = _f32(W).reshape(-1)
+    assert W.size == V * M
+    indptr, indices, values = _i32(indptr), _i32(indices), _f32(values)
+    assert values.size == indices.size
+    n = indptr.size - 1
+    if norms_ is None:
+        norms_ = norms(W, V, M, layout)
+    norms_ = np.ascontiguousarray(norms_, dtype=np.float64)
+    out = Top2(np.empty(n, np.int64), np.empty(n, np.float64), np.empty(n, np.int64), np.empty(n, np.float64))
+    _load().som_oracle_bmu_values(_p(W), layout, V, M, _p(norms_), _p(indptr), _p(indices), _p(values), n,
+                                  _p(out.b1), _p(out.d1), _p(out.b2), _p(out.d2))
+    return out
+
+
+def dist_at_values(W, V: int, M: int, indptr, indices, values, neuron, layout: int = FEATURE_MAJOR,
+                   norms_=None) -> np.ndarray:
+    """fp64 squared distance of real-valued sample n to neuron[n]."""
+    W = _f32(W).reshape(-1)
+    indptr, indices, values = _i32(indptr), _i32(indices), _f32(values)
+    n = indptr.size - 1
+    neuron = np.ascontiguousarray(neuron, dtype=np.int64)
+    if norms_ is None:
+        norms_ = norms(W, V, M, layout)
+    norms_ = np.ascontiguousarray(norms_, dtype=np.float64)
+    out = np.empty(n, np.float64)
+    _load().som_oracle_dist_at_values(_p(W), layout, V, M, _p(norms_), _p(indptr), _p(indices), _p(values), n,
+                                      _p(neuron), _p(out))
     return out
 
 

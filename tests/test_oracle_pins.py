@@ -245,3 +245,36 @@ def test_second_best_parity_rule_on_brute_force():
     assert swapped.ok
     wrong_dist = parity.check_second(t.b1, t.b2, D[ar, t.b2] * (1 + 1e-4), t, D[ar, t.b2], M)
     assert wrong_dist.dist_violations == n
+
+
+def test_real_valued_samples_against_dense_brute_force():
+    """Sparse real-valued samples: ||x||^2 - 2<x,w> + ||w||^2 against sum_v (x_v - w_iv)^2 on the
+    densified vector (numpy); all-ones values reduce to the binary search; a neuron equal to the
+    sample is at distance zero."""
+    rng = np.random.default_rng(21)
+    V, M, n = 48, 19, 120
+    W = rng.normal(size=(V, M)).astype(np.float32)
+    rows = [np.sort(rng.choice(V, size=int(rng.integers(0, 10)), replace=False)).astype(np.int32) for _ in range(n)]
+    indptr = np.zeros(n + 1, np.int32)
+    indptr[1:] = np.cumsum([len(r) for r in rows])
+    indices = np.concatenate(rows).astype(np.int32)
+    values = rng.normal(size=indices.size).astype(np.float32)
+    X = np.zeros((n, V))
+    for s_, r in enumerate(rows):
+        X[s_, r] = values[indptr[s_]:indptr[s_ + 1]].astype(np.float64)
+    D = ((X[:, :, None] - W.astype(np.float64)[None, :, :]) ** 2).sum(1)
+    t = orc.bmu_values(W.reshape(-1), V, M, indptr, indices, values)
+    order = np.argsort(D, axis=1, kind="stable")
+    np.testing.assert_array_equal(t.b1, order[:, 0])
+    np.testing.assert_array_equal(t.b2, order[:, 1])
+    np.testing.assert_allclose(t.d1, D[np.arange(n), t.b1], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(orc.dist_at_values(W.reshape(-1), V, M, indptr, indices, values, t.b2),
+                               D[np.arange(n), t.b2], rtol=1e-12, atol=1e-12)
+    ones = np.ones_like(values)
+    tb, tv = orc.bmu(W.reshape(-1), V, M, indptr, indices), orc.bmu_values(W.reshape(-1), V, M, indptr, indices, ones)
+    np.testing.assert_array_equal(tb.b1, tv.b1)
+    np.testing.assert_allclose(tb.d1, tv.d1, rtol=1e-13, atol=1e-13)
+    W2 = W.copy()
+    W2[:, 7] = X[3].astype(np.float32)  # neuron 7 becomes sample 3
+    t2 = orc.bmu_values(W2.reshape(-1), V, M, indptr, indices, values)
+    assert t2.b1[3] == 7 and abs(t2.d1[3]) < 1e-5
