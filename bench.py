@@ -224,13 +224,20 @@ def run_ours(args, w: synth.Workload):
         h.set_option(6, args.update_mib)
     if args.two_stage:
         h.set_option(7, 1)
+    sample_values = []
+    if args.values:
+        for bi, b in enumerate(batches):
+            k = torch.arange(b.nnz, dtype=torch.int64, device=dev)
+            sample_values.append(synth._u24_to_f32(synth.hash32(w.seed + 17, 5, k, bi), 0.25, 1.5))
     out_bmu = torch.empty(w.batch, dtype=torch.int32, device=dev)
     out_dist = torch.empty(w.batch, dtype=torch.float32, device=dev)
 
     def step(i):
         b = batches[i % n_batches]
         h.norms()
-        if args.top2:
+        if args.values:
+            h.bmu_values(b.indptr, b.indices, sample_values[i % n_batches])
+        elif args.top2:
             h.bmu2(b.indptr, b.indices)
         else:
             h.bmu(b.indptr, b.indices, out_bmu, out_dist)
@@ -293,7 +300,8 @@ def run_ours(args, w: synth.Workload):
 
     # ---- the same step with the two-stage search (library option 7), reported beside the headline ----
     two_stage = None
-    if args.store == "f32" and w.M % 128 == 0 and not args.top2 and not args.two_stage and not args.no_two_stage_leg:
+    if (args.store == "f32" and w.M % 128 == 0 and not args.top2 and not args.two_stage and not args.values
+            and not args.no_two_stage_leg):
         free_b, _ = torch.cuda.mem_get_info()
         if free_b > w.V * w.M * 2 + (4 << 30):
             try:
@@ -401,7 +409,7 @@ def run_ours(args, w: synth.Workload):
         "dtype": "f32" if args.store == "f32" else "f32 accumulate, f16-stored codebook",
         "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": nnz_mean,
-                   "step": "som_norms + %s on one batch" % ("som_bmu2" if args.top2 else "som_bmu"),
+                   "step": "som_norms + %s on one batch" % ("som_bmu_values" if args.values else ("som_bmu2" if args.top2 else "som_bmu")),
                    "replicas": ws,
                    "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
                        w.V * w.M * store_bytes / 1e6, batches[0].nnz * 4 / 1e6) if w.V * w.M * store_bytes > 126e6 else
@@ -452,6 +460,8 @@ def main():
                     help="fp32 storage: certified first pass over an fp16 copy, exact second pass (library option 7)")
     ap.add_argument("--no-two-stage-leg", action="store_true",
                     help="skip the extra measurement of the two-stage search that the default run reports beside the headline")
+    ap.add_argument("--values", action="store_true",
+                    help="time som_bmu_values (sparse real-valued samples: seeded values in [0.25, 1.75)) instead of som_bmu")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -123,6 +123,20 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
              int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream);
 
 /*
+ * som_bmu_values - the search for sparse REAL-VALUED samples (the paper's outlook, Section 7: "carrying
+ * ||x||^2 and a values array alongside the feature indices"; its SparseFloat variant, Table 6):
+ *   d_values   DEVICE pointer, fp32, parallel to d_indices: sample s has value d_values[k] at feature
+ *              d_indices[k] for k in [d_indptr[s], d_indptr[s+1]) and 0 elsewhere.
+ * BMU = argmin_i (||w_i||^2 - 2 * sum_k x_k * w_i[idx_k]), ties to the lowest index; d_min_dist is
+ * ||x||^2 - 2<x,w> + ||w||^2, recomputed in fp64 for the winner.  With all values 1 the result is
+ * som_bmu's.  The gather-sum becomes a gather-multiply (fused multiply-add, fp32), run by the
+ * direct-load kernel only (the row-table plan is specific to binary samples); other arguments,
+ * preconditions, asynchrony and determinism as in som_bmu.
+ */
+int som_bmu_values(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, const float* d_values,
+                   int64_t n_samples, int32_t* d_bmu, float* d_min_dist, void* stream);
+
+/*
  * som_update - the batch update that follows the search in an epoch (Section 3.4; Algorithm 2,
  * steps 8-9): scatter the samples onto the lattice (per cell the sum of its assigned samples
  * and their count), blur both fields with three unnormalised box passes per lattice axis of

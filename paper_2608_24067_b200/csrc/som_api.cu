@@ -314,6 +314,33 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
     return bmu_impl(h, d_indptr, d_indices, n_samples, d_bmu, d_min_dist, d_bmu2, d_dist2, stream);
 }
 
+int som_bmu_values(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, const float* d_values,
+                   int64_t n_samples, int32_t* d_bmu, float* d_min_dist, void* stream)
+{
+    if (!h || n_samples < 0) return SOM_ERR_INVALID_ARG;
+    if (n_samples == 0) return SOM_OK;
+    if (!d_indptr || !d_indices || !d_values || !d_bmu || !d_min_dist) return SOM_ERR_INVALID_ARG;
+    if (n_samples >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
+    if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t key_bytes = som_align_up((size_t)n_samples * sizeof(unsigned long long), 256);
+    int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, key_bytes);
+    if (rc) return rc;
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(h->ws);
+    if (h->timing && (rc = ensure_events(h))) return rc;
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
+    SOM_CK(h, cudaMemsetAsync(keys, 0xFF, key_bytes, st));
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+    if ((rc = som_launch_bmu_values(h, d_indptr, d_indices, d_values, n_samples, keys, st))) return rc;
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+    if ((rc = som_launch_finalize_values(h, d_indptr, d_indices, d_values, n_samples, keys, d_bmu, d_min_dist, st)))
+        return rc;
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
+    if (h->timing) h->ev_bmu_calls += 1;
+    return SOM_OK;
+}
+
 int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indptr, const int32_t* d_indices,
                int64_t n_samples, const int32_t* d_bmu, int32_t radius, void* stream)
 {

@@ -40,12 +40,15 @@ __device__ __forceinline__ void load4(const __half* p, float (&w)[4])
 
 // TOP2 also keeps the second-best unit in keys2 (Algorithm 2 keeps the two best units).
 // ST is the storage type of the codebook (float, or __half widened exactly before the fp32 add).
-template <int VEC, bool TOP2, typename ST>
+// VALUED: sparse real-valued samples (a values array parallel to the indices; the paper's outlook,
+// Section 7): the gather-sum becomes a gather-multiply, score = ||w||^2/2 - sum_k x_k * w[idx_k].
+template <int VEC, bool TOP2, typename ST, bool VALUED = false>
 __global__ void __launch_bounds__(DIRECT_THREADS)
 k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
              const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
              unsigned long long* __restrict__ keys, unsigned long long* __restrict__ keys2,
-             int64_t neuron_off, const int32_t* __restrict__ sample_list)
+             int64_t neuron_off, const int32_t* __restrict__ sample_list,
+             const float* __restrict__ values = nullptr)
 {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -69,21 +72,30 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
         for (int k = 0; k < VEC; ++k) acc[k] = seed[k];
         for (int base = beg; base < end; base += 32) {
             const int mine = (base + lane < end) ? indices[base + lane] : 0;
+            const float mine_x = (VALUED && base + lane < end) ? values[base + lane] : 1.f;
             const int cnt = min(32, end - base);
             for (int j = 0; j < cnt; ++j) {
                 const int v = __shfl_sync(0xffffffffu, mine, j);
+                const float x = VALUED ? __shfl_sync(0xffffffffu, mine_x, j) : 1.f;
                 const ST* p = W + (int64_t)v * M + i0;
                 if (VEC == 4) {
                     if (live) {
                         float w[4];
                         load4(p, w);
-                        acc[0] -= w[0];
-                        acc[1 % VEC] -= w[1];
-                        acc[2 % VEC] -= w[2];
-                        acc[3 % VEC] -= w[3];
+                        if (VALUED) {
+                            acc[0] = fmaf(-x, w[0], acc[0]);
+                            acc[1 % VEC] = fmaf(-x, w[1], acc[1 % VEC]);
+                            acc[2 % VEC] = fmaf(-x, w[2], acc[2 % VEC]);
+                            acc[3 % VEC] = fmaf(-x, w[3], acc[3 % VEC]);
+                        } else {
+                            acc[0] -= w[0];
+                            acc[1 % VEC] -= w[1];
+                            acc[2 % VEC] -= w[2];
+                            acc[3 % VEC] -= w[3];
+                        }
                     }
                 } else {
-                    if (live) acc[0] -= som_weight(p);
+                    if (live) acc[0] = VALUED ? fmaf(-x, som_weight(p), acc[0]) : acc[0] - som_weight(p);
                 }
             }
         }
@@ -146,7 +158,7 @@ __global__ void k_finalize(const ST* __restrict__ W, const double* __restrict__ 
                            const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                            int64_t n, const unsigned long long* __restrict__ keys,
                            int32_t* __restrict__ bmu, float* __restrict__ dist,
-                           const int32_t* __restrict__ sample_list)
+                           const int32_t* __restrict__ sample_list, const float* __restrict__ values = nullptr)
 {
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= n) return;
@@ -159,10 +171,19 @@ __global__ void k_finalize(const ST* __restrict__ W, const double* __restrict__ 
     }
     const int beg = indptr[s];
     const int end = indptr[s + 1];
-    double dot = 0.0;
-    for (int j = beg; j < end; ++j) dot += (double)som_weight(W + (int64_t)indices[j] * M + idx);
+    double dot = 0.0, xx = (double)(end - beg);
+    if (values) {
+        xx = 0.0;
+        for (int j = beg; j < end; ++j) {
+            const double x = (double)values[j];
+            xx += x * x;
+            dot += x * (double)som_weight(W + (int64_t)indices[j] * M + idx);
+        }
+    } else {
+        for (int j = beg; j < end; ++j) dot += (double)som_weight(W + (int64_t)indices[j] * M + idx);
+    }
     bmu[s] = (int32_t)idx;
-    dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
+    dist[s] = (float)(xx - 2.0 * dot + norm64[idx]);
 }
 
 __global__ void k_validate(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
@@ -219,6 +240,53 @@ int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* i
         SOM_CK(h, cudaGetLastError());
         h->launches += 1;
     }
+    return SOM_OK;
+}
+
+// Sparse real-valued samples: always the direct-load kernel, best unit only.
+int som_launch_bmu_values(som_handle* h, const int32_t* indptr, const int32_t* indices, const float* values,
+                          int64_t n, unsigned long long* keys, cudaStream_t st)
+{
+    const int vec = (h->M % 4 == 0) ? 4 : 1;
+    const int64_t per_block = (int64_t)DIRECT_WARPS * DIRECT_SAMPLES_PER_WARP;
+    const int64_t gx = (n + per_block - 1) / per_block;
+    const int64_t neurons_per_block = 32 * vec;
+    const int64_t gy = (h->M + neurons_per_block - 1) / neurons_per_block;
+    const int64_t max_gy = 65535;
+    for (int64_t y0 = 0; y0 < gy; y0 += max_gy) {
+        const int64_t ny = (gy - y0 < max_gy) ? gy - y0 : max_gy;
+        dim3 grid((unsigned)gx, (unsigned)ny);
+        const int64_t neuron_off = y0 * neurons_per_block;
+#define SOM_VALUED(VEC_, ST_, W_)                                                                     \
+    k_bmu_direct<VEC_, false, ST_, true><<<grid, DIRECT_THREADS, 0, st>>>(W_, h->hnorm, h->M, indptr, indices, n, \
+                                                                          keys, nullptr, neuron_off, nullptr, values)
+        if (h->Wh) {
+            if (vec == 4) SOM_VALUED(4, __half, h->Wh);
+            else SOM_VALUED(1, __half, h->Wh);
+        } else {
+            if (vec == 4) SOM_VALUED(4, float, h->W);
+            else SOM_VALUED(1, float, h->W);
+        }
+#undef SOM_VALUED
+        SOM_CK(h, cudaGetLastError());
+        h->launches += 1;
+    }
+    return SOM_OK;
+}
+
+int som_launch_finalize_values(som_handle* h, const int32_t* indptr, const int32_t* indices, const float* values,
+                               int64_t n, const unsigned long long* keys, int32_t* bmu, float* dist,
+                               cudaStream_t st)
+{
+    const int64_t blocks = (n + 255) / 256;
+    if (h->Wh)
+        k_finalize<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, indptr, indices, n, keys,
+                                                             bmu, dist, nullptr, values);
+    else
+        k_finalize<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, keys,
+                                                            bmu, dist, nullptr, values);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
     return SOM_OK;
 }
 

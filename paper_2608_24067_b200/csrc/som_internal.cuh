@@ -94,6 +94,11 @@ int som_launch_bmu_direct(som_handle* h, const int32_t* indptr, const int32_t* i
 int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                         const unsigned long long* keys, int32_t* bmu, float* dist, const int32_t* sample_list,
                         cudaStream_t st);
+int som_launch_bmu_values(som_handle* h, const int32_t* indptr, const int32_t* indices, const float* values,
+                          int64_t n, unsigned long long* keys, cudaStream_t st);
+int som_launch_finalize_values(som_handle* h, const int32_t* indptr, const int32_t* indices, const float* values,
+                               int64_t n, const unsigned long long* keys, int32_t* bmu, float* dist,
+                               cudaStream_t st);
 int som_launch_validate(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                         int* d_flag, cudaStream_t st);
 size_t som_norms_workspace_bytes(const som_handle* h);

@@ -24,7 +24,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
-    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain",
+    "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain", "som_bmu_values",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -61,6 +61,8 @@ def load_library():
     lib.som_bmu_host.argtypes = [P, P, P, I64, P, P, P]
     lib.som_bmu2.argtypes = [P, P, P, I64, P, P, P, P, P]
     lib.som_bmu2.restype = INT
+    lib.som_bmu_values.argtypes = [P, P, P, P, I64, P, P, P]
+    lib.som_bmu_values.restype = INT
     lib.som_update.argtypes = [P, I32, I32, P, P, I64, P, I32, P]
     lib.som_update.restype = INT
     lib.som_validate_csr.argtypes = [P, P, P, I64, P]
@@ -176,6 +178,19 @@ class Som:
                                 _stream_ptr(stream))
         self._check(rc, "som_bmu2")
         return tuple(out)
+
+    def bmu_values(self, indptr: torch.Tensor, indices: torch.Tensor, values: torch.Tensor, stream=None):
+        """som_bmu_values: sparse real-valued samples; returns (bmu int32 [n], squared distance fp32 [n])."""
+        n = indptr.numel() - 1
+        dev = self.codebook.device
+        out_bmu = torch.empty(n, dtype=torch.int32, device=dev)
+        out_dist = torch.empty(n, dtype=torch.float32, device=dev)
+        rc = self._lib.som_bmu_values(self._h, _dev_ptr(indptr, torch.int32, "indptr"),
+                                      _dev_ptr(indices, torch.int32, "indices"),
+                                      _dev_ptr(values, torch.float32, "values"), n,
+                                      out_bmu.data_ptr(), out_dist.data_ptr(), _stream_ptr(stream))
+        self._check(rc, "som_bmu_values")
+        return out_bmu, out_dist
 
     def update(self, rows: int, cols: int, indptr: torch.Tensor, indices: torch.Tensor, bmu: torch.Tensor,
                radius: int, stream=None):
