@@ -122,39 +122,55 @@ k_select_hot(const uint32_t* __restrict__ feat_count, int V, int n_mask, int n_h
     kth_largest(feat_count, V, n_mask + n_hot, sh_hist, sh_state, &thr_a, &gr_a);
     const int need_m = n_mask - gr_m;            // ties at thr_m to take (lowest ids first)
     const int need_a = n_mask + n_hot - gr_a;    // ties at thr_a to take
-    int tie_m_seen = 0, tie_a_seen = 0, mask_assigned = 0, hot_assigned = 0;
-    for (int v0 = 0; v0 < V; v0 += 1024) {
-        const int v = v0 + threadIdx.x;
-        const uint32_t c = (v < V) ? feat_count[v] : 0u;
-        const int e_m = (v < V && c == thr_m && c > 0) ? 1 : 0;
-        const int e_a = (v < V && c == thr_a && c > 0) ? 1 : 0;
-        int tot;
-        const int r_m = block_excl_scan_1024(e_m, warp_sums, &sh_total);
-        tot = sh_total;
-        const int is_mask = (v < V) && (c > thr_m || (e_m && tie_m_seen + r_m < need_m));
-        tie_m_seen += tot;
-        const int r_a = block_excl_scan_1024(e_a, warp_sums, &sh_total);
-        tot = sh_total;
-        const int is_sel = (v < V) && (c > thr_a || (e_a && tie_a_seen + r_a < need_a));
-        tie_a_seen += tot;
-        const int is_hot = is_sel && !is_mask;
-        const int s_m = block_excl_scan_1024(is_mask, warp_sums, &sh_total);
-        const int tot_m = sh_total;
-        const int s_h = block_excl_scan_1024(is_hot, warp_sums, &sh_total);
-        const int tot_h = sh_total;
-        if (v < V) {
-            int slot = -1;
-            if (is_mask) slot = mask_assigned + s_m;
-            else if (is_hot) slot = n_mask + hot_assigned + s_h;
-            feat_slot[v] = slot;
-            if (slot >= 0) {
-                slot_feat[slot] = v;
-                atomicAdd(&n_slots[SOM_PLAN_COVERED], (int)c);  // instances the table will serve
-            }
-        }
-        mask_assigned += tot_m;
-        hot_assigned += tot_h;
+    // Every thread owns a contiguous range of feature ids, so ranks in id order are "offset of my
+    // range (one block scan) + position inside it".  Pass 1 ranks the ties at the two thresholds
+    // (the lowest ids are taken), pass 2 decides mask / hot and counts them, pass 3 writes the
+    // slots: four block scans in all, whatever V is.
+    const int per = (V + 1023) / 1024;
+    const int v_lo = min(V, (int)threadIdx.x * per), v_hi = min(V, v_lo + per);
+    int my_em = 0, my_ea = 0;
+    for (int v = v_lo; v < v_hi; ++v) {
+        const uint32_t c = feat_count[v];
+        my_em += (c == thr_m && c > 0);
+        my_ea += (c == thr_a && c > 0);
     }
+    const int off_em = block_excl_scan_1024(my_em, warp_sums, &sh_total);
+    const int off_ea = block_excl_scan_1024(my_ea, warp_sums, &sh_total);
+    int my_mask = 0, my_hot = 0, seen_m = off_em, seen_a = off_ea;
+    for (int v = v_lo; v < v_hi; ++v) {
+        const uint32_t c = feat_count[v];
+        const bool e_m = c == thr_m && c > 0, e_a = c == thr_a && c > 0;
+        const bool is_mask = c > thr_m || (e_m && seen_m < need_m);
+        const bool is_sel = c > thr_a || (e_a && seen_a < need_a);
+        seen_m += e_m;
+        seen_a += e_a;
+        my_mask += is_mask;
+        my_hot += is_sel && !is_mask;
+    }
+    int slot_m = block_excl_scan_1024(my_mask, warp_sums, &sh_total);
+    const int mask_assigned = sh_total;
+    int slot_h = block_excl_scan_1024(my_hot, warp_sums, &sh_total);
+    const int hot_assigned = sh_total;
+    seen_m = off_em;
+    seen_a = off_ea;
+    int covered = 0;
+    for (int v = v_lo; v < v_hi; ++v) {
+        const uint32_t c = feat_count[v];
+        const bool e_m = c == thr_m && c > 0, e_a = c == thr_a && c > 0;
+        const bool is_mask = c > thr_m || (e_m && seen_m < need_m);
+        const bool is_sel = c > thr_a || (e_a && seen_a < need_a);
+        seen_m += e_m;
+        seen_a += e_a;
+        int slot = -1;
+        if (is_mask) slot = slot_m++;
+        else if (is_sel) slot = n_mask + slot_h++;
+        feat_slot[v] = slot;
+        if (slot >= 0) {
+            slot_feat[slot] = v;
+            covered += (int)c;  // instances the table will serve
+        }
+    }
+    if (covered) atomicAdd(&n_slots[SOM_PLAN_COVERED], covered);
     // unused slots (fewer distinct features than slots) point at no feature
     for (int s = threadIdx.x; s < n_mask + n_hot; s += blockDim.x) {
         const bool used = (s < n_mask) ? (s < mask_assigned) : (s - n_mask < hot_assigned);
