@@ -366,7 +366,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const int32_t* __restrict__ slot_feat, int n_rows,
             const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
             u64* __restrict__ keys, u64* __restrict__ keys2, int parts, int64_t part_len, int n_units,
-            int* __restrict__ unit_counter)
+            int n_whole, int* __restrict__ unit_counter)
 {
     constexpr int R = L::R;
     constexpr int T = L::T;
@@ -410,8 +410,11 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
         __syncthreads();
         const int unit = unit_sh;
         if (unit >= n_units) break;
-        const int range = unit / parts;
-        const int part = unit - range * parts;
+        // The last units of the launch are claimed in quarters, so that the blocks run out of
+        // work within a quarter of a unit of each other.
+        const int whole = unit < n_whole ? unit : n_whole + ((unit - n_whole) >> 2);
+        const int range = whole / parts;
+        const int part = whole - range * parts;
         const int64_t i0 = (int64_t)range * T;
         if (range != cur_range) {
             L::stage(tab, W, M, i0, slot_feat, n_rows, warp, lane, WARPS);
@@ -427,8 +430,13 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
         }
         __syncthreads();
 
-        const int64_t k_begin = (int64_t)part * part_len;
-        const int64_t k_end = min(n_pad, k_begin + part_len);  // a multiple of 4
+        int64_t k_begin = (int64_t)part * part_len;
+        int64_t k_end = min(n_pad, k_begin + part_len);  // a multiple of 4
+        if (unit >= n_whole) {
+            const int64_t quarter = ((part_len >> 2) + CHUNK - 1) / CHUNK * CHUNK;
+            k_begin += (int64_t)((unit - n_whole) & 3) * quarter;
+            k_end = min(k_end, k_begin + quarter);
+        }
         const int n_chunks = (int)((k_end - k_begin + CHUNK - 1) / CHUNK);
 
         uint32_t curmask = 0;
@@ -633,8 +641,12 @@ int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* he
     parts = (int)((n + part_len - 1) / part_len);
     const int64_t n_units64 = (int64_t)n_ranges * parts;
     if (n_units64 > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
-    const int n_units = (int)n_units64;
-    const int grid = n_units < h->sm_count ? n_units : h->sm_count;
+    const int grid = n_units64 < h->sm_count ? (int)n_units64 : h->sm_count;
+    // the last `grid` units are claimed as quarters (see the kernel)
+    const int n_split = (n_units64 >= 4 * (int64_t)grid && part_len >= 16 * CHUNK) ? grid : 0;
+    const int n_whole = (int)n_units64 - n_split;
+    if (n_units64 + 3 * (int64_t)n_split > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
+    const int n_units = n_whole + 4 * n_split;
     auto kern = k_bmu_table<L, THREADS, TOP2>;
     const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
     SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -644,7 +656,7 @@ int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* he
                                       reinterpret_cast<const uint4*>(ws + b.slots),
                                       reinterpret_cast<const uint32_t*>(ws + b.overflow), n,
                                       reinterpret_cast<u64*>(ws + b.keys),
-                                      TOP2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr, parts, part_len, n_units,
+                                      TOP2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr, parts, part_len, n_units, n_whole,
                                       reinterpret_cast<int*>(head + b.n_slots) + 3);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
