@@ -39,7 +39,8 @@
 
 namespace {
 
-constexpr int CHUNK = 128;  // samples a warp takes at a time
+constexpr int CHUNK = 128;  // samples a warp takes at a time ...
+constexpr int SMALL_CHUNK = 32;  // ... and near the end of a unit, so that its warps finish together
 constexpr int RING_STAGE = 224;  // bytes of one ring stage: 4 slots + 4 keys
 constexpr int SLOT_Q = SOM_SLOT_WORDS / 4;  // uint4 per slot
 
@@ -437,7 +438,12 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             k_begin += (int64_t)((unit - n_whole) & 3) * quarter;
             k_end = min(k_end, k_begin + quarter);
         }
-        const int n_chunks = (int)((k_end - k_begin + CHUNK - 1) / CHUNK);
+        // full chunks first; the last 64 samples per warp of the unit go out in small chunks
+        const int64_t unit_len = k_end > k_begin ? k_end - k_begin : 0;
+        const int64_t tail_len = min(unit_len, (int64_t)WARPS * 2 * SMALL_CHUNK);
+        const int n_big = (int)((unit_len - tail_len) / CHUNK);
+        const int64_t small_begin = k_begin + (int64_t)n_big * CHUNK;
+        const int n_chunks = n_big + (int)((k_end - small_begin + SMALL_CHUNK - 1) / SMALL_CHUNK);
 
         uint32_t curmask = 0;
         Scores base = L::seed(hn_sh, q);
@@ -446,8 +452,9 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
             chunk = __shfl_sync(0xffffffffu, chunk, 0);
             if (chunk >= n_chunks) break;
-            const int64_t w0 = k_begin + (int64_t)chunk * CHUNK;
-            const int rounds = (int)(min(k_end, w0 + CHUNK) - w0) >> 2;
+            const int64_t w0 = chunk < n_big ? k_begin + (int64_t)chunk * CHUNK
+                                              : small_begin + (int64_t)(chunk - n_big) * SMALL_CHUNK;
+            const int rounds = (int)(min(k_end, w0 + (chunk < n_big ? CHUNK : SMALL_CHUNK)) - w0) >> 2;
 
             // Ring feed: lanes 0..11 carry the twelve 16-byte pieces of a round's four slots,
             // lanes 12..13 the two 16-byte pieces of its four keys.
