@@ -108,22 +108,32 @@ def test_update_of_fp16_codebook(som_mod):
 
 
 def test_epoch_on_synthetic_workload(som_mod):
-    """One epoch of the tiny configuration end to end: search, update, norms, search again; the
-    update is checked against the oracle fed with the GPU's own assignment."""
+    """One epoch of the tiny configuration end to end: search, update, norms, search again.  The
+    update is driven by the ORACLE's assignment (no oracle input comes from the CUDA path; the
+    GPU's own assignment is checked against it first), and compared with the update oracle."""
+    from oracle import parity
+    from oracle import som_oracle as orc
     w = synth.CONFIGS[0]
     rows = cols = 16
     W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
     W_old = W.cpu().numpy().copy()
     b = synth.sample_csr(w.N, w.V, w.lam, w.seed, device="cuda")
+    ip, ix = b.indptr.cpu().numpy(), b.indices.cpu().numpy()
     h = som_mod.Som(w.V, w.M, W)
     h.norms()
-    bmu, _ = h.bmu(b.indptr, b.indices)
-    h.update(rows, cols, b.indptr, b.indices, bmu, 4)
+    bmu, dist = h.bmu(b.indptr, b.indices)
+    torch.cuda.synchronize()
+    nn = orc.norms(W_old, w.V, w.M)
+    top2 = orc.bmu(W_old, w.V, w.M, ip, ix, norms_=nn)
+    g = bmu.cpu().numpy()
+    rep = parity.check(g, dist.cpu().numpy(), top2, orc.dist_at(W_old, w.V, w.M, ip, ix, g.astype(np.int64), norms_=nn), w.M)
+    assert rep.ok, str(rep)
+    assign = top2.b1.astype(np.int32)
+    h.update(rows, cols, b.indptr, b.indices, torch.from_numpy(assign).cuda(), 4)
     h.norms()
     bmu2, dist2 = h.bmu(b.indptr, b.indices)
     torch.cuda.synchronize()
-    want = uorc.update(W_old, w.V, rows, cols, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
-                       bmu.cpu().numpy(), 4)
+    want = uorc.update(W_old, w.V, rows, cols, ip, ix, assign, 4)
     np.testing.assert_allclose(W.cpu().numpy().astype(np.float64), want, rtol=1e-6, atol=1e-12)
     assert np.isfinite(dist2.cpu().numpy()).all()
 
