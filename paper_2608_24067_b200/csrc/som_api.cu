@@ -356,7 +356,22 @@ int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indpt
     int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need);
     if (rc) return rc;
     h->norms_valid = 0;  // the codebook changes: som_norms must run before the next search
-    return som_launch_update(h, rows, cols, d_indptr, d_indices, n_samples, d_bmu, radius, planes, st);
+    // On small lattices with many samples the planes of the most frequent features are counted
+    // in shared memory (see k_upd_scatter_hot); the plan's selection phase names those features.
+    const int32_t* hot_slot = nullptr;
+    const int32_t* slot_feat = nullptr;
+    const int n_hot_slots = 16;
+    if (h->M * 4 <= 80 * 1024 && n_samples >= 8 * h->M && d_indices) {
+        SomPlanBuffers pb;
+        const size_t head_need = som_plan_head_bytes(h->V, n_hot_slots, &pb);
+        if ((rc = ensure_bytes(h, &h->head, &h->head_bytes, head_need))) return rc;
+        char* head = reinterpret_cast<char*>(h->head);
+        if ((rc = som_launch_plan_select(h, d_indptr, d_indices, n_samples, head, pb, n_hot_slots, 0, st))) return rc;
+        hot_slot = reinterpret_cast<const int32_t*>(head + pb.feat_slot);
+        slot_feat = reinterpret_cast<const int32_t*>(head + pb.slot_feat);
+    }
+    return som_launch_update(h, rows, cols, d_indptr, d_indices, n_samples, d_bmu, radius, planes, hot_slot,
+                             slot_feat, n_hot_slots, st);
 }
 
 int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,

@@ -104,4 +104,5 @@ int som_launch_validate(som_handle* h, const int32_t* indptr, const int32_t* ind
 size_t som_norms_workspace_bytes(const som_handle* h);
 size_t som_update_workspace_bytes(const som_handle* h, int64_t budget_bytes, int* planes_per_slab);
 int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, const int32_t* indices,
-                      int64_t n, const int32_t* bmu, int radius, int planes_per_slab, cudaStream_t st);
+                      int64_t n, const int32_t* bmu, int radius, int planes_per_slab, const int32_t* hot_slot,
+                      const int32_t* slot_feat, int n_hot_slots, cudaStream_t st);

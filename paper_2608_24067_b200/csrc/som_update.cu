@@ -62,7 +62,7 @@ __global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows
 // one thread per sample: its features inside [v0, v1) add 1 to the cell of its best unit
 __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                               int64_t n, const int32_t* __restrict__ bmu, int v0, int v1, int rows, int cols,
-                              float* __restrict__ num_t)
+                              const int32_t* __restrict__ hot_slot, float* __restrict__ num_t)
 {
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n) return;
@@ -74,7 +74,47 @@ __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t*
     for (int j = beg; j < end; ++j) {
         const int v = indices[j];
         if (v >= v1) break;  // ids ascend inside a row
-        if (v >= v0) atomicAdd(&num_t[(int64_t)(v - v0) * M + cell_t], 1.0f);
+        if (v >= v0 && !(hot_slot && hot_slot[v] >= 0)) atomicAdd(&num_t[(int64_t)(v - v0) * M + cell_t], 1.0f);
+    }
+}
+
+// The planes of the most frequent features take most of the batch's increments (a feature that
+// 84 % of a million samples carry puts 200 atomic adds on every cell of one 4096-cell plane, and
+// same-address atomics queue in L2).  Block (slice, group) counts the increments of its group of
+// hot features over its slice of the samples in shared memory, then adds each non-zero count to
+// the plane once.  hot_slot[v] = rank of feature v among the hot ones or -1; slot_feat is its
+// inverse.
+__global__ void k_upd_scatter_hot(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
+                                  int64_t n, const int32_t* __restrict__ bmu, int v0, int v1, int rows, int cols,
+                                  const int32_t* __restrict__ hot_slot, const int32_t* __restrict__ slot_feat,
+                                  int planes_per_block, float* __restrict__ num_t)
+{
+    extern __shared__ unsigned int cnt[];
+    const int M = rows * cols;
+    const int slot0 = blockIdx.y * planes_per_block;
+    for (int e = threadIdx.x; e < planes_per_block * M; e += blockDim.x) cnt[e] = 0u;
+    __syncthreads();
+    const int64_t per = (n + gridDim.x - 1) / gridDim.x;
+    const int64_t s_lo = (int64_t)blockIdx.x * per, s_hi = min(n, s_lo + per);
+    for (int64_t s = s_lo + threadIdx.x; s < s_hi; s += blockDim.x) {
+        const int c = bmu[s];
+        const int r = c / cols, q = c - r * cols;
+        const int cell_t = q * rows + r;  // transposed cell order
+        const int beg = indptr[s], end = indptr[s + 1];
+        for (int j = beg; j < end; ++j) {
+            const int slot = hot_slot[indices[j]] - slot0;
+            if (slot >= 0 && slot < planes_per_block) atomicAdd(&cnt[slot * M + cell_t], 1u);
+        }
+    }
+    __syncthreads();
+    for (int p = 0; p < planes_per_block; ++p) {
+        const int f = slot_feat[slot0 + p];
+        if (f < v0 || f >= v1) continue;  // unused slot, or a feature of another slab
+        float* plane = num_t + (int64_t)(f - v0) * M;
+        for (int e = threadIdx.x; e < M; e += blockDim.x) {
+            const unsigned int k = cnt[p * M + e];
+            if (k) atomicAdd(&plane[e], (float)k);
+        }
     }
 }
 
@@ -197,7 +237,8 @@ size_t som_update_workspace_bytes(const som_handle* h, int64_t budget_bytes, int
 }
 
 int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, const int32_t* indices,
-                      int64_t n, const int32_t* bmu, int radius, int planes_per_slab, cudaStream_t st)
+                      int64_t n, const int32_t* bmu, int radius, int planes_per_slab, const int32_t* hot_slot,
+                      const int32_t* slot_feat, int n_hot_slots, cudaStream_t st)
 {
     const int64_t M = h->M;
     const size_t mb = som_align_up((size_t)M * 4, 256);
@@ -245,8 +286,21 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         const int64_t planes = v1 - v0;
         SOM_CK(h, cudaMemsetAsync(slab_a, 0, (size_t)planes * M * 4, st));
         if (n > 0) {
-            k_upd_scatter<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols, slab_a);
+            k_upd_scatter<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols, hot_slot,
+                                                                 slab_a);
             h->launches += 1;
+            if (hot_slot) {
+                int ppb = (int)((160 * 1024) / (M * 4));
+                if (ppb > n_hot_slots) ppb = n_hot_slots;
+                const int groups = (n_hot_slots + ppb - 1) / ppb;
+                int slices = h->sm_count / groups;
+                slices = slices < 1 ? 1 : (slices > 16 ? 16 : slices);
+                const size_t sh = (size_t)ppb * M * 4;
+                SOM_CK(h, cudaFuncSetAttribute(k_upd_scatter_hot, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh));
+                k_upd_scatter_hot<<<dim3(slices, groups), 1024, sh, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols,
+                                                                        hot_slot, slot_feat, ppb, slab_a);
+                h->launches += 1;
+            }
         }
         float* x = three_passes<float, double>(h, slab_a, slab_b, planes, cols, rows, radius, st);
         float* y = (x == slab_a) ? slab_b : slab_a;

@@ -138,6 +138,21 @@ def test_epoch_on_synthetic_workload(som_mod):
     assert np.isfinite(dist2.cpu().numpy()).all()
 
 
+@pytest.mark.parametrize("mib", [0, 1])
+def test_update_with_frequent_features_counted_on_chip(som_mod, mib):
+    """Many samples on a small lattice with Zipf-shaped features: the most frequent features take the
+    shared-memory counting path; with a 1 MiB budget they are spread over four feature slabs."""
+    w = synth.CONFIGS[0]
+    rows = cols = 16
+    rng = np.random.default_rng(12)
+    W_old = rng.random(w.V * w.M).astype(np.float32)
+    b = synth.sample_csr(60_000, w.V, w.lam, 4, device="cpu")
+    bmu = rng.integers(0, w.M, size=b.n).astype(np.int32)
+    got = _run(som_mod, W_old, w.V, rows, cols, b.indptr.numpy(), b.indices.numpy(), bmu, 2,
+               options=((6, mib),) if mib else ())
+    _check(got, W_old, w.V, rows, cols, b.indptr.numpy(), b.indices.numpy(), bmu, 2, rtol=1e-6)
+
+
 def test_update_rejects_bad_lattice(som_mod):
     V, rows, cols = 10, 4, 4
     W = torch.zeros(V * rows * cols, device="cuda")
