@@ -115,3 +115,26 @@ def test_two_stage_needs_its_shadow_from_norms(som_mod):
     bmu, dist = h.bmu(b.indptr, b.indices)
     torch.cuda.synchronize()
     _check(W.cpu().numpy(), V, M, b, bmu.cpu().numpy(), dist.cpu().numpy(), np.arange(0, n, 13))
+
+
+def test_two_stage_option_leaves_the_other_entry_points_alone(som_mod):
+    """som_bmu2 never takes the two-stage route, an fp16-stored codebook has no use for it, and a
+    forced direct-load kernel overrides it: all must give what they give without the option."""
+    V, M, n = 2_000, 1_024, 30_000
+    W = synth.fill_codebook(V, M, 9, device="cuda")
+    b = synth.sample_csr(n, V, 7.0, 9, device="cuda")
+    plain, staged = som_mod.Som(V, M, W), som_mod.Som(V, M, W)
+    staged.set_option(7, 1)
+    plain.norms(); staged.norms()
+    for a, c in zip(plain.bmu2(b.indptr, b.indices), staged.bmu2(b.indptr, b.indices)):
+        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+    plain.set_option(0, 1); staged.set_option(0, 1)
+    for a, c in zip(plain.bmu(b.indptr, b.indices), staged.bmu(b.indptr, b.indices)):
+        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+    W16 = W.half()
+    h16a, h16b = som_mod.Som(V, M, W16), som_mod.Som(V, M, W16)
+    h16b.set_option(7, 1)
+    h16a.norms(); h16b.norms()
+    for a, c in zip(h16a.bmu(b.indptr, b.indices), h16b.bmu(b.indptr, b.indices)):
+        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+    torch.cuda.synchronize()
