@@ -154,12 +154,6 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     int rc = SOM_OK;
     if (h->timing && (rc = ensure_events(h))) return rc;
 
-    // Kernel selection.  The row-table kernel needs 128-bit aligned row segments (M % 4 == 0),
-    // feature ids that fit its 16-bit codes (V <= 65536) and enough (neuron range x sample
-    // part) units to occupy every SM; everything else goes to the direct-load kernel.  So do,
-    // in automatic mode, batches whose most frequent features cover too few feature instances
-    // for a shared-memory table to pay: there the direct-load kernel, bound by L2 bandwidth
-    // alone, is faster (measured cross-over: about half of the instances).
     // Two-stage search (option 7, fp32 storage): a first pass over the fp16 shadow of the
     // codebook with the wide fp16 layout, a certificate per sample, an exact fp32 pass for the
     // samples that fail it.  It needs the shadow written by the last som_norms and the row-table
@@ -167,6 +161,13 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     // the third).
     const bool two_stage_ok = h->opt_two_stage == 1 && h->shadow && h->shadow_valid && !h->Wh && !top2 &&
                               h->M % 128 == 0;
+    // Kernel selection.  The row-table kernel needs 128-bit aligned row segments (M % 4 == 0;
+    // M % 64 == 0 with fp16 storage), feature ids that fit its 16-bit codes (V <= 65536) and
+    // enough (neuron range x sample part) units to occupy every SM; everything else goes to
+    // the direct-load kernel.  So do, in automatic mode, batches whose most frequent features
+    // cover too few feature instances for a shared-memory table to pay: there the direct-load
+    // kernel, bound by L2 bandwidth alone, is faster (measured cross-over: about half of the
+    // instances).
     const SomTableGeom geom = som_table_geometry(h, two_stage_ok);
     bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
                      h->M < ((int64_t)1 << 30);
