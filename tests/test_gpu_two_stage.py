@@ -138,3 +138,18 @@ def test_two_stage_option_leaves_the_other_entry_points_alone(som_mod):
     for a, c in zip(h16a.bmu(b.indptr, b.indices), h16b.bmu(b.indptr, b.indices)):
         assert torch.equal(a.view(torch.int32), c.view(torch.int32))
     torch.cuda.synchronize()
+
+
+def test_two_stage_twins_that_fp16_cannot_tell_apart(som_mod):
+    """Second half of the map = first half scaled by 1 + 2^-12: the twins collapse (or nearly) in fp16,
+    but their fp32 distances differ by more than the near-tie band, so the certificate must send the
+    affected samples to the exact pass and the exact winner must come back."""
+    V, half, n = 4_000, 512, 40_000
+    Wh = synth.fill_codebook(V, half, 6, device="cuda").view(V, half)
+    W = torch.cat([Wh, Wh * (1.0 + 2.0 ** -12)], dim=1).contiguous().view(-1)
+    M = 2 * half
+    b = synth.sample_csr(n, V, 7.0, 6, device="cuda")
+    h, bmu, dist = _run(som_mod, W, V, M, b, True)
+    rep = _check(W.cpu().numpy(), V, M, b, bmu, dist, np.arange(0, n, 5))
+    assert rep.unambiguous > 0.9 * rep.n          # the twins are not near ties for the fp64 oracle
+    assert h.last_uncertain() > n // 2            # but the first pass cannot separate them
