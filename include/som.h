@@ -242,8 +242,9 @@ int som_last_cuda_error(const som_handle* h);
  * best first-pass scores are further apart than twice a bound on what the fp16 rounding and the fp32
  * summation can change (then the best unit of the exact weights is provably the same one), and searches
  * the other samples again with the fp32 weights.  Reported distances always come from the fp32 weights.
- * Needs M % 128 == 0 and the row-table kernel; som_bmu2 never uses it.  som_last_uncertain returns how many
- * samples the last two-stage search sent to its second pass.
+ * Needs M % 128 == 0 and the row-table kernel; som_bmu2 never uses it.  A two-stage call synchronises the
+ * stream a second time (it reads the length of the second pass's list back).  som_last_uncertain returns how
+ * many samples the last two-stage search sent to its second pass.
  */
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);
