@@ -171,6 +171,20 @@ int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indice
                  int32_t* h_bmu, float* h_min_dist, void* stream);
 
 /*
+ * som_bmu_host_async / som_host_sync - som_bmu_host for a STREAM of batches: the call returns once the
+ * batch's work is enqueued, and h_bmu / h_min_dist hold the results after som_host_sync(h).  The handle
+ * keeps two staging buffers and two copy streams of its own, so the host-to-device copy of one batch
+ * overlaps the search of the previous one and the results travel back while the next search runs
+ * (the paper streams the corpus from host memory, Section 4.2).  The search itself runs on `stream`.
+ * h_indptr / h_indices must stay unchanged until the NEXT call on the handle has returned (or
+ * som_host_sync); the output buffers of up to two calls are in flight at a time.  Use pinned host
+ * memory: pageable buffers make the copies synchronous and the overlap is lost.
+ */
+int som_bmu_host_async(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,
+                       int32_t* h_bmu, float* h_min_dist, void* stream);
+int som_host_sync(som_handle* h);
+
+/*
  * som_validate_csr - check the preconditions of som_bmu on a device-resident batch:
  * non-decreasing row pointers, ids in [0, V), strictly ascending inside each row
  * (Section 4.2, the sparse-binary CSR container).  Synchronises `stream`.

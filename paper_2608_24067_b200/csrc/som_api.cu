@@ -113,6 +113,18 @@ int som_destroy(som_handle* h)
     cudaFree(h->stage);
     cudaFree(h->head);
     cudaFree(h->shadow);
+    if (h->copy_stream) {
+        cudaStreamSynchronize(h->copy_stream);
+        cudaStreamSynchronize(h->back_stream);
+        for (int t = 0; t < 2; ++t) {
+            cudaEventDestroy(h->ev_h2d[t]);
+            cudaEventDestroy(h->ev_searched[t]);
+            cudaEventDestroy(h->ev_d2h[t]);
+            cudaFree(h->pipe_stage[t]);
+        }
+        cudaStreamDestroy(h->copy_stream);
+        cudaStreamDestroy(h->back_stream);
+    }
     cudaFree(h->wmax_bits);
     if (h->host_pair) cudaFreeHost(h->host_pair);
     if (h->events_made)
@@ -406,6 +418,76 @@ int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indice
     SOM_CK(h, cudaMemcpyAsync(h_bmu, d_bmu, (size_t)n_samples * 4, cudaMemcpyDeviceToHost, st));
     SOM_CK(h, cudaMemcpyAsync(h_min_dist, d_dist, (size_t)n_samples * 4, cudaMemcpyDeviceToHost, st));
     SOM_CK(h, cudaStreamSynchronize(st));
+    return SOM_OK;
+}
+
+// Pipelined host entry point: two staging buffers and two copy streams of the handle's own (one
+// per direction: a single in-order stream would hold the next batch's upload behind the previous
+// batch's download, which waits for its search), so that the host-to-device copy of one batch
+// overlaps the search of the previous one and the results travel back while the next search runs.
+static int pipe_setup(som_handle* h)
+{
+    if (h->copy_stream) return SOM_OK;
+    SOM_CK(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+    SOM_CK(h, cudaStreamCreateWithFlags(&h->back_stream, cudaStreamNonBlocking));
+    for (int t = 0; t < 2; ++t) {
+        SOM_CK(h, cudaEventCreateWithFlags(&h->ev_h2d[t], cudaEventDisableTiming));
+        SOM_CK(h, cudaEventCreateWithFlags(&h->ev_searched[t], cudaEventDisableTiming));
+        SOM_CK(h, cudaEventCreateWithFlags(&h->ev_d2h[t], cudaEventDisableTiming));
+    }
+    return SOM_OK;
+}
+
+int som_bmu_host_async(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,
+                       int32_t* h_bmu, float* h_min_dist, void* stream)
+{
+    if (!h || n_samples < 0) return SOM_ERR_INVALID_ARG;
+    if (n_samples == 0) return SOM_OK;
+    if (!h_indptr || !h_bmu || !h_min_dist) return SOM_ERR_INVALID_ARG;
+    if (h_indptr[0] != 0 || h_indptr[n_samples] < 0) return SOM_ERR_INVALID_ARG;
+    const int64_t nnz = h_indptr[n_samples];
+    if (nnz > 0 && !h_indices) return SOM_ERR_INVALID_ARG;
+    if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int rc = pipe_setup(h);
+    if (rc) return rc;
+    const int t = (int)(h->pipe_calls & 1);
+    // the buffer's previous batch (two calls ago) must have left it
+    if (h->pipe_calls >= 2) SOM_CK(h, cudaEventSynchronize(h->ev_d2h[t]));
+
+    const size_t b_ptr = som_align_up((size_t)(n_samples + 1) * 4, 256);
+    const size_t b_idx = som_align_up((size_t)(nnz > 0 ? nnz : 1) * 4, 256);
+    const size_t b_out = som_align_up((size_t)n_samples * 4, 256);
+    if ((rc = ensure_bytes(h, &h->pipe_stage[t], &h->pipe_stage_bytes[t], b_ptr + b_idx + 2 * b_out))) return rc;
+    char* base = reinterpret_cast<char*>(h->pipe_stage[t]);
+    int32_t* d_ptr = reinterpret_cast<int32_t*>(base);
+    int32_t* d_idx = reinterpret_cast<int32_t*>(base + b_ptr);
+    int32_t* d_bmu = reinterpret_cast<int32_t*>(base + b_ptr + b_idx);
+    float* d_dist = reinterpret_cast<float*>(base + b_ptr + b_idx + b_out);
+    SOM_CK(h, cudaMemcpyAsync(d_ptr, h_indptr, (size_t)(n_samples + 1) * 4, cudaMemcpyHostToDevice, h->copy_stream));
+    if (nnz > 0)
+        SOM_CK(h, cudaMemcpyAsync(d_idx, h_indices, (size_t)nnz * 4, cudaMemcpyHostToDevice, h->copy_stream));
+    SOM_CK(h, cudaEventRecord(h->ev_h2d[t], h->copy_stream));
+    SOM_CK(h, cudaStreamWaitEvent(st, h->ev_h2d[t], 0));
+    rc = som_bmu(h, d_ptr, d_idx, n_samples, d_bmu, d_dist, stream);
+    if (rc) return rc;
+    SOM_CK(h, cudaEventRecord(h->ev_searched[t], st));
+    SOM_CK(h, cudaStreamWaitEvent(h->back_stream, h->ev_searched[t], 0));
+    SOM_CK(h, cudaMemcpyAsync(h_bmu, d_bmu, (size_t)n_samples * 4, cudaMemcpyDeviceToHost, h->back_stream));
+    SOM_CK(h, cudaMemcpyAsync(h_min_dist, d_dist, (size_t)n_samples * 4, cudaMemcpyDeviceToHost, h->back_stream));
+    SOM_CK(h, cudaEventRecord(h->ev_d2h[t], h->back_stream));
+    h->pipe_calls += 1;
+    return SOM_OK;
+}
+
+int som_host_sync(som_handle* h)
+{
+    if (!h) return SOM_ERR_INVALID_ARG;
+    if (!h->copy_stream) return SOM_OK;
+    DeviceGuard g(h->device);
+    SOM_CK(h, cudaStreamSynchronize(h->copy_stream));
+    SOM_CK(h, cudaStreamSynchronize(h->back_stream));
     return SOM_OK;
 }
 

@@ -32,6 +32,12 @@ struct som_handle {
     size_t ws_bytes;
     void* stage;  // grow-only device staging for som_bmu_host
     size_t stage_bytes;
+    // pipelined host entry point (som_bmu_host_async): copy stream, two staging buffers, events
+    cudaStream_t copy_stream, back_stream;  // host-to-device and device-to-host
+    cudaEvent_t ev_h2d[2], ev_searched[2], ev_d2h[2];
+    void* pipe_stage[2];
+    size_t pipe_stage_bytes[2];
+    int64_t pipe_calls;
     void* head;  // small plan arrays that the selection phase fills before nnz is known
     size_t head_bytes;
 

@@ -25,6 +25,7 @@ EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
     "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain", "som_bmu_values",
+    "som_bmu_host_async", "som_host_sync",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -59,6 +60,10 @@ def load_library():
     lib.som_norms.argtypes = [P, P]
     lib.som_bmu.argtypes = [P, P, P, I64, P, P, P]
     lib.som_bmu_host.argtypes = [P, P, P, I64, P, P, P]
+    lib.som_bmu_host_async.argtypes = [P, P, P, I64, P, P, P]
+    lib.som_bmu_host_async.restype = INT
+    lib.som_host_sync.argtypes = [P]
+    lib.som_host_sync.restype = INT
     lib.som_bmu2.argtypes = [P, P, P, I64, P, P, P, P, P]
     lib.som_bmu2.restype = INT
     lib.som_bmu_values.argtypes = [P, P, P, P, I64, P, P, P]
@@ -211,6 +216,19 @@ class Som:
                                     _host_ptr(out_dist, torch.float32, "out_dist"), _stream_ptr(stream))
         self._check(rc, "som_bmu_host")
         return out_bmu, out_dist
+
+    def bmu_host_async(self, indptr: torch.Tensor, indices: torch.Tensor, out_bmu: torch.Tensor,
+                       out_dist: torch.Tensor, stream=None):
+        """som_bmu_host_async: pinned CPU tensors in and out; results are valid after host_sync()."""
+        n = indptr.numel() - 1
+        rc = self._lib.som_bmu_host_async(self._h, _host_ptr(indptr, torch.int32, "indptr"),
+                                          _host_ptr(indices, torch.int32, "indices"), n,
+                                          _host_ptr(out_bmu, torch.int32, "out_bmu"),
+                                          _host_ptr(out_dist, torch.float32, "out_dist"), _stream_ptr(stream))
+        self._check(rc, "som_bmu_host_async")
+
+    def host_sync(self):
+        self._check(self._lib.som_host_sync(self._h), "som_host_sync")
 
     def validate_csr(self, indptr: torch.Tensor, indices: torch.Tensor, stream=None) -> bool:
         n = indptr.numel() - 1

@@ -342,3 +342,23 @@ def test_batch_of_empty_samples(som_mod, variant):
     best = int(np.argmin(nn.astype(np.float32)))
     assert np.all(bmu.cpu().numpy() == best)
     np.testing.assert_allclose(dist.cpu().numpy(), np.float32(nn[best]), rtol=1e-6)
+
+
+def test_streamed_host_entry_point(som_mod):
+    """som_bmu_host_async over a stream of different batches equals som_bmu on each of them."""
+    w = synth.CONFIGS[0]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    h = som_mod.Som(w.V, w.M, W)
+    h.norms()
+    batches = [synth.sample_csr(4000 + 500 * k, w.V, w.lam, w.seed, device="cpu", first_sample=10_000 * k)
+               for k in range(5)]
+    pinned = [(b.indptr.pin_memory(), b.indices.pin_memory()) for b in batches]
+    outs = [(torch.empty(b.n, dtype=torch.int32).pin_memory(), torch.empty(b.n, dtype=torch.float32).pin_memory())
+            for b in batches]
+    for (ip, ix), (ob, od) in zip(pinned, outs):
+        h.bmu_host_async(ip, ix, ob, od)
+    h.host_sync()
+    for b, (ob, od) in zip(batches, outs):
+        d_bmu, d_dist = h.bmu(b.indptr.cuda(), b.indices.cuda())
+        torch.cuda.synchronize()
+        assert torch.equal(ob, d_bmu.cpu()) and torch.equal(od.view(torch.int32), d_dist.cpu().view(torch.int32))
