@@ -38,6 +38,14 @@ def test_host_only_calls_without_gpu():
     assert lib.som_create(ctypes.byref(out), 0, 0, None) == 1  # invalid arguments, checked first
     assert lib.som_norms(None, None) == 1
     assert lib.som_bmu(None, None, None, 0, None, None, None) == 1
+    assert lib.som_bmu2(None, None, None, 0, None, None, None, None, None) == 1
+    assert lib.som_bmu_values(None, None, None, None, 0, None, None, None) == 1
+    assert lib.som_update(None, 1, 1, None, None, 0, None, 1, None) == 1
+    assert lib.som_bmu_host_async(None, None, None, 0, None, None, None) == 1
+    assert lib.som_host_sync(None) == 1
+    assert lib.som_last_uncertain(None) == 0
+    assert lib.som_create_f16(ctypes.byref(out), 0, 0, None) == 1
+    assert lib.som_norms_noalloc(0, 0, None, None, None) == 1
 
 
 def test_no_signature_mentions_torch():
