@@ -224,6 +224,7 @@ def run_ours(args, w: synth.Workload):
         h.set_option(6, args.update_mib)
     if args.two_stage:
         h.set_option(7, 1)
+    plans = [h.plan(b.indptr, b.indices) for b in batches] if args.planned else []
     sample_values = []
     if args.values:
         for bi, b in enumerate(batches):
@@ -235,7 +236,9 @@ def run_ours(args, w: synth.Workload):
     def step(i):
         b = batches[i % n_batches]
         h.norms()
-        if args.values:
+        if args.planned:
+            plans[i % n_batches].bmu(out_bmu, out_dist)
+        elif args.values:
             h.bmu_values(b.indptr, b.indices, sample_values[i % n_batches])
         elif args.top2:
             h.bmu2(b.indptr, b.indices)
@@ -417,7 +420,8 @@ def run_ours(args, w: synth.Workload):
         "dtype": "f32" if args.store == "f32" else "f32 accumulate, f16-stored codebook",
         "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": nnz_mean,
-                   "step": "som_norms + %s on one batch" % ("som_bmu_values" if args.values else ("som_bmu2" if args.top2 else "som_bmu")),
+                   "step": "som_norms + %s on one batch" % ("som_bmu_planned (plans built once, outside)" if args.planned else
+                       ("som_bmu_values" if args.values else ("som_bmu2" if args.top2 else "som_bmu"))),
                    "replicas": ws,
                    "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
                        w.V * w.M * store_bytes / 1e6, batches[0].nnz * 4 / 1e6) if w.V * w.M * store_bytes > 126e6 else
@@ -470,6 +474,9 @@ def main():
                     help="skip the extra measurement of the two-stage search that the default run reports beside the headline")
     ap.add_argument("--values", action="store_true",
                     help="time som_bmu_values (sparse real-valued samples: seeded values in [0.25, 1.75)) instead of som_bmu")
+    ap.add_argument("--planned", action="store_true",
+                    help="epoch-loop mode: the batches' plans are built once (som_plan_create) outside the timed "
+                         "region and every step runs som_norms + som_bmu_planned")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
     ap.add_argument("--no-cpu-baseline", action="store_true")

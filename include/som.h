@@ -123,6 +123,28 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
              int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream);
 
 /*
+ * som_plan_create / som_bmu_planned / som_plan_destroy - a reusable batch plan for epoch loops.
+ * The per-batch preparation inside som_bmu (feature histogram, choice of the table's features, sort of the
+ * samples, re-encoded index lists: "the tile's merged feature lists", Section 3.3) depends on the batch
+ * alone, not on the codebook.  Training searches the same batches every epoch (Algorithm 2, step 2), so a
+ * caller can build each batch's plan once:
+ *   som_plan_create   builds the plan of the device-resident CSR batch (arguments as in som_bmu) in
+ *                     device memory of its own (about 70 bytes per sample) and synchronises `stream`.
+ *                     The plan BORROWS d_indptr / d_indices: they must stay valid and unchanged while
+ *                     the plan lives.  It is tied to the handle and to the handle's options and
+ *                     storage type at this moment.
+ *   som_bmu_planned   som_bmu for the plan's batch: same outputs (bit-identical to som_bmu's on the same
+ *                     batch), but only enqueues work on `stream` (no host synchronisation, no allocation).
+ *                     Two searches with the same plan must not overlap on the GPU.
+ *   som_plan_destroy  frees the plan (NULL is accepted); destroy plans before their handle.
+ */
+typedef struct som_plan som_plan; /* opaque */
+int som_plan_create(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+                    som_plan** out, void* stream);
+int som_bmu_planned(som_handle* h, som_plan* plan, int32_t* d_bmu, float* d_min_dist, void* stream);
+int som_plan_destroy(som_plan* plan);
+
+/*
  * som_bmu_values - the search for sparse REAL-VALUED samples (the paper's outlook, Section 7: "carrying
  * ||x||^2 and a values array alongside the feature indices"; its SparseFloat variant, Table 6):
  *   d_values   DEVICE pointer, fp32, parallel to d_indices: sample s has value d_values[k] at feature

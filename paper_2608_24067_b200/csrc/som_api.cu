@@ -354,6 +354,142 @@ int som_bmu_values(som_handle* h, const int32_t* d_indptr, const int32_t* d_indi
     return SOM_OK;
 }
 
+// ---- reusable batch plan ---------------------------------------------------------------------
+// The plan of a batch (hot set, sort, slots) depends on the batch alone, not on the codebook, so an
+// epoch loop that searches the same batches every epoch builds each plan once.
+struct som_plan {
+    som_handle* h;
+    int device;              // its own copy: the plan may outlive the handle until it is destroyed
+    const int32_t* indptr;   // borrowed
+    const int32_t* indices;  // borrowed
+    int64_t n, nnz;
+    int use_table;
+    int n_hot;
+    int f16;                 // storage layout the plan was built for
+    SomPlanBuffers pb;
+    char* head;
+    char* ws;                // table path: the plan's arrays; direct path: the keys
+};
+
+int som_plan_destroy(som_plan* p)
+{
+    if (!p) return SOM_OK;
+    DeviceGuard g(p->device);
+    cudaFree(p->head);
+    cudaFree(p->ws);
+    delete p;
+    return SOM_OK;
+}
+
+int som_plan_create(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
+                    som_plan** out, void* stream)
+{
+    if (!out) return SOM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!h || n_samples <= 0 || !d_indptr) return SOM_ERR_INVALID_ARG;
+    if (n_samples >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    som_plan* p = new (std::nothrow) som_plan();
+    if (!p) return SOM_ERR_INVALID_ARG;
+    p->h = h;
+    p->device = h->device;
+    p->indptr = d_indptr;
+    p->indices = d_indices;
+    p->n = n_samples;
+    p->f16 = h->Wh != nullptr;
+    int rc = SOM_OK;
+    // the same choice of kernel as som_bmu makes (see there)
+    const SomTableGeom geom = som_table_geometry(h, false);
+    p->n_hot = geom.n_hot;
+    bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
+                     h->M < ((int64_t)1 << 30);
+    if (use_table && h->opt_variant == 0) {
+        const int64_t units = ((h->M + geom.T - 1) / geom.T) * som_table_default_parts(n_samples, geom.T);
+        if (units < 2 * (int64_t)h->sm_count) use_table = false;
+    }
+    if (!h->host_pair && cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)) != cudaSuccess)
+        rc = SOM_ERR_CUDA;
+    if (!rc && use_table) {
+        const size_t head_need = som_plan_head_bytes(h->V, SOM_PLAN_MASK_FEATURES + geom.n_hot, &p->pb);
+        if (cudaMalloc(reinterpret_cast<void**>(&p->head), head_need) != cudaSuccess) rc = SOM_ERR_CUDA;
+        if (!rc) rc = som_launch_plan_select(h, d_indptr, d_indices, n_samples, p->head, p->pb,
+                                             SOM_PLAN_MASK_FEATURES, geom.n_hot, st);
+    }
+    if (!rc) {
+        cudaError_t e = cudaMemcpyAsync(h->host_pair, d_indptr, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(h->host_pair + 1, d_indptr + n_samples, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+        h->host_pair[2] = 0;
+        if (e == cudaSuccess && use_table)
+            e = cudaMemcpyAsync(h->host_pair + 2,
+                                reinterpret_cast<const int32_t*>(p->head + p->pb.n_slots) + SOM_PLAN_COVERED,
+                                sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) rc = SOM_ERR_CUDA;
+    }
+    if (!rc) {
+        p->nnz = (int64_t)h->host_pair[1] - (int64_t)h->host_pair[0];
+        if (p->nnz < 0 || (p->nnz > 0 && !d_indices)) rc = SOM_ERR_INVALID_ARG;
+    }
+    if (!rc && use_table) {
+        if (p->nnz + 6 * n_samples + 4 >= ((int64_t)1 << 31)) use_table = false;
+        const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 50;
+        if (h->opt_variant == 0 && (int64_t)h->host_pair[2] * 100 < cover_pct * p->nnz) use_table = false;
+    }
+    if (!rc) {
+        p->use_table = use_table ? 1 : 0;
+        const size_t need = use_table ? som_plan_workspace_bytes(n_samples, p->nnz, &p->pb)
+                                      : som_align_up((size_t)n_samples * sizeof(unsigned long long), 256);
+        if (cudaMalloc(reinterpret_cast<void**>(&p->ws), need) != cudaSuccess) rc = SOM_ERR_CUDA;
+        if (!rc && use_table)
+            rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, p->head, p->ws, p->pb,
+                                      SOM_PLAN_MASK_FEATURES, geom.n_hot, st);
+    }
+    if (rc) {
+        if (rc == SOM_ERR_CUDA && !h->last_cuda_error) h->last_cuda_error = (int)cudaGetLastError();
+        som_plan_destroy(p);
+        return rc;
+    }
+    *out = p;
+    return SOM_OK;
+}
+
+int som_bmu_planned(som_handle* h, som_plan* p, int32_t* d_bmu, float* d_min_dist, void* stream)
+{
+    if (!h || !p || p->h != h || !d_bmu || !d_min_dist) return SOM_ERR_INVALID_ARG;
+    if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
+    if (p->f16 != (h->Wh != nullptr)) return SOM_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int rc = SOM_OK;
+    if (h->timing && (rc = ensure_events(h))) return rc;
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
+    if (!p->use_table) {
+        unsigned long long* keys = reinterpret_cast<unsigned long long*>(p->ws);
+        SOM_CK(h, cudaMemsetAsync(keys, 0xFF, (size_t)p->n * sizeof(unsigned long long), st));
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+        if ((rc = som_launch_bmu_direct(h, p->indptr, p->indices, p->n, keys, nullptr, nullptr, st))) return rc;
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+        if ((rc = som_launch_finalize(h, p->indptr, p->indices, p->n, keys, d_bmu, d_min_dist, nullptr, st)))
+            return rc;
+    } else {
+        // the plan was built for a table of p->n_hot rows: the handle's options must still give it
+        if (som_table_geometry(h, false).n_hot != p->n_hot) return SOM_ERR_INVALID_ARG;
+        SOM_CK(h, cudaMemsetAsync(p->ws + p->pb.keys, 0xFF, (size_t)(p->n + 16) * sizeof(unsigned long long), st));
+        SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(p->head + p->pb.n_slots) + 3, 0, sizeof(int), st));
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, false, p->n, p->head, p->ws, p->pb, p->n_hot, false, st))) return rc;
+        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+        if ((rc = som_launch_finalize_sorted(h, p->indptr, p->indices, p->n, p->ws, p->pb, false, d_bmu,
+                                             d_min_dist, st)))
+            return rc;
+    }
+    if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
+    if (h->timing) h->ev_bmu_calls += 1;
+    return SOM_OK;
+}
+
 int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indptr, const int32_t* d_indices,
                int64_t n_samples, const int32_t* d_bmu, int32_t radius, void* stream)
 {

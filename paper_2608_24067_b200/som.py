@@ -25,7 +25,7 @@ EXPORTS = [
     "som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr", "som_get_norms",
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
     "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain", "som_bmu_values",
-    "som_bmu_host_async", "som_host_sync",
+    "som_bmu_host_async", "som_host_sync", "som_plan_create", "som_bmu_planned", "som_plan_destroy",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -64,6 +64,12 @@ def load_library():
     lib.som_bmu_host_async.restype = INT
     lib.som_host_sync.argtypes = [P]
     lib.som_host_sync.restype = INT
+    lib.som_plan_create.argtypes = [P, P, P, I64, ctypes.POINTER(P), P]
+    lib.som_plan_create.restype = INT
+    lib.som_bmu_planned.argtypes = [P, P, P, P, P]
+    lib.som_bmu_planned.restype = INT
+    lib.som_plan_destroy.argtypes = [P]
+    lib.som_plan_destroy.restype = INT
     lib.som_bmu2.argtypes = [P, P, P, I64, P, P, P, P, P]
     lib.som_bmu2.restype = INT
     lib.som_bmu_values.argtypes = [P, P, P, P, I64, P, P, P]
@@ -124,6 +130,43 @@ def norms_noalloc(V: int, M: int, codebook: torch.Tensor, out: torch.Tensor, str
     if rc != SOM_OK:
         raise SomError(rc, "som_norms_noalloc")
     return out
+
+
+class Plan:
+    """A batch plan (som_plan_create); search it with ``bmu()`` as often as the codebook changes."""
+
+    def __init__(self, som_handle: "Som", indptr: torch.Tensor, indices: torch.Tensor, stream=None):
+        self._som = som_handle
+        self._lib = som_handle._lib
+        self.indptr, self.indices = indptr, indices  # borrowed by the plan: keep them alive
+        self.n = indptr.numel() - 1
+        self._p = ctypes.c_void_p()
+        rc = self._lib.som_plan_create(som_handle._h, _dev_ptr(indptr, torch.int32, "indptr"),
+                                       _dev_ptr(indices, torch.int32, "indices"), self.n,
+                                       ctypes.byref(self._p), _stream_ptr(stream))
+        som_handle._check(rc, "som_plan_create")
+
+    def bmu(self, out_bmu: torch.Tensor | None = None, out_dist: torch.Tensor | None = None, stream=None):
+        dev = self._som.codebook.device
+        if out_bmu is None:
+            out_bmu = torch.empty(self.n, dtype=torch.int32, device=dev)
+        if out_dist is None:
+            out_dist = torch.empty(self.n, dtype=torch.float32, device=dev)
+        rc = self._lib.som_bmu_planned(self._som._h, self._p, _dev_ptr(out_bmu, torch.int32, "out_bmu"),
+                                       _dev_ptr(out_dist, torch.float32, "out_dist"), _stream_ptr(stream))
+        self._som._check(rc, "som_bmu_planned")
+        return out_bmu, out_dist
+
+    def destroy(self):
+        if self._p:
+            self._lib.som_plan_destroy(self._p)
+            self._p = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 class Som:
@@ -229,6 +272,10 @@ class Som:
 
     def host_sync(self):
         self._check(self._lib.som_host_sync(self._h), "som_host_sync")
+
+    def plan(self, indptr: torch.Tensor, indices: torch.Tensor, stream=None) -> "Plan":
+        """som_plan_create: a reusable plan of this device-resident batch (keeps the tensors alive)."""
+        return Plan(self, indptr, indices, stream)
 
     def validate_csr(self, indptr: torch.Tensor, indices: torch.Tensor, stream=None) -> bool:
         n = indptr.numel() - 1

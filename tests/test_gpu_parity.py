@@ -362,3 +362,33 @@ def test_streamed_host_entry_point(som_mod):
         d_bmu, d_dist = h.bmu(b.indptr.cuda(), b.indices.cuda())
         torch.cuda.synchronize()
         assert torch.equal(ob, d_bmu.cpu()) and torch.equal(od.view(torch.int32), d_dist.cpu().view(torch.int32))
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+def test_reusable_plan_matches_som_bmu(som_mod, variant):
+    """A plan built once serves several epochs: after each in-place change of the codebook (and
+    som_norms) the planned search equals som_bmu bit for bit, and both obey the oracle."""
+    V, M, n = 30_000, 1_024, 60_000
+    W = synth.fill_codebook(V, M, 4, device="cuda")
+    b = synth.sample_csr(n, V, 11.0, 4, device="cuda")
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, variant)
+    plan = h.plan(b.indptr, b.indices)
+    for epoch in range(3):
+        if epoch:
+            W.mul_(0.9)
+            W[epoch::7] += 0.01
+        h.norms()
+        p_bmu, p_dist = plan.bmu()
+        d_bmu, d_dist = h.bmu(b.indptr, b.indices)
+        torch.cuda.synchronize()
+        assert torch.equal(p_bmu, d_bmu) and torch.equal(p_dist.view(torch.int32), d_dist.view(torch.int32))
+    _check_against_oracle(W.cpu().numpy(), V, M, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
+                          p_bmu.cpu().numpy(), p_dist.cpu().numpy(), np.arange(0, n, 9))
+    plan.destroy()
+    # a plan is tied to its handle
+    other = som_mod.Som(V, M, W)
+    other.norms()
+    plan2 = h.plan(b.indptr, b.indices)
+    rc = other._lib.som_bmu_planned(other._h, plan2._p, p_bmu.data_ptr(), p_dist.data_ptr(), None)
+    assert rc == 1  # SOM_ERR_INVALID_ARG
