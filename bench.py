@@ -224,7 +224,10 @@ def run_ours(args, w: synth.Workload):
         h.set_option(6, args.update_mib)
     if args.two_stage:
         h.set_option(7, 1)
-    plans = [h.plan(b.indptr, b.indices) for b in batches] if args.planned else []
+    epoch_edge = int(round(w.M ** 0.5))
+    if args.epoch and epoch_edge * epoch_edge != w.M:
+        raise SystemExit("bench.py --epoch needs a square lattice")
+    plans = [h.plan(b.indptr, b.indices) for b in batches] if (args.planned or args.epoch) else []
     sample_values = []
     if args.values:
         for bi, b in enumerate(batches):
@@ -236,7 +239,10 @@ def run_ours(args, w: synth.Workload):
     def step(i):
         b = batches[i % n_batches]
         h.norms()
-        if args.planned:
+        if args.epoch:
+            plans[i % n_batches].bmu(out_bmu, out_dist)
+            h.update(epoch_edge, epoch_edge, b.indptr, b.indices, out_bmu, max(1, epoch_edge // 4))
+        elif args.planned:
             plans[i % n_batches].bmu(out_bmu, out_dist)
         elif args.values:
             h.bmu_values(b.indptr, b.indices, sample_values[i % n_batches])
@@ -312,7 +318,7 @@ def run_ours(args, w: synth.Workload):
     # ---- the same step with the two-stage search (library option 7), reported beside the headline ----
     two_stage = None
     if (args.store == "f32" and w.M % 128 == 0 and not args.top2 and not args.two_stage and not args.values
-            and not args.no_two_stage_leg):
+            and not args.epoch and not args.no_two_stage_leg):
         free_b, _ = torch.cuda.mem_get_info()
         if free_b > w.V * w.M * 2 + (4 << 30):
             try:
@@ -420,7 +426,8 @@ def run_ours(args, w: synth.Workload):
         "dtype": "f32" if args.store == "f32" else "f32 accumulate, f16-stored codebook",
         "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": nnz_mean,
-                   "step": "som_norms + %s on one batch" % ("som_bmu_planned (plans built once, outside)" if args.planned else
+                   "step": "som_norms + %s on one batch" % ("som_bmu_planned + som_update (a training-epoch step; plans built once, outside)" if args.epoch else
+                       "som_bmu_planned (plans built once, outside)" if args.planned else
                        ("som_bmu_values" if args.values else ("som_bmu2" if args.top2 else "som_bmu"))),
                    "replicas": ws,
                    "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
@@ -474,6 +481,9 @@ def main():
                     help="skip the extra measurement of the two-stage search that the default run reports beside the headline")
     ap.add_argument("--values", action="store_true",
                     help="time som_bmu_values (sparse real-valued samples: seeded values in [0.25, 1.75)) instead of som_bmu")
+    ap.add_argument("--epoch", action="store_true",
+                    help="time a whole training-epoch step on a square lattice: som_norms + som_bmu_planned + "
+                         "som_update (radius = edge / 4); implies --planned")
     ap.add_argument("--planned", action="store_true",
                     help="epoch-loop mode: the batches' plans are built once (som_plan_create) outside the timed "
                          "region and every step runs som_norms + som_bmu_planned")
