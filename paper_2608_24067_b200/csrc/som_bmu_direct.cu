@@ -4,7 +4,8 @@
 // a warp owns one sample at a time and a block of 32*VEC neurons; every lane keeps VEC
 // score accumulators in registers, seeded with ||w_i||^2 / 2, and for each active feature v
 // subtracts the contiguous segment W[v*M + i0 .. i0+VEC) fetched with one 128-bit load
-// (feature-major layout: the warp's 32 loads cover 512 contiguous bytes).  The per-block
+// (feature-major layout: the warp's 32 loads cover 512 contiguous bytes), four features at a
+// time so that their loads are in flight together.  The per-block
 // argmin is a warp-shuffle reduction on (score, index) with ties to the lower index, and
 // the cross-block combine is a 64-bit atomicMin on an order-preserving packed key, which is
 // commutative and associative and therefore deterministic.  No N x M score block is ever
@@ -58,7 +59,8 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
     float seed[VEC];
 #pragma unroll
     for (int k = 0; k < VEC; ++k) seed[k] = (i0 + k < M) ? hnorm[i0 + k] : inf;
-    const bool live = i0 < M;  // with VEC == 4, M % 4 == 0: all four or none
+    const bool live = i0 < M;  // with VEC >= 4, M % VEC == 0: all of the lane's neurons or none
+    const ST* W_lane = W + (live ? i0 : 0);
 
     const int64_t s0 = ((int64_t)blockIdx.x * DIRECT_WARPS + warp) * DIRECT_SAMPLES_PER_WARP;
     const int64_t s1 = min(n, s0 + DIRECT_SAMPLES_PER_WARP);
@@ -74,28 +76,59 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
             const int mine = (base + lane < end) ? indices[base + lane] : 0;
             const float mine_x = (VALUED && base + lane < end) ? values[base + lane] : 1.f;
             const int cnt = min(32, end - base);
-            for (int j = 0; j < cnt; ++j) {
-                const int v = __shfl_sync(0xffffffffu, mine, j);
-                const float x = VALUED ? __shfl_sync(0xffffffffu, mine_x, j) : 1.f;
-                const ST* p = W + (int64_t)v * M + i0;
-                if (VEC == 4) {
-                    if (live) {
-                        float w[4];
-                        load4(p, w);
-                        if (VALUED) {
-                            acc[0] = fmaf(-x, w[0], acc[0]);
-                            acc[1 % VEC] = fmaf(-x, w[1], acc[1 % VEC]);
-                            acc[2 % VEC] = fmaf(-x, w[2], acc[2 % VEC]);
-                            acc[3 % VEC] = fmaf(-x, w[3], acc[3 % VEC]);
+            int j = 0;
+            // four features at a time: their row segments are in flight together, the
+            // subtractions keep the ascending feature order
+            for (; j + 4 <= cnt; j += 4) {
+                int v[4];
+                float x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    v[u] = __shfl_sync(0xffffffffu, mine, j + u);
+                    x[u] = VALUED ? __shfl_sync(0xffffffffu, mine_x, j + u) : 1.f;
+                }
+                if (live) {
+                    float w[4][VEC];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const ST* p = W_lane + (int64_t)v[u] * M;
+                        if (VEC >= 4) {
+#pragma unroll
+                            for (int g = 0; g < VEC / 4; ++g) {
+                                float t[4];
+                                load4(p + 4 * g, t);
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) w[u][(4 * g + k) % VEC] = t[k];
+                            }
                         } else {
-                            acc[0] -= w[0];
-                            acc[1 % VEC] -= w[1];
-                            acc[2 % VEC] -= w[2];
-                            acc[3 % VEC] -= w[3];
+                            w[u][0] = som_weight(p);
                         }
                     }
-                } else {
-                    if (live) acc[0] = VALUED ? fmaf(-x, som_weight(p), acc[0]) : acc[0] - som_weight(p);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+#pragma unroll
+                        for (int k = 0; k < VEC; ++k)
+                            acc[k] = VALUED ? fmaf(-x[u], w[u][k], acc[k]) : acc[k] - w[u][k];
+                }
+            }
+            for (; j < cnt; ++j) {
+                const int v = __shfl_sync(0xffffffffu, mine, j);
+                const float x = VALUED ? __shfl_sync(0xffffffffu, mine_x, j) : 1.f;
+                if (live) {
+                    const ST* p = W_lane + (int64_t)v * M;
+                    if (VEC >= 4) {
+#pragma unroll
+                        for (int g = 0; g < VEC / 4; ++g) {
+                            float t[4];
+                            load4(p + 4 * g, t);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                acc[(4 * g + k) % VEC] = VALUED ? fmaf(-x, t[k], acc[(4 * g + k) % VEC])
+                                                                : acc[(4 * g + k) % VEC] - t[k];
+                        }
+                    } else {
+                        acc[0] = VALUED ? fmaf(-x, som_weight(p), acc[0]) : acc[0] - som_weight(p);
+                    }
                 }
             }
         }
