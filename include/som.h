@@ -270,7 +270,7 @@ int som_last_cuda_error(const som_handle* h);
  * 8, 16, where 16 needs M % 128 == 0); key 4 = sample parts per
  * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
  * feature instances that the row table's features must cover for the row-table kernel to be taken
- * (0 = default 50; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
+ * (0 = default 60; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
  * slab buffers in MiB (0 = default 4096); key 7 = two-stage search for fp32 storage (0 = off, the default;
  * 1 = on): som_norms then also keeps an fp16 copy of the codebook (V*M*2 more bytes of device memory,
  * allocated by this call, which fails with SOM_ERR_CUDA if they cannot be had) and the largest |weight|;

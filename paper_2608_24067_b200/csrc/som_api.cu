@@ -216,7 +216,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (nnz < 0) return SOM_ERR_INVALID_ARG;
         if (nnz + 6 * n_samples + 4 >= ((int64_t)1 << 31)) use_table = false;
         if (nnz > 0 && !d_indices) return SOM_ERR_INVALID_ARG;
-        const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 50;
+        const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 60;
         if (h->opt_variant == 0 && (int64_t)h->host_pair[2] * 100 < cover_pct * nnz) use_table = false;
     }
 
@@ -434,7 +434,7 @@ int som_plan_create(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     }
     if (!rc && use_table) {
         if (p->nnz + 6 * n_samples + 4 >= ((int64_t)1 << 31)) use_table = false;
-        const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 50;
+        const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 60;
         if (h->opt_variant == 0 && (int64_t)h->host_pair[2] * 100 < cover_pct * p->nnz) use_table = false;
     }
     if (!rc) {

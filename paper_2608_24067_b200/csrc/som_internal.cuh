@@ -56,7 +56,7 @@ struct som_handle {
     int plan_attr_set;
     int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)
     int64_t opt_two_stage;  // 0 = off, 1 = on where it applies (fp32 storage, M % 128 == 0, memory for the shadow)
-    int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 50)
+    int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 60)
     int32_t* host_pair;    // pinned, 4 ints: read-back of indptr[0], indptr[n], covered instances, uncertain samples
 };
 
