@@ -20,6 +20,8 @@
 // between passes are fp32.  Whether a neuron's blurred denominator is zero is decided exactly,
 // from an integer box count of the occupied cells over the reach of three passes (3 * radius):
 // a running sum that subtracts can leave a rounding residue where the exact sum is zero.
+// Lattices of up to 128 x 128 cells replace steps 2-4 by one kernel that blurs a plane in shared
+// memory (k_upd_blur_fused): one read and one write of the plane instead of seven.
 #include "som_internal.cuh"
 
 namespace {
@@ -178,6 +180,182 @@ __global__ void k_box_pass_divide(const float* __restrict__ in, int64_t planes, 
     }
 }
 
+// Small lattices: the whole blur of a plane in shared memory.  A block takes one plane at a time:
+// it loads the scattered counts (transposed cell order) into an fp64 buffer, runs the three box
+// passes along each axis between two fp64 buffers (counts and their window sums are integers, so
+// fp64 holds them exactly up to 2^53 and the order of the passes does not matter), multiplies by
+// the reciprocal denominator and writes the new weights: one read and one write of the plane
+// instead of seven trips through DRAM.  A line is cut into `seg` segments, each walked by its own
+// thread with a running window sum started from a plain sum over its first window, so that a
+// 64 x 64 plane keeps 256 threads busy; the row pitch is odd (in doubles), which keeps the walks
+// along either axis at the two shared-memory wavefronts a warp's 64-bit accesses need anyway.
+constexpr int FUSED_THREADS = 256;
+constexpr int FUSED_THREADS_WIDE = 1024;
+
+constexpr int FUSED_PREFETCH = 16;  // cells per thread held in registers: planes of up to 4096 cells
+
+// lines of `len` cells: cell j of line l at buf[l * line_stride + j * cell_stride]
+template <typename BT>
+__device__ __forceinline__ void box_lines(const BT* __restrict__ in, BT* __restrict__ out, int n_lines,
+                                          int len, int line_stride, int cell_stride, int radius, int seg)
+{
+    const int seg_len = (len + seg - 1) / seg;
+    for (int job = threadIdx.x; job < n_lines * seg; job += blockDim.x) {
+        const int line = job % n_lines;
+        const int a = (job / n_lines) * seg_len;
+        const int b = min(len, a + seg_len);
+        if (a >= b) continue;
+        const BT* src = in + line * line_stride;
+        BT* dst = out + line * line_stride;
+        const int lo = max(0, a - radius), hi = min(len - 1, a + radius);
+        double s0 = 0.0, s1 = 0.0;
+        const BT* p = src + lo * cell_stride;
+        int j = lo;
+        for (; j + 1 <= hi; j += 2, p += 2 * cell_stride) {
+            s0 += (double)p[0];
+            s1 += (double)p[cell_stride];
+        }
+        if (j <= hi) s0 += (double)p[0];
+        double sum = s0 + s1;
+        BT* pd = dst + a * cell_stride;
+        *pd = (BT)sum;
+        pd += cell_stride;
+        const BT* pe = src + (a + 1 + radius) * cell_stride;  // the cell entering the window
+        const BT* pl = src + (a - radius) * cell_stride;      // the cell leaving it
+        // i < len - radius: a cell enters; i > radius: a cell leaves
+        for (int i = a + 1; i < b; ++i, pe += cell_stride, pl += cell_stride, pd += cell_stride) {
+            const double enter = (i < len - radius) ? (double)*pe : 0.0;
+            const double leave = (i > radius) ? (double)*pl : 0.0;
+            sum += enter - leave;
+            *pd = (BT)sum;
+        }
+    }
+}
+
+// BT: type of the two plane buffers (double: exact; float: rounded between passes like the
+// device-memory route, for planes too large for two fp64 buffers); running sums are fp64 either way.
+template <typename ST, typename BT, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+k_upd_blur_fused(const float* __restrict__ slab, int planes, int rows, int cols, int radius, int seg_r, int seg_c,
+                 const double* __restrict__ rden, ST* __restrict__ W, int v0)
+{
+    extern __shared__ __align__(16) unsigned char fused_raw[];
+    const int pitch = cols | 1;  // odd, in cells
+    const int M = rows * cols;   // <= FUSED_PREFETCH * THREADS
+    BT* A = reinterpret_cast<BT*>(fused_raw);
+    BT* B = A + rows * pitch;
+    // the next plane's counts wait in registers while the current plane is blurred
+    float pre[FUSED_PREFETCH];
+    if ((int)blockIdx.x < planes) {
+        const float* src = slab + (int64_t)blockIdx.x * M;
+#pragma unroll
+        for (int k = 0; k < FUSED_PREFETCH; ++k) {
+            const int g = threadIdx.x + k * THREADS;
+            pre[k] = g < M ? __ldg(src + g) : 0.f;
+        }
+    }
+    // cell (r, c) of this thread's k-th element, in transposed order (g = c * rows + r) and in
+    // neuron order (i = r * cols + c): advanced by THREADS per element without divisions
+    const int t_c0 = threadIdx.x / rows, t_r0 = threadIdx.x % rows;
+    const int t_dc = THREADS / rows, t_dr = THREADS % rows;
+    const int n_r0 = threadIdx.x / cols, n_c0 = threadIdx.x % cols;
+    const int n_dr = THREADS / cols, n_dc = THREADS % cols;
+    for (int plane = blockIdx.x; plane < planes; plane += gridDim.x) {
+        {
+            int r = t_r0, c = t_c0;
+#pragma unroll
+            for (int k = 0; k < FUSED_PREFETCH; ++k) {
+                if ((int)threadIdx.x + k * THREADS < M) A[r * pitch + c] = (BT)pre[k];
+                r += t_dr; c += t_dc;
+                if (r >= rows) { r -= rows; c += 1; }
+            }
+        }
+        __syncthreads();
+        if (plane + (int)gridDim.x < planes) {
+            const float* src = slab + (int64_t)(plane + gridDim.x) * M;
+#pragma unroll
+            for (int k = 0; k < FUSED_PREFETCH; ++k) {
+                const int g = threadIdx.x + k * THREADS;
+                pre[k] = g < M ? __ldg(src + g) : 0.f;
+            }
+        }
+        BT* x = A;
+        BT* y = B;
+        for (int pass = 0; pass < 3; ++pass) {  // along the lattice rows: a line is a row
+            box_lines(x, y, rows, cols, pitch, 1, radius, seg_r);
+            __syncthreads();
+            BT* t = x; x = y; y = t;
+        }
+        for (int pass = 0; pass < 3; ++pass) {  // along the lattice columns: a line is a column
+            box_lines(x, y, cols, rows, 1, pitch, radius, seg_c);
+            __syncthreads();
+            BT* t = x; x = y; y = t;
+        }
+        ST* dst = W + (int64_t)(v0 + plane) * M;
+        {
+            int r = n_r0, c = n_c0;
+            for (int i = threadIdx.x; i < M; i += THREADS) {
+                const double rd = rden[i];
+                if (rd != 0.0) dst[i] = (ST)(float)((double)x[r * pitch + c] * rd);
+                r += n_dr; c += n_dc;
+                if (c >= cols) { c -= cols; r += 1; }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// The denominator's route on a small lattice, one block: blur the sample counts (transposed cell
+// order) like a numerator plane, count the occupied cells within the reach of three passes
+// (3 * radius) along each axis with the same box walk (the counts are integers, exact in fp64), and
+// write the reciprocal of the blurred denominator where the reach is not empty, else 0 (= keep).
+__global__ void __launch_bounds__(FUSED_THREADS)
+k_upd_den_fused(const float* __restrict__ den_t, const int32_t* __restrict__ occ, int rows, int cols, int radius,
+                int seg_r, int seg_c, double* __restrict__ rden)
+{
+    extern __shared__ __align__(16) unsigned char fused_raw[];
+    const int pitch = cols | 1;
+    const int M = rows * cols;
+    double* A = reinterpret_cast<double*>(fused_raw);
+    double* B = A + rows * pitch;
+    double* C = A + 2 * rows * pitch;
+    for (int g = threadIdx.x; g < M; g += blockDim.x) {
+        const int c = g / rows, r = g - c * rows;
+        A[r * pitch + c] = (double)den_t[g];
+    }
+    __syncthreads();
+    double* x = A;
+    double* y = B;
+    for (int pass = 0; pass < 3; ++pass) {
+        box_lines(x, y, rows, cols, pitch, 1, radius, seg_r);
+        __syncthreads();
+        double* t = x; x = y; y = t;
+    }
+    for (int pass = 0; pass < 3; ++pass) {
+        box_lines(x, y, cols, rows, 1, pitch, radius, seg_c);
+        __syncthreads();
+        double* t = x; x = y; y = t;
+    }
+    for (int i = threadIdx.x; i < M; i += blockDim.x) {
+        const int r = i / cols, c = i - r * cols;
+        C[r * pitch + c] = x[r * pitch + c];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < M; i += blockDim.x) {
+        const int r = i / cols, c = i - r * cols;
+        A[r * pitch + c] = occ[i] > 0 ? 1.0 : 0.0;
+    }
+    __syncthreads();
+    box_lines(A, B, rows, cols, pitch, 1, 3 * radius, seg_r);
+    __syncthreads();
+    box_lines(B, A, cols, rows, 1, pitch, 3 * radius, seg_c);
+    __syncthreads();
+    for (int i = threadIdx.x; i < M; i += blockDim.x) {
+        const int r = i / cols, c = i - r * cols;
+        rden[i] = A[r * pitch + c] > 0.0 ? 1.0 / C[r * pitch + c] : 0.0;
+    }
+}
+
 // [plane][a][b] -> [plane][b][a] through 32 x 32 shared-memory tiles
 template <typename T>
 __global__ void k_transpose(const T* __restrict__ in, T* __restrict__ out, int a, int b)
@@ -264,20 +442,35 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         }
         h->launches += 1;
     }
-    float* d = three_passes<float, double>(h, den_a, den_b, 1, cols, rows, radius, st);  // along the lattice rows
-    float* d_other = (d == den_a) ? den_b : den_a;
-    transpose<float>(h, d, d_other, 1, cols, rows, st);
-    float* den_blurred = three_passes<float, double>(h, d_other, d, 1, rows, cols, radius, st);
-    // occupied cells within 3 * radius along each axis (exact integer counts; the count of a cell
-    // is at most M, so int32 suffices)
-    const int reach_r = 3 * radius;
-    k_box_pass<int32_t, int32_t><<<blocks_for(cols), UPD_THREADS, 0, st>>>(occ_a, occ_b, 1, rows, cols, reach_r);
-    transpose<int32_t>(h, occ_b, occ_c, 1, rows, cols, st);
-    k_box_pass<int32_t, int32_t><<<blocks_for(rows), UPD_THREADS, 0, st>>>(occ_c, occ_b, 1, cols, rows, reach_r);
-    transpose<int32_t>(h, occ_b, occ_c, 1, cols, rows, st);  // occ_c: reach count in neuron order
     double* rden = reinterpret_cast<double*>(ws + 6 * mb);
-    k_upd_reciprocal<<<blocks_for(M), UPD_THREADS, 0, st>>>(den_blurred, occ_c, M, rden);
-    h->launches += 3;
+    // planes of up to 4096 cells are blurred on chip in fp64 buffers by 256 threads, planes of up to
+    // 16384 cells in fp32 buffers by 1024 threads; larger ones take the passes through device memory
+    const int wide = M > FUSED_PREFETCH * FUSED_THREADS;
+    const int f_threads = wide ? FUSED_THREADS_WIDE : FUSED_THREADS;
+    const bool fused = M <= FUSED_PREFETCH * f_threads && rows <= f_threads && cols <= f_threads;
+    const int seg_r = f_threads / rows > 1 ? f_threads / rows : 1;  // segments per lattice row
+    const int seg_c = f_threads / cols > 1 ? f_threads / cols : 1;  // segments per lattice column
+    const size_t plane_sh = (size_t)rows * (cols | 1) * (wide ? sizeof(float) : sizeof(double));
+    if (fused && !wide) {
+        SOM_CK(h, cudaFuncSetAttribute(k_upd_den_fused, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)(3 * plane_sh)));
+        k_upd_den_fused<<<1, FUSED_THREADS, 3 * plane_sh, st>>>(den_a, occ_a, rows, cols, radius, seg_r, seg_c, rden);
+        h->launches += 1;
+    } else {
+        float* d = three_passes<float, double>(h, den_a, den_b, 1, cols, rows, radius, st);  // along the lattice rows
+        float* d_other = (d == den_a) ? den_b : den_a;
+        transpose<float>(h, d, d_other, 1, cols, rows, st);
+        float* den_blurred = three_passes<float, double>(h, d_other, d, 1, rows, cols, radius, st);
+        // occupied cells within 3 * radius along each axis (exact integer counts; the count of a cell
+        // is at most M, so int32 suffices)
+        const int reach_r = 3 * radius;
+        k_box_pass<int32_t, int32_t><<<blocks_for(cols), UPD_THREADS, 0, st>>>(occ_a, occ_b, 1, rows, cols, reach_r);
+        transpose<int32_t>(h, occ_b, occ_c, 1, rows, cols, st);
+        k_box_pass<int32_t, int32_t><<<blocks_for(rows), UPD_THREADS, 0, st>>>(occ_c, occ_b, 1, cols, rows, reach_r);
+        transpose<int32_t>(h, occ_b, occ_c, 1, cols, rows, st);  // occ_c: reach count in neuron order
+        k_upd_reciprocal<<<blocks_for(M), UPD_THREADS, 0, st>>>(den_blurred, occ_c, M, rden);
+        h->launches += 3;
+    }
     SOM_CK(h, cudaGetLastError());
 
     // ---- numerator, slab by slab ------------------------------------------------------------------
@@ -301,6 +494,28 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
                                                                         hot_slot, slot_feat, ppb, slab_a);
                 h->launches += 1;
             }
+        }
+        // small lattices: everything after the scatter in one kernel, a plane at a time on chip
+        const size_t fused_sh = 2 * plane_sh;
+        if (fused) {
+            const int per_sm = (int)((size_t)216 * 1024 / (fused_sh + 1024));
+            int64_t grid = (int64_t)h->sm_count * per_sm;
+            if (grid > planes) grid = planes;
+#define SOM_FUSED(ST_, BT_, THREADS_, W_)                                                                       \
+    do {                                                                                                        \
+        SOM_CK(h, cudaFuncSetAttribute(k_upd_blur_fused<ST_, BT_, THREADS_>,                                    \
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused_sh));            \
+        k_upd_blur_fused<ST_, BT_, THREADS_><<<(unsigned)grid, THREADS_, fused_sh, st>>>(                       \
+            slab_a, (int)planes, rows, cols, radius, seg_r, seg_c, rden, W_, v0);                               \
+    } while (0)
+            if (h->Wh && wide) SOM_FUSED(__half, float, FUSED_THREADS_WIDE, const_cast<__half*>(h->Wh));
+            else if (h->Wh) SOM_FUSED(__half, double, FUSED_THREADS, const_cast<__half*>(h->Wh));
+            else if (wide) SOM_FUSED(float, float, FUSED_THREADS_WIDE, const_cast<float*>(h->W));
+            else SOM_FUSED(float, double, FUSED_THREADS, const_cast<float*>(h->W));
+#undef SOM_FUSED
+            h->launches += 1;
+            SOM_CK(h, cudaGetLastError());
+            continue;
         }
         float* x = three_passes<float, double>(h, slab_a, slab_b, planes, cols, rows, radius, st);
         float* y = (x == slab_a) ? slab_b : slab_a;

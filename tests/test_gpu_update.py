@@ -72,7 +72,11 @@ def _check(got, W_old_stored, V, rows, cols, indptr, indices, bmu, radius, rtol)
 @pytest.mark.parametrize("V,rows,cols,n,radius", [
     (40, 8, 8, 300, 1), (64, 16, 16, 2000, 2), (33, 12, 20, 500, 3), (50, 32, 32, 5000, 5),
     (20, 7, 5, 100, 1), (17, 16, 16, 400, 16), (25, 1, 40, 200, 2), (25, 40, 1, 200, 2),
-    (30, 9, 9, 0, 1), (12, 64, 64, 3000, 0), (70, 33, 65, 4000, 4)])
+    (30, 9, 9, 0, 1), (12, 64, 64, 3000, 0), (70, 33, 65, 4000, 4),
+    # more than 4096 cells: fp32 plane buffers in shared memory; more than 16384: the passes go
+    # through device memory
+    (6, 72, 80, 3000, 3), (5, 66, 64, 2000, 70), (4, 300, 20, 1500, 2), (3, 128, 128, 4000, 9),
+    (3, 130, 130, 2000, 4), (2, 2000, 9, 1500, 2)])
 def test_update_matches_oracle(som_mod, V, rows, cols, n, radius):
     indptr, indices, bmu, W_old = _problem(V * 7 + rows, V, rows, cols, n)
     got = _run(som_mod, W_old, V, rows, cols, indptr, indices, bmu, radius)
