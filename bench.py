@@ -9,6 +9,7 @@ som_bmu (plan, fused search, combine/finalize).  Prints ONE JSON line on rank 0.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -489,17 +490,18 @@ def main():
                          "region and every step runs som_norms + som_bmu_planned")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="samples per batch instead of the configuration's (a sweep variant, named in the workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]
     if args.features == "uniform":
-        import dataclasses
         w = dataclasses.replace(w, name=w.name + "-uniform", zipf_s=0.0)
+    if args.batch > 0:
+        w = dataclasses.replace(w, name="%s-batch%d" % (w.name, args.batch), batch=args.batch, N=max(w.N, args.batch))
     if args.zipf_s is not None:
-        import dataclasses
         w = dataclasses.replace(w, name="%s-zipf%g" % (w.name, args.zipf_s), zipf_s=args.zipf_s)
     if args.store == "f16":
-        import dataclasses
         w = dataclasses.replace(w, name=w.name + "-f16")
     if args.impl == "reference":
         run_reference(args, w)
