@@ -151,14 +151,24 @@ k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_s
     for (int k = 0; k < VEC; ++k) out[k] = acc[k];
 }
 
+// 32 neurons x 8 groups of splits per block: group g adds splits g, g + 8, ... in order, then
+// the eight group sums are added in order (a fixed order: the result does not depend on the run)
+constexpr int COMBINE_GROUPS = 8;
 __global__ void k_norms_combine(const double* __restrict__ partial, int64_t M, int splits,
                                 double* __restrict__ norm64, float* __restrict__ norm32,
                                 float* __restrict__ hnorm)
 {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= M) return;
+    __shared__ double sh[COMBINE_GROUPS][33];
+    const int64_t i = (int64_t)blockIdx.x * 32 + threadIdx.x;
     double s = 0.0;
-    for (int k = 0; k < splits; ++k) s += partial[(int64_t)k * M + i];
+    if (i < M)
+        for (int k = threadIdx.y; k < splits; k += COMBINE_GROUPS) s += partial[(int64_t)k * M + i];
+    sh[threadIdx.y][threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.y != 0 || i >= M) return;
+    s = sh[0][threadIdx.x];
+#pragma unroll
+    for (int g = 1; g < COMBINE_GROUPS; ++g) s += sh[g][threadIdx.x];
     norm64[i] = s;
     norm32[i] = (float)s;
     hnorm[i] = (float)(0.5 * s);
@@ -216,8 +226,8 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
         k_norms_partial<1, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
                                                                  nullptr, nullptr);
     SOM_CK(h, cudaGetLastError());
-    const int64_t blocks = (h->M + 255) / 256;
-    k_norms_combine<<<(unsigned)blocks, 256, 0, st>>>(partial, h->M, p.splits, h->norm64, h->norm32,
+    const int64_t blocks = (h->M + 31) / 32;
+    k_norms_combine<<<(unsigned)blocks, dim3(32, COMBINE_GROUPS), 0, st>>>(partial, h->M, p.splits, h->norm64, h->norm32,
                                                       h->hnorm);
     SOM_CK(h, cudaGetLastError());
     h->launches += 2;

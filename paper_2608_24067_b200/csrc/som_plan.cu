@@ -109,9 +109,17 @@ __device__ void kth_largest(const uint32_t* __restrict__ c, int V, int K, uint32
 }
 
 __global__ void __launch_bounds__(1024)
-k_select_hot(const uint32_t* __restrict__ feat_count, int V, int n_mask, int n_hot,
+k_select_hot(const uint32_t* __restrict__ feat_count_g, int V, int n_mask, int n_hot, int use_smem,
              int32_t* __restrict__ feat_slot, int32_t* __restrict__ slot_feat, int32_t* __restrict__ n_slots)
 {
+    // the counts are walked thirteen times: keep them in shared memory when they fit
+    extern __shared__ uint32_t sh_counts[];
+    const uint32_t* feat_count = feat_count_g;
+    if (use_smem) {
+        for (int v = threadIdx.x; v < V; v += blockDim.x) sh_counts[v] = feat_count_g[v];
+        feat_count = sh_counts;
+        __syncthreads();
+    }
     __shared__ uint32_t sh_hist[256];
     __shared__ uint32_t sh_state[4];
     __shared__ int warp_sums[32];
@@ -453,7 +461,12 @@ int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* 
         SOM_CK(h, cudaGetLastError());
     }
     // 2. select
-    k_select_hot<<<1, 1024, 0, st>>>(feat_count, h->V, n_mask, n_hot, feat_slot, slot_feat, n_slots);
+    const size_t counts_sh = (size_t)h->V * 4;
+    const int counts_fit = counts_sh <= 200 * 1024;
+    if (counts_fit)
+        SOM_CK(h, cudaFuncSetAttribute(k_select_hot, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)counts_sh));
+    k_select_hot<<<1, 1024, counts_fit ? counts_sh : 0, st>>>(feat_count, h->V, n_mask, n_hot, counts_fit, feat_slot,
+                                                             slot_feat, n_slots);
     SOM_CK(h, cudaGetLastError());
     h->launches += 2;
     return SOM_OK;
