@@ -75,11 +75,29 @@ k_feat_hist(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indi
     }
 }
 
+// Adds 1 to bins[bin] with one atomic per distinct bin in the warp; returns this thread's
+// rank inside the bin's increment (0-based) plus the old value.
+__device__ __forceinline__ uint32_t warp_agg_inc(uint32_t* bins, uint32_t bin, bool active)
+{
+    const unsigned act = __ballot_sync(0xffffffffu, active);
+    uint32_t res = 0;
+    if (active) {
+        const unsigned peers = __match_any_sync(act, bin);
+        const int lane = threadIdx.x & 31;
+        const int leader = __ffs(peers) - 1;
+        uint32_t old = 0;
+        if (lane == leader) old = atomicAdd(&bins[bin], (uint32_t)__popc(peers));
+        old = __shfl_sync(peers, old, leader);
+        res = old + (uint32_t)__popc(peers & ((1u << lane) - 1u));
+    }
+    return res;
+}
+
 // ---- 2. hot-set selection --------------------------------------------------------------------
 // K-th largest count by a 4-pass radix select.  thr = that count, n_greater = how many counts
 // are strictly larger.  All threads of the 1024-thread block call it.
 __device__ void kth_largest(const uint32_t* __restrict__ c, int V, int K, uint32_t* sh_hist,
-                            uint32_t* sh_state, uint32_t* thr, int* n_greater)
+                            uint32_t* sh_state, int* scan_ws, uint32_t* thr, int* n_greater)
 {
     if (threadIdx.x == 0) { sh_state[0] = 0; sh_state[1] = (uint32_t)K; sh_state[2] = 0; }
     __syncthreads();
@@ -88,18 +106,27 @@ __device__ void kth_largest(const uint32_t* __restrict__ c, int V, int K, uint32
         __syncthreads();
         const uint32_t prefix = sh_state[0];
         const uint32_t hi_mask = (shift == 24) ? 0u : (0xffffffffu << (shift + 8));
-        for (int v = threadIdx.x; v < V; v += blockDim.x) {
-            const uint32_t x = c[v];
-            if ((x & hi_mask) == prefix) atomicAdd(&sh_hist[(x >> shift) & 255u], 1u);
+        // (nearly all counts share their high bytes: one atomic per distinct digit and warp)
+        for (int v0 = 0; v0 < V; v0 += blockDim.x) {
+            const int v = v0 + threadIdx.x;
+            const uint32_t x = v < V ? c[v] : 0u;
+            warp_agg_inc(sh_hist, (x >> shift) & 255u, v < V && (x & hi_mask) == prefix);
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t need = sh_state[1], cum = 0;
-            int d = 255;
-            while (d > 0 && cum + sh_hist[d] < need) { cum += sh_hist[d]; --d; }
-            sh_state[2] += cum;
-            sh_state[1] = need - cum;
-            sh_state[0] = prefix | ((uint32_t)d << shift);
+        // the digit d whose bin holds the K-th largest: the counts above it (an exclusive scan
+        // over the digits in descending order) stay below `need`, with bin d they reach it;
+        // digit 0 when even all bins together do not (fewer counts than K)
+        {
+            const uint32_t need = sh_state[1];
+            const int d = 255 - (int)threadIdx.x;
+            const uint32_t mine = d >= 0 ? sh_hist[d] : 0u;
+            int total;
+            const uint32_t above = (uint32_t)block_excl_scan_1024((int)mine, scan_ws, &total);
+            if (d >= 0 && ((above < need && need <= above + mine) || (d == 0 && above + mine < need))) {
+                sh_state[2] += above;
+                sh_state[1] = need - above;
+                sh_state[0] = prefix | ((uint32_t)d << shift);
+            }
         }
         __syncthreads();
     }
@@ -126,8 +153,8 @@ k_select_hot(const uint32_t* __restrict__ feat_count_g, int V, int n_mask, int n
     __shared__ int sh_total;
     uint32_t thr_m, thr_a;
     int gr_m, gr_a;
-    kth_largest(feat_count, V, n_mask, sh_hist, sh_state, &thr_m, &gr_m);
-    kth_largest(feat_count, V, n_mask + n_hot, sh_hist, sh_state, &thr_a, &gr_a);
+    kth_largest(feat_count, V, n_mask, sh_hist, sh_state, warp_sums, &thr_m, &gr_m);
+    kth_largest(feat_count, V, n_mask + n_hot, sh_hist, sh_state, warp_sums, &thr_a, &gr_a);
     const int need_m = n_mask - gr_m;            // ties at thr_m to take (lowest ids first)
     const int need_a = n_mask + n_hot - gr_a;    // ties at thr_a to take
     // Every thread owns a contiguous range of feature ids, so ranks in id order are "offset of my
@@ -195,24 +222,6 @@ __device__ __forceinline__ uint32_t sort_bin(uint32_t mask, uint32_t n_hot, uint
     const uint32_t ch = n_hot > 15u ? 15u : n_hot;
     const uint32_t ct = n_tail > 7u ? 7u : n_tail;
     return (mask << SOM_PLAN_LEN_BITS) | (ch << 3) | ct;
-}
-
-// Adds 1 to bins[bin] with one atomic per distinct bin in the warp; returns this thread's
-// rank inside the bin's increment (0-based) plus the old value.
-__device__ __forceinline__ uint32_t warp_agg_inc(uint32_t* bins, uint32_t bin, bool active)
-{
-    const unsigned act = __ballot_sync(0xffffffffu, active);
-    uint32_t res = 0;
-    if (active) {
-        const unsigned peers = __match_any_sync(act, bin);
-        const int lane = threadIdx.x & 31;
-        const int leader = __ffs(peers) - 1;
-        uint32_t old = 0;
-        if (lane == leader) old = atomicAdd(&bins[bin], (uint32_t)__popc(peers));
-        old = __shfl_sync(peers, old, leader);
-        res = old + (uint32_t)__popc(peers & ((1u << lane) - 1u));
-    }
-    return res;
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS)
