@@ -273,12 +273,14 @@ int som_last_cuda_error(const som_handle* h);
  * (0 = default 60; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
  * slab buffers in MiB (0 = default 4096); key 7 = two-stage search for fp32 storage (0 = off, the default;
  * 1 = on): som_norms then also keeps an fp16 copy of the codebook (V*M*2 more bytes of device memory,
- * allocated by this call, which fails with SOM_ERR_CUDA if they cannot be had) and the largest |weight|;
- * som_bmu ranks the neurons by a first pass over that copy, keeps the result for every sample whose two
- * best first-pass scores are further apart than twice a bound on what the fp16 rounding and the fp32
- * summation can change (then the best unit of the exact weights is provably the same one), and searches
- * the other samples again with the fp32 weights.  Reported distances always come from the fp32 weights.
- * Needs M % 128 == 0 and the row-table kernel; som_bmu2 never uses it.  A two-stage call synchronises the
+ * allocated by this call, which fails with SOM_ERR_CUDA if they cannot be had), the largest |weight|, the
+ * largest ||w||^2 and whether any weight is negative; som_bmu ranks the neurons by a first pass over that
+ * copy, keeps the result for every sample whose two best first-pass scores are further apart than a bound on
+ * what the fp16 rounding and the fp32 summation can change (then the best unit of the exact weights is
+ * provably the same one; the bound is tighter when no weight is negative), and searches the other samples
+ * again with the fp32 weights.  som_bmu2 does the same with the three best first-pass scores (both units
+ * and their order certified).  Reported distances always come from the fp32 weights.
+ * Needs M % 128 == 0 and the row-table kernel.  A two-stage call synchronises the
  * stream a second time (it reads the length of the second pass's list back).  som_last_uncertain returns how
  * many samples the last two-stage search sent to its second pass.
  */

@@ -169,9 +169,9 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     // Two-stage search (option 7, fp32 storage): a first pass over the fp16 shadow of the
     // codebook with the wide fp16 layout, a certificate per sample, an exact fp32 pass for the
     // samples that fail it.  It needs the shadow written by the last som_norms and the row-table
-    // kernel; the two-best search does not use it (a certificate for the second unit would need
-    // the third).
-    const bool two_stage_ok = h->opt_two_stage == 1 && h->shadow && h->shadow_valid && !h->Wh && !top2 &&
+    // kernel; the two-best search keeps the three best of the first pass (the certificate for the
+    // second unit needs the third).
+    const bool two_stage_ok = h->opt_two_stage == 1 && h->shadow && h->shadow_valid && !h->Wh &&
                               h->M % 128 == 0;
     // Kernel selection.  The row-table kernel needs 128-bit aligned row segments (M % 4 == 0;
     // M % 64 == 0 with fp16 storage), feature ids that fit its 16-bit codes (V <= 65536) and
@@ -246,13 +246,14 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
                                        geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        // first pass: two best units by the fp16-rounded weights
-        if ((rc = som_launch_bmu_table(h, true, n_samples, head, ws, pb, geom.n_hot, true, st))) return rc;
+        // first pass: two (three) best units by the fp16-rounded weights
+        if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
+        if ((rc = som_launch_bmu_table(h, true, n_samples, head, ws, pb, geom.n_hot, top2 ? 3 : 2, st))) return rc;
         // certificate; certain samples are finalised, the others listed
         int32_t* uncertain = reinterpret_cast<int32_t*>(ws + pb.uncertain);
         int* n_unc_dev = reinterpret_cast<int*>(head + pb.n_slots) + SOM_PLAN_UNCERTAIN;
-        if ((rc = som_launch_certify(h, d_indptr, d_indices, n_samples, ws, pb, d_bmu, d_min_dist, uncertain,
-                                     n_unc_dev, st)))
+        if ((rc = som_launch_certify(h, d_indptr, d_indices, n_samples, ws, pb, d_bmu, d_min_dist, d_bmu2, d_dist2,
+                                     uncertain, n_unc_dev, st)))
             return rc;
         SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
         SOM_CK(h, cudaStreamSynchronize(st));
@@ -263,27 +264,37 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
             // them the row-table kernel runs again on their compacted slots (same plan: both
             // layouts hold the same number of hot rows), else the direct-load kernel.
             unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
+            unsigned long long* ukeys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.ukeys2) : nullptr;
             const SomTableGeom exact = som_table_geometry(h, false);
             const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T);
+            const size_t ub = (size_t)(n_unc + 16) * sizeof(unsigned long long);
+            SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, ub, st));
+            if (top2) SOM_CK(h, cudaMemsetAsync(ukeys2, 0xFF, ub, st));
             if (exact.n_hot == geom.n_hot && units >= 2 * (int64_t)h->sm_count) {
                 SomPlanBuffers pe = pb;
                 pe.slots = pb.slots2;
                 pe.keys = pb.ukeys;
-                SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, (size_t)(n_unc + 16) * sizeof(unsigned long long), st));
+                pe.keys2 = pb.ukeys2;
                 SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(head + pb.n_slots) + 3, 0, sizeof(int), st));
                 if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_unc, st))) return rc;
-                if ((rc = som_launch_bmu_table(h, false, n_unc, head, ws, pe, exact.n_hot, false, st))) return rc;
+                if ((rc = som_launch_bmu_table(h, false, n_unc, head, ws, pe, exact.n_hot, top2 ? 2 : 1, st)))
+                    return rc;
                 if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
                 if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_unc, ws, pe, false, d_bmu,
                                                      d_min_dist, st)))
                     return rc;
+                if (top2 && (rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_unc, ws, pe, true, d_bmu2,
+                                                             d_dist2, st)))
+                    return rc;
             } else {
-                SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, (size_t)n_unc * sizeof(unsigned long long), st));
-                if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_unc, ukeys, nullptr, uncertain, st)))
+                if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_unc, ukeys, ukeys2, uncertain, st)))
                     return rc;
                 if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
                 if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_unc, ukeys, d_bmu, d_min_dist, uncertain,
                                               st)))
+                    return rc;
+                if (top2 && (rc = som_launch_finalize(h, d_indptr, d_indices, n_unc, ukeys2, d_bmu2, d_dist2,
+                                                      uncertain, st)))
                     return rc;
             }
         } else if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) {
@@ -300,7 +311,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
                                        geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_table(h, false, n_samples, head, ws, pb, geom.n_hot, top2, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, false, n_samples, head, ws, pb, geom.n_hot, top2 ? 2 : 1, st))) return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, false, d_bmu,
                                              d_min_dist, st)))
@@ -479,7 +490,7 @@ int som_bmu_planned(som_handle* h, som_plan* p, int32_t* d_bmu, float* d_min_dis
         SOM_CK(h, cudaMemsetAsync(p->ws + p->pb.keys, 0xFF, (size_t)(p->n + 16) * sizeof(unsigned long long), st));
         SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(p->head + p->pb.n_slots) + 3, 0, sizeof(int), st));
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_table(h, false, p->n, p->head, p->ws, p->pb, p->n_hot, false, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, false, p->n, p->head, p->ws, p->pb, p->n_hot, 1, st))) return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, p->indptr, p->indices, p->n, p->ws, p->pb, false, d_bmu,
                                              d_min_dist, st)))

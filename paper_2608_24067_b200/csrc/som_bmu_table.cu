@@ -359,16 +359,18 @@ struct LayF16W {
 #define SOM_TAIL(code) L::ldg(row_ptr(w_q, (code), stride_b))
 
 // L = storage layout (R = neurons per lane, 4 or 8; a team of 8 lanes covers T = 8*R neurons of
-// one sample).  TOP2 also keeps the second-best unit of every sample in keys2 (Algorithm 2 keeps the two
+// one sample).  KEEP = 2 also keeps the second-best unit of every sample in keys2 (Algorithm 2 keeps the two
 // best units); the candidate filter then tests against the second-best score.
-template <typename L, int THREADS, bool TOP2>
+// KEEP = 3 (first pass of the two-stage two-best search) keeps the third best as well, in keys3.
+template <typename L, int THREADS, int KEEP>
 __global__ void __launch_bounds__(THREADS, 1)
 k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
             const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
-            u64* __restrict__ keys, u64* __restrict__ keys2, int parts, int64_t part_len, int n_units,
-            int n_whole, int* __restrict__ unit_counter)
+            u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
+            int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter)
 {
+    constexpr bool TOP2 = KEEP >= 2;
     constexpr int R = L::R;
     constexpr int T = L::T;
     constexpr int ROWB = L::ROWB;
@@ -460,8 +462,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             // lanes 12..13 the two 16-byte pieces of its four keys.
             unsigned char* ring = ring_sh + warp * 2 * RING_STAGE;
             // the keys a round tests its candidates against: the best so far, or with TOP2 the
-            // second best so far (a stale, larger value only lets more candidates through)
-            const u64* filter_keys = TOP2 ? keys2 : keys;
+            // second (third) best so far (a stale, larger value only lets more candidates through)
+            const u64* filter_keys = KEEP == 3 ? keys3 : (TOP2 ? keys2 : keys);
             const uint4* feed = (lane < 12) ? slots + w0 * SLOT_Q + lane
                                             : reinterpret_cast<const uint4*>(filter_keys + w0) + (lane - 12);
             const int feed_step = (lane < 12) ? 4 * SLOT_Q : 2;  // uint4 per round
@@ -591,17 +593,34 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         // not beat the best of its time) or when a later, smaller candidate
                         // displaces it from keys, so keys2 ends as the second smallest.  Both
                         // are minima of fixed sets: order-independent, ties to the lower index.
+                        // With KEEP = 3 the chain has one more level: what loses at keys2 goes
+                        // on to keys3; the lane's second best (never the overall best) enters at
+                        // keys2, its third best (never among the overall two best) at keys3.
                         u64* k1 = pk - 4;
                         u64* k2 = keys2 + (k1 - keys);
+                        u64* k3 = KEEP == 3 ? keys3 + (k1 - keys) : nullptr;
                         const u64 old = atomicMin(k1, c1);
-                        atomicMin(k2, old > c1 ? old : c1);
+                        const u64 l1 = old > c1 ? old : c1;
+                        const u64 old2 = atomicMin(k2, l1);
+                        if (KEEP == 3) atomicMin(k3, old2 > l1 ? old2 : l1);
                         float m2 = inf;
                         int r2 = 0;
 #pragma unroll
                         for (int j = R - 1; j >= 0; --j)
                             if (j != rr && a[j] <= m2) { m2 = a[j]; r2 = j; }
-                        if (!(m2 > cs))
-                            atomicMin(k2, som_pack_key(m2, i_first + L::neuron_of(r2)));
+                        if (!(m2 > cs)) {
+                            const u64 c2 = som_pack_key(m2, i_first + L::neuron_of(r2));
+                            const u64 o2 = atomicMin(k2, c2);
+                            if (KEEP == 3) {
+                                atomicMin(k3, o2 > c2 ? o2 : c2);
+                                float m3 = inf;
+                                int r3 = 0;
+#pragma unroll
+                                for (int j = R - 1; j >= 0; --j)
+                                    if (j != rr && j != r2 && a[j] <= m3) { m3 = a[j]; r3 = j; }
+                                if (!(m3 > cs)) atomicMin(k3, som_pack_key(m3, i_first + L::neuron_of(r3)));
+                            }
+                        }
                     }
                 }
             }
@@ -633,7 +652,7 @@ __global__ void k_finalize_sorted(const ST* __restrict__ W, const double* __rest
     dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
 }
 
-template <typename L, int THREADS, bool TOP2>
+template <typename L, int THREADS, int KEEP>
 int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* head, char* ws,
                  const SomPlanBuffers& b, int n_hot, size_t smem, cudaStream_t st)
 {
@@ -654,7 +673,7 @@ int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* he
     const int n_whole = (int)n_units64 - n_split;
     if (n_units64 + 3 * (int64_t)n_split > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
     const int n_units = n_whole + 4 * n_split;
-    auto kern = k_bmu_table<L, THREADS, TOP2>;
+    auto kern = k_bmu_table<L, THREADS, KEEP>;
     const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
     SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<grid, THREADS, smem, st>>>(codebook, h->hnorm, h->M,
@@ -663,7 +682,9 @@ int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* he
                                       reinterpret_cast<const uint4*>(ws + b.slots),
                                       reinterpret_cast<const uint32_t*>(ws + b.overflow), n,
                                       reinterpret_cast<u64*>(ws + b.keys),
-                                      TOP2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr, parts, part_len, n_units, n_whole,
+                                      KEEP >= 2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr,
+                                      KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
+                                      n_units, n_whole,
                                       reinterpret_cast<int*>(head + b.n_slots) + 3);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
@@ -700,19 +721,21 @@ SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
     return g;
 }
 
-template <bool TOP2>
+template <int KEEP>
 static int launch_table_any(som_handle* h, bool shadow, int64_t n, char* head, char* ws,
                             const SomPlanBuffers& b, int n_hot, cudaStream_t st)
 {
     const SomTableGeom g = som_table_geometry(h, shadow);
     const bool f16 = h->Wh != nullptr || shadow;
     const void* cb = shadow ? (const void*)h->shadow : (h->Wh ? (const void*)h->Wh : (const void*)h->W);
-#define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, TOP2>(h, cb, n, head, ws, b, n_hot, g.smem, st)
+#define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, KEEP>(h, cb, n, head, ws, b, n_hot, g.smem, st)
     if (f16 && g.R == 16) {
-        if (g.threads == 768) SOM_TABLE(LayF16W, 768);
-        if (g.threads == 640) SOM_TABLE(LayF16W, 640);
+        if (KEEP < 3 && g.threads == 768) SOM_TABLE(LayF16W, 768);
+        if (KEEP < 3 && g.threads == 640) SOM_TABLE(LayF16W, 640);
         SOM_TABLE(LayF16W, 512);
     }
+    if constexpr (KEEP == 3) return SOM_ERR_UNSUPPORTED;  // three best: the wide fp16 layout only
+    else {
     if (f16) {
         if (g.threads == 1024) SOM_TABLE(LayF16, 1024);
         if (g.threads == 896) SOM_TABLE(LayF16, 896);
@@ -732,25 +755,31 @@ static int launch_table_any(som_handle* h, bool shadow, int64_t n, char* head, c
     if (g.threads == 768) SOM_TABLE(LayF32<4>, 768);
     if (g.threads == 640) SOM_TABLE(LayF32<4>, 640);
     SOM_TABLE(LayF32<4>, 512);
+    }
 #undef SOM_TABLE
 }
 
 int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
-                         int n_hot, bool top2, cudaStream_t st)
+                         int n_hot, int keep, cudaStream_t st)
 {
-    return top2 ? launch_table_any<true>(h, shadow, n, head, ws, b, n_hot, st)
-                : launch_table_any<false>(h, shadow, n, head, ws, b, n_hot, st);
+    if (keep == 3) return launch_table_any<3>(h, shadow, n, head, ws, b, n_hot, st);
+    return keep == 2 ? launch_table_any<2>(h, shadow, n, head, ws, b, n_hot, st)
+                     : launch_table_any<1>(h, shadow, n, head, ws, b, n_hot, st);
 }
 
 // ---- two-stage search: certification of the first pass ----------------------------------------
 // The first pass ranked the neurons by fp32 sums of the fp16-rounded weights.  For a sample with
-// k active features every such score differs from the fp32 score of the exact weights by at most
-//   eps = k * max(wmax * 2^-11, 2^-25)  (rounding of each weight to fp16, round to nearest;
-//                                        the second term covers fp16's subnormal range)
-//       + 2 * (k + 2) * 2^-24 * B  (fp32 summation, either path; B bounds every partial sum),
-// so when the two best first-pass scores are more than 2 * eps apart the best unit of the exact
-// weights is the first pass's best unit.  Such samples are finalised here (distance recomputed in
-// fp64 from the fp32 weights, as always); the others are listed for an exact fp32 search.
+// k active features such a score differs from the fp32 score of the exact weights by at most
+//   k * max(wmax * 2^-11, 2^-25)  (rounding of each weight to fp16, round to nearest; the second
+//                                  term covers fp16's subnormal range)
+//   + 2 * (k + 2) * 2^-24 * B     (fp32 summation, either path; B bounds every partial sum).
+// When no weight is negative (the norm pass records it) the first term tightens to 2^-11 times the
+// unit's own dot product with the sample, i.e. ||w||^2/2 minus its score, plus k * 2^-25; for a unit
+// that is not named, to 2^-11 * (max ||w||^2/2 - its score), largest at the lowest score it can have.
+// When the two best first-pass scores are further apart than the bounds of the best unit and of
+// any other unit together, the best unit of the exact weights is the first pass's best unit.  Such
+// samples are finalised here (distance recomputed in fp64 from the fp32 weights, as always); the
+// others are listed for an exact fp32 search.
 namespace {
 __device__ __forceinline__ float score_of_key(u64 key)
 {
@@ -758,11 +787,18 @@ __device__ __forceinline__ float score_of_key(u64 key)
     return __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
 }
 
+// SECOND: the two-best search.  With the three best first-pass scores s1 <= s2 <= s3, the two
+// first-pass winners are the two best units of the exact weights, in that order, when both gaps
+// exceed the bounds of their two sides (s3 - s2: no third unit can overtake either; s2 - s1: they
+// cannot swap).
+template <bool SECOND>
 __global__ void k_certify(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
                           const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
                           const uint4* __restrict__ slots, const u64* __restrict__ keys,
-                          const u64* __restrict__ keys2, const unsigned int* __restrict__ wmax_bits,
+                          const u64* __restrict__ keys2, const u64* __restrict__ keys3,
+                          const unsigned int* __restrict__ wmax_bits, const float* __restrict__ hnorm,
                           int32_t* __restrict__ bmu, float* __restrict__ dist,
+                          int32_t* __restrict__ bmu2, float* __restrict__ dist2,
                           int32_t* __restrict__ uncertain, uint4* __restrict__ slots2,
                           int* __restrict__ n_uncertain)
 {
@@ -777,21 +813,56 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
         const u64 k1 = keys[k], k2 = keys2[k];
         const int beg = indptr[s];
         const int end = indptr[s + 1];
-        const float wmax = __uint_as_float(*wmax_bits);
+        const float wmax = __uint_as_float(wmax_bits[0]);
+        const bool has_negative = wmax_bits[SOM_AUX_HAS_NEGATIVE] != 0u;
+        const float hmax = __uint_as_float(wmax_bits[SOM_AUX_HMAX]);
         const float s1 = score_of_key(k1), s2 = score_of_key(k2);
+        const uint32_t i1 = (uint32_t)(k1 & 0xffffffffull), i2 = (uint32_t)(k2 & 0xffffffffull);
         const float cnt = (float)(end - beg);
-        const float bound = fmaxf(fabsf(s1), fabsf(s2)) + 2.f * cnt * wmax;
-        // per weight: 2^-11 relative in fp16's normal range, at most 2^-25 absolute below it
-        const float per_weight = fmaxf(wmax * 4.8828125e-4f, 2.9802322e-8f) * 1.0001f;
-        const float eps = cnt * per_weight + 2.f * (cnt + 2.f) * 5.9604645e-8f * bound;
-        const bool certain = (s2 - s1) > 2.f * eps;  // false for NaN or an empty second key
+        float top = fmaxf(fabsf(s1), fabsf(s2));
+        float s3 = 0.f;
+        if (SECOND) {
+            s3 = score_of_key(keys3[k]);
+            top = fmaxf(top, fabsf(s3));
+        }
+        // fp32 summation of either pass: 2 (k + 2) 2^-24 B, B a bound on every partial sum
+        const float fsum = 2.f * (cnt + 2.f) * 5.9604645e-8f * (top + 2.f * cnt * wmax);
+        // rounding of the weights to fp16: at most 2^-11 relative in fp16's normal range, at most
+        // 2^-25 absolute below it
+        float e1, e2, eo;  // error bounds of the first, the second and of any other unit's score
+        if (!has_negative && i1 < M && i2 < M) {
+            // All weights >= 0: a unit's rounding errors add up to at most 2^-11 times its dot
+            // product, which is ||w||^2/2 minus its score (first-pass values, hence the margins).
+            // For a unit that is not named its dot product is at most hmax minus the lowest score
+            // it can have; the bound shrinks as the score grows, so that lowest score is the worst case.
+            const float c = 4.8828125e-4f * 1.002f;
+            const float sub = cnt * 2.9802322e-8f;
+            e1 = c * fmaxf(hnorm[i1] - s1 + fsum, 0.f) + sub + fsum;
+            e2 = c * fmaxf(hnorm[i2] - s2 + fsum, 0.f) + sub + fsum;
+            eo = c * fmaxf(hmax - (SECOND ? s3 : s2) + fsum, 0.f) + sub + fsum;
+        } else {
+            e1 = e2 = eo = cnt * fmaxf(wmax * 4.8828125e-4f, 2.9802322e-8f) * 1.0001f + fsum;
+        }
+        // comparisons are false for NaN or an empty key
+        bool certain;
+        if (!SECOND) certain = (s2 - s1) > e1 + eo;
+        else certain = (s2 - s1) > e1 + e2 && (s3 - s2) > e2 + eo;  // (a map of two units has no third: exact pass)
         flag = !certain;
         if (certain) {
             const uint32_t idx = (uint32_t)(k1 & 0xffffffffull);
-            double dot = 0.0;
-            for (int j = beg; j < end; ++j) dot += (double)__ldg(W + (int64_t)indices[j] * M + idx);
+            const uint32_t idx2 = (uint32_t)(k2 & 0xffffffffull);
+            double dot = 0.0, dot2 = 0.0;
+            for (int j = beg; j < end; ++j) {
+                const float* row = W + (int64_t)indices[j] * M;
+                dot += (double)__ldg(row + idx);
+                if (SECOND) dot2 += (double)__ldg(row + idx2);
+            }
             bmu[s] = (int32_t)idx;
             dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
+            if (SECOND) {
+                bmu2[s] = (int32_t)idx2;
+                dist2[s] = (float)((double)(end - beg) - 2.0 * dot2 + norm64[idx2]);
+            }
         }
     }
     // The uncertain samples of a block keep their (mask-sorted) order: their ids and their
@@ -816,16 +887,23 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
 }  // namespace
 
 int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
-                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* uncertain,
-                       int* n_uncertain, cudaStream_t st)
+                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* bmu2, float* dist2,
+                       int32_t* uncertain, int* n_uncertain, cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
-    k_certify<<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n,
-                                                reinterpret_cast<const uint4*>(ws + b.slots),
-                                                reinterpret_cast<const u64*>(ws + b.keys),
-                                                reinterpret_cast<const u64*>(ws + b.keys2), h->wmax_bits, bmu,
-                                                dist, uncertain, reinterpret_cast<uint4*>(ws + b.slots2),
-                                                n_uncertain);
+    const uint4* slots = reinterpret_cast<const uint4*>(ws + b.slots);
+    const u64* keys = reinterpret_cast<const u64*>(ws + b.keys);
+    const u64* keys2 = reinterpret_cast<const u64*>(ws + b.keys2);
+    const u64* keys3 = reinterpret_cast<const u64*>(ws + b.keys3);
+    uint4* slots2 = reinterpret_cast<uint4*>(ws + b.slots2);
+    if (bmu2)
+        k_certify<true><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, slots, keys,
+                                                          keys2, keys3, h->wmax_bits, h->hnorm, bmu, dist, bmu2, dist2,
+                                                          uncertain, slots2, n_uncertain);
+    else
+        k_certify<false><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, slots, keys,
+                                                           keys2, nullptr, h->wmax_bits, h->hnorm, bmu, dist, nullptr,
+                                                           nullptr, uncertain, slots2, n_uncertain);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

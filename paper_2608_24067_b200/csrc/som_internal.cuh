@@ -11,6 +11,9 @@
 #define SOM_EV_RING 32
 #define SOM_N_EVENTS (SOM_EV_PER_CALL * SOM_EV_RING)
 
+#define SOM_AUX_HAS_NEGATIVE 1
+#define SOM_AUX_HMAX 2
+
 struct som_handle {
     int device;
     int sm_count;
@@ -19,7 +22,8 @@ struct som_handle {
     const float* W;    // borrowed, feature-major fp32 codebook (nullptr when stored as fp16)
     const __half* Wh;  // borrowed, feature-major fp16 codebook (som_create_f16), else nullptr
     __half* shadow;    // owned fp16 copy of an fp32 codebook for the two-stage search (nullptr = none)
-    unsigned int* wmax_bits;  // device: float bits of max |weight|, written by som_norms with the shadow
+    unsigned int* wmax_bits;  // device, written by som_norms with the shadow: [0] float bits of max |weight|,
+                              // [SOM_AUX_HAS_NEGATIVE] 1 if a weight is negative, [SOM_AUX_HMAX] float bits of max ||w||^2/2
     int shadow_valid;         // the last som_norms wrote the shadow
     int64_t last_uncertain;   // samples the last two-stage search sent to its exact pass
 

@@ -40,7 +40,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
     for (int k = 0; k < VEC; ++k) acc[k] = 0.0;
     const float* p = W + (int64_t)v0 * M + i;
     __half* ps = SHADOW ? shadow + (int64_t)v0 * M + i : nullptr;
-    float wmax = 0.f;
+    float wmax = 0.f, wmin = 0.f;
     int v = v0;
     if (VEC == 4) {
         for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
@@ -53,6 +53,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
                 if (SHADOW) {
                     store_half4(ps + (int64_t)u * M, w[u]);
                     wmax = fmaxf(wmax, fmaxf(fmaxf(fabsf(w[u].x), fabsf(w[u].y)), fmaxf(fabsf(w[u].z), fabsf(w[u].w))));
+                    wmin = fminf(wmin, fminf(fminf(w[u].x, w[u].y), fminf(w[u].z, w[u].w)));
                 }
                 acc[0] = fma((double)w[u].x, (double)w[u].x, acc[0]);
                 acc[1 % VEC] = fma((double)w[u].y, (double)w[u].y, acc[1 % VEC]);
@@ -67,6 +68,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
             if (SHADOW) {
                 store_half4(ps, w);
                 wmax = fmaxf(wmax, fmaxf(fmaxf(fabsf(w.x), fabsf(w.y)), fmaxf(fabsf(w.z), fabsf(w.w))));
+                wmin = fminf(wmin, fminf(fminf(w.x, w.y), fminf(w.z, w.w)));
                 ps += M;
             }
             acc[0] = fma((double)w.x, (double)w.x, acc[0]);
@@ -91,6 +93,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
         const unsigned int active = __activemask();
         const unsigned int best = __reduce_max_sync(active, __float_as_uint(wmax));
         if ((threadIdx.x & 31) == (__ffs(active) - 1)) atomicMax(wmax_bits, best);
+        if (wmin < 0.f) wmax_bits[SOM_AUX_HAS_NEGATIVE] = 1u;  // (every writer stores the same value)
     }
 }
 
@@ -156,7 +159,7 @@ k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_s
 constexpr int COMBINE_GROUPS = 8;
 __global__ void k_norms_combine(const double* __restrict__ partial, int64_t M, int splits,
                                 double* __restrict__ norm64, float* __restrict__ norm32,
-                                float* __restrict__ hnorm)
+                                float* __restrict__ hnorm, unsigned int* __restrict__ hmax_bits)
 {
     __shared__ double sh[COMBINE_GROUPS][33];
     const int64_t i = (int64_t)blockIdx.x * 32 + threadIdx.x;
@@ -172,6 +175,8 @@ __global__ void k_norms_combine(const double* __restrict__ partial, int64_t M, i
     norm64[i] = s;
     norm32[i] = (float)s;
     hnorm[i] = (float)(0.5 * s);
+    // largest ||w||^2 / 2 over the map (non-negative: its float bits order like unsigned integers)
+    if (hmax_bits) atomicMax(hmax_bits, __float_as_uint((float)(0.5 * s)));
 }
 
 struct NormPlan {
@@ -216,7 +221,7 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
     else if (h->Wh)
         k_norms_partial_h<1><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
     else if (p.vec == 4 && h->shadow) {
-        SOM_CK(h, cudaMemsetAsync(h->wmax_bits, 0, sizeof(unsigned int), st));
+        SOM_CK(h, cudaMemsetAsync(h->wmax_bits, 0, 4 * sizeof(unsigned int), st));
         k_norms_partial<4, true><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
                                                                 h->shadow, h->wmax_bits);
     } else if (p.vec == 4)
@@ -227,8 +232,9 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
                                                                  nullptr, nullptr);
     SOM_CK(h, cudaGetLastError());
     const int64_t blocks = (h->M + 31) / 32;
-    k_norms_combine<<<(unsigned)blocks, dim3(32, COMBINE_GROUPS), 0, st>>>(partial, h->M, p.splits, h->norm64, h->norm32,
-                                                      h->hnorm);
+    k_norms_combine<<<(unsigned)blocks, dim3(32, COMBINE_GROUPS), 0, st>>>(
+        partial, h->M, p.splits, h->norm64, h->norm32, h->hnorm,
+        (p.vec == 4 && h->shadow && !h->Wh) ? h->wmax_bits + SOM_AUX_HMAX : nullptr);
     SOM_CK(h, cudaGetLastError());
     h->launches += 2;
     return SOM_OK;

@@ -418,6 +418,7 @@ size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b)
     };
     b->keys = take((size_t)(n + 16) * 8);
     b->keys2 = take((size_t)(n + 16) * 8);
+    b->keys3 = take((size_t)(n + 16) * 8);
     b->pk = take((size_t)n * 4);
     b->ntail = take((size_t)n * 4);
     b->bin_count = take((size_t)SOM_PLAN_BINS * 4);
@@ -427,6 +428,7 @@ size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b)
     b->overflow = take((size_t)(nnz + 6 * n + 4) * 4);
     b->uncertain = take((size_t)n * 4);
     b->ukeys = take((size_t)(n + 16) * 8);
+    b->ukeys2 = take((size_t)(n + 16) * 8);
     b->slots2 = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
     return off;
 }

@@ -45,6 +45,7 @@ struct SomPlanBuffers {
     // workspace
     size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
     size_t keys2;       // u64 [n]      the same for the second-best unit (two-best search only)
+    size_t keys3;       // u64 [n]      and for the third best (first pass of the two-stage two-best search)
     size_t pk;          // u32 [n]      mask | n_hot << 16, by sample
     size_t ntail;       // u32 [n]
     size_t bin_count;   // u32 [bins]
@@ -54,6 +55,7 @@ struct SomPlanBuffers {
     size_t overflow;    // u32 [nnz + 6n]
     size_t uncertain;   // i32 [n]      samples the two-stage search sends to its exact pass
     size_t ukeys;       // u64 [n + 16] their packed keys, by position in that list
+    size_t ukeys2;      // u64 [n + 16] and their second-best keys (two-best search)
     size_t slots2;      // 48 B [n + 16] their slots, compacted in list order
 };
 #define SOM_PLAN_N_SLOTS_INTS 8
@@ -85,16 +87,18 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
                          char* head, char* ws, const SomPlanBuffers& b, int n_mask, int n_hot,
                          cudaStream_t st);
 
-// shadow = read the handle's fp16 shadow of an fp32 codebook (first pass of the two-stage search)
+// shadow = read the handle's fp16 shadow of an fp32 codebook (first pass of the two-stage search);
+// keep = how many best units per sample are kept (1, 2; 3 with the shadow's wide layout only)
 int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
-                         int n_hot, bool top2, cudaStream_t st);
+                         int n_hot, int keep, cudaStream_t st);
 
 // pads a slot array of n slots to a multiple of four with copies of the last one
 int som_launch_pad_slots(som_handle* h, char* ws, size_t slots_offset, int64_t n, cudaStream_t st);
 
+// bmu2 / dist2 non-null: the two-best search (needs the three best first-pass keys)
 int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
-                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* uncertain,
-                       int* n_uncertain, cudaStream_t st);
+                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* bmu2, float* dist2,
+                       int32_t* uncertain, int* n_uncertain, cudaStream_t st);
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                                char* ws, const SomPlanBuffers& b, bool second, int32_t* bmu, float* dist,

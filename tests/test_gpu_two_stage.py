@@ -117,19 +117,92 @@ def test_two_stage_needs_its_shadow_from_norms(som_mod):
     _check(W.cpu().numpy(), V, M, b, bmu.cpu().numpy(), dist.cpu().numpy(), np.arange(0, n, 13))
 
 
+def _run2(som_mod, W, V, M, b, two_stage, variant=2):
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, variant)
+    if two_stage:
+        h.set_option(7, 1)
+    h.norms()
+    out = h.bmu2(b.indptr, b.indices)
+    again = h.bmu2(b.indptr, b.indices)
+    torch.cuda.synchronize()
+    for a, c in zip(out, again):
+        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+    return h, [t.cpu().numpy() for t in out]
+
+
+def _check2(W_host, V, M, b, out, rows):
+    g1, gd1, g2, gd2 = [x[rows] for x in out]
+    ip, ix = _subset(b.indptr.cpu().numpy(), b.indices.cpu().numpy(), rows)
+    nn = orc.norms(W_host, V, M)
+    top2 = orc.bmu(W_host, V, M, ip, ix, norms_=nn)
+    rep1 = parity.check(g1, gd1, top2, orc.dist_at(W_host, V, M, ip, ix, np.clip(g1.astype(np.int64), 0, M - 1), norms_=nn), M)
+    assert rep1.ok, str(rep1)
+    rep2 = parity.check_second(g1, g2, gd2, top2,
+                               orc.dist_at(W_host, V, M, ip, ix, np.clip(g2.astype(np.int64), 0, M - 1), norms_=nn), M)
+    assert rep2.ok, str(rep2)
+
+
+@pytest.mark.parametrize("scale", [1.0, 37.0, 1.0 / 64.0, 1e-6, 1e5])
+def test_two_stage_two_best_matches_oracle_and_plain_search(som_mod, scale):
+    """som_bmu2 with the option: three best of the first pass, both gaps certified."""
+    V, M, n = 30_000, 1_024, 80_000
+    W = synth.fill_codebook(V, M, 5, device="cuda") * scale
+    b = synth.sample_csr(n, V, 11.0, 5, device="cuda")
+    hs, staged = _run2(som_mod, W, V, M, b, True)
+    hp, plain = _run2(som_mod, W, V, M, b, False)
+    unc = hs.last_uncertain()
+    if 1e-3 < scale < 1e3:
+        assert 0 < unc < n // 2
+    differ = np.flatnonzero((plain[0] != staged[0]) | (plain[2] != staged[2]))
+    assert differ.size <= unc  # only samples of the exact pass can differ (near ties, other summation order)
+    same = (plain[0] == staged[0]) & (plain[2] == staged[2])
+    assert np.array_equal(plain[1][same].view(np.uint32), staged[1][same].view(np.uint32))
+    assert np.array_equal(plain[3][same].view(np.uint32), staged[3][same].view(np.uint32))
+    assert np.all(staged[2] != staged[0]) and staged[2].min() >= 0 and staged[2].max() < M
+    rows = np.unique(np.concatenate([np.arange(0, n, 9), differ]))
+    _check2(W.cpu().numpy(), V, M, b, staged, rows)
+
+
+def test_two_stage_two_best_config2_sampled_rows(som_mod):
+    w = synth.CONFIGS[1]
+    W = synth.fill_codebook(w.V, w.M, w.seed, device="cuda")
+    b = synth.sample_csr(w.N, w.V, w.lam, w.seed, device="cuda")
+    h, out = _run2(som_mod, W, w.V, w.M, b, True, variant=0)
+    assert 0 < h.last_uncertain() < w.N // 3
+    rows = np.concatenate([np.arange(0, w.N, 40), [w.N - 1]])
+    _check2(W.cpu().numpy(), w.V, w.M, b, out, rows)
+
+
+def test_two_stage_two_best_with_duplicate_neurons(som_mod):
+    """Two identical halves of the map: the best unit's twin is the second best at the same distance;
+    nothing can be certified and the lower index comes first."""
+    V, half, n = 2_000, 1_024, 40_000
+    Wh = synth.fill_codebook(V, half, 2, device="cuda").view(V, half)
+    W = torch.cat([Wh, Wh], dim=1).contiguous().view(-1)
+    M = 2 * half
+    b = synth.sample_csr(n, V, 7.0, 2, device="cuda")
+    h, out = _run2(som_mod, W, V, M, b, True)
+    assert h.last_uncertain() == n
+    assert out[0].max() < half
+    assert np.array_equal(out[2], out[0] + half)
+    assert np.array_equal(out[1].view(np.uint32), out[3].view(np.uint32))
+    _check2(W.cpu().numpy(), V, M, b, out, np.arange(0, n, 11))
+
+
 def test_two_stage_option_leaves_the_other_entry_points_alone(som_mod):
-    """som_bmu2 never takes the two-stage route, an fp16-stored codebook has no use for it, and a
-    forced direct-load kernel overrides it: all must give what they give without the option."""
+    """An fp16-stored codebook has no use for the option and a forced direct-load kernel overrides
+    it: both must give what they give without the option."""
     V, M, n = 2_000, 1_024, 30_000
     W = synth.fill_codebook(V, M, 9, device="cuda")
     b = synth.sample_csr(n, V, 7.0, 9, device="cuda")
     plain, staged = som_mod.Som(V, M, W), som_mod.Som(V, M, W)
     staged.set_option(7, 1)
     plain.norms(); staged.norms()
-    for a, c in zip(plain.bmu2(b.indptr, b.indices), staged.bmu2(b.indptr, b.indices)):
-        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
     plain.set_option(0, 1); staged.set_option(0, 1)
     for a, c in zip(plain.bmu(b.indptr, b.indices), staged.bmu(b.indptr, b.indices)):
+        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+    for a, c in zip(plain.bmu2(b.indptr, b.indices), staged.bmu2(b.indptr, b.indices)):
         assert torch.equal(a.view(torch.int32), c.view(torch.int32))
     W16 = W.half()
     h16a, h16b = som_mod.Som(V, M, W16), som_mod.Som(V, M, W16)
@@ -137,19 +210,6 @@ def test_two_stage_option_leaves_the_other_entry_points_alone(som_mod):
     h16a.norms(); h16b.norms()
     for a, c in zip(h16a.bmu(b.indptr, b.indices), h16b.bmu(b.indptr, b.indices)):
         assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+    for a, c in zip(h16a.bmu2(b.indptr, b.indices), h16b.bmu2(b.indptr, b.indices)):
+        assert torch.equal(a.view(torch.int32), c.view(torch.int32))
     torch.cuda.synchronize()
-
-
-def test_two_stage_twins_that_fp16_cannot_tell_apart(som_mod):
-    """Second half of the map = first half scaled by 1 + 2^-12: the twins collapse (or nearly) in fp16,
-    but their fp32 distances differ by more than the near-tie band, so the certificate must send the
-    affected samples to the exact pass and the exact winner must come back."""
-    V, half, n = 4_000, 512, 40_000
-    Wh = synth.fill_codebook(V, half, 6, device="cuda").view(V, half)
-    W = torch.cat([Wh, Wh * (1.0 + 2.0 ** -12)], dim=1).contiguous().view(-1)
-    M = 2 * half
-    b = synth.sample_csr(n, V, 7.0, 6, device="cuda")
-    h, bmu, dist = _run(som_mod, W, V, M, b, True)
-    rep = _check(W.cpu().numpy(), V, M, b, bmu, dist, np.arange(0, n, 5))
-    assert rep.unambiguous > 0.9 * rep.n          # the twins are not near ties for the fp64 oracle
-    assert h.last_uncertain() > n // 2            # but the first pass cannot separate them
