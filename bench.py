@@ -242,7 +242,8 @@ def run_ours(args, w: synth.Workload):
         h.norms()
         if args.epoch:
             plans[i % n_batches].bmu(out_bmu, out_dist)
-            h.update(epoch_edge, epoch_edge, b.indptr, b.indices, out_bmu, max(1, epoch_edge // 4))
+            h.update(epoch_edge, epoch_edge, b.indptr, b.indices, out_bmu,
+                     args.radius if args.radius > 0 else max(1, epoch_edge // 4))
         elif args.planned:
             plans[i % n_batches].bmu(out_bmu, out_dist)
         elif args.values:
@@ -363,7 +364,7 @@ def run_ours(args, w: synth.Workload):
         b0 = batches[0]
         h.norms()
         bm, _ = h.bmu(b0.indptr, b0.indices)
-        radius = max(1, edge // 4)
+        radius = args.radius if args.radius > 0 else max(1, edge // 4)
         h.update(edge, edge, b0.indptr, b0.indices, bm, radius)  # warm-up (allocates the workspace)
         barrier()
         u_steps = max(1, min(args.steps, 5))
@@ -490,6 +491,7 @@ def main():
                          "region and every step runs som_norms + som_bmu_planned")
     ap.add_argument("--top2", action="store_true",
                     help="time som_bmu2 (best and second-best unit) instead of som_bmu")
+    ap.add_argument("--radius", type=int, default=0, help="som_update: blur radius (default edge / 4)")
     ap.add_argument("--batch", type=int, default=0,
                     help="samples per batch instead of the configuration's (a sweep variant, named in the workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -129,12 +129,15 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
  * alone, not on the codebook.  Training searches the same batches every epoch (Algorithm 2, step 2), so a
  * caller can build each batch's plan once:
  *   som_plan_create   builds the plan of the device-resident CSR batch (arguments as in som_bmu) in
- *                     device memory of its own (about 70 bytes per sample) and synchronises `stream`.
+ *                     device memory of its own (about 220 bytes per sample plus 70 MB, scratch of the
+ *                     search included) and synchronises `stream`.
  *                     The plan BORROWS d_indptr / d_indices: they must stay valid and unchanged while
  *                     the plan lives.  It is tied to the handle and to the handle's options and
  *                     storage type at this moment.
  *   som_bmu_planned   som_bmu for the plan's batch: same outputs (bit-identical to som_bmu's on the same
- *                     batch), but only enqueues work on `stream` (no host synchronisation, no allocation).
+ *                     batch with the same options), but only enqueues work on `stream` (no host
+ *                     synchronisation, no allocation), except with the two-stage search (option 7), which
+ *                     it takes like som_bmu and which synchronises the stream once.
  *                     Two searches with the same plan must not overlap on the GPU.
  *   som_plan_destroy  frees the plan (NULL is accepted); destroy plans before their handle.
  */
@@ -280,6 +283,9 @@ int som_last_cuda_error(const som_handle* h);
  * provably the same one; the bound is tighter when no weight is negative), and searches the other samples
  * again with the fp32 weights.  som_bmu2 does the same with the three best first-pass scores (both units
  * and their order certified).  Reported distances always come from the fp32 weights.
+ * It pays on maps whose units are distinct at fp16 resolution (random initialisation, small final radius); on
+ * a map that a wide blur has just smoothed most samples fail the certificate and the call is slower than
+ * the plain search: read som_last_uncertain and switch the option off while that share is high.
  * Needs M % 128 == 0 and the row-table kernel.  A two-stage call synchronises the
  * stream a second time (it reads the length of the second pass's list back).  som_last_uncertain returns how
  * many samples the last two-stage search sent to its second pass.

@@ -150,6 +150,77 @@ int som_norms(som_handle* h, void* stream)
     return SOM_OK;
 }
 
+// The two-stage search on a batch whose plan (slots in ws, table features in head) is ready: first
+// pass over the fp16 shadow keeping the two (som_bmu2: three) best units, certificate, exact fp32
+// pass for the samples it leaves open.  Synchronises the stream once (length of that list).
+static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
+                            char* ws, const SomPlanBuffers& pb, int n_hot, int32_t* bmu, float* dist,
+                            int32_t* bmu2, float* dist2, cudaStream_t st)
+{
+    int rc = SOM_OK;
+    const bool top2 = bmu2 != nullptr;
+    const size_t kb = (size_t)(n + 16) * sizeof(unsigned long long);
+    int* counters = reinterpret_cast<int*>(head + pb.n_slots);
+    SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, kb, st));
+    SOM_CK(h, cudaMemsetAsync(ws + pb.keys2, 0xFF, kb, st));
+    if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
+    SOM_CK(h, cudaMemsetAsync(counters + 3, 0, sizeof(int), st));                   // search unit counter
+    SOM_CK(h, cudaMemsetAsync(counters + SOM_PLAN_UNCERTAIN, 0, sizeof(int), st));  // length of the list
+    if ((rc = som_launch_bmu_table(h, true, n, head, ws, pb, n_hot, top2 ? 3 : 2, st))) return rc;
+    // certificate; certain samples are finalised, the others listed
+    int32_t* uncertain = reinterpret_cast<int32_t*>(ws + pb.uncertain);
+    int* n_unc_dev = reinterpret_cast<int*>(head + pb.n_slots) + SOM_PLAN_UNCERTAIN;
+    if ((rc = som_launch_certify(h, indptr, indices, n, ws, pb, bmu, dist, bmu2, dist2,
+                                 uncertain, n_unc_dev, st)))
+        return rc;
+    SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SOM_CK(h, cudaStreamSynchronize(st));
+    const int64_t n_unc = h->host_pair[3];
+    h->last_uncertain = n_unc;
+    if (n_unc > 0) {
+        // exact pass over the listed samples: fp32 weights, all neurons.  With enough of
+        // them the row-table kernel runs again on their compacted slots (same plan: both
+        // layouts hold the same number of hot rows), else the direct-load kernel.
+        unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
+        unsigned long long* ukeys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.ukeys2) : nullptr;
+        const SomTableGeom exact = som_table_geometry(h, false);
+        const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T);
+        const size_t ub = (size_t)(n_unc + 16) * sizeof(unsigned long long);
+        SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, ub, st));
+        if (top2) SOM_CK(h, cudaMemsetAsync(ukeys2, 0xFF, ub, st));
+        if (exact.n_hot == n_hot && units >= 2 * (int64_t)h->sm_count) {
+            SomPlanBuffers pe = pb;
+            pe.slots = pb.slots2;
+            pe.keys = pb.ukeys;
+            pe.keys2 = pb.ukeys2;
+            SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(head + pb.n_slots) + 3, 0, sizeof(int), st));
+            if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_unc, st))) return rc;
+            if ((rc = som_launch_bmu_table(h, false, n_unc, head, ws, pe, exact.n_hot, top2 ? 2 : 1, st)))
+                return rc;
+            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+            if ((rc = som_launch_finalize_sorted(h, indptr, indices, n_unc, ws, pe, false, bmu,
+                                                 dist, st)))
+                return rc;
+            if (top2 && (rc = som_launch_finalize_sorted(h, indptr, indices, n_unc, ws, pe, true, bmu2,
+                                                         dist2, st)))
+                return rc;
+        } else {
+            if ((rc = som_launch_bmu_direct(h, indptr, indices, n_unc, ukeys, ukeys2, uncertain, st)))
+                return rc;
+            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+            if ((rc = som_launch_finalize(h, indptr, indices, n_unc, ukeys, bmu, dist, uncertain,
+                                          st)))
+                return rc;
+            if (top2 && (rc = som_launch_finalize(h, indptr, indices, n_unc, ukeys2, bmu2, dist2,
+                                                  uncertain, st)))
+                return rc;
+        }
+    } else if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) {
+        return rc;
+    }
+    return SOM_OK;
+}
+
 // The search behind som_bmu (d_bmu2 == nullptr) and som_bmu2 (both second-best outputs given).
 static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
                     int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream)
@@ -239,67 +310,13 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         const size_t need = som_plan_workspace_bytes(n_samples, nnz, &pb);
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
         char* ws = reinterpret_cast<char*>(h->ws);
-        const size_t kb = (size_t)(n_samples + 16) * sizeof(unsigned long long);
-        SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, kb, st));
-        SOM_CK(h, cudaMemsetAsync(ws + pb.keys2, 0xFF, kb, st));
         if ((rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, head, ws, pb, SOM_PLAN_MASK_FEATURES,
                                        geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        // first pass: two (three) best units by the fp16-rounded weights
-        if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
-        if ((rc = som_launch_bmu_table(h, true, n_samples, head, ws, pb, geom.n_hot, top2 ? 3 : 2, st))) return rc;
-        // certificate; certain samples are finalised, the others listed
-        int32_t* uncertain = reinterpret_cast<int32_t*>(ws + pb.uncertain);
-        int* n_unc_dev = reinterpret_cast<int*>(head + pb.n_slots) + SOM_PLAN_UNCERTAIN;
-        if ((rc = som_launch_certify(h, d_indptr, d_indices, n_samples, ws, pb, d_bmu, d_min_dist, d_bmu2, d_dist2,
-                                     uncertain, n_unc_dev, st)))
+        if ((rc = two_stage_search(h, d_indptr, d_indices, n_samples, head, ws, pb, geom.n_hot, d_bmu, d_min_dist,
+                                   d_bmu2, d_dist2, st)))
             return rc;
-        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-        SOM_CK(h, cudaStreamSynchronize(st));
-        const int64_t n_unc = h->host_pair[3];
-        h->last_uncertain = n_unc;
-        if (n_unc > 0) {
-            // exact pass over the listed samples: fp32 weights, all neurons.  With enough of
-            // them the row-table kernel runs again on their compacted slots (same plan: both
-            // layouts hold the same number of hot rows), else the direct-load kernel.
-            unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
-            unsigned long long* ukeys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.ukeys2) : nullptr;
-            const SomTableGeom exact = som_table_geometry(h, false);
-            const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T);
-            const size_t ub = (size_t)(n_unc + 16) * sizeof(unsigned long long);
-            SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, ub, st));
-            if (top2) SOM_CK(h, cudaMemsetAsync(ukeys2, 0xFF, ub, st));
-            if (exact.n_hot == geom.n_hot && units >= 2 * (int64_t)h->sm_count) {
-                SomPlanBuffers pe = pb;
-                pe.slots = pb.slots2;
-                pe.keys = pb.ukeys;
-                pe.keys2 = pb.ukeys2;
-                SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(head + pb.n_slots) + 3, 0, sizeof(int), st));
-                if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_unc, st))) return rc;
-                if ((rc = som_launch_bmu_table(h, false, n_unc, head, ws, pe, exact.n_hot, top2 ? 2 : 1, st)))
-                    return rc;
-                if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-                if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_unc, ws, pe, false, d_bmu,
-                                                     d_min_dist, st)))
-                    return rc;
-                if (top2 && (rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_unc, ws, pe, true, d_bmu2,
-                                                             d_dist2, st)))
-                    return rc;
-            } else {
-                if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_unc, ukeys, ukeys2, uncertain, st)))
-                    return rc;
-                if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-                if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_unc, ukeys, d_bmu, d_min_dist, uncertain,
-                                              st)))
-                    return rc;
-                if (top2 && (rc = som_launch_finalize(h, d_indptr, d_indices, n_unc, ukeys2, d_bmu2, d_dist2,
-                                                      uncertain, st)))
-                    return rc;
-            }
-        } else if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) {
-            return rc;
-        }
     } else {
         const size_t need = som_plan_workspace_bytes(n_samples, nnz, &pb);
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
@@ -487,6 +504,17 @@ int som_bmu_planned(som_handle* h, som_plan* p, int32_t* d_bmu, float* d_min_dis
     } else {
         // the plan was built for a table of p->n_hot rows: the handle's options must still give it
         if (som_table_geometry(h, false).n_hot != p->n_hot) return SOM_ERR_INVALID_ARG;
+        // two-stage search (option 7), as in som_bmu, when the shadow's layout holds the same table
+        if (h->opt_two_stage == 1 && h->shadow && h->shadow_valid && !h->Wh && h->M % 128 == 0 &&
+            som_table_geometry(h, true).n_hot == p->n_hot) {
+            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+            if ((rc = two_stage_search(h, p->indptr, p->indices, p->n, p->head, p->ws, p->pb, p->n_hot, d_bmu,
+                                       d_min_dist, nullptr, nullptr, st)))
+                return rc;
+            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
+            if (h->timing) h->ev_bmu_calls += 1;
+            return SOM_OK;
+        }
         SOM_CK(h, cudaMemsetAsync(p->ws + p->pb.keys, 0xFF, (size_t)(p->n + 16) * sizeof(unsigned long long), st));
         SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(p->head + p->pb.n_slots) + 3, 0, sizeof(int), st));
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;

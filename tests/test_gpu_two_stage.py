@@ -213,3 +213,27 @@ def test_two_stage_option_leaves_the_other_entry_points_alone(som_mod):
     for a, c in zip(h16a.bmu2(b.indptr, b.indices), h16b.bmu2(b.indptr, b.indices)):
         assert torch.equal(a.view(torch.int32), c.view(torch.int32))
     torch.cuda.synchronize()
+
+
+def test_two_stage_with_a_reusable_plan(som_mod):
+    """The planned search takes the two-stage route like som_bmu and gives the same bits, epoch after epoch."""
+    V, M, n = 30_000, 1_024, 60_000
+    W = synth.fill_codebook(V, M, 4, device="cuda")
+    b = synth.sample_csr(n, V, 11.0, 4, device="cuda")
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, 2)
+    h.set_option(7, 1)
+    plan = h.plan(b.indptr, b.indices)
+    for epoch in range(3):
+        if epoch:
+            W.mul_(0.9)
+            W[epoch::7] += 0.01
+        h.norms()
+        p_bmu, p_dist = plan.bmu()
+        unc_planned = h.last_uncertain()
+        d_bmu, d_dist = h.bmu(b.indptr, b.indices)
+        torch.cuda.synchronize()
+        assert 0 < unc_planned < n // 2 and unc_planned == h.last_uncertain()
+        assert torch.equal(p_bmu, d_bmu) and torch.equal(p_dist.view(torch.int32), d_dist.view(torch.int32))
+    _check(W.cpu().numpy(), V, M, b, p_bmu.cpu().numpy(), p_dist.cpu().numpy(), np.arange(0, n, 9))
+    plan.destroy()
