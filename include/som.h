@@ -284,11 +284,13 @@ int som_last_cuda_error(const som_handle* h);
  * again with the fp32 weights.  som_bmu2 does the same with the three best first-pass scores (both units
  * and their order certified).  Reported distances always come from the fp32 weights.
  * It pays on maps whose units are distinct at fp16 resolution (random initialisation, small final radius); on
- * a map that a wide blur has just smoothed most samples fail the certificate and the call is slower than
- * the plain search: read som_last_uncertain and switch the option off while that share is high.
+ * a map that a wide blur has just smoothed most samples fail the certificate.  A batch of at least 65536
+ * samples is therefore probed first (one sample in 256, chosen by sample index; one more stream
+ * synchronisation): if more than a fifth of those fail, the call runs the plain search instead.
  * Needs M % 128 == 0 and the row-table kernel.  A two-stage call synchronises the
  * stream a second time (it reads the length of the second pass's list back).  som_last_uncertain returns how
- * many samples the last two-stage search sent to its second pass.
+ * many samples the last two-stage search sent to its second pass (all of them when the probe chose the plain
+ * search).
  */
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);

@@ -152,7 +152,8 @@ int som_norms(som_handle* h, void* stream)
 
 // The two-stage search on a batch whose plan (slots in ws, table features in head) is ready: first
 // pass over the fp16 shadow keeping the two (som_bmu2: three) best units, certificate, exact fp32
-// pass for the samples it leaves open.  Synchronises the stream once (length of that list).
+// pass for the samples it leaves open.  Synchronises the stream once (length of that list), twice when
+// the batch is large enough to be probed first.
 static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
                             char* ws, const SomPlanBuffers& pb, int n_hot, int32_t* bmu, float* dist,
                             int32_t* bmu2, float* dist2, cudaStream_t st)
@@ -166,12 +167,58 @@ static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t*
     if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
     SOM_CK(h, cudaMemsetAsync(counters + 3, 0, sizeof(int), st));                   // search unit counter
     SOM_CK(h, cudaMemsetAsync(counters + SOM_PLAN_UNCERTAIN, 0, sizeof(int), st));  // length of the list
+    int32_t* uncertain = reinterpret_cast<int32_t*>(ws + pb.uncertain);
+    int* n_unc_dev = counters + SOM_PLAN_UNCERTAIN;
+    const SomTableGeom exact = som_table_geometry(h, false);
+
+    // Probe.  On a map whose neighbouring units differ by less than fp16 resolves (one that a wide
+    // blur has just smoothed) most samples fail the certificate, and a first pass over the whole
+    // batch is wasted.  So one sample in SOM_PROBE_STRIDE goes through first pass and certificate
+    // first; if more than a fifth of those fail, the batch takes the plain fp32 search.
+    if (n >= SOM_PROBE_MIN_BATCH && exact.n_hot == n_hot) {
+        const int64_t n_probe = (n + SOM_PROBE_STRIDE - 1) / SOM_PROBE_STRIDE;
+        const size_t pkb = (size_t)(n_probe + 16) * sizeof(unsigned long long);
+        SomPlanBuffers pp = pb;
+        pp.slots = pb.slots2;
+        pp.keys = pb.ukeys;
+        pp.keys2 = pb.ukeys2;  // (keys3 is not in use yet: its head serves the probe)
+        SOM_CK(h, cudaMemsetAsync(ws + pp.keys, 0xFF, pkb, st));
+        SOM_CK(h, cudaMemsetAsync(ws + pp.keys2, 0xFF, pkb, st));
+        if ((rc = som_launch_probe_gather(h, n, ws, pb, st))) return rc;
+        if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_probe, st))) return rc;
+        // (enough sample parts per neuron range that the short launch still occupies every SM)
+        const SomTableGeom first = som_table_geometry(h, true);
+        const int64_t n_ranges = (h->M + first.T - 1) / first.T;
+        const int64_t saved_parts = h->opt_parts;
+        h->opt_parts = (2 * (int64_t)h->sm_count + n_ranges - 1) / n_ranges;
+        rc = som_launch_bmu_table(h, true, n_probe, head, ws, pp, n_hot, top2 ? 3 : 2, st);
+        h->opt_parts = saved_parts;
+        if (rc) return rc;
+        if ((rc = som_launch_certify(h, indptr, indices, n_probe, ws, pp, top2, true, nullptr, nullptr, nullptr,
+                                     nullptr, nullptr, n_unc_dev, st)))
+            return rc;
+        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        SOM_CK(h, cudaStreamSynchronize(st));
+        const int64_t probe_unc = h->host_pair[3];
+        SOM_CK(h, cudaMemsetAsync(counters + 3, 0, sizeof(int), st));
+        SOM_CK(h, cudaMemsetAsync(n_unc_dev, 0, sizeof(int), st));
+        if (probe_unc * 5 > n_probe) {
+            // plain search on the same plan (keys and keys2 are still empty)
+            h->last_uncertain = n;
+            if ((rc = som_launch_bmu_table(h, false, n, head, ws, pb, n_hot, top2 ? 2 : 1, st))) return rc;
+            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+            if ((rc = som_launch_finalize_sorted(h, indptr, indices, n, ws, pb, false, bmu, dist, st))) return rc;
+            if (top2 && (rc = som_launch_finalize_sorted(h, indptr, indices, n, ws, pb, true, bmu2, dist2, st)))
+                return rc;
+            return SOM_OK;
+        }
+        if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
+    }
+
     if ((rc = som_launch_bmu_table(h, true, n, head, ws, pb, n_hot, top2 ? 3 : 2, st))) return rc;
     // certificate; certain samples are finalised, the others listed
-    int32_t* uncertain = reinterpret_cast<int32_t*>(ws + pb.uncertain);
-    int* n_unc_dev = reinterpret_cast<int*>(head + pb.n_slots) + SOM_PLAN_UNCERTAIN;
-    if ((rc = som_launch_certify(h, indptr, indices, n, ws, pb, bmu, dist, bmu2, dist2,
-                                 uncertain, n_unc_dev, st)))
+    if ((rc = som_launch_certify(h, indptr, indices, n, ws, pb, top2, false, bmu, dist, bmu2, dist2, uncertain,
+                                 n_unc_dev, st)))
         return rc;
     SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     SOM_CK(h, cudaStreamSynchronize(st));
@@ -183,7 +230,6 @@ static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t*
         // layouts hold the same number of hot rows), else the direct-load kernel.
         unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
         unsigned long long* ukeys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.ukeys2) : nullptr;
-        const SomTableGeom exact = som_table_geometry(h, false);
         const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T);
         const size_t ub = (size_t)(n_unc + 16) * sizeof(unsigned long long);
         SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, ub, st));

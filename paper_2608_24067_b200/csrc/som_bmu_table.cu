@@ -791,7 +791,9 @@ __device__ __forceinline__ float score_of_key(u64 key)
 // first-pass winners are the two best units of the exact weights, in that order, when both gaps
 // exceed the bounds of their two sides (s3 - s2: no third unit can overtake either; s2 - s1: they
 // cannot swap).
-template <bool SECOND>
+// COUNT_ONLY: the probe of the two-stage search; nothing is finalised or listed, the samples that fail the
+// certificate are only counted.
+template <bool SECOND, bool COUNT_ONLY>
 __global__ void k_certify(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
                           const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
                           const uint4* __restrict__ slots, const u64* __restrict__ keys,
@@ -848,7 +850,7 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
         if (!SECOND) certain = (s2 - s1) > e1 + eo;
         else certain = (s2 - s1) > e1 + e2 && (s3 - s2) > e2 + eo;  // (a map of two units has no third: exact pass)
         flag = !certain;
-        if (certain) {
+        if (certain && !COUNT_ONLY) {
             const uint32_t idx = (uint32_t)(k1 & 0xffffffffull);
             const uint32_t idx2 = (uint32_t)(k2 & 0xffffffffull);
             double dot = 0.0, dot2 = 0.0;
@@ -869,6 +871,10 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
     // slots are compacted to one contiguous run of the lists, so that the exact pass can run
     // the row-table kernel on the same plan.
     const unsigned int votes = __ballot_sync(0xffffffffu, flag);
+    if (COUNT_ONLY) {
+        if (lane == 0 && votes) atomicAdd(n_uncertain, __popc(votes));
+        return;
+    }
     if (lane == 0) warp_count[warp] = __popc(votes);
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -887,23 +893,49 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
 }  // namespace
 
 int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
-                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* bmu2, float* dist2,
-                       int32_t* uncertain, int* n_uncertain, cudaStream_t st)
+                       const SomPlanBuffers& b, bool second, bool count_only, int32_t* bmu, float* dist,
+                       int32_t* bmu2, float* dist2, int32_t* uncertain, int* n_uncertain, cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
     const uint4* slots = reinterpret_cast<const uint4*>(ws + b.slots);
     const u64* keys = reinterpret_cast<const u64*>(ws + b.keys);
     const u64* keys2 = reinterpret_cast<const u64*>(ws + b.keys2);
-    const u64* keys3 = reinterpret_cast<const u64*>(ws + b.keys3);
+    const u64* keys3 = second ? reinterpret_cast<const u64*>(ws + b.keys3) : nullptr;
     uint4* slots2 = reinterpret_cast<uint4*>(ws + b.slots2);
-    if (bmu2)
-        k_certify<true><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, slots, keys,
-                                                          keys2, keys3, h->wmax_bits, h->hnorm, bmu, dist, bmu2, dist2,
-                                                          uncertain, slots2, n_uncertain);
-    else
-        k_certify<false><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, slots, keys,
-                                                           keys2, nullptr, h->wmax_bits, h->hnorm, bmu, dist, nullptr,
-                                                           nullptr, uncertain, slots2, n_uncertain);
+#define SOM_CERTIFY(SECOND_, COUNT_)                                                                            \
+    k_certify<SECOND_, COUNT_><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, slots, \
+                                                                 keys, keys2, keys3, h->wmax_bits, h->hnorm, bmu,  \
+                                                                 dist, bmu2, dist2, uncertain, slots2, n_uncertain)
+    if (second && count_only) SOM_CERTIFY(true, true);
+    else if (second) SOM_CERTIFY(true, false);
+    else if (count_only) SOM_CERTIFY(false, true);
+    else SOM_CERTIFY(false, false);
+#undef SOM_CERTIFY
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
+    return SOM_OK;
+}
+
+// Probe of the two-stage search: the slot of every SOM_PROBE_STRIDE-th sample (by sample index) goes to
+// position index / SOM_PROBE_STRIDE of a second slot array.
+namespace {
+__global__ void k_probe_gather(const uint4* __restrict__ slots, int64_t n, uint4* __restrict__ probe)
+{
+    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n) return;
+    const uint32_t s = slots[k * SLOT_Q].y;
+    if (s % SOM_PROBE_STRIDE) return;
+    const int64_t pos = s / SOM_PROBE_STRIDE;
+#pragma unroll
+    for (int x = 0; x < SLOT_Q; ++x) probe[pos * SLOT_Q + x] = slots[k * SLOT_Q + x];
+}
+}  // namespace
+
+int som_launch_probe_gather(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, cudaStream_t st)
+{
+    const int64_t blocks = (n + 255) / 256;
+    k_probe_gather<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(ws + b.slots), n,
+                                                     reinterpret_cast<uint4*>(ws + b.slots2));
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

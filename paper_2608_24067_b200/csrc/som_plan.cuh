@@ -95,10 +95,17 @@ int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char
 // pads a slot array of n slots to a multiple of four with copies of the last one
 int som_launch_pad_slots(som_handle* h, char* ws, size_t slots_offset, int64_t n, cudaStream_t st);
 
-// bmu2 / dist2 non-null: the two-best search (needs the three best first-pass keys)
+// second: the two-best search (needs the three best first-pass keys); count_only: only count the
+// samples that fail the certificate into *n_uncertain (the probe; no outputs are touched)
 int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* ws,
-                       const SomPlanBuffers& b, int32_t* bmu, float* dist, int32_t* bmu2, float* dist2,
-                       int32_t* uncertain, int* n_uncertain, cudaStream_t st);
+                       const SomPlanBuffers& b, bool second, bool count_only, int32_t* bmu, float* dist,
+                       int32_t* bmu2, float* dist2, int32_t* uncertain, int* n_uncertain, cudaStream_t st);
+
+// The two-stage search first tries its certificate on one sample in SOM_PROBE_STRIDE (by sample index, so
+// the choice depends on the batch alone); batches below SOM_PROBE_MIN_BATCH samples are not probed.
+#define SOM_PROBE_STRIDE 256
+#define SOM_PROBE_MIN_BATCH 65536
+int som_launch_probe_gather(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, cudaStream_t st);
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                                char* ws, const SomPlanBuffers& b, bool second, int32_t* bmu, float* dist,

@@ -237,3 +237,28 @@ def test_two_stage_with_a_reusable_plan(som_mod):
         assert torch.equal(p_bmu, d_bmu) and torch.equal(p_dist.view(torch.int32), d_dist.view(torch.int32))
     _check(W.cpu().numpy(), V, M, b, p_bmu.cpu().numpy(), p_dist.cpu().numpy(), np.arange(0, n, 9))
     plan.destroy()
+
+
+def test_two_stage_probe_sends_a_smooth_map_to_the_plain_search(som_mod):
+    """Units that differ by less than fp16 resolves: the probe (one sample in 256 of a batch of at least
+    65536) fails the certificate nearly everywhere and the call takes the plain search on the same plan,
+    whose bits it must then reproduce; a smaller batch is not probed and goes through the exact pass."""
+    V, M, n = 4_000, 1_024, 100_000
+    base = synth.fill_codebook(V, 1, 3, device="cuda").view(V, 1)
+    noise = synth.fill_codebook(V, M, 8, device="cuda").view(V, M)
+    W = (base + 1e-5 * noise).contiguous().view(-1)
+    b = synth.sample_csr(n, V, 9.0, 3, device="cuda")
+    hs, bs, ds = _run(som_mod, W, V, M, b, True)
+    hp, bp, dp = _run(som_mod, W, V, M, b, False)
+    assert hs.last_uncertain() == n
+    assert np.array_equal(bs, bp) and np.array_equal(ds.view(np.uint32), dp.view(np.uint32))
+    _check(W.cpu().numpy(), V, M, b, bs, ds, np.arange(0, n, 23))
+    hs2, out_s = _run2(som_mod, W, V, M, b, True)
+    hp2, out_p = _run2(som_mod, W, V, M, b, False)
+    assert hs2.last_uncertain() == n
+    for a, c in zip(out_s, out_p):
+        assert np.array_equal(a.view(np.uint32), c.view(np.uint32))
+    small = synth.sample_csr(20_000, V, 9.0, 4, device="cuda")
+    h3, b3, d3 = _run(som_mod, W, V, M, small, True)
+    assert h3.last_uncertain() > 15_000
+    _check(W.cpu().numpy(), V, M, small, b3, d3, np.arange(0, 20_000, 7))
