@@ -195,51 +195,75 @@ constexpr int FUSED_THREADS_WIDE = 1024;
 constexpr int FUSED_PREFETCH = 16;  // cells per thread held in registers: planes of up to 4096 cells
 
 // lines of `len` cells: cell j of line l at buf[l * line_stride + j * cell_stride]
-template <typename BT>
+// All threads of the block call it; n_lines * seg <= blockDim.x, so a thread has at most one
+// segment.  With use_totals (worth it when the window is much longer than a segment; it costs
+// one block synchronisation) a segment's first window sum is put together from the totals of the
+// segments that lie wholly inside the window (each thread sums its own segment first; `tot` holds
+// one double per thread) and the few cells at the window's two ends; else from the window's cells.
+template <bool use_totals, typename BT>
 __device__ __forceinline__ void box_lines(const BT* __restrict__ in, BT* __restrict__ out, int n_lines,
-                                          int len, int line_stride, int cell_stride, int radius, int seg)
+                                          int len, int line_stride, int cell_stride, int radius, int seg,
+                                          double* __restrict__ tot)
 {
     const int seg_len = (len + seg - 1) / seg;
-    for (int job = threadIdx.x; job < n_lines * seg; job += blockDim.x) {
-        const int line = job % n_lines;
-        const int a = (job / n_lines) * seg_len;
-        const int b = min(len, a + seg_len);
-        if (a >= b) continue;
-        const BT* src = in + line * line_stride;
-        BT* dst = out + line * line_stride;
-        const int lo = max(0, a - radius), hi = min(len - 1, a + radius);
-        double s0 = 0.0, s1 = 0.0;
-        const BT* p = src + lo * cell_stride;
-        int j = lo;
-        for (; j + 1 <= hi; j += 2, p += 2 * cell_stride) {
-            s0 += (double)p[0];
-            s1 += (double)p[cell_stride];
+    const int job = threadIdx.x;
+    const bool busy = job < n_lines * seg;
+    const int line = busy ? job % n_lines : 0;
+    const int g = busy ? job / n_lines : 0;
+    const int a = g * seg_len;
+    const int b = min(len, a + seg_len);
+    const BT* src = in + line * line_stride;
+    if (busy && use_totals) {
+        double t0 = 0.0, t1 = 0.0;
+        const BT* p = src + a * cell_stride;
+        int j = a;
+        for (; j + 1 < b; j += 2, p += 2 * cell_stride) {
+            t0 += (double)p[0];
+            t1 += (double)p[cell_stride];
         }
-        if (j <= hi) s0 += (double)p[0];
-        double sum = s0 + s1;
-        BT* pd = dst + a * cell_stride;
+        if (j < b) t0 += (double)p[0];
+        tot[job] = t0 + t1;  // (an empty segment, a >= b, holds 0)
+    }
+    if (use_totals) __syncthreads();  // (the same for every thread of the block)
+    if (!busy || a >= b) return;
+    BT* dst = out + line * line_stride;
+    const int lo = max(0, a - radius), hi = min(len - 1, a + radius);
+    // segments g_lo .. g_hi lie wholly inside [lo, hi]
+    const int g_lo = (lo + seg_len - 1) / seg_len;
+    int g_hi = (hi + 1) / seg_len - 1;
+    if (hi == len - 1) g_hi = (len - 1) / seg_len;  // the last segment may be short; it ends at len - 1
+    double sum = 0.0;
+    int left_end = hi + 1, right_begin = hi + 1;  // cells [lo, left_end) and [right_begin, hi] are added singly
+    if (use_totals && g_lo <= g_hi) {
+        for (int q = g_lo; q <= g_hi; ++q) sum += tot[line + n_lines * q];
+        left_end = g_lo * seg_len;
+        right_begin = min(len, (g_hi + 1) * seg_len);
+    }
+    for (int j = lo; j < left_end; ++j) sum += (double)src[j * cell_stride];
+    for (int j = right_begin; j <= hi; ++j) sum += (double)src[j * cell_stride];
+    BT* pd = dst + a * cell_stride;
+    *pd = (BT)sum;
+    pd += cell_stride;
+    const BT* pe = src + (a + 1 + radius) * cell_stride;  // the cell entering the window
+    const BT* pl = src + (a - radius) * cell_stride;      // the cell leaving it
+    // i < len - radius: a cell enters; i > radius: a cell leaves
+    for (int i = a + 1; i < b; ++i, pe += cell_stride, pl += cell_stride, pd += cell_stride) {
+        const double enter = (i < len - radius) ? (double)*pe : 0.0;
+        const double leave = (i > radius) ? (double)*pl : 0.0;
+        sum += enter - leave;
         *pd = (BT)sum;
-        pd += cell_stride;
-        const BT* pe = src + (a + 1 + radius) * cell_stride;  // the cell entering the window
-        const BT* pl = src + (a - radius) * cell_stride;      // the cell leaving it
-        // i < len - radius: a cell enters; i > radius: a cell leaves
-        for (int i = a + 1; i < b; ++i, pe += cell_stride, pl += cell_stride, pd += cell_stride) {
-            const double enter = (i < len - radius) ? (double)*pe : 0.0;
-            const double leave = (i > radius) ? (double)*pl : 0.0;
-            sum += enter - leave;
-            *pd = (BT)sum;
-        }
     }
 }
 
 // BT: type of the two plane buffers (double: exact; float: rounded between passes like the
 // device-memory route, for planes too large for two fp64 buffers); running sums are fp64 either way.
-template <typename ST, typename BT, int THREADS>
+template <typename ST, typename BT, int THREADS, bool TOTALS>
 __global__ void __launch_bounds__(THREADS)
 k_upd_blur_fused(const float* __restrict__ slab, int planes, int rows, int cols, int radius, int seg_r, int seg_c,
                  const double* __restrict__ rden, ST* __restrict__ W, int v0)
 {
     extern __shared__ __align__(16) unsigned char fused_raw[];
+    __shared__ double tot[THREADS];
     const int pitch = cols | 1;  // odd, in cells
     const int M = rows * cols;   // <= FUSED_PREFETCH * THREADS
     BT* A = reinterpret_cast<BT*>(fused_raw);
@@ -282,12 +306,12 @@ k_upd_blur_fused(const float* __restrict__ slab, int planes, int rows, int cols,
         BT* x = A;
         BT* y = B;
         for (int pass = 0; pass < 3; ++pass) {  // along the lattice rows: a line is a row
-            box_lines(x, y, rows, cols, pitch, 1, radius, seg_r);
+            box_lines<TOTALS>(x, y, rows, cols, pitch, 1, radius, seg_r, tot);
             __syncthreads();
             BT* t = x; x = y; y = t;
         }
         for (int pass = 0; pass < 3; ++pass) {  // along the lattice columns: a line is a column
-            box_lines(x, y, cols, rows, 1, pitch, radius, seg_c);
+            box_lines<TOTALS>(x, y, cols, rows, 1, pitch, radius, seg_c, tot);
             __syncthreads();
             BT* t = x; x = y; y = t;
         }
@@ -314,6 +338,7 @@ k_upd_den_fused(const float* __restrict__ den_t, const int32_t* __restrict__ occ
                 int seg_r, int seg_c, double* __restrict__ rden)
 {
     extern __shared__ __align__(16) unsigned char fused_raw[];
+    __shared__ double tot[FUSED_THREADS];
     const int pitch = cols | 1;
     const int M = rows * cols;
     double* A = reinterpret_cast<double*>(fused_raw);
@@ -327,12 +352,12 @@ k_upd_den_fused(const float* __restrict__ den_t, const int32_t* __restrict__ occ
     double* x = A;
     double* y = B;
     for (int pass = 0; pass < 3; ++pass) {
-        box_lines(x, y, rows, cols, pitch, 1, radius, seg_r);
+        box_lines<false>(x, y, rows, cols, pitch, 1, radius, seg_r, tot);
         __syncthreads();
         double* t = x; x = y; y = t;
     }
     for (int pass = 0; pass < 3; ++pass) {
-        box_lines(x, y, cols, rows, 1, pitch, radius, seg_c);
+        box_lines<false>(x, y, cols, rows, 1, pitch, radius, seg_c, tot);
         __syncthreads();
         double* t = x; x = y; y = t;
     }
@@ -346,9 +371,9 @@ k_upd_den_fused(const float* __restrict__ den_t, const int32_t* __restrict__ occ
         A[r * pitch + c] = occ[i] > 0 ? 1.0 : 0.0;
     }
     __syncthreads();
-    box_lines(A, B, rows, cols, pitch, 1, 3 * radius, seg_r);
+    box_lines<false>(A, B, rows, cols, pitch, 1, 3 * radius, seg_r, tot);
     __syncthreads();
-    box_lines(B, A, cols, rows, 1, pitch, 3 * radius, seg_c);
+    box_lines<false>(B, A, cols, rows, 1, pitch, 3 * radius, seg_c, tot);
     __syncthreads();
     for (int i = threadIdx.x; i < M; i += blockDim.x) {
         const int r = i / cols, c = i - r * cols;
@@ -498,20 +523,29 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         // small lattices: everything after the scatter in one kernel, a plane at a time on chip
         const size_t fused_sh = 2 * plane_sh;
         if (fused) {
+            // segment totals for the first window sums where the window spans more than three segments
+            const bool totals = 2 * radius + 1 > 3 * ((cols + seg_r - 1) / seg_r) &&
+                                2 * radius + 1 > 3 * ((rows + seg_c - 1) / seg_c);
             const int per_sm = (int)((size_t)216 * 1024 / (fused_sh + 1024));
             int64_t grid = (int64_t)h->sm_count * per_sm;
             if (grid > planes) grid = planes;
-#define SOM_FUSED(ST_, BT_, THREADS_, W_)                                                                       \
+#define SOM_FUSED(ST_, BT_, THREADS_, TOT_, W_)                                                                 \
     do {                                                                                                        \
-        SOM_CK(h, cudaFuncSetAttribute(k_upd_blur_fused<ST_, BT_, THREADS_>,                                    \
+        SOM_CK(h, cudaFuncSetAttribute(k_upd_blur_fused<ST_, BT_, THREADS_, TOT_>,                              \
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused_sh));            \
-        k_upd_blur_fused<ST_, BT_, THREADS_><<<(unsigned)grid, THREADS_, fused_sh, st>>>(                       \
+        k_upd_blur_fused<ST_, BT_, THREADS_, TOT_><<<(unsigned)grid, THREADS_, fused_sh, st>>>(                 \
             slab_a, (int)planes, rows, cols, radius, seg_r, seg_c, rden, W_, v0);                               \
     } while (0)
-            if (h->Wh && wide) SOM_FUSED(__half, float, FUSED_THREADS_WIDE, const_cast<__half*>(h->Wh));
-            else if (h->Wh) SOM_FUSED(__half, double, FUSED_THREADS, const_cast<__half*>(h->Wh));
-            else if (wide) SOM_FUSED(float, float, FUSED_THREADS_WIDE, const_cast<float*>(h->W));
-            else SOM_FUSED(float, double, FUSED_THREADS, const_cast<float*>(h->W));
+#define SOM_FUSED_T(ST_, BT_, THREADS_, W_)                                                                     \
+    do {                                                                                                        \
+        if (totals) SOM_FUSED(ST_, BT_, THREADS_, true, W_);                                                    \
+        else SOM_FUSED(ST_, BT_, THREADS_, false, W_);                                                          \
+    } while (0)
+            if (h->Wh && wide) SOM_FUSED_T(__half, float, FUSED_THREADS_WIDE, const_cast<__half*>(h->Wh));
+            else if (h->Wh) SOM_FUSED_T(__half, double, FUSED_THREADS, const_cast<__half*>(h->Wh));
+            else if (wide) SOM_FUSED_T(float, float, FUSED_THREADS_WIDE, const_cast<float*>(h->W));
+            else SOM_FUSED_T(float, double, FUSED_THREADS, const_cast<float*>(h->W));
+#undef SOM_FUSED_T
 #undef SOM_FUSED
             h->launches += 1;
             SOM_CK(h, cudaGetLastError());
