@@ -586,7 +586,8 @@ int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indpt
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int planes = 1;
     const int64_t budget = (h->opt_update_mib > 0 ? h->opt_update_mib : 4096) << 20;
-    const size_t need = som_update_workspace_bytes(h, budget, &planes);
+    // (n_samples more words: the per-sample masks of the most frequent features, see below)
+    const size_t need = som_update_workspace_bytes(h, budget, &planes) + som_align_up((size_t)n_samples * 4, 256);
     int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need);
     if (rc) return rc;
     h->norms_valid = 0;  // the codebook changes: som_norms must run before the next search

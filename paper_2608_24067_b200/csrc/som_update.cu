@@ -82,37 +82,60 @@ __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t*
 
 // The planes of the most frequent features take most of the batch's increments (a feature that
 // 84 % of a million samples carry puts 200 atomic adds on every cell of one 4096-cell plane, and
-// same-address atomics queue in L2).  Block (slice, group) counts the increments of its group of
-// hot features over its slice of the samples in shared memory, then adds each non-zero count to
-// the plane once.  hot_slot[v] = rank of feature v among the hot ones or -1; slot_feat is its
-// inverse.
-__global__ void k_upd_scatter_hot(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
-                                  int64_t n, const int32_t* __restrict__ bmu, int v0, int v1, int rows, int cols,
-                                  const int32_t* __restrict__ hot_slot, const int32_t* __restrict__ slot_feat,
+// same-address atomics queue in L2).  k_upd_hot_mask notes per sample which of the (at most 16) hot
+// features it has; block (slice, group) of k_upd_scatter_hot then counts the increments of its group
+// of hot features over its slice of the samples in shared memory, reading only mask and best unit of
+// a sample, and adds each non-zero count to the plane once.  hot_slot[v] = rank of feature v among the
+// hot ones or -1; slot_feat is its inverse.
+__global__ void k_upd_hot_mask(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
+                               const int32_t* __restrict__ hot_slot, uint32_t* __restrict__ mask)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n) return;
+    uint32_t m = 0;
+    const int beg = indptr[s], end = indptr[s + 1];
+    for (int j = beg; j < end; ++j) {
+        const int slot = hot_slot[indices[j]];
+        if (slot >= 0) m |= 1u << slot;
+    }
+    mask[s] = m;
+}
+
+__global__ void k_upd_scatter_hot(const uint32_t* __restrict__ mask, int64_t n, const int32_t* __restrict__ bmu,
+                                  int v0, int v1, int rows, int cols, const int32_t* __restrict__ slot_feat,
                                   int planes_per_block, float* __restrict__ num_t)
 {
     extern __shared__ unsigned int cnt[];
     const int M = rows * cols;
     const int slot0 = blockIdx.y * planes_per_block;
     for (int e = threadIdx.x; e < planes_per_block * M; e += blockDim.x) cnt[e] = 0u;
+    // the group's slots whose feature lies in this slab
+    uint32_t group = 0;
+    for (int p = 0; p < planes_per_block && slot0 + p < 32; ++p) {
+        const int f = slot_feat[slot0 + p];
+        if (f >= v0 && f < v1) group |= 1u << (slot0 + p);
+    }
     __syncthreads();
     const int64_t per = (n + gridDim.x - 1) / gridDim.x;
     const int64_t s_lo = (int64_t)blockIdx.x * per, s_hi = min(n, s_lo + per);
-    for (int64_t s = s_lo + threadIdx.x; s < s_hi; s += blockDim.x) {
-        const int c = bmu[s];
-        const int r = c / cols, q = c - r * cols;
-        const int cell_t = q * rows + r;  // transposed cell order
-        const int beg = indptr[s], end = indptr[s + 1];
-        for (int j = beg; j < end; ++j) {
-            const int slot = hot_slot[indices[j]] - slot0;
-            if (slot >= 0 && slot < planes_per_block) atomicAdd(&cnt[slot * M + cell_t], 1u);
+    if (group) {
+        for (int64_t s = s_lo + threadIdx.x; s < s_hi; s += blockDim.x) {
+            uint32_t m = mask[s] & group;
+            if (!m) continue;
+            const int c = bmu[s];
+            const int r = c / cols, q = c - r * cols;
+            const int cell_t = q * rows + r;  // transposed cell order
+            while (m) {
+                const int slot = __ffs(m) - 1;
+                m &= m - 1;
+                atomicAdd(&cnt[(slot - slot0) * M + cell_t], 1u);
+            }
         }
     }
     __syncthreads();
     for (int p = 0; p < planes_per_block; ++p) {
-        const int f = slot_feat[slot0 + p];
-        if (f < v0 || f >= v1) continue;  // unused slot, or a feature of another slab
-        float* plane = num_t + (int64_t)(f - v0) * M;
+        if (!((group >> (slot0 + p)) & 1u)) continue;  // unused slot, or a feature of another slab
+        float* plane = num_t + (int64_t)(slot_feat[slot0 + p] - v0) * M;
         for (int e = threadIdx.x; e < M; e += blockDim.x) {
             const unsigned int k = cnt[p * M + e];
             if (k) atomicAdd(&plane[e], (float)k);
@@ -499,6 +522,12 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
     SOM_CK(h, cudaGetLastError());
 
     // ---- numerator, slab by slab ------------------------------------------------------------------
+    // (the per-sample masks of the hot features live behind the two slab buffers)
+    uint32_t* hot_mask = reinterpret_cast<uint32_t*>(ws + 8 * mb + 2 * som_align_up((size_t)planes_per_slab * M * 4, 256));
+    if (hot_slot && n > 0) {
+        k_upd_hot_mask<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, hot_slot, hot_mask);
+        h->launches += 1;
+    }
     for (int v0 = 0; v0 < h->V; v0 += planes_per_slab) {
         const int v1 = (v0 + planes_per_slab < h->V) ? v0 + planes_per_slab : h->V;
         const int64_t planes = v1 - v0;
@@ -515,8 +544,8 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
                 slices = slices < 1 ? 1 : (slices > 16 ? 16 : slices);
                 const size_t sh = (size_t)ppb * M * 4;
                 SOM_CK(h, cudaFuncSetAttribute(k_upd_scatter_hot, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh));
-                k_upd_scatter_hot<<<dim3(slices, groups), 1024, sh, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols,
-                                                                        hot_slot, slot_feat, ppb, slab_a);
+                k_upd_scatter_hot<<<dim3(slices, groups), 1024, sh, st>>>(hot_mask, n, bmu, v0, v1, rows, cols, slot_feat,
+                                                                        ppb, slab_a);
                 h->launches += 1;
             }
         }
