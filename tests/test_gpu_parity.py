@@ -392,3 +392,36 @@ def test_reusable_plan_matches_som_bmu(som_mod, variant):
     plan2 = h.plan(b.indptr, b.indices)
     rc = other._lib.som_bmu_planned(other._h, plan2._p, p_bmu.data_ptr(), p_dist.data_ptr(), None)
     assert rc == 1  # SOM_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("variant,store,two_stage", [(1, "f32", False), (2, "f32", False), (2, "f16", False),
+                                                      (2, "f32", True)])
+def test_search_on_a_smoothed_map(som_mod, variant, store, two_stage):
+    """A map right after a batch update with a wide blur (built by the update ORACLE from random
+    assignments): neighbouring units are nearly equal, so near ties abound.  Every kernel must stay
+    inside the parity rule there, and the two-stage search must fall back to exact scores."""
+    from oracle import som_update_oracle as uorc
+    V, rows, cols, n = 2_000, 32, 32, 70_000
+    M = rows * cols
+    rng = np.random.default_rng(21)
+    b = synth.sample_csr(n, V, 7.0, 6, device="cpu")
+    ip, ix = b.indptr.numpy(), b.indices.numpy()
+    W0 = synth.fill_codebook(V, M, 6, device="cpu").numpy()
+    assign = rng.integers(0, M, size=n).astype(np.int32)
+    W_host = uorc.update(W0, V, rows, cols, ip, ix, assign, 5).astype(np.float32)
+    if store == "f16":
+        W_dev = torch.from_numpy(W_host).cuda().half()
+        W_host = W_dev.float().cpu().numpy()  # the oracle sees the stored values
+    else:
+        W_dev = torch.from_numpy(W_host).cuda()
+    h = som_mod.Som(V, M, W_dev)
+    h.set_option(0, variant)
+    if two_stage:
+        h.set_option(7, 1)
+    h.norms()
+    g_bmu, g_dist = h.bmu(b.indptr.cuda(), b.indices.cuda())
+    torch.cuda.synchronize()
+    if two_stage:
+        assert h.last_uncertain() > n // 5
+    rep = _check_against_oracle(W_host, V, M, ip, ix, g_bmu.cpu().numpy(), g_dist.cpu().numpy(), np.arange(0, n, 7))
+    assert rep.near_ties > 0
