@@ -156,6 +156,12 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
     int end = __shfl_sync(0xffffffffu, end_l, 0);
     int first = (beg + lane < end) ? indices[beg + lane] : 0;
     float first_x = (VALUED && beg + lane < end) ? values[beg + lane] : 1.f;
+    // The key a sample's candidates are tested against before any index is tracked: its best so
+    // far, or with TOP2 its second best so far (a stale, larger value only lets more through).
+    // Lane q reads the key of the warp's q-th sample; volatile: other blocks lower it meanwhile.
+    const unsigned long long* filter_keys = TOP2 ? keys2 : keys;
+    unsigned long long key_l = ~0ull;
+    if (lane < n_mine) key_l = *reinterpret_cast<const volatile unsigned long long*>(filter_keys + s0 + lane);
 
     for (int q = 0; q < n_mine; ++q) {
         // the next sample's first 32 features are fetched while this one is searched
@@ -209,13 +215,29 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
                 }
             }
         }
-        // the lane's best (and second best) in ascending neuron order, then across the warp
         if (NEG) {
 #pragma unroll
             for (int t = 0; t < TILES; ++t)
 #pragma unroll
                 for (int k = 0; k < VEC; ++k) acc[t][k] = -acc[t][k];
         }
+        // Most visits change nothing: unless some lane's smallest score reaches the sample's
+        // current key, the indices, the shuffles and the atomics are skipped.
+        {
+            float mn = acc[0][0];
+#pragma unroll
+            for (int e = 1; e < TILES * VEC; ++e) mn = fminf(mn, acc[e / VEC][e % VEC]);
+            const uint32_t cu = (uint32_t)(__shfl_sync(0xffffffffu, key_l, q) >> 32);
+            const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);  // NaN for an empty key
+            if (!__any_sync(0xffffffffu, !(mn > cs))) {
+                beg = nbeg;
+                end = nend;
+                first = next;
+                first_x = next_x;
+                continue;
+            }
+        }
+        // the lane's best (and second best) in ascending neuron order, then across the warp
         float best = acc[0][0];
         uint32_t bi = (uint32_t)i0;
         float second = inf;            // TOP2: the lane's, then the warp's, second best
