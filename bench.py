@@ -439,7 +439,8 @@ def run_ours(args, w: synth.Workload):
         "roofline": roofline,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms},
+                "ms_per_step": e2e_ms,
+                "path": "som_norms + som_bmu_host_async / som_host_sync (binary samples, best unit) on the same batches"},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
