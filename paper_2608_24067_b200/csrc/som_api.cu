@@ -113,6 +113,12 @@ int som_destroy(som_handle* h)
     cudaFree(h->stage);
     cudaFree(h->head);
     cudaFree(h->shadow);
+    if (h->aux_stream) {
+        cudaStreamSynchronize(h->aux_stream);
+        cudaEventDestroy(h->ev_fork);
+        cudaEventDestroy(h->ev_join);
+        cudaStreamDestroy(h->aux_stream);
+    }
     if (h->copy_stream) {
         cudaStreamSynchronize(h->copy_stream);
         cudaStreamSynchronize(h->back_stream);
@@ -591,6 +597,14 @@ int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indpt
     int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need);
     if (rc) return rc;
     h->norms_valid = 0;  // the codebook changes: som_norms must run before the next search
+    // a side stream for the denominator's route, forked from `stream` here and joined inside
+    if (!h->aux_stream) {
+        SOM_CK(h, cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking));
+        SOM_CK(h, cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+        SOM_CK(h, cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+    }
+    SOM_CK(h, cudaEventRecord(h->ev_fork, st));
+    SOM_CK(h, cudaStreamWaitEvent(h->aux_stream, h->ev_fork, 0));
     // On small lattices with many samples the planes of the most frequent features are counted
     // in shared memory (see k_upd_scatter_hot); the plan's selection phase names those features.
     const int32_t* hot_slot = nullptr;
@@ -606,7 +620,7 @@ int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indpt
         slot_feat = reinterpret_cast<const int32_t*>(head + pb.slot_feat);
     }
     return som_launch_update(h, rows, cols, d_indptr, d_indices, n_samples, d_bmu, radius, planes, hot_slot,
-                             slot_feat, n_hot_slots, st);
+                             slot_feat, n_hot_slots, st, h->aux_stream, h->ev_join);
 }
 
 int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indices, int64_t n_samples,

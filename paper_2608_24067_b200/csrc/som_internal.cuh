@@ -38,6 +38,8 @@ struct som_handle {
     size_t stage_bytes;
     // pipelined host entry point (som_bmu_host_async): copy stream, two staging buffers, events
     cudaStream_t copy_stream, back_stream;  // host-to-device and device-to-host
+    cudaStream_t aux_stream;                // som_update: side stream of the denominator's route
+    cudaEvent_t ev_fork, ev_join;
     cudaEvent_t ev_h2d[2], ev_searched[2], ev_d2h[2];
     void* pipe_stage[2];
     size_t pipe_stage_bytes[2];
@@ -115,4 +117,5 @@ size_t som_norms_workspace_bytes(const som_handle* h);
 size_t som_update_workspace_bytes(const som_handle* h, int64_t budget_bytes, int* planes_per_slab);
 int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, const int32_t* indices,
                       int64_t n, const int32_t* bmu, int radius, int planes_per_slab, const int32_t* hot_slot,
-                      const int32_t* slot_feat, int n_hot_slots, cudaStream_t st);
+                      const int32_t* slot_feat, int n_hot_slots, cudaStream_t st, cudaStream_t aux,
+                      cudaEvent_t ev_join);

@@ -464,8 +464,14 @@ size_t som_update_workspace_bytes(const som_handle* h, int64_t budget_bytes, int
 
 int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, const int32_t* indices,
                       int64_t n, const int32_t* bmu, int radius, int planes_per_slab, const int32_t* hot_slot,
-                      const int32_t* slot_feat, int n_hot_slots, cudaStream_t st)
+                      const int32_t* slot_feat, int n_hot_slots, cudaStream_t st, cudaStream_t aux,
+                      cudaEvent_t ev_join)
 {
+    // The denominator's route (single-block kernels) and the clearing of the first slab run on the
+    // side stream `aux`, which the caller has made wait for `st`; `st` joins it before the scatter.
+    // Meanwhile `st` runs the selection of the frequent features and their masks.
+    cudaStream_t main_st = st;
+    if (aux) st = aux;
     const int64_t M = h->M;
     const size_t mb = som_align_up((size_t)M * 4, 256);
     char* ws = reinterpret_cast<char*>(h->ws);
@@ -521,6 +527,12 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
     }
     SOM_CK(h, cudaGetLastError());
 
+    if (aux) {
+        const int64_t first = planes_per_slab < h->V ? planes_per_slab : h->V;
+        SOM_CK(h, cudaMemsetAsync(slab_a, 0, (size_t)first * M * 4, aux));
+        SOM_CK(h, cudaEventRecord(ev_join, aux));
+        st = main_st;
+    }
     // ---- numerator, slab by slab ------------------------------------------------------------------
     // (the per-sample masks of the hot features live behind the two slab buffers)
     uint32_t* hot_mask = reinterpret_cast<uint32_t*>(ws + 8 * mb + 2 * som_align_up((size_t)planes_per_slab * M * 4, 256));
@@ -531,7 +543,8 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
     for (int v0 = 0; v0 < h->V; v0 += planes_per_slab) {
         const int v1 = (v0 + planes_per_slab < h->V) ? v0 + planes_per_slab : h->V;
         const int64_t planes = v1 - v0;
-        SOM_CK(h, cudaMemsetAsync(slab_a, 0, (size_t)planes * M * 4, st));
+        if (aux && v0 == 0) SOM_CK(h, cudaStreamWaitEvent(st, ev_join, 0));  // first slab cleared, denominator ready
+        else SOM_CK(h, cudaMemsetAsync(slab_a, 0, (size_t)planes * M * 4, st));
         if (n > 0) {
             k_upd_scatter<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols, hot_slot,
                                                                  slab_a);
