@@ -301,8 +301,8 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     // enough (neuron range x sample part) units to occupy every SM; everything else goes to
     // the direct-load kernel.  So do, in automatic mode, batches whose most frequent features
     // cover too few feature instances for a shared-memory table to pay: there the direct-load
-    // kernel, bound by L2 bandwidth alone, is faster (measured cross-over: about half of the
-    // instances).
+    // kernel, bound by L2 bandwidth alone, is faster (measured cross-over: between a half and
+    // two thirds of the instances).
     const SomTableGeom geom = som_table_geometry(h, two_stage_ok);
     bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
                      h->M < ((int64_t)1 << 30);
