@@ -603,12 +603,15 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         const u64 l1 = old > c1 ? old : c1;
                         const u64 old2 = atomicMin(k2, l1);
                         if (KEEP == 3) atomicMin(k3, old2 > l1 ? old2 : l1);
+                        // the lane's second smallest score first; its index only if it can matter
                         float m2 = inf;
-                        int r2 = 0;
 #pragma unroll
-                        for (int j = R - 1; j >= 0; --j)
-                            if (j != rr && a[j] <= m2) { m2 = a[j]; r2 = j; }
+                        for (int j = 0; j < R; ++j) m2 = fminf(m2, j == rr ? inf : a[j]);
                         if (!(m2 > cs)) {
+                            int r2 = rr == R - 1 ? R - 2 : R - 1;
+#pragma unroll
+                            for (int j = R - 1; j >= 0; --j)
+                                if (j != rr && a[j] == m2) r2 = j;  // lowest such neuron
                             const u64 c2 = som_pack_key(m2, i_first + L::neuron_of(r2));
                             const u64 o2 = atomicMin(k2, c2);
                             if (KEEP == 3) {
