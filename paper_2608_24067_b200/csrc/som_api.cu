@@ -590,6 +590,8 @@ int som_update(som_handle* h, int32_t rows, int32_t cols, const int32_t* d_indpt
     if (n_samples >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
     DeviceGuard g(h->device);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // a window that already spans the lattice along both axes does not grow any more
+    if (radius > (rows > cols ? rows : cols)) radius = rows > cols ? rows : cols;
     int planes = 1;
     const int64_t budget = (h->opt_update_mib > 0 ? h->opt_update_mib : 4096) << 20;
     // (n_samples more words: the per-sample masks of the most frequent features, see below)

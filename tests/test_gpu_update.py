@@ -157,6 +157,15 @@ def test_update_with_frequent_features_counted_on_chip(som_mod, mib):
     _check(got, W_old, w.V, rows, cols, b.indptr.numpy(), b.indices.numpy(), bmu, 2, rtol=1e-6)
 
 
+def test_update_with_a_huge_radius_equals_a_radius_that_spans_the_lattice(som_mod):
+    V, rows, cols, n = 9, 12, 20, 300
+    indptr, indices, bmu, W_old = _problem(2, V, rows, cols, n)
+    huge = _run(som_mod, W_old, V, rows, cols, indptr, indices, bmu, 2 ** 30)
+    spans = _run(som_mod, W_old, V, rows, cols, indptr, indices, bmu, 20)
+    assert np.array_equal(huge, spans)
+    _check(spans, W_old, V, rows, cols, indptr, indices, bmu, 20, rtol=1e-6)
+
+
 def test_update_rejects_bad_lattice(som_mod):
     V, rows, cols = 10, 4, 4
     W = torch.zeros(V * rows * cols, device="cuda")
