@@ -120,7 +120,8 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
              const float* __restrict__ values = nullptr)
 {
     constexpr int TILE = 32 * VEC;  // neurons per tile
-    constexpr int FEATS = 4;        // features whose row segments are in flight together
+    // features whose row segments are in flight together (fp16 rows are half as long: twice as many)
+    constexpr int FEATS = sizeof(ST) == 2 ? 8 : 4;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int64_t i0 = neuron_off + (int64_t)blockIdx.y * (TILES * TILE) + lane * VEC;
