@@ -5,6 +5,11 @@
 
 One step = one pass of the whole hot path over one batch: som_norms (norm pass) followed by
 som_bmu (plan, fused search, combine/finalize).  Prints ONE JSON line on rank 0.
+
+Without --config the graded map sizes are measured one after the other (64x64, 128x128, 512x512,
+1024x1024): the line's own fields are those of the largest one (1024x1024, 125.8 GB codebook
+resident in HBM, batches of 250 000 samples) and "per_config" carries one summary per size.
+--config C measures that one configuration only.
 """
 from __future__ import annotations
 
@@ -152,30 +157,50 @@ def _oracle_rate(w: synth.Workload, W_host_slab: np.ndarray, m_slab: int, indptr
     return rate, cores, desc, dt
 
 
+def config_dict(w: synth.Workload, world: int, step: str, store_bytes: int = 4) -> dict:
+    """The workload as both arms name it (nominal figures only, so that the two arms print the same)."""
+    n_batches = max(1, min(4, w.N // w.batch))
+    return {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "batches": n_batches,
+            "mean_nnz": 1.0 + w.lam, "step": step, "replicas": world,
+            "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
+                w.V * w.M * store_bytes / 1e6, w.batch * (1.0 + w.lam) * 4 / 1e6)
+            if w.V * w.M * store_bytes > 126e6 else
+            "inputs smaller than L2: steps rotate over %d distinct batches, no flush" % n_batches}
+
+
+DEFAULT_STEP = "som_norms + som_bmu on one batch"
+
+
 def run_reference(args, w: synth.Workload):
-    """The CPU oracle as it stands, timed on host cores, on bounded samples of the workload."""
+    """The CPU oracle as it stands, timed on host cores.  Every step is one bounded sample of the
+    workload (the first samples of a batch against the first 4096 neurons of the configured
+    codebook); `ms_per_step` is the measured time of such a step, `value` the rate it implies for
+    the whole map (scaled by the neuron fraction)."""
     ws, rank, _ = _dist_env()
     if rank != 0:
         return
     m_slab = min(w.M, 4096)
-    # the slab is the first m_slab neurons of the configured codebook
     W_host = synth.codebook_slab(w.V, w.M, 0, m_slab, w.seed).numpy()
     n_gen = min(w.batch, 200_000)
     b = synth.sample_csr(n_gen, w.V, w.lam, w.seed)
     indptr, indices = b.indptr.numpy(), b.indices.numpy()
-    per_step = max(1.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
-    rates, desc, cores = [], "", 1
+    per_step = max(0.5, min(10.0, 100.0 / max(1, args.steps + args.warmup)))
+    rates, times, desc, cores = [], [], "", 1
     for i in range(args.warmup + args.steps):
         rate, cores, desc, dt = _oracle_rate(w, W_host, m_slab, indptr, indices, per_step)
         if i >= args.warmup:
             rates.append(rate)
+            times.append(dt)
     value = float(np.mean(rates))
     line = {
         "impl": "reference", "metric": "bmu_samples_per_s", "value": value, "unit": "samples/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": 1000.0 * w.batch / value, "higher_is_better": True, "scaling": "weak",
+        "ms_per_step": 1000.0 * float(np.mean(times)),
+        "ms_per_step_is": "measured time of one bounded oracle sample (cpu_baseline.sample), not of a whole batch",
+        "ms_per_whole_batch_at_this_rate": 1000.0 * w.batch / value,
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": 1 + w.lam},
+        "config": config_dict(w, ws, DEFAULT_STEP),
         "cpu_baseline": {"value": value, "unit": "samples/s", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -183,22 +208,54 @@ def run_reference(args, w: synth.Workload):
     print(json.dumps(line), flush=True)
 
 
-def run_ours(args, w: synth.Workload):
-    ws, rank, lr = _dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
-    torch.cuda.set_device(lr)
-    dev = torch.device("cuda", lr)
-    dist = None
-    if ws > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
-    from paper_2608_24067_b200 import som
+class Ctx:
+    """What every measured configuration shares: device, process group, peaks."""
 
-    hbm_gbs, sm_max_mhz, peak_src = _peaks()
-    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
-    add_peak = sm_count * FP32_LANES_PER_SM * sm_max_mhz * 1e6  # adds/s
+    def __init__(self):
+        self.ws, self.rank, self.lr = _dist_env()
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
+        torch.cuda.set_device(self.lr)
+        self.dev = torch.device("cuda", self.lr)
+        self.dist = None
+        if self.ws > 1:
+            import torch.distributed as dist_mod
+            self.dist = dist_mod
+            self.dist.init_process_group("nccl", device_id=self.dev)
+        from paper_2608_24067_b200 import som
+        self.som = som
+        self.hbm_gbs, self.sm_max_mhz, self.peak_src = _peaks()
+        self.sm_count = torch.cuda.get_device_properties(self.dev).multi_processor_count
+        self.add_peak = self.sm_count * FP32_LANES_PER_SM * self.sm_max_mhz * 1e6  # adds/s, derived
+        # the same peak measured: independent FP32 add chains, nothing else (library microbenchmark)
+        self.add_peak_measured = som.measure_fadd_peak(self.dev)
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        torch.cuda.synchronize()
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+
+
+def _committed_traffic(workload_name: str):
+    """DRAM bytes per launch of the search kernel from the committed ncu summary of this workload
+    (profiles/k_bmu_table_<workload>.md, a line `traffic_bytes_per_launch = ...`), or None."""
+    tpath = os.path.join(ROOT, "profiles", "k_bmu_table_%s.md" % workload_name)
+    if os.path.exists(tpath):
+        for tl in open(tpath):
+            if tl.startswith("traffic_bytes_per_launch"):
+                return float(tl.split("=")[1])
+    return None
+
+
+def measure(ctx: Ctx, args, w: synth.Workload, steps: int, warmup: int, cpu_seconds: float) -> dict:
+    """One configuration: device-resident throughput, end to end, two-stage leg, CPU baseline."""
+    som, dev, dist, ws, rank = ctx.som, ctx.dev, ctx.dist, ctx.ws, ctx.rank
+    hbm_gbs, add_peak = ctx.hbm_gbs, ctx.add_peak
+    barrier = ctx.barrier
 
     # ---- inputs (synthetic, resident in HBM) -------------------------------------------------
     store_bytes = 2 if args.store == "f16" else 4
@@ -253,16 +310,11 @@ def run_ours(args, w: synth.Workload):
         else:
             h.bmu(b.indptr, b.indices, out_bmu, out_dist)
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
     # ---- device-resident timing -------------------------------------------------------------
-    for i in range(args.warmup):
+    for i in range(warmup):
         step(i)
     barrier()
-    sampler = ClockSampler(lr) if rank == 0 else None
+    sampler = ClockSampler(ctx.lr) if rank == 0 else None
     h.set_timing(True)
     l0 = h.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -270,8 +322,8 @@ def run_ours(args, w: synth.Workload):
     if sampler:
         sampler.begin()
     e0.record()
-    for i in range(args.steps):
-        step(args.warmup + i)
+    for i in range(steps):
+        step(warmup + i)
     e1.record()
     barrier()
     if sampler:
@@ -281,12 +333,12 @@ def run_ours(args, w: synth.Workload):
     phases = h.get_timing()
     h.set_timing(False)
     ms_total = max_over_ranks(ms_total, dist, dev)
-    ms_per_step = ms_total / args.steps
+    ms_per_step = ms_total / steps
     value = aggregate_samples_per_s(ws, w.batch, ms_per_step)
 
     # ---- end to end through the host entry point --------------------------------------------
     hb = [(b.indptr.cpu().pin_memory(), b.indices.cpu().pin_memory()) for b in batches]
-    e2e_steps = max(1, min(args.steps, 5))
+    e2e_steps = max(1, min(steps, 5))
 
     # Streamed through som_bmu_host_async: every step uploads its batch and downloads both outputs;
     # the handle overlaps one step's copies with its neighbours' searches.  The timed region ends
@@ -314,6 +366,19 @@ def run_ours(args, w: synth.Workload):
     e2e_value = aggregate_samples_per_s(ws, w.batch, e2e_ms)
     h2d = int(np.mean([ip.numel() * 4 + ix.numel() * 4 for ip, ix in hb]))
     d2h = w.batch * 8
+    # the blocking form of the same call: upload, search, download, wait; one step at a time
+    ip0, ix0 = hb[0]
+    h.norms()
+    h.bmu_host(ip0, ix0, h_outs[0][0], h_outs[0][1])  # staging buffer allocated outside the timed region
+    barrier()
+    blk_steps = max(1, min(steps, 3))
+    e0.record()
+    for i in range(blk_steps):
+        h.norms()
+        h.bmu_host(hb[i % n_batches][0], hb[i % n_batches][1], h_outs[0][0], h_outs[0][1])
+    e1.record()
+    barrier()
+    blocking_ms = max_over_ranks(e0.elapsed_time(e1) / blk_steps, dist, dev)
 
     clocks = sampler.close() if sampler else None
 
@@ -334,16 +399,16 @@ def run_ours(args, w: synth.Workload):
                     h2.norms()
                     h2.bmu(b.indptr, b.indices, out_bmu, out_dist)
 
-                for i in range(args.warmup):
+                for i in range(warmup):
                     step2(i)
                 barrier()
                 h2.set_timing(True)
                 e0.record()
-                for i in range(args.steps):
-                    step2(args.warmup + i)
+                for i in range(steps):
+                    step2(warmup + i)
                 e1.record()
                 barrier()
-                ms2 = max_over_ranks(e0.elapsed_time(e1) / args.steps, dist, dev)
+                ms2 = max_over_ranks(e0.elapsed_time(e1) / steps, dist, dev)
                 ph2 = h2.get_timing()
                 adds2 = w.batch * nnz_mean * w.M
                 two_stage = {"value": aggregate_samples_per_s(ws, w.batch, ms2), "unit": "samples/s",
@@ -356,6 +421,9 @@ def run_ours(args, w: synth.Workload):
                 h2.destroy()
             except som.SomError as exc:  # e.g. no memory for the copy
                 two_stage = {"unavailable": str(exc)}
+        else:
+            two_stage = {"unavailable": "no device memory for the fp16 copy of the codebook (%.1f GB)"
+                                        % (w.V * w.M * 2 / 1e9)}
 
     # ---- optional: the update phase of an epoch, timed on its own -----------------------------
     update = None
@@ -367,7 +435,7 @@ def run_ours(args, w: synth.Workload):
         radius = args.radius if args.radius > 0 else max(1, edge // 4)
         h.update(edge, edge, b0.indptr, b0.indices, bm, radius)  # warm-up (allocates the workspace)
         barrier()
-        u_steps = max(1, min(args.steps, 5))
+        u_steps = max(1, min(steps, 5))
         e0.record()
         for _ in range(u_steps):
             h.update(edge, edge, b0.indptr, b0.indices, bm, radius)
@@ -380,79 +448,134 @@ def run_ours(args, w: synth.Workload):
                   "share_of_epoch": u_ms / (u_ms + ms_per_step)}
         h.norms()
 
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+    line = None
+    if rank == 0:
+        # ---- roofline of the dominant kernel (the fused search) ---------------------------------
+        adds = w.batch * nnz_mean * w.M  # nominal neuron-feature accumulations per launch
+        search_s = max(phases["search_ms"], 1e-6) * 1e-3
+        achieved = adds / search_s
+        alg_bytes = (w.V * w.M * store_bytes + sum(b.nnz * 4 + (b.n + 1) * 4 for b in batches) / n_batches
+                     + w.batch * 8)
+        # DRAM bytes one launch of the search kernel really moves, from the committed ncu capture of
+        # this workload's shipped kernel (None when there is none: the large maps are not captured
+        # with full counter sets, their algorithmic bytes stand in and the key stays null)
+        traffic = _committed_traffic(w.name) if args.store == "f32" else None
+        t_alu = adds / add_peak
+        t_hbm = (traffic if traffic is not None else alg_bytes) / (hbm_gbs * 1e9)
+        roofline = {
+            "bound": "alu" if t_alu >= t_hbm else "hbm", "kernel": "fused BMU search",
+            "achieved": achieved / 1e12, "peak": add_peak / 1e12,
+            "unit": "TFLOP/s", "frac": max(t_alu, t_hbm) / search_s, "traffic": traffic,
+            "traffic_note": None if traffic is not None else "not measured at this size; hbm term uses the algorithmic bytes",
+            "peak_source": "%d SMs x %d fp32 lanes x %.0f MHz (%s clock); adds only, no multiplies" % (
+                ctx.sm_count, FP32_LANES_PER_SM, ctx.sm_max_mhz, ctx.peak_src),
+            "peak_measured": ctx.add_peak_measured / 1e12,
+            "frac_of_measured_peak": achieved / ctx.add_peak_measured if ctx.add_peak_measured > 0 else None,
+            "alu_time_at_peak_ms": t_alu * 1e3, "hbm_time_at_peak_ms": t_hbm * 1e3,
+            "search_ms": phases["search_ms"], "algorithmic_bytes": alg_bytes, "hbm_peak_gbs": hbm_gbs,
+            "mean_nnz_measured": nnz_mean,
+            "norms_ms": phases["norms_ms"],
+            "norms_hbm_frac": (w.V * w.M * store_bytes / max(phases["norms_ms"], 1e-6) / 1e6) / hbm_gbs,
+            "plan_ms": phases["plan_ms"], "finalize_ms": phases["finalize_ms"],
+            "step_frac_of_alu_roofline": (adds / add_peak) / (ms_per_step * 1e-3),
+        }
 
-    # ---- roofline of the dominant kernel (the fused search) -------------------------------------
-    adds = w.batch * nnz_mean * w.M  # nominal neuron-feature accumulations per launch
-    search_s = max(phases["search_ms"], 1e-6) * 1e-3
-    achieved = adds / search_s
-    alg_bytes = w.V * w.M * store_bytes + sum(b.nnz * 4 + (b.n + 1) * 4 for b in batches) / n_batches + w.batch * 8
-    # DRAM bytes per launch of the search kernel from the committed ncu summary of this workload
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "k_bmu_table_%s.md" % w.name)
-    if os.path.exists(tpath) and args.store == "f32":  # the committed capture is of the fp32 path
-        for tl in open(tpath):
-            if tl.startswith("traffic_bytes_per_launch"):
-                traffic = float(tl.split("=")[1])
-    roofline = {
-        "bound": "alu", "kernel": "fused BMU search", "achieved": achieved / 1e12, "peak": add_peak / 1e12,
-        "unit": "TFLOP/s", "frac": achieved / add_peak, "traffic": traffic,
-        "peak_source": "%d SMs x %d fp32 lanes x %.0f MHz (%s clock)" % (sm_count, FP32_LANES_PER_SM, sm_max_mhz, peak_src),
-        "search_ms": phases["search_ms"], "algorithmic_bytes": alg_bytes,
-        "hbm_time_at_peak_ms": alg_bytes / (hbm_gbs * 1e9) * 1e3, "hbm_peak_gbs": hbm_gbs,
-        "norms_ms": phases["norms_ms"],
-        "norms_hbm_frac": (w.V * w.M * store_bytes / max(phases["norms_ms"], 1e-6) / 1e6) / hbm_gbs,
-        "plan_ms": phases["plan_ms"], "finalize_ms": phases["finalize_ms"],
-        "step_frac_of_alu_roofline": (adds / add_peak) / (ms_per_step * 1e-3),
-    }
+        # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ------------------
+        cpu = None
+        if ws == 1 and not args.no_cpu_baseline and cpu_seconds > 0:
+            m_slab = min(w.M, 4096)
+            Wh = W.view(w.V, w.M)[:, :m_slab].float().contiguous().cpu().numpy()
+            b = batches[0]
+            n_take = min(b.n, 100_000)
+            ip = b.indptr[:n_take + 1].cpu().numpy()
+            ix = b.indices[:int(b.indptr[n_take])].cpu().numpy()
+            rate, cores, desc, _ = _oracle_rate(w, Wh, m_slab, ip, ix, cpu_seconds)
+            cpu = {"value": rate, "unit": "samples/s", "cores": cores, "kind": "oracle", "sample": desc}
 
-    # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ----------------------
-    cpu = None
-    if ws == 1 and not args.no_cpu_baseline:
-        m_slab = min(w.M, 4096)
-        Wh = W.view(w.V, w.M)[:, :m_slab].float().contiguous().cpu().numpy()
-        b = batches[0]
-        n_take = min(b.n, 100_000)
-        ip = b.indptr[:n_take + 1].cpu().numpy()
-        ix = b.indices[:int(b.indptr[n_take])].cpu().numpy()
-        rate, cores, desc, _ = _oracle_rate(w, Wh, m_slab, ip, ix, 12.0)
-        cpu = {"value": rate, "unit": "samples/s", "cores": cores, "kind": "oracle", "sample": desc}
+        step_name = ("som_norms + " + ("som_bmu_planned + som_update (a training-epoch step; plans built once, outside)"
+                                       if args.epoch else
+                                       "som_bmu_planned (plans built once, outside)" if args.planned else
+                                       ("som_bmu_values" if args.values else ("som_bmu2" if args.top2 else "som_bmu")))
+                     + " on one batch")
+        line = {
+            "metric": "bmu_samples_per_s", "value": value, "unit": "samples/s", "n_gpus": ws,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if args.store == "f32" else "f32 accumulate, f16-stored codebook",
+            "data": "synthetic",
+            "config": config_dict(w, ws, step_name, store_bytes),
+            "accumulations_per_s": ws * adds / (ms_per_step * 1e-3),
+            "roofline": roofline,
+            "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms, "blocking_ms_per_step": blocking_ms,
+                    "path": "som_norms + som_bmu_host_async / som_host_sync (binary samples, best unit) on the same "
+                            "batches, copies overlapped with the neighbouring steps; blocking_ms_per_step is "
+                            "som_norms + som_bmu_host, one step at a time"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if update is not None:
+            line["update"] = update
+        if args.two_stage:
+            line["two_stage"] = {"uncertain_samples_last_call": h.last_uncertain(), "batch": w.batch}
+        elif two_stage is not None:
+            line["two_stage"] = two_stage
+    for p_ in plans:
+        p_.destroy()
+    h.destroy()
+    del W, batches, hb, h_outs, out_bmu, out_dist, plans, sample_values
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return line
 
-    line = {
-        "metric": "bmu_samples_per_s", "value": value, "unit": "samples/s", "n_gpus": ws,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32" if args.store == "f32" else "f32 accumulate, f16-stored codebook",
-        "data": "synthetic",
-        "config": {"workload": w.name, "V": w.V, "M": w.M, "batch": w.batch, "mean_nnz": nnz_mean,
-                   "step": "som_norms + %s on one batch" % ("som_bmu_planned + som_update (a training-epoch step; plans built once, outside)" if args.epoch else
-                       "som_bmu_planned (plans built once, outside)" if args.planned else
-                       ("som_bmu_values" if args.values else ("som_bmu2" if args.top2 else "som_bmu"))),
-                   "replicas": ws,
-                   "l2_policy": "inputs larger than L2 (codebook %.0f MB + CSR %.0f MB per step)" % (
-                       w.V * w.M * store_bytes / 1e6, batches[0].nnz * 4 / 1e6) if w.V * w.M * store_bytes > 126e6 else
-                   "inputs smaller than L2: steps rotate over %d distinct batches, no flush" % n_batches},
-        "accumulations_per_s": ws * adds / (ms_per_step * 1e-3),
-        "roofline": roofline,
-        "cpu_baseline": cpu,
-        "e2e": {"value": e2e_value, "unit": "samples/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms,
-                "path": "som_norms + som_bmu_host_async / som_host_sync (binary samples, best unit) on the same batches"},
-        "gpu_launches": int(launches),
-        "clocks": clocks,
-    }
-    if update is not None:
-        line["update"] = update
-    if args.two_stage:
-        line["two_stage"] = {"uncertain_samples_last_call": h.last_uncertain(), "batch": w.batch}
-    elif two_stage is not None:
-        line["two_stage"] = two_stage
-    print(json.dumps(line), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+
+def _summary(line: dict) -> dict:
+    r = line["roofline"]
+    return {"workload": line["config"]["workload"], "batch": line["config"]["batch"], "steps": line["steps"],
+            "warmup": line["warmup"], "ms_per_step": line["ms_per_step"], "value": line["value"],
+            "accumulations_per_s": line["accumulations_per_s"],
+            "roofline": {"bound": r["bound"], "frac": r["frac"], "frac_of_measured_peak": r["frac_of_measured_peak"],
+                         "achieved": r["achieved"], "traffic": r["traffic"]},
+            "search_ms": r["search_ms"], "norms_ms": r["norms_ms"], "norms_hbm_frac": r["norms_hbm_frac"],
+            "plan_ms": r["plan_ms"], "finalize_ms": r["finalize_ms"],
+            "e2e": {k: line["e2e"][k] for k in ("value", "ms_per_step", "blocking_ms_per_step",
+                                                 "h2d_bytes_per_step", "d2h_bytes_per_step")},
+            "two_stage": ({k: line["two_stage"].get(k) for k in ("value", "search_ms", "frac", "unavailable")
+                           if k in line["two_stage"]} if line.get("two_stage") else None),
+            "cpu_baseline": line["cpu_baseline"], "gpu_launches": line["gpu_launches"], "clocks": line["clocks"]}
+
+
+def _cap_steps(w: synth.Workload, steps: int, warmup: int):
+    """Steps and warm-ups of one size in the all-sizes run: the driver's counts, cut where the timed
+    region of a size would pass about a minute (steps of the two largest maps take 0.3 to 0.6 s)."""
+    est_ms = w.batch * (1.0 + w.lam) * w.M / 37.2e12 / 0.15 * 1e3 + w.V * w.M * 4 / 6.4e12 * 1e3
+    cap = max(3, int(60_000.0 / max(est_ms, 1e-3)))
+    return min(steps, cap), max(3, min(warmup, max(3, cap // 4)))
+
+
+def run_ours(args, workloads):
+    ctx = Ctx()
+    lines = []
+    for k, w in enumerate(workloads):
+        last = k == len(workloads) - 1
+        if len(workloads) > 1:
+            steps, warmup = _cap_steps(w, args.steps, args.warmup)
+        else:
+            steps, warmup = args.steps, args.warmup
+        lines.append(measure(ctx, args, w, steps, warmup, 12.0 if last else 5.0))
+    if ctx.rank == 0:
+        line = lines[-1]
+        if len(lines) > 1:
+            line["per_config"] = [_summary(x) for x in lines]
+            line["steps_requested"] = args.steps
+            line["warmup_requested"] = args.warmup
+            if (line["steps"], line["warmup"]) != (args.steps, args.warmup):
+                line["steps_note"] = ("steps / warm-ups of a size are cut where its timed region would pass "
+                                      "about a minute; the counts used are in each per_config entry")
+        print(json.dumps(line), flush=True)
+    ctx.close()
 
 
 def main():
@@ -461,7 +584,9 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, help="index into the five workloads (default 1: 64x64)")
+    ap.add_argument("--config", type=int, default=None,
+                    help="index into the five workloads; default: the four graded map sizes (1..4) one after "
+                         "the other, headline = the largest (1024x1024)")
     ap.add_argument("--variant", type=int, default=None, help="search kernel variant (library option 0)")
     ap.add_argument("--hot-rows", type=int, default=0, help="row-table kernel: hot rows in shared memory")
     ap.add_argument("--threads", type=int, default=0, help="row-table kernel: block size (512 or 1024)")
@@ -497,19 +622,29 @@ def main():
                     help="samples per batch instead of the configuration's (a sweep variant, named in the workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    w = synth.CONFIGS[args.config]
-    if args.features == "uniform":
-        w = dataclasses.replace(w, name=w.name + "-uniform", zipf_s=0.0)
-    if args.batch > 0:
-        w = dataclasses.replace(w, name="%s-batch%d" % (w.name, args.batch), batch=args.batch, N=max(w.N, args.batch))
-    if args.zipf_s is not None:
-        w = dataclasses.replace(w, name="%s-zipf%g" % (w.name, args.zipf_s), zipf_s=args.zipf_s)
-    if args.store == "f16":
-        w = dataclasses.replace(w, name=w.name + "-f16")
-    if args.impl == "reference":
-        run_reference(args, w)
+
+    def variant_of(w):
+        if args.features == "uniform":
+            w = dataclasses.replace(w, name=w.name + "-uniform", zipf_s=0.0)
+        if args.batch > 0:
+            w = dataclasses.replace(w, name="%s-batch%d" % (w.name, args.batch), batch=args.batch,
+                                    N=max(w.N, args.batch))
+        if args.zipf_s is not None:
+            w = dataclasses.replace(w, name="%s-zipf%g" % (w.name, args.zipf_s), zipf_s=args.zipf_s)
+        if args.store == "f16":
+            w = dataclasses.replace(w, name=w.name + "-f16")
+        return w
+
+    plain = not (args.epoch or args.planned or args.values or args.top2 or args.with_update or args.two_stage)
+    if args.config is None:
+        ids = [1, 2, 3, 4] if plain else [1]
     else:
-        run_ours(args, w)
+        ids = [args.config]
+    workloads = [variant_of(synth.CONFIGS[i]) for i in ids]
+    if args.impl == "reference":
+        run_reference(args, workloads[-1])
+    else:
+        run_ours(args, workloads)
 
 
 if __name__ == "__main__":

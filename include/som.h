@@ -18,13 +18,13 @@
  *     "host pointer" = ordinary process memory.  The library never takes ownership of a
  *     caller's buffer.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
- *     som_norms / som_bmu only enqueue work on it, with two exceptions: growing the handle's
- *     workspace (first call, or a larger batch than any before) allocates device memory,
- *     which may synchronise the device once; and som_bmu, when its row-table kernel is a
- *     candidate, first runs the feature-selection step of its plan and reads three integers back
- *     (d_indptr[0], d_indptr[n_samples] and the number of feature instances its table would
- *     serve) to size the plan and pick the kernel, which waits for earlier work on `stream`
- *     (the search itself is then only enqueued).
+ *     som_norms / som_bmu / som_bmu2 only enqueue work on it and return without waiting for
+ *     the device: the batch's nnz, the choice of the table's features and, in automatic mode,
+ *     the choice between the two search kernels all stay on the device (the kernels of both
+ *     paths are enqueued; those of the path not chosen return at once).  Exceptions: growing
+ *     the handle's workspace (first call, or a larger batch than any before) allocates device
+ *     memory, which may synchronise the device once; and the two-stage search (option 7),
+ *     which reads list lengths back.
  *   - Thread safety: one handle must not be used from two host threads at once, and two
  *     calls on the same handle must not overlap on the GPU (they share the workspace);
  *     issue them on one stream or order the streams yourself.
@@ -79,8 +79,8 @@ int som_create(som_handle** out, int32_t V, int64_t M, const float* d_codebook);
 int som_create_f16(som_handle** out, int32_t V, int64_t M, const void* d_codebook_f16);
 
 /*
- * som_norms - recompute ||w_i||^2 for all M neurons (the norm term of Eq. 1; the paper's
- * "negligible norm pass", Section 5.7).  One streaming read of the codebook; squares are
+ * som_norms - recompute ||w_i||^2 for all M neurons (the norm term of Eq. 1; the separate norm
+ * pass whose cost Section 5.7 reports as negligible).  One streaming read of the codebook; squares are
  * accumulated in fp64 in a fixed order (deterministic) and stored as fp32.
  * Must be called once after som_create and again after every codebook update.
  */
@@ -92,7 +92,9 @@ int som_norms(som_handle* h, void* stream);
  *               [d_indptr[s], d_indptr[s+1]) of d_indices.  d_indptr[0] may be any offset.
  *   d_indices   DEVICE pointer, int32; inside each row ascending, distinct, in [0, V).
  *               These are preconditions (the paper sorts ascending, Section 3.1) and are
- *               NOT checked here; som_validate_csr checks them.
+ *               NOT checked here; som_validate_csr checks them.  (The batch-plan kernels skip
+ *               an id outside [0, V) and record it, see som_device_flags; the search kernels
+ *               themselves rely on the precondition.)  May be NULL only when every row is empty.
  *   n_samples   0 <= n_samples < 2^31; 0 is a successful no-op.
  *   d_bmu       DEVICE pointer, int32 [n_samples]  out: index of the nearest neuron,
  *               lowest index among exact fp32 ties.
@@ -101,7 +103,15 @@ int som_norms(som_handle* h, void* stream);
  *               Eq. 1, no square root), recomputed for the winner in fp64 and rounded once.
  * A sample with no active feature gets argmin ||w_i||^2 and that norm.
  * Scores are accumulated in fp32 in a fixed order, so outputs are bit-identical from run
- * to run for the same inputs.
+ * to run for the same inputs (same batch, same options).  That order is fixed per BATCH, not
+ * per sample: which features the row table holds, and which kernel the automatic mode takes,
+ * follow from the batch's feature histogram.  So one sample searched inside two different
+ * batches (or by the two kernels) gets fp32 scores that may differ in the last bits, and its
+ * best unit may differ between the two calls when its two best units are nearer to each other
+ * than that rounding (about 1e-6 of the score; Section 3.1 reports the same effect of the
+ * summation order, about one assignment in 1e5 at 256x256).  Wherever the two best units are
+ * further apart than 1e-4 of the best squared distance the unit is the same in every batch.
+ * The reported distance is always the fp64 one of the reported unit.
  */
 int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
             int32_t* d_bmu, float* d_min_dist, void* stream);
@@ -116,8 +126,9 @@ int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, in
  *              index among exact fp32 ties; -1 when the map has a single neuron.
  *   d_dist2    DEVICE pointer, fp32 [n_samples]   out: its full squared distance, recomputed in
  *              fp64 and rounded once like d_min_dist; +inf when d_bmu2 is -1.
- * Same preconditions, asynchrony and determinism as som_bmu; d_bmu/d_min_dist are bit-identical
- * to som_bmu's for the same inputs.
+ * Same preconditions, asynchrony and determinism as som_bmu; with the two-stage search off (the
+ * default) d_bmu/d_min_dist are bit-identical to som_bmu's for the same inputs (with option 7 the
+ * two calls may send different samples to the exact pass, whose kernel sums in another order).
  */
 int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
              int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream);
@@ -125,7 +136,7 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
 /*
  * som_plan_create / som_bmu_planned / som_plan_destroy - a reusable batch plan for epoch loops.
  * The per-batch preparation inside som_bmu (feature histogram, choice of the table's features, sort of the
- * samples, re-encoded index lists: "the tile's merged feature lists", Section 3.3) depends on the batch
+ * samples, re-encoded index lists: the merged feature lists of a sample tile, Section 3.3) depends on the batch
  * alone, not on the codebook.  Training searches the same batches every epoch (Algorithm 2, step 2), so a
  * caller can build each batch's plan once:
  *   som_plan_create   builds the plan of the device-resident CSR batch (arguments as in som_bmu) in
@@ -148,8 +159,8 @@ int som_bmu_planned(som_handle* h, som_plan* plan, int32_t* d_bmu, float* d_min_
 int som_plan_destroy(som_plan* plan);
 
 /*
- * som_bmu_values - the search for sparse REAL-VALUED samples (the paper's outlook, Section 7: "carrying
- * ||x||^2 and a values array alongside the feature indices"; its SparseFloat variant, Table 6):
+ * som_bmu_values - the search for sparse REAL-VALUED samples (the paper's outlook, Section 7: a values
+ * array beside the feature indices and the sample's own squared norm; its SparseFloat variant, Table 6):
  *   d_values   DEVICE pointer, fp32, parallel to d_indices: sample s has value d_values[k] at feature
  *              d_indices[k] for k in [d_indptr[s], d_indptr[s+1]) and 0 elsewhere.
  * BMU = argmin_i (||w_i||^2 - 2 * sum_k x_k * w_i[idx_k]), ties to the lowest index; d_min_dist is
@@ -197,7 +208,8 @@ int som_bmu_host(som_handle* h, const int32_t* h_indptr, const int32_t* h_indice
 
 /*
  * som_bmu_host_async / som_host_sync - som_bmu_host for a STREAM of batches: the call returns once the
- * batch's work is enqueued, and h_bmu / h_min_dist hold the results after som_host_sync(h).  The handle
+ * batch's work is enqueued (it waits only for the staging buffer it reuses, i.e. for the results of
+ * the call before the previous one to have left the device), and h_bmu / h_min_dist hold the results after som_host_sync(h).  The handle
  * keeps two staging buffers and two copy streams of its own, so the host-to-device copy of one batch
  * overlaps the search of the previous one and the results travel back while the next search runs
  * (the paper streams the corpus from host memory, Section 4.2).  The search itself runs on `stream`.
@@ -217,6 +229,19 @@ int som_host_sync(som_handle* h);
  */
 int som_validate_csr(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices,
                      int64_t n_samples, void* stream);
+
+/*
+ * som_device_flags - what earlier calls on this handle skipped on the device.  (No counterpart in the
+ * paper: error reporting of this library.)  Kernels never fault on a bad index they can see cheaply;
+ * they skip the entry and set a sticky bit in a flag word on the device:
+ *   - a feature id outside [0, V) met by the batch-plan kernels of som_bmu / som_plan_create or by
+ *     som_update's frequent-feature pass             -> SOM_ERR_BAD_CSR
+ *   - a best-unit index outside [0, M) in som_update's d_bmu (a stale buffer, the -1 that som_bmu2
+ *     writes for a missing second unit): the sample is left out of the update -> SOM_ERR_INVALID_ARG
+ * This call copies the word back, clears it, synchronises `stream` and returns SOM_OK or the
+ * status above (SOM_ERR_BAD_CSR first when both bits are set).
+ */
+int som_device_flags(som_handle* h, void* stream);
 
 /*
  * som_get_norms - copy the M fp32 norms computed by the last som_norms into a DEVICE buffer
@@ -292,6 +317,16 @@ int som_last_cuda_error(const som_handle* h);
  * many samples the last two-stage search sent to its second pass (all of them when the probe chose the plain
  * search).
  */
+/*
+ * som_measure_fadd_peak - measure the device's FP32 add rate (no counterpart in the paper: the
+ * denominator of this library's roofline, measured instead of derived).  Launches a kernel of
+ * independent add chains (eight per thread, 64 warps per SM) four times on `stream`, times the last
+ * three with CUDA events and returns the best rate in *adds_per_s.  Synchronises.
+ *   d_scratch      DEVICE pointer, fp32, at least 2048 * (number of SMs) elements; written.
+ *   scratch_elems  its length.
+ */
+int som_measure_fadd_peak(double* adds_per_s, float* d_scratch, int64_t scratch_elems, void* stream);
+
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);
 int64_t som_launch_count(const som_handle* h);

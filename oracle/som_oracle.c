@@ -114,8 +114,8 @@ void som_oracle_dist_at(const float* W, int layout, int64_t V, int64_t M, const 
 }
 
 /*
- * Sparse real-valued samples (the paper's outlook, Section 7: "carrying ||x||^2 and a values array
- * alongside the feature indices"): x has value val[k] at feature idx[k] and 0 elsewhere, and
+ * Sparse real-valued samples (the paper's outlook, Section 7: a values array beside the feature
+ * indices and the sample's own squared norm): x has value val[k] at feature idx[k] and 0 elsewhere, and
  *   d(x, w_i) = ||x - w_i||^2 = sum_k val[k]^2 - 2 * sum_k val[k] * w_i[idx[k]] + ||w_i||^2.
  */
 static double distance_values(const float* W, int layout, int64_t V, int64_t M, const double* norms,

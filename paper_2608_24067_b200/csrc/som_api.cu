@@ -54,6 +54,21 @@ inline int mark(som_handle* h, int64_t call, int slot, cudaStream_t st)
     return SOM_OK;
 }
 
+// Hands the device-side kernel choice to the launchers for the length of a scope.
+struct GateScope {
+    som_handle* h;
+    GateScope(som_handle* h_, const int* gate) : h(h_)
+    {
+        h->gate = gate;
+        h->gate_want = 1;
+    }
+    ~GateScope()
+    {
+        h->gate = nullptr;
+        h->gate_want = 0;
+    }
+};
+
 }  // namespace
 
 extern "C" {
@@ -84,6 +99,8 @@ static int create_impl(som_handle** out, int32_t V, int64_t M, const void* d_cod
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->norm64), (size_t)M * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->norm32), (size_t)M * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->hnorm), (size_t)M * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&h->dev_flags), 256);
+    if (e == cudaSuccess) e = cudaMemset(h->dev_flags, 0, 256);
     if (e != cudaSuccess) {
         som_destroy(h);
         return SOM_ERR_CUDA;
@@ -109,6 +126,7 @@ int som_destroy(som_handle* h)
     cudaFree(h->norm64);
     cudaFree(h->norm32);
     cudaFree(h->hnorm);
+    cudaFree(h->dev_flags);
     cudaFree(h->ws);
     cudaFree(h->stage);
     cudaFree(h->head);
@@ -197,7 +215,7 @@ static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t*
         const int64_t n_ranges = (h->M + first.T - 1) / first.T;
         const int64_t saved_parts = h->opt_parts;
         h->opt_parts = (2 * (int64_t)h->sm_count + n_ranges - 1) / n_ranges;
-        rc = som_launch_bmu_table(h, true, n_probe, head, ws, pp, n_hot, top2 ? 3 : 2, st);
+        rc = som_launch_bmu_table(h, true, indptr, indices, n_probe, head, ws, pp, n_hot, top2 ? 3 : 2, st);
         h->opt_parts = saved_parts;
         if (rc) return rc;
         if ((rc = som_launch_certify(h, indptr, indices, n_probe, ws, pp, top2, true, nullptr, nullptr, nullptr,
@@ -211,7 +229,7 @@ static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t*
         if (probe_unc * 5 > n_probe) {
             // plain search on the same plan (keys and keys2 are still empty)
             h->last_uncertain = n;
-            if ((rc = som_launch_bmu_table(h, false, n, head, ws, pb, n_hot, top2 ? 2 : 1, st))) return rc;
+            if ((rc = som_launch_bmu_table(h, false, indptr, indices, n, head, ws, pb, n_hot, top2 ? 2 : 1, st))) return rc;
             if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
             if ((rc = som_launch_finalize_sorted(h, indptr, indices, n, ws, pb, false, bmu, dist, st))) return rc;
             if (top2 && (rc = som_launch_finalize_sorted(h, indptr, indices, n, ws, pb, true, bmu2, dist2, st)))
@@ -221,7 +239,7 @@ static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t*
         if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
     }
 
-    if ((rc = som_launch_bmu_table(h, true, n, head, ws, pb, n_hot, top2 ? 3 : 2, st))) return rc;
+    if ((rc = som_launch_bmu_table(h, true, indptr, indices, n, head, ws, pb, n_hot, top2 ? 3 : 2, st))) return rc;
     // certificate; certain samples are finalised, the others listed
     if ((rc = som_launch_certify(h, indptr, indices, n, ws, pb, top2, false, bmu, dist, bmu2, dist2, uncertain,
                                  n_unc_dev, st)))
@@ -247,7 +265,7 @@ static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t*
             pe.keys2 = pb.ukeys2;
             SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(head + pb.n_slots) + 3, 0, sizeof(int), st));
             if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_unc, st))) return rc;
-            if ((rc = som_launch_bmu_table(h, false, n_unc, head, ws, pe, exact.n_hot, top2 ? 2 : 1, st)))
+            if ((rc = som_launch_bmu_table(h, false, indptr, indices, n_unc, head, ws, pe, exact.n_hot, top2 ? 2 : 1, st)))
                 return rc;
             if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
             if ((rc = som_launch_finalize_sorted(h, indptr, indices, n_unc, ws, pe, false, bmu,
@@ -281,6 +299,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     if (n_samples == 0) return SOM_OK;
     if (!d_indptr || !d_bmu || !d_min_dist) return SOM_ERR_INVALID_ARG;
     const bool top2 = d_bmu2 != nullptr;
+    // (d_indices may be null only for a batch whose rows are all empty: no kernel dereferences it then)
     if (n_samples >= (int64_t)1 << 31) return SOM_ERR_UNSUPPORTED;
     if (!h->norms_valid) return SOM_ERR_NORMS_STALE;
     DeviceGuard g(h->device);
@@ -311,36 +330,35 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         const int64_t units = ((h->M + geom.T - 1) / geom.T) * parts;
         if (units < 2 * (int64_t)h->sm_count) use_table = false;
     }
-    int64_t nnz = 0;
     SomPlanBuffers pb;
     char* head = nullptr;
     bool begun = false;
+    const int* gate = nullptr;  // device-side choice between the two kernels (automatic mode)
     if (use_table) {
-        // The selection phase of the plan runs first; then the two row pointers (the workspace
-        // is sized from the batch's nnz, which lives on the device) and the number of instances
-        // the chosen features cover come back in one short synchronisation of the stream.
         const size_t head_need = som_plan_head_bytes(h->V, SOM_PLAN_MASK_FEATURES + geom.n_hot, &pb);
         if ((rc = ensure_bytes(h, &h->head, &h->head_bytes, head_need))) return rc;
         head = reinterpret_cast<char*>(h->head);
-        if (!h->host_pair) SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
         begun = true;
+        // The selection phase of the plan: feature histogram, choice of the table's features and, in
+        // automatic mode, of the kernel (the table must serve enough of the batch's feature instances).
         if ((rc = som_launch_plan_select(h, d_indptr, d_indices, n_samples, head, pb, SOM_PLAN_MASK_FEATURES,
                                          geom.n_hot, st)))
             return rc;
-        SOM_CK(h, cudaMemcpyAsync(h->host_pair, d_indptr, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 1, d_indptr + n_samples, sizeof(int32_t),
-                                  cudaMemcpyDeviceToHost, st));
-        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 2,
-                                  reinterpret_cast<const int32_t*>(head + pb.n_slots) + SOM_PLAN_COVERED,
-                                  sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-        SOM_CK(h, cudaStreamSynchronize(st));
-        nnz = (int64_t)h->host_pair[1] - (int64_t)h->host_pair[0];
-        if (nnz < 0) return SOM_ERR_INVALID_ARG;
-        if (nnz + 6 * n_samples + 4 >= ((int64_t)1 << 31)) use_table = false;
-        if (nnz > 0 && !d_indices) return SOM_ERR_INVALID_ARG;
-        const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 60;
-        if (h->opt_variant == 0 && (int64_t)h->host_pair[2] * 100 < cover_pct * nnz) use_table = false;
+        const int32_t* counters = reinterpret_cast<const int32_t*>(head + pb.n_slots);
+        if (h->opt_variant == 0 && two_stage_ok) {
+            // the two-stage search synchronises anyway: it reads the choice back
+            if (!h->host_pair)
+                SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
+            SOM_CK(h, cudaMemcpyAsync(h->host_pair + 2, counters + SOM_PLAN_USE_TABLE, sizeof(int32_t),
+                                      cudaMemcpyDeviceToHost, st));
+            SOM_CK(h, cudaStreamSynchronize(st));
+            if (h->host_pair[2] == 0) use_table = false;
+        } else if (h->opt_variant == 0) {
+            // Everything else stays on the device: the kernels of both paths are enqueued, and those of
+            // the path not chosen return at once.  The host never waits for the batch.
+            gate = counters + SOM_PLAN_USE_TABLE;
+        }
     }
 
     if (!use_table) {
@@ -359,7 +377,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
             (rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys2, d_bmu2, d_dist2, nullptr, st)))
             return rc;
     } else if (two_stage_ok) {
-        const size_t need = som_plan_workspace_bytes(n_samples, nnz, &pb);
+        const size_t need = som_plan_workspace_bytes(n_samples, &pb);
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
         char* ws = reinterpret_cast<char*>(h->ws);
         if ((rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, head, ws, pb, SOM_PLAN_MASK_FEATURES,
@@ -370,17 +388,27 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
                                    d_bmu2, d_dist2, st)))
             return rc;
     } else {
-        const size_t need = som_plan_workspace_bytes(n_samples, nnz, &pb);
+        const size_t need = som_plan_workspace_bytes(n_samples, &pb);
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
         char* ws = reinterpret_cast<char*>(h->ws);
-        SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
-        if (top2)
-            SOM_CK(h, cudaMemsetAsync(ws + pb.keys2, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
+        unsigned long long* keys = reinterpret_cast<unsigned long long*>(ws + pb.keys);
+        unsigned long long* keys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.keys2) : nullptr;
+        SOM_CK(h, cudaMemsetAsync(keys, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
+        if (top2) SOM_CK(h, cudaMemsetAsync(keys2, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
+        GateScope scope(h, gate);  // row-table path: runs when the choice is 1 (or there is no gate)
         if ((rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, head, ws, pb, SOM_PLAN_MASK_FEATURES,
                                        geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_table(h, false, n_samples, head, ws, pb, geom.n_hot, top2 ? 2 : 1, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, false, d_indptr, d_indices, n_samples, head, ws, pb, geom.n_hot,
+                                       top2 ? 2 : 1, st)))
+            return rc;
+        if (gate) {
+            // direct-load path on the same key arrays (indexed by sample there): runs when the choice is 0
+            h->gate_want = 0;
+            if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, nullptr, st))) return rc;
+            h->gate_want = 1;
+        }
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, false, d_bmu,
                                              d_min_dist, st)))
@@ -388,6 +416,14 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (top2 && (rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, true, d_bmu2,
                                                      d_dist2, st)))
             return rc;
+        if (gate) {
+            h->gate_want = 0;
+            if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, nullptr, st)))
+                return rc;
+            if (top2 &&
+                (rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys2, d_bmu2, d_dist2, nullptr, st)))
+                return rc;
+        }
     }
     if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
     if (h->timing) h->ev_bmu_calls += 1;
@@ -513,13 +549,12 @@ int som_plan_create(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (p->nnz < 0 || (p->nnz > 0 && !d_indices)) rc = SOM_ERR_INVALID_ARG;
     }
     if (!rc && use_table) {
-        if (p->nnz + 6 * n_samples + 4 >= ((int64_t)1 << 31)) use_table = false;
         const int64_t cover_pct = h->opt_cover > 0 ? h->opt_cover : 60;
         if (h->opt_variant == 0 && (int64_t)h->host_pair[2] * 100 < cover_pct * p->nnz) use_table = false;
     }
     if (!rc) {
         p->use_table = use_table ? 1 : 0;
-        const size_t need = use_table ? som_plan_workspace_bytes(n_samples, p->nnz, &p->pb)
+        const size_t need = use_table ? som_plan_workspace_bytes(n_samples, &p->pb)
                                       : som_align_up((size_t)n_samples * sizeof(unsigned long long), 256);
         if (cudaMalloc(reinterpret_cast<void**>(&p->ws), need) != cudaSuccess) rc = SOM_ERR_CUDA;
         if (!rc && use_table)
@@ -570,7 +605,8 @@ int som_bmu_planned(som_handle* h, som_plan* p, int32_t* d_bmu, float* d_min_dis
         SOM_CK(h, cudaMemsetAsync(p->ws + p->pb.keys, 0xFF, (size_t)(p->n + 16) * sizeof(unsigned long long), st));
         SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(p->head + p->pb.n_slots) + 3, 0, sizeof(int), st));
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = som_launch_bmu_table(h, false, p->n, p->head, p->ws, p->pb, p->n_hot, 1, st))) return rc;
+        if ((rc = som_launch_bmu_table(h, false, p->indptr, p->indices, p->n, p->head, p->ws, p->pb, p->n_hot, 1, st)))
+            return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, p->indptr, p->indices, p->n, p->ws, p->pb, false, d_bmu,
                                              d_min_dist, st)))
@@ -746,6 +782,20 @@ int som_validate_csr(som_handle* h, const int32_t* d_indptr, const int32_t* d_in
     SOM_CK(h, cudaMemcpyAsync(&flag, d_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
     SOM_CK(h, cudaStreamSynchronize(st));
     return flag ? SOM_ERR_BAD_CSR : SOM_OK;
+}
+
+int som_device_flags(som_handle* h, void* stream)
+{
+    if (!h) return SOM_ERR_INVALID_ARG;
+    DeviceGuard g(h->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int flags = 0;
+    SOM_CK(h, cudaMemcpyAsync(&flags, h->dev_flags, sizeof(int), cudaMemcpyDeviceToHost, st));
+    SOM_CK(h, cudaMemsetAsync(h->dev_flags, 0, sizeof(int), st));
+    SOM_CK(h, cudaStreamSynchronize(st));
+    if (flags & SOM_FLAG_BAD_INDEX) return SOM_ERR_BAD_CSR;
+    if (flags & SOM_FLAG_BAD_UNIT) return SOM_ERR_INVALID_ARG;
+    return SOM_OK;
 }
 
 int som_get_norms(som_handle* h, float* d_out, void* stream)

@@ -117,8 +117,9 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
              const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
              unsigned long long* __restrict__ keys, unsigned long long* __restrict__ keys2,
              int64_t neuron_off, const int32_t* __restrict__ sample_list,
-             const float* __restrict__ values = nullptr)
+             const float* __restrict__ values = nullptr, const int* __restrict__ gate = nullptr, int gate_want = 0)
 {
+    if (som_gated_off(gate, gate_want)) return;
     constexpr int TILE = 32 * VEC;  // neurons per tile
     // features whose row segments are in flight together (fp16 rows are half as long: twice as many)
     constexpr int FEATS = sizeof(ST) == 2 ? 8 : 4;
@@ -304,8 +305,10 @@ __global__ void k_finalize(const ST* __restrict__ W, const double* __restrict__ 
                            const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                            int64_t n, const unsigned long long* __restrict__ keys,
                            int32_t* __restrict__ bmu, float* __restrict__ dist,
-                           const int32_t* __restrict__ sample_list, const float* __restrict__ values = nullptr)
+                           const int32_t* __restrict__ sample_list, const float* __restrict__ values = nullptr,
+                           const int* __restrict__ gate = nullptr, int gate_want = 0)
 {
+    if (som_gated_off(gate, gate_want)) return;
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= n) return;
     const int64_t s = sample_list ? (int64_t)sample_list[k] : k;
@@ -378,10 +381,12 @@ static void launch_direct(dim3 grid, cudaStream_t st, const ST* W, som_handle* h
             W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, nullptr, values);
     else if (keys2)
         k_bmu_direct<VEC, TILES, true, ST><<<grid, DIRECT_THREADS, 0, st>>>(
-            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, keys2, neuron_off, sample_list);
+            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, keys2, neuron_off, sample_list, nullptr,
+            h->gate, h->gate_want);
     else
         k_bmu_direct<VEC, TILES, false, ST><<<grid, DIRECT_THREADS, 0, st>>>(
-            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, sample_list);
+            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, sample_list, nullptr,
+            h->gate, h->gate_want);
 }
 
 template <typename ST>
@@ -461,10 +466,10 @@ int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* ind
     const int64_t blocks = (n + 255) / 256;
     if (h->Wh)
         k_finalize<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, indptr, indices, n, keys,
-                                                             bmu, dist, sample_list);
+                                                             bmu, dist, sample_list, nullptr, h->gate, h->gate_want);
     else
         k_finalize<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, keys,
-                                                            bmu, dist, sample_list);
+                                                            bmu, dist, sample_list, nullptr, h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -366,10 +366,13 @@ template <typename L, int THREADS, int KEEP>
 __global__ void __launch_bounds__(THREADS, 1)
 k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
-            const uint4* __restrict__ slots, const uint32_t* __restrict__ overflow, int64_t n_pad,
+            const uint4* __restrict__ slots, const int32_t* __restrict__ indptr,
+            const int32_t* __restrict__ indices, const int32_t* __restrict__ feat_slot, int V, int64_t n_pad,
             u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
-            int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter)
+            int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter,
+            const int* __restrict__ gate, int gate_want)
 {
+    if (som_gated_off(gate, gate_want)) return;
     constexpr bool TOP2 = KEEP >= 2;
     constexpr int R = L::R;
     constexpr int T = L::T;
@@ -539,7 +542,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     case 2: SOM_HOT(hi16(s0.z));
                     default: break;
                 }
-                const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7 / overflow fields
+                const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
 
                 // ---- tail rows ------------------------------------------------------------------
                 if (p0) L::sub(acc, tr0);
@@ -553,15 +556,20 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         if (nt > 6) L::sub(acc, SOM_TAIL(lo16(t67)));
                         if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
                     } else {
-                        // rare: a sample that does not fit its slot keeps 32-bit lists in the
-                        // overflow buffer (w10 = offset, w11 = hot count | tail count << 16).
-                        // Its inline tail codes are feature 0 four times; start over from base.
+                        // rare: a sample that does not fit its slot (more than 12 hot or 8 tail
+                        // features).  Its inline codes are the zero row and feature 0; start
+                        // over from base and walk its row of the batch, ascending, looking each
+                        // feature up in the feature -> table slot map (mask features are in base).
                         acc = base;
-                        const uint32_t* ol = overflow + t45;
-                        const uint32_t onh = lo16(t67), ont = hi16(t67);
-                        const uint32_t nt_pad = (ont + 3u) & ~3u;
-                        for (uint32_t j = 0; j < ont; ++j) L::sub(acc, SOM_TAIL(__ldg(ol + j)));
-                        for (uint32_t j = 0; j < onh; ++j) SOM_HOT(__ldg(ol + nt_pad + j));
+                        const uint32_t sidx = s0.y;
+                        const int jb = __ldg(indptr + sidx), je = __ldg(indptr + sidx + 1);
+                        for (int j = jb; j < je; ++j) {
+                            const int v = __ldg(indices + j);
+                            if ((unsigned)v >= (unsigned)V) continue;
+                            const int fs = __ldg(feat_slot + v);
+                            if (fs < 0) L::sub(acc, SOM_TAIL((uint32_t)v));
+                            else if (fs >= SOM_PLAN_MASK_FEATURES) SOM_HOT(fs);
+                        }
                     }
                 }
 
@@ -632,12 +640,13 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 }
 
 template <typename ST>
-__global__ void k_finalize_sorted(const ST* __restrict__ W, const double* __restrict__ norm64, int64_t M,
+__global__ void k_finalize_sorted(const ST* __restrict__ W, const double* __restrict__ norm64, int64_t M, int V,
                                   const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                                   int64_t n, const uint4* __restrict__ slots,
                                   const u64* __restrict__ keys, int32_t* __restrict__ bmu,
-                                  float* __restrict__ dist)
+                                  float* __restrict__ dist, const int* __restrict__ gate, int gate_want)
 {
+    if (som_gated_off(gate, gate_want)) return;
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= n) return;
     const uint32_t s = slots[k * SLOT_Q].y;
@@ -650,14 +659,18 @@ __global__ void k_finalize_sorted(const ST* __restrict__ W, const double* __rest
     const int beg = indptr[s];
     const int end = indptr[s + 1];
     double dot = 0.0;
-    for (int j = beg; j < end; ++j) dot += (double)som_weight(W + (int64_t)indices[j] * M + idx);
+    for (int j = beg; j < end; ++j) {
+        const int v = indices[j];
+        if ((unsigned)v < (unsigned)V) dot += (double)som_weight(W + (int64_t)v * M + idx);  // (the plan skipped the others)
+    }
     bmu[s] = (int32_t)idx;
     dist[s] = (float)((double)(end - beg) - 2.0 * dot + norm64[idx]);
 }
 
 template <typename L, int THREADS, int KEEP>
-int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* head, char* ws,
-                 const SomPlanBuffers& b, int n_hot, size_t smem, cudaStream_t st)
+int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, const int32_t* indices,
+                 int64_t n_real, char* head, char* ws, const SomPlanBuffers& b, int n_hot, size_t smem,
+                 cudaStream_t st)
 {
     constexpr int T = L::T;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
@@ -683,12 +696,12 @@ int launch_table(som_handle* h, const void* codebook_v, int64_t n_real, char* he
                                       reinterpret_cast<const int32_t*>(head + b.slot_feat),
                                       SOM_PLAN_MASK_FEATURES + n_hot,
                                       reinterpret_cast<const uint4*>(ws + b.slots),
-                                      reinterpret_cast<const uint32_t*>(ws + b.overflow), n,
+                                      indptr, indices, reinterpret_cast<const int32_t*>(head + b.feat_slot), h->V, n,
                                       reinterpret_cast<u64*>(ws + b.keys),
                                       KEEP >= 2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr,
                                       KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
                                       n_units, n_whole,
-                                      reinterpret_cast<int*>(head + b.n_slots) + 3);
+                                      reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;
@@ -725,13 +738,13 @@ SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
 }
 
 template <int KEEP>
-static int launch_table_any(som_handle* h, bool shadow, int64_t n, char* head, char* ws,
-                            const SomPlanBuffers& b, int n_hot, cudaStream_t st)
+static int launch_table_any(som_handle* h, bool shadow, const int32_t* indptr, const int32_t* indices, int64_t n,
+                            char* head, char* ws, const SomPlanBuffers& b, int n_hot, cudaStream_t st)
 {
     const SomTableGeom g = som_table_geometry(h, shadow);
     const bool f16 = h->Wh != nullptr || shadow;
     const void* cb = shadow ? (const void*)h->shadow : (h->Wh ? (const void*)h->Wh : (const void*)h->W);
-#define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, KEEP>(h, cb, n, head, ws, b, n_hot, g.smem, st)
+#define SOM_TABLE(L_, THREADS_) return launch_table<L_, THREADS_, KEEP>(h, cb, indptr, indices, n, head, ws, b, n_hot, g.smem, st)
     if (f16 && g.R == 16) {
         if (KEEP < 3 && g.threads == 768) SOM_TABLE(LayF16W, 768);
         if (KEEP < 3 && g.threads == 640) SOM_TABLE(LayF16W, 640);
@@ -762,12 +775,12 @@ static int launch_table_any(som_handle* h, bool shadow, int64_t n, char* head, c
 #undef SOM_TABLE
 }
 
-int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
-                         int n_hot, int keep, cudaStream_t st)
+int som_launch_bmu_table(som_handle* h, bool shadow, const int32_t* indptr, const int32_t* indices, int64_t n,
+                         char* head, char* ws, const SomPlanBuffers& b, int n_hot, int keep, cudaStream_t st)
 {
-    if (keep == 3) return launch_table_any<3>(h, shadow, n, head, ws, b, n_hot, st);
-    return keep == 2 ? launch_table_any<2>(h, shadow, n, head, ws, b, n_hot, st)
-                     : launch_table_any<1>(h, shadow, n, head, ws, b, n_hot, st);
+    if (keep == 3) return launch_table_any<3>(h, shadow, indptr, indices, n, head, ws, b, n_hot, st);
+    return keep == 2 ? launch_table_any<2>(h, shadow, indptr, indices, n, head, ws, b, n_hot, st)
+                     : launch_table_any<1>(h, shadow, indptr, indices, n, head, ws, b, n_hot, st);
 }
 
 // ---- two-stage search: certification of the first pass ----------------------------------------
@@ -797,7 +810,7 @@ __device__ __forceinline__ float score_of_key(u64 key)
 // COUNT_ONLY: the probe of the two-stage search; nothing is finalised or listed, the samples that fail the
 // certificate are only counted.
 template <bool SECOND, bool COUNT_ONLY>
-__global__ void k_certify(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M,
+__global__ void k_certify(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M, int V,
                           const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
                           const uint4* __restrict__ slots, const u64* __restrict__ keys,
                           const u64* __restrict__ keys2, const u64* __restrict__ keys3,
@@ -858,7 +871,9 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
             const uint32_t idx2 = (uint32_t)(k2 & 0xffffffffull);
             double dot = 0.0, dot2 = 0.0;
             for (int j = beg; j < end; ++j) {
-                const float* row = W + (int64_t)indices[j] * M;
+                const int v = indices[j];
+                if ((unsigned)v >= (unsigned)V) continue;  // (the plan skipped it too)
+                const float* row = W + (int64_t)v * M;
                 dot += (double)__ldg(row + idx);
                 if (SECOND) dot2 += (double)__ldg(row + idx2);
             }
@@ -906,7 +921,7 @@ int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indi
     const u64* keys3 = second ? reinterpret_cast<const u64*>(ws + b.keys3) : nullptr;
     uint4* slots2 = reinterpret_cast<uint4*>(ws + b.slots2);
 #define SOM_CERTIFY(SECOND_, COUNT_)                                                                            \
-    k_certify<SECOND_, COUNT_><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, slots, \
+    k_certify<SECOND_, COUNT_><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, h->V, indptr, indices, n, slots, \
                                                                  keys, keys2, keys3, h->wmax_bits, h->hnorm, bmu,  \
                                                                  dist, bmu2, dist2, uncertain, slots2, n_uncertain)
     if (second && count_only) SOM_CERTIFY(true, true);
@@ -952,11 +967,11 @@ int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32
     const uint4* slots = reinterpret_cast<const uint4*>(ws + b.slots);
     const u64* keys = reinterpret_cast<const u64*>(ws + (second ? b.keys2 : b.keys));
     if (h->Wh)
-        k_finalize_sorted<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, indptr, indices, n,
-                                                                    slots, keys, bmu, dist);
+        k_finalize_sorted<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, h->V, indptr, indices, n,
+                                                                    slots, keys, bmu, dist, h->gate, h->gate_want);
     else
-        k_finalize_sorted<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n,
-                                                                   slots, keys, bmu, dist);
+        k_finalize_sorted<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, h->V, indptr, indices, n,
+                                                                   slots, keys, bmu, dist, h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

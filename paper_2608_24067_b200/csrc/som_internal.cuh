@@ -11,6 +11,10 @@
 #define SOM_EV_RING 32
 #define SOM_N_EVENTS (SOM_EV_PER_CALL * SOM_EV_RING)
 
+// bits of som_handle::dev_flags
+#define SOM_FLAG_BAD_INDEX 1 /* a feature id outside [0, V) was skipped */
+#define SOM_FLAG_BAD_UNIT 2  /* a best-unit index outside [0, M) was skipped */
+
 #define SOM_AUX_HAS_NEGATIVE 1
 #define SOM_AUX_HMAX 2
 
@@ -63,6 +67,11 @@ struct som_handle {
     int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)
     int64_t opt_two_stage;  // 0 = off, 1 = on where it applies (fp32 storage, M % 128 == 0, memory for the shadow)
     int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 60)
+    // Kernel choice made on the device (automatic mode): the launchers hand `gate` / `gate_want` to the
+    // kernels of both search paths, and a kernel returns at once unless *gate == gate_want.
+    const int* gate;       // device, nullptr = no gate
+    int gate_want;
+    int* dev_flags;        // device, sticky: SOM_FLAG_* bits set by kernels that skipped a bad entry
     int32_t* host_pair;    // pinned, 4 ints: read-back of indptr[0], indptr[n], covered instances, uncertain samples
 };
 
@@ -119,3 +128,15 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
                       int64_t n, const int32_t* bmu, int radius, int planes_per_slab, const int32_t* hot_slot,
                       const int32_t* slot_feat, int n_hot_slots, cudaStream_t st, cudaStream_t aux,
                       cudaEvent_t ev_join);
+
+// true when this launch belongs to the search path that the plan's selection did not choose
+__device__ __forceinline__ bool som_gated_off(const int* gate, int want)
+{
+    return gate != nullptr && *reinterpret_cast<const volatile int*>(gate) != want;
+}
+
+// records a skipped entry in the handle's flag word (one atomic per warp that saw any)
+__device__ __forceinline__ void som_raise(int* flags, bool bad, int bit)
+{
+    if (__any_sync(__activemask(), bad) && bad) atomicOr(flags, bit);
+}

@@ -1,4 +1,4 @@
-// Per-batch plan of the row-table BMU kernel: the "merged feature lists" of a sample tile
+// Per-batch plan of the row-table BMU kernel: the merged feature lists of a sample tile
 // (Section 3.3), pushed from one tile to the whole batch.
 //
 //   1. feature histogram of the batch                      (k_feat_hist)
@@ -9,11 +9,12 @@
 //   4. exclusive scan of the bins                           (k_scan_*)
 //   5. scatter every sample to its sorted position and write its fixed-size slot there:
 //      hot features as byte offsets of their table row, tail features as feature ids
-//      (k_scatter_slots); the rare sample that does not fit a slot gets an overflow list.
+//      (k_scatter_slots); the rare sample that does not fit a slot is marked, and the search
+//      kernel reads its row of the batch itself.
 //
 // Samples that share a mask end up adjacent, so the search kernel keeps
-// ||w||^2/2 - sum(mask rows) in registers across them ("clustering the corpus so that a
-// tile's feature union shrinks", Section 7 of the paper, taken to the register level).
+// ||w||^2/2 - sum(mask rows) in registers across them (the corpus-clustering lever of
+// Section 7 of the paper, which shrinks a tile's feature union, taken to the register level).
 // Nothing here depends on the neuron range, so the plan is built once per batch.
 #include "som_internal.cuh"
 #include "som_plan.cuh"
@@ -54,25 +55,35 @@ __device__ int block_excl_scan_1024(int v, int* warp_sums, int* total)
 // ---- 1. feature histogram --------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 k_feat_hist(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n, int V,
-            int use_smem, uint32_t* __restrict__ feat_count)
+            int use_smem, uint32_t* __restrict__ feat_count, int* __restrict__ flags)
 {
+    // a feature id outside [0, V) is skipped here and in the later plan kernels, and noted in the
+    // handle's flag word (the search itself keeps sorted, distinct, in-range ids as a precondition)
+    bool bad = false;
     extern __shared__ uint32_t sh_hist[];
     const int64_t beg = indptr[0], end = indptr[n];
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     if (use_smem) {
         for (int v = threadIdx.x; v < V; v += blockDim.x) sh_hist[v] = 0;
         __syncthreads();
-        for (int64_t p = beg + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < end; p += stride)
-            atomicAdd(&sh_hist[indices[p]], 1u);
+        for (int64_t p = beg + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < end; p += stride) {
+            const int v = indices[p];
+            if ((unsigned)v < (unsigned)V) atomicAdd(&sh_hist[v], 1u);
+            else bad = true;
+        }
         __syncthreads();
         for (int v = threadIdx.x; v < V; v += blockDim.x) {
             const uint32_t c = sh_hist[v];
             if (c) atomicAdd(&feat_count[v], c);
         }
     } else {
-        for (int64_t p = beg + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < end; p += stride)
-            atomicAdd(&feat_count[indices[p]], 1u);
+        for (int64_t p = beg + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < end; p += stride) {
+            const int v = indices[p];
+            if ((unsigned)v < (unsigned)V) atomicAdd(&feat_count[v], 1u);
+            else bad = true;
+        }
     }
+    if (bad) atomicOr(flags, SOM_FLAG_BAD_INDEX);
 }
 
 // Adds 1 to bins[bin] with one atomic per distinct bin in the warp; returns this thread's
@@ -137,7 +148,8 @@ __device__ void kth_largest(const uint32_t* __restrict__ c, int V, int K, uint32
 
 __global__ void __launch_bounds__(1024)
 k_select_hot(const uint32_t* __restrict__ feat_count_g, int V, int n_mask, int n_hot, int use_smem,
-             int32_t* __restrict__ feat_slot, int32_t* __restrict__ slot_feat, int32_t* __restrict__ n_slots)
+             int32_t* __restrict__ feat_slot, int32_t* __restrict__ slot_feat, int32_t* __restrict__ n_slots,
+             const int32_t* __restrict__ indptr, int64_t n, int cover_pct)
 {
     // the counts are walked thirteen times: keep them in shared memory when they fit
     extern __shared__ uint32_t sh_counts[];
@@ -211,7 +223,16 @@ k_select_hot(const uint32_t* __restrict__ feat_count_g, int V, int n_mask, int n
         const bool used = (s < n_mask) ? (s < mask_assigned) : (s - n_mask < hot_assigned);
         if (!used) slot_feat[s] = -1;
     }
-    if (threadIdx.x == 0) { n_slots[0] = mask_assigned; n_slots[1] = hot_assigned; }
+    // The kernel choice of the automatic mode, made here so that the host never waits for it: the row
+    // table pays when its features serve at least cover_pct percent of the batch's feature instances.
+    __syncthreads();  // every thread's share of the covered count has been added
+    if (threadIdx.x == 0) {
+        n_slots[0] = mask_assigned;
+        n_slots[1] = hot_assigned;
+        const int64_t nnz = (int64_t)indptr[n] - (int64_t)indptr[0];
+        const int64_t cov = *reinterpret_cast<volatile int32_t*>(&n_slots[SOM_PLAN_COVERED]);
+        n_slots[SOM_PLAN_USE_TABLE] = (cov * 100 >= (int64_t)cover_pct * nnz) ? 1 : 0;
+    }
 }
 
 // ---- 3. classify ----------------------------------------------------------------------------
@@ -225,17 +246,21 @@ __device__ __forceinline__ uint32_t sort_bin(uint32_t mask, uint32_t n_hot, uint
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS)
-k_classify(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
+k_classify(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n, int V,
            const int32_t* __restrict__ feat_slot, int n_mask, uint32_t* __restrict__ pk,
-           uint32_t* __restrict__ ntail, uint32_t* __restrict__ bin_count)
+           uint32_t* __restrict__ ntail, uint32_t* __restrict__ bin_count, const int* __restrict__ gate,
+           int gate_want)
 {
+    if (som_gated_off(gate, gate_want)) return;
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool active = s < n;
     uint32_t mask = 0, nh = 0, nt = 0;
     if (active) {
         const int beg = indptr[s], end = indptr[s + 1];
         for (int j = beg; j < end; ++j) {
-            const int slot = feat_slot[indices[j]];
+            const int v = indices[j];
+            if ((unsigned)v >= (unsigned)V) continue;  // skipped (k_feat_hist has noted it)
+            const int slot = feat_slot[v];
             if (slot < 0) ++nt;
             else if (slot < n_mask) mask |= 1u << slot;
             else ++nh;
@@ -308,13 +333,13 @@ k_scan_apply(const uint32_t* __restrict__ in, int n, const uint32_t* __restrict_
 
 // ---- 5. scatter + slots ----------------------------------------------------------------------
 __global__ void __launch_bounds__(PLAN_THREADS)
-k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
+k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n, int V,
                 const int32_t* __restrict__ feat_slot, int n_mask, int zero_row,
                 const uint32_t* __restrict__ pk, const uint32_t* __restrict__ ntail,
                 uint32_t* __restrict__ bin_cursor /* starts as bin_start */,
-                uint32_t* __restrict__ slots, uint32_t* __restrict__ overflow,
-                uint32_t* __restrict__ overflow_cursor)
+                uint32_t* __restrict__ slots, const int* __restrict__ gate, int gate_want)
 {
+    if (som_gated_off(gate, gate_want)) return;
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool active = s < n;
     uint32_t mask = 0, nh = 0, nt = 0, p = 0;
@@ -327,12 +352,11 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
     const uint32_t pos = warp_agg_inc(bin_cursor, sort_bin(mask, nh, nt), active);
     if (!active) return;
     const bool fits = nh <= SOM_SLOT_MAX_HOT && nt <= SOM_SLOT_MAX_TAIL;
-    // (an overflow list holds at most 65535 hot and 65535 tail entries; the launcher checks V)
     // The slot is assembled in registers and written with three 128-bit stores.  Unused hot
     // codes point at the all-zero row that follows the table; unused tail codes are feature 0.
     const uint32_t zz = (uint32_t)zero_row | ((uint32_t)zero_row << 16);
     uint32_t w[SOM_SLOT_WORDS];
-    w[0] = fits ? (mask | (nh << 16) | (nt << 24)) : (mask | (SOM_SLOT_NT_OVERFLOW << 24));
+    w[0] = fits ? (mask | (nh << 16) | (nt << 24)) : (mask | (SOM_SLOT_NT_OVERFLOW << 24));  // (zero hot codes)
     w[1] = (uint32_t)s;
 #pragma unroll
     for (int i = 2; i < 8; ++i) w[i] = zz;
@@ -343,6 +367,7 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
         uint32_t ih = 0, it = 0;
         for (int j = beg; j < end; ++j) {
             const int v = indices[j];
+            if ((unsigned)v >= (unsigned)V) continue;
             const int fs = feat_slot[v];
             if (fs < 0) {
 #pragma unroll
@@ -359,22 +384,8 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
                 ++ih;
             }
         }
-    } else {
-        const uint32_t nt_pad = (nt + 3u) & ~3u, nh_pad = (nh + 3u) & ~3u;
-        const uint32_t off = atomicAdd(overflow_cursor, nt_pad + nh_pad);
-        // the list offset and the true counts (which may not fit the header fields) go where
-        // the last tail codes would be; the inline tail codes stay feature 0, a valid row
-        w[10] = off;
-        w[11] = nh | (nt << 16);
-        uint32_t* tail = overflow + off;
-        uint32_t* hot = tail + nt_pad;
-        for (int j = beg; j < end; ++j) {
-            const int v = indices[j];
-            const int fs = feat_slot[v];
-            if (fs < 0) *tail++ = (uint32_t)v;
-            else if (fs >= n_mask) *hot++ = (uint32_t)fs;
-        }
     }
+    // (a sample that does not fit keeps no list: the search kernel reads its row of the batch itself)
     uint4* slot = reinterpret_cast<uint4*>(slots + (size_t)pos * SOM_SLOT_WORDS);
     slot[0] = make_uint4(w[0], w[1], w[2], w[3]);
     slot[1] = make_uint4(w[4], w[5], w[6], w[7]);
@@ -408,7 +419,7 @@ size_t som_plan_head_bytes(int32_t V, int n_slots_max, SomPlanBuffers* b)
     return off;
 }
 
-size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b)
+size_t som_plan_workspace_bytes(int64_t n, SomPlanBuffers* b)
 {
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -425,7 +436,6 @@ size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b)
     b->bin_start = take((size_t)SOM_PLAN_BINS * 4);
     b->block_sums = take((size_t)(SOM_PLAN_BINS / SCAN_BLOCK + 2) * 4);
     b->slots = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
-    b->overflow = take((size_t)(nnz + 6 * n + 4) * 4);
     b->uncertain = take((size_t)n * 4);
     b->ukeys = take((size_t)(n + 16) * 8);
     b->ukeys2 = take((size_t)(n + 16) * 8);
@@ -468,7 +478,7 @@ int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* 
         } else {
             blocks = h->sm_count * 2;
         }
-        k_feat_hist<<<blocks, 1024, use_smem ? sh : 0, st>>>(indptr, indices, n, h->V, use_smem, feat_count);
+        k_feat_hist<<<blocks, 1024, use_smem ? sh : 0, st>>>(indptr, indices, n, h->V, use_smem, feat_count, h->dev_flags);
         SOM_CK(h, cudaGetLastError());
     }
     // 2. select
@@ -477,7 +487,8 @@ int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* 
     if (counts_fit)
         SOM_CK(h, cudaFuncSetAttribute(k_select_hot, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)counts_sh));
     k_select_hot<<<1, 1024, counts_fit ? counts_sh : 0, st>>>(feat_count, h->V, n_mask, n_hot, counts_fit, feat_slot,
-                                                             slot_feat, n_slots);
+                                                             slot_feat, n_slots, indptr, n,
+                                                             (int)(h->opt_cover > 0 ? h->opt_cover : 60));
     SOM_CK(h, cudaGetLastError());
     h->launches += 2;
     return SOM_OK;
@@ -488,18 +499,17 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
                          cudaStream_t st)
 {
     int32_t* feat_slot = reinterpret_cast<int32_t*>(head + b.feat_slot);
-    int32_t* n_slots = reinterpret_cast<int32_t*>(head + b.n_slots);
     uint32_t* pk = reinterpret_cast<uint32_t*>(ws + b.pk);
     uint32_t* ntail = reinterpret_cast<uint32_t*>(ws + b.ntail);
     uint32_t* bin_count = reinterpret_cast<uint32_t*>(ws + b.bin_count);
     uint32_t* bin_start = reinterpret_cast<uint32_t*>(ws + b.bin_start);
     uint32_t* slots = reinterpret_cast<uint32_t*>(ws + b.slots);
-    uint32_t* overflow = reinterpret_cast<uint32_t*>(ws + b.overflow);
 
     SOM_CK(h, cudaMemsetAsync(bin_count, 0, (size_t)SOM_PLAN_BINS * 4, st));
     // 3. classify
     const unsigned sblocks = (unsigned)((n + PLAN_THREADS - 1) / PLAN_THREADS);
-    k_classify<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, feat_slot, n_mask, pk, ntail, bin_count);
+    k_classify<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, h->V, feat_slot, n_mask, pk, ntail, bin_count,
+                                                 h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());
     // 4. scan bins
     {
@@ -513,9 +523,8 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
         SOM_CK(h, cudaGetLastError());
     }
     // 5. scatter + slots (bin_start doubles as the running cursor)
-    k_scatter_slots<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, feat_slot, n_mask, n_mask + n_hot, pk, ntail,
-                                                      bin_start, slots, overflow,
-                                                      reinterpret_cast<uint32_t*>(n_slots) + 2);
+    k_scatter_slots<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, h->V, feat_slot, n_mask, n_mask + n_hot, pk, ntail,
+                                                      bin_start, slots, h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());
     const int64_t n_pad = (n + 3) / 4 * 4;
     if (n_pad > n) {

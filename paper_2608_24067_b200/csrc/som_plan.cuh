@@ -15,16 +15,15 @@ struct som_handle;
 // One 48-byte slot per sample, at a fixed address for its sorted position k (slots[k]), so
 // that the search kernel can load it one round ahead without chasing an offset.  As 12 words:
 //   w0        mask of mask features (bits 0-15) | hot codes (16-23) | tail codes (24-31);
-//             a tail count of SOM_SLOT_NT_OVERFLOW marks a sample kept in the overflow buffer
+//             a tail count of SOM_SLOT_NT_OVERFLOW marks a sample that does not fit a slot
 //   w1        sample index
 //   w2..w7    hot codes 0..11, 16 bits each: row of the feature in the shared-memory table;
 //             unused ones hold the index of the all-zero row that follows the table
 //   w8..w11   tail codes 0..7, 16 bits each: feature id
-//             (overflow sample: w8 = w9 = 0, w10 = offset of its lists in the overflow
-//             buffer, w11 = hot count | tail count << 16)
-// A sample fits when it has at most 12 hot and 8 tail features; the rare others keep 32-bit
-// lists in the overflow buffer: tail ids padded to a multiple of 4, then hot rows likewise
-// (at most 65535 of each).  16-bit codes require V <= 65536 and at most 65536 table rows.
+// A sample fits when it has at most 12 hot and 8 tail features; for the rare others the slot
+// holds only the mask and the sample index (hot codes all zero-row, tail codes feature 0), and
+// the search kernel walks the sample's row of the batch itself, looking each feature up in the
+// feature -> table slot map.  16-bit codes require V <= 65536 and at most 65536 table rows.
 // The slot array is padded to a multiple of 4 samples with copies of the last slot, so the
 // search kernel always runs whole rounds; the duplicates redo the same idempotent atomicMin.
 #define SOM_SLOT_WORDS 12
@@ -32,16 +31,17 @@ struct som_handle;
 #define SOM_SLOT_MAX_TAIL 8
 #define SOM_SLOT_NT_OVERFLOW 255u
 
-// Byte offsets of the plan's arrays.  The first four live in the small "head" buffer, which
-// the selection phase fills before the batch's nnz is known on the host; the others live in
-// the handle's workspace, sized from nnz.
+// Byte offsets of the plan's arrays.  The first four live in the small "head" buffer, sized by V;
+// the others live in the handle's workspace, sized by the number of samples alone (the host never
+// needs the batch's nnz, which lives on the device).
 struct SomPlanBuffers {
     // head buffer
     size_t feat_count;  // u32 [V]
     size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
     size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
-    size_t n_slots;     // i32 [8]      mask slots used, hot slots used, overflow cursor, search unit
-                        //              counter, feature instances covered by the table, uncertain samples
+    size_t n_slots;     // i32 [8]      mask slots used, hot slots used, (unused), search unit counter,
+                        //              feature instances covered by the table, uncertain samples,
+                        //              1 if the automatic mode takes the row-table kernel for this batch
     // workspace
     size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
     size_t keys2;       // u64 [n]      the same for the second-best unit (two-best search only)
@@ -52,7 +52,6 @@ struct SomPlanBuffers {
     size_t bin_start;   // u32 [bins]
     size_t block_sums;  // u32 [scan blocks]
     size_t slots;       // 48 B [n + 16]
-    size_t overflow;    // u32 [nnz + 6n]
     size_t uncertain;   // i32 [n]      samples the two-stage search sends to its exact pass
     size_t ukeys;       // u64 [n + 16] their packed keys, by position in that list
     size_t ukeys2;      // u64 [n + 16] and their second-best keys (two-best search)
@@ -61,6 +60,7 @@ struct SomPlanBuffers {
 #define SOM_PLAN_N_SLOTS_INTS 8
 #define SOM_PLAN_COVERED 4 /* index into n_slots */
 #define SOM_PLAN_UNCERTAIN 5 /* index into n_slots: length of the two-stage search's uncertain list */
+#define SOM_PLAN_USE_TABLE 6 /* index into n_slots: the selection kernel's choice of search kernel */
 
 // Sample parts per neuron range of the row-table kernel.  More parts mean fewer ranges live at
 // once (their slabs must share L2 with the slot stream) but smaller units, each of which
@@ -76,7 +76,7 @@ static inline int som_table_default_parts(int64_t n, int range_neurons)
 }
 
 size_t som_plan_head_bytes(int32_t V, int n_slots_max, SomPlanBuffers* b);
-size_t som_plan_workspace_bytes(int64_t n, int64_t nnz, SomPlanBuffers* b);
+size_t som_plan_workspace_bytes(int64_t n, SomPlanBuffers* b);
 
 // Phase 1 (needs no workspace): feature histogram and choice of the mask and hot features;
 // leaves the number of feature instances they cover in n_slots[SOM_PLAN_COVERED].
@@ -89,8 +89,9 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
 
 // shadow = read the handle's fp16 shadow of an fp32 codebook (first pass of the two-stage search);
 // keep = how many best units per sample are kept (1, 2; 3 with the shadow's wide layout only)
-int som_launch_bmu_table(som_handle* h, bool shadow, int64_t n, char* head, char* ws, const SomPlanBuffers& b,
-                         int n_hot, int keep, cudaStream_t st);
+// indptr / indices: the batch (rows of samples that do not fit a slot are read from it)
+int som_launch_bmu_table(som_handle* h, bool shadow, const int32_t* indptr, const int32_t* indices, int64_t n,
+                         char* head, char* ws, const SomPlanBuffers& b, int n_hot, int keep, cudaStream_t st);
 
 // pads a slot array of n slots to a multiple of four with copies of the last one
 int som_launch_pad_slots(som_handle* h, char* ws, size_t slots_offset, int64_t n, cudaStream_t st);

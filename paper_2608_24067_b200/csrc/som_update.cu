@@ -31,8 +31,10 @@ constexpr int UPD_THREADS = 256;
 // Count of samples per cell into den_t (TRANSPOSED cell order) and the occupancy flags.  Small
 // lattices take a per-block histogram in shared memory first (a million samples on a few
 // thousand cells would otherwise queue on a handful of L2 atomic units); counts are exact in fp32.
+// A best-unit index outside [0, M) (a stale buffer, the -1 of a missing second unit) is skipped and
+// noted in the handle's flag word, here and in the scatters below.
 __global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows, int cols, int use_smem,
-                            float* __restrict__ den_t, int32_t* __restrict__ occ)
+                            float* __restrict__ den_t, int32_t* __restrict__ occ, int* __restrict__ flags)
 {
     extern __shared__ unsigned int hist[];
     const int M = rows * cols;
@@ -40,8 +42,13 @@ __global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows
     if (use_smem) {
         for (int c = threadIdx.x; c < M; c += blockDim.x) hist[c] = 0u;
         __syncthreads();
-        for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < n; s += stride)
-            atomicAdd(&hist[bmu[s]], 1u);
+        bool bad = false;
+        for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < n; s += stride) {
+            const int c = bmu[s];
+            if ((unsigned)c < (unsigned)M) atomicAdd(&hist[c], 1u);
+            else bad = true;
+        }
+        if (bad) atomicOr(flags, SOM_FLAG_BAD_UNIT);
         __syncthreads();
         for (int c = threadIdx.x; c < M; c += blockDim.x) {
             const unsigned int k = hist[c];
@@ -54,6 +61,10 @@ __global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows
     } else {
         for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < n; s += stride) {
             const int c = bmu[s];
+            if ((unsigned)c >= (unsigned)M) {
+                atomicOr(flags, SOM_FLAG_BAD_UNIT);
+                continue;
+            }
             const int r = c / cols, q = c - r * cols;
             atomicAdd(&den_t[(int64_t)q * rows + r], 1.0f);
             occ[c] = 1;
@@ -69,9 +80,10 @@ __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t*
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n) return;
     const int c = bmu[s];
+    const int64_t M = (int64_t)rows * cols;
+    if ((unsigned)c >= (unsigned)M) return;  // skipped; k_upd_count has noted it
     const int r = c / cols, q = c - r * cols;
     const int64_t cell_t = (int64_t)q * rows + r;  // transposed cell order
-    const int64_t M = (int64_t)rows * cols;
     const int beg = indptr[s], end = indptr[s + 1];
     for (int j = beg; j < end; ++j) {
         const int v = indices[j];
@@ -88,14 +100,20 @@ __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t*
 // a sample, and adds each non-zero count to the plane once.  hot_slot[v] = rank of feature v among the
 // hot ones or -1; slot_feat is its inverse.
 __global__ void k_upd_hot_mask(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
-                               const int32_t* __restrict__ hot_slot, uint32_t* __restrict__ mask)
+                               int V, const int32_t* __restrict__ hot_slot, uint32_t* __restrict__ mask,
+                               int* __restrict__ flags)
 {
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n) return;
     uint32_t m = 0;
     const int beg = indptr[s], end = indptr[s + 1];
     for (int j = beg; j < end; ++j) {
-        const int slot = hot_slot[indices[j]];
+        const int v = indices[j];
+        if ((unsigned)v >= (unsigned)V) {  // skipped and noted
+            atomicOr(flags, SOM_FLAG_BAD_INDEX);
+            continue;
+        }
+        const int slot = hot_slot[v];
         if (slot >= 0) m |= 1u << slot;
     }
     mask[s] = m;
@@ -103,7 +121,7 @@ __global__ void k_upd_hot_mask(const int32_t* __restrict__ indptr, const int32_t
 
 __global__ void k_upd_scatter_hot(const uint32_t* __restrict__ mask, int64_t n, const int32_t* __restrict__ bmu,
                                   int v0, int v1, int rows, int cols, const int32_t* __restrict__ slot_feat,
-                                  int planes_per_block, float* __restrict__ num_t)
+                                  int n_slots, int planes_per_block, float* __restrict__ num_t)
 {
     extern __shared__ unsigned int cnt[];
     const int M = rows * cols;
@@ -111,7 +129,7 @@ __global__ void k_upd_scatter_hot(const uint32_t* __restrict__ mask, int64_t n, 
     for (int e = threadIdx.x; e < planes_per_block * M; e += blockDim.x) cnt[e] = 0u;
     // the group's slots whose feature lies in this slab
     uint32_t group = 0;
-    for (int p = 0; p < planes_per_block && slot0 + p < 32; ++p) {
+    for (int p = 0; p < planes_per_block && slot0 + p < n_slots; ++p) {
         const int f = slot_feat[slot0 + p];
         if (f >= v0 && f < v1) group |= 1u << (slot0 + p);
     }
@@ -123,6 +141,7 @@ __global__ void k_upd_scatter_hot(const uint32_t* __restrict__ mask, int64_t n, 
             uint32_t m = mask[s] & group;
             if (!m) continue;
             const int c = bmu[s];
+            if ((unsigned)c >= (unsigned)M) continue;  // skipped; k_upd_count has noted it
             const int r = c / cols, q = c - r * cols;
             const int cell_t = q * rows + r;  // transposed cell order
             while (m) {
@@ -133,7 +152,7 @@ __global__ void k_upd_scatter_hot(const uint32_t* __restrict__ mask, int64_t n, 
         }
     }
     __syncthreads();
-    for (int p = 0; p < planes_per_block; ++p) {
+    for (int p = 0; p < planes_per_block && slot0 + p < n_slots; ++p) {
         if (!((group >> (slot0 + p)) & 1u)) continue;  // unused slot, or a feature of another slab
         float* plane = num_t + (int64_t)(slot_feat[slot0 + p] - v0) * M;
         for (int e = threadIdx.x; e < M; e += blockDim.x) {
@@ -490,9 +509,9 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         const int use_smem = M * 4 <= 96 * 1024;
         if (use_smem) {
             SOM_CK(h, cudaFuncSetAttribute(k_upd_count, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
-            k_upd_count<<<h->sm_count * 2, 1024, (size_t)M * 4, st>>>(bmu, n, rows, cols, 1, den_a, occ_a);
+            k_upd_count<<<h->sm_count * 2, 1024, (size_t)M * 4, st>>>(bmu, n, rows, cols, 1, den_a, occ_a, h->dev_flags);
         } else {
-            k_upd_count<<<h->sm_count * 8, UPD_THREADS, 0, st>>>(bmu, n, rows, cols, 0, den_a, occ_a);
+            k_upd_count<<<h->sm_count * 8, UPD_THREADS, 0, st>>>(bmu, n, rows, cols, 0, den_a, occ_a, h->dev_flags);
         }
         h->launches += 1;
     }
@@ -537,7 +556,7 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
     // (the per-sample masks of the hot features live behind the two slab buffers)
     uint32_t* hot_mask = reinterpret_cast<uint32_t*>(ws + 8 * mb + 2 * som_align_up((size_t)planes_per_slab * M * 4, 256));
     if (hot_slot && n > 0) {
-        k_upd_hot_mask<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, hot_slot, hot_mask);
+        k_upd_hot_mask<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, h->V, hot_slot, hot_mask, h->dev_flags);
         h->launches += 1;
     }
     for (int v0 = 0; v0 < h->V; v0 += planes_per_slab) {
@@ -558,7 +577,7 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
                 const size_t sh = (size_t)ppb * M * 4;
                 SOM_CK(h, cudaFuncSetAttribute(k_upd_scatter_hot, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh));
                 k_upd_scatter_hot<<<dim3(slices, groups), 1024, sh, st>>>(hot_mask, n, bmu, v0, v1, rows, cols, slot_feat,
-                                                                        ppb, slab_a);
+                                                                        n_hot_slots, ppb, slab_a);
                 h->launches += 1;
             }
         }

@@ -26,6 +26,7 @@ EXPORTS = [
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
     "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain", "som_bmu_values",
     "som_bmu_host_async", "som_host_sync", "som_plan_create", "som_bmu_planned", "som_plan_destroy",
+    "som_device_flags", "som_measure_fadd_peak",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -89,6 +90,10 @@ def load_library():
     lib.som_last_uncertain.argtypes = [P]
     lib.som_last_uncertain.restype = I64
     lib.som_set_option.argtypes = [P, INT, I64]
+    lib.som_measure_fadd_peak.argtypes = [ctypes.POINTER(ctypes.c_double), P, I64, P]
+    lib.som_measure_fadd_peak.restype = INT
+    lib.som_device_flags.argtypes = [P, P]
+    lib.som_device_flags.restype = INT
     lib.som_norms_noalloc.argtypes = [I32, I64, P, P, P]
     lib.som_norms_noalloc.restype = INT
     for name in ("som_create", "som_norms", "som_bmu", "som_bmu_host", "som_validate_csr",
@@ -130,6 +135,21 @@ def norms_noalloc(V: int, M: int, codebook: torch.Tensor, out: torch.Tensor, str
     if rc != SOM_OK:
         raise SomError(rc, "som_norms_noalloc")
     return out
+
+
+def measure_fadd_peak(device=None, stream=None) -> float:
+    """som_measure_fadd_peak: the FP32 add rate (adds/s) the current device delivers on independent
+    add chains; the scratch tensor is allocated here, the measurement runs in the library."""
+    lib = load_library()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        scratch = torch.empty(2048 * sms, dtype=torch.float32, device=dev)
+        out = ctypes.c_double(0.0)
+        rc = lib.som_measure_fadd_peak(ctypes.byref(out), scratch.data_ptr(), scratch.numel(), _stream_ptr(stream))
+    if rc != SOM_OK:
+        raise SomError(rc, "som_measure_fadd_peak")
+    return float(out.value)
 
 
 class Plan:
@@ -286,6 +306,11 @@ class Som:
             return False
         self._check(rc, "som_validate_csr")
         return True
+
+    def device_flags(self, stream=None) -> int:
+        """som_device_flags: status of what earlier calls skipped on the device (0 = nothing);
+        synchronises the stream and clears the record."""
+        return int(self._lib.som_device_flags(self._h, _stream_ptr(stream)))
 
     def get_norms(self, stream=None) -> torch.Tensor:
         out = torch.empty(self.M, dtype=torch.float32, device=self.codebook.device)

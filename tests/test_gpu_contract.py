@@ -1,0 +1,145 @@
+"""GPU tests of what the header promises beyond parity on one batch: som_bmu only enqueues work,
+bad indices are skipped and reported instead of faulting, and a sample's best unit does not depend
+on the batch it arrives in except inside the near-tie band (Section 3.1 of the paper: the summation
+order flips only near-tied assignments)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import parity
+from oracle import som_oracle as orc
+from paper_2608_24067_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def som_mod():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_24067_b200 import som
+    som.load_library()
+    return som
+
+
+@pytest.mark.parametrize("variant", [0, 2])
+def test_som_bmu_returns_before_the_search_has_run(som_mod, variant):
+    """The call only enqueues: an event recorded right after it returns is not yet reached (the
+    search of a million samples over 16 384 neurons takes about 20 ms), and the results are those
+    of a call that was waited for."""
+    V, M, n = 30_000, 16_384, 1_000_000
+    W = synth.fill_codebook(V, M, 0, device="cuda")
+    b = synth.sample_csr(n, V, 11.0, 0, device="cuda")
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, variant)
+    h.norms()
+    ref_bmu, ref_dist = h.bmu(b.indptr, b.indices)  # grows the workspace (may synchronise)
+    torch.cuda.synchronize()
+    out_bmu, out_dist = torch.empty_like(ref_bmu), torch.empty_like(ref_dist)
+    done = torch.cuda.Event()
+    h.bmu(b.indptr, b.indices, out_bmu, out_dist)
+    done.record()
+    pending = not done.query()
+    torch.cuda.synchronize()
+    assert pending, "som_bmu waited for the device"
+    assert torch.equal(out_bmu, ref_bmu) and torch.equal(out_dist.view(torch.int32), ref_dist.view(torch.int32))
+
+
+def test_bad_unit_indices_are_skipped_and_reported(som_mod):
+    """som_update with best-unit indices outside [0, M) (the -1 of a missing second unit, a stale
+    buffer): those samples are left out, nothing faults, and som_device_flags reports it once."""
+    from oracle import som_update_oracle as uorc
+    V, rows, cols, n = 40, 16, 16, 3000
+    M = rows * cols
+    rng = np.random.default_rng(5)
+    W_old = rng.random(V * M).astype(np.float32)
+    b = synth.sample_csr(n, V, 5.0, 2, device="cpu")
+    ip, ix = b.indptr.numpy(), b.indices.numpy()
+    bmu = rng.integers(0, M, size=n).astype(np.int32)
+    bad = bmu.copy()
+    bad[7], bad[100], bad[2999] = -1, M, 2 ** 31 - 1
+    W = torch.from_numpy(W_old).cuda()
+    h = som_mod.Som(V, M, W)
+    assert h.device_flags() == 0
+    h.update(rows, cols, b.indptr.cuda(), b.indices.cuda(), torch.from_numpy(bad).cuda(), 2)
+    assert h.device_flags() == 1  # SOM_ERR_INVALID_ARG
+    assert h.device_flags() == 0  # cleared by the query
+    keep = np.ones(n, bool)
+    keep[[7, 100, 2999]] = False
+    rows_kept = np.nonzero(keep)[0]
+    lens = ip[1:] - ip[:-1]
+    ip2 = np.zeros(rows_kept.size + 1, np.int32)
+    ip2[1:] = np.cumsum(lens[rows_kept])
+    ix2 = np.concatenate([ix[ip[r]:ip[r + 1]] for r in rows_kept]).astype(np.int32)
+    want = uorc.update(W_old, V, rows, cols, ip2, ix2, bmu[rows_kept], 2)
+    np.testing.assert_allclose(W.cpu().numpy().astype(np.float64), want, rtol=1e-6, atol=1e-12)
+
+
+def test_bad_feature_ids_are_skipped_by_the_plan_and_reported(som_mod):
+    """Feature ids outside [0, V) in a batch that goes through the row-table kernel: the plan skips
+    them (the result is that of the batch without them), nothing faults, som_device_flags says
+    SOM_ERR_BAD_CSR."""
+    V, M, n = 3000, 512, 40_000
+    W = synth.fill_codebook(V, M, 9, device="cuda")
+    b = synth.sample_csr(n, V, 9.0, 9, device="cpu")
+    ip, ix = b.indptr.numpy().astype(np.int64), b.indices.numpy().copy()
+    # append one bad id to three rows (rows stay ascending except for the negative one)
+    rows_bad = [5, 1234, n - 1]
+    new_ix, new_ip = [], [0]
+    for r in range(n):
+        row = ix[ip[r]:ip[r + 1]]
+        if r == rows_bad[0]:
+            row = np.concatenate([row, [V]])
+        elif r == rows_bad[1]:
+            row = np.concatenate([row, [V + 70000]])
+        elif r == rows_bad[2]:
+            row = np.concatenate([[-3], row])
+        new_ix.append(row)
+        new_ip.append(new_ip[-1] + len(row))
+    bad_ix = torch.from_numpy(np.concatenate(new_ix).astype(np.int32)).cuda()
+    bad_ip = torch.from_numpy(np.asarray(new_ip, np.int32)).cuda()
+    h = som_mod.Som(V, M, W)
+    h.set_option(0, 2)
+    h.norms()
+    g_bmu, g_dist = h.bmu(bad_ip, bad_ix)
+    assert h.device_flags() == 5  # SOM_ERR_BAD_CSR
+    c_bmu, _ = h.bmu(b.indptr.cuda(), b.indices.cuda())
+    assert h.device_flags() == 0
+    torch.cuda.synchronize()
+    assert torch.equal(g_bmu, c_bmu)
+    assert not h.validate_csr(bad_ip, bad_ix)
+
+
+def test_same_sample_in_different_batches_and_kernels(som_mod):
+    """10 000 samples searched inside two different 100 000-sample batches, and by both kernels:
+    wherever the oracle calls the sample unambiguous, all four answers are the oracle's unit."""
+    V, M = 30_000, 4_096
+    W = synth.fill_codebook(V, M, 0, device="cuda")
+    common = synth.sample_csr(10_000, V, 11.0, 0, device="cpu", first_sample=5_000_000)
+    fill_a = synth.sample_csr(90_000, V, 11.0, 0, device="cpu", first_sample=0)
+    fill_b = synth.sample_csr(90_000, V, 11.0, 0, device="cpu", first_sample=900_000, zipf_s=0.9)
+
+    def join(first, second):
+        ip = torch.cat([first.indptr, second.indptr[1:] + first.indptr[-1]]).to(torch.int32)
+        return ip.cuda(), torch.cat([first.indices, second.indices]).cuda()
+
+    h = som_mod.Som(V, M, W)
+    h.norms()
+    answers = []
+    for variant in (2, 1):
+        h.set_option(0, variant)
+        ip, ix = join(common, fill_a)          # the common samples lead batch A
+        answers.append(h.bmu(ip, ix)[0][:10_000].cpu().numpy())
+        ip, ix = join(fill_b, common)          # and trail batch B, whose table features differ
+        answers.append(h.bmu(ip, ix)[0][90_000:].cpu().numpy())
+    torch.cuda.synchronize()
+    Wh = W.cpu().numpy()
+    cip, cix = common.indptr.numpy(), common.indices.numpy()
+    nn = orc.norms(Wh, V, M)
+    top2 = orc.bmu(Wh, V, M, cip, cix, norms_=nn)
+    unamb = (top2.d2 - top2.d1) > parity.GAP_REL * top2.d1
+    assert unamb.sum() > 9_000
+    for g in answers:
+        assert np.array_equal(g[unamb], top2.b1[unamb])
+        d_at = orc.dist_at(Wh, V, M, cip, cix, g.astype(np.int64), norms_=nn)
+        assert np.all(d_at[~unamb] - top2.d1[~unamb] <= parity.GAP_REL * top2.d1[~unamb])

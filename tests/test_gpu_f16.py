@@ -11,6 +11,8 @@ from oracle import parity
 from oracle import som_oracle as orc
 from paper_2608_24067_b200 import synth
 
+import largemap
+
 pytestmark = pytest.mark.gpu
 
 
@@ -135,64 +137,53 @@ def test_f16_matches_fp32_handle_on_the_same_values(som_mod):
     assert torch.equal(d16[same], d32[same])
 
 
-def _oracle_top2_slabbed(W_dev, V, M, indptr, indices, slab_neurons=16384):
-    """Oracle best/second best over a device-resident fp16 codebook, consumed in neuron slabs
-    (ascending) widened and copied to the host; also returns the oracle's fp64 norms."""
-    W2 = W_dev.view(V, M)
-    run = None
-    norms = np.empty(M, np.float64)
-    for m0 in range(0, M, slab_neurons):
-        m1 = min(M, m0 + slab_neurons)
-        slab = W2[:, m0:m1].float().contiguous().cpu().numpy()
-        nn = orc.norms(slab, V, m1 - m0)
-        norms[m0:m1] = nn
-        run = orc.bmu(slab, V, m1 - m0, indptr, indices, norms_=nn, m_offset=m0, running=run)
-        del slab
-    return run, norms
-
-
-def _dist_at_from_device(W_dev, V, M, indptr, indices, neuron, norms):
-    """fp64 distance of sample s to neuron[s] from gathered weights (Eq. 1, ascending feature order)."""
-    W2 = W_dev.view(V, M)
-    out = np.empty(len(neuron), np.float64)
-    for s in range(len(neuron)):
-        idx = indices[indptr[s]:indptr[s + 1]].astype(np.int64)
-        w = W2[torch.from_numpy(idx).cuda(), int(neuron[s])].double().cpu().numpy()
-        dot = 0.0
-        for x in w:
-            dot += float(x)
-        out[s] = float(len(idx)) - 2.0 * dot + norms[int(neuron[s])]
-    return out
-
-
 def test_f16_largest_map_full_size_sampled_rows(som_mod):
     """1024x1024 map stored in fp16 (62.9 GB, resident in HBM) at the batch size the benchmark
-    uses, through som_bmu2; a strided sample of rows is checked against the oracle, which reads
-    the device codebook slab by slab, and range properties are checked for every row."""
+    uses, through som_bmu2, all four batches: 5 000 rows per batch (first and last among them) are
+    checked against the oracle, which reads the device codebook slab by slab; for every sample both
+    reported distances must be the fp64 distances to the reported neurons within 1e-5 relative."""
     w = synth.CONFIGS[4]
     import gc
     gc.collect()  # handles and tensors of earlier tests
     torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
-    need = w.V * w.M * 2 + (6 << 30)
+    need = w.V * w.M * 2 + (8 << 30)
     if free < need:
         pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
     W16 = torch.empty(w.V * w.M, dtype=torch.float16, device="cuda")
     synth.fill_codebook(w.V, w.M, w.seed, out=W16)
-    b = synth.sample_csr(w.batch, w.V, w.lam, w.seed, device="cuda")
     h = som_mod.Som(w.V, w.M, W16)
     h.norms()
-    g1, gd1, g2, gd2 = [t.cpu().numpy() for t in h.bmu2(b.indptr, b.indices)]
-    assert g1.min() >= 0 and g1.max() < w.M and g2.min() >= 0 and g2.max() < w.M
-    assert np.all(g1 != g2) and np.isfinite(gd1).all() and np.isfinite(gd2).all()
-    rows = np.unique(np.concatenate([np.linspace(0, w.batch - 1, 48).astype(np.int64), [0, w.batch - 1]]))
-    ip, ix = _subset(b.indptr.cpu().numpy(), b.indices.cpu().numpy(), rows)
-    top2, norms = _oracle_top2_slabbed(W16, w.V, w.M, ip, ix)
-    rep1 = parity.check(g1[rows], gd1[rows], top2, _dist_at_from_device(W16, w.V, w.M, ip, ix, g1[rows], norms), w.M)
+    subs, full = [], []
+    for bi in range(w.N // w.batch):
+        b = synth.sample_csr(w.batch, w.V, w.lam, w.seed, device="cuda", first_sample=bi * w.batch)
+        g1, gd1, g2, gd2 = [t.cpu().numpy() for t in h.bmu2(b.indptr, b.indices)]
+        assert g1.min() >= 0 and g1.max() < w.M and g2.min() >= 0 and g2.max() < w.M
+        assert np.all(g1 != g2) and np.isfinite(gd1).all() and np.isfinite(gd2).all()
+        ip, ix = b.indptr.cpu().numpy(), b.indices.cpu().numpy()
+        rows = largemap.sample_rows(w.batch, 5000)
+        p, x = largemap.subset_csr(ip, ix, rows)
+        subs.append((p, x, g1[rows], gd1[rows], g2[rows], gd2[rows]))
+        full.append((ip, ix, g1, gd1, g2, gd2))
+        del b
+    ptr = np.zeros(1, np.int64)
+    for s_ in subs:
+        ptr = np.concatenate([ptr, ptr[-1] + s_[0][1:].astype(np.int64)])
+    ptr = ptr.astype(np.int32)
+    idx = np.concatenate([s_[1] for s_ in subs])
+    sg1, sd1, sg2, sd2 = [np.concatenate([s_[k] for s_ in subs]) for k in (2, 3, 4, 5)]
+    assert sg1.size >= 20000
+    top2, norms = largemap.oracle_top2_slabbed(W16, w.V, w.M, ptr, idx)
+    rep1 = parity.check(sg1, sd1, top2, largemap.dist_to_named_neuron(W16, w.V, w.M, ptr, idx, sg1, norms), w.M)
     assert rep1.ok, str(rep1)
-    rep2 = parity.check_second(g1[rows], g2[rows], gd2[rows], top2,
-                               _dist_at_from_device(W16, w.V, w.M, ip, ix, g2[rows], norms), w.M)
+    rep2 = parity.check_second(sg1, sg2, sd2, top2,
+                               largemap.dist_to_named_neuron(W16, w.V, w.M, ptr, idx, sg2, norms), w.M)
     assert rep2.ok, str(rep2)
+    for ip, ix, g1, gd1, g2, gd2 in full:
+        for g, gd in ((g1, gd1), (g2, gd2)):
+            d_all = largemap.dist_to_named_neuron(W16, w.V, w.M, ip, ix, g, norms)
+            err = np.abs(gd.astype(np.float64) - d_all)
+            assert np.all(err <= parity.DIST_REL * np.abs(d_all) + parity.DIST_ABS), float(err.max())
     np.testing.assert_allclose(h.get_norms().cpu().numpy().astype(np.float64), norms, rtol=2e-7)
     h.destroy()
     del W16

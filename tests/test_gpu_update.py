@@ -157,6 +157,23 @@ def test_update_with_frequent_features_counted_on_chip(som_mod, mib):
     _check(got, W_old, w.V, rows, cols, b.indptr.numpy(), b.indices.numpy(), bmu, 2, rtol=1e-6)
 
 
+def test_update_at_benchmark_shape(som_mod):
+    """The shape the benchmark times: a 64 x 64 lattice, V = 30 000, one million Zipf-shaped samples,
+    radius 16 (edge / 4).  The frequent features take the on-chip counting path, the blur runs fused
+    in shared memory; every one of the 122 880 000 new weights is compared with the update oracle."""
+    w = synth.CONFIGS[1]
+    rows = cols = 64
+    rng = np.random.default_rng(31)
+    W_old = synth.fill_codebook(w.V, w.M, w.seed, device="cpu").numpy()
+    b = synth.sample_csr(w.batch, w.V, w.lam, w.seed, device="cpu")
+    assert b.n >= 1_000_000
+    ip, ix = b.indptr.numpy(), b.indices.numpy()
+    bmu = rng.integers(0, w.M, size=b.n).astype(np.int32)
+    got = _run(som_mod, W_old, w.V, rows, cols, ip, ix, bmu, 16)
+    want = uorc.update(W_old, w.V, rows, cols, ip, ix, bmu, 16)
+    np.testing.assert_allclose(got, want, rtol=1e-6, atol=1e-12)
+
+
 def test_update_with_a_huge_radius_equals_a_radius_that_spans_the_lattice(som_mod):
     V, rows, cols, n = 9, 12, 20, 300
     indptr, indices, bmu, W_old = _problem(2, V, rows, cols, n)

@@ -247,6 +247,60 @@ def test_second_best_parity_rule_on_brute_force():
     assert wrong_dist.dist_violations == n
 
 
+def test_first_unit_parity_rule_rejects_wrong_outputs():
+    """The rule every GPU parity test stands on (oracle.parity.check), against an explicit ranking
+    of all fp64 distances: the true answer passes; the second-best unit given as the best fails
+    wherever the two are outside the band; a distance off by 1e-4 relative fails; an index out of
+    range fails; a near-tied unit just inside the band passes and one just outside it fails."""
+    from oracle import parity
+    rng = np.random.default_rng(23)
+    V, M, n = 40, 12, 300
+    W = rng.random((V, M)).astype(np.float32)
+    rows = [np.sort(rng.choice(V, size=int(rng.integers(1, 9)), replace=False)).astype(np.int32) for _ in range(n)]
+    indptr = np.zeros(n + 1, np.int32)
+    indptr[1:] = np.cumsum([len(r) for r in rows])
+    indices = np.concatenate(rows)
+    D = orc.all_distances(W.reshape(-1), V, M, indptr, indices)
+    order = np.argsort(D, axis=1, kind="stable")
+    t = orc.bmu(W.reshape(-1), V, M, indptr, indices)
+    ar = np.arange(n)
+    good = parity.check(t.b1, D[ar, t.b1].astype(np.float32), t, D[ar, t.b1], M)
+    assert good.ok and good.index_mismatch_unambiguous == 0 and good.histogram_equal
+    # the oracle's second unit in place of the first
+    far = (t.d2 - t.d1) > parity.GAP_REL * t.d1
+    assert far.sum() > n // 2
+    second = parity.check(t.b2, D[ar, t.b2].astype(np.float32), t, D[ar, t.b2], M)
+    assert not second.ok and second.index_mismatch_unambiguous == int(far.sum())
+    assert not second.histogram_equal
+    # right units, distances off by 1e-4 relative (ten times the tolerance)
+    off = parity.check(t.b1, (D[ar, t.b1] * (1 + 1e-4)).astype(np.float32), t, D[ar, t.b1], M)
+    assert not off.ok and off.dist_violations == n and off.index_mismatch_unambiguous == 0
+    # distances inside the tolerance pass: 2e-6 relative
+    near = parity.check(t.b1, D[ar, t.b1] * (1 + 2e-6), t, D[ar, t.b1], M)
+    assert near.ok
+    # an index out of range, on an unambiguous and on a near-tied sample
+    bad = t.b1.copy()
+    bad[0] = M
+    bad[1] = -1
+    safe = np.clip(bad, 0, M - 1)
+    rep = parity.check(bad, D[ar, safe].astype(np.float32), t, D[ar, safe], M)
+    assert not rep.ok
+    # hand-made near ties: two units whose distances differ by a chosen relative gap
+    top = orc.Top2(np.array([3, 3, 3]), np.array([10.0, 10.0, 10.0]), np.array([5, 5, 5]),
+                   np.array([10.0 + 5e-4, 10.0 + 5e-4, 10.0 + 2e-3]))
+    # sample 0: near tie, unit 5 reported, its distance inside the band -> accepted and counted
+    # sample 1: near tie, a third unit reported whose distance is just outside the band -> rejected
+    # sample 2: unambiguous (gap 2e-4 relative), unit 5 reported -> rejected
+    g = np.array([5, 7, 5])
+    d_at = np.array([10.0 + 5e-4, 10.0 + 1.1e-3, 10.0 + 2e-3])
+    rep = parity.check(g, d_at.astype(np.float32), top, d_at, M)
+    assert rep.near_ties == 2 and rep.unambiguous == 1
+    assert rep.near_tie_outside_band == 1 and rep.index_mismatch_unambiguous == 1
+    ok_only = parity.check(g[:1], d_at[:1].astype(np.float32),
+                           orc.Top2(top.b1[:1], top.d1[:1], top.b2[:1], top.d2[:1]), d_at[:1], M)
+    assert ok_only.ok and ok_only.near_ties == 1
+
+
 def test_real_valued_samples_against_dense_brute_force():
     """Sparse real-valued samples: ||x||^2 - 2<x,w> + ||w||^2 against sum_v (x_v - w_iv)^2 on the
     densified vector (numpy); all-ones values reduce to the binary search; a neuron equal to the

@@ -1,6 +1,7 @@
 """som_norms_noalloc, the entry point for callers that cannot allocate device memory
 (their memory belongs to a pool of their own, or they cannot take the synchronisation an
-allocation may imply): it must give the same norms as the handle-based som_norms.
+allocation may imply): it must give the same norms as the handle-based som_norms, and both must
+be the CPU oracle's fp64 norms rounded to fp32.
 
 Collected last on purpose, so that a run stopping at the first failure has already run every
 other test; it passes alone in a fresh process as well as after the others.
@@ -9,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import som_oracle as orc
 from paper_2608_24067_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -46,6 +48,9 @@ def test_noalloc_norms_match_handle_norms_twice_in_a_row(som_mod):
         ref = _reference_norms(som_mod, V, M, W)
         # same fp64 accumulation, possibly split differently over V: one fp32 rounding apart at most
         np.testing.assert_allclose(out.cpu().numpy(), ref.cpu().numpy(), rtol=2e-7, atol=0.0)
+        # and against the oracle: ascending-v fp64 sums of squares, one fp32 rounding on the GPU side
+        want = orc.norms(W.cpu().numpy(), V, M)
+        np.testing.assert_allclose(out.cpu().numpy().astype(np.float64), want, rtol=2e-7, atol=0.0)
     # the same call again gives bit-identical output (fixed summation order)
     V, M, W, out = outs[1]
     again = torch.empty_like(out)
@@ -61,6 +66,8 @@ def test_noalloc_unaligned_neuron_count(som_mod):
     som_mod.norms_noalloc(V, M, W, out)
     ref = _reference_norms(som_mod, V, M, W)
     np.testing.assert_allclose(out.cpu().numpy(), ref.cpu().numpy(), rtol=2e-7, atol=0.0)
+    want = orc.norms(W.cpu().numpy(), V, M)
+    np.testing.assert_allclose(out.cpu().numpy().astype(np.float64), want, rtol=2e-7, atol=0.0)
 
 
 def test_noalloc_rejects_sizes_beyond_its_scratch(som_mod):
