@@ -174,11 +174,34 @@ int som_norms(som_handle* h, void* stream)
     return SOM_OK;
 }
 
+// Samples that do not fit a slot of the row-table plan (more than 12 hot or 8 tail features; the plan
+// lists them, the row-table kernel skips them): the direct-load kernel searches the list, whose length
+// only the device knows, and their outputs are written last.  Two small launches that return at once
+// when the list is empty.
+static int rare_pass(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head, char* ws,
+                     const SomPlanBuffers& pb, int32_t* bmu, float* dist, int32_t* bmu2, float* dist2,
+                     cudaStream_t st)
+{
+    const bool top2 = bmu2 != nullptr;
+    unsigned long long* rk = reinterpret_cast<unsigned long long*>(ws + pb.rare_keys);
+    unsigned long long* rk2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.rare_keys2) : nullptr;
+    const int32_t* list = reinterpret_cast<const int32_t*>(ws + pb.rare_list);
+    const size_t kb = (size_t)(n + 16) * sizeof(unsigned long long);
+    SOM_CK(h, cudaMemsetAsync(rk, 0xFF, kb, st));
+    if (top2) SOM_CK(h, cudaMemsetAsync(rk2, 0xFF, kb, st));
+    h->list_len_dev = reinterpret_cast<const int*>(head + pb.n_slots) + SOM_PLAN_RARE;
+    int rc = som_launch_bmu_direct(h, indptr, indices, n, rk, rk2, list, st);
+    if (!rc) rc = som_launch_finalize(h, indptr, indices, n, rk, bmu, dist, list, st);
+    if (!rc && top2) rc = som_launch_finalize(h, indptr, indices, n, rk2, bmu2, dist2, list, st);
+    h->list_len_dev = nullptr;
+    return rc;
+}
+
 // The two-stage search on a batch whose plan (slots in ws, table features in head) is ready: first
 // pass over the fp16 shadow keeping the two (som_bmu2: three) best units, certificate, exact fp32
 // pass for the samples it leaves open.  Synchronises the stream once (length of that list), twice when
 // the batch is large enough to be probed first.
-static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
+static int two_stage_passes(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
                             char* ws, const SomPlanBuffers& pb, int n_hot, int32_t* bmu, float* dist,
                             int32_t* bmu2, float* dist2, cudaStream_t st)
 {
@@ -291,6 +314,15 @@ static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t*
     return SOM_OK;
 }
 
+static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
+                            char* ws, const SomPlanBuffers& pb, int n_hot, int32_t* bmu, float* dist,
+                            int32_t* bmu2, float* dist2, cudaStream_t st)
+{
+    int rc = two_stage_passes(h, indptr, indices, n, head, ws, pb, n_hot, bmu, dist, bmu2, dist2, st);
+    if (!rc) rc = rare_pass(h, indptr, indices, n, head, ws, pb, bmu, dist, bmu2, dist2, st);
+    return rc;
+}
+
 // The search behind som_bmu (d_bmu2 == nullptr) and som_bmu2 (both second-best outputs given).
 static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
                     int32_t* d_bmu, float* d_min_dist, int32_t* d_bmu2, float* d_dist2, void* stream)
@@ -346,10 +378,11 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
                                          geom.n_hot, st)))
             return rc;
         const int32_t* counters = reinterpret_cast<const int32_t*>(head + pb.n_slots);
+        // (pinned words for the read-backs of the two-stage search)
+        if (two_stage_ok && !h->host_pair)
+            SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
         if (h->opt_variant == 0 && two_stage_ok) {
             // the two-stage search synchronises anyway: it reads the choice back
-            if (!h->host_pair)
-                SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
             SOM_CK(h, cudaMemcpyAsync(h->host_pair + 2, counters + SOM_PLAN_USE_TABLE, sizeof(int32_t),
                                       cudaMemcpyDeviceToHost, st));
             SOM_CK(h, cudaStreamSynchronize(st));
@@ -415,6 +448,8 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
             return rc;
         if (top2 && (rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, true, d_bmu2,
                                                      d_dist2, st)))
+            return rc;
+        if ((rc = rare_pass(h, d_indptr, d_indices, n_samples, head, ws, pb, d_bmu, d_min_dist, d_bmu2, d_dist2, st)))
             return rc;
         if (gate) {
             h->gate_want = 0;
@@ -610,6 +645,9 @@ int som_bmu_planned(som_handle* h, som_plan* p, int32_t* d_bmu, float* d_min_dis
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, p->indptr, p->indices, p->n, p->ws, p->pb, false, d_bmu,
                                              d_min_dist, st)))
+            return rc;
+        if ((rc = rare_pass(h, p->indptr, p->indices, p->n, p->head, p->ws, p->pb, d_bmu, d_min_dist, nullptr,
+                            nullptr, st)))
             return rc;
     }
     if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;

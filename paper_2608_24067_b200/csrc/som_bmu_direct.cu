@@ -117,9 +117,11 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
              const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
              unsigned long long* __restrict__ keys, unsigned long long* __restrict__ keys2,
              int64_t neuron_off, const int32_t* __restrict__ sample_list,
-             const float* __restrict__ values = nullptr, const int* __restrict__ gate = nullptr, int gate_want = 0)
+             const float* __restrict__ values = nullptr, const int* __restrict__ gate = nullptr, int gate_want = 0,
+             int sample_groups = 0, const int* __restrict__ n_dev = nullptr)
 {
     if (som_gated_off(gate, gate_want)) return;
+    if (n_dev) n = *n_dev;  // length of a sample list that lives on the device
     constexpr int TILE = 32 * VEC;  // neurons per tile
     // features whose row segments are in flight together (fp16 rows are half as long: twice as many)
     constexpr int FEATS = sizeof(ST) == 2 ? 8 : 4;
@@ -143,9 +145,12 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
     // byte address of the lane's first neuron in feature row 0; row v is row_bytes * v further on
     const char* W_lane = reinterpret_cast<const char*>(W + (live[0] ? i0 : 0));
 
-    const int64_t s0 = ((int64_t)blockIdx.x * DIRECT_WARPS + warp) * DIRECT_SAMPLES_PER_WARP;
+    // A block takes the sample groups blockIdx.x, blockIdx.x + gridDim.x, ...: one group per block in the
+    // plain launch; a gated launch (which mostly returns at once) comes with a small grid instead.
+    for (int bx = blockIdx.x; bx < sample_groups; bx += gridDim.x) {
+    const int64_t s0 = ((int64_t)bx * DIRECT_WARPS + warp) * DIRECT_SAMPLES_PER_WARP;
     const int n_mine = (int)min((int64_t)DIRECT_SAMPLES_PER_WARP, n - s0);
-    if (n_mine <= 0) return;
+    if (n_mine <= 0) break;  // (later groups lie further on)
     // lane q holds the row bounds of the warp's q-th sample
     // (with a sample list, position s of the list and of the key arrays is sample list[s])
     int beg_l = 0, end_l = 0;
@@ -296,6 +301,7 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
         first = next;
         first_x = next_x;
     }
+    }
 }
 
 // One thread per sample: unpack the winner and recompute its full squared distance
@@ -306,17 +312,18 @@ __global__ void k_finalize(const ST* __restrict__ W, const double* __restrict__ 
                            int64_t n, const unsigned long long* __restrict__ keys,
                            int32_t* __restrict__ bmu, float* __restrict__ dist,
                            const int32_t* __restrict__ sample_list, const float* __restrict__ values = nullptr,
-                           const int* __restrict__ gate = nullptr, int gate_want = 0)
+                           const int* __restrict__ gate = nullptr, int gate_want = 0,
+                           const int* __restrict__ n_dev = nullptr)
 {
     if (som_gated_off(gate, gate_want)) return;
-    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= n) return;
+    if (n_dev) n = *n_dev;  // length of a sample list that lives on the device
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n; k += (int64_t)gridDim.x * blockDim.x) {
     const int64_t s = sample_list ? (int64_t)sample_list[k] : k;
     const uint32_t idx = (uint32_t)(keys[k] & 0xffffffffull);
     if (idx >= M) {  // only a second-best key can be empty: fewer than two neurons
         bmu[s] = -1;
         dist[s] = __int_as_float(0x7f800000);
-        return;
+        continue;
     }
     const int beg = indptr[s];
     const int end = indptr[s + 1];
@@ -333,6 +340,7 @@ __global__ void k_finalize(const ST* __restrict__ W, const double* __restrict__ 
     }
     bmu[s] = (int32_t)idx;
     dist[s] = (float)(xx - 2.0 * dot + norm64[idx]);
+    }
 }
 
 __global__ void k_validate(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
@@ -373,20 +381,21 @@ template <int VEC, int TILES, typename ST>
 static void launch_direct(dim3 grid, cudaStream_t st, const ST* W, som_handle* h, const int32_t* indptr,
                           const int32_t* indices, int64_t n, unsigned long long* keys,
                           unsigned long long* keys2, int64_t neuron_off, const int32_t* sample_list,
-                          const float* values)
+                          const float* values, int sample_groups)
 {
     const uint32_t row_bytes = (uint32_t)(h->M * (int64_t)sizeof(ST));
     if (values)
         k_bmu_direct<VEC, TILES, false, ST, true><<<grid, DIRECT_THREADS, 0, st>>>(
-            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, nullptr, values);
+            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, nullptr, values, nullptr, 0,
+            sample_groups);
     else if (keys2)
         k_bmu_direct<VEC, TILES, true, ST><<<grid, DIRECT_THREADS, 0, st>>>(
             W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, keys2, neuron_off, sample_list, nullptr,
-            h->gate, h->gate_want);
+            h->gate, h->gate_want, sample_groups, h->list_len_dev);
     else
         k_bmu_direct<VEC, TILES, false, ST><<<grid, DIRECT_THREADS, 0, st>>>(
             W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, sample_list, nullptr,
-            h->gate, h->gate_want);
+            h->gate, h->gate_want, sample_groups, h->list_len_dev);
 }
 
 template <typename ST>
@@ -405,10 +414,14 @@ static int launch_direct_any(som_handle* h, const ST* W, const int32_t* indptr, 
     const int64_t max_gy = 65535;
     for (int64_t y0 = 0; y0 < gy; y0 += max_gy) {
         const int64_t ny = (gy - y0 < max_gy) ? gy - y0 : max_gy;
-        dim3 grid((unsigned)gx, (unsigned)ny);
+        // a gated launch returns at once on most calls: keep it to about 2048 blocks, each of which walks
+        // several sample groups when it does run
+        int64_t gx_launch = gx;
+        if ((h->gate || h->list_len_dev) && gx * ny > 2048) gx_launch = 2048 / ny > 1 ? 2048 / ny : 1;
+        dim3 grid((unsigned)gx_launch, (unsigned)ny);
         const int64_t neuron_off = y0 * neurons_per_block;
 #define SOM_DIRECT(VEC_, TILES_) \
-    launch_direct<VEC_, TILES_, ST>(grid, st, W, h, indptr, indices, n, keys, keys2, neuron_off, sample_list, values)
+    launch_direct<VEC_, TILES_, ST>(grid, st, W, h, indptr, indices, n, keys, keys2, neuron_off, sample_list, values, (int)gx)
         if constexpr (sizeof(ST) == 2) {
             if (vec == 8 && tiles == 2) SOM_DIRECT(8, 2);
             else if (vec == 8) SOM_DIRECT(8, 1);
@@ -463,13 +476,16 @@ int som_launch_finalize(som_handle* h, const int32_t* indptr, const int32_t* ind
                         const unsigned long long* keys, int32_t* bmu, float* dist, const int32_t* sample_list,
                         cudaStream_t st)
 {
-    const int64_t blocks = (n + 255) / 256;
+    int64_t blocks = (n + 255) / 256;
+    if (h->list_len_dev && blocks > 64) blocks = 64;  // a list whose (short) length lives on the device
     if (h->Wh)
         k_finalize<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, indptr, indices, n, keys,
-                                                             bmu, dist, sample_list, nullptr, h->gate, h->gate_want);
+                                                             bmu, dist, sample_list, nullptr, h->gate, h->gate_want,
+                                                             h->list_len_dev);
     else
         k_finalize<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, indptr, indices, n, keys,
-                                                            bmu, dist, sample_list, nullptr, h->gate, h->gate_want);
+                                                            bmu, dist, sample_list, nullptr, h->gate, h->gate_want,
+                                                            h->list_len_dev);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -164,6 +164,14 @@ struct LayF32 {
     {
         return lds_acc<H>(reinterpret_cast<const unsigned char*>(hn) + q * 16);
     }
+    static __device__ __forceinline__ Scores worst()
+    {
+        Scores r;
+        const u64 two_inf = 0x7f8000007f800000ull;
+#pragma unroll
+        for (int x = 0; x < H; ++x) r.g[x].lo = r.g[x].hi = two_inf;
+        return r;
+    }
     static __device__ __forceinline__ void unpack(const Scores& s, float (&a)[R_])
     {
 #pragma unroll
@@ -247,6 +255,13 @@ struct LayF16 {
         r.v[4] = hi.x; r.v[5] = hi.y; r.v[6] = hi.z; r.v[7] = hi.w;
         return r;
     }
+    static __device__ __forceinline__ Scores worst()
+    {
+        Scores r;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r.v[j] = __int_as_float(0xff800000);  // negated scores: -inf
+        return r;
+    }
     static __device__ __forceinline__ void unpack(const Scores& s, float (&a)[8])
     {
 #pragma unroll
@@ -322,6 +337,13 @@ struct LayF16W {
         }
         return r;
     }
+    static __device__ __forceinline__ Scores worst()
+    {
+        Scores r;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) r.v[j] = __int_as_float(0xff800000);  // negated scores: -inf
+        return r;
+    }
     static __device__ __forceinline__ void unpack(const Scores& s, float (&a)[16])
     {
 #pragma unroll
@@ -366,8 +388,7 @@ template <typename L, int THREADS, int KEEP>
 __global__ void __launch_bounds__(THREADS, 1)
 k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
-            const uint4* __restrict__ slots, const int32_t* __restrict__ indptr,
-            const int32_t* __restrict__ indices, const int32_t* __restrict__ feat_slot, int V, int64_t n_pad,
+            const uint4* __restrict__ slots, int64_t n_pad,
             u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
             int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter,
             const int* __restrict__ gate, int gate_want)
@@ -557,19 +578,11 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
                     } else {
                         // rare: a sample that does not fit its slot (more than 12 hot or 8 tail
-                        // features).  Its inline codes are the zero row and feature 0; start
-                        // over from base and walk its row of the batch, ascending, looking each
-                        // feature up in the feature -> table slot map (mask features are in base).
-                        acc = base;
-                        const uint32_t sidx = s0.y;
-                        const int jb = __ldg(indptr + sidx), je = __ldg(indptr + sidx + 1);
-                        for (int j = jb; j < je; ++j) {
-                            const int v = __ldg(indices + j);
-                            if ((unsigned)v >= (unsigned)V) continue;
-                            const int fs = __ldg(feat_slot + v);
-                            if (fs < 0) L::sub(acc, SOM_TAIL((uint32_t)v));
-                            else if (fs >= SOM_PLAN_MASK_FEATURES) SOM_HOT(fs);
-                        }
+                        // features) is not searched here: its scores are made the worst possible,
+                        // so that it offers no candidate; the direct-load kernel searches the
+                        // list of such samples afterwards.  (Walking its row of the batch here,
+                        // even out of line, cost the hot loop of every sample 15 to 20 %.)
+                        acc = L::worst();
                     }
                 }
 
@@ -696,7 +709,7 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
                                       reinterpret_cast<const int32_t*>(head + b.slot_feat),
                                       SOM_PLAN_MASK_FEATURES + n_hot,
                                       reinterpret_cast<const uint4*>(ws + b.slots),
-                                      indptr, indices, reinterpret_cast<const int32_t*>(head + b.feat_slot), h->V, n,
+                                      n,
                                       reinterpret_cast<u64*>(ws + b.keys),
                                       KEEP >= 2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr,
                                       KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,

@@ -71,6 +71,10 @@ struct som_handle {
     // kernels of both search paths, and a kernel returns at once unless *gate == gate_want.
     const int* gate;       // device, nullptr = no gate
     int gate_want;
+    // Length of a sample list that only the device knows (the samples that do not fit a slot of the
+    // row-table plan): while set, the direct-load kernel and its finalisation read their sample count
+    // from it and are launched with small grids that walk the list.
+    const int* list_len_dev;
     int* dev_flags;        // device, sticky: SOM_FLAG_* bits set by kernels that skipped a bad entry
     int32_t* host_pair;    // pinned, 4 ints: read-back of indptr[0], indptr[n], covered instances, uncertain samples
 };

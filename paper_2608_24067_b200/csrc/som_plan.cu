@@ -9,8 +9,8 @@
 //   4. exclusive scan of the bins                           (k_scan_*)
 //   5. scatter every sample to its sorted position and write its fixed-size slot there:
 //      hot features as byte offsets of their table row, tail features as feature ids
-//      (k_scatter_slots); the rare sample that does not fit a slot is marked, and the search
-//      kernel reads its row of the batch itself.
+//      (k_scatter_slots); the rare sample that does not fit a slot is marked and listed, and the
+//      direct-load kernel searches that list after the row-table kernel.
 //
 // Samples that share a mask end up adjacent, so the search kernel keeps
 // ||w||^2/2 - sum(mask rows) in registers across them (the corpus-clustering lever of
@@ -337,7 +337,8 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
                 const int32_t* __restrict__ feat_slot, int n_mask, int zero_row,
                 const uint32_t* __restrict__ pk, const uint32_t* __restrict__ ntail,
                 uint32_t* __restrict__ bin_cursor /* starts as bin_start */,
-                uint32_t* __restrict__ slots, const int* __restrict__ gate, int gate_want)
+                uint32_t* __restrict__ slots, int32_t* __restrict__ rare_list, int32_t* __restrict__ rare_count,
+                const int* __restrict__ gate, int gate_want)
 {
     if (som_gated_off(gate, gate_want)) return;
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -384,8 +385,10 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
                 ++ih;
             }
         }
+    } else {
+        // a sample that does not fit a slot goes on the list that the direct-load kernel searches
+        rare_list[atomicAdd(rare_count, 1)] = (int32_t)s;
     }
-    // (a sample that does not fit keeps no list: the search kernel reads its row of the batch itself)
     uint4* slot = reinterpret_cast<uint4*>(slots + (size_t)pos * SOM_SLOT_WORDS);
     slot[0] = make_uint4(w[0], w[1], w[2], w[3]);
     slot[1] = make_uint4(w[4], w[5], w[6], w[7]);
@@ -440,6 +443,9 @@ size_t som_plan_workspace_bytes(int64_t n, SomPlanBuffers* b)
     b->ukeys = take((size_t)(n + 16) * 8);
     b->ukeys2 = take((size_t)(n + 16) * 8);
     b->slots2 = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
+    b->rare_list = take((size_t)n * 4);
+    b->rare_keys = take((size_t)(n + 16) * 8);
+    b->rare_keys2 = take((size_t)(n + 16) * 8);
     return off;
 }
 
@@ -524,7 +530,9 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
     }
     // 5. scatter + slots (bin_start doubles as the running cursor)
     k_scatter_slots<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, h->V, feat_slot, n_mask, n_mask + n_hot, pk, ntail,
-                                                      bin_start, slots, h->gate, h->gate_want);
+                                                      bin_start, slots, reinterpret_cast<int32_t*>(ws + b.rare_list),
+                                                      reinterpret_cast<int32_t*>(head + b.n_slots) + SOM_PLAN_RARE,
+                                                      h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());
     const int64_t n_pad = (n + 3) / 4 * 4;
     if (n_pad > n) {

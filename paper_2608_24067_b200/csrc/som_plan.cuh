@@ -21,9 +21,10 @@ struct som_handle;
 //             unused ones hold the index of the all-zero row that follows the table
 //   w8..w11   tail codes 0..7, 16 bits each: feature id
 // A sample fits when it has at most 12 hot and 8 tail features; for the rare others the slot
-// holds only the mask and the sample index (hot codes all zero-row, tail codes feature 0), and
-// the search kernel walks the sample's row of the batch itself, looking each feature up in the
-// feature -> table slot map.  16-bit codes require V <= 65536 and at most 65536 table rows.
+// holds only the mask and the sample index (hot codes all zero-row, tail codes feature 0): the
+// row-table kernel gives such a sample no candidate, and its index goes on a list (rare_list)
+// that the direct-load kernel searches afterwards, writing its outputs last.
+// 16-bit codes require V <= 65536 and at most 65536 table rows.
 // The slot array is padded to a multiple of 4 samples with copies of the last slot, so the
 // search kernel always runs whole rounds; the duplicates redo the same idempotent atomicMin.
 #define SOM_SLOT_WORDS 12
@@ -39,7 +40,7 @@ struct SomPlanBuffers {
     size_t feat_count;  // u32 [V]
     size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
     size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
-    size_t n_slots;     // i32 [8]      mask slots used, hot slots used, (unused), search unit counter,
+    size_t n_slots;     // i32 [8]      mask slots used, hot slots used, length of rare_list, search unit counter,
                         //              feature instances covered by the table, uncertain samples,
                         //              1 if the automatic mode takes the row-table kernel for this batch
     // workspace
@@ -56,8 +57,12 @@ struct SomPlanBuffers {
     size_t ukeys;       // u64 [n + 16] their packed keys, by position in that list
     size_t ukeys2;      // u64 [n + 16] and their second-best keys (two-best search)
     size_t slots2;      // 48 B [n + 16] their slots, compacted in list order
+    size_t rare_list;   // i32 [n]      samples that do not fit a slot (searched by the direct-load kernel)
+    size_t rare_keys;   // u64 [n + 16] their packed keys, by position in that list
+    size_t rare_keys2;  // u64 [n + 16] and their second-best keys (two-best search)
 };
 #define SOM_PLAN_N_SLOTS_INTS 8
+#define SOM_PLAN_RARE 2 /* index into n_slots: length of rare_list */
 #define SOM_PLAN_COVERED 4 /* index into n_slots */
 #define SOM_PLAN_UNCERTAIN 5 /* index into n_slots: length of the two-stage search's uncertain list */
 #define SOM_PLAN_USE_TABLE 6 /* index into n_slots: the selection kernel's choice of search kernel */
@@ -89,7 +94,6 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
 
 // shadow = read the handle's fp16 shadow of an fp32 codebook (first pass of the two-stage search);
 // keep = how many best units per sample are kept (1, 2; 3 with the shadow's wide layout only)
-// indptr / indices: the batch (rows of samples that do not fit a slot are read from it)
 int som_launch_bmu_table(som_handle* h, bool shadow, const int32_t* indptr, const int32_t* indices, int64_t n,
                          char* head, char* ws, const SomPlanBuffers& b, int n_hot, int keep, cudaStream_t st);
 
