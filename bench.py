@@ -578,6 +578,56 @@ def run_ours(args, workloads):
     ctx.close()
 
 
+def run_tc_probe(args):
+    """Go / no-go microbenchmark of the densified hot-feature tile on tcgen05 (library call som_tc_probe):
+    cycles per tile of 128 samples x 64 neurons for building the 0/1 tile, the MMAs and the drain, alone and
+    pipelined, on every SM at once, with membership bits of the workload's H most frequent features."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device")
+    from paper_2608_24067_b200 import som
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    w = synth.CONFIGS[2]
+    n_tiles, repeats = 64, 40
+    b = synth.sample_csr(n_tiles * 128, w.V, w.lam, w.seed, device="cpu")
+    ip, ix = b.indptr.numpy().astype(np.int64), b.indices.numpy()
+    row = np.repeat(np.arange(b.n), np.diff(ip))
+    rng = np.random.default_rng(0)
+    results = []
+    modes = [(1, "build"), (2, "mma"), (4, "drain"), (6, "mma+drain"), (7, "build+mma+drain"),
+             (15, "build+mma+drain+redistribute"), (16, "lds"), (18, "mma+lds")]
+    for H in (32, 64, 128, 256):
+        # the workload's ids are frequency ranks: the H most frequent features are ids 0 .. H-1
+        sel = ix < H
+        words = np.zeros((b.n, H // 32), np.uint32)
+        np.bitwise_or.at(words, (row[sel], ix[sel] // 32), (np.uint32(1) << (ix[sel] % 32).astype(np.uint32)))
+        inst = float(sel.sum()) / b.n
+        rows = (rng.random((H, 64)) * 0.05).astype(np.float32)
+        hnorm = (17.0 + rng.random(64)).astype(np.float32)
+        member = ((words[:128, :, None] >> np.arange(32, dtype=np.uint32)[None, None, :]) & 1).reshape(128, H)
+        want = hnorm.astype(np.float64)[None, :] - member.astype(np.float64) @ rows.astype(np.float64)
+        d_rows, d_h = torch.from_numpy(rows).to(dev), torch.from_numpy(hnorm).to(dev)
+        d_bits = torch.from_numpy(words.view(np.int32)).to(dev)
+        for terms in (1, 2):
+            entry = {"H": H, "terms": terms, "dense_instances_per_sample": inst, "cycles_per_tile": {}}
+            for mode, name in modes:
+                som.tc_probe(d_rows, d_h, d_bits, H, terms, n_tiles, mode, 2, sms)  # warm-up
+                r = som.tc_probe(d_rows, d_h, d_bits, H, terms, n_tiles, mode, repeats, sms)
+                torch.cuda.synchronize()
+                if int(r["status"].item()) != 0:
+                    raise SystemExit("tc probe: a bounded wait gave up (H=%d terms=%d mode=%d)" % (H, terms, mode))
+                cyc = float(r["cycles"].double().mean().item()) / (n_tiles * repeats)
+                entry["cycles_per_tile"][name] = cyc
+                if mode == 7:
+                    entry["max_abs_err_first_tile"] = float(np.abs(r["out"].cpu().numpy() - want).max())
+                    entry["pairs_per_clk_per_sm"] = 128 * 64 / cyc
+            results.append(entry)
+    print(json.dumps({"tc_probe": results, "tile": "128 samples x 64 neurons", "blocks": sms,
+                      "note": "cycles per tile, mean over blocks, every SM busy; membership of the 128x128 "
+                              "workload's H most frequent features"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -620,8 +670,13 @@ def main():
     ap.add_argument("--radius", type=int, default=0, help="som_update: blur radius (default edge / 4)")
     ap.add_argument("--batch", type=int, default=0,
                     help="samples per batch instead of the configuration's (a sweep variant, named in the workload)")
+    ap.add_argument("--tc-probe", action="store_true",
+                    help="run the tcgen05 microbenchmark of the densified hot-feature tile and print its numbers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.tc_probe:
+        run_tc_probe(args)
+        return
 
     def variant_of(w):
         if args.features == "uniform":

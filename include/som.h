@@ -327,6 +327,35 @@ int som_last_cuda_error(const som_handle* h);
  */
 int som_measure_fadd_peak(double* adds_per_s, float* d_scratch, int64_t scratch_elems, void* stream);
 
+/*
+ * som_tc_probe - measured probe of a densified hot-feature tile on the tensor cores (no counterpart in
+ * the paper, whose kernels run on plain CUDA cores; Section 3.3 is the gather it restates).  For the H
+ * most frequent features of a batch the gather-sum of a tile of 128 samples over 64 neurons is the dense
+ * product of the samples' 0/1 membership matrix with those features' rows.  The probe runs that product on
+ * tcgen05.mma (fp16 operands, fp32 accumulation in tensor memory) with the steps a fused search kernel
+ * would need around it - building the 0/1 tile in shared memory from membership bits, the MMAs, draining
+ * the accumulator into registers - and reports the clock cycles, so that the cost can be compared with the
+ * shared-memory reads the product would replace.  The accumulator is seeded with ||w||^2 / 2 and the rows
+ * are subtracted, i.e. it holds the samples' partial scores.
+ *   d_rows     DEVICE, fp32 [H][64]: rows of the H dense features for one range of 64 neurons.
+ *   d_hnorm    DEVICE, fp32 [64]: ||w||^2 / 2 of those neurons.
+ *   d_bits     DEVICE, uint32 [n_tiles * 128][H / 32]: bit f % 32 of word f / 32 = sample has feature f.
+ *   H          32 ... 256, a multiple of 32.   terms: fp16 terms per weight, 1 (rounded) or 2 (hi + lo).
+ *   mode       bit 0 build the 0/1 tile for every tile (else only the first two), bit 1 issue the MMAs,
+ *              bit 2 drain the accumulators, bit 3 also redistribute the drained values by shuffles to
+ *              eight threads per sample, bit 4 the drain warps also stream 1024 wavefronts of 128-bit
+ *              shared-memory reads per tile (to see whether they and the MMAs' operand fetch contend).
+ *   repeats    every block walks the n_tiles tiles this many times; blocks: thread blocks (one per SM).
+ *   d_out      DEVICE, fp32 [128][64] or NULL: partial scores of the first tile (written by block 0).
+ *   d_mins     DEVICE, fp32 [blocks][128] or NULL: per-sample minimum score of the last tile walked.
+ *   d_cycles   DEVICE, int64 [blocks]: clock cycles of each block's loop.
+ *   d_status   DEVICE, int: 0, or 1 if a bounded wait inside the kernel gave up (results invalid).
+ * Enqueues one kernel on `stream`; does not synchronise.
+ */
+int som_tc_probe(const float* d_rows, const float* d_hnorm, const uint32_t* d_bits, int32_t H, int32_t terms,
+                 int32_t n_tiles, int32_t mode, int32_t repeats, int32_t blocks, float* d_out, float* d_mins,
+                 long long* d_cycles, int* d_status, void* stream);
+
 int som_set_timing(som_handle* h, int enable);
 int som_get_timing(som_handle* h, float* out_ms, int n_out);
 int64_t som_launch_count(const som_handle* h);

@@ -26,7 +26,7 @@ EXPORTS = [
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
     "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain", "som_bmu_values",
     "som_bmu_host_async", "som_host_sync", "som_plan_create", "som_bmu_planned", "som_plan_destroy",
-    "som_device_flags", "som_measure_fadd_peak",
+    "som_device_flags", "som_measure_fadd_peak", "som_tc_probe",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -92,6 +92,8 @@ def load_library():
     lib.som_set_option.argtypes = [P, INT, I64]
     lib.som_measure_fadd_peak.argtypes = [ctypes.POINTER(ctypes.c_double), P, I64, P]
     lib.som_measure_fadd_peak.restype = INT
+    lib.som_tc_probe.argtypes = [P, P, P, I32, I32, I32, I32, I32, I32, P, P, P, P, P]
+    lib.som_tc_probe.restype = INT
     lib.som_device_flags.argtypes = [P, P]
     lib.som_device_flags.restype = INT
     lib.som_norms_noalloc.argtypes = [I32, I64, P, P, P]
@@ -150,6 +152,28 @@ def measure_fadd_peak(device=None, stream=None) -> float:
     if rc != SOM_OK:
         raise SomError(rc, "som_measure_fadd_peak")
     return float(out.value)
+
+
+def tc_probe(rows: torch.Tensor, hnorm: torch.Tensor, bits: torch.Tensor, H: int, terms: int, n_tiles: int,
+             mode: int = 7, repeats: int = 1, blocks: int = 1, stream=None) -> dict:
+    """som_tc_probe: the densified hot-feature tile on tcgen05 (argument marshalling only).  Returns the
+    first tile's partial scores [128, 64], the per-sample minima [blocks, 128], the cycles per block and
+    the kernel's status word (tensors on the device; synchronise before reading)."""
+    lib = load_library()
+    dev = rows.device
+    out = torch.zeros(128, 64, dtype=torch.float32, device=dev)
+    mins = torch.zeros(blocks, 128, dtype=torch.float32, device=dev)
+    cycles = torch.zeros(blocks, dtype=torch.int64, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    if bits.dtype != torch.int32 or bits.numel() != n_tiles * 128 * (H // 32):
+        raise ValueError("bits must be int32 [n_tiles * 128, H / 32]")
+    with torch.cuda.device(dev):
+        rc = lib.som_tc_probe(_dev_ptr(rows, torch.float32, "rows"), _dev_ptr(hnorm, torch.float32, "hnorm"),
+                              bits.data_ptr(), H, terms, n_tiles, mode, repeats, blocks, out.data_ptr(),
+                              mins.data_ptr(), cycles.data_ptr(), status.data_ptr(), _stream_ptr(stream))
+    if rc != SOM_OK:
+        raise SomError(rc, "som_tc_probe")
+    return {"out": out, "mins": mins, "cycles": cycles, "status": status}
 
 
 class Plan:
