@@ -227,6 +227,7 @@ static int two_stage_passes(som_handle* h, const int32_t* indptr, const int32_t*
         const size_t pkb = (size_t)(n_probe + 16) * sizeof(unsigned long long);
         SomPlanBuffers pp = pb;
         pp.slots = pb.slots2;
+        pp.order = pb.uncertain;
         pp.keys = pb.ukeys;
         pp.keys2 = pb.ukeys2;  // (keys3 is not in use yet: its head serves the probe)
         SOM_CK(h, cudaMemsetAsync(ws + pp.keys, 0xFF, pkb, st));
@@ -284,6 +285,7 @@ static int two_stage_passes(som_handle* h, const int32_t* indptr, const int32_t*
         if (exact.n_hot == n_hot && units >= 2 * (int64_t)h->sm_count) {
             SomPlanBuffers pe = pb;
             pe.slots = pb.slots2;
+            pe.order = pb.uncertain;  // the list holds the sample index of every compacted slot
             pe.keys = pb.ukeys;
             pe.keys2 = pb.ukeys2;
             SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(head + pb.n_slots) + 3, 0, sizeof(int), st));

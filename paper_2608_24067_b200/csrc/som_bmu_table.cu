@@ -576,8 +576,10 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         if (nt > 5) L::sub(acc, SOM_TAIL(hi16(t45)));
                         if (nt > 6) L::sub(acc, SOM_TAIL(lo16(t67)));
                         if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
+                        if (nt > 8) L::sub(acc, SOM_TAIL(lo16(s0.y)));
+                        if (nt > 9) L::sub(acc, SOM_TAIL(hi16(s0.y)));
                     } else {
-                        // rare: a sample that does not fit its slot (more than 12 hot or 8 tail
+                        // rare: a sample that does not fit its slot (more than 12 hot or 10 tail
                         // features) is not searched here: its scores are made the worst possible,
                         // so that it offers no candidate; the direct-load kernel searches the
                         // list of such samples afterwards.  (Walking its row of the batch here,
@@ -655,14 +657,14 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 template <typename ST>
 __global__ void k_finalize_sorted(const ST* __restrict__ W, const double* __restrict__ norm64, int64_t M, int V,
                                   const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
-                                  int64_t n, const uint4* __restrict__ slots,
+                                  int64_t n, const uint32_t* __restrict__ order,
                                   const u64* __restrict__ keys, int32_t* __restrict__ bmu,
                                   float* __restrict__ dist, const int* __restrict__ gate, int gate_want)
 {
     if (som_gated_off(gate, gate_want)) return;
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= n) return;
-    const uint32_t s = slots[k * SLOT_Q].y;
+    const uint32_t s = order[k];
     const uint32_t idx = (uint32_t)(keys[k] & 0xffffffffull);
     if (idx >= M) {  // only a second-best key can be empty: fewer than two neurons
         bmu[s] = -1;
@@ -825,8 +827,8 @@ __device__ __forceinline__ float score_of_key(u64 key)
 template <bool SECOND, bool COUNT_ONLY>
 __global__ void k_certify(const float* __restrict__ W, const double* __restrict__ norm64, int64_t M, int V,
                           const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
-                          const uint4* __restrict__ slots, const u64* __restrict__ keys,
-                          const u64* __restrict__ keys2, const u64* __restrict__ keys3,
+                          const uint4* __restrict__ slots, const uint32_t* __restrict__ order,
+                          const u64* __restrict__ keys, const u64* __restrict__ keys2, const u64* __restrict__ keys3,
                           const unsigned int* __restrict__ wmax_bits, const float* __restrict__ hnorm,
                           int32_t* __restrict__ bmu, float* __restrict__ dist,
                           int32_t* __restrict__ bmu2, float* __restrict__ dist2,
@@ -840,7 +842,7 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
     bool flag = false;
     uint32_t s = 0;
     if (k < n) {
-        s = slots[k * SLOT_Q].y;
+        s = order[k];
         const u64 k1 = keys[k], k2 = keys2[k];
         const int beg = indptr[s];
         const int end = indptr[s + 1];
@@ -929,13 +931,14 @@ int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indi
 {
     const int64_t blocks = (n + 255) / 256;
     const uint4* slots = reinterpret_cast<const uint4*>(ws + b.slots);
+    const uint32_t* order = reinterpret_cast<const uint32_t*>(ws + b.order);
     const u64* keys = reinterpret_cast<const u64*>(ws + b.keys);
     const u64* keys2 = reinterpret_cast<const u64*>(ws + b.keys2);
     const u64* keys3 = second ? reinterpret_cast<const u64*>(ws + b.keys3) : nullptr;
     uint4* slots2 = reinterpret_cast<uint4*>(ws + b.slots2);
 #define SOM_CERTIFY(SECOND_, COUNT_)                                                                            \
     k_certify<SECOND_, COUNT_><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, h->V, indptr, indices, n, slots, \
-                                                                 keys, keys2, keys3, h->wmax_bits, h->hnorm, bmu,  \
+                                                                 order, keys, keys2, keys3, h->wmax_bits, h->hnorm, bmu,  \
                                                                  dist, bmu2, dist2, uncertain, slots2, n_uncertain)
     if (second && count_only) SOM_CERTIFY(true, true);
     else if (second) SOM_CERTIFY(true, false);
@@ -950,13 +953,15 @@ int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indi
 // Probe of the two-stage search: the slot of every SOM_PROBE_STRIDE-th sample (by sample index) goes to
 // position index / SOM_PROBE_STRIDE of a second slot array.
 namespace {
-__global__ void k_probe_gather(const uint4* __restrict__ slots, int64_t n, uint4* __restrict__ probe)
+__global__ void k_probe_gather(const uint4* __restrict__ slots, const uint32_t* __restrict__ order, int64_t n,
+                               uint4* __restrict__ probe, uint32_t* __restrict__ probe_order)
 {
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= n) return;
-    const uint32_t s = slots[k * SLOT_Q].y;
+    const uint32_t s = order[k];
     if (s % SOM_PROBE_STRIDE) return;
     const int64_t pos = s / SOM_PROBE_STRIDE;
+    probe_order[pos] = s;
 #pragma unroll
     for (int x = 0; x < SLOT_Q; ++x) probe[pos * SLOT_Q + x] = slots[k * SLOT_Q + x];
 }
@@ -965,8 +970,12 @@ __global__ void k_probe_gather(const uint4* __restrict__ slots, int64_t n, uint4
 int som_launch_probe_gather(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
-    k_probe_gather<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(ws + b.slots), n,
-                                                     reinterpret_cast<uint4*>(ws + b.slots2));
+    // (the probe's slots go to slots2, their sample indices to the uncertain list, which is free until
+    //  the certificate of the full batch fills it)
+    k_probe_gather<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(ws + b.slots),
+                                                     reinterpret_cast<const uint32_t*>(ws + b.order), n,
+                                                     reinterpret_cast<uint4*>(ws + b.slots2),
+                                                     reinterpret_cast<uint32_t*>(ws + b.uncertain));
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;
@@ -977,14 +986,14 @@ int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32
                                cudaStream_t st)
 {
     const int64_t blocks = (n + 255) / 256;
-    const uint4* slots = reinterpret_cast<const uint4*>(ws + b.slots);
+    const uint32_t* order = reinterpret_cast<const uint32_t*>(ws + b.order);
     const u64* keys = reinterpret_cast<const u64*>(ws + (second ? b.keys2 : b.keys));
     if (h->Wh)
         k_finalize_sorted<__half><<<(unsigned)blocks, 256, 0, st>>>(h->Wh, h->norm64, h->M, h->V, indptr, indices, n,
-                                                                    slots, keys, bmu, dist, h->gate, h->gate_want);
+                                                                    order, keys, bmu, dist, h->gate, h->gate_want);
     else
         k_finalize_sorted<float><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, h->V, indptr, indices, n,
-                                                                   slots, keys, bmu, dist, h->gate, h->gate_want);
+                                                                   order, keys, bmu, dist, h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -337,7 +337,8 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
                 const int32_t* __restrict__ feat_slot, int n_mask, int zero_row,
                 const uint32_t* __restrict__ pk, const uint32_t* __restrict__ ntail,
                 uint32_t* __restrict__ bin_cursor /* starts as bin_start */,
-                uint32_t* __restrict__ slots, int32_t* __restrict__ rare_list, int32_t* __restrict__ rare_count,
+                uint32_t* __restrict__ slots, uint32_t* __restrict__ order, int32_t* __restrict__ rare_list,
+                int32_t* __restrict__ rare_count,
                 const int* __restrict__ gate, int gate_want)
 {
     if (som_gated_off(gate, gate_want)) return;
@@ -358,7 +359,7 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
     const uint32_t zz = (uint32_t)zero_row | ((uint32_t)zero_row << 16);
     uint32_t w[SOM_SLOT_WORDS];
     w[0] = fits ? (mask | (nh << 16) | (nt << 24)) : (mask | (SOM_SLOT_NT_OVERFLOW << 24));  // (zero hot codes)
-    w[1] = (uint32_t)s;
+    w[1] = 0u;  // tail codes 8..9
 #pragma unroll
     for (int i = 2; i < 8; ++i) w[i] = zz;
 #pragma unroll
@@ -375,6 +376,8 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
                 for (int i = 0; i < 4; ++i)
                     if ((it >> 1) == (uint32_t)i)
                         w[8 + i] = (it & 1u) ? (w[8 + i] | ((uint32_t)v << 16)) : (uint32_t)v;
+                if (it == 8u) w[1] = (uint32_t)v;
+                if (it == 9u) w[1] |= (uint32_t)v << 16;
                 ++it;
             } else if (fs >= n_mask) {
 #pragma unroll
@@ -389,6 +392,7 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
         // a sample that does not fit a slot goes on the list that the direct-load kernel searches
         rare_list[atomicAdd(rare_count, 1)] = (int32_t)s;
     }
+    order[pos] = (uint32_t)s;
     uint4* slot = reinterpret_cast<uint4*>(slots + (size_t)pos * SOM_SLOT_WORDS);
     slot[0] = make_uint4(w[0], w[1], w[2], w[3]);
     slot[1] = make_uint4(w[4], w[5], w[6], w[7]);
@@ -439,6 +443,7 @@ size_t som_plan_workspace_bytes(int64_t n, SomPlanBuffers* b)
     b->bin_start = take((size_t)SOM_PLAN_BINS * 4);
     b->block_sums = take((size_t)(SOM_PLAN_BINS / SCAN_BLOCK + 2) * 4);
     b->slots = take((size_t)(n + 16) * SOM_SLOT_WORDS * 4);
+    b->order = take((size_t)(n + 16) * 4);
     b->uncertain = take((size_t)n * 4);
     b->ukeys = take((size_t)(n + 16) * 8);
     b->ukeys2 = take((size_t)(n + 16) * 8);
@@ -530,7 +535,8 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
     }
     // 5. scatter + slots (bin_start doubles as the running cursor)
     k_scatter_slots<<<sblocks, PLAN_THREADS, 0, st>>>(indptr, indices, n, h->V, feat_slot, n_mask, n_mask + n_hot, pk, ntail,
-                                                      bin_start, slots, reinterpret_cast<int32_t*>(ws + b.rare_list),
+                                                      bin_start, slots, reinterpret_cast<uint32_t*>(ws + b.order),
+                                                      reinterpret_cast<int32_t*>(ws + b.rare_list),
                                                       reinterpret_cast<int32_t*>(head + b.n_slots) + SOM_PLAN_RARE,
                                                       h->gate, h->gate_want);
     SOM_CK(h, cudaGetLastError());

@@ -16,11 +16,13 @@ struct som_handle;
 // that the search kernel can load it one round ahead without chasing an offset.  As 12 words:
 //   w0        mask of mask features (bits 0-15) | hot codes (16-23) | tail codes (24-31);
 //             a tail count of SOM_SLOT_NT_OVERFLOW marks a sample that does not fit a slot
-//   w1        sample index
+//   w1        tail codes 8..9
 //   w2..w7    hot codes 0..11, 16 bits each: row of the feature in the shared-memory table;
 //             unused ones hold the index of the all-zero row that follows the table
 //   w8..w11   tail codes 0..7, 16 bits each: feature id
-// A sample fits when it has at most 12 hot and 8 tail features; for the rare others the slot
+// (the sample index of a sorted position lives in a separate array, `order`: only the
+// finalisation needs it).
+// A sample fits when it has at most 12 hot and 10 tail features; for the rare others the slot
 // holds only the mask and the sample index (hot codes all zero-row, tail codes feature 0): the
 // row-table kernel gives such a sample no candidate, and its index goes on a list (rare_list)
 // that the direct-load kernel searches afterwards, writing its outputs last.
@@ -29,7 +31,7 @@ struct som_handle;
 // search kernel always runs whole rounds; the duplicates redo the same idempotent atomicMin.
 #define SOM_SLOT_WORDS 12
 #define SOM_SLOT_MAX_HOT 12
-#define SOM_SLOT_MAX_TAIL 8
+#define SOM_SLOT_MAX_TAIL 10
 #define SOM_SLOT_NT_OVERFLOW 255u
 
 // Byte offsets of the plan's arrays.  The first four live in the small "head" buffer, sized by V;
@@ -53,6 +55,7 @@ struct SomPlanBuffers {
     size_t bin_start;   // u32 [bins]
     size_t block_sums;  // u32 [scan blocks]
     size_t slots;       // 48 B [n + 16]
+    size_t order;       // u32 [n + 16]  sample index of every sorted position
     size_t uncertain;   // i32 [n]      samples the two-stage search sends to its exact pass
     size_t ukeys;       // u64 [n + 16] their packed keys, by position in that list
     size_t ukeys2;      // u64 [n + 16] and their second-best keys (two-best search)
