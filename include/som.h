@@ -294,8 +294,8 @@ int som_last_cuda_error(const som_handle* h);
  * som_set_option tunes kernel selection: key 0 = search kernel variant (0 auto, 1 direct-load
  * kernel, 2 shared-memory row-table kernel where M % 4 == 0 and V <= 65536); key 1 = hot rows kept in shared
  * memory by the row-table kernel (0 = default); key 2 = its block size (0 = default, 512, 640, 768, 896, 1024);
- * key 3 = neurons per lane there (0 = default; fp32 storage: 4, 8, where 8 needs M % 64 == 0; fp16 storage:
- * 8, 16, where 16 needs M % 128 == 0); key 4 = sample parts per
+ * key 3 = neurons per lane there (0 = default: the widest that divides M; fp32 storage: 4, 8, 16, where 8 needs
+ * M % 64 == 0 and 16 M % 128 == 0; fp16 storage: 8, 16, where 16 needs M % 128 == 0); key 4 = sample parts per
  * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
  * feature instances that the row table's features must cover for the row-table kernel to be taken
  * (0 = default 60; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
@@ -311,7 +311,8 @@ int som_last_cuda_error(const som_handle* h);
  * It pays on maps whose units are distinct at fp16 resolution (random initialisation, small final radius); on
  * a map that a wide blur has just smoothed most samples fail the certificate.  A batch of at least 65536
  * samples is therefore probed first (one sample in 256, chosen by sample index; one more stream
- * synchronisation): if more than a fifth of those fail, the call runs the plain search instead.
+ * synchronisation): if more than a fifth of those fail, the call runs the plain search instead (on the
+ * same plan, i.e. with 8 neurons per lane: bit-identical to a plain call with key 3 = 8).
  * Needs M % 128 == 0 and the row-table kernel.  A two-stage call synchronises the
  * stream a second time (it reads the length of the second pass's list back).  som_last_uncertain returns how
  * many samples the last two-stage search sent to its second pass (all of them when the probe chose the plain

@@ -278,7 +278,7 @@ static int two_stage_passes(som_handle* h, const int32_t* indptr, const int32_t*
         // layouts hold the same number of hot rows), else the direct-load kernel.
         unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
         unsigned long long* ukeys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.ukeys2) : nullptr;
-        const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T);
+        const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T, exact.row_bytes);
         const size_t ub = (size_t)(n_unc + 16) * sizeof(unsigned long long);
         SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, ub, st));
         if (top2) SOM_CK(h, cudaMemsetAsync(ukeys2, 0xFF, ub, st));
@@ -360,7 +360,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
                      h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
-        const int64_t parts = som_table_default_parts(n_samples, geom.T);
+        const int64_t parts = som_table_default_parts(n_samples, geom.T, geom.row_bytes);
         const int64_t units = ((h->M + geom.T - 1) / geom.T) * parts;
         if (units < 2 * (int64_t)h->sm_count) use_table = false;
     }
@@ -558,7 +558,7 @@ int som_plan_create(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     bool use_table = h->opt_variant != 1 && (h->M % (h->Wh ? 64 : 4) == 0) && h->V <= 65536 &&
                      h->M < ((int64_t)1 << 30);
     if (use_table && h->opt_variant == 0) {
-        const int64_t units = ((h->M + geom.T - 1) / geom.T) * som_table_default_parts(n_samples, geom.T);
+        const int64_t units = ((h->M + geom.T - 1) / geom.T) * som_table_default_parts(n_samples, geom.T, geom.row_bytes);
         if (units < 2 * (int64_t)h->sm_count) use_table = false;
     }
     if (!h->host_pair && cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)) != cudaSuccess)
@@ -955,7 +955,7 @@ int som_set_option(som_handle* h, int key, int64_t value)
         return SOM_OK;
     }
     if (key == 2) {
-        if (value != 0 && value != 512 && value != 640 && value != 768 &&
+        if (value != 0 && value != 512 && value != 576 && value != 640 && value != 768 &&
             value != 896 && value != 1024)
             return SOM_ERR_INVALID_ARG;
         h->opt_threads = value;

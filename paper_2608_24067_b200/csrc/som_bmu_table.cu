@@ -150,6 +150,8 @@ template <int R_>
 struct LayF32 {
     typedef float Store;
     static constexpr int R = R_, H = R_ / 4, T = 8 * R_, ROWB = T * 4;
+    // tail rows of a sample whose loads go in flight before its hot rows (each holds R registers)
+    static constexpr int TAILS_AHEAD = R_ >= 16 ? 2 : 4;
     static constexpr float SEED_SIGN = 1.f;     // scores are held as they are
     typedef Acc<H> Scores;
     typedef Acc<H> Slice;
@@ -220,6 +222,7 @@ struct LayF32 {
 struct LayF16 {
     typedef __half Store;
     static constexpr int R = 8, T = 64, ROWB = T * 2;
+    static constexpr int TAILS_AHEAD = 4;
     static constexpr float SEED_SIGN = -1.f;  // the seed array holds -||w||^2/2
     struct Scores { float v[8]; };
     typedef uint4 Slice;
@@ -295,6 +298,7 @@ struct LayF16 {
 struct LayF16W {
     typedef __half Store;
     static constexpr int R = 16, T = 128, ROWB = T * 2;
+    static constexpr int TAILS_AHEAD = 4;
     static constexpr float SEED_SIGN = -1.f;
     struct Scores { float v[16]; };
     struct Slice { uint4 g[2]; };
@@ -529,8 +533,12 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 Slice tr0, tr1, tr2, tr3;
                 if (p0) tr0 = SOM_TAIL(lo16(s2.x));
                 if (p1) tr1 = SOM_TAIL(hi16(s2.x));
-                if (p2) tr2 = SOM_TAIL(lo16(s2.y));
-                if (p3) tr3 = SOM_TAIL(hi16(s2.y));
+                if constexpr (L::TAILS_AHEAD >= 3) {
+                    if (p2) tr2 = SOM_TAIL(lo16(s2.y));
+                }
+                if constexpr (L::TAILS_AHEAD >= 4) {
+                    if (p3) tr3 = SOM_TAIL(hi16(s2.y));
+                }
 
                 // ---- mask prefix ------------------------------------------------------------
                 if (mask != curmask) {
@@ -568,8 +576,16 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 // ---- tail rows ------------------------------------------------------------------
                 if (p0) L::sub(acc, tr0);
                 if (p1) L::sub(acc, tr1);
-                if (p2) L::sub(acc, tr2);
-                if (p3) L::sub(acc, tr3);
+                if constexpr (L::TAILS_AHEAD >= 3) {
+                    if (p2) L::sub(acc, tr2);
+                } else {
+                    if (p2) L::sub(acc, SOM_TAIL(lo16(s2.y)));
+                }
+                if constexpr (L::TAILS_AHEAD >= 4) {
+                    if (p3) L::sub(acc, tr3);
+                } else {
+                    if (p3) L::sub(acc, SOM_TAIL(hi16(s2.y)));
+                }
                 if (nt > 4) {
                     if (nt != SOM_SLOT_NT_OVERFLOW) {
                         L::sub(acc, SOM_TAIL(lo16(t45)));
@@ -690,7 +706,7 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     constexpr int T = L::T;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
     const int n_ranges = (int)((h->M + T - 1) / T);
-    int parts = h->opt_parts > 0 ? (int)h->opt_parts : som_table_default_parts(n, T);
+    int parts = h->opt_parts > 0 ? (int)h->opt_parts : som_table_default_parts(n, T, L::ROWB);
     if ((int64_t)parts * 1024 > n) parts = (int)(n / 1024);
     if (parts < 1) parts = 1;
     int64_t part_len = (n + parts - 1) / parts;
@@ -734,20 +750,27 @@ SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
     // (an fp16-stored codebook has the 8-neuron layout only; som_table_usable checks M % 64)
     g.R = (f16 || (h->opt_r != 4 && h->M % 64 == 0)) ? 8 : 4;
     if (f16 && h->opt_r != 8 && h->M % 128 == 0) g.R = 16;  // wide fp16 layout wherever it divides M
+    // fp32 storage: 16 neurons per lane (128-neuron ranges, 512-byte rows) wherever 128 divides M: half the
+    // per-round bookkeeping and half the row visits per add (3 to 5 % faster; 11 % on the largest map,
+    // where every row visit is another 2 MB page)
+    // (not with the two-stage search, whose exact pass shares the plan of the fp16 first pass: 720 hot rows)
+    if (!f16 && h->opt_r != 4 && h->opt_r != 8 && h->M % 128 == 0 && h->opt_two_stage != 1) g.R = 16;
     g.T = 8 * g.R;
     const int row_bytes = g.T * (f16 ? 2 : 4);
     // (the fp16 layout holds half as many row registers: 896 threads at 72 registers measured best)
-    const int def_threads = f16 ? (g.R == 16 ? 512 : 896) : (g.R == 8 ? 640 : 1024);
-    g.threads = (h->opt_threads == 512 || h->opt_threads == 640 || h->opt_threads == 768 ||
+    const int def_threads = f16 ? (g.R == 16 ? 512 : 896) : (g.R == 16 ? 512 : (g.R == 8 ? 640 : 1024));
+    g.threads = (h->opt_threads == 512 || h->opt_threads == 576 || h->opt_threads == 640 || h->opt_threads == 768 ||
                  h->opt_threads == 896 || h->opt_threads == 1024)
                     ? (int)h->opt_threads : def_threads;
     // 227 KB per block, minus the static shared memory (slot rings, norms) of the kernel
     int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
     // Defaults keep dynamic + static shared memory under 196 KB: one step more and the SM's
     // carve-out leaves 28 KB instead of 60 KB of L1, which costs 12 % at 128x128 (measured).
-    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows : (row_bytes == 128 ? (f16 ? 1456 : 1376) : 720);
+    int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows
+                                   : (row_bytes == 128 ? (f16 ? 1456 : 1376) : (row_bytes == 512 ? 352 : 720));
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
+    g.row_bytes = row_bytes;
     g.smem = (size_t)(SOM_PLAN_MASK_FEATURES + g.n_hot + 1) * row_bytes;  // + the zero row
     return g;
 }
@@ -773,6 +796,10 @@ static int launch_table_any(som_handle* h, bool shadow, const int32_t* indptr, c
         if (g.threads == 768) SOM_TABLE(LayF16, 768);
         if (g.threads == 640) SOM_TABLE(LayF16, 640);
         SOM_TABLE(LayF16, 512);
+    }
+    if (g.R == 16) {
+        if (g.threads == 576) SOM_TABLE(LayF32<16>, 576);
+        SOM_TABLE(LayF32<16>, 512);
     }
     if (g.R == 8) {
         if (g.threads == 1024) SOM_TABLE(LayF32<8>, 1024);

@@ -103,9 +103,10 @@ def test_config2_sampled_rows(som_mod, variant):
     assert np.array_equal(dist2.cpu().numpy().view(np.uint32), g_dist.view(np.uint32))
 
 
-@pytest.mark.parametrize("lane_neurons,threads", [(4, 1024), (4, 768), (8, 512), (8, 768)])
+@pytest.mark.parametrize("lane_neurons,threads", [(4, 1024), (4, 768), (8, 512), (8, 768), (8, 640), (16, 512),
+                                                  (16, 576)])
 def test_row_table_geometries(som_mod, lane_neurons, threads):
-    """Both lane widths of the row-table kernel (32- and 64-neuron ranges) and block sizes,
+    """The lane widths of the row-table kernel (32-, 64- and 128-neuron ranges) and block sizes,
     with permuted feature ids so that the hot features are not the low ids."""
     V, M, n = 30_000, 1_024, 60_000
     W = synth.fill_codebook(V, M, 3, device="cuda")

@@ -96,7 +96,7 @@ def test_top2_config2_sampled_rows(som_mod, variant):
     assert rep.differs_from_oracle < 0.05 * rows.size
 
 
-@pytest.mark.parametrize("lane_neurons,threads", [(4, 1024), (8, 640)])
+@pytest.mark.parametrize("lane_neurons,threads", [(4, 1024), (8, 640), (16, 512)])
 def test_top2_row_table_geometries(som_mod, lane_neurons, threads):
     V, M, n = 30_000, 1_024, 60_000
     W = synth.fill_codebook(V, M, 3, device="cuda")

@@ -30,9 +30,11 @@ def _subset(indptr, indices, rows):
     return out_ptr, out_idx
 
 
-def _run(som_mod, W, V, M, b, two_stage, variant=2):
+def _run(som_mod, W, V, M, b, two_stage, variant=2, lane_neurons=0):
     h = som_mod.Som(V, M, W)
     h.set_option(0, variant)
+    if lane_neurons:
+        h.set_option(3, lane_neurons)
     if two_stage:
         h.set_option(7, 1)
     h.norms()
@@ -117,9 +119,11 @@ def test_two_stage_needs_its_shadow_from_norms(som_mod):
     _check(W.cpu().numpy(), V, M, b, bmu.cpu().numpy(), dist.cpu().numpy(), np.arange(0, n, 13))
 
 
-def _run2(som_mod, W, V, M, b, two_stage, variant=2):
+def _run2(som_mod, W, V, M, b, two_stage, variant=2, lane_neurons=0):
     h = som_mod.Som(V, M, W)
     h.set_option(0, variant)
+    if lane_neurons:
+        h.set_option(3, lane_neurons)
     if two_stage:
         h.set_option(7, 1)
     h.norms()
@@ -242,19 +246,20 @@ def test_two_stage_with_a_reusable_plan(som_mod):
 def test_two_stage_probe_sends_a_smooth_map_to_the_plain_search(som_mod):
     """Units that differ by less than fp16 resolves: the probe (one sample in 256 of a batch of at least
     65536) fails the certificate nearly everywhere and the call takes the plain search on the same plan,
-    whose bits it must then reproduce; a smaller batch is not probed and goes through the exact pass."""
+    whose bits it must then reproduce (the plain search with 8 neurons per lane: the layout whose table
+    matches the first pass's plan); a smaller batch is not probed and goes through the exact pass."""
     V, M, n = 4_000, 1_024, 100_000
     base = synth.fill_codebook(V, 1, 3, device="cuda").view(V, 1)
     noise = synth.fill_codebook(V, M, 8, device="cuda").view(V, M)
     W = (base + 1e-5 * noise).contiguous().view(-1)
     b = synth.sample_csr(n, V, 9.0, 3, device="cuda")
     hs, bs, ds = _run(som_mod, W, V, M, b, True)
-    hp, bp, dp = _run(som_mod, W, V, M, b, False)
+    hp, bp, dp = _run(som_mod, W, V, M, b, False, lane_neurons=8)
     assert hs.last_uncertain() == n
     assert np.array_equal(bs, bp) and np.array_equal(ds.view(np.uint32), dp.view(np.uint32))
     _check(W.cpu().numpy(), V, M, b, bs, ds, np.arange(0, n, 23))
     hs2, out_s = _run2(som_mod, W, V, M, b, True)
-    hp2, out_p = _run2(som_mod, W, V, M, b, False)
+    hp2, out_p = _run2(som_mod, W, V, M, b, False, lane_neurons=8)
     assert hs2.last_uncertain() == n
     for a, c in zip(out_s, out_p):
         assert np.array_equal(a.view(np.uint32), c.view(np.uint32))
