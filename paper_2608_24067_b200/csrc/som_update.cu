@@ -75,7 +75,7 @@ __global__ void k_upd_count(const int32_t* __restrict__ bmu, int64_t n, int rows
 // one thread per sample: its features inside [v0, v1) add 1 to the cell of its best unit
 __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices,
                               int64_t n, const int32_t* __restrict__ bmu, int v0, int v1, int rows, int cols,
-                              const int32_t* __restrict__ hot_slot, float* __restrict__ num_t)
+                              const int32_t* __restrict__ hot_slot, float* __restrict__ num_t, int natural_order)
 {
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n) return;
@@ -83,7 +83,9 @@ __global__ void k_upd_scatter(const int32_t* __restrict__ indptr, const int32_t*
     const int64_t M = (int64_t)rows * cols;
     if ((unsigned)c >= (unsigned)M) return;  // skipped; k_upd_count has noted it
     const int r = c / cols, q = c - r * cols;
-    const int64_t cell_t = (int64_t)q * rows + r;  // transposed cell order
+    // transposed cell order for the routes that blur along the lattice rows first with walks along the
+    // slow index; neuron order for the strip route
+    const int64_t cell_t = natural_order ? (int64_t)c : (int64_t)q * rows + r;
     const int beg = indptr[s], end = indptr[s + 1];
     for (int j = beg; j < end; ++j) {
         const int v = indices[j];
@@ -294,6 +296,71 @@ __device__ __forceinline__ void box_lines(const BT* __restrict__ in, BT* __restr
         const double leave = (i > radius) ? (double)*pl : 0.0;
         sum += enter - leave;
         *pd = (BT)sum;
+    }
+}
+
+// Lattices too large for one plane to be blurred on chip (more than 16384 cells) take the blur in two
+// strip kernels through shared memory instead of seven trips through device memory.  A box pass
+// along one lattice axis never mixes the lines of the other, so a block can take a strip of `tc`
+// adjacent lines over their whole length: k_upd_strip loads the strip as a tile [len][tc] (the walk
+// index slow, the strip's lines fast: consecutive banks for every access of the walks, whatever the
+// radius), runs the three passes between two fp32 buffers with fp64 running sums (the fields between
+// passes are rounded to fp32, as on the device-memory route), and writes once:
+//   first launch  (FINAL = false): input in TRANSPOSED cell order (cell (r, c) at c * rows + r, as the
+//                 scatter leaves it): the walk runs along a lattice row; the result is written in
+//                 neuron order, i.e. the tile is transposed on its way out;
+//   second launch (FINAL = true):  input in neuron order, the walk runs down a lattice column; the
+//                 result is multiplied by the reciprocal blurred denominator and written as the new
+//                 weights of features v0 + plane (a zero reciprocal keeps the prototype).
+// A plane crosses device memory five times in all (scatter, in, out, in, weights out).
+constexpr int STRIP_THREADS = 256;
+typedef float STRIP_BT;  // type of the two tile buffers (fp64 buffers measured twice as slow: fewer blocks per SM)
+
+// in: [plane][len][width]; the block's strip is the `tc` fast indices f0 .. f0 + tc - 1
+template <typename ST, bool TOTALS, bool FINAL>
+__global__ void __launch_bounds__(STRIP_THREADS)
+k_upd_strip(const float* __restrict__ in, float* __restrict__ out, int64_t planes, int len, int width, int radius,
+            int tc, int seg, const double* __restrict__ rden, ST* __restrict__ W, int v0)
+{
+    extern __shared__ __align__(16) unsigned char strip_raw[];
+    __shared__ double tot[STRIP_THREADS];
+    const int pitch = tc | 1;
+    STRIP_BT* A = reinterpret_cast<STRIP_BT*>(strip_raw);
+    STRIP_BT* B = A + (size_t)len * pitch;
+    const int64_t M = (int64_t)len * width;
+    const int groups = (width + tc - 1) / tc;
+    const int64_t items = planes * groups;
+    const int ti = STRIP_THREADS / tc;  // walk positions one sweep of the block's threads covers
+    const int lf = threadIdx.x % tc, li = threadIdx.x / tc;
+    for (int64_t it = blockIdx.x; it < items; it += gridDim.x) {
+        const int64_t plane = it / groups;
+        const int f0 = (int)(it - plane * groups) * tc;
+        const int nf = min(tc, width - f0);
+        const float* src = in + plane * M + f0;
+        for (int i = li; i < len; i += ti) A[i * pitch + lf] = lf < nf ? (STRIP_BT)src[(int64_t)i * width + lf] : (STRIP_BT)0;
+        __syncthreads();
+        box_lines<TOTALS>(A, B, nf, len, 1, pitch, radius, seg, tot);
+        __syncthreads();
+        box_lines<TOTALS>(B, A, nf, len, 1, pitch, radius, seg, tot);
+        __syncthreads();
+        box_lines<TOTALS>(A, B, nf, len, 1, pitch, radius, seg, tot);
+        __syncthreads();
+        if (FINAL) {
+            // (len = rows, width = cols: neuron (i, f0 + lf) is cell i * width + f0 + lf)
+            ST* dst = W + (int64_t)(v0 + plane) * M + f0;
+            const double* rd_base = rden + f0;
+            if (lf < nf)
+                for (int i = li; i < len; i += ti) {
+                    const double rd = rd_base[(int64_t)i * width + lf];
+                    if (rd != 0.0) dst[(int64_t)i * width + lf] = (ST)(float)((double)B[i * pitch + lf] * rd);
+                }
+        } else {
+            // (len = cols, width = rows: line f0 + f is lattice row r, its cells go to r * len + i)
+            float* dst = out + plane * M + (int64_t)f0 * len;
+            for (int f = 0; f < nf; ++f)
+                for (int i = threadIdx.x; i < len; i += STRIP_THREADS) dst[(int64_t)f * len + i] = (float)B[i * pitch + f];
+        }
+        __syncthreads();
     }
 }
 
@@ -552,6 +619,25 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         SOM_CK(h, cudaEventRecord(ev_join, aux));
         st = main_st;
     }
+    // Larger lattices: the strip route wherever a strip of at least four lines over the whole length of
+    // either axis fits in shared memory twice over (fp32); else the passes through device memory.
+    const size_t strip_budget = 200 * 1024;
+    auto strip_width = [&](int len, int width) {
+        // lines per strip: a thread walks a segment of len / (256 / tc) cells, and about 16 cells per thread with
+        // as many blocks per SM as shared memory holds measured best (512 x 512, radius 128: 8 lines per
+        // strip 127 ms, 4: 190 ms, 16: 147 ms, 32: 360 ms for 30 000 planes)
+        int tc = len > 256 ? 8 : (len > 128 ? 16 : 32);
+        while (tc >= 4 && (size_t)len * (tc | 1) * sizeof(STRIP_BT) * 2 > strip_budget) tc /= 2;
+        if (tc >= 4 && tc > width) {  // few lines: all of them in one strip
+            int t2 = 4;
+            while (t2 < width) t2 *= 2;
+            tc = t2 < tc ? t2 : tc;
+        }
+        return tc >= 4 ? tc : 0;
+    };
+    const int strip_tc_r = fused ? 0 : strip_width(cols, rows);  // walk along a lattice row, strip of rows
+    const int strip_tc_c = fused ? 0 : strip_width(rows, cols);  // walk down a lattice column, strip of columns
+    const bool strip = !fused && strip_tc_r >= 4 && strip_tc_c >= 4;
     // ---- numerator, slab by slab ------------------------------------------------------------------
     // (the per-sample masks of the hot features live behind the two slab buffers)
     uint32_t* hot_mask = reinterpret_cast<uint32_t*>(ws + 8 * mb + 2 * som_align_up((size_t)planes_per_slab * M * 4, 256));
@@ -566,7 +652,7 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         else SOM_CK(h, cudaMemsetAsync(slab_a, 0, (size_t)planes * M * 4, st));
         if (n > 0) {
             k_upd_scatter<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols, hot_slot,
-                                                                 slab_a);
+                                                                 slab_a, 0);
             h->launches += 1;
             if (hot_slot) {
                 int ppb = (int)((160 * 1024) / (M * 4));
@@ -609,6 +695,45 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
 #undef SOM_FUSED_T
 #undef SOM_FUSED
             h->launches += 1;
+            SOM_CK(h, cudaGetLastError());
+            continue;
+        }
+        if (strip) {
+            // slab_a holds the counts in transposed cell order: [plane][cols][rows]
+            const int seg_r = STRIP_THREADS / strip_tc_r, seg_c = STRIP_THREADS / strip_tc_c;
+            const size_t sh_r = (size_t)cols * (strip_tc_r | 1) * sizeof(STRIP_BT) * 2;
+            const size_t sh_c = (size_t)rows * (strip_tc_c | 1) * sizeof(STRIP_BT) * 2;
+            const bool tot_r = 2 * radius + 1 > 3 * ((cols + seg_r - 1) / seg_r);
+            const bool tot_c = 2 * radius + 1 > 3 * ((rows + seg_c - 1) / seg_c);
+            const int64_t items_r = planes * ((rows + strip_tc_r - 1) / strip_tc_r);
+            const int64_t items_c = planes * ((cols + strip_tc_c - 1) / strip_tc_c);
+            auto grid_for = [&](size_t sh, int64_t items) {
+                int per_sm = (int)((size_t)220 * 1024 / (sh + 3072));
+                per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+                const int64_t g = (int64_t)h->sm_count * per_sm;
+                return (unsigned)(g < items ? g : items);
+            };
+#define SOM_STRIP(ST_, TOT_, FINAL_, IN_, OUT_, LEN_, WIDTH_, TC_, SEG_, SH_, ITEMS_, W_)                          \
+    do {                                                                                                         \
+        SOM_CK(h, cudaFuncSetAttribute(k_upd_strip<ST_, TOT_, FINAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                       (int)(SH_)));                                                             \
+        k_upd_strip<ST_, TOT_, FINAL_><<<grid_for(SH_, ITEMS_), STRIP_THREADS, SH_, st>>>(                        \
+            IN_, OUT_, planes, LEN_, WIDTH_, radius, TC_, SEG_, rden, W_, v0);                                     \
+    } while (0)
+            float* none_w = nullptr;
+            if (tot_r) SOM_STRIP(float, true, false, slab_a, slab_b, cols, rows, strip_tc_r, seg_r, sh_r, items_r, none_w);
+            else SOM_STRIP(float, false, false, slab_a, slab_b, cols, rows, strip_tc_r, seg_r, sh_r, items_r, none_w);
+            if (h->Wh) {
+                __half* wh = const_cast<__half*>(h->Wh);
+                if (tot_c) SOM_STRIP(__half, true, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wh);
+                else SOM_STRIP(__half, false, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wh);
+            } else {
+                float* wf = const_cast<float*>(h->W);
+                if (tot_c) SOM_STRIP(float, true, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wf);
+                else SOM_STRIP(float, false, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wf);
+            }
+#undef SOM_STRIP
+            h->launches += 2;
             SOM_CK(h, cudaGetLastError());
             continue;
         }

@@ -76,7 +76,13 @@ def _check(got, W_old_stored, V, rows, cols, indptr, indices, bmu, radius, rtol)
     # more than 4096 cells: fp32 plane buffers in shared memory; more than 16384: the passes go
     # through device memory
     (6, 72, 80, 3000, 3), (5, 66, 64, 2000, 70), (4, 300, 20, 1500, 2), (3, 128, 128, 4000, 9),
-    (3, 130, 130, 2000, 4), (2, 2000, 9, 1500, 2)])
+    (3, 130, 130, 2000, 4), (2, 2000, 9, 1500, 2),
+    # the strip route (rows, then column strips, through shared memory): square and oblong lattices,
+    # windows shorter and much longer than a thread's segment, a radius beyond the lattice
+    (2, 512, 512, 20000, 37), (2, 512, 512, 3000, 1), (2, 40, 1000, 3000, 5), (1, 3000, 11, 2000, 3),
+    (2, 256, 300, 5000, 128), (1, 1024, 1024, 50000, 200), (2, 200, 150, 4000, 400),
+    # shapes beyond the strip route's shared memory: the passes through device memory
+    (1, 5000, 8, 3000, 2), (1, 3, 30000, 3000, 6)])
 def test_update_matches_oracle(som_mod, V, rows, cols, n, radius):
     indptr, indices, bmu, W_old = _problem(V * 7 + rows, V, rows, cols, n)
     got = _run(som_mod, W_old, V, rows, cols, indptr, indices, bmu, radius)
@@ -101,6 +107,14 @@ def test_update_in_slabs_equals_single_slab(som_mod):
     slabs = _run(som_mod, W_old, V, rows, cols, indptr, indices, bmu, radius, options=((6, 1),))  # 1 MiB: 32 planes
     assert np.array_equal(whole, slabs)
     _check(whole, W_old, V, rows, cols, indptr, indices, bmu, radius, rtol=1e-6)
+
+
+def test_update_of_fp16_codebook_on_a_large_lattice(som_mod):
+    V, rows, cols, n, radius = 3, 192, 160, 6000, 7
+    indptr, indices, bmu, W_old = _problem(16, V, rows, cols, n)
+    W_old16 = torch.from_numpy(W_old).half().float().numpy()
+    got = _run(som_mod, W_old16, V, rows, cols, indptr, indices, bmu, radius, dtype=torch.float16)
+    _check(got, W_old16, V, rows, cols, indptr, indices, bmu, radius, rtol=2.0 ** -11 + 1e-6)
 
 
 def test_update_of_fp16_codebook(som_mod):
