@@ -368,6 +368,7 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     char* head = nullptr;
     bool begun = false;
     const int* gate = nullptr;  // device-side choice between the two kernels (automatic mode)
+    bool table_hint = true;     // what an earlier call's batch chose
     if (use_table) {
         const size_t head_need = som_plan_head_bytes(h->V, SOM_PLAN_MASK_FEATURES + geom.n_hot, &pb);
         if ((rc = ensure_bytes(h, &h->head, &h->head_bytes, head_need))) return rc;
@@ -393,6 +394,16 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
             // Everything else stays on the device: the kernels of both paths are enqueued, and those of
             // the path not chosen return at once.  The host never waits for the batch.
             gate = counters + SOM_PLAN_USE_TABLE;
+            // The choice also travels to a pinned host word, unwaited for: a later call reads what an
+            // earlier call chose (batches of one stream mostly agree) and gives the launch it expects to
+            // be idle a small grid.  Only the cost of a wrong guess depends on it, never the result.
+            if (!h->host_pair) {
+                SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
+                h->host_pair[2] = 1;
+            }
+            table_hint = *reinterpret_cast<volatile int32_t*>(h->host_pair + 2) != 0;
+            SOM_CK(h, cudaMemcpyAsync(h->host_pair + 2, counters + SOM_PLAN_USE_TABLE, sizeof(int32_t),
+                                      cudaMemcpyDeviceToHost, st));
         }
     }
 
@@ -441,8 +452,11 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (gate) {
             // direct-load path on the same key arrays (indexed by sample there): runs when the choice is 0
             h->gate_want = 0;
-            if ((rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, nullptr, st))) return rc;
+            h->gate_small_grid = table_hint ? 1 : 0;
+            rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, nullptr, st);
+            h->gate_small_grid = 0;
             h->gate_want = 1;
+            if (rc) return rc;
         }
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
         if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, false, d_bmu,

@@ -111,7 +111,9 @@ template <> struct Seg<__half, 8> {
 // Section 7): the gather-sum becomes a gather-multiply, score = ||w||^2/2 - sum_k x_k * w[idx_k].
 // TILES: a warp covers TILES adjacent tiles of 32*VEC neurons per sample, so that the feature
 // broadcast, the row address and the shuffle argmin are paid once per TILES tiles.
-template <int VEC, int TILES, bool TOP2, typename ST, bool VALUED = false>
+// WALK: the block walks the sample groups blockIdx.x, blockIdx.x + gridDim.x, ... instead of taking one
+// (launches that mostly return at once, or whose sample count only the device knows, come with a small grid).
+template <int VEC, int TILES, bool TOP2, typename ST, bool VALUED = false, bool WALK = false>
 __global__ void __launch_bounds__(DIRECT_THREADS, 2)
 k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t M, uint32_t row_bytes,
              const int32_t* __restrict__ indptr, const int32_t* __restrict__ indices, int64_t n,
@@ -120,8 +122,10 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
              const float* __restrict__ values = nullptr, const int* __restrict__ gate = nullptr, int gate_want = 0,
              int sample_groups = 0, const int* __restrict__ n_dev = nullptr)
 {
-    if (som_gated_off(gate, gate_want)) return;
-    if (n_dev) n = *n_dev;  // length of a sample list that lives on the device
+    if constexpr (WALK) {  // (gates and device-side sample counts come with the walking form only)
+        if (som_gated_off(gate, gate_want)) return;
+        if (n_dev) n = *n_dev;  // length of a sample list that lives on the device
+    }
     constexpr int TILE = 32 * VEC;  // neurons per tile
     // features whose row segments are in flight together (fp16 rows are half as long: twice as many)
     constexpr int FEATS = sizeof(ST) == 2 ? 8 : 4;
@@ -145,9 +149,9 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
     // byte address of the lane's first neuron in feature row 0; row v is row_bytes * v further on
     const char* W_lane = reinterpret_cast<const char*>(W + (live[0] ? i0 : 0));
 
-    // A block takes the sample groups blockIdx.x, blockIdx.x + gridDim.x, ...: one group per block in the
-    // plain launch; a gated launch (which mostly returns at once) comes with a small grid instead.
-    for (int bx = blockIdx.x; bx < sample_groups; bx += gridDim.x) {
+    int bx = blockIdx.x;
+    if (WALK && bx >= sample_groups) return;
+    do {
     const int64_t s0 = ((int64_t)bx * DIRECT_WARPS + warp) * DIRECT_SAMPLES_PER_WARP;
     const int n_mine = (int)min((int64_t)DIRECT_SAMPLES_PER_WARP, n - s0);
     if (n_mine <= 0) break;  // (later groups lie further on)
@@ -301,7 +305,7 @@ k_bmu_direct(const ST* __restrict__ W, const float* __restrict__ hnorm, int64_t 
         first = next;
         first_x = next_x;
     }
-    }
+    } while (WALK && (bx += (int)gridDim.x) < sample_groups);
 }
 
 // One thread per sample: unpack the winner and recompute its full squared distance
@@ -381,21 +385,19 @@ template <int VEC, int TILES, typename ST>
 static void launch_direct(dim3 grid, cudaStream_t st, const ST* W, som_handle* h, const int32_t* indptr,
                           const int32_t* indices, int64_t n, unsigned long long* keys,
                           unsigned long long* keys2, int64_t neuron_off, const int32_t* sample_list,
-                          const float* values, int sample_groups)
+                          const float* values, int sample_groups, bool walk)
 {
     const uint32_t row_bytes = (uint32_t)(h->M * (int64_t)sizeof(ST));
-    if (values)
-        k_bmu_direct<VEC, TILES, false, ST, true><<<grid, DIRECT_THREADS, 0, st>>>(
-            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, nullptr, values, nullptr, 0,
-            sample_groups);
-    else if (keys2)
-        k_bmu_direct<VEC, TILES, true, ST><<<grid, DIRECT_THREADS, 0, st>>>(
-            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, keys2, neuron_off, sample_list, nullptr,
-            h->gate, h->gate_want, sample_groups, h->list_len_dev);
-    else
-        k_bmu_direct<VEC, TILES, false, ST><<<grid, DIRECT_THREADS, 0, st>>>(
-            W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, nullptr, neuron_off, sample_list, nullptr,
-            h->gate, h->gate_want, sample_groups, h->list_len_dev);
+#define SOM_DIRECT_GO(TOP2_, VALUED_, WALK_, K2_, SL_, VAL_)                                                      \
+    k_bmu_direct<VEC, TILES, TOP2_, ST, VALUED_, WALK_><<<grid, DIRECT_THREADS, 0, st>>>(                         \
+        W, h->hnorm, h->M, row_bytes, indptr, indices, n, keys, K2_, neuron_off, SL_, VAL_, h->gate, h->gate_want, \
+        sample_groups, h->list_len_dev)
+    if (values) SOM_DIRECT_GO(false, true, false, nullptr, nullptr, values);
+    else if (keys2 && walk) SOM_DIRECT_GO(true, false, true, keys2, sample_list, nullptr);
+    else if (keys2) SOM_DIRECT_GO(true, false, false, keys2, sample_list, nullptr);
+    else if (walk) SOM_DIRECT_GO(false, false, true, nullptr, sample_list, nullptr);
+    else SOM_DIRECT_GO(false, false, false, nullptr, sample_list, nullptr);
+#undef SOM_DIRECT_GO
 }
 
 template <typename ST>
@@ -417,11 +419,14 @@ static int launch_direct_any(som_handle* h, const ST* W, const int32_t* indptr, 
         // a gated launch returns at once on most calls: keep it to about 2048 blocks, each of which walks
         // several sample groups when it does run
         int64_t gx_launch = gx;
-        if ((h->gate || h->list_len_dev) && gx * ny > 2048) gx_launch = 2048 / ny > 1 ? 2048 / ny : 1;
+        // gated launches and launches over a device-side list take the walking form of the kernel; those
+        // expected to be idle, and the lists (short), come with a small grid
+        const bool walk = (h->gate || h->list_len_dev) && !values;
+        if ((h->gate_small_grid || h->list_len_dev) && walk && gx * ny > 2048) gx_launch = 2048 / ny > 1 ? 2048 / ny : 1;
         dim3 grid((unsigned)gx_launch, (unsigned)ny);
         const int64_t neuron_off = y0 * neurons_per_block;
 #define SOM_DIRECT(VEC_, TILES_) \
-    launch_direct<VEC_, TILES_, ST>(grid, st, W, h, indptr, indices, n, keys, keys2, neuron_off, sample_list, values, (int)gx)
+    launch_direct<VEC_, TILES_, ST>(grid, st, W, h, indptr, indices, n, keys, keys2, neuron_off, sample_list, values, (int)gx, walk)
         if constexpr (sizeof(ST) == 2) {
             if (vec == 8 && tiles == 2) SOM_DIRECT(8, 2);
             else if (vec == 8) SOM_DIRECT(8, 1);

@@ -71,6 +71,7 @@ struct som_handle {
     // kernels of both search paths, and a kernel returns at once unless *gate == gate_want.
     const int* gate;       // device, nullptr = no gate
     int gate_want;
+    int gate_small_grid;   // the gated launch in hand is expected to return at once: give it a small grid
     // Length of a sample list that only the device knows (the samples that do not fit a slot of the
     // row-table plan): while set, the direct-load kernel and its finalisation read their sample count
     // from it and are launched with small grids that walk the list.
