@@ -23,8 +23,7 @@
  *     the choice between the two search kernels all stay on the device (the kernels of both
  *     paths are enqueued; those of the path not chosen return at once).  Exceptions: growing
  *     the handle's workspace (first call, or a larger batch than any before) allocates device
- *     memory, which may synchronise the device once; and the two-stage search (option 7),
- *     which reads list lengths back.
+ *     memory, which may synchronise the device once.
  *   - Thread safety: one handle must not be used from two host threads at once, and two
  *     calls on the same handle must not overlap on the GPU (they share the workspace);
  *     issue them on one stream or order the streams yourself.
@@ -147,8 +146,7 @@ int som_bmu2(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, i
  *                     storage type at this moment.
  *   som_bmu_planned   som_bmu for the plan's batch: same outputs (bit-identical to som_bmu's on the same
  *                     batch with the same options), but only enqueues work on `stream` (no host
- *                     synchronisation, no allocation), except with the two-stage search (option 7), which
- *                     it takes like som_bmu and which synchronises the stream once.
+ *                     synchronisation, no allocation); it takes the two-stage search (option 7) like som_bmu.
  *                     Two searches with the same plan must not overlap on the GPU.
  *   som_plan_destroy  frees the plan (NULL is accepted); destroy plans before their handle.
  */
@@ -291,32 +289,38 @@ int som_last_cuda_error(const som_handle* h);
  *   out_ms[0] som_norms total, out_ms[1] som_bmu total, out_ms[2] som_bmu plan phase,
  *   out_ms[3] som_bmu search kernel(s), out_ms[4] som_bmu finalize.
  * som_launch_count returns how many kernels this handle has launched since creation.
- * som_set_option tunes kernel selection: key 0 = search kernel variant (0 auto, 1 direct-load
- * kernel, 2 shared-memory row-table kernel where M % 4 == 0 and V <= 65536); key 1 = hot rows kept in shared
- * memory by the row-table kernel (0 = default); key 2 = its block size (0 = default, 512, 640, 768, 896, 1024);
- * key 3 = neurons per lane there (0 = default: the widest that divides M; fp32 storage: 4, 8, 16, where 8 needs
- * M % 64 == 0 and 16 M % 128 == 0; fp16 storage: 8, 16, where 16 needs M % 128 == 0); key 4 = sample parts per
- * neuron range there (0 = default); key 5 = in automatic selection, the least percentage of the batch's
- * feature instances that the row table's features must cover for the row-table kernel to be taken
- * (0 = default 60; batches below it go to the direct-load kernel); key 6 = workspace budget of som_update's
- * slab buffers in MiB (0 = default 4096); key 7 = two-stage search for fp32 storage (0 = off, the default;
- * 1 = on): som_norms then also keeps an fp16 copy of the codebook (V*M*2 more bytes of device memory,
- * allocated by this call, which fails with SOM_ERR_CUDA if they cannot be had), the largest |weight|, the
- * largest ||w||^2 and whether any weight is negative; som_bmu ranks the neurons by a first pass over that
- * copy, keeps the result for every sample whose two best first-pass scores are further apart than a bound on
- * what the fp16 rounding and the fp32 summation can change (then the best unit of the exact weights is
- * provably the same one; the bound is tighter when no weight is negative), and searches the other samples
- * again with the fp32 weights.  som_bmu2 does the same with the three best first-pass scores (both units
- * and their order certified).  Reported distances always come from the fp32 weights.
- * It pays on maps whose units are distinct at fp16 resolution (random initialisation, small final radius); on
- * a map that a wide blur has just smoothed most samples fail the certificate.  A batch of at least 65536
- * samples is therefore probed first (one sample in 256, chosen by sample index; one more stream
- * synchronisation): if more than a fifth of those fail, the call runs the plain search instead (on the
- * same plan, i.e. with 8 neurons per lane: bit-identical to a plain call with key 3 = 8).
- * Needs M % 128 == 0 and the row-table kernel.  A two-stage call synchronises the
- * stream a second time (it reads the length of the second pass's list back).  som_last_uncertain returns how
- * many samples the last two-stage search sent to its second pass (all of them when the probe chose the plain
- * search).
+ * som_set_option sets a per-handle option (SOM_ERR_INVALID_ARG for an unknown key or value):
+ *   key 0  search kernel: 0 automatic (default), 1 direct-load kernel, 2 shared-memory row-table kernel (where
+ *          M % 4 == 0 and V <= 65536).
+ *   key 5  automatic selection: least percentage of the batch's feature instances that the row table's
+ *          features must cover for the row-table kernel to be taken (0 = default 60; batches below it go to
+ *          the direct-load kernel).
+ *   key 6  workspace budget of som_update's slab buffers in MiB (0 = default 4096).
+ *   key 7  two-stage search for fp32 storage (0 = off, the default; 1 = on): som_norms then also keeps an fp16
+ *          copy of the codebook (V*M*2 more bytes of device memory, allocated by this call, which fails with
+ *          SOM_ERR_CUDA if they cannot be had), the largest |weight|, the largest ||w||^2 and whether any weight
+ *          is negative; som_bmu ranks the neurons by a first pass over that copy, keeps the result for every
+ *          sample whose two best first-pass scores are further apart than a bound on what the fp16 rounding and
+ *          the fp32 summation can change (then the best unit of the exact weights is provably the same one; the
+ *          bound is tighter when no weight is negative), and searches the other samples again with the fp32
+ *          weights.  som_bmu2 does the same with the three best first-pass scores (both units and their order
+ *          certified).  Reported distances always come from the fp32 weights.  It pays on maps whose units are
+ *          distinct at fp16 resolution (random initialisation, small final radius); on a map that a wide blur
+ *          has just smoothed most samples fail the certificate.  A batch of at least 65536 samples is therefore
+ *          probed first (one sample in 256, chosen by sample index): if more
+ *          than a fifth of those fail, the call runs the plain search instead (on the same plan, i.e. with 8
+ *          neurons per lane: bit-identical to a plain call with key 3 = 8).  Needs M % 128 == 0 and the
+ *          row-table kernel.  A two-stage call only enqueues, like any other: the probe's verdict, the choice
+ *          between the two-stage path and the plain search and the length of the second pass's list all stay on
+ *          the device (the kernels of both paths are enqueued; those of the path not taken return at once; the
+ *          second pass is run by the direct-load kernel, which reads the list's length on the device).
+ *          som_last_uncertain returns how many samples the last two-stage search sent to its second pass (all
+ *          of them when the probe chose the plain search); the figure travels back unwaited for and is valid
+ *          once the call's stream has been synchronised.
+ *   keys 1 to 4 are geometry tunables of the row-table kernel for benchmarking (hot rows in shared memory, block
+ *          size, neurons per lane, sample parts per neuron range; 0 = the measured default): described in
+ *          paper_2608_24067_b200/csrc/som_tuning.h.  Callers need not touch them; a plan (som_plan_create) is
+ *          tied to their values at its creation.
  */
 /*
  * som_measure_fadd_peak - measure the device's FP32 add rate (no counterpart in the paper: the

@@ -60,7 +60,7 @@ struct GateScope {
     GateScope(som_handle* h_, const int* gate) : h(h_)
     {
         h->gate = gate;
-        h->gate_want = 1;
+        h->gate_want = SOM_GATE_TABLE;
     }
     ~GateScope()
     {
@@ -199,39 +199,42 @@ static int rare_pass(som_handle* h, const int32_t* indptr, const int32_t* indice
 
 // The two-stage search on a batch whose plan (slots in ws, table features in head) is ready: first
 // pass over the fp16 shadow keeping the two (som_bmu2: three) best units, certificate, exact fp32
-// pass for the samples it leaves open.  Synchronises the stream once (length of that list), twice when
-// the batch is large enough to be probed first.
-static int two_stage_passes(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
-                            char* ws, const SomPlanBuffers& pb, int n_hot, int32_t* bmu, float* dist,
-                            int32_t* bmu2, float* dist2, cudaStream_t st)
+// pass for the samples it leaves open.  Everything is enqueued; nothing is read back.  `gate` is the
+// device word that says which path this batch takes: the probe and the decision kernel may raise it from
+// 1 (row-table kernel) to 2 (row-table kernel, two-stage search); the kernels enqueued here for the
+// two-stage path run only then, and the caller enqueues the plain search for the other case.
+// Key arrays (keys, keys2, keys3) must have been cleared by the caller.
+static int two_stage_enqueue(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
+                             char* ws, const SomPlanBuffers& pb, int n_hot, int32_t* bmu, float* dist,
+                             int32_t* bmu2, float* dist2, cudaStream_t st)
 {
     int rc = SOM_OK;
     const bool top2 = bmu2 != nullptr;
-    const size_t kb = (size_t)(n + 16) * sizeof(unsigned long long);
     int* counters = reinterpret_cast<int*>(head + pb.n_slots);
-    SOM_CK(h, cudaMemsetAsync(ws + pb.keys, 0xFF, kb, st));
-    SOM_CK(h, cudaMemsetAsync(ws + pb.keys2, 0xFF, kb, st));
-    if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
-    SOM_CK(h, cudaMemsetAsync(counters + 3, 0, sizeof(int), st));                   // search unit counter
-    SOM_CK(h, cudaMemsetAsync(counters + SOM_PLAN_UNCERTAIN, 0, sizeof(int), st));  // length of the list
     int32_t* uncertain = reinterpret_cast<int32_t*>(ws + pb.uncertain);
     int* n_unc_dev = counters + SOM_PLAN_UNCERTAIN;
-    const SomTableGeom exact = som_table_geometry(h, false);
+    SOM_CK(h, cudaMemsetAsync(counters + 3, 0, sizeof(int), st));   // search unit counter
+    SOM_CK(h, cudaMemsetAsync(n_unc_dev, 0, sizeof(int), st));      // length of the uncertain list
 
     // Probe.  On a map whose neighbouring units differ by less than fp16 resolves (one that a wide
     // blur has just smoothed) most samples fail the certificate, and a first pass over the whole
     // batch is wasted.  So one sample in SOM_PROBE_STRIDE goes through first pass and certificate
-    // first; if more than a fifth of those fail, the batch takes the plain fp32 search.
-    if (n >= SOM_PROBE_MIN_BATCH && exact.n_hot == n_hot) {
-        const int64_t n_probe = (n + SOM_PROBE_STRIDE - 1) / SOM_PROBE_STRIDE;
+    // first (count only); the decision kernel sends the batch to the plain fp32 search if more than a
+    // fifth of those fail.
+    int n_probe = 0;
+    h->gate_want = SOM_GATE_TABLE;
+    if (n >= SOM_PROBE_MIN_BATCH) {
+        n_probe = (int)((n + SOM_PROBE_STRIDE - 1) / SOM_PROBE_STRIDE);
         const size_t pkb = (size_t)(n_probe + 16) * sizeof(unsigned long long);
         SomPlanBuffers pp = pb;
         pp.slots = pb.slots2;
         pp.order = pb.uncertain;
         pp.keys = pb.ukeys;
-        pp.keys2 = pb.ukeys2;  // (keys3 is not in use yet: its head serves the probe)
+        pp.keys2 = pb.ukeys2;
+        pp.keys3 = pb.rare_keys;  // (free until the rare pass at the end of the call)
         SOM_CK(h, cudaMemsetAsync(ws + pp.keys, 0xFF, pkb, st));
         SOM_CK(h, cudaMemsetAsync(ws + pp.keys2, 0xFF, pkb, st));
+        if (top2) SOM_CK(h, cudaMemsetAsync(ws + pp.keys3, 0xFF, pkb, st));
         if ((rc = som_launch_probe_gather(h, n, ws, pb, st))) return rc;
         if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_probe, st))) return rc;
         // (enough sample parts per neuron range that the short launch still occupies every SM)
@@ -245,84 +248,35 @@ static int two_stage_passes(som_handle* h, const int32_t* indptr, const int32_t*
         if ((rc = som_launch_certify(h, indptr, indices, n_probe, ws, pp, top2, true, nullptr, nullptr, nullptr,
                                      nullptr, nullptr, n_unc_dev, st)))
             return rc;
-        SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-        SOM_CK(h, cudaStreamSynchronize(st));
-        const int64_t probe_unc = h->host_pair[3];
-        SOM_CK(h, cudaMemsetAsync(counters + 3, 0, sizeof(int), st));
-        SOM_CK(h, cudaMemsetAsync(n_unc_dev, 0, sizeof(int), st));
-        if (probe_unc * 5 > n_probe) {
-            // plain search on the same plan (keys and keys2 are still empty)
-            h->last_uncertain = n;
-            if ((rc = som_launch_bmu_table(h, false, indptr, indices, n, head, ws, pb, n_hot, top2 ? 2 : 1, st))) return rc;
-            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-            if ((rc = som_launch_finalize_sorted(h, indptr, indices, n, ws, pb, false, bmu, dist, st))) return rc;
-            if (top2 && (rc = som_launch_finalize_sorted(h, indptr, indices, n, ws, pb, true, bmu2, dist2, st)))
-                return rc;
-            return SOM_OK;
-        }
-        if (top2) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
     }
+    if ((rc = som_launch_two_stage_decide(h, head, pb, n_probe, n, st))) return rc;
+    SOM_CK(h, cudaMemsetAsync(counters + 3, 0, sizeof(int), st));
 
+    // ---- the two-stage path proper: runs when the gate word is 2 -------------------------------------
+    h->gate_want = SOM_GATE_TABLE_TS;
     if ((rc = som_launch_bmu_table(h, true, indptr, indices, n, head, ws, pb, n_hot, top2 ? 3 : 2, st))) return rc;
     // certificate; certain samples are finalised, the others listed
     if ((rc = som_launch_certify(h, indptr, indices, n, ws, pb, top2, false, bmu, dist, bmu2, dist2, uncertain,
                                  n_unc_dev, st)))
         return rc;
-    SOM_CK(h, cudaMemcpyAsync(h->host_pair + 3, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    SOM_CK(h, cudaStreamSynchronize(st));
-    const int64_t n_unc = h->host_pair[3];
-    h->last_uncertain = n_unc;
-    if (n_unc > 0) {
-        // exact pass over the listed samples: fp32 weights, all neurons.  With enough of
-        // them the row-table kernel runs again on their compacted slots (same plan: both
-        // layouts hold the same number of hot rows), else the direct-load kernel.
-        unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
-        unsigned long long* ukeys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.ukeys2) : nullptr;
-        const int64_t units = ((h->M + exact.T - 1) / exact.T) * som_table_default_parts(n_unc, exact.T, exact.row_bytes);
-        const size_t ub = (size_t)(n_unc + 16) * sizeof(unsigned long long);
-        SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, ub, st));
-        if (top2) SOM_CK(h, cudaMemsetAsync(ukeys2, 0xFF, ub, st));
-        if (exact.n_hot == n_hot && units >= 2 * (int64_t)h->sm_count) {
-            SomPlanBuffers pe = pb;
-            pe.slots = pb.slots2;
-            pe.order = pb.uncertain;  // the list holds the sample index of every compacted slot
-            pe.keys = pb.ukeys;
-            pe.keys2 = pb.ukeys2;
-            SOM_CK(h, cudaMemsetAsync(reinterpret_cast<int*>(head + pb.n_slots) + 3, 0, sizeof(int), st));
-            if ((rc = som_launch_pad_slots(h, ws, pb.slots2, n_unc, st))) return rc;
-            if ((rc = som_launch_bmu_table(h, false, indptr, indices, n_unc, head, ws, pe, exact.n_hot, top2 ? 2 : 1, st)))
-                return rc;
-            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-            if ((rc = som_launch_finalize_sorted(h, indptr, indices, n_unc, ws, pe, false, bmu,
-                                                 dist, st)))
-                return rc;
-            if (top2 && (rc = som_launch_finalize_sorted(h, indptr, indices, n_unc, ws, pe, true, bmu2,
-                                                         dist2, st)))
-                return rc;
-        } else {
-            if ((rc = som_launch_bmu_direct(h, indptr, indices, n_unc, ukeys, ukeys2, uncertain, st)))
-                return rc;
-            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
-            if ((rc = som_launch_finalize(h, indptr, indices, n_unc, ukeys, bmu, dist, uncertain,
-                                          st)))
-                return rc;
-            if (top2 && (rc = som_launch_finalize(h, indptr, indices, n_unc, ukeys2, bmu2, dist2,
-                                                  uncertain, st)))
-                return rc;
-        }
-    } else if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) {
-        return rc;
-    }
+    // exact pass over the listed samples: fp32 weights, all neurons, by the direct-load kernel, which reads
+    // the length of the list on the device
+    unsigned long long* ukeys = reinterpret_cast<unsigned long long*>(ws + pb.ukeys);
+    unsigned long long* ukeys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.ukeys2) : nullptr;
+    const size_t ub = (size_t)(n + 16) * sizeof(unsigned long long);
+    SOM_CK(h, cudaMemsetAsync(ukeys, 0xFF, ub, st));
+    if (top2) SOM_CK(h, cudaMemsetAsync(ukeys2, 0xFF, ub, st));
+    h->list_len_dev = n_unc_dev;
+    rc = som_launch_bmu_direct(h, indptr, indices, n, ukeys, ukeys2, uncertain, st);
+    if (!rc) rc = som_launch_finalize(h, indptr, indices, n, ukeys, bmu, dist, uncertain, st);
+    if (!rc && top2) rc = som_launch_finalize(h, indptr, indices, n, ukeys2, bmu2, dist2, uncertain, st);
+    h->list_len_dev = nullptr;
+    if (rc) return rc;
+    // what som_last_uncertain reports travels to pinned host words, unwaited for
+    SOM_CK(h, cudaMemcpyAsync(h->host_pair, counters + SOM_PLAN_REPORT, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SOM_CK(h, cudaMemcpyAsync(h->host_pair + 1, n_unc_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    h->last_uncertain = -1;  // (read from the pinned words on demand)
     return SOM_OK;
-}
-
-static int two_stage_search(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n, char* head,
-                            char* ws, const SomPlanBuffers& pb, int n_hot, int32_t* bmu, float* dist,
-                            int32_t* bmu2, float* dist2, cudaStream_t st)
-{
-    int rc = two_stage_passes(h, indptr, indices, n, head, ws, pb, n_hot, bmu, dist, bmu2, dist2, st);
-    if (!rc) rc = rare_pass(h, indptr, indices, n, head, ws, pb, bmu, dist, bmu2, dist2, st);
-    return rc;
 }
 
 // The search behind som_bmu (d_bmu2 == nullptr) and som_bmu2 (both second-best outputs given).
@@ -367,40 +321,36 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
     SomPlanBuffers pb;
     char* head = nullptr;
     bool begun = false;
-    const int* gate = nullptr;  // device-side choice between the two kernels (automatic mode)
-    bool table_hint = true;     // what an earlier call's batch chose
+    const int* gate = nullptr;  // device-side choice between the search paths
+    bool table_hint = true;     // what an earlier call's batch chose (automatic mode)
     if (use_table) {
         const size_t head_need = som_plan_head_bytes(h->V, SOM_PLAN_MASK_FEATURES + geom.n_hot, &pb);
         if ((rc = ensure_bytes(h, &h->head, &h->head_bytes, head_need))) return rc;
         head = reinterpret_cast<char*>(h->head);
+        if (!h->host_pair) {
+            SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
+            h->host_pair[0] = h->host_pair[1] = 0;
+            h->host_pair[2] = 1;
+        }
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_BEGIN, st))) return rc;
         begun = true;
-        // The selection phase of the plan: feature histogram, choice of the table's features and, in
-        // automatic mode, of the kernel (the table must serve enough of the batch's feature instances).
-        if ((rc = som_launch_plan_select(h, d_indptr, d_indices, n_samples, head, pb, SOM_PLAN_MASK_FEATURES,
-                                         geom.n_hot, st)))
-            return rc;
+        // The selection phase of the plan: feature histogram, choice of the table's features and of the
+        // kernel (in automatic mode the table must serve enough of the batch's feature instances; a forced
+        // row-table kernel always gets 1), written to the gate word on the device.
+        const int64_t saved_cover = h->opt_cover;
+        if (h->opt_variant == 2) h->opt_cover = -1;  // (coverage threshold of zero percent)
+        rc = som_launch_plan_select(h, d_indptr, d_indices, n_samples, head, pb, SOM_PLAN_MASK_FEATURES, geom.n_hot, st);
+        h->opt_cover = saved_cover;
+        if (rc) return rc;
         const int32_t* counters = reinterpret_cast<const int32_t*>(head + pb.n_slots);
-        // (pinned words for the read-backs of the two-stage search)
-        if (two_stage_ok && !h->host_pair)
-            SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
-        if (h->opt_variant == 0 && two_stage_ok) {
-            // the two-stage search synchronises anyway: it reads the choice back
-            SOM_CK(h, cudaMemcpyAsync(h->host_pair + 2, counters + SOM_PLAN_USE_TABLE, sizeof(int32_t),
-                                      cudaMemcpyDeviceToHost, st));
-            SOM_CK(h, cudaStreamSynchronize(st));
-            if (h->host_pair[2] == 0) use_table = false;
-        } else if (h->opt_variant == 0) {
-            // Everything else stays on the device: the kernels of both paths are enqueued, and those of
-            // the path not chosen return at once.  The host never waits for the batch.
-            gate = counters + SOM_PLAN_USE_TABLE;
+        // Everything stays on the device: the kernels of every path are enqueued, and those of the paths
+        // not chosen return at once.  The host never waits for the batch.  (A forced row-table kernel
+        // without the two-stage search has one path only and needs no gate.)
+        if (h->opt_variant == 0 || two_stage_ok) gate = counters + SOM_PLAN_USE_TABLE;
+        if (h->opt_variant == 0) {
             // The choice also travels to a pinned host word, unwaited for: a later call reads what an
             // earlier call chose (batches of one stream mostly agree) and gives the launch it expects to
             // be idle a small grid.  Only the cost of a wrong guess depends on it, never the result.
-            if (!h->host_pair) {
-                SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
-                h->host_pair[2] = 1;
-            }
             table_hint = *reinterpret_cast<volatile int32_t*>(h->host_pair + 2) != 0;
             SOM_CK(h, cudaMemcpyAsync(h->host_pair + 2, counters + SOM_PLAN_USE_TABLE, sizeof(int32_t),
                                       cudaMemcpyDeviceToHost, st));
@@ -422,53 +372,51 @@ static int bmu_impl(som_handle* h, const int32_t* d_indptr, const int32_t* d_ind
         if (top2 &&
             (rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys2, d_bmu2, d_dist2, nullptr, st)))
             return rc;
-    } else if (two_stage_ok) {
-        const size_t need = som_plan_workspace_bytes(n_samples, &pb);
-        if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
-        char* ws = reinterpret_cast<char*>(h->ws);
-        if ((rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, head, ws, pb, SOM_PLAN_MASK_FEATURES,
-                                       geom.n_hot, st)))
-            return rc;
-        if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-        if ((rc = two_stage_search(h, d_indptr, d_indices, n_samples, head, ws, pb, geom.n_hot, d_bmu, d_min_dist,
-                                   d_bmu2, d_dist2, st)))
-            return rc;
     } else {
         const size_t need = som_plan_workspace_bytes(n_samples, &pb);
         if ((rc = ensure_bytes(h, &h->ws, &h->ws_bytes, need))) return rc;
         char* ws = reinterpret_cast<char*>(h->ws);
         unsigned long long* keys = reinterpret_cast<unsigned long long*>(ws + pb.keys);
-        unsigned long long* keys2 = top2 ? reinterpret_cast<unsigned long long*>(ws + pb.keys2) : nullptr;
-        SOM_CK(h, cudaMemsetAsync(keys, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
-        if (top2) SOM_CK(h, cudaMemsetAsync(keys2, 0xFF, (size_t)(n_samples + 16) * sizeof(unsigned long long), st));
-        GateScope scope(h, gate);  // row-table path: runs when the choice is 1 (or there is no gate)
+        unsigned long long* keys2 = reinterpret_cast<unsigned long long*>(ws + pb.keys2);
+        const size_t kb = (size_t)(n_samples + 16) * sizeof(unsigned long long);
+        SOM_CK(h, cudaMemsetAsync(keys, 0xFF, kb, st));
+        if (top2 || two_stage_ok) SOM_CK(h, cudaMemsetAsync(keys2, 0xFF, kb, st));
+        if (top2 && two_stage_ok) SOM_CK(h, cudaMemsetAsync(ws + pb.keys3, 0xFF, kb, st));
+        GateScope scope(h, gate);  // the plan: runs when a row-table path is chosen (or there is no gate)
         if ((rc = som_launch_plan_sort(h, d_indptr, d_indices, n_samples, head, ws, pb, SOM_PLAN_MASK_FEATURES,
                                        geom.n_hot, st)))
             return rc;
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
+        if (two_stage_ok &&
+            (rc = two_stage_enqueue(h, d_indptr, d_indices, n_samples, head, ws, pb, geom.n_hot, d_bmu, d_min_dist,
+                                    d_bmu2, d_dist2, st)))
+            return rc;
+        // plain row-table search (with the two-stage search enabled: only when the gate word stayed at 1)
+        h->gate_want = two_stage_ok ? SOM_GATE_TABLE_PLAIN : SOM_GATE_TABLE;
         if ((rc = som_launch_bmu_table(h, false, d_indptr, d_indices, n_samples, head, ws, pb, geom.n_hot,
                                        top2 ? 2 : 1, st)))
             return rc;
-        if (gate) {
+        if (gate && h->opt_variant == 0) {
             // direct-load path on the same key arrays (indexed by sample there): runs when the choice is 0
-            h->gate_want = 0;
+            h->gate_want = SOM_GATE_DIRECT;
             h->gate_small_grid = table_hint ? 1 : 0;
-            rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, keys2, nullptr, st);
+            rc = som_launch_bmu_direct(h, d_indptr, d_indices, n_samples, keys, top2 ? keys2 : nullptr, nullptr, st);
             h->gate_small_grid = 0;
-            h->gate_want = 1;
             if (rc) return rc;
         }
         if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+        h->gate_want = two_stage_ok ? SOM_GATE_TABLE_PLAIN : SOM_GATE_TABLE;
         if ((rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, false, d_bmu,
                                              d_min_dist, st)))
             return rc;
         if (top2 && (rc = som_launch_finalize_sorted(h, d_indptr, d_indices, n_samples, ws, pb, true, d_bmu2,
                                                      d_dist2, st)))
             return rc;
+        h->gate_want = SOM_GATE_TABLE;
         if ((rc = rare_pass(h, d_indptr, d_indices, n_samples, head, ws, pb, d_bmu, d_min_dist, d_bmu2, d_dist2, st)))
             return rc;
-        if (gate) {
-            h->gate_want = 0;
+        if (gate && h->opt_variant == 0) {
+            h->gate_want = SOM_GATE_DIRECT;
             if ((rc = som_launch_finalize(h, d_indptr, d_indices, n_samples, keys, d_bmu, d_min_dist, nullptr, st)))
                 return rc;
             if (top2 &&
@@ -645,9 +593,36 @@ int som_bmu_planned(som_handle* h, som_plan* p, int32_t* d_bmu, float* d_min_dis
         // two-stage search (option 7), as in som_bmu, when the shadow's layout holds the same table
         if (h->opt_two_stage == 1 && h->shadow && h->shadow_valid && !h->Wh && h->M % 128 == 0 &&
             som_table_geometry(h, true).n_hot == p->n_hot) {
+            // as in som_bmu: both the two-stage path and the plain search are enqueued, the gate word (set
+            // to 1 here: this plan takes the row-table kernel) is raised to 2 on the device unless the probe
+            // sends the batch to the plain search
+            static const int32_t one = 1;
+            int* counters = reinterpret_cast<int*>(p->head + p->pb.n_slots);
+            if (!h->host_pair) {
+                SOM_CK(h, cudaMallocHost(reinterpret_cast<void**>(&h->host_pair), 4 * sizeof(int32_t)));
+                h->host_pair[0] = h->host_pair[1] = 0;
+                h->host_pair[2] = 1;
+            }
+            SOM_CK(h, cudaMemcpyAsync(counters + SOM_PLAN_USE_TABLE, &one, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+            const size_t kb = (size_t)(p->n + 16) * sizeof(unsigned long long);
+            SOM_CK(h, cudaMemsetAsync(p->ws + p->pb.keys, 0xFF, kb, st));
+            SOM_CK(h, cudaMemsetAsync(p->ws + p->pb.keys2, 0xFF, kb, st));
             if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_PLAN_END, st))) return rc;
-            if ((rc = two_stage_search(h, p->indptr, p->indices, p->n, p->head, p->ws, p->pb, p->n_hot, d_bmu,
-                                       d_min_dist, nullptr, nullptr, st)))
+            GateScope scope(h, counters + SOM_PLAN_USE_TABLE);
+            if ((rc = two_stage_enqueue(h, p->indptr, p->indices, p->n, p->head, p->ws, p->pb, p->n_hot, d_bmu,
+                                        d_min_dist, nullptr, nullptr, st)))
+                return rc;
+            h->gate_want = SOM_GATE_TABLE_PLAIN;
+            if ((rc = som_launch_bmu_table(h, false, p->indptr, p->indices, p->n, p->head, p->ws, p->pb, p->n_hot, 1,
+                                           st)))
+                return rc;
+            if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_SEARCH_END, st))) return rc;
+            if ((rc = som_launch_finalize_sorted(h, p->indptr, p->indices, p->n, p->ws, p->pb, false, d_bmu,
+                                                 d_min_dist, st)))
+                return rc;
+            h->gate_want = SOM_GATE_TABLE;
+            if ((rc = rare_pass(h, p->indptr, p->indices, p->n, p->head, p->ws, p->pb, d_bmu, d_min_dist, nullptr,
+                                nullptr, st)))
                 return rc;
             if ((rc = mark(h, h->ev_bmu_calls, EV_BMU_END, st))) return rc;
             if (h->timing) h->ev_bmu_calls += 1;
@@ -918,7 +893,16 @@ int som_get_timing(som_handle* h, float* out_ms, int n_out)
     return SOM_OK;
 }
 
-int64_t som_last_uncertain(const som_handle* h) { return h ? h->last_uncertain : 0; }
+int64_t som_last_uncertain(const som_handle* h)
+{
+    if (!h) return 0;
+    if (h->last_uncertain >= 0 || !h->host_pair) return h->last_uncertain < 0 ? 0 : h->last_uncertain;
+    // the last two-stage call left its report in pinned host words (valid once its stream has been waited for):
+    // word 0 = all samples when the probe sent the batch to the plain search, else -1; word 1 = the length of
+    // the certificate's list
+    const int32_t report = *reinterpret_cast<volatile int32_t*>(h->host_pair);
+    return report >= 0 ? (int64_t)report : (int64_t) * reinterpret_cast<volatile int32_t*>(h->host_pair + 1);
+}
 
 int64_t som_launch_count(const som_handle* h) { return h ? h->launches : 0; }
 

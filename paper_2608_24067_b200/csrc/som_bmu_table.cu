@@ -860,8 +860,9 @@ __global__ void k_certify(const float* __restrict__ W, const double* __restrict_
                           int32_t* __restrict__ bmu, float* __restrict__ dist,
                           int32_t* __restrict__ bmu2, float* __restrict__ dist2,
                           int32_t* __restrict__ uncertain, uint4* __restrict__ slots2,
-                          int* __restrict__ n_uncertain)
+                          int* __restrict__ n_uncertain, const int* __restrict__ gate, int gate_want)
 {
+    if (som_gated_off(gate, gate_want)) return;
     __shared__ int warp_count[8];
     __shared__ int block_base;
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -966,7 +967,8 @@ int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indi
 #define SOM_CERTIFY(SECOND_, COUNT_)                                                                            \
     k_certify<SECOND_, COUNT_><<<(unsigned)blocks, 256, 0, st>>>(h->W, h->norm64, h->M, h->V, indptr, indices, n, slots, \
                                                                  order, keys, keys2, keys3, h->wmax_bits, h->hnorm, bmu,  \
-                                                                 dist, bmu2, dist2, uncertain, slots2, n_uncertain)
+                                                                 dist, bmu2, dist2, uncertain, slots2, n_uncertain, \
+                                                                 h->gate, h->gate_want)
     if (second && count_only) SOM_CERTIFY(true, true);
     else if (second) SOM_CERTIFY(true, false);
     else if (count_only) SOM_CERTIFY(false, true);
@@ -981,8 +983,10 @@ int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indi
 // position index / SOM_PROBE_STRIDE of a second slot array.
 namespace {
 __global__ void k_probe_gather(const uint4* __restrict__ slots, const uint32_t* __restrict__ order, int64_t n,
-                               uint4* __restrict__ probe, uint32_t* __restrict__ probe_order)
+                               uint4* __restrict__ probe, uint32_t* __restrict__ probe_order,
+                               const int* __restrict__ gate, int gate_want)
 {
+    if (som_gated_off(gate, gate_want)) return;
     const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= n) return;
     const uint32_t s = order[k];
@@ -1002,7 +1006,40 @@ int som_launch_probe_gather(som_handle* h, int64_t n, char* ws, const SomPlanBuf
     k_probe_gather<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(ws + b.slots),
                                                      reinterpret_cast<const uint32_t*>(ws + b.order), n,
                                                      reinterpret_cast<uint4*>(ws + b.slots2),
-                                                     reinterpret_cast<uint32_t*>(ws + b.uncertain));
+                                                     reinterpret_cast<uint32_t*>(ws + b.uncertain), h->gate, h->gate_want);
+    SOM_CK(h, cudaGetLastError());
+    h->launches += 1;
+    return SOM_OK;
+}
+
+// The two-stage search's own choice, made on the device: with the row-table kernel chosen (gate word 1),
+// the batch takes the two-stage search (gate word 2) unless its probe failed the certificate for more than
+// a fifth of the probed samples.  *report receives what som_last_uncertain is to say for a batch that takes the
+// plain search (all its samples), else -1 (the certificate's own count follows later).
+namespace {
+__global__ void k_two_stage_decide(int* __restrict__ choice, const int* __restrict__ probe_uncertain, int n_probe,
+                                   int64_t n, int* __restrict__ counters_to_clear, int* __restrict__ report)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int r = -1;
+    if (*choice >= 1) {  // (2 is what an earlier search of the same plan left)
+        const bool plain = n_probe > 0 && (int64_t)(*probe_uncertain) * 5 > (int64_t)n_probe;
+        *choice = plain ? 1 : 2;
+        if (plain) r = (int)n;
+    } else if (*choice == 0) {
+        r = 0;
+    }
+    *report = r;
+    counters_to_clear[0] = 0;  // the probe's uncertain count: the full batch's certificate starts from zero
+}
+}  // namespace
+
+int som_launch_two_stage_decide(som_handle* h, char* head, const SomPlanBuffers& b, int n_probe, int64_t n,
+                                cudaStream_t st)
+{
+    int* counters = reinterpret_cast<int*>(head + b.n_slots);
+    k_two_stage_decide<<<1, 32, 0, st>>>(counters + SOM_PLAN_USE_TABLE, counters + SOM_PLAN_UNCERTAIN, n_probe, n,
+                                         counters + SOM_PLAN_UNCERTAIN, counters + SOM_PLAN_REPORT);
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -11,6 +11,12 @@
 #define SOM_EV_RING 32
 #define SOM_N_EVENTS (SOM_EV_PER_CALL * SOM_EV_RING)
 
+// which choices of the device-side gate a launch belongs to (bit number = value of the gate word)
+#define SOM_GATE_DIRECT 1      /* choice 0 */
+#define SOM_GATE_TABLE_PLAIN 2 /* choice 1 */
+#define SOM_GATE_TABLE_TS 4    /* choice 2 */
+#define SOM_GATE_TABLE 6       /* choice 1 or 2: the plan, the rare pass */
+
 // bits of som_handle::dev_flags
 #define SOM_FLAG_BAD_INDEX 1 /* a feature id outside [0, V) was skipped */
 #define SOM_FLAG_BAD_UNIT 2  /* a best-unit index outside [0, M) was skipped */
@@ -67,8 +73,9 @@ struct som_handle {
     int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)
     int64_t opt_two_stage;  // 0 = off, 1 = on where it applies (fp32 storage, M % 128 == 0, memory for the shadow)
     int64_t opt_cover;     // auto selection: least percentage of instances the row table must cover (0 = 60)
-    // Kernel choice made on the device (automatic mode): the launchers hand `gate` / `gate_want` to the
-    // kernels of both search paths, and a kernel returns at once unless *gate == gate_want.
+    // Kernel choice made on the device: the launchers hand `gate` / `gate_want` to the kernels of every
+    // search path, and a kernel returns at once unless bit *gate of gate_want is set (SOM_GATE_* masks).
+    // *gate is 0 = direct-load kernel, 1 = row-table kernel, 2 = row-table kernel with the two-stage search.
     const int* gate;       // device, nullptr = no gate
     int gate_want;
     int gate_small_grid;   // the gated launch in hand is expected to return at once: give it a small grid
@@ -135,9 +142,9 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
                       cudaEvent_t ev_join);
 
 // true when this launch belongs to the search path that the plan's selection did not choose
-__device__ __forceinline__ bool som_gated_off(const int* gate, int want)
+__device__ __forceinline__ bool som_gated_off(const int* gate, int want_mask)
 {
-    return gate != nullptr && *reinterpret_cast<const volatile int*>(gate) != want;
+    return gate != nullptr && !((want_mask >> *reinterpret_cast<const volatile int*>(gate)) & 1);
 }
 
 // records a skipped entry in the handle's flag word (one atomic per warp that saw any)

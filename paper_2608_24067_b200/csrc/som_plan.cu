@@ -499,7 +499,7 @@ int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* 
         SOM_CK(h, cudaFuncSetAttribute(k_select_hot, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)counts_sh));
     k_select_hot<<<1, 1024, counts_fit ? counts_sh : 0, st>>>(feat_count, h->V, n_mask, n_hot, counts_fit, feat_slot,
                                                              slot_feat, n_slots, indptr, n,
-                                                             (int)(h->opt_cover > 0 ? h->opt_cover : 60));
+                                                             (int)(h->opt_cover > 0 ? h->opt_cover : (h->opt_cover < 0 ? 0 : 60)));
     SOM_CK(h, cudaGetLastError());
     h->launches += 2;
     return SOM_OK;

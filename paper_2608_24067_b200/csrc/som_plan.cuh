@@ -43,8 +43,8 @@ struct SomPlanBuffers {
     size_t feat_slot;   // i32 [V]      table slot of a feature, -1 = tail
     size_t slot_feat;   // i32 [slots]  feature of a table slot, -1 = unused
     size_t n_slots;     // i32 [8]      mask slots used, hot slots used, length of rare_list, search unit counter,
-                        //              feature instances covered by the table, uncertain samples,
-                        //              1 if the automatic mode takes the row-table kernel for this batch
+                        //              feature instances covered by the table, uncertain samples, the gate
+                        //              word (SOM_PLAN_USE_TABLE), the two-stage report (SOM_PLAN_REPORT)
     // workspace
     size_t keys;        // u64 [n]      packed (score, neuron) per sorted position
     size_t keys2;       // u64 [n]      the same for the second-best unit (two-best search only)
@@ -68,7 +68,9 @@ struct SomPlanBuffers {
 #define SOM_PLAN_RARE 2 /* index into n_slots: length of rare_list */
 #define SOM_PLAN_COVERED 4 /* index into n_slots */
 #define SOM_PLAN_UNCERTAIN 5 /* index into n_slots: length of the two-stage search's uncertain list */
-#define SOM_PLAN_USE_TABLE 6 /* index into n_slots: the selection kernel's choice of search kernel */
+#define SOM_PLAN_USE_TABLE 6 /* index into n_slots: the device-side choice (the gate word): 0 direct-load kernel,
+                                1 row-table kernel, 2 row-table kernel with the two-stage search */
+#define SOM_PLAN_REPORT 7    /* index into n_slots: the two-stage search's report (see k_two_stage_decide) */
 
 // Sample parts per neuron range of the row-table kernel.  More parts mean fewer ranges live at
 // once (their slabs must share L2 with the slot stream) but smaller units, each of which
@@ -118,6 +120,8 @@ int som_launch_certify(som_handle* h, const int32_t* indptr, const int32_t* indi
 #define SOM_PROBE_STRIDE 256
 #define SOM_PROBE_MIN_BATCH 65536
 int som_launch_probe_gather(som_handle* h, int64_t n, char* ws, const SomPlanBuffers& b, cudaStream_t st);
+int som_launch_two_stage_decide(som_handle* h, char* head, const SomPlanBuffers& b, int n_probe, int64_t n,
+                                cudaStream_t st);
 
 int som_launch_finalize_sorted(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                                char* ws, const SomPlanBuffers& b, bool second, int32_t* bmu, float* dist,

@@ -1,0 +1,16 @@
+// Geometry tunables of the row-table search kernel, set through som_set_option (include/som.h).
+// They exist for benchmarking and for the tests that walk every template instance; 0 always means
+// "the measured default".  A reusable plan (som_plan_create) is tied to their values at its creation.
+//
+//   key 1  hot rows kept in shared memory beside the 16 mask rows (default: 352 rows of 512 bytes, 720 of
+//          256 bytes, 1376 / 1456 of 128 bytes: what keeps table + slot rings under 196 KB, so that the
+//          SM keeps a 60 KB L1)
+//   key 2  block size: 512, 576 (wide fp32 layout only), 640, 768, 896, 1024
+//   key 3  neurons per lane: fp32 storage 4, 8 (needs M % 64 == 0), 16 (M % 128 == 0); fp16 storage 8,
+//          16 (M % 128 == 0); default: the widest that divides M (fp32 with the two-stage search: 8)
+//   key 4  sample parts per neuron range (default: see som_table_default_parts in som_plan.cuh)
+#pragma once
+#define SOM_OPT_HOT_ROWS 1
+#define SOM_OPT_THREADS 2
+#define SOM_OPT_LANE_NEURONS 3
+#define SOM_OPT_PARTS 4

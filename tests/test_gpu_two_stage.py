@@ -234,6 +234,7 @@ def test_two_stage_with_a_reusable_plan(som_mod):
             W[epoch::7] += 0.01
         h.norms()
         p_bmu, p_dist = plan.bmu()
+        torch.cuda.synchronize()  # (the count travels back unwaited for: read it once the stream is done)
         unc_planned = h.last_uncertain()
         d_bmu, d_dist = h.bmu(b.indptr, b.indices)
         torch.cuda.synchronize()
