@@ -150,8 +150,10 @@ template <int R_>
 struct LayF32 {
     typedef float Store;
     static constexpr int R = R_, H = R_ / 4, T = 8 * R_, ROWB = T * 4;
-    // tail rows of a sample whose loads go in flight before its hot rows (each holds R registers)
-    static constexpr int TAILS_AHEAD = R_ >= 16 ? 2 : 4;
+    // tail rows of a sample whose loads go in flight before its hot rows (each holds R registers; with 16
+    // neurons per lane three fit 128 registers at the price of a 36-byte spill, and measure 1 to 3 % faster
+    // than two)
+    static constexpr int TAILS_AHEAD = R_ >= 16 ? 3 : 4;
     static constexpr float SEED_SIGN = 1.f;     // scores are held as they are
     typedef Acc<H> Scores;
     typedef Acc<H> Slice;
