@@ -924,6 +924,11 @@ int som_set_option(som_handle* h, int key, int64_t value)
         h->opt_parts = value;
         return SOM_OK;
     }
+    if (key == 8) {
+        if (value < 0 || value > SOM_PLAN_MASK_FEATURES) return SOM_ERR_INVALID_ARG;
+        h->opt_mask_bits = value;
+        return SOM_OK;
+    }
     if (key == 7) {
         if (value != 0 && value != 1) return SOM_ERR_INVALID_ARG;
         if (value == 1 && !h->shadow && !h->Wh) {

@@ -465,6 +465,28 @@ int som_launch_pad_slots(som_handle* h, char* ws, size_t slots_offset, int64_t n
     return SOM_OK;
 }
 
+// How many of the table's first SOM_PLAN_MASK_FEATURES rows are handled as mask bits (the others are
+// ordinary hot rows).  A mask feature costs a sample nothing while its mask equals that of the sample its
+// team handled before (four positions earlier in the sorted list), and a rebuild of the whole prefix,
+// which stalls the other three teams of the warp, when it does not.  The sorted list has one run per
+// distinct mask, so the smaller the batch, the shorter the runs and the fewer bits pay.  Measured on the
+// MeSH-shaped batches, whole call, fp32: 250k samples on the 1024 x 1024 map 430 ms with 16 bits, 379 with 9
+// (the optimum: 387 with 7, 386 with 11); 1M samples on 512 x 512: 359 / 337 (10 or 11 bits); 4M samples
+// on 128 x 128: 82.0 / 80.4 (12 or 13 bits).  fp16 storage moves the same way (269 -> 226 ms at 9 bits).
+static void plan_split(const som_handle* h, int64_t n, int* n_mask, int* n_hot)
+{
+    int bits = (int)h->opt_mask_bits;
+    if (bits == 0) {
+        int lg = 0;
+        while (lg < 40 && ((int64_t)1 << (lg + 1)) <= n) ++lg;  // floor(log2 n)
+        bits = lg - 8;                                            // 250k -> 9, 1M -> 11, 4M -> 13
+        if (bits < 4) bits = 4;
+    }
+    if (bits > *n_mask) bits = *n_mask;
+    *n_hot += *n_mask - bits;
+    *n_mask = bits;
+}
+
 int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* indices, int64_t n,
                            char* head, const SomPlanBuffers& b, int n_mask, int n_hot, cudaStream_t st)
 {
@@ -472,6 +494,7 @@ int som_launch_plan_select(som_handle* h, const int32_t* indptr, const int32_t* 
     int32_t* feat_slot = reinterpret_cast<int32_t*>(head + b.feat_slot);
     int32_t* slot_feat = reinterpret_cast<int32_t*>(head + b.slot_feat);
     int32_t* n_slots = reinterpret_cast<int32_t*>(head + b.n_slots);
+    plan_split(h, n, &n_mask, &n_hot);
 
     SOM_CK(h, cudaMemsetAsync(feat_count, 0, (size_t)h->V * 4, st));
     SOM_CK(h, cudaMemsetAsync(n_slots, 0, SOM_PLAN_N_SLOTS_INTS * 4, st));
@@ -515,6 +538,7 @@ int som_launch_plan_sort(som_handle* h, const int32_t* indptr, const int32_t* in
     uint32_t* bin_count = reinterpret_cast<uint32_t*>(ws + b.bin_count);
     uint32_t* bin_start = reinterpret_cast<uint32_t*>(ws + b.bin_start);
     uint32_t* slots = reinterpret_cast<uint32_t*>(ws + b.slots);
+    plan_split(h, n, &n_mask, &n_hot);
 
     SOM_CK(h, cudaMemsetAsync(bin_count, 0, (size_t)SOM_PLAN_BINS * 4, st));
     // 3. classify

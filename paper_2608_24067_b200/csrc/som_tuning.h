@@ -9,8 +9,11 @@
 //   key 3  neurons per lane: fp32 storage 4, 8 (needs M % 64 == 0), 16 (M % 128 == 0); fp16 storage 8,
 //          16 (M % 128 == 0); default: the widest that divides M (fp32 with the two-stage search: 8)
 //   key 4  sample parts per neuron range (default: see som_table_default_parts in som_plan.cuh)
+//   key 8  how many of the 16 most frequent features of a batch are handled as mask bits (1..16); default:
+//          floor(log2(samples)) - 8, at least 4, at most 16 (see plan_split in som_plan.cu)
 #pragma once
 #define SOM_OPT_HOT_ROWS 1
 #define SOM_OPT_THREADS 2
 #define SOM_OPT_LANE_NEURONS 3
 #define SOM_OPT_PARTS 4
+#define SOM_OPT_MASK_BITS 8

@@ -123,6 +123,27 @@ def test_row_table_geometries(som_mod, lane_neurons, threads):
                           bmu.cpu().numpy(), dist.cpu().numpy(), rows)
 
 
+@pytest.mark.parametrize("mask_bits", [1, 5, 9, 16])
+def test_mask_feature_counts(som_mod, mask_bits):
+    """How many of the batch's most frequent features the plan handles as mask bits (the rest of the 16
+    become ordinary hot rows) is a matter of speed only: every split matches the oracle, on fp32 and on the
+    wide fp16 layout (permuted feature ids, so that the frequent features are not the low ids)."""
+    V, M, n = 30_000, 1_024, 50_000
+    b = synth.sample_csr(n, V, 11.0, 4, device="cuda", permute_ids=True)
+    rows = np.arange(0, n, 9)
+    for dtype in (torch.float32, torch.float16):
+        W = synth.fill_codebook(V, M, 4, device="cuda").to(dtype)
+        h = som_mod.Som(V, M, W)
+        h.set_option(0, 2)
+        h.set_option(8, mask_bits)
+        h.norms()
+        bmu, dist = h.bmu(b.indptr, b.indices)
+        torch.cuda.synchronize()
+        _check_against_oracle(W.float().cpu().numpy(), V, M, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
+                              bmu.cpu().numpy(), dist.cpu().numpy(), rows)
+        assert h.device_flags() == 0
+
+
 def test_config3_full_size_sampled_rows(som_mod):
     """128x128 map at its full size (4M samples, the benchmark's launch configuration);
     a strided sample of rows against the oracle, plus properties that hold for all rows."""
