@@ -78,11 +78,11 @@ struct SomPlanBuffers {
 //   64-neuron ranges (fp32, 256-byte rows): flat optimum at about 20,000 samples per unit, at most 32 parts;
 //   128-neuron ranges of the wide fp16 layout (256-byte rows): half as many ranges, smaller units;
 //   128-neuron ranges of the wide fp32 layout (512-byte rows, slabs of 15 MB): the fewer ranges are
-//     live the better - 56 parts on a 250k-sample batch (units of 4,500 samples) are 10 % faster than
-//     16 on the largest map, 96 to 128 parts are best on 4M samples.
+//     live the better - 40 to 48 parts on a 250k-sample batch (units of 6,000 samples) are 10 % faster
+//     than 16 on the largest map, 64 to 80 are best on 1M samples, 96 to 128 on 4M samples.
 static inline int som_table_default_parts(int64_t n, int range_neurons, int row_bytes)
 {
-    if (row_bytes >= 512) return n < 48 * 1024 ? (n < 1024 ? 1 : (int)(n / 1024)) : (n < 600000 ? 56 : 96);
+    if (row_bytes >= 512) return n < 48 * 1024 ? (n < 1024 ? 1 : (int)(n / 1024)) : (n < 600000 ? 44 : (n < 2500000 ? 64 : 96));
     const bool wide = range_neurons >= 128;
     const int64_t parts = n / (wide ? 15000 : 20000);
     const int64_t cap = wide ? 64 : 32;

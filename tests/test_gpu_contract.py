@@ -22,16 +22,18 @@ def som_mod():
     return som
 
 
-@pytest.mark.parametrize("variant", [0, 2])
-def test_som_bmu_returns_before_the_search_has_run(som_mod, variant):
+@pytest.mark.parametrize("variant,two_stage", [(0, 0), (2, 0), (0, 1), (2, 1)])
+def test_som_bmu_returns_before_the_search_has_run(som_mod, variant, two_stage):
     """The call only enqueues: an event recorded right after it returns is not yet reached (the
     search of a million samples over 16 384 neurons takes about 20 ms), and the results are those
-    of a call that was waited for."""
+    of a call that was waited for.  The two-stage search (probe, verdict, second pass) is no
+    exception: its decisions are taken on the device."""
     V, M, n = 30_000, 16_384, 1_000_000
     W = synth.fill_codebook(V, M, 0, device="cuda")
     b = synth.sample_csr(n, V, 11.0, 0, device="cuda")
     h = som_mod.Som(V, M, W)
     h.set_option(0, variant)
+    h.set_option(7, two_stage)
     h.norms()
     ref_bmu, ref_dist = h.bmu(b.indptr, b.indices)  # grows the workspace (may synchronise)
     torch.cuda.synchronize()
