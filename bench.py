@@ -670,6 +670,9 @@ def main():
     ap.add_argument("--radius", type=int, default=0, help="som_update: blur radius (default edge / 4)")
     ap.add_argument("--batch", type=int, default=0,
                     help="samples per batch instead of the configuration's (a sweep variant, named in the workload)")
+    ap.add_argument("--V", type=int, default=0,
+                    help="features instead of the configuration's 30 000 (a smaller variant of the same map for "
+                         "profiler captures that must hold few GB; named in the workload)")
     ap.add_argument("--tc-probe", action="store_true",
                     help="run the tcgen05 microbenchmark of the densified hot-feature tile and print its numbers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -684,6 +687,8 @@ def main():
         if args.batch > 0:
             w = dataclasses.replace(w, name="%s-batch%d" % (w.name, args.batch), batch=args.batch,
                                     N=max(w.N, args.batch))
+        if args.V > 0:
+            w = dataclasses.replace(w, name="%s-V%d" % (w.name, args.V), V=args.V)
         if args.zipf_s is not None:
             w = dataclasses.replace(w, name="%s-zipf%g" % (w.name, args.zipf_s), zipf_s=args.zipf_s)
         if args.store == "f16":

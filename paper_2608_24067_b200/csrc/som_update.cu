@@ -21,7 +21,9 @@
 // from an integer box count of the occupied cells over the reach of three passes (3 * radius):
 // a running sum that subtracts can leave a rounding residue where the exact sum is zero.
 // Lattices of up to 128 x 128 cells replace steps 2-4 by one kernel that blurs a plane in shared
-// memory (k_upd_blur_fused): one read and one write of the plane instead of seven.
+// memory (k_upd_blur_fused): one read and one write of the plane instead of seven.  Larger lattices
+// scatter in neuron order and take two strip kernels through shared memory (k_upd_strip), as long as
+// a strip of eight lines fits there; only shapes beyond that walk steps 1-4 through device memory.
 #include "som_internal.cuh"
 
 namespace {
@@ -123,7 +125,7 @@ __global__ void k_upd_hot_mask(const int32_t* __restrict__ indptr, const int32_t
 
 __global__ void k_upd_scatter_hot(const uint32_t* __restrict__ mask, int64_t n, const int32_t* __restrict__ bmu,
                                   int v0, int v1, int rows, int cols, const int32_t* __restrict__ slot_feat,
-                                  int n_slots, int planes_per_block, float* __restrict__ num_t)
+                                  int n_slots, int planes_per_block, float* __restrict__ num_t, int natural_order)
 {
     extern __shared__ unsigned int cnt[];
     const int M = rows * cols;
@@ -145,7 +147,7 @@ __global__ void k_upd_scatter_hot(const uint32_t* __restrict__ mask, int64_t n, 
             const int c = bmu[s];
             if ((unsigned)c >= (unsigned)M) continue;  // skipped; k_upd_count has noted it
             const int r = c / cols, q = c - r * cols;
-            const int cell_t = q * rows + r;  // transposed cell order
+            const int cell_t = natural_order ? c : q * rows + r;  // (transposed cell order unless the strip route follows)
             while (m) {
                 const int slot = __ffs(m) - 1;
                 m &= m - 1;
@@ -302,63 +304,247 @@ __device__ __forceinline__ void box_lines(const BT* __restrict__ in, BT* __restr
 // Lattices too large for one plane to be blurred on chip (more than 16384 cells) take the blur in two
 // strip kernels through shared memory instead of seven trips through device memory.  A box pass
 // along one lattice axis never mixes the lines of the other, so a block can take a strip of `tc`
-// adjacent lines over their whole length: k_upd_strip loads the strip as a tile [len][tc] (the walk
-// index slow, the strip's lines fast: consecutive banks for every access of the walks, whatever the
-// radius), runs the three passes between two fp32 buffers with fp64 running sums (the fields between
-// passes are rounded to fp32, as on the device-memory route), and writes once:
-//   first launch  (FINAL = false): input in TRANSPOSED cell order (cell (r, c) at c * rows + r, as the
-//                 scatter leaves it): the walk runs along a lattice row; the result is written in
-//                 neuron order, i.e. the tile is transposed on its way out;
-//   second launch (FINAL = true):  input in neuron order, the walk runs down a lattice column; the
-//                 result is multiplied by the reciprocal blurred denominator and written as the new
-//                 weights of features v0 + plane (a zero reciprocal keeps the prototype).
+// adjacent lines over their whole length, run the three passes of that axis between two fp32 tiles
+// [line][cell] with fp64 running sums (the fields between passes are rounded to fp32, as on the
+// device-memory route) and write once:
+//   first launch  (ROWS = true):  a line is a lattice row, contiguous in memory; in and out in neuron order;
+//   second launch (ROWS = false): a line is a lattice column (cell i of line f at i * width + f); the result
+//                 is multiplied by the reciprocal blurred denominator and written as the new weights of
+//                 features v0 + plane (a zero reciprocal keeps the prototype).
 // A plane crosses device memory five times in all (scatter, in, out, in, weights out).
-constexpr int STRIP_THREADS = 256;
-typedef float STRIP_BT;  // type of the two tile buffers (fp64 buffers measured twice as slow: fewer blocks per SM)
+//
+// One thread walks a segment of 16 cells: the window sum at the segment's first cell is put together from
+// the totals of the segments that lie wholly inside the window (fp64, one per segment, kept in shared memory)
+// and the few cells at the window's two ends; then every step adds the entering cell and subtracts the
+// leaving one.  The totals of the next pass's input are summed on the way (the thread has just produced
+// those 16 cells).  What counts is the instruction budget: the first version of this kernel spent 58
+// instructions per cell and pass (generic strides, bounds tests and pointer updates per cell, a totals
+// pass of its own, three fp32 <-> fp64 conversions per cell on the 16-lane conversion unit); here the walk of
+// a segment whose window stays inside the line is fully unrolled with immediate offsets, the other
+// segments clamp their indices into a zero cell instead of testing bounds, and the widening of the value
+// just rounded goes through integer instructions instead of the conversion unit.
+// Layout: the line pitch is 1 modulo 32 words and a warp holds 16 lines x 2 neighbouring segments (or 32 lines
+// x 1), so every access of a walk touches 32 different banks.  Cells [len, pitch) of every line and the word
+// before the first line stay zero: they are what out-of-range window ends read.
+constexpr int STRIP_THREADS = 512;
+constexpr int STRIP_SEG = 16;
+constexpr int STRIP_MAX_ITERS = 4;  // segments of a strip per thread, at most
 
-// in: [plane][len][width]; the block's strip is the `tc` fast indices f0 .. f0 + tc - 1
-template <typename ST, bool TOTALS, bool FINAL>
-__global__ void __launch_bounds__(STRIP_THREADS)
+// A window sum rounded to the 24 significant bits of the fp32 field it is stored in, still as an fp64 value
+// (Veltkamp's splitting with 2^29 + 1: one multiplication and two additions on the fp64 pipe, result the
+// nearest 24-bit value).  The thread stores it (its conversion to fp32 is then exact) and adds the same
+// value to the total of the next pass's input, so cells and totals agree bit for bit without widening the
+// stored value again: the conversion unit (16 lanes per SM) sees three conversions per cell, not four, and
+// an integer emulation of the widening cost seven instructions per cell.
+__device__ __forceinline__ double strip_round24(double x)
+{
+    // (intrinsics: the compiler must not contract the product into the subtraction)
+    const double gamma = __dmul_rn(x, 536870913.0);  // 2^29 + 1
+    const double delta = __dsub_rn(x, gamma);
+    return __dadd_rn(gamma, delta);
+}
+
+// The walk of one segment: y[k] = window sum at cell a + k for k = 1 .. 15, given the sum at cell a.
+// ENTER / LEAVE say whether the segment's steps have an entering / a leaving cell at all (they have all or none
+// on these paths; pe[k] enters and pl[k] leaves at step k); returns the fp64 total of the rounded outputs.
+template <bool ENTER, bool LEAVE>
+__device__ __forceinline__ double strip_walk(const float* __restrict__ pe, const float* __restrict__ pl,
+                                             float* __restrict__ y, double sum, double t_next)
+{
+#pragma unroll
+    for (int k = 1; k < STRIP_SEG; ++k) {
+        if (ENTER && LEAVE) sum += (double)pe[k] - (double)pl[k];
+        else if (ENTER) sum += (double)pe[k];
+        else if (LEAVE) sum -= (double)pl[k];
+        const double o = strip_round24(sum);
+        y[k] = (float)o;
+        t_next += o;
+    }
+    return t_next;
+}
+
+// in: plane-major; ROWS: cell i of line f at f * len + i, else at i * width + f.  The block's strip is lines
+// f0 .. f0 + tc - 1 (tc a power of two).  Shared memory: the segment totals tot[tc][n_seg | 1] and their
+// running sums cum[tc][(n_seg + 1) | 1] (fp64), then 1 + 2 * tc * pitch floats.
+template <typename ST, bool ROWS>
+__global__ void __launch_bounds__(STRIP_THREADS, 3)
 k_upd_strip(const float* __restrict__ in, float* __restrict__ out, int64_t planes, int len, int width, int radius,
-            int tc, int seg, const double* __restrict__ rden, ST* __restrict__ W, int v0)
+            int tc, int tc_shift, int pitch, const double* __restrict__ rden, ST* __restrict__ W, int v0)
 {
     extern __shared__ __align__(16) unsigned char strip_raw[];
-    __shared__ double tot[STRIP_THREADS];
-    const int pitch = tc | 1;
-    STRIP_BT* A = reinterpret_cast<STRIP_BT*>(strip_raw);
-    STRIP_BT* B = A + (size_t)len * pitch;
+    const int n_seg = (len + STRIP_SEG - 1) / STRIP_SEG;
+    const int len_pad = n_seg * STRIP_SEG;
+    const int n_jobs = n_seg << tc_shift;
+    const int tot_pitch = n_seg | 1, cum_pitch = (n_seg + 1) | 1;  // odd: 16 lines at one segment, 32 banks
+    double* tot = reinterpret_cast<double*>(strip_raw);
+    double* cum = tot + tc * tot_pitch;
+    float* A = reinterpret_cast<float*>(cum + tc * cum_pitch) + 1;
+    float* B = A + (size_t)tc * pitch;
+    for (int c = threadIdx.x; c < 1 + 2 * tc * pitch; c += STRIP_THREADS) A[c - 1] = 0.f;
     const int64_t M = (int64_t)len * width;
     const int groups = (width + tc - 1) / tc;
     const int64_t items = planes * groups;
-    const int ti = STRIP_THREADS / tc;  // walk positions one sweep of the block's threads covers
-    const int lf = threadIdx.x % tc, li = threadIdx.x / tc;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // Column strips (ROWS = false) are moved with line f = thread % tc and walk index col_first, col_first +
+    // 512 / tc, ...  A warp of up to 32 lines holds 32 / tc walk indices; they are taken tc apart, so that the
+    // warp's 32 tile cells [f][i] (bank f + i) fall into 32 banks; the sweep of the block still covers
+    // 512 / tc consecutive indices.
+    const int col_first = tc <= 32 ? (lane >> tc_shift) * tc + (warp & (tc - 1)) + 32 * (warp >> tc_shift)
+                                   : threadIdx.x >> tc_shift;
+    __syncthreads();
     for (int64_t it = blockIdx.x; it < items; it += gridDim.x) {
         const int64_t plane = it / groups;
         const int f0 = (int)(it - plane * groups) * tc;
         const int nf = min(tc, width - f0);
-        const float* src = in + plane * M + f0;
-        for (int i = li; i < len; i += ti) A[i * pitch + lf] = lf < nf ? (STRIP_BT)src[(int64_t)i * width + lf] : (STRIP_BT)0;
+        // ---- load the strip -------------------------------------------------------------------------
+        if (ROWS) {
+            for (int f = warp; f < nf; f += STRIP_THREADS / 32) {
+                const float* s = in + plane * M + (int64_t)(f0 + f) * len + lane;
+                float* d = A + f * pitch + lane;
+                int i = lane;
+                for (; i + 96 < len; i += 128, s += 128, d += 128) {  // four loads in flight
+                    const float v0 = s[0], v1 = s[32], v2 = s[64], v3 = s[96];
+                    d[0] = v0;
+                    d[32] = v1;
+                    d[64] = v2;
+                    d[96] = v3;
+                }
+                for (; i < len; i += 32, s += 32, d += 32) d[0] = s[0];
+            }
+        } else {
+            const int f = threadIdx.x & (tc - 1);
+            const int step = STRIP_THREADS >> tc_shift;
+            if (f < nf) {
+                int i = col_first;
+                const float* s = in + plane * M + f0 + (int64_t)i * width + f;
+                const int64_t hop = (int64_t)step * width;
+                float* d = A + f * pitch + i;
+                for (; i + 3 * step < len; i += 4 * step, s += 4 * hop, d += 4 * step) {
+                    const float v0 = s[0], v1 = s[hop], v2 = s[2 * hop], v3 = s[3 * hop];
+                    d[0] = v0;
+                    d[step] = v1;
+                    d[2 * step] = v2;
+                    d[3 * step] = v3;
+                }
+                for (; i < len; i += step, s += hop, d += step) d[0] = s[0];
+            }
+        }
         __syncthreads();
-        box_lines<TOTALS>(A, B, nf, len, 1, pitch, radius, seg, tot);
+        // ---- totals of the first pass's input -------------------------------------------------------
+#pragma unroll 1
+        for (int job = threadIdx.x; job < n_jobs; job += STRIP_THREADS) {
+            {
+                const int line = job & (tc - 1), g = job >> tc_shift;
+                const float* x = A + line * pitch + g * STRIP_SEG;
+                double t0 = 0.0, t1 = 0.0;
+#pragma unroll
+                for (int k = 0; k < STRIP_SEG; k += 2) {
+                    t0 += (double)x[k];
+                    t1 += (double)x[k + 1];
+                }
+                tot[line * tot_pitch + g] = t0 + t1;
+            }
+        }
+        // ---- three passes --------------------------------------------------------------------------
+        float* X = A;
+        float* Y = B;
+#pragma unroll 1
+        for (int pass = 0; pass < 3; ++pass) {
+            __syncthreads();  // the totals of this pass's input are written
+            // running sums of a line's totals, a warp per line: cum[q] = tot[0] + ... + tot[q - 1]
+            for (int line = warp; line < tc; line += STRIP_THREADS / 32) {
+                double carry = 0.0;
+                for (int q0 = 0; q0 < n_seg; q0 += 32) {
+                    const int q = q0 + lane;
+                    double v = q < n_seg ? tot[line * tot_pitch + q] : 0.0;
+#pragma unroll
+                    for (int d = 1; d < 32; d *= 2) {
+                        const double up = __shfl_up_sync(0xffffffffu, v, d);
+                        if (lane >= d) v += up;
+                    }
+                    if (q < n_seg) cum[line * cum_pitch + q + 1] = carry + v;
+                    carry += __shfl_sync(0xffffffffu, v, 31);
+                }
+                if (lane == 0) cum[line * cum_pitch] = 0.0;
+            }
+            __syncthreads();
+#pragma unroll 1
+            for (int job = threadIdx.x; job < n_jobs; job += STRIP_THREADS) {
+                {
+                    const int line = job & (tc - 1), g = job >> tc_shift;
+                    const int a = g * STRIP_SEG;
+                    const float* x = X + line * pitch;
+                    // window sum at the segment's first cell: whole segments from the running sums, the
+                    // cells at the window's two ends singly
+                    const int lo = max(0, a - radius), hi = min(len_pad - 1, a + radius);
+                    const int q_lo = (lo + STRIP_SEG - 1) / STRIP_SEG, q_hi = (hi + 1) / STRIP_SEG - 1;
+                    int left_end = hi + 1, right_begin = hi + 1;  // cells [lo, left_end) and [right_begin, hi] singly
+                    double sum = 0.0;
+                    if (q_lo <= q_hi) {
+                        const double* cl = cum + line * cum_pitch;
+                        sum = cl[q_hi + 1] - cl[q_lo];
+                        left_end = q_lo * STRIP_SEG;
+                        right_begin = (q_hi + 1) * STRIP_SEG;
+                    }
+                    for (int j = lo; j < left_end; ++j) sum += (double)x[j];
+                    for (int j = right_begin; j <= hi; ++j) sum += (double)x[j];
+                    float* y = Y + line * pitch + a;
+                    double t_next = a < len ? strip_round24(sum) : 0.0;
+                    y[0] = (float)t_next;
+                    const float* pe = x + a + radius;      // pe[k] enters at cell a + k
+                    const float* pl = x + a - radius - 1;  // pl[k] leaves
+                    const bool whole = a + STRIP_SEG <= len;
+                    const bool e_all = a + STRIP_SEG - 1 + radius <= len_pad;  // (cells [len, len_pad] are zero)
+                    const bool e_none = a + 1 + radius >= len;
+                    const bool l_all = a >= radius;
+                    const bool l_none = a + STRIP_SEG - 1 <= radius;
+                    if (whole && e_all && l_all) t_next = strip_walk<true, true>(pe, pl, y, sum, t_next);
+                    else if (whole && e_all && l_none) t_next = strip_walk<true, false>(pe, pl, y, sum, t_next);
+                    else if (whole && e_none && l_all) t_next = strip_walk<false, true>(pe, pl, y, sum, t_next);
+                    else if (whole && e_none && l_none) t_next = strip_walk<false, false>(pe, pl, y, sum, t_next);
+                    else {
+                        // a window end crosses the line's end inside the segment: indices are clamped into a zero cell
+#pragma unroll 5
+                        for (int k = 1; k < STRIP_SEG; ++k) {
+                            const int i = a + k;
+                            const float enter = x[min(i + radius, len_pad)];  // (cell len_pad is zero)
+                            const float leave = x[max(i - radius - 1, -1)];   // (so is cell -1)
+                            sum += (double)enter - (double)leave;
+                            const double o = i < len ? strip_round24(sum) : 0.0;
+                            y[k] = (float)o;
+                            t_next += o;
+                        }
+                    }
+                    tot[line * tot_pitch + g] = t_next;
+                }
+            }
+            float* t = X; X = Y; Y = t;
+        }
         __syncthreads();
-        box_lines<TOTALS>(B, A, nf, len, 1, pitch, radius, seg, tot);
-        __syncthreads();
-        box_lines<TOTALS>(A, B, nf, len, 1, pitch, radius, seg, tot);
-        __syncthreads();
-        if (FINAL) {
-            // (len = rows, width = cols: neuron (i, f0 + lf) is cell i * width + f0 + lf)
+        // ---- write (X holds the result) --------------------------------------------------------------
+        if (ROWS) {
+            for (int f = warp; f < nf; f += STRIP_THREADS / 32) {
+                float* d = out + plane * M + (int64_t)(f0 + f) * len + lane;
+                const float* s = X + f * pitch + lane;
+                int i = lane;
+                for (; i + 96 < len; i += 128, s += 128, d += 128) {
+                    d[0] = s[0];
+                    d[32] = s[32];
+                    d[64] = s[64];
+                    d[96] = s[96];
+                }
+                for (; i < len; i += 32, s += 32, d += 32) d[0] = s[0];
+            }
+        } else {
+            // (len = rows, width = cols: cell i of line f0 + f is neuron i * width + f0 + f)
             ST* dst = W + (int64_t)(v0 + plane) * M + f0;
             const double* rd_base = rden + f0;
-            if (lf < nf)
-                for (int i = li; i < len; i += ti) {
-                    const double rd = rd_base[(int64_t)i * width + lf];
-                    if (rd != 0.0) dst[(int64_t)i * width + lf] = (ST)(float)((double)B[i * pitch + lf] * rd);
+            const int f = threadIdx.x & (tc - 1);
+            if (f < nf)
+                for (int i = col_first; i < len; i += STRIP_THREADS >> tc_shift) {
+                    const double rd = rd_base[(int64_t)i * width + f];
+                    if (rd != 0.0) dst[(int64_t)i * width + f] = (ST)(float)((double)X[f * pitch + i] * rd);
                 }
-        } else {
-            // (len = cols, width = rows: line f0 + f is lattice row r, its cells go to r * len + i)
-            float* dst = out + plane * M + (int64_t)f0 * len;
-            for (int f = 0; f < nf; ++f)
-                for (int i = threadIdx.x; i < len; i += STRIP_THREADS) dst[(int64_t)f * len + i] = (float)B[i * pitch + f];
         }
         __syncthreads();
     }
@@ -619,25 +805,31 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         SOM_CK(h, cudaEventRecord(ev_join, aux));
         st = main_st;
     }
-    // Larger lattices: the strip route wherever a strip of at least four lines over the whole length of
+    // Larger lattices: the strip route wherever a strip of at least eight lines over the whole length of
     // either axis fits in shared memory twice over (fp32); else the passes through device memory.
-    const size_t strip_budget = 200 * 1024;
-    auto strip_width = [&](int len, int width) {
-        // lines per strip: a thread walks a segment of len / (256 / tc) cells, and about 16 cells per thread with
-        // as many blocks per SM as shared memory holds measured best (512 x 512, radius 128: 8 lines per
-        // strip 127 ms, 4: 190 ms, 16: 147 ms, 32: 360 ms for 30 000 planes)
-        int tc = len > 256 ? 8 : (len > 128 ? 16 : 32);
-        while (tc >= 4 && (size_t)len * (tc | 1) * sizeof(STRIP_BT) * 2 > strip_budget) tc /= 2;
-        if (tc >= 4 && tc > width) {  // few lines: all of them in one strip
-            int t2 = 4;
-            while (t2 < width) t2 *= 2;
-            tc = t2 < tc ? t2 : tc;
-        }
-        return tc >= 4 ? tc : 0;
+    struct StripGeom { int tc, shift, pitch; size_t sh; };
+    auto strip_geom = [&](int len, int width) {
+        StripGeom g = {0, 0, 0, 0};
+        const int n_seg = (len + STRIP_SEG - 1) / STRIP_SEG;
+        const int pitch = (n_seg * STRIP_SEG + 31) / 32 * 32 + 1;  // > the padded length, 1 modulo 32
+        auto bytes = [&](int tc) {
+            return (size_t)tc * ((n_seg | 1) + ((n_seg + 1) | 1)) * 8 + (size_t)(2 * tc * pitch + 1) * 4;
+        };
+        // as many lines as give every thread one or two segments, three blocks per SM where that leaves at
+        // least 16 lines (a warp then covers 32 banks), never fewer than 8 lines
+        int tc = 256;
+        while (tc > 8 && (tc * n_seg > 2 * STRIP_THREADS || bytes(tc) > (size_t)80 * 1024)) tc /= 2;
+        while (tc > 8 && tc / 2 >= width) tc /= 2;  // few lines: all of them in one strip
+        if (tc * n_seg > STRIP_MAX_ITERS * STRIP_THREADS || bytes(tc) > (size_t)200 * 1024) return g;
+        g.tc = tc;
+        while ((1 << g.shift) < tc) ++g.shift;
+        g.pitch = pitch;
+        g.sh = bytes(tc);
+        return g;
     };
-    const int strip_tc_r = fused ? 0 : strip_width(cols, rows);  // walk along a lattice row, strip of rows
-    const int strip_tc_c = fused ? 0 : strip_width(rows, cols);  // walk down a lattice column, strip of columns
-    const bool strip = !fused && strip_tc_r >= 4 && strip_tc_c >= 4;
+    const StripGeom sg_r = fused ? StripGeom{0, 0, 0, 0} : strip_geom(cols, rows);  // walk along a lattice row
+    const StripGeom sg_c = fused ? StripGeom{0, 0, 0, 0} : strip_geom(rows, cols);  // walk down a lattice column
+    const bool strip = !fused && sg_r.tc > 0 && sg_c.tc > 0;
     // ---- numerator, slab by slab ------------------------------------------------------------------
     // (the per-sample masks of the hot features live behind the two slab buffers)
     uint32_t* hot_mask = reinterpret_cast<uint32_t*>(ws + 8 * mb + 2 * som_align_up((size_t)planes_per_slab * M * 4, 256));
@@ -652,7 +844,7 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
         else SOM_CK(h, cudaMemsetAsync(slab_a, 0, (size_t)planes * M * 4, st));
         if (n > 0) {
             k_upd_scatter<<<blocks_for(n), UPD_THREADS, 0, st>>>(indptr, indices, n, bmu, v0, v1, rows, cols, hot_slot,
-                                                                 slab_a, 0);
+                                                                 slab_a, strip ? 1 : 0);
             h->launches += 1;
             if (hot_slot) {
                 int ppb = (int)((160 * 1024) / (M * 4));
@@ -663,7 +855,7 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
                 const size_t sh = (size_t)ppb * M * 4;
                 SOM_CK(h, cudaFuncSetAttribute(k_upd_scatter_hot, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh));
                 k_upd_scatter_hot<<<dim3(slices, groups), 1024, sh, st>>>(hot_mask, n, bmu, v0, v1, rows, cols, slot_feat,
-                                                                        n_hot_slots, ppb, slab_a);
+                                                                        n_hot_slots, ppb, slab_a, strip ? 1 : 0);
                 h->launches += 1;
             }
         }
@@ -699,39 +891,26 @@ int som_launch_update(som_handle* h, int rows, int cols, const int32_t* indptr, 
             continue;
         }
         if (strip) {
-            // slab_a holds the counts in transposed cell order: [plane][cols][rows]
-            const int seg_r = STRIP_THREADS / strip_tc_r, seg_c = STRIP_THREADS / strip_tc_c;
-            const size_t sh_r = (size_t)cols * (strip_tc_r | 1) * sizeof(STRIP_BT) * 2;
-            const size_t sh_c = (size_t)rows * (strip_tc_c | 1) * sizeof(STRIP_BT) * 2;
-            const bool tot_r = 2 * radius + 1 > 3 * ((cols + seg_r - 1) / seg_r);
-            const bool tot_c = 2 * radius + 1 > 3 * ((rows + seg_c - 1) / seg_c);
-            const int64_t items_r = planes * ((rows + strip_tc_r - 1) / strip_tc_r);
-            const int64_t items_c = planes * ((cols + strip_tc_c - 1) / strip_tc_c);
+            // slab_a holds the counts in neuron order
             auto grid_for = [&](size_t sh, int64_t items) {
-                int per_sm = (int)((size_t)220 * 1024 / (sh + 3072));
-                per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+                int per_sm = (int)((size_t)226 * 1024 / (sh + 1024));
+                per_sm = per_sm < 1 ? 1 : (per_sm > 3 ? 3 : per_sm);  // (the kernel's launch bound: three blocks)
                 const int64_t g = (int64_t)h->sm_count * per_sm;
                 return (unsigned)(g < items ? g : items);
             };
-#define SOM_STRIP(ST_, TOT_, FINAL_, IN_, OUT_, LEN_, WIDTH_, TC_, SEG_, SH_, ITEMS_, W_)                          \
+            const int64_t items_r = planes * ((rows + sg_r.tc - 1) / sg_r.tc);
+            const int64_t items_c = planes * ((cols + sg_c.tc - 1) / sg_c.tc);
+#define SOM_STRIP(ST_, ROWS_, IN_, OUT_, LEN_, WIDTH_, G_, ITEMS_, W_)                                           \
     do {                                                                                                         \
-        SOM_CK(h, cudaFuncSetAttribute(k_upd_strip<ST_, TOT_, FINAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                       (int)(SH_)));                                                             \
-        k_upd_strip<ST_, TOT_, FINAL_><<<grid_for(SH_, ITEMS_), STRIP_THREADS, SH_, st>>>(                        \
-            IN_, OUT_, planes, LEN_, WIDTH_, radius, TC_, SEG_, rden, W_, v0);                                     \
+        SOM_CK(h, cudaFuncSetAttribute(k_upd_strip<ST_, ROWS_>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+                                       (int)(G_).sh));                                                           \
+        k_upd_strip<ST_, ROWS_><<<grid_for((G_).sh, ITEMS_), STRIP_THREADS, (G_).sh, st>>>(                      \
+            IN_, OUT_, planes, LEN_, WIDTH_, radius, (G_).tc, (G_).shift, (G_).pitch, rden, W_, v0);            \
     } while (0)
             float* none_w = nullptr;
-            if (tot_r) SOM_STRIP(float, true, false, slab_a, slab_b, cols, rows, strip_tc_r, seg_r, sh_r, items_r, none_w);
-            else SOM_STRIP(float, false, false, slab_a, slab_b, cols, rows, strip_tc_r, seg_r, sh_r, items_r, none_w);
-            if (h->Wh) {
-                __half* wh = const_cast<__half*>(h->Wh);
-                if (tot_c) SOM_STRIP(__half, true, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wh);
-                else SOM_STRIP(__half, false, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wh);
-            } else {
-                float* wf = const_cast<float*>(h->W);
-                if (tot_c) SOM_STRIP(float, true, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wf);
-                else SOM_STRIP(float, false, true, slab_b, nullptr, rows, cols, strip_tc_c, seg_c, sh_c, items_c, wf);
-            }
+            SOM_STRIP(float, true, slab_a, slab_b, cols, rows, sg_r, items_r, none_w);
+            if (h->Wh) SOM_STRIP(__half, false, slab_b, nullptr, rows, cols, sg_c, items_c, const_cast<__half*>(h->Wh));
+            else SOM_STRIP(float, false, slab_b, nullptr, rows, cols, sg_c, items_c, const_cast<float*>(h->W));
 #undef SOM_STRIP
             h->launches += 2;
             SOM_CK(h, cudaGetLastError());
