@@ -171,6 +171,19 @@ def test_update_with_frequent_features_counted_on_chip(som_mod, mib):
     _check(got, W_old, w.V, rows, cols, b.indptr.numpy(), b.indices.numpy(), bmu, 2, rtol=1e-6)
 
 
+def test_update_with_frequent_features_on_the_strip_route(som_mod):
+    """A 130 x 130 lattice (above the on-chip blur, so the strip kernels run, which take the counts in neuron
+    order) with enough Zipf-shaped samples for the frequent features' shared-memory counting path: both
+    scatters must write the order the strips read."""
+    V, rows, cols = 300, 130, 130
+    rng = np.random.default_rng(21)
+    W_old = rng.random(V * rows * cols).astype(np.float32)
+    b = synth.sample_csr(150_000, V, 6.0, 8, device="cpu")
+    bmu = rng.integers(0, rows * cols, size=b.n).astype(np.int32)
+    got = _run(som_mod, W_old, V, rows, cols, b.indptr.numpy(), b.indices.numpy(), bmu, 5)
+    _check(got, W_old, V, rows, cols, b.indptr.numpy(), b.indices.numpy(), bmu, 5, rtol=1e-6)
+
+
 def test_update_at_benchmark_shape(som_mod):
     """The shape the benchmark times: a 64 x 64 lattice, V = 30 000, one million Zipf-shaped samples,
     radius 16 (edge / 4).  The frequent features take the on-chip counting path, the blur runs fused
