@@ -317,8 +317,8 @@ int som_last_cuda_error(const som_handle* h);
  *          som_last_uncertain returns how many samples the last two-stage search sent to its second pass (all
  *          of them when the probe chose the plain search); the figure travels back unwaited for and is valid
  *          once the call's stream has been synchronised.
- *   keys 1 to 4 and 8 are tunables of the row-table kernel and its plan for benchmarking (hot rows in shared
- *          memory, block size, neurons per lane, sample parts per neuron range, mask features; 0 = the measured
+ *   keys 1 to 4, 8 and 9 are tunables of the row-table kernel and its plan for benchmarking (hot rows in shared
+ *          memory, block size, neurons per lane, sample parts per neuron range, mask features, L2 policy of the slot stream; 0 = the measured
  *          default): described in
  *          paper_2608_24067_b200/csrc/som_tuning.h.  Callers need not touch them; a plan (som_plan_create) is
  *          tied to their values at its creation.

@@ -924,6 +924,11 @@ int som_set_option(som_handle* h, int key, int64_t value)
         h->opt_parts = value;
         return SOM_OK;
     }
+    if (key == 9) {
+        if (value < 0 || value > 2) return SOM_ERR_INVALID_ARG;
+        h->opt_feed_keep = value;
+        return SOM_OK;
+    }
     if (key == 8) {
         if (value < 0 || value > SOM_PLAN_MASK_FEATURES) return SOM_ERR_INVALID_ARG;
         h->opt_mask_bits = value;

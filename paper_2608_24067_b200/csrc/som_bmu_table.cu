@@ -128,6 +128,20 @@ __device__ __forceinline__ Acc<H> ldg_acc(const float* p)
     return r;
 }
 
+// 128-bit load of slot or key bytes past L1 (the keys change under atomics).  `keep` asks L2 to evict the line
+// last: on a small batch the whole slot and key stream then stays L2-resident from one neuron range to the
+// next instead of being fetched from device memory once per range.
+__device__ __forceinline__ uint4 ld_feed(const uint4* p, uint64_t keep_policy)
+{
+    uint4 v;
+    if (keep_policy)
+        asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(keep_policy));
+    else
+        v = __ldcg(p);
+    return v;
+}
+
 __device__ __forceinline__ uint32_t lo16(uint32_t w) { return w & 0xffffu; }
 __device__ __forceinline__ uint32_t hi16(uint32_t w) { return w >> 16; }
 
@@ -427,9 +441,11 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const uint4* __restrict__ slots, int64_t n_pad,
             u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
             int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter,
-            const int* __restrict__ gate, int gate_want)
+            const int* __restrict__ gate, int gate_want, int feed_keep_arg)
 {
     if (som_gated_off(gate, gate_want)) return;
+    uint64_t feed_keep = 0;  // L2 cache policy "evict last" for the slot and key stream, or none
+    if (feed_keep_arg) asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(feed_keep));
     constexpr bool TOP2 = KEEP >= 2;
     constexpr int R = L::R;
     constexpr int T = L::T;
@@ -539,8 +555,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             uint4 g = make_uint4(0u, 0u, 0u, 0u);
             __syncwarp();  // the previous chunk's last reads of the ring are done
             if (feeder) {
-                *reinterpret_cast<uint4*>(my_store) = __ldcg(feed);  // round 0 -> stage 0
-                g = __ldcg(feed + feed_step);                        // round 1, in flight
+                *reinterpret_cast<uint4*>(my_store) = ld_feed(feed, feed_keep);  // round 0 -> stage 0
+                g = ld_feed(feed + feed_step, feed_keep);             // round 1, in flight
             }
             feed += 2 * feed_step;
             __syncwarp();
@@ -556,7 +572,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 // are padded, so the loads past the chunk's end stay in bounds.
                 if (feeder) {
                     *reinterpret_cast<uint4*>(my_store + (RING_STAGE - st)) = g;
-                    g = __ldcg(feed);
+                    g = ld_feed(feed, feed_keep);
                 }
                 feed += feed_step;
                 __syncwarp();
@@ -769,7 +785,8 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
                                       KEEP >= 2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr,
                                       KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
                                       n_units, n_whole,
-                                      reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want);
+                                      reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want,
+                                      h->opt_feed_keep == 1 || (h->opt_feed_keep == 0 && n * 56 <= ((int64_t)24 << 20)));
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

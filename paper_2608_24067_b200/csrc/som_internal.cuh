@@ -69,6 +69,7 @@ struct som_handle {
     int64_t opt_threads;   // block size of the row-table kernel: 0 (default 512), 512 or 1024
     int64_t opt_r;         // neurons per lane of the row-table kernel: 0 = default, 4, 8 or 16
     int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
+    int64_t opt_feed_keep; // row-table kernel: slot stream kept in L2 (0 = by batch size, 1 = always, 2 = never)
     int64_t opt_mask_bits; // plan: features handled as mask bits (0 = default by batch size, else 1..16)
     int plan_attr_set;
     int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)
