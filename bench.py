@@ -229,6 +229,9 @@ class Ctx:
         self.add_peak = self.sm_count * FP32_LANES_PER_SM * self.sm_max_mhz * 1e6  # adds/s, derived
         # the same peak measured: independent FP32 add chains, nothing else (library microbenchmark)
         self.add_peak_measured = som.measure_fadd_peak(self.dev)
+        # bytes per clock and SM along the paths an add's operand takes (shared memory, L2): what the search
+        # kernel's time per sample is made of (library microbenchmark, about 40 ms)
+        self.operand_paths = som.measure_operand_paths(self.dev)
 
     def barrier(self):
         if self.dist is not None:
@@ -478,6 +481,10 @@ def measure(ctx: Ctx, args, w: synth.Workload, steps: int, warmup: int, cpu_seco
             "norms_hbm_frac": (w.V * w.M * store_bytes / max(phases["norms_ms"], 1e-6) / 1e6) / hbm_gbs,
             "plan_ms": phases["plan_ms"], "finalize_ms": phases["finalize_ms"],
             "step_frac_of_alu_roofline": (adds / add_peak) / (ms_per_step * 1e-3),
+            # operand delivery, the unit that really bounds the kernel: measured bytes per clock and SM from
+            # shared memory (hot rows) and from L2 (tail rows), and the search's SM clocks per sample and 128 neurons
+            "operand_paths_bytes_per_clk_per_sm": ctx.operand_paths,
+            "sm_clk_per_sample_and_128_neurons": search_s * ctx.sm_max_mhz * 1e6 * ctx.sm_count / (w.batch * w.M / 128.0),
         }
 
         # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ------------------
@@ -537,7 +544,8 @@ def _summary(line: dict) -> dict:
             "warmup": line["warmup"], "ms_per_step": line["ms_per_step"], "value": line["value"],
             "accumulations_per_s": line["accumulations_per_s"],
             "roofline": {"bound": r["bound"], "frac": r["frac"], "frac_of_measured_peak": r["frac_of_measured_peak"],
-                         "achieved": r["achieved"], "traffic": r["traffic"]},
+                         "achieved": r["achieved"], "traffic": r["traffic"],
+                         "sm_clk_per_sample_and_128_neurons": r["sm_clk_per_sample_and_128_neurons"]},
             "search_ms": r["search_ms"], "norms_ms": r["norms_ms"], "norms_hbm_frac": r["norms_hbm_frac"],
             "plan_ms": r["plan_ms"], "finalize_ms": r["finalize_ms"],
             "e2e": {k: line["e2e"][k] for k in ("value", "ms_per_step", "blocking_ms_per_step",
@@ -628,6 +636,27 @@ def run_tc_probe(args):
                               "workload's H most frequent features"}), flush=True)
 
 
+def run_operand_probe():
+    """Bytes per clock and SM along the paths an operand takes into a register (library microbenchmark), and
+    what they make of a sample of the headline workload: clocks per sample and 128-neuron range if every hot
+    row came at the shared-memory rate and every tail row at the L2 rate, one after the other."""
+    from paper_2608_24067_b200 import som
+    som.load_library()
+    torch.cuda.set_device(0)
+    p = som.measure_operand_paths()
+    # rows per sample of the MeSH-shaped batches with the 368-row table (hot rows as issued, i.e. padded to the
+    # warp's longest list, and prefix rebuilds; tail rows), by batch size and its number of mask features
+    mix = {"250k samples, 9 mask features": (4.85, 3.92), "1M samples, 11": (4.60, 3.93), "4M samples, 13": (4.40, 3.93)}
+    model = {}
+    for name, (hot_rows, tail_rows) in mix.items():
+        t_sh, t_l2 = 512.0 * hot_rows / p["shared"], 512.0 * tail_rows / p["l2_global"]
+        model[name] = {"hot_rows": hot_rows, "tail_rows": tail_rows, "clk_shared": t_sh, "clk_l2": t_l2,
+                       "clk_one_after_the_other": t_sh + t_l2, "clk_fully_overlapped": max(t_sh, t_l2),
+                       "clk_at_the_probe's_two-stream_rate": 512.0 * (hot_rows + tail_rows) / p["shared_and_l2"]}
+    print(json.dumps({"probe": "operand paths, 512-byte rows, eight lanes per row, one 512-thread block per SM",
+                      "bytes_per_clk_per_sm": p, "model_clk_per_sample_and_128_neuron_range": model}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -675,10 +704,16 @@ def main():
                          "profiler captures that must hold few GB; named in the workload)")
     ap.add_argument("--tc-probe", action="store_true",
                     help="run the tcgen05 microbenchmark of the densified hot-feature tile and print its numbers")
+    ap.add_argument("--operand-probe", action="store_true",
+                    help="run the microbenchmark of the operand paths (shared memory, L2 by global loads, both, "
+                         "L2 by texture fetches: bytes per clock and SM) and print its numbers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.tc_probe:
         run_tc_probe(args)
+        return
+    if args.operand_probe:
+        run_operand_probe()
         return
 
     def variant_of(w):

@@ -334,6 +334,24 @@ int som_last_cuda_error(const som_handle* h);
 int som_measure_fadd_peak(double* adds_per_s, float* d_scratch, int64_t scratch_elems, void* stream);
 
 /*
+ * som_measure_operand_paths - measure how many bytes per clock and SM reach registers along the paths that an
+ * add's operand takes in the row-table search kernel (no counterpart in the paper; Section 5.7 only says that
+ * its kernel executes adds and no multiplies: what bounds such a kernel is operand delivery).  One block of 512
+ * threads per SM reads 512-byte rows, eight lanes per row, as that kernel's wide fp32 layout does:
+ *   bytes_per_clk[0]  rows of a 180 KB table in shared memory,
+ *   bytes_per_clk[1]  rows of the caller's buffer with read-only global loads (L2-resident when the buffer is a
+ *                     few tens of MB),
+ *   bytes_per_clk[2]  both streams in one loop (the sum of both streams' bytes over the loop's time),
+ *   bytes_per_clk[3]  the buffer's rows through a linear texture.
+ * Times with the SM cycle counter, mean over the blocks.  Synchronises.
+ *   n_out          length of bytes_per_clk, at least 4.
+ *   d_rows         DEVICE pointer, 512-byte aligned, rows_bytes bytes (512 .. 2^31) of finite fp32 values; read.
+ *   d_scratch      DEVICE pointer, fp32, at least 514 * (number of SMs) + 2 elements; written.
+ */
+int som_measure_operand_paths(double* bytes_per_clk, int n_out, const void* d_rows, int64_t rows_bytes,
+                              float* d_scratch, int64_t scratch_elems, void* stream);
+
+/*
  * som_tc_probe - measured probe of a densified hot-feature tile on the tensor cores (no counterpart in
  * the paper, whose kernels run on plain CUDA cores; Section 3.3 is the gather it restates).  For the H
  * most frequent features of a batch the gather-sum of a tile of 128 samples over 64 neurons is the dense

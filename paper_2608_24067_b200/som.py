@@ -26,7 +26,7 @@ EXPORTS = [
     "som_destroy", "som_status_string", "som_last_cuda_error", "som_set_timing", "som_get_timing",
     "som_launch_count", "som_set_option", "som_norms_noalloc", "som_bmu2", "som_create_f16", "som_update", "som_last_uncertain", "som_bmu_values",
     "som_bmu_host_async", "som_host_sync", "som_plan_create", "som_bmu_planned", "som_plan_destroy",
-    "som_device_flags", "som_measure_fadd_peak", "som_tc_probe",
+    "som_device_flags", "som_measure_fadd_peak", "som_measure_operand_paths", "som_tc_probe",
 ]
 
 NOALLOC_MAX_M = 524288
@@ -92,6 +92,8 @@ def load_library():
     lib.som_set_option.argtypes = [P, INT, I64]
     lib.som_measure_fadd_peak.argtypes = [ctypes.POINTER(ctypes.c_double), P, I64, P]
     lib.som_measure_fadd_peak.restype = INT
+    lib.som_measure_operand_paths.argtypes = [ctypes.POINTER(ctypes.c_double), INT, P, I64, P, I64, P]
+    lib.som_measure_operand_paths.restype = INT
     lib.som_tc_probe.argtypes = [P, P, P, I32, I32, I32, I32, I32, I32, P, P, P, P, P]
     lib.som_tc_probe.restype = INT
     lib.som_device_flags.argtypes = [P, P]
@@ -137,6 +139,23 @@ def norms_noalloc(V: int, M: int, codebook: torch.Tensor, out: torch.Tensor, str
     if rc != SOM_OK:
         raise SomError(rc, "som_norms_noalloc")
     return out
+
+
+def measure_operand_paths(device=None, stream=None, buffer_mb: int = 16) -> dict:
+    """som_measure_operand_paths: bytes per clock and SM that reach registers from shared memory, from an
+    L2-resident buffer (global loads), from both at once, and through a linear texture."""
+    lib = load_library()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        rows = torch.zeros(buffer_mb << 18, dtype=torch.float32, device=dev)
+        scratch = torch.empty(514 * sms + 2, dtype=torch.float32, device=dev)
+        out = (ctypes.c_double * 4)()
+        rc = lib.som_measure_operand_paths(out, 4, rows.data_ptr(), rows.numel() * 4, scratch.data_ptr(),
+                                           scratch.numel(), _stream_ptr(stream))
+    if rc != SOM_OK:
+        raise SomError(rc, "som_measure_operand_paths")
+    return {"shared": float(out[0]), "l2_global": float(out[1]), "shared_and_l2": float(out[2]), "l2_texture": float(out[3])}
 
 
 def measure_fadd_peak(device=None, stream=None) -> float:
