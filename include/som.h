@@ -82,6 +82,10 @@ int som_create_f16(som_handle** out, int32_t V, int64_t M, const void* d_codeboo
  * pass whose cost Section 5.7 reports as negligible).  One streaming read of the codebook; squares are
  * accumulated in fp64 in a fixed order (deterministic) and stored as fp32.
  * Must be called once after som_create and again after every codebook update.
+ * With fp32 storage and M % 128 == 0 the same read also records, for every feature and every range of 128
+ * neurons, the largest weight (V * M / 128 floats, allocated by the first call; if that memory cannot be had
+ * the call carries on without them).  The search uses them to skip rows that cannot change a sample's result
+ * (som_bmu below); they cost the norm pass nothing measurable.
  */
 int som_norms(som_handle* h, void* stream);
 
@@ -111,6 +115,12 @@ int som_norms(som_handle* h, void* stream);
  * summation order, about one assignment in 1e5 at 256x256).  Wherever the two best units are
  * further apart than 1e-4 of the best squared distance the unit is the same in every batch.
  * The reported distance is always the fp64 one of the reported unit.
+ * Not every row of the sparse x dense product is formed: where som_norms has recorded the per-range
+ * maxima (fp32 storage, M % 128 == 0; by default on maps of at least 65 536 neurons), the kernel skips
+ * a sample's infrequent-feature rows for a range of 128 neurons when even the range's smallest partial
+ * score, lowered by those features' largest weights in the range, stays above the sample's best score so
+ * far, with a margin for fp32 rounding: no neuron of the range can then be the best unit.  The outputs
+ * are bit for bit those of the search that forms every row (tests/test_gpu_parity.py forces it both ways).
  */
 int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
             int32_t* d_bmu, float* d_min_dist, void* stream);
@@ -317,8 +327,8 @@ int som_last_cuda_error(const som_handle* h);
  *          som_last_uncertain returns how many samples the last two-stage search sent to its second pass (all
  *          of them when the probe chose the plain search); the figure travels back unwaited for and is valid
  *          once the call's stream has been synchronised.
- *   keys 1 to 4, 8 and 9 are tunables of the row-table kernel and its plan for benchmarking (hot rows in shared
- *          memory, block size, neurons per lane, sample parts per neuron range, mask features, L2 policy of the slot stream; 0 = the measured
+ *   keys 1 to 4 and 8 to 10 are tunables of the row-table kernel and its plan for benchmarking (hot rows in shared
+ *          memory, block size, neurons per lane, sample parts per neuron range, mask features, L2 policy of the slot stream, pruning by range maxima; 0 = the measured
  *          default): described in
  *          paper_2608_24067_b200/csrc/som_tuning.h.  Callers need not touch them; a plan (som_plan_create) is
  *          tied to their values at its creation.

@@ -131,6 +131,7 @@ int som_destroy(som_handle* h)
     cudaFree(h->stage);
     cudaFree(h->head);
     cudaFree(h->shadow);
+    cudaFree(h->range_max);
     if (h->aux_stream) {
         cudaStreamSynchronize(h->aux_stream);
         cudaEventDestroy(h->ev_fork);
@@ -165,6 +166,15 @@ int som_norms(som_handle* h, void* stream)
     int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, som_norms_workspace_bytes(h));
     if (rc) return rc;
     if (h->timing && (rc = ensure_events(h))) return rc;
+    // per-range maxima of the feature rows for the search's pruning (fp32 storage, M % 128 == 0): V * M / 128
+    // floats, allocated by the first call; without the memory the search simply does not prune
+    if (!h->range_max && !h->Wh && h->M % 128 == 0 && h->opt_prune != 2) {
+        if (cudaMalloc(reinterpret_cast<void**>(&h->range_max), (size_t)h->V * (size_t)(h->M / 128) * sizeof(float)) !=
+            cudaSuccess) {
+            h->range_max = nullptr;
+            (void)cudaGetLastError();
+        }
+    }
     if ((rc = mark(h, h->ev_norms_calls, EV_NORMS_BEGIN, st))) return rc;
     if ((rc = som_launch_norms(h, st))) return rc;
     h->shadow_valid = h->shadow != nullptr && h->M % 4 == 0;
@@ -922,6 +932,11 @@ int som_set_option(som_handle* h, int key, int64_t value)
     if (key == 4) {
         if (value < 0 || value > 1024) return SOM_ERR_INVALID_ARG;
         h->opt_parts = value;
+        return SOM_OK;
+    }
+    if (key == 10) {
+        if (value < 0 || value > 2) return SOM_ERR_INVALID_ARG;
+        h->opt_prune = value;
         return SOM_OK;
     }
     if (key == 9) {

@@ -39,6 +39,7 @@
 
 namespace {
 
+constexpr int SOM_PRUNE_MIN_RANGES = 512;  // pruning by range maxima from this many neuron ranges (see launch_table)
 constexpr int CHUNK = 128;  // samples a warp takes at a time ...
 constexpr int SMALL_CHUNK = 32;  // ... and near the end of a unit, so that its warps finish together
 constexpr int RING_STAGE = 224;  // bytes of one ring stage: 4 slots + 4 keys
@@ -198,6 +199,7 @@ struct LayF32 {
     // neurons per lane three fit 128 registers at the price of a 36-byte spill, and measure 1 to 3 % faster
     // than two)
     static constexpr int TAILS_AHEAD = R_ >= 16 ? 3 : 4;
+    static constexpr bool CAN_PRUNE = true;     // scores are held as they are: a lower bound on them is one on the result
     static constexpr float SEED_SIGN = 1.f;     // scores are held as they are
     typedef Acc<H> Scores;
     typedef Acc<H> Slice;
@@ -269,6 +271,7 @@ struct LayF16 {
     typedef __half Store;
     static constexpr int R = 8, T = 64, ROWB = T * 2;
     static constexpr int TAILS_AHEAD = 4;
+    static constexpr bool CAN_PRUNE = false;
     static constexpr float SEED_SIGN = -1.f;  // the seed array holds -||w||^2/2
     struct Scores { float v[8]; };
     typedef uint4 Slice;
@@ -345,6 +348,7 @@ struct LayF16W {
     typedef __half Store;
     static constexpr int R = 16, T = 128, ROWB = T * 2;
     static constexpr int TAILS_AHEAD = 4;
+    static constexpr bool CAN_PRUNE = false;
     static constexpr float SEED_SIGN = -1.f;
     struct Scores { float v[16]; };
     struct Slice { uint4 g[2]; };
@@ -434,14 +438,14 @@ struct LayF16W {
 // one sample).  KEEP = 2 also keeps the second-best unit of every sample in keys2 (Algorithm 2 keeps the two
 // best units); the candidate filter then tests against the second-best score.
 // KEEP = 3 (first pass of the two-stage two-best search) keeps the third best as well, in keys3.
-template <typename L, int THREADS, int KEEP>
+template <typename L, int THREADS, int KEEP, bool PRUNE>
 __global__ void __launch_bounds__(THREADS, 1)
 k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ hnorm, int64_t M,
             const int32_t* __restrict__ slot_feat, int n_rows,
             const uint4* __restrict__ slots, int64_t n_pad,
             u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
             int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter,
-            const int* __restrict__ gate, int gate_want, int feed_keep_arg)
+            const int* __restrict__ gate, int gate_want, int feed_keep_arg, const float* __restrict__ range_max, int V)
 {
     if (som_gated_off(gate, gate_want)) return;
     uint64_t feed_keep = 0;  // L2 cache policy "evict last" for the slot and key stream, or none
@@ -474,6 +478,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
         reinterpret_cast<uint32_t*>(tab)[n_rows * (ROWB / 4) + c] = 0u;
 
     int cur_range = -1;
+    const float* rmax_range = nullptr;  // (pruning) largest weight of every feature row in the live 128-neuron range
     const unsigned char* w_q = reinterpret_cast<const unsigned char*>(W);
     uint32_t i_first = 0;
     for (;;) {
@@ -509,6 +514,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const int64_t i_lane = i0 + L::lane_first(q);
             i_first = (uint32_t)i_lane;
             w_q = reinterpret_cast<const unsigned char*>(W + (i_lane < M ? i_lane : 0));
+            if constexpr (PRUNE) rmax_range = range_max + (i0 >> 7) * (int64_t)V;
             for (int c = threadIdx.x; c < T; c += THREADS)
                 hn_sh[c] = L::SEED_SIGN * ((i0 + c < M) ? hnorm[i0 + c] : inf);
         }
@@ -582,15 +588,26 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 const uint32_t mask = hdr & 0xffffu;
                 const bool p0 = nt > 0, p1 = nt > 1, p2 = nt > 2, p3 = nt > 3;
 
-                // ---- the first four tail rows of this sample go in flight first ---------------
+                // ---- the first tail rows of this sample go in flight first; with pruning, only the bounds
+                //      on what the tail rows can take off this range's scores (one 4-byte load per lane:
+                //      lane q of the team reads the range maximum of tail feature q, and of q + 8)
                 Slice tr0, tr1, tr2, tr3;
-                if (p0) tr0 = SOM_TAIL(lo16(s2.x));
-                if (p1) tr1 = SOM_TAIL(hi16(s2.x));
-                if constexpr (L::TAILS_AHEAD >= 3) {
-                    if (p2) tr2 = SOM_TAIL(lo16(s2.y));
-                }
-                if constexpr (L::TAILS_AHEAD >= 4) {
-                    if (p3) tr3 = SOM_TAIL(hi16(s2.y));
+                float bnd = 0.f;
+                if constexpr (PRUNE) {
+                    const uint32_t ntc = nt == SOM_SLOT_NT_OVERFLOW ? 0u : nt;
+                    if ((uint32_t)q < ntc)
+                        bnd = __ldg(rmax_range + *reinterpret_cast<const uint16_t*>(my_slot + st + 32 + 2 * q));
+                    if ((uint32_t)q + 8u < ntc)
+                        bnd += __ldg(rmax_range + *reinterpret_cast<const uint16_t*>(my_slot + st + 4 + 2 * q));
+                } else {
+                    if (p0) tr0 = SOM_TAIL(lo16(s2.x));
+                    if (p1) tr1 = SOM_TAIL(hi16(s2.x));
+                    if constexpr (L::TAILS_AHEAD >= 3) {
+                        if (p2) tr2 = SOM_TAIL(lo16(s2.y));
+                    }
+                    if constexpr (L::TAILS_AHEAD >= 4) {
+                        if (p3) tr3 = SOM_TAIL(hi16(s2.y));
+                    }
                 }
 
                 // ---- mask prefix ------------------------------------------------------------
@@ -625,26 +642,76 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     default: break;
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
+                const uint32_t cu = (uint32_t)(key0 >> 32);
+                const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
+                pk += 4;
+
+                // ---- pruning (fp32 storage, range maxima from som_norms): the tail rows lower a score by at most
+                //      the sum of their largest weights in this range.  If even the smallest score of the team's
+                //      neurons, lowered by that much, stays above the sample's key (with a margin for the rounding
+                //      of the sums), no neuron of this range can become a candidate, whatever the tail rows hold:
+                //      they are not loaded.  The result is that of the full search, bit for bit (a neuron that
+                //      is skipped would have lost the comparison below).  A live sample's tail rows go out only
+                //      now, four at a time: their latency is no longer hidden behind the hot rows, which is why
+                //      the launcher prunes only where nearly all pairs of sample and range are skipped.
+                constexpr int TA = PRUNE ? 4 : L::TAILS_AHEAD;
+                if constexpr (PRUNE) {
+                    bnd += __shfl_xor_sync(0xffffffffu, bnd, 1);
+                    bnd += __shfl_xor_sync(0xffffffffu, bnd, 2);
+                    bnd += __shfl_xor_sync(0xffffffffu, bnd, 4);
+                    float h[R];
+                    L::unpack(acc, h);
+                    float lo = fminf(fminf(h[0], h[1]), fminf(h[2], h[3]));
+                    if (R >= 8) lo = fminf(lo, fminf(fminf(h[4 % R], h[5 % R]), fminf(h[6 % R], h[7 % R])));
+                    if (R == 16) {
+                        lo = fminf(lo, fminf(fminf(h[8 % R], h[9 % R]), fminf(h[10 % R], h[11 % R])));
+                        lo = fminf(lo, fminf(fminf(h[12 % R], h[13 % R]), fminf(h[14 % R], h[15 % R])));
+                    }
+                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, 1));
+                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, 2));
+                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, 4));
+                    // (an empty key decodes to NaN: the comparison is false and the sample stays live)
+                    const bool live = nt != SOM_SLOT_NT_OVERFLOW &&
+                                      !(lo - bnd > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd)));
+                    if (!live) continue;
+                    if (p0) tr0 = SOM_TAIL(lo16(s2.x));
+                    if (p1) tr1 = SOM_TAIL(hi16(s2.x));
+                    if (p2) tr2 = SOM_TAIL(lo16(s2.y));
+                    if (p3) tr3 = SOM_TAIL(hi16(s2.y));
+                }
 
                 // ---- tail rows ------------------------------------------------------------------
                 if (p0) L::sub(acc, tr0);
                 if (p1) L::sub(acc, tr1);
-                if constexpr (L::TAILS_AHEAD >= 3) {
+                if constexpr (TA >= 3) {
                     if (p2) L::sub(acc, tr2);
                 } else {
                     if (p2) L::sub(acc, SOM_TAIL(lo16(s2.y)));
                 }
-                if constexpr (L::TAILS_AHEAD >= 4) {
+                if constexpr (TA >= 4) {
                     if (p3) L::sub(acc, tr3);
                 } else {
                     if (p3) L::sub(acc, SOM_TAIL(hi16(s2.y)));
                 }
                 if (nt > 4) {
                     if (nt != SOM_SLOT_NT_OVERFLOW) {
-                        L::sub(acc, SOM_TAIL(lo16(t45)));
-                        if (nt > 5) L::sub(acc, SOM_TAIL(hi16(t45)));
-                        if (nt > 6) L::sub(acc, SOM_TAIL(lo16(t67)));
-                        if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
+                        if constexpr (PRUNE) {
+                            // nothing was loaded ahead of the decision: the next four go out together
+                            const bool p5 = nt > 5, p6 = nt > 6, p7 = nt > 7;
+                            tr0 = SOM_TAIL(lo16(t45));
+                            if (p5) tr1 = SOM_TAIL(hi16(t45));
+                            if (p6) tr2 = SOM_TAIL(lo16(t67));
+                            if (p7) tr3 = SOM_TAIL(hi16(t67));
+                            L::sub(acc, tr0);
+                            if (p5) L::sub(acc, tr1);
+                            if (p6) L::sub(acc, tr2);
+                            if (p7) L::sub(acc, tr3);
+                        } else {
+                            L::sub(acc, SOM_TAIL(lo16(t45)));
+                            if (nt > 5) L::sub(acc, SOM_TAIL(hi16(t45)));
+                            if (nt > 6) L::sub(acc, SOM_TAIL(lo16(t67)));
+                            if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
+                        }
                         if (nt > 8) L::sub(acc, SOM_TAIL(lo16(s0.y)));
                         if (nt > 9) L::sub(acc, SOM_TAIL(hi16(s0.y)));
                     } else {
@@ -657,8 +724,6 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     }
                 }
 
-                pk += 4;
-
                 // ---- lane-local argmin, rare atomic combine ------------------------------------
                 float a[R];
                 L::unpack(acc, a);
@@ -668,8 +733,6 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     mn = fminf(mn, fminf(fminf(a[8 % R], a[9 % R]), fminf(a[10 % R], a[11 % R])));
                     mn = fminf(mn, fminf(fminf(a[12 % R], a[13 % R]), fminf(a[14 % R], a[15 % R])));
                 }
-                const uint32_t cu = (uint32_t)(key0 >> 32);
-                const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
                 if (!(mn > cs)) {
                     int rr = R - 1;
 #pragma unroll
@@ -773,20 +836,39 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     const int n_whole = (int)n_units64 - n_split;
     if (n_units64 + 3 * (int64_t)n_split > 0x7fffffff) return SOM_ERR_UNSUPPORTED;
     const int n_units = n_whole + 4 * n_split;
-    auto kern = k_bmu_table<L, THREADS, KEEP>;
     const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
-    SOM_CK(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<grid, THREADS, smem, st>>>(codebook, h->hnorm, h->M,
-                                      reinterpret_cast<const int32_t*>(head + b.slot_feat),
-                                      SOM_PLAN_MASK_FEATURES + n_hot,
-                                      reinterpret_cast<const uint4*>(ws + b.slots),
-                                      n,
-                                      reinterpret_cast<u64*>(ws + b.keys),
-                                      KEEP >= 2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr,
-                                      KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
-                                      n_units, n_whole,
-                                      reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want,
-                                      h->opt_feed_keep == 1 || (h->opt_feed_keep == 0 && n * 56 <= ((int64_t)24 << 20)));
+    const int feed_keep = h->opt_feed_keep == 1 || (h->opt_feed_keep == 0 && n * 56 <= ((int64_t)24 << 20));
+    // Pruning by range maxima: fp32 storage, when som_norms has written them (the codebook this launch reads
+    // must be the handle's own fp32 codebook, not a shadow).  It pays where nearly every pair of sample and
+    // range is skipped, which takes many ranges: measured 67 % of the pairs skipped with 32 ranges (64 x 64:
+    // 11 % slower, the live samples' tail rows now wait for L2 in the open), 77 % with 128 ranges (11 % slower),
+    // 96 % with 2048 (512 x 512: 21 % faster), 93 % with 8192 (1024 x 1024: 19 % faster).
+    bool prune = false;
+    if constexpr (L::CAN_PRUNE)
+        prune = h->range_max != nullptr && codebook_v == static_cast<const void*>(h->W) &&
+                (h->opt_prune == 1 || (h->opt_prune == 0 && n_ranges >= SOM_PRUNE_MIN_RANGES));
+    auto launch = [&](auto kern) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, THREADS, smem, st>>>(codebook, h->hnorm, h->M,
+                                          reinterpret_cast<const int32_t*>(head + b.slot_feat),
+                                          SOM_PLAN_MASK_FEATURES + n_hot,
+                                          reinterpret_cast<const uint4*>(ws + b.slots),
+                                          n,
+                                          reinterpret_cast<u64*>(ws + b.keys),
+                                          KEEP >= 2 ? reinterpret_cast<u64*>(ws + b.keys2) : nullptr,
+                                          KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
+                                          n_units, n_whole,
+                                          reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want,
+                                          feed_keep, prune ? h->range_max : nullptr, (int)h->V);
+        return cudaGetLastError();
+    };
+    if constexpr (L::CAN_PRUNE) {
+        if (prune) SOM_CK(h, launch(k_bmu_table<L, THREADS, KEEP, true>));
+        else SOM_CK(h, launch(k_bmu_table<L, THREADS, KEEP, false>));
+    } else {
+        SOM_CK(h, launch(k_bmu_table<L, THREADS, KEEP, false>));
+    }
     SOM_CK(h, cudaGetLastError());
     h->launches += 1;
     return SOM_OK;

@@ -31,6 +31,8 @@ struct som_handle {
     int64_t M;
     const float* W;    // borrowed, feature-major fp32 codebook (nullptr when stored as fp16)
     const __half* Wh;  // borrowed, feature-major fp16 codebook (som_create_f16), else nullptr
+    float* range_max;  // owned, [M / 128][V]: per feature row and 128-neuron range the largest weight (written by
+                       // som_norms when M % 128 == 0 and fp32 storage; nullptr = none); bounds for the search's pruning
     __half* shadow;    // owned fp16 copy of an fp32 codebook for the two-stage search (nullptr = none)
     unsigned int* wmax_bits;  // device, written by som_norms with the shadow: [0] float bits of max |weight|,
                               // [SOM_AUX_HAS_NEGATIVE] 1 if a weight is negative, [SOM_AUX_HMAX] float bits of max ||w||^2/2
@@ -70,6 +72,8 @@ struct som_handle {
     int64_t opt_r;         // neurons per lane of the row-table kernel: 0 = default, 4, 8 or 16
     int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
     int64_t opt_feed_keep; // row-table kernel: slot stream kept in L2 (0 = by batch size, 1 = always, 2 = never)
+    int64_t opt_prune;     // row-table kernel: skip a sample's tail rows for ranges that cannot hold its best unit
+                           // (0 = where range_max exists and the map has at least 512 ranges, 1 = wherever range_max exists, 2 = off)
     int64_t opt_mask_bits; // plan: features handled as mask bits (0 = default by batch size, else 1..16)
     int plan_attr_set;
     int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)

@@ -26,10 +26,25 @@ __device__ __forceinline__ void store_half4(__half* dst, const float4 w)
 // SHADOW (VEC == 4 only): the pass also writes an fp16 copy of the codebook and the largest
 // |weight| (as float bits, through atomicMax: non-negative floats order like their bits), which
 // the two-stage search uses for its first pass and its error bound.
-template <int VEC, bool SHADOW>
+// RMAX (VEC == 4 and M % 128 == 0 only): the pass also writes, for every feature row and every range of 128
+// neurons (the 128 neurons a warp holds), the largest weight of the row in the range: range_max[range * V + v].
+// The row-table search uses it to bound what a sample's tail features can still take off the scores of a
+// whole range (see k_bmu_table).
+__device__ __forceinline__ void store_range_max(float* __restrict__ dst, float m)
+{
+    // max over the warp in one instruction: floats ordered as signed integers
+    int key = __float_as_int(m);
+    key ^= (key >> 31) & 0x7fffffff;
+    key = __reduce_max_sync(0xffffffffu, key);
+    key ^= (key >> 31) & 0x7fffffff;
+    if ((threadIdx.x & 31) == 0) *dst = __int_as_float(key);
+}
+
+template <int VEC, bool SHADOW, bool RMAX>
 __global__ void __launch_bounds__(NORM_THREADS)
 k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_split,
-                double* __restrict__ partial, __half* __restrict__ shadow, unsigned int* __restrict__ wmax_bits)
+                double* __restrict__ partial, __half* __restrict__ shadow, unsigned int* __restrict__ wmax_bits,
+                float* __restrict__ range_max)
 {
     const int64_t i = ((int64_t)blockIdx.x * NORM_THREADS + threadIdx.x) * VEC;
     if (i >= M) return;
@@ -41,6 +56,8 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
     const float* p = W + (int64_t)v0 * M + i;
     __half* ps = SHADOW ? shadow + (int64_t)v0 * M + i : nullptr;
     float wmax = 0.f, wmin = 0.f;
+    // (RMAX: M % 128 == 0, so a warp is all inside M and holds exactly range i / 128)
+    float* pr = RMAX ? range_max + (i / 128) * (int64_t)V + v0 : nullptr;
     int v = v0;
     if (VEC == 4) {
         for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
@@ -55,6 +72,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
                     wmax = fmaxf(wmax, fmaxf(fmaxf(fabsf(w[u].x), fabsf(w[u].y)), fmaxf(fabsf(w[u].z), fabsf(w[u].w))));
                     wmin = fminf(wmin, fminf(fminf(w[u].x, w[u].y), fminf(w[u].z, w[u].w)));
                 }
+                if (RMAX) store_range_max(pr + u, fmaxf(fmaxf(w[u].x, w[u].y), fmaxf(w[u].z, w[u].w)));
                 acc[0] = fma((double)w[u].x, (double)w[u].x, acc[0]);
                 acc[1 % VEC] = fma((double)w[u].y, (double)w[u].y, acc[1 % VEC]);
                 acc[2 % VEC] = fma((double)w[u].z, (double)w[u].z, acc[2 % VEC]);
@@ -62,6 +80,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
             }
             p += (int64_t)NORM_UNROLL * M;
             if (SHADOW) ps += (int64_t)NORM_UNROLL * M;
+            if (RMAX) pr += NORM_UNROLL;
         }
         for (; v < v1; ++v) {
             float4 w = __ldcs(reinterpret_cast<const float4*>(p));
@@ -71,6 +90,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
                 wmin = fminf(wmin, fminf(fminf(w.x, w.y), fminf(w.z, w.w)));
                 ps += M;
             }
+            if (RMAX) store_range_max(pr++, fmaxf(fmaxf(w.x, w.y), fmaxf(w.z, w.w)));
             acc[0] = fma((double)w.x, (double)w.x, acc[0]);
             acc[1 % VEC] = fma((double)w.y, (double)w.y, acc[1 % VEC]);
             acc[2 % VEC] = fma((double)w.z, (double)w.z, acc[2 % VEC]);
@@ -222,14 +242,21 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
         k_norms_partial_h<1><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
     else if (p.vec == 4 && h->shadow) {
         SOM_CK(h, cudaMemsetAsync(h->wmax_bits, 0, 4 * sizeof(unsigned int), st));
-        k_norms_partial<4, true><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
-                                                                h->shadow, h->wmax_bits);
-    } else if (p.vec == 4)
-        k_norms_partial<4, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
-                                                                 nullptr, nullptr);
+        if (h->range_max)
+            k_norms_partial<4, true, true><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                          h->shadow, h->wmax_bits, h->range_max);
+        else
+            k_norms_partial<4, true, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                           h->shadow, h->wmax_bits, nullptr);
+    } else if (p.vec == 4 && h->range_max)
+        k_norms_partial<4, false, true><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                       nullptr, nullptr, h->range_max);
+    else if (p.vec == 4)
+        k_norms_partial<4, false, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                        nullptr, nullptr, nullptr);
     else
-        k_norms_partial<1, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
-                                                                 nullptr, nullptr);
+        k_norms_partial<1, false, false><<<grid, NORM_THREADS, 0, st>>>(h->W, h->M, h->V, p.rows_per_split, partial,
+                                                                        nullptr, nullptr, nullptr);
     SOM_CK(h, cudaGetLastError());
     const int64_t blocks = (h->M + 31) / 32;
     k_norms_combine<<<(unsigned)blocks, dim3(32, COMBINE_GROUPS), 0, st>>>(

@@ -144,6 +144,44 @@ def test_mask_feature_counts(som_mod, mask_bits):
         assert h.device_flags() == 0
 
 
+@pytest.mark.parametrize("lane_neurons", [4, 8, 16])
+@pytest.mark.parametrize("codebook", ["recipe", "smooth", "constant", "negative"])
+def test_pruning_by_range_maxima_changes_nothing(som_mod, lane_neurons, codebook):
+    """The row-table kernel may skip a sample's tail rows for a neuron range whose scores cannot reach the
+    sample's key (bounds from the per-range maxima that som_norms writes).  Forced on (by default it runs on
+    maps of 512 ranges and more), its outputs are bit-identical to those of the full search and match the
+    oracle: on the benchmark's codebook recipe, on a smooth map (nearly everything is skipped), on a map of
+    equal neurons (nothing can be skipped: every range ties) and on weights of both signs."""
+    V, M, n = 30_000, 2_048, 40_000
+    W = synth.fill_codebook(V, M, 5, device="cuda")
+    if codebook == "smooth":
+        ramp = torch.linspace(0.0, 1.0, M, device="cuda")
+        W = (W.view(V, M) * 0.2 + ramp[None, :] * torch.rand(V, 1, device="cuda")).reshape(-1).contiguous()
+    elif codebook == "constant":
+        W = W.view(V, M)[:, :1].repeat(1, M).reshape(-1).contiguous()
+    elif codebook == "negative":
+        W = (W - 0.3).contiguous()
+    b = synth.sample_csr(n, V, 11.0, 5, device="cuda", permute_ids=True)
+    outs = []
+    for prune in (2, 1):
+        h = som_mod.Som(V, M, W)
+        h.set_option(0, 2)
+        h.set_option(3, lane_neurons)
+        h.set_option(10, prune)
+        h.norms()
+        bmu, dist = h.bmu(b.indptr, b.indices)
+        b1, d1, b2, d2 = h.bmu2(b.indptr, b.indices)
+        torch.cuda.synchronize()
+        assert h.device_flags() == 0
+        outs.append([t.cpu().numpy() for t in (bmu, dist, b1, d1, b2, d2)])
+    for full, pruned in zip(*outs):
+        assert np.array_equal(full.view(np.uint32) if full.dtype == np.float32 else full,
+                              pruned.view(np.uint32) if pruned.dtype == np.float32 else pruned)
+    rows = np.arange(0, n, 11)
+    _check_against_oracle(W.cpu().numpy(), V, M, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
+                          outs[1][0], outs[1][1], rows)
+
+
 def test_config3_full_size_sampled_rows(som_mod):
     """128x128 map at its full size (4M samples, the benchmark's launch configuration);
     a strided sample of rows against the oracle, plus properties that hold for all rows."""
