@@ -132,14 +132,11 @@ __device__ __forceinline__ Acc<H> ldg_acc(const float* p)
 // 128-bit load of slot or key bytes past L1 (the keys change under atomics).  `keep` asks L2 to evict the line
 // last: on a small batch the whole slot and key stream then stays L2-resident from one neuron range to the
 // next instead of being fetched from device memory once per range.
-__device__ __forceinline__ uint4 ld_feed(const uint4* p, uint64_t keep_policy)
+__device__ __forceinline__ uint4 ld_feed(const uint4* p, uint64_t policy)
 {
     uint4 v;
-    if (keep_policy)
-        asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
-                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(keep_policy));
-    else
-        v = __ldcg(p);
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(policy));
     return v;
 }
 
@@ -448,8 +445,9 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const int* __restrict__ gate, int gate_want, int feed_keep_arg, const float* __restrict__ range_max, int V)
 {
     if (som_gated_off(gate, gate_want)) return;
-    uint64_t feed_keep = 0;  // L2 cache policy "evict last" for the slot and key stream, or none
+    uint64_t feed_keep;  // L2 cache policy of the slot and key stream: "evict last" on small batches, else normal
     if (feed_keep_arg) asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(feed_keep));
+    else asm("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(feed_keep));
     constexpr bool TOP2 = KEEP >= 2;
     constexpr int R = L::R;
     constexpr int T = L::T;
@@ -642,9 +640,11 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     default: break;
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
+                // the sample's key as a score (decoded here when pruning needs it, else where the argmin does)
                 const uint32_t cu = (uint32_t)(key0 >> 32);
-                const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
-                pk += 4;
+                float cs = 0.f;
+                if constexpr (PRUNE) cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
+                if constexpr (PRUNE) pk += 4;
 
                 // ---- pruning (fp32 storage, range maxima from som_norms): the tail rows lower a score by at most
                 //      the sum of their largest weights in this range.  If even the smallest score of the team's
@@ -732,6 +732,10 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 if (R == 16) {
                     mn = fminf(mn, fminf(fminf(a[8 % R], a[9 % R]), fminf(a[10 % R], a[11 % R])));
                     mn = fminf(mn, fminf(fminf(a[12 % R], a[13 % R]), fminf(a[14 % R], a[15 % R])));
+                }
+                if constexpr (!PRUNE) {
+                    pk += 4;
+                    cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
                 }
                 if (!(mn > cs)) {
                     int rr = R - 1;
