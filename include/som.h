@@ -82,7 +82,7 @@ int som_create_f16(som_handle** out, int32_t V, int64_t M, const void* d_codeboo
  * pass whose cost Section 5.7 reports as negligible).  One streaming read of the codebook; squares are
  * accumulated in fp64 in a fixed order (deterministic) and stored as fp32.
  * Must be called once after som_create and again after every codebook update.
- * With fp32 storage and M % 128 == 0 the same read also records, for every feature and every range of 128
+ * With M % 128 == 0 the same read also records, for every feature and every range of 128
  * neurons, the largest weight (V * M / 128 floats, allocated by the first call; if that memory cannot be had
  * the call carries on without them).  The search uses them to skip rows that cannot change a sample's result
  * (som_bmu below); they cost the norm pass nothing measurable.
@@ -116,7 +116,7 @@ int som_norms(som_handle* h, void* stream);
  * further apart than 1e-4 of the best squared distance the unit is the same in every batch.
  * The reported distance is always the fp64 one of the reported unit.
  * Not every row of the sparse x dense product is formed: where som_norms has recorded the per-range
- * maxima (fp32 storage, M % 128 == 0; by default on maps of at least 65 536 neurons), the kernel skips
+ * maxima (M % 128 == 0; by default on maps of at least 65 536 neurons), the kernel skips
  * a sample's infrequent-feature rows for a range of 128 neurons when even the range's smallest partial
  * score, lowered by those features' largest weights in the range, stays above the sample's best score so
  * far, with a margin for fp32 rounding: no neuron of the range can then be the best unit.  The outputs

@@ -196,7 +196,7 @@ struct LayF32 {
     // neurons per lane three fit 128 registers at the price of a 36-byte spill, and measure 1 to 3 % faster
     // than two)
     static constexpr int TAILS_AHEAD = R_ >= 16 ? 3 : 4;
-    static constexpr bool CAN_PRUNE = true;     // scores are held as they are: a lower bound on them is one on the result
+    static constexpr bool CAN_PRUNE = true;
     static constexpr float SEED_SIGN = 1.f;     // scores are held as they are
     typedef Acc<H> Scores;
     typedef Acc<H> Slice;
@@ -268,7 +268,7 @@ struct LayF16 {
     typedef __half Store;
     static constexpr int R = 8, T = 64, ROWB = T * 2;
     static constexpr int TAILS_AHEAD = 4;
-    static constexpr bool CAN_PRUNE = false;
+    static constexpr bool CAN_PRUNE = true;
     static constexpr float SEED_SIGN = -1.f;  // the seed array holds -||w||^2/2
     struct Scores { float v[8]; };
     typedef uint4 Slice;
@@ -345,7 +345,7 @@ struct LayF16W {
     typedef __half Store;
     static constexpr int R = 16, T = 128, ROWB = T * 2;
     static constexpr int TAILS_AHEAD = 4;
-    static constexpr bool CAN_PRUNE = false;
+    static constexpr bool CAN_PRUNE = true;
     static constexpr float SEED_SIGN = -1.f;
     struct Scores { float v[16]; };
     struct Slice { uint4 g[2]; };
@@ -842,15 +842,19 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     const int n_units = n_whole + 4 * n_split;
     const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
     const int feed_keep = h->opt_feed_keep == 1 || (h->opt_feed_keep == 0 && n * 56 <= ((int64_t)24 << 20));
-    // Pruning by range maxima: fp32 storage, when som_norms has written them (the codebook this launch reads
-    // must be the handle's own fp32 codebook, not a shadow).  It pays where nearly every pair of sample and
+    // Pruning by range maxima, when som_norms has written them.  It pays where nearly every pair of sample and
     // range is skipped, which takes many ranges: measured 67 % of the pairs skipped with 32 ranges (64 x 64:
     // 11 % slower, the live samples' tail rows now wait for L2 in the open), 77 % with 128 ranges (11 % slower),
-    // 96 % with 2048 (512 x 512: 21 % faster), 93 % with 8192 (1024 x 1024: 19 % faster).
+    // 96 % with 2048 (512 x 512: 23 % faster), 93 % with 8192 (1024 x 1024: 24 % faster); break-even at 512 ranges.
+    // fp16 storage, whose tail rows are half as long: 5 % (512 x 512) and 8 % (1024 x 1024) faster.
     bool prune = false;
     if constexpr (L::CAN_PRUNE)
-        prune = h->range_max != nullptr && codebook_v == static_cast<const void*>(h->W) &&
-                (h->opt_prune == 1 || (h->opt_prune == 0 && n_ranges >= SOM_PRUNE_MIN_RANGES));
+        prune = h->range_max != nullptr &&
+                (h->opt_prune == 1 || (h->opt_prune == 0 && (h->M + 127) / 128 >= SOM_PRUNE_MIN_RANGES));
+    // (the maxima are those of the handle's own codebook: the first pass of the two-stage search, which reads
+    //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
+    //  slower at 512 x 512: it tests against the second-best key, which skips less)
+    if (codebook_v != static_cast<const void*>(h->W) && codebook_v != static_cast<const void*>(h->Wh)) prune = false;
     auto launch = [&](auto kern) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;

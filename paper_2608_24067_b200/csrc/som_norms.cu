@@ -119,10 +119,22 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
 
 // The same pass over an fp16-stored codebook: VEC = 8 neurons per thread (one 128-bit load of
 // eight halves per row) or 1; every weight is widened exactly and squared in fp64.
-template <int VEC>
+// RMAX (VEC == 8, M % 128 == 0): a half-warp (16 threads x 8 neurons) holds one range of 128
+// neurons; its largest weight of every row goes to range_max[range * V + v] (see k_norms_partial).
+__device__ __forceinline__ void store_range_max_half(float* __restrict__ dst, float m)
+{
+    int key = __float_as_int(m);
+    key ^= (key >> 31) & 0x7fffffff;
+    const unsigned int half_lanes = (threadIdx.x & 16) ? 0xffff0000u : 0x0000ffffu;
+    key = __reduce_max_sync(half_lanes, key);
+    key ^= (key >> 31) & 0x7fffffff;
+    if ((threadIdx.x & 15) == 0) *dst = __int_as_float(key);
+}
+
+template <int VEC, bool RMAX>
 __global__ void __launch_bounds__(NORM_THREADS)
 k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_split,
-                  double* __restrict__ partial)
+                  double* __restrict__ partial, float* __restrict__ range_max)
 {
     const int64_t i = ((int64_t)blockIdx.x * NORM_THREADS + threadIdx.x) * VEC;
     if (i >= M) return;
@@ -132,6 +144,8 @@ k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_s
 #pragma unroll
     for (int k = 0; k < VEC; ++k) acc[k] = 0.0;
     const __half* p = W + (int64_t)v0 * M + i;
+    // (RMAX: M % 128 == 0, so a half-warp, 16 threads x 8 neurons, is all inside M and holds range i / 128)
+    float* pr = RMAX ? range_max + (i / 128) * (int64_t)V + v0 : nullptr;
     int v = v0;
     if (VEC == 8) {
         for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
@@ -142,24 +156,31 @@ k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_s
 #pragma unroll
             for (int u = 0; u < NORM_UNROLL; ++u) {
                 const uint32_t word[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+                float wm = -3.0e38f;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&word[k]));
+                    if (RMAX) wm = fmaxf(wm, fmaxf(f.x, f.y));
                     acc[(2 * k) % VEC] = fma((double)f.x, (double)f.x, acc[(2 * k) % VEC]);
                     acc[(2 * k + 1) % VEC] = fma((double)f.y, (double)f.y, acc[(2 * k + 1) % VEC]);
                 }
+                if (RMAX) store_range_max_half(pr + u, wm);
             }
             p += (int64_t)NORM_UNROLL * M;
+            if (RMAX) pr += NORM_UNROLL;
         }
         for (; v < v1; ++v) {
             const uint4 w = __ldcs(reinterpret_cast<const uint4*>(p));
             const uint32_t word[4] = {w.x, w.y, w.z, w.w};
+            float wm = -3.0e38f;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&word[k]));
+                if (RMAX) wm = fmaxf(wm, fmaxf(f.x, f.y));
                 acc[(2 * k) % VEC] = fma((double)f.x, (double)f.x, acc[(2 * k) % VEC]);
                 acc[(2 * k + 1) % VEC] = fma((double)f.y, (double)f.y, acc[(2 * k + 1) % VEC]);
             }
+            if (RMAX) store_range_max_half(pr++, wm);
             p += M;
         }
     } else {
@@ -236,10 +257,13 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
     NormPlan p = plan_norms(h);
     double* partial = reinterpret_cast<double*>(h->ws);
     dim3 grid((unsigned)p.col_blocks, (unsigned)p.splits);
-    if (h->Wh && p.vec == 8)
-        k_norms_partial_h<8><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
+    if (h->Wh && p.vec == 8 && h->range_max)
+        k_norms_partial_h<8, true><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial,
+                                                                  h->range_max);
+    else if (h->Wh && p.vec == 8)
+        k_norms_partial_h<8, false><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial, nullptr);
     else if (h->Wh)
-        k_norms_partial_h<1><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial);
+        k_norms_partial_h<1, false><<<grid, NORM_THREADS, 0, st>>>(h->Wh, h->M, h->V, p.rows_per_split, partial, nullptr);
     else if (p.vec == 4 && h->shadow) {
         SOM_CK(h, cudaMemsetAsync(h->wmax_bits, 0, 4 * sizeof(unsigned int), st));
         if (h->range_max)

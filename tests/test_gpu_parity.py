@@ -182,6 +182,44 @@ def test_pruning_by_range_maxima_changes_nothing(som_mod, lane_neurons, codebook
                           outs[1][0], outs[1][1], rows)
 
 
+@pytest.mark.parametrize("mode", ["f16-8", "f16-16", "two-stage"])
+@pytest.mark.parametrize("codebook", ["recipe", "smooth", "negative"])
+def test_pruning_with_fp16_rows(som_mod, mode, codebook):
+    """The same for an fp16-stored codebook (maxima of the stored halves, both fp16 layouts) and with the
+    two-stage search switched on over an fp32 codebook (its first pass over the fp16 copy does not prune; the
+    plain fallback and the option's bookkeeping must not be disturbed by the maxima)."""
+    V, M, n = 30_000, 2_048, 40_000
+    W = synth.fill_codebook(V, M, 6, device="cuda")
+    if codebook == "smooth":
+        ramp = torch.linspace(0.0, 1.0, M, device="cuda")
+        W = (W.view(V, M) * 0.2 + ramp[None, :] * torch.rand(V, 1, device="cuda")).reshape(-1).contiguous()
+    elif codebook == "negative":
+        W = (W - 0.3).contiguous()
+    if mode != "two-stage":
+        W = W.half()
+    b = synth.sample_csr(n, V, 11.0, 6, device="cuda", permute_ids=True)
+    outs = []
+    for prune in (2, 1):
+        h = som_mod.Som(V, M, W)
+        h.set_option(0, 2)
+        if mode == "two-stage":
+            h.set_option(7, 1)
+        else:
+            h.set_option(3, int(mode.split("-")[1]))
+        h.set_option(10, prune)
+        h.norms()
+        bmu, dist = h.bmu(b.indptr, b.indices)
+        b1, d1, b2, d2 = h.bmu2(b.indptr, b.indices)
+        torch.cuda.synchronize()
+        outs.append([t.cpu().numpy() for t in (bmu, dist, b1, d1, b2, d2)])
+    for full, pruned in zip(*outs):
+        assert np.array_equal(full.view(np.uint32) if full.dtype == np.float32 else full,
+                              pruned.view(np.uint32) if pruned.dtype == np.float32 else pruned)
+    rows = np.arange(0, n, 11)
+    _check_against_oracle(W.float().cpu().numpy(), V, M, b.indptr.cpu().numpy(), b.indices.cpu().numpy(),
+                          outs[1][0], outs[1][1], rows)
+
+
 def test_config3_full_size_sampled_rows(som_mod):
     """128x128 map at its full size (4M samples, the benchmark's launch configuration);
     a strided sample of rows against the oracle, plus properties that hold for all rows."""
