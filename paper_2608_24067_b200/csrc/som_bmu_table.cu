@@ -428,6 +428,48 @@ struct LayF16W {
     }
 };
 
+// ---- pruning helpers ---------------------------------------------------------------------------
+// smallest score over the team's 8 * R neurons (all lanes of the team call it together)
+template <typename L>
+__device__ __forceinline__ float team_min(const typename L::Scores& s, uint32_t team_lanes)
+{
+    constexpr int R = L::R;
+    float a[R];
+    L::unpack(s, a);
+    float lo = fminf(fminf(a[0], a[1]), fminf(a[2], a[3]));
+    if (R >= 8) lo = fminf(lo, fminf(fminf(a[4 % R], a[5 % R]), fminf(a[6 % R], a[7 % R])));
+    if (R == 16) {
+        lo = fminf(lo, fminf(fminf(a[8 % R], a[9 % R]), fminf(a[10 % R], a[11 % R])));
+        lo = fminf(lo, fminf(fminf(a[12 % R], a[13 % R]), fminf(a[14 % R], a[15 % R])));
+    }
+    lo = fminf(lo, __shfl_xor_sync(team_lanes, lo, 1));
+    lo = fminf(lo, __shfl_xor_sync(team_lanes, lo, 2));
+    lo = fminf(lo, __shfl_xor_sync(team_lanes, lo, 4));
+    return lo;
+}
+
+// Lane q's share of the bounds of one sample: the largest weights, in the live 128-neuron range, of tail
+// features q and q + 8 (from the table som_norms wrote; returned) and of hot codes q and q + 8 (from the
+// per-range copy in shared memory; *hot_part).  `slot` points at the sample's 48-byte slot in the ring.
+__device__ __forceinline__ float prune_bounds(const unsigned char* slot, int q, const float* __restrict__ rmax_hot,
+                                              const float* __restrict__ rmax_range, float* hot_part)
+{
+    const uint32_t hdr = *reinterpret_cast<const uint32_t*>(slot);
+    const uint32_t nt = hdr >> 24, nh = (hdr >> 16) & 0xffu;
+    *hot_part = 0.f;
+    if (nt == SOM_SLOT_NT_OVERFLOW) return 0.f;
+    const uint16_t* hot = reinterpret_cast<const uint16_t*>(slot + 8);
+    const uint16_t* tail = reinterpret_cast<const uint16_t*>(slot + 32);
+    const uint16_t* tail8 = reinterpret_cast<const uint16_t*>(slot + 4);
+    float bh = 0.f, bt = 0.f;
+    if ((uint32_t)q < nh) bh = rmax_hot[hot[q]];
+    if ((uint32_t)q + 8u < nh) bh += rmax_hot[hot[q + 8]];
+    if ((uint32_t)q < nt) bt = __ldg(rmax_range + tail[q]);
+    if ((uint32_t)q + 8u < nt) bt += __ldg(rmax_range + tail8[q]);
+    *hot_part = bh;
+    return bt;
+}
+
 #define SOM_HOT(code) L::sub(acc, L::lds(tab_q + (code) * ROWB))
 #define SOM_TAIL(code) L::ldg(row_ptr(w_q, (code), stride_b))
 
@@ -476,7 +518,11 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
         reinterpret_cast<uint32_t*>(tab)[n_rows * (ROWB / 4) + c] = 0u;
 
     int cur_range = -1;
-    const float* rmax_range = nullptr;  // (pruning) largest weight of every feature row in the live 128-neuron range
+    // pruning: largest weight of every feature row in the live 128-neuron range (global), a copy for the table's
+    // rows behind the table in shared memory, the lanes of this lane's team
+    const float* rmax_range = nullptr;
+    float* rmax_hot = reinterpret_cast<float*>(tab + (size_t)(n_rows + 1) * ROWB);
+    const uint32_t team_lanes = 0xffu << (8 * sub);
     const unsigned char* w_q = reinterpret_cast<const unsigned char*>(W);
     uint32_t i_first = 0;
     for (;;) {
@@ -512,7 +558,13 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const int64_t i_lane = i0 + L::lane_first(q);
             i_first = (uint32_t)i_lane;
             w_q = reinterpret_cast<const unsigned char*>(W + (i_lane < M ? i_lane : 0));
-            if constexpr (PRUNE) rmax_range = range_max + (i0 >> 7) * (int64_t)V;
+            if constexpr (PRUNE) {
+                rmax_range = range_max + (i0 >> 7) * (int64_t)V;
+                for (int c = threadIdx.x; c <= n_rows; c += THREADS) {
+                    const int f = c < n_rows ? slot_feat[c] : -1;
+                    rmax_hot[c] = f >= 0 ? rmax_range[f] : 0.f;  // (the zero row and unused rows take nothing off)
+                }
+            }
             for (int c = threadIdx.x; c < T; c += THREADS)
                 hn_sh[c] = L::SEED_SIGN * ((i0 + c < M) ? hnorm[i0 + c] : inf);
         }
@@ -534,6 +586,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 
         uint32_t curmask = 0;
         Scores base = L::seed(hn_sh, q);
+        float base_lo = 0.f, bt_next = 0.f, bh_next = 0.f;
+        if constexpr (PRUNE) base_lo = team_min<L>(base, team_lanes);
         for (;;) {
             int chunk = 0;
             if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
@@ -564,6 +618,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             }
             feed += 2 * feed_step;
             __syncwarp();
+            if constexpr (PRUNE) bt_next = prune_bounds(my_slot, q, rmax_hot, rmax_range, &bh_next);  // round 0
             u64* pk = keys + w0 + sub;
             for (int r = 0; r < rounds; ++r) {
                 const int st = (r & 1) * RING_STAGE;
@@ -590,13 +645,14 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 //      on what the tail rows can take off this range's scores (one 4-byte load per lane:
                 //      lane q of the team reads the range maximum of tail feature q, and of q + 8)
                 Slice tr0, tr1, tr2, tr3;
-                float bnd = 0.f;
+                float bnd = 0.f, bnd_hot = 0.f;
                 if constexpr (PRUNE) {
-                    const uint32_t ntc = nt == SOM_SLOT_NT_OVERFLOW ? 0u : nt;
-                    if ((uint32_t)q < ntc)
-                        bnd = __ldg(rmax_range + *reinterpret_cast<const uint16_t*>(my_slot + st + 32 + 2 * q));
-                    if ((uint32_t)q + 8u < ntc)
-                        bnd += __ldg(rmax_range + *reinterpret_cast<const uint16_t*>(my_slot + st + 4 + 2 * q));
+                    // this round's bounds arrive from the previous round; the next round's go in flight (they are
+                    // read from the ring's other stage, which the feeders have just filled; past the chunk's
+                    // last round that stage holds bytes that are no slot)
+                    bnd = bt_next;
+                    bnd_hot = bh_next;
+                    bt_next = r + 1 < rounds ? prune_bounds(my_slot + (RING_STAGE - st), q, rmax_hot, rmax_range, &bh_next) : 0.f;
                 } else {
                     if (p0) tr0 = SOM_TAIL(lo16(s2.x));
                     if (p1) tr1 = SOM_TAIL(hi16(s2.x));
@@ -618,12 +674,36 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         L::sub(base, L::lds(tab_q + b * ROWB));
                     }
                     curmask = mask;
+                    if constexpr (PRUNE) base_lo = team_min<L>(base, team_lanes);
                 }
 
                 // ---- hot rows: exactly max(nh over the warp, 1) steps; shorter lists are padded
                 //      with the zero row, so a step carries no predicate.  The first step also
                 //      moves the running score out of `base` (which the next sample may reuse).
-                const uint32_t nh_max = __reduce_max_sync(0xffffffffu, nh);
+                // the sample's key as a score (decoded here when pruning needs it, else where the argmin does)
+                const uint32_t cu = (uint32_t)(key0 >> 32);
+                float cs = 0.f;
+                bool live = true;
+                if constexpr (PRUNE) {
+                    // ---- first test, before any row of the sample is read: even the range's smallest PREFIX
+                    //      score (kept per team beside the prefix), lowered by the largest weights of all the
+                    //      sample's hot and tail rows in this range, stays above the sample's key: nothing of
+                    //      this sample is read for this range.
+                    cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
+                    pk += 4;
+                    bnd += __shfl_xor_sync(team_lanes, bnd, 1);
+                    bnd_hot += __shfl_xor_sync(team_lanes, bnd_hot, 1);
+                    bnd += __shfl_xor_sync(team_lanes, bnd, 2);
+                    bnd_hot += __shfl_xor_sync(team_lanes, bnd_hot, 2);
+                    bnd += __shfl_xor_sync(team_lanes, bnd, 4);
+                    bnd_hot += __shfl_xor_sync(team_lanes, bnd_hot, 4);
+                    const float all = bnd + bnd_hot;
+                    // (an empty key decodes to NaN: the comparison is false and the sample stays live)
+                    live = nt != SOM_SLOT_NT_OVERFLOW &&
+                           !(base_lo - all > cs + 1e-5f * (fabsf(base_lo) + fabsf(cs) + fabsf(all)));
+                }
+                const uint32_t nh_max = __reduce_max_sync(0xffffffffu, live ? nh : 0u);
+                if (!live) continue;
                 Scores acc = L::sub3(base, L::lds(tab_q + lo16(s0.z) * ROWB));
                 switch (nh_max) {
                     case 12: SOM_HOT(hi16(s1.w));
@@ -641,38 +721,21 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
                 // the sample's key as a score (decoded here when pruning needs it, else where the argmin does)
-                const uint32_t cu = (uint32_t)(key0 >> 32);
-                float cs = 0.f;
-                if constexpr (PRUNE) cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
-                if constexpr (PRUNE) pk += 4;
 
-                // ---- pruning (fp32 storage, range maxima from som_norms): the tail rows lower a score by at most
-                //      the sum of their largest weights in this range.  If even the smallest score of the team's
-                //      neurons, lowered by that much, stays above the sample's key (with a margin for the rounding
-                //      of the sums), no neuron of this range can become a candidate, whatever the tail rows hold:
-                //      they are not loaded.  The result is that of the full search, bit for bit (a neuron that
-                //      is skipped would have lost the comparison below).  A live sample's tail rows go out only
-                //      now, four at a time: their latency is no longer hidden behind the hot rows, which is why
-                //      the launcher prunes only where nearly all pairs of sample and range are skipped.
+                // ---- pruning, second test (after the hot rows): the tail rows lower a score by at most the sum of
+                //      their largest weights in this range.  If even the smallest score of the team's neurons as
+                //      it stands, lowered by that much, stays above the sample's key (with a margin for the
+                //      rounding of the sums), no neuron of this range can become a candidate, whatever the tail
+                //      rows hold: they are not loaded.  Either way the result is that of the full search, bit for
+                //      bit (a neuron that is skipped would have lost the comparison below).  A live sample's tail
+                //      rows go out only now, four at a time: their latency is no longer hidden behind the hot
+                //      rows, which is why the launcher prunes only where nearly all pairs of sample and range are
+                //      skipped.
                 constexpr int TA = PRUNE ? 4 : L::TAILS_AHEAD;
                 if constexpr (PRUNE) {
-                    bnd += __shfl_xor_sync(0xffffffffu, bnd, 1);
-                    bnd += __shfl_xor_sync(0xffffffffu, bnd, 2);
-                    bnd += __shfl_xor_sync(0xffffffffu, bnd, 4);
-                    float h[R];
-                    L::unpack(acc, h);
-                    float lo = fminf(fminf(h[0], h[1]), fminf(h[2], h[3]));
-                    if (R >= 8) lo = fminf(lo, fminf(fminf(h[4 % R], h[5 % R]), fminf(h[6 % R], h[7 % R])));
-                    if (R == 16) {
-                        lo = fminf(lo, fminf(fminf(h[8 % R], h[9 % R]), fminf(h[10 % R], h[11 % R])));
-                        lo = fminf(lo, fminf(fminf(h[12 % R], h[13 % R]), fminf(h[14 % R], h[15 % R])));
-                    }
-                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, 1));
-                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, 2));
-                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, 4));
-                    // (an empty key decodes to NaN: the comparison is false and the sample stays live)
-                    const bool live = nt != SOM_SLOT_NT_OVERFLOW &&
-                                      !(lo - bnd > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd)));
+                    // ---- second test, after the hot rows: the tail rows alone against the scores as they stand
+                    const float lo = team_min<L>(acc, team_lanes);
+                    live = !(lo - bnd > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd)));
                     if (!live) continue;
                     if (p0) tr0 = SOM_TAIL(lo16(s2.x));
                     if (p1) tr1 = SOM_TAIL(hi16(s2.x));
@@ -846,7 +909,9 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     // range is skipped, which takes many ranges: measured 67 % of the pairs skipped with 32 ranges (64 x 64:
     // 11 % slower, the live samples' tail rows now wait for L2 in the open), 77 % with 128 ranges (11 % slower),
     // 96 % with 2048 (512 x 512: 23 % faster), 93 % with 8192 (1024 x 1024: 24 % faster); break-even at 512 ranges.
-    // fp16 storage, whose tail rows are half as long: 5 % (512 x 512) and 8 % (1024 x 1024) faster.
+    // (Those figures are for the test after the hot rows alone; the test before them, which skips about half as
+    // many pairs but spares their hot rows too, took 512 x 512 from 255 to 239 ms and cost 1024 x 1024 1.5 %.)
+    // fp16 storage, whose tail rows are half as long: 10 % (512 x 512) and 8 % (1024 x 1024) faster.
     bool prune = false;
     if constexpr (L::CAN_PRUNE)
         prune = h->range_max != nullptr &&
@@ -855,6 +920,7 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
     //  slower at 512 x 512: it tests against the second-best key, which skips less)
     if (codebook_v != static_cast<const void*>(h->W) && codebook_v != static_cast<const void*>(h->Wh)) prune = false;
+    if (prune) smem += ((size_t)(SOM_PLAN_MASK_FEATURES + n_hot + 1) * sizeof(float) + 15) / 16 * 16;  // the table rows' maxima
     auto launch = [&](auto kern) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
