@@ -116,7 +116,7 @@ int som_norms(som_handle* h, void* stream);
  * further apart than 1e-4 of the best squared distance the unit is the same in every batch.
  * The reported distance is always the fp64 one of the reported unit.
  * Not every row of the sparse x dense product is formed: where som_norms has recorded the per-range
- * maxima (M % 128 == 0; by default on maps of at least 65 536 neurons), the kernel skips a sample's rows
+ * maxima (M % 128 == 0; by default on maps of at least 98 304 neurons), the kernel skips a sample's rows
  * for a range of 128 neurons when even the range's smallest partial score, lowered by the largest weights
  * in the range of the features not yet added, stays above the sample's best score so far, with a margin
  * for fp32 rounding: no neuron of the range can then be the best unit.  It tests once before the sample's

@@ -39,7 +39,7 @@
 
 namespace {
 
-constexpr int SOM_PRUNE_MIN_RANGES = 512;  // pruning by range maxima from this many neuron ranges (see launch_table)
+constexpr int SOM_PRUNE_MIN_RANGES = 768;  // pruning by range maxima from this many neuron ranges (see launch_table)
 constexpr int CHUNK = 128;  // samples a warp takes at a time ...
 constexpr int SMALL_CHUNK = 32;  // ... and near the end of a unit, so that its warps finish together
 constexpr int RING_STAGE = 224;  // bytes of one ring stage: 4 slots + 4 keys
@@ -910,7 +910,9 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     // 11 % slower, the live samples' tail rows now wait for L2 in the open), 77 % with 128 ranges (11 % slower),
     // 96 % with 2048 (512 x 512: 23 % faster), 93 % with 8192 (1024 x 1024: 24 % faster); break-even at 512 ranges.
     // (Those figures are for the test after the hot rows alone; the test before them, which skips about half as
-    // many pairs but spares their hot rows too, took 512 x 512 from 255 to 239 ms and cost 1024 x 1024 1.5 %.)
+    // many pairs but spares their hot rows too, took 512 x 512 from 255 to 239 ms and cost 1024 x 1024 1.5 %; with
+    // both tests 256 x 256 is 8 % slower than the full search, 320 x 320 and 384 x 384 2 to 4 % faster, 448 x 448
+    // 13 %: on from 768 ranges.)
     // fp16 storage, whose tail rows are half as long: 10 % (512 x 512) and 8 % (1024 x 1024) faster.
     bool prune = false;
     if constexpr (L::CAN_PRUNE)
