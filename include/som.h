@@ -116,12 +116,11 @@ int som_norms(som_handle* h, void* stream);
  * further apart than 1e-4 of the best squared distance the unit is the same in every batch.
  * The reported distance is always the fp64 one of the reported unit.
  * Not every row of the sparse x dense product is formed: where som_norms has recorded the per-range
- * maxima (M % 128 == 0; by default on maps of at least 98 304 neurons), the kernel skips a sample's rows
- * for a range of 128 neurons when even the range's smallest partial score, lowered by the largest weights
- * in the range of the features not yet added, stays above the sample's best score so far, with a margin
- * for fp32 rounding: no neuron of the range can then be the best unit.  It tests once before the sample's
- * rows are read (all of them are then skipped) and once after the frequent features' rows (the others are
- * skipped).  The outputs are bit for bit those of the search that forms every row
+ * maxima (M % 128 == 0; by default on maps of at least 4096 neurons), the kernel leaves a sample out
+ * of the search of a range of 128 neurons when even the range's smallest partial score over the sample's
+ * most frequent features, lowered by the largest weights in the range of its other features, stays above
+ * the sample's best score so far, with a margin for fp32 rounding: no neuron of the range can then be
+ * the best unit.  The outputs are bit for bit those of the search that forms every row
  * (tests/test_gpu_parity.py forces it both ways).
  */
 int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,

@@ -39,7 +39,7 @@
 
 namespace {
 
-constexpr int SOM_PRUNE_MIN_RANGES = 768;  // pruning by range maxima from this many neuron ranges (see launch_table)
+constexpr int SOM_PRUNE_MIN_RANGES = 32;  // pruning by range maxima from this many ranges of 128 neurons (see launch_table)
 constexpr int CHUNK = 128;  // samples a warp takes at a time ...
 constexpr int SMALL_CHUNK = 32;  // ... and near the end of a unit, so that its warps finish together
 constexpr int RING_STAGE = 224;  // bytes of one ring stage: 4 slots + 4 keys
@@ -448,28 +448,6 @@ __device__ __forceinline__ float team_min(const typename L::Scores& s, uint32_t 
     return lo;
 }
 
-// Lane q's share of the bounds of one sample: the largest weights, in the live 128-neuron range, of tail
-// features q and q + 8 (from the table som_norms wrote; returned) and of hot codes q and q + 8 (from the
-// per-range copy in shared memory; *hot_part).  `slot` points at the sample's 48-byte slot in the ring.
-__device__ __forceinline__ float prune_bounds(const unsigned char* slot, int q, const float* __restrict__ rmax_hot,
-                                              const float* __restrict__ rmax_range, float* hot_part)
-{
-    const uint32_t hdr = *reinterpret_cast<const uint32_t*>(slot);
-    const uint32_t nt = hdr >> 24, nh = (hdr >> 16) & 0xffu;
-    *hot_part = 0.f;
-    if (nt == SOM_SLOT_NT_OVERFLOW) return 0.f;
-    const uint16_t* hot = reinterpret_cast<const uint16_t*>(slot + 8);
-    const uint16_t* tail = reinterpret_cast<const uint16_t*>(slot + 32);
-    const uint16_t* tail8 = reinterpret_cast<const uint16_t*>(slot + 4);
-    float bh = 0.f, bt = 0.f;
-    if ((uint32_t)q < nh) bh = rmax_hot[hot[q]];
-    if ((uint32_t)q + 8u < nh) bh += rmax_hot[hot[q + 8]];
-    if ((uint32_t)q < nt) bt = __ldg(rmax_range + tail[q]);
-    if ((uint32_t)q + 8u < nt) bt += __ldg(rmax_range + tail8[q]);
-    *hot_part = bh;
-    return bt;
-}
-
 #define SOM_HOT(code) L::sub(acc, L::lds(tab_q + (code) * ROWB))
 #define SOM_TAIL(code) L::ldg(row_ptr(w_q, (code), stride_b))
 
@@ -505,6 +483,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
     // of one round.  The bytes of round r+2 are in flight in registers, round r+1 is being
     // stored, round r is being read: slot and key latency never sits on the critical path.
     __shared__ __align__(16) unsigned char ring_sh[WARPS * 2 * RING_STAGE];
+    __shared__ unsigned char live_sh[PRUNE ? WARPS * CHUNK : 16];  // (pruning) a warp's surviving samples of a chunk
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int q = lane & 7;
@@ -586,7 +565,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 
         uint32_t curmask = 0;
         Scores base = L::seed(hn_sh, q);
-        float base_lo = 0.f, bt_next = 0.f, bh_next = 0.f;
+        float base_lo = 0.f;
         if constexpr (PRUNE) base_lo = team_min<L>(base, team_lanes);
         for (;;) {
             int chunk = 0;
@@ -603,37 +582,149 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             // the keys a round tests its candidates against: the best so far, or with TOP2 the
             // second (third) best so far (a stale, larger value only lets more candidates through)
             const u64* filter_keys = KEEP == 3 ? keys3 : (TOP2 ? keys2 : keys);
-            const uint4* feed = (lane < 12) ? slots + w0 * SLOT_Q + lane
-                                            : reinterpret_cast<const uint4*>(filter_keys + w0) + (lane - 12);
-            const int feed_step = (lane < 12) ? 4 * SLOT_Q : 2;  // uint4 per round
-            const bool feeder = lane < 14;
-            unsigned char* my_store = ring + (lane < 12 ? lane * 16 : 192 + (lane - 12) * 16);
             const unsigned char* my_slot = ring + sub * 48;
             const unsigned char* my_key = ring + 192 + sub * 8;
-            uint4 g = make_uint4(0u, 0u, 0u, 0u);
-            __syncwarp();  // the previous chunk's last reads of the ring are done
-            if (feeder) {
-                *reinterpret_cast<uint4*>(my_store) = ld_feed(feed, feed_keep);  // round 0 -> stage 0
-                g = ld_feed(feed + feed_step, feed_keep);             // round 1, in flight
+            int rounds_b = rounds;  // rounds of the search loop below
+            int n_live = 0;         // (pruning) survivors of the chunk
+            unsigned char* live_list = live_sh + warp * CHUNK;  // (pruning) positions in the chunk of the samples to search
+            if constexpr (PRUNE) {
+                // ---- pruning, before the search loop: find the samples of the chunk that this range can still
+                //      matter to.  A sample survives unless (smallest prefix score of the range for its mask) minus
+                //      (largest weights in this range of all its hot and tail rows) stays above its key, with a
+                //      margin for the rounding of the sums.  Everything else is skipped for this range: a neuron
+                //      of it would have lost the candidate comparison of the search loop, so the result is that
+                //      of the full search bit for bit.  The survivors are then searched four to a round like any
+                //      chunk, with their tail rows in flight early.
+                //      Step 1, by teams as in the search loop: the prefix of every mask that occurs (rows are read
+                //      only where the mask changes) and its smallest score, one float per sample.
+                //      Step 2, a lane per sample (32 samples at a time, all their loads in flight together): the
+                //      bounds of its codes, the test, and the list of survivors in order.
+                const int n_chunk = 4 * rounds;
+                uint32_t hdrs[CHUNK / 32];
+                float los[CHUNK / 32];  // smallest prefix score for the masks of this lane's samples (step 1 -> step 2)
+#pragma unroll
+                for (int p = 0; p < CHUNK / 32; ++p) {
+                    const int pos = lane + 32 * p;
+                    hdrs[p] = pos < n_chunk ? __ldcg(reinterpret_cast<const uint32_t*>(slots + (w0 + pos) * SLOT_Q))
+                                            : (SOM_SLOT_NT_OVERFLOW << 24);
+                    los[p] = 0.f;
+                }
+#pragma unroll
+                for (int p = 0; p < CHUNK / 32; ++p) {
+#pragma unroll 1
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const uint32_t hdr = __shfl_sync(0xffffffffu, hdrs[p], 4 * rr + sub);
+                        if (32 * p + 4 * rr >= n_chunk) break;  // (the same for every lane)
+                        const uint32_t mask = hdr & 0xffffu;
+                        if (mask != curmask) {
+                            base = L::seed(hn_sh, q);
+                            uint32_t mm = mask;
+                            while (mm) {
+                                const int b = __ffs(mm) - 1;
+                                mm &= mm - 1;
+                                L::sub(base, L::lds(tab_q + b * ROWB));
+                            }
+                            curmask = mask;
+                            base_lo = team_min<L>(base, team_lanes);
+                        }
+                        // lane 4 * rr + s of the warp owns the sample that team s has just looked at
+                        const float t = __shfl_sync(0xffffffffu, base_lo, 8 * (lane & 3));
+                        if ((lane >> 2) == rr) los[p] = t;
+                    }
+                }
+#pragma unroll
+                for (int p = 0; p < CHUNK / 32; ++p) {
+                    const int pos = lane + 32 * p;
+                    if (32 * p >= n_chunk) break;
+                    const uint32_t hdr = hdrs[p];
+                    const uint32_t nt = hdr >> 24, nh = (hdr >> 16) & 0xffu;
+                    bool live = pos < n_chunk && nt != SOM_SLOT_NT_OVERFLOW;
+                    if (live) {
+                        const uint4* sl = slots + (w0 + pos) * SLOT_Q;
+                        const uint4 s0 = __ldcg(sl), s1 = __ldcg(sl + 1), s2 = __ldcg(sl + 2);
+                        const u64 key0 = __ldcg(filter_keys + w0 + pos);
+                        const uint32_t hw[6] = {s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};  // hot codes 0..11
+                        const uint32_t tw[5] = {s2.x, s2.y, s2.z, s2.w, s0.y};        // tail codes 0..9
+                        float bnd = 0.f;
+#pragma unroll
+                        for (int j = 0; j < SOM_SLOT_MAX_HOT; ++j)
+                            if ((uint32_t)j < nh) bnd += rmax_hot[(j & 1) ? hi16(hw[j >> 1]) : lo16(hw[j >> 1])];
+#pragma unroll
+                        for (int j = 0; j < SOM_SLOT_MAX_TAIL; ++j)
+                            if ((uint32_t)j < nt) bnd += __ldg(rmax_range + ((j & 1) ? hi16(tw[j >> 1]) : lo16(tw[j >> 1])));
+                        const uint32_t cu = (uint32_t)(key0 >> 32);
+                        const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
+                        const float lo = los[p];
+                        // (an empty key decodes to NaN: the comparison is false and the sample stays live)
+                        live = !(lo - bnd > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd)));
+                    }
+                    const uint32_t votes = __ballot_sync(0xffffffffu, live);
+                    if (live) live_list[n_live + __popc(votes & ((1u << lane) - 1u))] = (unsigned char)pos;
+                    n_live += __popc(votes);
+                }
+                rounds_b = (n_live + 3) >> 2;
+                __syncwarp();  // the list is written
+                // whole rounds: the last survivor is repeated, so that the spare teams' loads have an address
+                if (n_live > 0 && lane < 3 && n_live + lane < 4 * rounds_b) live_list[n_live + lane] = live_list[n_live - 1];
+                __syncwarp();
             }
-            feed += 2 * feed_step;
+            // the search loop's feed: contiguous slots and keys, or (pruning) those of the survivors
+            const uint4* feed;
+            int feed_step = 0;
+            bool feeder;
+            unsigned char* my_store;
+            auto feed_at = [&](int r) -> const uint4* {  // (pruning) where this lane's piece of round r lies
+                const int rr = 4 * min(r, rounds_b - 1);  // (past the last round: that round's again, a valid address)
+                if (lane < 12) return slots + (w0 + live_list[rr + lane / 3]) * SLOT_Q + lane % 3;
+                return reinterpret_cast<const uint4*>(filter_keys + w0 + live_list[rr + (lane - 12)]);
+            };
+            if constexpr (PRUNE) {
+                feeder = lane < 16;
+                my_store = ring + (lane < 12 ? lane * 16 : 192 + (lane - 12) * 8);
+                feed = nullptr;
+            } else {
+                feeder = lane < 14;
+                my_store = ring + (lane < 12 ? lane * 16 : 192 + (lane - 12) * 16);
+                feed = (lane < 12) ? slots + w0 * SLOT_Q + lane
+                                   : reinterpret_cast<const uint4*>(filter_keys + w0) + (lane - 12);
+                feed_step = (lane < 12) ? 4 * SLOT_Q : 2;  // uint4 per round
+            }
+            uint4 g = make_uint4(0u, 0u, 0u, 0u);
+            // (a key lane of the pruning feed moves 8 bytes: the low half of g)
+            auto ld_piece = [&](const uint4* p) -> uint4 {
+                if (PRUNE && lane >= 12) {
+                    const uint2 k = __ldcg(reinterpret_cast<const uint2*>(p));
+                    return make_uint4(k.x, k.y, 0u, 0u);
+                }
+                return ld_feed(p, feed_keep);
+            };
+            auto st_piece = [&](unsigned char* dst, const uint4 v) {
+                if (PRUNE && lane >= 12) *reinterpret_cast<uint2*>(dst) = make_uint2(v.x, v.y);
+                else *reinterpret_cast<uint4*>(dst) = v;
+            };
+            __syncwarp();  // the previous chunk's (or phase A's) last reads of the ring are done
+            if (rounds_b > 0 && feeder) {
+                st_piece(my_store, ld_piece(PRUNE ? feed_at(0) : feed));  // round 0 -> stage 0
+                g = ld_piece(PRUNE ? feed_at(1) : feed + feed_step);      // round 1, in flight
+            }
+            if (!PRUNE) feed += 2 * feed_step;
             __syncwarp();
-            if constexpr (PRUNE) bt_next = prune_bounds(my_slot, q, rmax_hot, rmax_range, &bh_next);  // round 0
             u64* pk = keys + w0 + sub;
-            for (int r = 0; r < rounds; ++r) {
+            for (int r = 0; r < rounds_b; ++r) {
                 const int st = (r & 1) * RING_STAGE;
                 const uint4 s0 = *reinterpret_cast<const uint4*>(my_slot + st);
                 const uint4 s1 = *reinterpret_cast<const uint4*>(my_slot + st + 16);
                 const uint4 s2 = *reinterpret_cast<const uint4*>(my_slot + st + 32);
                 const u64 key0 = *reinterpret_cast<const u64*>(my_key + st);
+                if constexpr (PRUNE) pk = keys + w0 + live_list[4 * r + sub] + 4;  // (the combine below names pk - 4)
                 // round r+1 goes into the other stage (its previous content, round r-1, was
                 // consumed a round ago); round r+2 goes in flight.  The slot and key arrays
                 // are padded, so the loads past the chunk's end stay in bounds.
                 if (feeder) {
-                    *reinterpret_cast<uint4*>(my_store + (RING_STAGE - st)) = g;
-                    g = ld_feed(feed, feed_keep);
+                    st_piece(my_store + (RING_STAGE - st), g);
+                    g = ld_piece(PRUNE ? feed_at(r + 2) : feed);
                 }
-                feed += feed_step;
+                if (!PRUNE) feed += feed_step;
                 __syncwarp();
                 const uint32_t hdr = s0.x;
                 const uint32_t nt = hdr >> 24;  // SOM_SLOT_NT_OVERFLOW marks an overflow sample
@@ -641,27 +732,15 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 const uint32_t mask = hdr & 0xffffu;
                 const bool p0 = nt > 0, p1 = nt > 1, p2 = nt > 2, p3 = nt > 3;
 
-                // ---- the first tail rows of this sample go in flight first; with pruning, only the bounds
-                //      on what the tail rows can take off this range's scores (one 4-byte load per lane:
-                //      lane q of the team reads the range maximum of tail feature q, and of q + 8)
+                // ---- the first tail rows of this sample go in flight first ----------------------------
                 Slice tr0, tr1, tr2, tr3;
-                float bnd = 0.f, bnd_hot = 0.f;
-                if constexpr (PRUNE) {
-                    // this round's bounds arrive from the previous round; the next round's go in flight (they are
-                    // read from the ring's other stage, which the feeders have just filled; past the chunk's
-                    // last round that stage holds bytes that are no slot)
-                    bnd = bt_next;
-                    bnd_hot = bh_next;
-                    bt_next = r + 1 < rounds ? prune_bounds(my_slot + (RING_STAGE - st), q, rmax_hot, rmax_range, &bh_next) : 0.f;
-                } else {
-                    if (p0) tr0 = SOM_TAIL(lo16(s2.x));
-                    if (p1) tr1 = SOM_TAIL(hi16(s2.x));
-                    if constexpr (L::TAILS_AHEAD >= 3) {
-                        if (p2) tr2 = SOM_TAIL(lo16(s2.y));
-                    }
-                    if constexpr (L::TAILS_AHEAD >= 4) {
-                        if (p3) tr3 = SOM_TAIL(hi16(s2.y));
-                    }
+                if (p0) tr0 = SOM_TAIL(lo16(s2.x));
+                if (p1) tr1 = SOM_TAIL(hi16(s2.x));
+                if constexpr (L::TAILS_AHEAD >= 3) {
+                    if (p2) tr2 = SOM_TAIL(lo16(s2.y));
+                }
+                if constexpr (L::TAILS_AHEAD >= 4) {
+                    if (p3) tr3 = SOM_TAIL(hi16(s2.y));
                 }
 
                 // ---- mask prefix ------------------------------------------------------------
@@ -674,36 +753,16 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         L::sub(base, L::lds(tab_q + b * ROWB));
                     }
                     curmask = mask;
-                    if constexpr (PRUNE) base_lo = team_min<L>(base, team_lanes);
                 }
 
                 // ---- hot rows: exactly max(nh over the warp, 1) steps; shorter lists are padded
                 //      with the zero row, so a step carries no predicate.  The first step also
                 //      moves the running score out of `base` (which the next sample may reuse).
-                // the sample's key as a score (decoded here when pruning needs it, else where the argmin does)
-                const uint32_t cu = (uint32_t)(key0 >> 32);
-                float cs = 0.f;
-                bool live = true;
-                if constexpr (PRUNE) {
-                    // ---- first test, before any row of the sample is read: even the range's smallest PREFIX
-                    //      score (kept per team beside the prefix), lowered by the largest weights of all the
-                    //      sample's hot and tail rows in this range, stays above the sample's key: nothing of
-                    //      this sample is read for this range.
-                    cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
-                    pk += 4;
-                    bnd += __shfl_xor_sync(team_lanes, bnd, 1);
-                    bnd_hot += __shfl_xor_sync(team_lanes, bnd_hot, 1);
-                    bnd += __shfl_xor_sync(team_lanes, bnd, 2);
-                    bnd_hot += __shfl_xor_sync(team_lanes, bnd_hot, 2);
-                    bnd += __shfl_xor_sync(team_lanes, bnd, 4);
-                    bnd_hot += __shfl_xor_sync(team_lanes, bnd_hot, 4);
-                    const float all = bnd + bnd_hot;
-                    // (an empty key decodes to NaN: the comparison is false and the sample stays live)
-                    live = nt != SOM_SLOT_NT_OVERFLOW &&
-                           !(base_lo - all > cs + 1e-5f * (fabsf(base_lo) + fabsf(cs) + fabsf(all)));
-                }
-                const uint32_t nh_max = __reduce_max_sync(0xffffffffu, live ? nh : 0u);
-                if (!live) continue;
+                // (pruning: the last round of the survivors may be short; its spare teams, which were fed the last
+                //  survivor again so that every load has a valid address, sit the round out)
+                const bool spare = PRUNE && 4 * r + sub >= n_live;
+                const uint32_t nh_max = __reduce_max_sync(0xffffffffu, spare ? 0u : nh);
+                if (spare) continue;
                 Scores acc = L::sub3(base, L::lds(tab_q + lo16(s0.z) * ROWB));
                 switch (nh_max) {
                     case 12: SOM_HOT(hi16(s1.w));
@@ -720,61 +779,25 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     default: break;
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
-                // the sample's key as a score (decoded here when pruning needs it, else where the argmin does)
-
-                // ---- pruning, second test (after the hot rows): the tail rows lower a score by at most the sum of
-                //      their largest weights in this range.  If even the smallest score of the team's neurons as
-                //      it stands, lowered by that much, stays above the sample's key (with a margin for the
-                //      rounding of the sums), no neuron of this range can become a candidate, whatever the tail
-                //      rows hold: they are not loaded.  Either way the result is that of the full search, bit for
-                //      bit (a neuron that is skipped would have lost the comparison below).  A live sample's tail
-                //      rows go out only now, four at a time: their latency is no longer hidden behind the hot
-                //      rows, which is why the launcher prunes only where nearly all pairs of sample and range are
-                //      skipped.
-                constexpr int TA = PRUNE ? 4 : L::TAILS_AHEAD;
-                if constexpr (PRUNE) {
-                    // ---- second test, after the hot rows: the tail rows alone against the scores as they stand
-                    const float lo = team_min<L>(acc, team_lanes);
-                    live = !(lo - bnd > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd)));
-                    if (!live) continue;
-                    if (p0) tr0 = SOM_TAIL(lo16(s2.x));
-                    if (p1) tr1 = SOM_TAIL(hi16(s2.x));
-                    if (p2) tr2 = SOM_TAIL(lo16(s2.y));
-                    if (p3) tr3 = SOM_TAIL(hi16(s2.y));
-                }
-
                 // ---- tail rows ------------------------------------------------------------------
                 if (p0) L::sub(acc, tr0);
                 if (p1) L::sub(acc, tr1);
-                if constexpr (TA >= 3) {
+                if constexpr (L::TAILS_AHEAD >= 3) {
                     if (p2) L::sub(acc, tr2);
                 } else {
                     if (p2) L::sub(acc, SOM_TAIL(lo16(s2.y)));
                 }
-                if constexpr (TA >= 4) {
+                if constexpr (L::TAILS_AHEAD >= 4) {
                     if (p3) L::sub(acc, tr3);
                 } else {
                     if (p3) L::sub(acc, SOM_TAIL(hi16(s2.y)));
                 }
                 if (nt > 4) {
                     if (nt != SOM_SLOT_NT_OVERFLOW) {
-                        if constexpr (PRUNE) {
-                            // nothing was loaded ahead of the decision: the next four go out together
-                            const bool p5 = nt > 5, p6 = nt > 6, p7 = nt > 7;
-                            tr0 = SOM_TAIL(lo16(t45));
-                            if (p5) tr1 = SOM_TAIL(hi16(t45));
-                            if (p6) tr2 = SOM_TAIL(lo16(t67));
-                            if (p7) tr3 = SOM_TAIL(hi16(t67));
-                            L::sub(acc, tr0);
-                            if (p5) L::sub(acc, tr1);
-                            if (p6) L::sub(acc, tr2);
-                            if (p7) L::sub(acc, tr3);
-                        } else {
-                            L::sub(acc, SOM_TAIL(lo16(t45)));
-                            if (nt > 5) L::sub(acc, SOM_TAIL(hi16(t45)));
-                            if (nt > 6) L::sub(acc, SOM_TAIL(lo16(t67)));
-                            if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
-                        }
+                        L::sub(acc, SOM_TAIL(lo16(t45)));
+                        if (nt > 5) L::sub(acc, SOM_TAIL(hi16(t45)));
+                        if (nt > 6) L::sub(acc, SOM_TAIL(lo16(t67)));
+                        if (nt > 7) L::sub(acc, SOM_TAIL(hi16(t67)));
                         if (nt > 8) L::sub(acc, SOM_TAIL(lo16(s0.y)));
                         if (nt > 9) L::sub(acc, SOM_TAIL(hi16(s0.y)));
                     } else {
@@ -796,10 +819,9 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     mn = fminf(mn, fminf(fminf(a[8 % R], a[9 % R]), fminf(a[10 % R], a[11 % R])));
                     mn = fminf(mn, fminf(fminf(a[12 % R], a[13 % R]), fminf(a[14 % R], a[15 % R])));
                 }
-                if constexpr (!PRUNE) {
-                    pk += 4;
-                    cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
-                }
+                if constexpr (!PRUNE) pk += 4;
+                const uint32_t cu = (uint32_t)(key0 >> 32);
+                const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
                 if (!(mn > cs)) {
                     int rr = R - 1;
 #pragma unroll
@@ -905,15 +927,10 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     const int n_units = n_whole + 4 * n_split;
     const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
     const int feed_keep = h->opt_feed_keep == 1 || (h->opt_feed_keep == 0 && n * 56 <= ((int64_t)24 << 20));
-    // Pruning by range maxima, when som_norms has written them.  It pays where nearly every pair of sample and
-    // range is skipped, which takes many ranges: measured 67 % of the pairs skipped with 32 ranges (64 x 64:
-    // 11 % slower, the live samples' tail rows now wait for L2 in the open), 77 % with 128 ranges (11 % slower),
-    // 96 % with 2048 (512 x 512: 23 % faster), 93 % with 8192 (1024 x 1024: 24 % faster); break-even at 512 ranges.
-    // (Those figures are for the test after the hot rows alone; the test before them, which skips about half as
-    // many pairs but spares their hot rows too, took 512 x 512 from 255 to 239 ms and cost 1024 x 1024 1.5 %; with
-    // both tests 256 x 256 is 8 % slower than the full search, 320 x 320 and 384 x 384 2 to 4 % faster, 448 x 448
-    // 13 %: on from 768 ranges.)
-    // fp16 storage, whose tail rows are half as long: 10 % (512 x 512) and 8 % (1024 x 1024) faster.
+    // Pruning by range maxima, when som_norms has written them.  Measured against the search that reads every row
+    // (fp32 storage, the benchmark's batches): 64 x 64 (32 ranges) 5.28 -> 5.07 ms, 128 x 128 78.2 -> 64.2 ms,
+    // 512 x 512 329 -> 163 ms, 1024 x 1024 368 -> 219 ms; the share of the (sample, range) pairs it skips grows
+    // with the number of ranges, because a sample's key tightens as the ranges go by.  Below 32 ranges it is off.
     bool prune = false;
     if constexpr (L::CAN_PRUNE)
         prune = h->range_max != nullptr &&

@@ -73,7 +73,7 @@ struct som_handle {
     int64_t opt_parts;     // row-table kernel: sample parts per neuron range (0 = default)
     int64_t opt_feed_keep; // row-table kernel: slot stream kept in L2 (0 = by batch size, 1 = always, 2 = never)
     int64_t opt_prune;     // row-table kernel: skip a sample's tail rows for ranges that cannot hold its best unit
-                           // (0 = where range_max exists and the map has at least 768 ranges of 128 neurons, 1 = wherever range_max exists, 2 = off)
+                           // (0 = where range_max exists and the map has at least 32 ranges of 128 neurons, 1 = wherever range_max exists, 2 = off)
     int64_t opt_mask_bits; // plan: features handled as mask bits (0 = default by batch size, else 1..16)
     int plan_attr_set;
     int64_t opt_update_mib;  // som_update: workspace budget for its slab buffers in MiB (0 = 4096)

@@ -15,7 +15,7 @@
 //          it stays L2-resident from one neuron range to the next: 1024 x 1024 with 250k samples moves 223 GB
 //          instead of 257 GB and runs 0.4 % faster), 1 = always, 2 = never
 //   key 10 pruning by range maxima in the row-table kernel (M % 128 == 0; exact, see k_bmu_table): 0 = on
-//          maps of at least 768 ranges of 128 neurons (where it pays), 1 = wherever som_norms has written the maxima, 2 = off
+//          maps of at least 32 ranges of 128 neurons, 1 = wherever som_norms has written the maxima, 2 = off
 //          (set before the first som_norms, it also spares the V * M / 128 floats of the maxima)
 #pragma once
 #define SOM_OPT_HOT_ROWS 1

@@ -149,7 +149,7 @@ def test_mask_feature_counts(som_mod, mask_bits):
 def test_pruning_by_range_maxima_changes_nothing(som_mod, lane_neurons, codebook):
     """The row-table kernel may skip a sample's tail rows for a neuron range whose scores cannot reach the
     sample's key (bounds from the per-range maxima that som_norms writes).  Forced on (by default it runs on
-    maps of 768 ranges of 128 neurons and more), its outputs are bit-identical to those of the full search and match the
+    maps of 32 ranges of 128 neurons and more; this map has 16), its outputs are bit-identical to those of the full search and match the
     oracle: on the benchmark's codebook recipe, on a smooth map (nearly everything is skipped), on a map of
     equal neurons (nothing can be skipped: every range ties) and on weights of both signs."""
     V, M, n = 30_000, 2_048, 40_000
