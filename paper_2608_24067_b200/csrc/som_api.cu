@@ -132,6 +132,7 @@ int som_destroy(som_handle* h)
     cudaFree(h->head);
     cudaFree(h->shadow);
     cudaFree(h->range_max);
+    cudaFree(h->range_order);
     if (h->aux_stream) {
         cudaStreamSynchronize(h->aux_stream);
         cudaEventDestroy(h->ev_fork);
@@ -172,6 +173,11 @@ int som_norms(som_handle* h, void* stream)
         if (cudaMalloc(reinterpret_cast<void**>(&h->range_max), (size_t)h->V * (size_t)(h->M / 128) * sizeof(float)) !=
             cudaSuccess) {
             h->range_max = nullptr;
+            (void)cudaGetLastError();
+        } else if (h->M / 128 <= 8192 &&  // (the order of the ranges: what one block sorts in shared memory)
+                   cudaMalloc(reinterpret_cast<void**>(&h->range_order), (size_t)(h->M / 128) * sizeof(int32_t)) !=
+                       cudaSuccess) {
+            h->range_order = nullptr;
             (void)cudaGetLastError();
         }
     }

@@ -462,7 +462,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const uint4* __restrict__ slots, int64_t n_pad,
             u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
             int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter,
-            const int* __restrict__ gate, int gate_want, int feed_keep_arg, const float* __restrict__ range_max, int V)
+            const int* __restrict__ gate, int gate_want, int feed_keep_arg, const float* __restrict__ range_max, int V,
+            const int32_t* __restrict__ range_order)
 {
     if (som_gated_off(gate, gate_want)) return;
     uint64_t feed_keep;  // L2 cache policy of the slot and key stream: "evict last" on small batches, else normal
@@ -520,9 +521,16 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
         // The last units of the launch are claimed in quarters, so that the blocks run out of
         // work within a quarter of a unit of each other.
         const int whole = unit < n_whole ? unit : n_whole + ((unit - n_whole) >> 2);
-        const int range = whole / parts;
+        const int range = whole / parts;  // (position in the launch's order of ranges)
         const int part = whole - range * parts;
-        const int64_t i0 = (int64_t)range * T;
+        // With pruning the 128-neuron ranges are taken in the order of their smallest ||w||^2 (written by
+        // som_norms): the ranges that are likeliest to hold a sample's best unit come first, its key is tight
+        // sooner and more of the later ranges are skipped.  (The result does not depend on the order.)
+        int64_t i0 = (int64_t)range * T;
+        if (PRUNE && range_order) {
+            constexpr int PER = 128 / T;  // ranges of this layout per 128 neurons
+            i0 = (int64_t)range_order[range / PER] * 128 + (int64_t)(range % PER) * T;
+        }
         if (range != cur_range) {
             // rows start on 16-byte boundaries when M * sizeof(weight) does (the range offset always does)
             if (((M * (int64_t)sizeof(typename L::Store)) & 15) == 0 && (reinterpret_cast<uintptr_t>(W) & 15) == 0 &&
@@ -953,7 +961,7 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
                                           KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
                                           n_units, n_whole,
                                           reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want,
-                                          feed_keep, prune ? h->range_max : nullptr, (int)h->V);
+                                          feed_keep, prune ? h->range_max : nullptr, (int)h->V, prune ? h->range_order : nullptr);
         return cudaGetLastError();
     };
     if constexpr (L::CAN_PRUNE) {

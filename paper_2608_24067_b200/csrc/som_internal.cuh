@@ -33,6 +33,7 @@ struct som_handle {
     const __half* Wh;  // borrowed, feature-major fp16 codebook (som_create_f16), else nullptr
     float* range_max;  // owned, [M / 128][V]: per feature row and 128-neuron range the largest weight (written by
                        // som_norms when M % 128 == 0; nullptr = none); bounds for the search's pruning
+    int32_t* range_order;  // owned, [M / 128]: the 128-neuron ranges by ascending smallest ||w||^2 (nullptr = none)
     __half* shadow;    // owned fp16 copy of an fp32 codebook for the two-stage search (nullptr = none)
     unsigned int* wmax_bits;  // device, written by som_norms with the shadow: [0] float bits of max |weight|,
                               // [SOM_AUX_HAS_NEGATIVE] 1 if a weight is negative, [SOM_AUX_HMAX] float bits of max ||w||^2/2

@@ -220,6 +220,44 @@ __global__ void k_norms_combine(const double* __restrict__ partial, int64_t M, i
     if (hmax_bits) atomicMax(hmax_bits, __float_as_uint((float)(0.5 * s)));
 }
 
+// The 128-neuron ranges ordered by their smallest ||w||^2 / 2 (one block; bitonic sort in shared memory of up to
+// 8192 ranges, ties by range number): the search kernel visits them in this order when it prunes.
+constexpr int ORDER_MAX_RANGES = 8192;
+__global__ void __launch_bounds__(1024)
+k_range_order(const float* __restrict__ hnorm, int n_ranges, int32_t* __restrict__ order)
+{
+    extern __shared__ unsigned long long okeys[];  // (ordered float bits << 32) | range
+    int n_pow = 1;
+    while (n_pow < n_ranges) n_pow *= 2;
+    for (int r = threadIdx.x; r < n_pow; r += 1024) {
+        unsigned long long k = ~0ull;
+        if (r < n_ranges) {
+            float m = 3.0e38f;
+            for (int j = 0; j < 128; ++j) m = fminf(m, hnorm[(int64_t)r * 128 + j]);
+            unsigned int b = __float_as_uint(m);  // (norms are non-negative: their bits order like unsigned integers)
+            k = ((unsigned long long)b << 32) | (unsigned int)r;
+        }
+        okeys[r] = k;
+    }
+    __syncthreads();
+    for (int size = 2; size <= n_pow; size *= 2)
+        for (int stride = size / 2; stride > 0; stride /= 2) {
+            for (int i = threadIdx.x; i < n_pow; i += 1024) {
+                const int j = i ^ stride;
+                if (j > i) {
+                    const bool up = (i & size) == 0;
+                    const unsigned long long a = okeys[i], b = okeys[j];
+                    if ((a > b) == up) {
+                        okeys[i] = b;
+                        okeys[j] = a;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    for (int r = threadIdx.x; r < n_ranges; r += 1024) order[r] = (int32_t)(okeys[r] & 0xffffffffull);
+}
+
 struct NormPlan {
     int vec;
     int splits;
@@ -288,5 +326,14 @@ int som_launch_norms(som_handle* h, cudaStream_t st)
         (p.vec == 4 && h->shadow && !h->Wh) ? h->wmax_bits + SOM_AUX_HMAX : nullptr);
     SOM_CK(h, cudaGetLastError());
     h->launches += 2;
+    if (h->range_order) {
+        const int n_ranges = (int)(h->M / 128);
+        int n_pow = 1;
+        while (n_pow < n_ranges) n_pow *= 2;
+        SOM_CK(h, cudaFuncSetAttribute(k_range_order, cudaFuncAttributeMaxDynamicSharedMemorySize, n_pow * 8));
+        k_range_order<<<1, 1024, (size_t)n_pow * 8, st>>>(h->hnorm, n_ranges, h->range_order);
+        SOM_CK(h, cudaGetLastError());
+        h->launches += 1;
+    }
     return SOM_OK;
 }
