@@ -167,10 +167,10 @@ int som_norms(som_handle* h, void* stream)
     int rc = ensure_bytes(h, &h->ws, &h->ws_bytes, som_norms_workspace_bytes(h));
     if (rc) return rc;
     if (h->timing && (rc = ensure_events(h))) return rc;
-    // per-range maxima of the feature rows for the search's pruning (M % 128 == 0): V * M / 128
+    // per-range maxima of the feature rows for the search's pruning (M % 128 == 0): V * M / 32
     // floats, allocated by the first call; without the memory the search simply does not prune
     if (!h->range_max && h->M % 128 == 0 && h->opt_prune != 2) {
-        if (cudaMalloc(reinterpret_cast<void**>(&h->range_max), (size_t)h->V * (size_t)(h->M / 128) * sizeof(float)) !=
+        if (cudaMalloc(reinterpret_cast<void**>(&h->range_max), (size_t)h->V * (size_t)(h->M / 32) * sizeof(float)) !=
             cudaSuccess) {
             h->range_max = nullptr;
             (void)cudaGetLastError();

@@ -197,6 +197,7 @@ struct LayF32 {
     // than two)
     static constexpr int TAILS_AHEAD = R_ >= 16 ? 3 : 4;
     static constexpr bool CAN_PRUNE = true;
+    static constexpr int GROUPS = R_ / 4;       // (pruning) 32-neuron groups of a team's range with bounds of their own
     static constexpr float SEED_SIGN = 1.f;     // scores are held as they are
     typedef Acc<H> Scores;
     typedef Acc<H> Slice;
@@ -269,6 +270,7 @@ struct LayF16 {
     static constexpr int R = 8, T = 64, ROWB = T * 2;
     static constexpr int TAILS_AHEAD = 4;
     static constexpr bool CAN_PRUNE = true;
+    static constexpr int GROUPS = 1;  // (a lane's eight neurons lie in one 32-neuron group, but which depends on the lane)
     static constexpr float SEED_SIGN = -1.f;  // the seed array holds -||w||^2/2
     struct Scores { float v[8]; };
     typedef uint4 Slice;
@@ -346,6 +348,7 @@ struct LayF16W {
     static constexpr int R = 16, T = 128, ROWB = T * 2;
     static constexpr int TAILS_AHEAD = 4;
     static constexpr bool CAN_PRUNE = true;
+    static constexpr int GROUPS = 1;
     static constexpr float SEED_SIGN = -1.f;
     struct Scores { float v[16]; };
     struct Slice { uint4 g[2]; };
@@ -429,23 +432,52 @@ struct LayF16W {
 };
 
 // ---- pruning helpers ---------------------------------------------------------------------------
-// smallest score over the team's 8 * R neurons (all lanes of the team call it together)
+// Smallest score of the team's neurons, per 32-neuron group where the layout keeps the groups apart (fp32: the
+// lane's x-th quad of neurons lies in group x), else over the whole range (all lanes of the team call it together).
 template <typename L>
-__device__ __forceinline__ float team_min(const typename L::Scores& s, uint32_t team_lanes)
+__device__ __forceinline__ void group_min(const typename L::Scores& s, uint32_t team_lanes, float (&lo)[L::GROUPS])
 {
-    constexpr int R = L::R;
+    constexpr int R = L::R, G = L::GROUPS;
     float a[R];
     L::unpack(s, a);
-    float lo = fminf(fminf(a[0], a[1]), fminf(a[2], a[3]));
-    if (R >= 8) lo = fminf(lo, fminf(fminf(a[4 % R], a[5 % R]), fminf(a[6 % R], a[7 % R])));
-    if (R == 16) {
-        lo = fminf(lo, fminf(fminf(a[8 % R], a[9 % R]), fminf(a[10 % R], a[11 % R])));
-        lo = fminf(lo, fminf(fminf(a[12 % R], a[13 % R]), fminf(a[14 % R], a[15 % R])));
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        constexpr int PER = R / G;  // neurons of the lane per group
+        float m = a[g * PER];
+#pragma unroll
+        for (int j = 1; j < PER; ++j) m = fminf(m, a[g * PER + j]);
+        m = fminf(m, __shfl_xor_sync(team_lanes, m, 1));
+        m = fminf(m, __shfl_xor_sync(team_lanes, m, 2));
+        m = fminf(m, __shfl_xor_sync(team_lanes, m, 4));
+        lo[g] = m;
     }
-    lo = fminf(lo, __shfl_xor_sync(team_lanes, lo, 1));
-    lo = fminf(lo, __shfl_xor_sync(team_lanes, lo, 2));
-    lo = fminf(lo, __shfl_xor_sync(team_lanes, lo, 4));
-    return lo;
+}
+
+// The bounds of one table entry (four floats: the largest weight of a feature in the four 32-neuron groups of a
+// 128-neuron range) for a layout whose range starts at group g0 and spans SPAN groups: G = SPAN values, or their
+// maximum (G = 1).  `e` points at the entry's first float.
+template <int G, int SPAN>
+__device__ __forceinline__ void entry_bounds(const float* __restrict__ e, int g0, float (&b)[G])
+{
+    float v[SPAN];
+    if constexpr (SPAN == 4) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(e));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else if constexpr (SPAN == 2) {
+        const float2 t = __ldg(reinterpret_cast<const float2*>(e + g0));
+        v[0] = t.x; v[1] = t.y;
+    } else {
+        v[0] = __ldg(e + g0);
+    }
+    if constexpr (G == SPAN) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) b[g] = v[g];
+    } else {
+        float m = v[0];
+#pragma unroll
+        for (int g = 1; g < SPAN; ++g) m = fmaxf(m, v[g]);
+        b[0] = m;
+    }
 }
 
 #define SOM_HOT(code) L::sub(acc, L::lds(tab_q + (code) * ROWB))
@@ -501,6 +533,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
     // pruning: largest weight of every feature row in the live 128-neuron range (global), a copy for the table's
     // rows behind the table in shared memory, the lanes of this lane's team
     const float* rmax_range = nullptr;
+    int rmax_g0 = 0;  // first 32-neuron group of this layout's range inside its 128-neuron range
     float* rmax_hot = reinterpret_cast<float*>(tab + (size_t)(n_rows + 1) * ROWB);
     const uint32_t team_lanes = 0xffu << (8 * sub);
     const unsigned char* w_q = reinterpret_cast<const unsigned char*>(W);
@@ -546,10 +579,16 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             i_first = (uint32_t)i_lane;
             w_q = reinterpret_cast<const unsigned char*>(W + (i_lane < M ? i_lane : 0));
             if constexpr (PRUNE) {
-                rmax_range = range_max + (i0 >> 7) * (int64_t)V;
+                rmax_range = range_max + (i0 >> 7) * (int64_t)V * 4;  // (four floats per feature)
+                rmax_g0 = (int)((i0 & 127) >> 5);
                 for (int c = threadIdx.x; c <= n_rows; c += THREADS) {
                     const int f = c < n_rows ? slot_feat[c] : -1;
-                    rmax_hot[c] = f >= 0 ? rmax_range[f] : 0.f;  // (the zero row and unused rows take nothing off)
+                    float hb[L::GROUPS];
+#pragma unroll
+                    for (int g = 0; g < L::GROUPS; ++g) hb[g] = 0.f;  // (the zero row and unused rows take nothing off)
+                    if (f >= 0) entry_bounds<L::GROUPS, T / 32>(rmax_range + (int64_t)f * 4, rmax_g0, hb);
+#pragma unroll
+                    for (int g = 0; g < L::GROUPS; ++g) rmax_hot[c * L::GROUPS + g] = hb[g];
                 }
             }
             for (int c = threadIdx.x; c < T; c += THREADS)
@@ -573,8 +612,10 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 
         uint32_t curmask = 0;
         Scores base = L::seed(hn_sh, q);
-        float base_lo = 0.f;
-        if constexpr (PRUNE) base_lo = team_min<L>(base, team_lanes);
+        float base_lo[L::GROUPS];
+#pragma unroll
+        for (int g = 0; g < L::GROUPS; ++g) base_lo[g] = 0.f;
+        if constexpr (PRUNE) group_min<L>(base, team_lanes, base_lo);
         for (;;) {
             int chunk = 0;
             if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
@@ -609,13 +650,14 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 //      bounds of its codes, the test, and the list of survivors in order.
                 const int n_chunk = 4 * rounds;
                 uint32_t hdrs[CHUNK / 32];
-                float los[CHUNK / 32];  // smallest prefix score for the masks of this lane's samples (step 1 -> step 2)
+                float los[CHUNK / 32][L::GROUPS];  // smallest prefix scores for the masks of this lane's samples (step 1 -> 2)
 #pragma unroll
                 for (int p = 0; p < CHUNK / 32; ++p) {
                     const int pos = lane + 32 * p;
                     hdrs[p] = pos < n_chunk ? __ldcg(reinterpret_cast<const uint32_t*>(slots + (w0 + pos) * SLOT_Q))
                                             : (SOM_SLOT_NT_OVERFLOW << 24);
-                    los[p] = 0.f;
+#pragma unroll
+                    for (int g = 0; g < L::GROUPS; ++g) los[p][g] = 0.f;
                 }
 #pragma unroll
                 for (int p = 0; p < CHUNK / 32; ++p) {
@@ -633,11 +675,14 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                                 L::sub(base, L::lds(tab_q + b * ROWB));
                             }
                             curmask = mask;
-                            base_lo = team_min<L>(base, team_lanes);
+                            group_min<L>(base, team_lanes, base_lo);
                         }
                         // lane 4 * rr + s of the warp owns the sample that team s has just looked at
-                        const float t = __shfl_sync(0xffffffffu, base_lo, 8 * (lane & 3));
-                        if ((lane >> 2) == rr) los[p] = t;
+#pragma unroll
+                        for (int g = 0; g < L::GROUPS; ++g) {
+                            const float t = __shfl_sync(0xffffffffu, base_lo[g], 8 * (lane & 3));
+                            if ((lane >> 2) == rr) los[p][g] = t;
+                        }
                     }
                 }
 #pragma unroll
@@ -653,18 +698,35 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         const u64 key0 = __ldcg(filter_keys + w0 + pos);
                         const uint32_t hw[6] = {s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};  // hot codes 0..11
                         const uint32_t tw[5] = {s2.x, s2.y, s2.z, s2.w, s0.y};        // tail codes 0..9
-                        float bnd = 0.f;
+                        float bnd[L::GROUPS];
+#pragma unroll
+                        for (int g = 0; g < L::GROUPS; ++g) bnd[g] = 0.f;
 #pragma unroll
                         for (int j = 0; j < SOM_SLOT_MAX_HOT; ++j)
-                            if ((uint32_t)j < nh) bnd += rmax_hot[(j & 1) ? hi16(hw[j >> 1]) : lo16(hw[j >> 1])];
+                            if ((uint32_t)j < nh) {
+                                const float* hb = rmax_hot + ((j & 1) ? hi16(hw[j >> 1]) : lo16(hw[j >> 1])) * L::GROUPS;
+#pragma unroll
+                                for (int g = 0; g < L::GROUPS; ++g) bnd[g] += hb[g];
+                            }
 #pragma unroll
                         for (int j = 0; j < SOM_SLOT_MAX_TAIL; ++j)
-                            if ((uint32_t)j < nt) bnd += __ldg(rmax_range + ((j & 1) ? hi16(tw[j >> 1]) : lo16(tw[j >> 1])));
+                            if ((uint32_t)j < nt) {
+                                float tb[L::GROUPS];
+                                entry_bounds<L::GROUPS, T / 32>(
+                                    rmax_range + (size_t)((j & 1) ? hi16(tw[j >> 1]) : lo16(tw[j >> 1])) * 4, rmax_g0, tb);
+#pragma unroll
+                                for (int g = 0; g < L::GROUPS; ++g) bnd[g] += tb[g];
+                            }
                         const uint32_t cu = (uint32_t)(key0 >> 32);
                         const float cs = __uint_as_float((cu & 0x80000000u) ? (cu ^ 0x80000000u) : ~cu);
-                        const float lo = los[p];
-                        // (an empty key decodes to NaN: the comparison is false and the sample stays live)
-                        live = !(lo - bnd > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd)));
+                        // the sample survives if some group of the range may still hold a candidate
+                        // (an empty key decodes to NaN: the comparisons are false and the sample stays live)
+                        live = false;
+#pragma unroll
+                        for (int g = 0; g < L::GROUPS; ++g) {
+                            const float lo = los[p][g];
+                            live = live || !(lo - bnd[g] > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd[g])));
+                        }
                     }
                     const uint32_t votes = __ballot_sync(0xffffffffu, live);
                     if (live) live_list[n_live + __popc(votes & ((1u << lane) - 1u))] = (unsigned char)pos;
@@ -947,7 +1009,7 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
     //  slower at 512 x 512: it tests against the second-best key, which skips less)
     if (codebook_v != static_cast<const void*>(h->W) && codebook_v != static_cast<const void*>(h->Wh)) prune = false;
-    if (prune) smem += ((size_t)(SOM_PLAN_MASK_FEATURES + n_hot + 1) * sizeof(float) + 15) / 16 * 16;  // the table rows' maxima
+    if (prune) smem += ((size_t)(SOM_PLAN_MASK_FEATURES + n_hot + 1) * L::GROUPS * sizeof(float) + 15) / 16 * 16;  // the table rows' maxima
     auto launch = [&](auto kern) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -1004,7 +1066,7 @@ SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
     // Defaults keep dynamic + static shared memory under 196 KB: one step more and the SM's
     // carve-out leaves 28 KB instead of 60 KB of L1, which costs 12 % at 128x128 (measured).
     int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows
-                                   : (row_bytes == 128 ? (f16 ? 1456 : 1376) : (row_bytes == 512 ? 352 : 720));
+                                   : (row_bytes == 128 ? (f16 ? 1456 : 1376) : (row_bytes == 512 ? 343 : 720));
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
     g.row_bytes = row_bytes;

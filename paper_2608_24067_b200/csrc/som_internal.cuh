@@ -31,7 +31,7 @@ struct som_handle {
     int64_t M;
     const float* W;    // borrowed, feature-major fp32 codebook (nullptr when stored as fp16)
     const __half* Wh;  // borrowed, feature-major fp16 codebook (som_create_f16), else nullptr
-    float* range_max;  // owned, [M / 128][V]: per feature row and 128-neuron range the largest weight (written by
+    float* range_max;  // owned, [M / 128][V][4]: per feature row, 128-neuron range and 32-neuron group the largest weight (written by
                        // som_norms when M % 128 == 0; nullptr = none); bounds for the search's pruning
     int32_t* range_order;  // owned, [M / 128]: the 128-neuron ranges by ascending smallest ||w||^2 (nullptr = none)
     __half* shadow;    // owned fp16 copy of an fp32 codebook for the two-stage search (nullptr = none)

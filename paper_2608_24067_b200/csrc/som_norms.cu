@@ -27,17 +27,18 @@ __device__ __forceinline__ void store_half4(__half* dst, const float4 w)
 // |weight| (as float bits, through atomicMax: non-negative floats order like their bits), which
 // the two-stage search uses for its first pass and its error bound.
 // RMAX (VEC == 4 and M % 128 == 0 only): the pass also writes, for every feature row and every range of 128
-// neurons (the 128 neurons a warp holds), the largest weight of the row in the range: range_max[range * V + v].
-// The row-table search uses it to bound what a sample's tail features can still take off the scores of a
-// whole range (see k_bmu_table).
+// neurons (the 128 neurons a warp holds), the largest weight of the row in each of the range's four groups of
+// 32 neurons: range_max[(range * V + v) * 4 + group].  The row-table search uses them to bound what a sample's
+// rows can still take off the scores of a range (see k_bmu_table).
 __device__ __forceinline__ void store_range_max(float* __restrict__ dst, float m)
 {
-    // max over the warp in one instruction: floats ordered as signed integers
+    // max over each group of eight lanes (32 neurons) in one instruction: floats ordered as signed integers
     int key = __float_as_int(m);
     key ^= (key >> 31) & 0x7fffffff;
-    key = __reduce_max_sync(0xffffffffu, key);
+    const unsigned int lane = threadIdx.x & 31;
+    key = __reduce_max_sync(0xffu << (lane & 24), key);
     key ^= (key >> 31) & 0x7fffffff;
-    if ((threadIdx.x & 31) == 0) *dst = __int_as_float(key);
+    if ((lane & 7) == 0) dst[lane >> 3] = __int_as_float(key);
 }
 
 template <int VEC, bool SHADOW, bool RMAX>
@@ -57,7 +58,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
     __half* ps = SHADOW ? shadow + (int64_t)v0 * M + i : nullptr;
     float wmax = 0.f, wmin = 0.f;
     // (RMAX: M % 128 == 0, so a warp is all inside M and holds exactly range i / 128)
-    float* pr = RMAX ? range_max + (i / 128) * (int64_t)V + v0 : nullptr;
+    float* pr = RMAX ? range_max + ((i / 128) * (int64_t)V + v0) * 4 : nullptr;
     int v = v0;
     if (VEC == 4) {
         for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
@@ -72,7 +73,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
                     wmax = fmaxf(wmax, fmaxf(fmaxf(fabsf(w[u].x), fabsf(w[u].y)), fmaxf(fabsf(w[u].z), fabsf(w[u].w))));
                     wmin = fminf(wmin, fminf(fminf(w[u].x, w[u].y), fminf(w[u].z, w[u].w)));
                 }
-                if (RMAX) store_range_max(pr + u, fmaxf(fmaxf(w[u].x, w[u].y), fmaxf(w[u].z, w[u].w)));
+                if (RMAX) store_range_max(pr + 4 * u, fmaxf(fmaxf(w[u].x, w[u].y), fmaxf(w[u].z, w[u].w)));
                 acc[0] = fma((double)w[u].x, (double)w[u].x, acc[0]);
                 acc[1 % VEC] = fma((double)w[u].y, (double)w[u].y, acc[1 % VEC]);
                 acc[2 % VEC] = fma((double)w[u].z, (double)w[u].z, acc[2 % VEC]);
@@ -80,7 +81,7 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
             }
             p += (int64_t)NORM_UNROLL * M;
             if (SHADOW) ps += (int64_t)NORM_UNROLL * M;
-            if (RMAX) pr += NORM_UNROLL;
+            if (RMAX) pr += 4 * NORM_UNROLL;
         }
         for (; v < v1; ++v) {
             float4 w = __ldcs(reinterpret_cast<const float4*>(p));
@@ -90,7 +91,10 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
                 wmin = fminf(wmin, fminf(fminf(w.x, w.y), fminf(w.z, w.w)));
                 ps += M;
             }
-            if (RMAX) store_range_max(pr++, fmaxf(fmaxf(w.x, w.y), fmaxf(w.z, w.w)));
+            if (RMAX) {
+                store_range_max(pr, fmaxf(fmaxf(w.x, w.y), fmaxf(w.z, w.w)));
+                pr += 4;
+            }
             acc[0] = fma((double)w.x, (double)w.x, acc[0]);
             acc[1 % VEC] = fma((double)w.y, (double)w.y, acc[1 % VEC]);
             acc[2 % VEC] = fma((double)w.z, (double)w.z, acc[2 % VEC]);
@@ -119,16 +123,17 @@ k_norms_partial(const float* __restrict__ W, int64_t M, int V, int rows_per_spli
 
 // The same pass over an fp16-stored codebook: VEC = 8 neurons per thread (one 128-bit load of
 // eight halves per row) or 1; every weight is widened exactly and squared in fp64.
-// RMAX (VEC == 8, M % 128 == 0): a half-warp (16 threads x 8 neurons) holds one range of 128
+// RMAX (VEC == 8, M % 128 == 0): a half-warp (16 threads x 8 neurons) holds one range of 128, four threads a group of 32
 // neurons; its largest weight of every row goes to range_max[range * V + v] (see k_norms_partial).
 __device__ __forceinline__ void store_range_max_half(float* __restrict__ dst, float m)
 {
+    // a thread holds 8 neurons, four threads a group of 32, a half-warp the range of 128
     int key = __float_as_int(m);
     key ^= (key >> 31) & 0x7fffffff;
-    const unsigned int half_lanes = (threadIdx.x & 16) ? 0xffff0000u : 0x0000ffffu;
-    key = __reduce_max_sync(half_lanes, key);
+    const unsigned int lane = threadIdx.x & 31;
+    key = __reduce_max_sync(0xfu << (lane & 28), key);
     key ^= (key >> 31) & 0x7fffffff;
-    if ((threadIdx.x & 15) == 0) *dst = __int_as_float(key);
+    if ((lane & 3) == 0) dst[(lane & 15) >> 2] = __int_as_float(key);
 }
 
 template <int VEC, bool RMAX>
@@ -145,7 +150,7 @@ k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_s
     for (int k = 0; k < VEC; ++k) acc[k] = 0.0;
     const __half* p = W + (int64_t)v0 * M + i;
     // (RMAX: M % 128 == 0, so a half-warp, 16 threads x 8 neurons, is all inside M and holds range i / 128)
-    float* pr = RMAX ? range_max + (i / 128) * (int64_t)V + v0 : nullptr;
+    float* pr = RMAX ? range_max + ((i / 128) * (int64_t)V + v0) * 4 : nullptr;
     int v = v0;
     if (VEC == 8) {
         for (; v + NORM_UNROLL <= v1; v += NORM_UNROLL) {
@@ -164,10 +169,10 @@ k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_s
                     acc[(2 * k) % VEC] = fma((double)f.x, (double)f.x, acc[(2 * k) % VEC]);
                     acc[(2 * k + 1) % VEC] = fma((double)f.y, (double)f.y, acc[(2 * k + 1) % VEC]);
                 }
-                if (RMAX) store_range_max_half(pr + u, wm);
+                if (RMAX) store_range_max_half(pr + 4 * u, wm);
             }
             p += (int64_t)NORM_UNROLL * M;
-            if (RMAX) pr += NORM_UNROLL;
+            if (RMAX) pr += 4 * NORM_UNROLL;
         }
         for (; v < v1; ++v) {
             const uint4 w = __ldcs(reinterpret_cast<const uint4*>(p));
@@ -180,7 +185,10 @@ k_norms_partial_h(const __half* __restrict__ W, int64_t M, int V, int rows_per_s
                 acc[(2 * k) % VEC] = fma((double)f.x, (double)f.x, acc[(2 * k) % VEC]);
                 acc[(2 * k + 1) % VEC] = fma((double)f.y, (double)f.y, acc[(2 * k + 1) % VEC]);
             }
-            if (RMAX) store_range_max_half(pr++, wm);
+            if (RMAX) {
+                store_range_max_half(pr, wm);
+                pr += 4;
+            }
             p += M;
         }
     } else {
