@@ -182,7 +182,7 @@ def test_pruning_by_range_maxima_changes_nothing(som_mod, lane_neurons, codebook
                           outs[1][0], outs[1][1], rows)
 
 
-@pytest.mark.parametrize("mode", ["f16-8", "f16-16", "two-stage"])
+@pytest.mark.parametrize("mode", ["f16-8", "f16-16", "two-stage"])  # (the 8-neuron fp16 layout does not prune)
 @pytest.mark.parametrize("codebook", ["recipe", "smooth", "negative"])
 def test_pruning_with_fp16_rows(som_mod, mode, codebook):
     """The same for an fp16-stored codebook (maxima of the stored halves, both fp16 layouts) and with the
