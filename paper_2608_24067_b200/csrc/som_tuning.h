@@ -2,7 +2,7 @@
 // They exist for benchmarking and for the tests that walk every template instance; 0 always means
 // "the measured default".  A reusable plan (som_plan_create) is tied to their values at its creation.
 //
-//   key 1  hot rows kept in shared memory beside the 16 mask rows (default: 352 rows of 512 bytes, 720 of
+//   key 1  hot rows kept in shared memory beside the 16 mask rows (default: 343 rows of 512 bytes, 720 of
 //          256 bytes, 1376 / 1456 of 128 bytes: what keeps table + slot rings under 196 KB, so that the
 //          SM keeps a 60 KB L1)
 //   key 2  block size: 512, 576 (wide fp32 layout only), 640, 768, 896, 1024
