@@ -662,24 +662,36 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 #pragma unroll
                     for (int g = 0; g < L::GROUPS; ++g) los[p][g] = 0.f;
                 }
+                auto to_mask = [&](uint32_t mask) {  // the team's prefix scores and their minima for this mask
+                    if (mask == curmask) return;
+                    base = L::seed(hn_sh, q);
+                    uint32_t mm = mask;
+                    while (mm) {
+                        const int b = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        L::sub(base, L::lds(tab_q + b * ROWB));
+                    }
+                    curmask = mask;
+                    group_min<L>(base, team_lanes, base_lo);
+                };
 #pragma unroll
                 for (int p = 0; p < CHUNK / 32; ++p) {
+                    if (32 * p >= n_chunk) break;  // (the same for every lane)
+                    // The samples are sorted by mask, so nearly always the 32 of this step share one: then every
+                    // team holds the same minima and every lane takes them as they are.
+                    const uint32_t my_mask = hdrs[p] & 0xffffu;
+                    const uint32_t first_mask = __shfl_sync(0xffffffffu, my_mask, 0);
+                    if (__all_sync(0xffffffffu, lane + 32 * p >= n_chunk || my_mask == first_mask)) {
+                        to_mask(first_mask);
+#pragma unroll
+                        for (int g = 0; g < L::GROUPS; ++g) los[p][g] = base_lo[g];
+                        continue;
+                    }
 #pragma unroll 1
                     for (int rr = 0; rr < 8; ++rr) {
                         const uint32_t hdr = __shfl_sync(0xffffffffu, hdrs[p], 4 * rr + sub);
                         if (32 * p + 4 * rr >= n_chunk) break;  // (the same for every lane)
-                        const uint32_t mask = hdr & 0xffffu;
-                        if (mask != curmask) {
-                            base = L::seed(hn_sh, q);
-                            uint32_t mm = mask;
-                            while (mm) {
-                                const int b = __ffs(mm) - 1;
-                                mm &= mm - 1;
-                                L::sub(base, L::lds(tab_q + b * ROWB));
-                            }
-                            curmask = mask;
-                            group_min<L>(base, team_lanes, base_lo);
-                        }
+                        to_mask(hdr & 0xffffu);
                         // lane 4 * rr + s of the warp owns the sample that team s has just looked at
 #pragma unroll
                         for (int g = 0; g < L::GROUPS; ++g) {
