@@ -652,16 +652,6 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 //      Step 2, a lane per sample (32 samples at a time, all their loads in flight together): the
                 //      bounds of its codes, the test, and the list of survivors in order.
                 const int n_chunk = 4 * rounds;
-                uint32_t hdrs[CHUNK / 32];
-                float los[CHUNK / 32][L::GROUPS];  // smallest prefix scores for the masks of this lane's samples (step 1 -> 2)
-#pragma unroll
-                for (int p = 0; p < CHUNK / 32; ++p) {
-                    const int pos = lane + 32 * p;
-                    hdrs[p] = pos < n_chunk ? __ldcg(reinterpret_cast<const uint32_t*>(slots + (w0 + pos) * SLOT_Q))
-                                            : (SOM_SLOT_NT_OVERFLOW << 24);
-#pragma unroll
-                    for (int g = 0; g < L::GROUPS; ++g) los[p][g] = 0.f;
-                }
                 auto to_mask = [&](uint32_t mask) {  // the team's prefix scores and their minima for this mask
                     if (mask == curmask) return;
                     base = L::seed(hn_sh, q);
@@ -674,43 +664,60 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     curmask = mask;
                     group_min<L>(base, team_lanes, base_lo);
                 };
+                // the slot and key of this lane's sample of step p (a step's loads are issued one step ahead)
+                uint4 n0, n1, n2;
+                u64 nkey;
+                auto load_step = [&](int p) {
+                    const int pos = lane + 32 * p;
+                    n0 = make_uint4(SOM_SLOT_NT_OVERFLOW << 24, 0u, 0u, 0u);
+                    n1 = n2 = make_uint4(0u, 0u, 0u, 0u);
+                    nkey = 0;
+                    if (pos < n_chunk) {
+                        const uint4* sl = slots + (w0 + pos) * SLOT_Q;
+                        n0 = __ldcg(sl);
+                        n1 = __ldcg(sl + 1);
+                        n2 = __ldcg(sl + 2);
+                        nkey = __ldcg(filter_keys + w0 + pos);
+                    }
+                };
+                load_step(0);
 #pragma unroll
                 for (int p = 0; p < CHUNK / 32; ++p) {
                     if (32 * p >= n_chunk) break;  // (the same for every lane)
-                    // The samples are sorted by mask, so nearly always the 32 of this step share one: then every
-                    // team holds the same minima and every lane takes them as they are.
-                    const uint32_t my_mask = hdrs[p] & 0xffffu;
+                    const int pos = lane + 32 * p;
+                    const uint4 s0 = n0, s1 = n1, s2 = n2;
+                    const u64 key0 = nkey;
+                    if (p + 1 < CHUNK / 32 && 32 * (p + 1) < n_chunk) load_step(p + 1);
+                    const uint32_t hdr = s0.x;
+                    float lo[L::GROUPS];
+                    // Step 1.  The samples are sorted by mask, so nearly always the 32 of this step share one: then
+                    // every team holds the same minima and every lane takes them as they are.
+                    const uint32_t my_mask = hdr & 0xffffu;
                     const uint32_t first_mask = __shfl_sync(0xffffffffu, my_mask, 0);
-                    if (__all_sync(0xffffffffu, lane + 32 * p >= n_chunk || my_mask == first_mask)) {
+                    if (__all_sync(0xffffffffu, pos >= n_chunk || my_mask == first_mask)) {
                         to_mask(first_mask);
 #pragma unroll
-                        for (int g = 0; g < L::GROUPS; ++g) los[p][g] = base_lo[g];
-                        continue;
-                    }
-#pragma unroll 1
-                    for (int rr = 0; rr < 8; ++rr) {
-                        const uint32_t hdr = __shfl_sync(0xffffffffu, hdrs[p], 4 * rr + sub);
-                        if (32 * p + 4 * rr >= n_chunk) break;  // (the same for every lane)
-                        to_mask(hdr & 0xffffu);
-                        // lane 4 * rr + s of the warp owns the sample that team s has just looked at
+                        for (int g = 0; g < L::GROUPS; ++g) lo[g] = base_lo[g];
+                    } else {
 #pragma unroll
-                        for (int g = 0; g < L::GROUPS; ++g) {
-                            const float t = __shfl_sync(0xffffffffu, base_lo[g], 8 * (lane & 3));
-                            if ((lane >> 2) == rr) los[p][g] = t;
+                        for (int g = 0; g < L::GROUPS; ++g) lo[g] = 0.f;
+#pragma unroll 1
+                        for (int rr = 0; rr < 8; ++rr) {
+                            const uint32_t h = __shfl_sync(0xffffffffu, hdr, 4 * rr + sub);
+                            if (32 * p + 4 * rr >= n_chunk) break;  // (the same for every lane)
+                            to_mask(h & 0xffffu);
+                            // lane 4 * rr + s of the warp owns the sample that team s has just looked at
+#pragma unroll
+                            for (int g = 0; g < L::GROUPS; ++g) {
+                                const float t = __shfl_sync(0xffffffffu, base_lo[g], 8 * (lane & 3));
+                                if ((lane >> 2) == rr) lo[g] = t;
+                            }
                         }
                     }
-                }
-#pragma unroll
-                for (int p = 0; p < CHUNK / 32; ++p) {
-                    const int pos = lane + 32 * p;
-                    if (32 * p >= n_chunk) break;
-                    const uint32_t hdr = hdrs[p];
+                    // Step 2.
                     const uint32_t nt = hdr >> 24, nh = (hdr >> 16) & 0xffu;
                     bool live = pos < n_chunk && nt != SOM_SLOT_NT_OVERFLOW;
                     if (live) {
-                        const uint4* sl = slots + (w0 + pos) * SLOT_Q;
-                        const uint4 s0 = __ldcg(sl), s1 = __ldcg(sl + 1), s2 = __ldcg(sl + 2);
-                        const u64 key0 = __ldcg(filter_keys + w0 + pos);
                         const uint32_t hw[6] = {s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};  // hot codes 0..11
                         const uint32_t tw[5] = {s2.x, s2.y, s2.z, s2.w, s0.y};        // tail codes 0..9
                         float bnd[L::GROUPS];
@@ -738,10 +745,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         // (an empty key decodes to NaN: the comparisons are false and the sample stays live)
                         live = false;
 #pragma unroll
-                        for (int g = 0; g < L::GROUPS; ++g) {
-                            const float lo = los[p][g];
-                            live = live || !(lo - bnd[g] > cs + 1e-5f * (fabsf(lo) + fabsf(cs) + fabsf(bnd[g])));
-                        }
+                        for (int g = 0; g < L::GROUPS; ++g)
+                            live = live || !(lo[g] - bnd[g] > cs + 1e-5f * (fabsf(lo[g]) + fabsf(cs) + fabsf(bnd[g])));
                     }
                     const uint32_t votes = __ballot_sync(0xffffffffu, live);
                     if (live) live_list[n_live + __popc(votes & ((1u << lane) - 1u))] = (unsigned char)pos;
