@@ -872,6 +872,38 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 // ---- tail rows ------------------------------------------------------------------
                 if (p0) L::sub(acc, tr0);
                 if (p1) L::sub(acc, tr1);
+                if constexpr (PRUNE) {
+                    // A survivor's rows are mostly cold (few samples of the batch read a given row of this range),
+                    // and a step of the warp waits for the slowest of its four teams: the later rows are loaded
+                    // as many at a time as the first ones, not one after the other.
+                    constexpr int A = L::TAILS_AHEAD;
+                    if constexpr (A >= 3) {
+                        if (p2) L::sub(acc, tr2);
+                    }
+                    if constexpr (A >= 4) {
+                        if (p3) L::sub(acc, tr3);
+                    }
+                    if (nt == SOM_SLOT_NT_OVERFLOW) {
+                        acc = L::worst();  // (never a survivor; see the other branch)
+                    } else {
+                        const uint32_t tc[5] = {s2.x, s2.y, s2.z, s2.w, s0.y};
+#pragma unroll
+                        for (int b = A; b < SOM_SLOT_MAX_TAIL; b += A) {
+                            if (nt > (uint32_t)b) {
+#pragma unroll
+                                for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
+                                    Slice& t = (j - b == 0) ? tr0 : ((j - b == 1) ? tr1 : ((j - b == 2) ? tr2 : tr3));
+                                    if (nt > (uint32_t)j) t = SOM_TAIL((j & 1) ? hi16(tc[j >> 1]) : lo16(tc[j >> 1]));
+                                }
+#pragma unroll
+                                for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
+                                    Slice& t = (j - b == 0) ? tr0 : ((j - b == 1) ? tr1 : ((j - b == 2) ? tr2 : tr3));
+                                    if (nt > (uint32_t)j) L::sub(acc, t);
+                                }
+                            }
+                        }
+                    }
+                } else {
                 if constexpr (L::TAILS_AHEAD >= 3) {
                     if (p2) L::sub(acc, tr2);
                 } else {
@@ -898,6 +930,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         // even out of line, cost the hot loop of every sample 15 to 20 %.)
                         acc = L::worst();
                     }
+                }
+
                 }
 
                 // ---- lane-local argmin, rare atomic combine ------------------------------------
