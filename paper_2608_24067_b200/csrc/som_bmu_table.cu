@@ -508,6 +508,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
     constexpr int R = L::R;
     constexpr int T = L::T;
     constexpr int ROWB = L::ROWB;
+    constexpr bool SECOND_TEST = PRUNE;  // (pruning) the search rounds test again before their tail rows
     constexpr int WARPS = THREADS / 32;
     typedef typename L::Scores Scores;
     typedef typename L::Slice Slice;
@@ -824,13 +825,32 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 
                 // ---- the first tail rows of this sample go in flight first ----------------------------
                 Slice tr0, tr1, tr2, tr3;
-                if (p0) tr0 = SOM_TAIL(lo16(s2.x));
-                if (p1) tr1 = SOM_TAIL(hi16(s2.x));
-                if constexpr (L::TAILS_AHEAD >= 3) {
-                    if (p2) tr2 = SOM_TAIL(lo16(s2.y));
-                }
-                if constexpr (L::TAILS_AHEAD >= 4) {
-                    if (p3) tr3 = SOM_TAIL(hi16(s2.y));
+                float tail_bound[L::GROUPS];  // (second test) this lane's share of the tail rows' bounds
+#pragma unroll
+                for (int g = 0; g < L::GROUPS; ++g) tail_bound[g] = 0.f;
+                if constexpr (!SECOND_TEST) {
+                    if (p0) tr0 = SOM_TAIL(lo16(s2.x));
+                    if (p1) tr1 = SOM_TAIL(hi16(s2.x));
+                    if constexpr (L::TAILS_AHEAD >= 3) {
+                        if (p2) tr2 = SOM_TAIL(lo16(s2.y));
+                    }
+                    if constexpr (L::TAILS_AHEAD >= 4) {
+                        if (p3) tr3 = SOM_TAIL(hi16(s2.y));
+                    }
+                } else {
+                    // Second test (below, after the hot rows): lane q of the team fetches the bounds of tail rows
+                    // q and q + 8; the rows themselves wait for the test.
+                    const uint32_t w = (q >> 1) == 0 ? s2.x : ((q >> 1) == 1 ? s2.y : ((q >> 1) == 2 ? s2.z : s2.w));
+                    if ((uint32_t)q < nt && nt <= (uint32_t)SOM_SLOT_MAX_TAIL)
+                        entry_bounds<L::GROUPS, T / 32>(rmax_range + (size_t)((q & 1) ? hi16(w) : lo16(w)) * 4, rmax_g0,
+                                                        tail_bound);
+                    if ((uint32_t)q + 8u < nt && nt <= (uint32_t)SOM_SLOT_MAX_TAIL) {
+                        float more[L::GROUPS];
+                        entry_bounds<L::GROUPS, T / 32>(rmax_range + (size_t)((q & 1) ? hi16(s0.y) : lo16(s0.y)) * 4, rmax_g0,
+                                                        more);
+#pragma unroll
+                        for (int g = 0; g < L::GROUPS; ++g) tail_bound[g] += more[g];
+                    }
                 }
 
                 // ---- mask prefix ------------------------------------------------------------
@@ -870,25 +890,45 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
                 // ---- tail rows ------------------------------------------------------------------
-                if (p0) L::sub(acc, tr0);
-                if (p1) L::sub(acc, tr1);
-                if constexpr (PRUNE) {
-                    // A survivor's rows are mostly cold (few samples of the batch read a given row of this range),
-                    // and a step of the warp waits for the slowest of its four teams: the later rows are loaded
-                    // as many at a time as the first ones, not one after the other.
+                if constexpr (SECOND_TEST) {
+                    // Second test, now that the scores hold the mask and hot rows exactly: if no neuron of the
+                    // team can get under the sample's key even when every tail row takes its largest weight of
+                    // the neuron's group off, the tail rows (mostly cold: few samples of a batch read a given row
+                    // of this range) are not read at all.  Such a sample offers no candidate either way.
+#pragma unroll
+                    for (int g = 0; g < L::GROUPS; ++g) {
+                        float t = tail_bound[g];
+                        t += __shfl_xor_sync(team_lanes, t, 1);
+                        t += __shfl_xor_sync(team_lanes, t, 2);
+                        t += __shfl_xor_sync(team_lanes, t, 4);
+                        tail_bound[g] = t;
+                    }
+                    const uint32_t cu2 = (uint32_t)(key0 >> 32);
+                    const float cs2 = __uint_as_float((cu2 & 0x80000000u) ? (cu2 ^ 0x80000000u) : ~cu2);
+                    bool may = false;
+                    {
+                        float sc[R];
+                        L::unpack(acc, sc);
+                        constexpr int PER = R / L::GROUPS;
+#pragma unroll
+                        for (int g = 0; g < L::GROUPS; ++g) {
+                            float m = sc[g * PER];
+#pragma unroll
+                            for (int j = 1; j < PER; ++j) m = fminf(m, sc[g * PER + j]);
+                            // (an empty key decodes to NaN: the comparison is false and the rows are read)
+                            may = may || !(m - tail_bound[g] > cs2 + 1e-5f * (fabsf(m) + fabsf(cs2) + fabsf(tail_bound[g])));
+                        }
+                    }
+                    if (!__any_sync(team_lanes, may)) continue;
+                    // A step of the warp waits for the slowest of its four teams: the rows are loaded
+                    // as many at a time as the registers allow, not one after the other.
                     constexpr int A = L::TAILS_AHEAD;
-                    if constexpr (A >= 3) {
-                        if (p2) L::sub(acc, tr2);
-                    }
-                    if constexpr (A >= 4) {
-                        if (p3) L::sub(acc, tr3);
-                    }
                     if (nt == SOM_SLOT_NT_OVERFLOW) {
                         acc = L::worst();  // (never a survivor; see the other branch)
                     } else {
                         const uint32_t tc[5] = {s2.x, s2.y, s2.z, s2.w, s0.y};
 #pragma unroll
-                        for (int b = A; b < SOM_SLOT_MAX_TAIL; b += A) {
+                        for (int b = 0; b < SOM_SLOT_MAX_TAIL; b += A) {
                             if (nt > (uint32_t)b) {
 #pragma unroll
                                 for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
@@ -904,6 +944,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         }
                     }
                 } else {
+                if (p0) L::sub(acc, tr0);
+                if (p1) L::sub(acc, tr1);
                 if constexpr (L::TAILS_AHEAD >= 3) {
                     if (p2) L::sub(acc, tr2);
                 } else {
