@@ -498,7 +498,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
             int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter,
             const int* __restrict__ gate, int gate_want, int feed_keep_arg, const float* __restrict__ range_max, int V,
-            const int32_t* __restrict__ range_order)
+            const int32_t* __restrict__ range_order, int second_test_arg)
 {
     if (som_gated_off(gate, gate_want)) return;
     uint64_t feed_keep;  // L2 cache policy of the slot and key stream: "evict last" on small batches, else normal
@@ -508,7 +508,10 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
     constexpr int R = L::R;
     constexpr int T = L::T;
     constexpr int ROWB = L::ROWB;
-    constexpr bool SECOND_TEST = PRUNE;  // (pruning) the search rounds test again before their tail rows
+    // (pruning) the search rounds test again before their tail rows: always where the bounds are kept per 32-neuron
+    // group; with one bound per range (fp16 layouts) only where the launcher says so (large maps), because the
+    // test makes the rows that are read after all wait for it
+    const bool second_test = PRUNE && (L::GROUPS > 1 || second_test_arg != 0);
     constexpr int WARPS = THREADS / 32;
     typedef typename L::Scores Scores;
     typedef typename L::Slice Slice;
@@ -828,7 +831,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 float tail_bound[L::GROUPS];  // (second test) this lane's share of the tail rows' bounds
 #pragma unroll
                 for (int g = 0; g < L::GROUPS; ++g) tail_bound[g] = 0.f;
-                if constexpr (!SECOND_TEST) {
+                if (!second_test) {
                     if (p0) tr0 = SOM_TAIL(lo16(s2.x));
                     if (p1) tr1 = SOM_TAIL(hi16(s2.x));
                     if constexpr (L::TAILS_AHEAD >= 3) {
@@ -890,23 +893,23 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
                 // ---- tail rows ------------------------------------------------------------------
-                if constexpr (SECOND_TEST) {
-                    // Second test, now that the scores hold the mask and hot rows exactly: if no neuron of the
-                    // team can get under the sample's key even when every tail row takes its largest weight of
-                    // the neuron's group off, the tail rows (mostly cold: few samples of a batch read a given row
-                    // of this range) are not read at all.  Such a sample offers no candidate either way.
+                if constexpr (PRUNE) {
+                    if (second_test) {
+                        // Second test, now that the scores hold the mask and hot rows exactly: if no neuron of the
+                        // team can get under the sample's key even when every tail row takes its largest weight of
+                        // the neuron's group off, the tail rows (mostly cold: few samples of a batch read a given
+                        // row of this range) are not read at all.  Such a sample offers no candidate either way.
 #pragma unroll
-                    for (int g = 0; g < L::GROUPS; ++g) {
-                        float t = tail_bound[g];
-                        t += __shfl_xor_sync(team_lanes, t, 1);
-                        t += __shfl_xor_sync(team_lanes, t, 2);
-                        t += __shfl_xor_sync(team_lanes, t, 4);
-                        tail_bound[g] = t;
-                    }
-                    const uint32_t cu2 = (uint32_t)(key0 >> 32);
-                    const float cs2 = __uint_as_float((cu2 & 0x80000000u) ? (cu2 ^ 0x80000000u) : ~cu2);
-                    bool may = false;
-                    {
+                        for (int g = 0; g < L::GROUPS; ++g) {
+                            float t = tail_bound[g];
+                            t += __shfl_xor_sync(team_lanes, t, 1);
+                            t += __shfl_xor_sync(team_lanes, t, 2);
+                            t += __shfl_xor_sync(team_lanes, t, 4);
+                            tail_bound[g] = t;
+                        }
+                        const uint32_t cu2 = (uint32_t)(key0 >> 32);
+                        const float cs2 = __uint_as_float((cu2 & 0x80000000u) ? (cu2 ^ 0x80000000u) : ~cu2);
+                        bool may = false;
                         float sc[R];
                         L::unpack(acc, sc);
                         constexpr int PER = R / L::GROUPS;
@@ -918,10 +921,11 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                             // (an empty key decodes to NaN: the comparison is false and the rows are read)
                             may = may || !(m - tail_bound[g] > cs2 + 1e-5f * (fabsf(m) + fabsf(cs2) + fabsf(tail_bound[g])));
                         }
+                        if (!__any_sync(team_lanes, may)) continue;
                     }
-                    if (!__any_sync(team_lanes, may)) continue;
                     // A step of the warp waits for the slowest of its four teams: the rows are loaded
-                    // as many at a time as the registers allow, not one after the other.
+                    // as many at a time as the registers allow, not one after the other (the first ones are in
+                    // flight since the round's start, unless they had to wait for the second test).
                     constexpr int A = L::TAILS_AHEAD;
                     if (nt == SOM_SLOT_NT_OVERFLOW) {
                         acc = L::worst();  // (never a survivor; see the other branch)
@@ -930,10 +934,12 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 #pragma unroll
                         for (int b = 0; b < SOM_SLOT_MAX_TAIL; b += A) {
                             if (nt > (uint32_t)b) {
+                                if (b > 0 || second_test) {
 #pragma unroll
-                                for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
-                                    Slice& t = (j - b == 0) ? tr0 : ((j - b == 1) ? tr1 : ((j - b == 2) ? tr2 : tr3));
-                                    if (nt > (uint32_t)j) t = SOM_TAIL((j & 1) ? hi16(tc[j >> 1]) : lo16(tc[j >> 1]));
+                                    for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
+                                        Slice& t = (j - b == 0) ? tr0 : ((j - b == 1) ? tr1 : ((j - b == 2) ? tr2 : tr3));
+                                        if (nt > (uint32_t)j) t = SOM_TAIL((j & 1) ? hi16(tc[j >> 1]) : lo16(tc[j >> 1]));
+                                    }
                                 }
 #pragma unroll
                                 for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
@@ -1105,6 +1111,10 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
     //  slower at 512 x 512: it tests against the second-best key, which skips less)
     if (codebook_v != static_cast<const void*>(h->W) && codebook_v != static_cast<const void*>(h->Wh)) prune = false;
+    // second test of the search rounds with one bound per range (wide fp16 layout): measured 12 to 14 % slower at
+    // 64 x 64 and 128 x 128 (most samples pass it and their rows then start late), 11 to 13 % faster at 512 x 512
+    // and 1024 x 1024; on from 1024 ranges
+    const int second_test = (h->M + 127) / 128 >= 1024;
     if (prune) smem += ((size_t)(SOM_PLAN_MASK_FEATURES + n_hot + 1) * L::GROUPS * sizeof(float) + 15) / 16 * 16;  // the table rows' maxima
     auto launch = [&](auto kern) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -1119,7 +1129,8 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
                                           KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
                                           n_units, n_whole,
                                           reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want,
-                                          feed_keep, prune ? h->range_max : nullptr, (int)h->V, prune ? h->range_order : nullptr);
+                                          feed_keep, prune ? h->range_max : nullptr, (int)h->V, prune ? h->range_order : nullptr,
+                                          second_test);
         return cudaGetLastError();
     };
     if constexpr (L::CAN_PRUNE) {
