@@ -198,6 +198,7 @@ struct LayF32 {
     static constexpr int TAILS_AHEAD = R_ >= 16 ? 3 : 4;
     static constexpr bool CAN_PRUNE = true;
     static constexpr int GROUPS = R_ / 4;       // (pruning) 32-neuron groups of a team's range with bounds of their own
+    static constexpr bool HALF_GROUPS = false;  // every lane's x-th quad of neurons lies in group x
     static constexpr float SEED_SIGN = 1.f;     // scores are held as they are
     typedef Acc<H> Scores;
     typedef Acc<H> Slice;
@@ -274,6 +275,7 @@ struct LayF16 {
     //  by reading, so it is not built)
     static constexpr bool CAN_PRUNE = false;
     static constexpr int GROUPS = 1;
+    static constexpr bool HALF_GROUPS = false;
     static constexpr float SEED_SIGN = -1.f;  // the seed array holds -||w||^2/2
     struct Scores { float v[8]; };
     typedef uint4 Slice;
@@ -351,7 +353,10 @@ struct LayF16W {
     static constexpr int R = 16, T = 128, ROWB = T * 2;
     static constexpr int TAILS_AHEAD = 4;
     static constexpr bool CAN_PRUNE = true;
-    static constexpr int GROUPS = 1;
+    // (pruning) the four 32-neuron groups of the range have bounds of their own; a lane's first eight neurons lie
+    // in group q >> 2, its second eight in group 2 + (q >> 2)
+    static constexpr int GROUPS = 4;
+    static constexpr bool HALF_GROUPS = true;
     static constexpr float SEED_SIGN = -1.f;
     struct Scores { float v[16]; };
     struct Slice { uint4 g[2]; };
@@ -435,24 +440,41 @@ struct LayF16W {
 };
 
 // ---- pruning helpers ---------------------------------------------------------------------------
-// Smallest score of the team's neurons, per 32-neuron group where the layout keeps the groups apart (fp32: the
-// lane's x-th quad of neurons lies in group x), else over the whole range (all lanes of the team call it together).
+// Smallest score of the team's neurons, per 32-neuron group where the layout keeps the groups apart, else over
+// the whole range.  fp32: every lane's x-th quad of neurons lies in group x.  Wide fp16 rows (HALF_GROUPS): a
+// lane's c-th eight neurons lie in group 2 c + (q >> 2), so lanes 0..3 and lanes 4..7 of the team each reduce among
+// themselves and then swap.  All lanes of the team call it together and all end up with all the minima.
 template <typename L>
-__device__ __forceinline__ void group_min(const typename L::Scores& s, uint32_t team_lanes, float (&lo)[L::GROUPS])
+__device__ __forceinline__ void group_min(const typename L::Scores& s, uint32_t team_lanes, int q, float (&lo)[L::GROUPS])
 {
     constexpr int R = L::R, G = L::GROUPS;
     float a[R];
     L::unpack(s, a);
+    if constexpr (L::HALF_GROUPS) {
+        constexpr int PER = 2 * R / G;  // neurons of the lane per group it has a share in
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        constexpr int PER = R / G;  // neurons of the lane per group
-        float m = a[g * PER];
+        for (int c = 0; c < G / 2; ++c) {
+            float m = a[c * PER];
 #pragma unroll
-        for (int j = 1; j < PER; ++j) m = fminf(m, a[g * PER + j]);
-        m = fminf(m, __shfl_xor_sync(team_lanes, m, 1));
-        m = fminf(m, __shfl_xor_sync(team_lanes, m, 2));
-        m = fminf(m, __shfl_xor_sync(team_lanes, m, 4));
-        lo[g] = m;
+            for (int j = 1; j < PER; ++j) m = fminf(m, a[c * PER + j]);
+            m = fminf(m, __shfl_xor_sync(team_lanes, m, 1));
+            m = fminf(m, __shfl_xor_sync(team_lanes, m, 2));
+            const float o = __shfl_xor_sync(team_lanes, m, 4);
+            lo[2 * c] = (q & 4) ? o : m;
+            lo[2 * c + 1] = (q & 4) ? m : o;
+        }
+    } else {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            constexpr int PER = R / G;  // neurons of the lane per group
+            float m = a[g * PER];
+#pragma unroll
+            for (int j = 1; j < PER; ++j) m = fminf(m, a[g * PER + j]);
+            m = fminf(m, __shfl_xor_sync(team_lanes, m, 1));
+            m = fminf(m, __shfl_xor_sync(team_lanes, m, 2));
+            m = fminf(m, __shfl_xor_sync(team_lanes, m, 4));
+            lo[g] = m;
+        }
     }
 }
 
@@ -498,7 +520,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             u64* __restrict__ keys, u64* __restrict__ keys2, u64* __restrict__ keys3, int parts,
             int64_t part_len, int n_units, int n_whole, int* __restrict__ unit_counter,
             const int* __restrict__ gate, int gate_want, int feed_keep_arg, const float* __restrict__ range_max, int V,
-            const int32_t* __restrict__ range_order, int second_test_arg)
+            const int32_t* __restrict__ range_order)
 {
     if (som_gated_off(gate, gate_want)) return;
     uint64_t feed_keep;  // L2 cache policy of the slot and key stream: "evict last" on small batches, else normal
@@ -508,10 +530,10 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
     constexpr int R = L::R;
     constexpr int T = L::T;
     constexpr int ROWB = L::ROWB;
-    // (pruning) the search rounds test again before their tail rows: always where the bounds are kept per 32-neuron
-    // group; with one bound per range (fp16 layouts) only where the launcher says so (large maps), because the
-    // test makes the rows that are read after all wait for it
-    const bool second_test = PRUNE && (L::GROUPS > 1 || second_test_arg != 0);
+    // (pruning) the search rounds test again before their tail rows.  (With one bound per range instead of one per
+    // 32-neuron group, as the wide fp16 layout first had it, this test lost 12 to 14 % at 64 x 64 and 128 x 128:
+    // most samples passed it and their rows then started late.)
+    constexpr bool SECOND_TEST = PRUNE;
     constexpr int WARPS = THREADS / 32;
     typedef typename L::Scores Scores;
     typedef typename L::Slice Slice;
@@ -622,7 +644,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
         float base_lo[L::GROUPS];
 #pragma unroll
         for (int g = 0; g < L::GROUPS; ++g) base_lo[g] = 0.f;
-        if constexpr (PRUNE) group_min<L>(base, team_lanes, base_lo);
+        if constexpr (PRUNE) group_min<L>(base, team_lanes, q, base_lo);
         for (;;) {
             int chunk = 0;
             if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
@@ -646,15 +668,16 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             if constexpr (PRUNE) {
                 // ---- pruning, before the search loop: find the samples of the chunk that this range can still
                 //      matter to.  A sample survives unless (smallest prefix score of the range for its mask) minus
-                //      (largest weights in this range of all its hot and tail rows) stays above its key, with a
-                //      margin for the rounding of the sums.  Everything else is skipped for this range: a neuron
-                //      of it would have lost the candidate comparison of the search loop, so the result is that
-                //      of the full search bit for bit.  The survivors are then searched four to a round like any
-                //      chunk, with their tail rows in flight early.
-                //      Step 1, by teams as in the search loop: the prefix of every mask that occurs (rows are read
-                //      only where the mask changes) and its smallest score, one float per sample.
-                //      Step 2, a lane per sample (32 samples at a time, all their loads in flight together): the
-                //      bounds of its codes, the test, and the list of survivors in order.
+                //      (largest weights in this range of all its hot and tail rows) stays above its key, per group
+                //      of 32 neurons, with a margin for the rounding of the sums.  Everything else is skipped for
+                //      this range: a neuron of it would have lost the candidate comparison of the search loop, so
+                //      the result is that of the full search bit for bit.  The survivors are then searched four to
+                //      a round like any chunk; a round tests once more before it reads tail rows (see there).
+                //      32 samples of the chunk at a time, the next 32's slots and keys already in flight:
+                //      step 1, by teams as in the search loop: the prefix of the mask and its smallest scores (the
+                //      samples are sorted by mask, so nearly always one mask serves all 32);
+                //      step 2, a lane per sample: the bounds of its codes, the test, and the list of survivors in
+                //      order.
                 const int n_chunk = 4 * rounds;
                 auto to_mask = [&](uint32_t mask) {  // the team's prefix scores and their minima for this mask
                     if (mask == curmask) return;
@@ -666,7 +689,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                         L::sub(base, L::lds(tab_q + b * ROWB));
                     }
                     curmask = mask;
-                    group_min<L>(base, team_lanes, base_lo);
+                    group_min<L>(base, team_lanes, q, base_lo);
                 };
                 // the slot and key of this lane's sample of step p (a step's loads are issued one step ahead)
                 uint4 n0, n1, n2;
@@ -831,7 +854,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 float tail_bound[L::GROUPS];  // (second test) this lane's share of the tail rows' bounds
 #pragma unroll
                 for (int g = 0; g < L::GROUPS; ++g) tail_bound[g] = 0.f;
-                if (!second_test) {
+                if constexpr (!SECOND_TEST) {
                     if (p0) tr0 = SOM_TAIL(lo16(s2.x));
                     if (p1) tr1 = SOM_TAIL(hi16(s2.x));
                     if constexpr (L::TAILS_AHEAD >= 3) {
@@ -893,39 +916,41 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 }
                 const uint32_t t45 = s2.z, t67 = s2.w;  // tail codes 4..7
                 // ---- tail rows ------------------------------------------------------------------
-                if constexpr (PRUNE) {
-                    if (second_test) {
-                        // Second test, now that the scores hold the mask and hot rows exactly: if no neuron of the
-                        // team can get under the sample's key even when every tail row takes its largest weight of
-                        // the neuron's group off, the tail rows (mostly cold: few samples of a batch read a given
-                        // row of this range) are not read at all.  Such a sample offers no candidate either way.
+                if constexpr (SECOND_TEST) {
+                    // Second test, now that the scores hold the mask and hot rows exactly: if no neuron of the
+                    // team can get under the sample's key even when every tail row takes its largest weight of
+                    // the neuron's group off, the tail rows (mostly cold: few samples of a batch read a given
+                    // row of this range) are not read at all.  Such a sample offers no candidate either way.
 #pragma unroll
-                        for (int g = 0; g < L::GROUPS; ++g) {
-                            float t = tail_bound[g];
-                            t += __shfl_xor_sync(team_lanes, t, 1);
-                            t += __shfl_xor_sync(team_lanes, t, 2);
-                            t += __shfl_xor_sync(team_lanes, t, 4);
-                            tail_bound[g] = t;
-                        }
-                        const uint32_t cu2 = (uint32_t)(key0 >> 32);
-                        const float cs2 = __uint_as_float((cu2 & 0x80000000u) ? (cu2 ^ 0x80000000u) : ~cu2);
-                        bool may = false;
-                        float sc[R];
-                        L::unpack(acc, sc);
-                        constexpr int PER = R / L::GROUPS;
-#pragma unroll
-                        for (int g = 0; g < L::GROUPS; ++g) {
-                            float m = sc[g * PER];
-#pragma unroll
-                            for (int j = 1; j < PER; ++j) m = fminf(m, sc[g * PER + j]);
-                            // (an empty key decodes to NaN: the comparison is false and the rows are read)
-                            may = may || !(m - tail_bound[g] > cs2 + 1e-5f * (fabsf(m) + fabsf(cs2) + fabsf(tail_bound[g])));
-                        }
-                        if (!__any_sync(team_lanes, may)) continue;
+                    for (int g = 0; g < L::GROUPS; ++g) {
+                        float t = tail_bound[g];
+                        t += __shfl_xor_sync(team_lanes, t, 1);
+                        t += __shfl_xor_sync(team_lanes, t, 2);
+                        t += __shfl_xor_sync(team_lanes, t, 4);
+                        tail_bound[g] = t;
                     }
+                    const uint32_t cu2 = (uint32_t)(key0 >> 32);
+                    const float cs2 = __uint_as_float((cu2 & 0x80000000u) ? (cu2 ^ 0x80000000u) : ~cu2);
+                    bool may = false;
+                    float sc[R];
+                    L::unpack(acc, sc);
+                    // (the lane's neurons group by group, as in group_min; an empty key decodes to NaN: the
+                    //  comparison is false and the rows are read)
+                    constexpr int SHARES = L::HALF_GROUPS ? L::GROUPS / 2 : L::GROUPS;
+                    constexpr int PER = R / SHARES;
+#pragma unroll
+                    for (int c = 0; c < SHARES; ++c) {
+                        float m = sc[c * PER];
+#pragma unroll
+                        for (int j = 1; j < PER; ++j) m = fminf(m, sc[c * PER + j]);
+                        float tb;
+                        if constexpr (L::HALF_GROUPS) tb = (q & 4) ? tail_bound[2 * c + 1] : tail_bound[2 * c];
+                        else tb = tail_bound[c];
+                        may = may || !(m - tb > cs2 + 1e-5f * (fabsf(m) + fabsf(cs2) + fabsf(tb)));
+                    }
+                    if (!__any_sync(team_lanes, may)) continue;
                     // A step of the warp waits for the slowest of its four teams: the rows are loaded
-                    // as many at a time as the registers allow, not one after the other (the first ones are in
-                    // flight since the round's start, unless they had to wait for the second test).
+                    // as many at a time as the registers allow, not one after the other.
                     constexpr int A = L::TAILS_AHEAD;
                     if (nt == SOM_SLOT_NT_OVERFLOW) {
                         acc = L::worst();  // (never a survivor; see the other branch)
@@ -934,12 +959,10 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
 #pragma unroll
                         for (int b = 0; b < SOM_SLOT_MAX_TAIL; b += A) {
                             if (nt > (uint32_t)b) {
-                                if (b > 0 || second_test) {
 #pragma unroll
-                                    for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
-                                        Slice& t = (j - b == 0) ? tr0 : ((j - b == 1) ? tr1 : ((j - b == 2) ? tr2 : tr3));
-                                        if (nt > (uint32_t)j) t = SOM_TAIL((j & 1) ? hi16(tc[j >> 1]) : lo16(tc[j >> 1]));
-                                    }
+                                for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
+                                    Slice& t = (j - b == 0) ? tr0 : ((j - b == 1) ? tr1 : ((j - b == 2) ? tr2 : tr3));
+                                    if (nt > (uint32_t)j) t = SOM_TAIL((j & 1) ? hi16(tc[j >> 1]) : lo16(tc[j >> 1]));
                                 }
 #pragma unroll
                                 for (int j = b; j < b + A && j < SOM_SLOT_MAX_TAIL; ++j) {
@@ -1100,8 +1123,8 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
     const int feed_keep = h->opt_feed_keep == 1 || (h->opt_feed_keep == 0 && n * 56 <= ((int64_t)24 << 20));
     // Pruning by range maxima, when som_norms has written them.  Measured against the search that reads every row
-    // (fp32 storage, the benchmark's batches): 64 x 64 (32 ranges) 5.28 -> 5.07 ms, 128 x 128 78.2 -> 64.2 ms,
-    // 512 x 512 329 -> 163 ms, 1024 x 1024 368 -> 219 ms; the share of the (sample, range) pairs it skips grows
+    // (fp32 storage, the benchmark's batches): 64 x 64 (32 ranges) 5.28 -> 3.96 ms, 128 x 128 78.2 -> 50.0 ms,
+    // 512 x 512 329 -> 113 ms, 1024 x 1024 368 -> 130 ms; the share of the (sample, range) pairs it skips grows
     // with the number of ranges, because a sample's key tightens as the ranges go by.  Below 32 ranges it is off.
     bool prune = false;
     if constexpr (L::CAN_PRUNE)
@@ -1111,10 +1134,6 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
     //  slower at 512 x 512: it tests against the second-best key, which skips less)
     if (codebook_v != static_cast<const void*>(h->W) && codebook_v != static_cast<const void*>(h->Wh)) prune = false;
-    // second test of the search rounds with one bound per range (wide fp16 layout): measured 12 to 14 % slower at
-    // 64 x 64 and 128 x 128 (most samples pass it and their rows then start late), 11 to 13 % faster at 512 x 512
-    // and 1024 x 1024; on from 1024 ranges
-    const int second_test = (h->M + 127) / 128 >= 1024;
     if (prune) smem += ((size_t)(SOM_PLAN_MASK_FEATURES + n_hot + 1) * L::GROUPS * sizeof(float) + 15) / 16 * 16;  // the table rows' maxima
     auto launch = [&](auto kern) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -1129,8 +1148,7 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
                                           KEEP == 3 ? reinterpret_cast<u64*>(ws + b.keys3) : nullptr, parts, part_len,
                                           n_units, n_whole,
                                           reinterpret_cast<int*>(head + b.n_slots) + 3, h->gate, h->gate_want,
-                                          feed_keep, prune ? h->range_max : nullptr, (int)h->V, prune ? h->range_order : nullptr,
-                                          second_test);
+                                          feed_keep, prune ? h->range_max : nullptr, (int)h->V, prune ? h->range_order : nullptr);
         return cudaGetLastError();
     };
     if constexpr (L::CAN_PRUNE) {
