@@ -83,9 +83,10 @@ int som_create_f16(som_handle** out, int32_t V, int64_t M, const void* d_codeboo
  * accumulated in fp64 in a fixed order (deterministic) and stored as fp32.
  * Must be called once after som_create and again after every codebook update.
  * With M % 128 == 0 the same read also records, for every feature and every range of 128
- * neurons, the largest weight (V * M / 128 floats, allocated by the first call; if that memory cannot be had
- * the call carries on without them).  The search uses them to skip rows that cannot change a sample's result
- * (som_bmu below); they cost the norm pass nothing measurable.
+ * neurons, the largest weight in each of the range's four groups of 32 neurons (V * M / 32 floats, allocated by
+ * the first call; if that memory cannot be had the call carries on without them), and the order of the ranges by
+ * their smallest norm.  The search uses them to skip rows that cannot change a sample's result (som_bmu below);
+ * writing them makes the pass about a fifth longer on the largest map (18 -> 22 ms at 1024 x 1024).
  */
 int som_norms(som_handle* h, void* stream);
 
@@ -120,8 +121,9 @@ int som_norms(som_handle* h, void* stream);
  * of the search of a range of 128 neurons when even the range's smallest partial score over the sample's
  * most frequent features, lowered by the largest weights in the range of its other features, stays above
  * the sample's best score so far, with a margin for fp32 rounding: no neuron of the range can then be
- * the best unit.  The outputs are bit for bit those of the search that forms every row
- * (tests/test_gpu_parity.py forces it both ways).
+ * the best unit.  A sample that stays in is tested once more, with the partial scores of its frequent
+ * features exact for every neuron, before any row of its rare features is read.  The outputs are bit for bit
+ * those of the search that forms every row (tests/test_gpu_parity.py forces it both ways).
  */
 int som_bmu(som_handle* h, const int32_t* d_indptr, const int32_t* d_indices, int64_t n_samples,
             int32_t* d_bmu, float* d_min_dist, void* stream);
