@@ -1106,7 +1106,23 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     constexpr int T = L::T;
     const int64_t n = (n_real + 3) / 4 * 4;  // the plan pads the slot array to whole rounds
     const int n_ranges = (int)((h->M + T - 1) / T);
+    // Pruning by range maxima, when som_norms has written them.  Measured against the search that reads every row
+    // (fp32 storage, the benchmark's batches): 64 x 64 (32 ranges) 5.28 -> 3.96 ms, 128 x 128 78.2 -> 50.0 ms,
+    // 512 x 512 329 -> 113 ms, 1024 x 1024 368 -> 130 ms; the share of the (sample, range) pairs it skips grows
+    // with the number of ranges, because a sample's key tightens as the ranges go by.  Below 32 ranges it is off.
+    bool prune = false;
+    if constexpr (L::CAN_PRUNE)
+        prune = h->range_max != nullptr &&
+                (h->opt_prune == 1 || (h->opt_prune == 0 && (h->M + 127) / 128 >= SOM_PRUNE_MIN_RANGES));
+    // (the maxima are those of the handle's own codebook: the first pass of the two-stage search, which reads
+    //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
+    //  slower at 512 x 512: it tests against the second-best key, which skips less)
+    if (codebook_v != static_cast<const void*>(h->W) && codebook_v != static_cast<const void*>(h->Wh)) prune = false;
     int parts = h->opt_parts > 0 ? (int)h->opt_parts : som_table_default_parts(n, T, L::ROWB);
+    // (with pruning a unit's search is three times shorter on the large maps but its table costs the same: on a
+    //  250k-sample batch 16 parts instead of 44 measure 4 % faster at 512 x 512 and 1024 x 1024; the small maps,
+    //  whose units are few, keep theirs)
+    if (prune && h->opt_parts <= 0 && L::ROWB >= 512 && n >= 200000 && n < 600000 && n_ranges >= 1024) parts = 16;
     if ((int64_t)parts * 1024 > n) parts = (int)(n / 1024);
     if (parts < 1) parts = 1;
     int64_t part_len = (n + parts - 1) / parts;
@@ -1122,18 +1138,6 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     const int n_units = n_whole + 4 * n_split;
     const typename L::Store* codebook = reinterpret_cast<const typename L::Store*>(codebook_v);
     const int feed_keep = h->opt_feed_keep == 1 || (h->opt_feed_keep == 0 && n * 56 <= ((int64_t)24 << 20));
-    // Pruning by range maxima, when som_norms has written them.  Measured against the search that reads every row
-    // (fp32 storage, the benchmark's batches): 64 x 64 (32 ranges) 5.28 -> 3.96 ms, 128 x 128 78.2 -> 50.0 ms,
-    // 512 x 512 329 -> 113 ms, 1024 x 1024 368 -> 130 ms; the share of the (sample, range) pairs it skips grows
-    // with the number of ranges, because a sample's key tightens as the ranges go by.  Below 32 ranges it is off.
-    bool prune = false;
-    if constexpr (L::CAN_PRUNE)
-        prune = h->range_max != nullptr &&
-                (h->opt_prune == 1 || (h->opt_prune == 0 && (h->M + 127) / 128 >= SOM_PRUNE_MIN_RANGES));
-    // (the maxima are those of the handle's own codebook: the first pass of the two-stage search, which reads
-    //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
-    //  slower at 512 x 512: it tests against the second-best key, which skips less)
-    if (codebook_v != static_cast<const void*>(h->W) && codebook_v != static_cast<const void*>(h->Wh)) prune = false;
     if (prune) smem += ((size_t)(SOM_PLAN_MASK_FEATURES + n_hot + 1) * L::GROUPS * sizeof(float) + 15) / 16 * 16;  // the table rows' maxima
     auto launch = [&](auto kern) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -80,6 +80,8 @@ struct SomPlanBuffers {
 //   128-neuron ranges of the wide fp32 layout (512-byte rows, slabs of 15 MB): the fewer ranges are
 //     live the better - 40 to 48 parts on a 250k-sample batch (units of 6,000 samples) are 10 % faster
 //     than 16 on the largest map, 64 to 80 are best on 1M samples, 96 to 128 on 4M samples.
+//     (Those are the figures of the search that reads every row; where it prunes, the launcher takes 16 parts
+//     for batches of that size on the large maps, see launch_table.)
 static inline int som_table_default_parts(int64_t n, int range_neurons, int row_bytes)
 {
     if (row_bytes >= 512) return n < 48 * 1024 ? (n < 1024 ? 1 : (int)(n / 1024)) : (n < 600000 ? 44 : (n < 2500000 ? 64 : 96));
