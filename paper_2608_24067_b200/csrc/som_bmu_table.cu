@@ -951,7 +951,8 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                     if (!__any_sync(team_lanes, may)) continue;
                     // A step of the warp waits for the slowest of its four teams: the rows are loaded
                     // as many at a time as the registers allow, not one after the other.
-                    constexpr int A = L::TAILS_AHEAD;
+                    // (fp32 blocks of more than 640 threads have 80 registers: one row at a time)
+                    constexpr int A = (sizeof(typename L::Store) == 4 && THREADS > 640) ? 1 : L::TAILS_AHEAD;
                     if (nt == SOM_SLOT_NT_OVERFLOW) {
                         acc = L::worst();  // (never a survivor; see the other branch)
                     } else {
@@ -1186,16 +1187,26 @@ SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
     g.T = 8 * g.R;
     const int row_bytes = g.T * (f16 ? 2 : 4);
     // (the fp16 layout holds half as many row registers: 896 threads at 72 registers measured best)
-    const int def_threads = f16 ? (g.R == 16 ? 512 : 896) : (g.R == 16 ? 512 : (g.R == 8 ? 640 : 1024));
+    // fp32, 16 neurons per lane: where the launch prunes (launch_table) its rounds seldom read tail rows, so they
+    // are loaded one at a time, the kernel fits 80 registers and 24 warps hide more of its latency than 16 do:
+    // 768 threads measure 7 % faster than 512 (512 x 512: 103 -> 96 ms).  The search that reads every row keeps
+    // three rows in flight and 512 threads (576 and more spill and measure slower).
+    const bool prunes = !shadow && h->range_max != nullptr &&
+                        (h->opt_prune == 1 || (h->opt_prune == 0 && (h->M + 127) / 128 >= SOM_PRUNE_MIN_RANGES));
+    const int def_threads = f16 ? (g.R == 16 ? 512 : 896) : (g.R == 16 ? (prunes ? 768 : 512) : (g.R == 8 ? 640 : 1024));
     g.threads = (h->opt_threads == 512 || h->opt_threads == 576 || h->opt_threads == 640 || h->opt_threads == 768 ||
                  h->opt_threads == 896 || h->opt_threads == 1024)
                     ? (int)h->opt_threads : def_threads;
     // 227 KB per block, minus the static shared memory (slot rings, norms) of the kernel
     int max_rows = (int)((227 * 1024 - 16 * 1024) / row_bytes) - SOM_PLAN_MASK_FEATURES - 1;
-    // Defaults keep dynamic + static shared memory under 196 KB: one step more and the SM's
-    // carve-out leaves 28 KB instead of 60 KB of L1, which costs 12 % at 128x128 (measured).
+    // Defaults keep dynamic + static shared memory (and the KB that the system reserves per block) under 196 KB: one
+    // step more and the SM's carve-out leaves 28 KB instead of 60 KB of L1, which costs 9 to 12 % (measured at
+    // every map size).  The wide layouts count in the bounds of the table's rows that a pruning launch keeps behind
+    // the table (16 bytes per row) and the rings of a 768-thread block: 334 rows of 512 bytes and 680 of 256
+    // bytes (fp16) are the most that stay below the step; the defaults leave a KB of room.
     int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows
-                                   : (row_bytes == 128 ? (f16 ? 1456 : 1376) : (row_bytes == 512 ? 343 : 720));
+                                   : (row_bytes == 128 ? (f16 ? 1456 : 1376)
+                                                       : (row_bytes == 512 ? 330 : (f16 && g.R == 16 ? 676 : 720)));
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
     g.row_bytes = row_bytes;
@@ -1226,6 +1237,7 @@ static int launch_table_any(som_handle* h, bool shadow, const int32_t* indptr, c
         SOM_TABLE(LayF16, 512);
     }
     if (g.R == 16) {
+        if (g.threads == 768) SOM_TABLE(LayF32<16>, 768);
         if (g.threads == 576) SOM_TABLE(LayF32<16>, 576);
         SOM_TABLE(LayF32<16>, 512);
     }
