@@ -39,7 +39,6 @@
 
 namespace {
 
-constexpr int SOM_PRUNE_MIN_RANGES = 32;  // pruning by range maxima from this many ranges of 128 neurons (see launch_table)
 constexpr int CHUNK = 128;  // samples a warp takes at a time ...
 constexpr int SMALL_CHUNK = 32;  // ... and near the end of a unit, so that its warps finish together
 constexpr int RING_STAGE = 224;  // bytes of one ring stage: 4 slots + 4 keys
@@ -1113,8 +1112,7 @@ int launch_table(som_handle* h, const void* codebook_v, const int32_t* indptr, c
     // with the number of ranges, because a sample's key tightens as the ranges go by.  Below 32 ranges it is off.
     bool prune = false;
     if constexpr (L::CAN_PRUNE)
-        prune = h->range_max != nullptr &&
-                (h->opt_prune == 1 || (h->opt_prune == 0 && (h->M + 127) / 128 >= SOM_PRUNE_MIN_RANGES));
+        prune = som_table_prunes(h);
     // (the maxima are those of the handle's own codebook: the first pass of the two-stage search, which reads
     //  the fp16 copy of an fp32 codebook, does not prune; with the copy's rounding allowed for it measured 3 %
     //  slower at 512 x 512: it tests against the second-best key, which skips less)
@@ -1191,8 +1189,7 @@ SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
     // are loaded one at a time, the kernel fits 80 registers and 24 warps hide more of its latency than 16 do:
     // 768 threads measure 7 % faster than 512 (512 x 512: 103 -> 96 ms).  The search that reads every row keeps
     // three rows in flight and 512 threads (576 and more spill and measure slower).
-    const bool prunes = !shadow && h->range_max != nullptr &&
-                        (h->opt_prune == 1 || (h->opt_prune == 0 && (h->M + 127) / 128 >= SOM_PRUNE_MIN_RANGES));
+    const bool prunes = !shadow && som_table_prunes(h);
     const int def_threads = f16 ? (g.R == 16 ? 512 : 896) : (g.R == 16 ? (prunes ? 768 : 512) : (g.R == 8 ? 640 : 1024));
     g.threads = (h->opt_threads == 512 || h->opt_threads == 576 || h->opt_threads == 640 || h->opt_threads == 768 ||
                  h->opt_threads == 896 || h->opt_threads == 1024)

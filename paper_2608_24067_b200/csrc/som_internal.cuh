@@ -94,6 +94,16 @@ struct som_handle {
     int32_t* host_pair;    // pinned, 4 ints: read-back of indptr[0], indptr[n], covered instances, uncertain samples
 };
 
+// pruning by range maxima in the row-table search: on from this many ranges of 128 neurons (option 10 = 0)
+constexpr int SOM_PRUNE_MIN_RANGES = 32;
+// whether the row-table search over the handle's own codebook prunes (the launcher also wants a layout that can)
+static inline bool som_table_prunes(const som_handle* h)
+{
+    return h->range_max != nullptr &&
+           (h->opt_prune == 1 || (h->opt_prune == 0 && (h->M + 127) / 128 >= SOM_PRUNE_MIN_RANGES));
+}
+
+
 // event slots
 enum { EV_NORMS_BEGIN = 0, EV_NORMS_END, EV_BMU_BEGIN, EV_BMU_PLAN_END, EV_BMU_SEARCH_END, EV_BMU_END };
 

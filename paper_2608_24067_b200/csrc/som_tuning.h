@@ -2,7 +2,7 @@
 // They exist for benchmarking and for the tests that walk every template instance; 0 always means
 // "the measured default".  A reusable plan (som_plan_create) is tied to their values at its creation.
 //
-//   key 1  hot rows kept in shared memory beside the 16 mask rows (default: 343 rows of 512 bytes, 720 of
+//   key 1  hot rows kept in shared memory beside the 16 mask rows (default: 330 rows of 512 bytes, 720 (fp16 wide rows: 676) of
 //          256 bytes, 1376 / 1456 of 128 bytes: what keeps table + slot rings under 196 KB, so that the
 //          SM keeps a 60 KB L1)
 //   key 2  block size: 512, 576 (wide fp32 layout only), 640, 768, 896, 1024
@@ -10,7 +10,8 @@
 //          16 (M % 128 == 0); default: the widest that divides M (fp32 with the two-stage search: 8)
 //   key 4  sample parts per neuron range (default: see som_table_default_parts in som_plan.cuh)
 //   key 8  how many of the 16 most frequent features of a batch are handled as mask bits (1..16); default:
-//          floor(log2(samples)) - 8, at least 4, at most 16 (see plan_split in som_plan.cu)
+//          floor(log2(samples)) - 8, less floor((floor(log2(ranges of 128 neurons)) - 3) / 2) (at most 4) where the
+//          search prunes; at least 4, at most 16 (see plan_split in som_plan.cu)
 //   key 9  slot and key stream loaded with the L2 "evict last" policy: 0 = when the stream is at most 24 MB (then
 //          it stays L2-resident from one neuron range to the next: 1024 x 1024 with 250k samples moves 223 GB
 //          instead of 257 GB and runs 0.4 % faster), 1 = always, 2 = never
