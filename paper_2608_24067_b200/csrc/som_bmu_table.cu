@@ -1200,10 +1200,11 @@ SomTableGeom som_table_geometry(const som_handle* h, bool shadow)
     // step more and the SM's carve-out leaves 28 KB instead of 60 KB of L1, which costs 9 to 12 % (measured at
     // every map size).  The wide layouts count in the bounds of the table's rows that a pruning launch keeps behind
     // the table (16 bytes per row) and the rings of a 768-thread block: 334 rows of 512 bytes and 680 of 256
-    // bytes (fp16) are the most that stay below the step; the defaults leave a KB of room.
+    // bytes (fp16) are the most that stay below the step; the defaults leave a KB of room.  (The fp16 copy that
+    // the two-stage search reads first does not prune, and its plan is also that of the exact pass: 720 rows.)
     int want = h->opt_hot_rows > 0 ? (int)h->opt_hot_rows
                                    : (row_bytes == 128 ? (f16 ? 1456 : 1376)
-                                                       : (row_bytes == 512 ? 330 : (f16 && g.R == 16 ? 676 : 720)));
+                                                       : (row_bytes == 512 ? 330 : (f16 && g.R == 16 && !shadow ? 676 : 720)));
     if (want > max_rows) want = max_rows;
     g.n_hot = want;
     g.row_bytes = row_bytes;
