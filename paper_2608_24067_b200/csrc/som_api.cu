@@ -190,7 +190,7 @@ int som_norms(som_handle* h, void* stream)
     return SOM_OK;
 }
 
-// Samples that do not fit a slot of the row-table plan (more than 12 hot or 8 tail features; the plan
+// Samples that do not fit a slot of the row-table plan (more than 10 tail features, counting the hot features beyond 12 among them; the plan
 // lists them, the row-table kernel skips them): the direct-load kernel searches the list, whose length
 // only the device knows, and their outputs are written last.  Two small launches that return at once
 // when the list is empty.

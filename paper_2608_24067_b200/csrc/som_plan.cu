@@ -265,6 +265,12 @@ k_classify(const int32_t* __restrict__ indptr, const int32_t* __restrict__ indic
             else if (slot < n_mask) mask |= 1u << slot;
             else ++nh;
         }
+        // hot features beyond a slot's twelve go with the tail features (their rows are then read from the
+        // codebook like any tail row) as long as those have room: far fewer samples are left to the list
+        if (nh > (uint32_t)SOM_SLOT_MAX_HOT && nt + (nh - SOM_SLOT_MAX_HOT) <= (uint32_t)SOM_SLOT_MAX_TAIL) {
+            nt += nh - SOM_SLOT_MAX_HOT;
+            nh = SOM_SLOT_MAX_HOT;
+        }
         pk[s] = mask | (nh << 16);
         ntail[s] = nt;
     }
@@ -371,7 +377,7 @@ k_scatter_slots(const int32_t* __restrict__ indptr, const int32_t* __restrict__ 
             const int v = indices[j];
             if ((unsigned)v >= (unsigned)V) continue;
             const int fs = feat_slot[v];
-            if (fs < 0) {
+            if (fs < 0 || (fs >= n_mask && ih >= (uint32_t)SOM_SLOT_MAX_HOT)) {  // tail feature, or a hot one too many
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if ((it >> 1) == (uint32_t)i)
