@@ -469,6 +469,10 @@ def measure(ctx: Ctx, args, w: synth.Workload, steps: int, warmup: int, cpu_seco
             "bound": "alu" if t_alu >= t_hbm else "hbm", "kernel": "fused BMU search",
             "achieved": achieved / 1e12, "peak": add_peak / 1e12,
             "unit": "TFLOP/s", "frac": max(t_alu, t_hbm) / search_s, "traffic": traffic,
+            # achieved and frac count the adds of the plain definition (every row of every sample against every
+            # neuron) over the measured time; where the kernel prunes (bit-identical outputs) it executes only
+            # part of them, so frac is the job done against the add pipe's peak, not the pipe's load, and can pass 1
+            "frac_note": "algorithmic adds of the full product / time; the pruning kernel executes a fraction of them",
             "traffic_note": None if traffic is not None else "not measured at this size; hbm term uses the algorithmic bytes",
             "peak_source": "%d SMs x %d fp32 lanes x %.0f MHz (%s clock); adds only, no multiplies" % (
                 ctx.sm_count, FP32_LANES_PER_SM, ctx.sm_max_mhz, ctx.peak_src),
