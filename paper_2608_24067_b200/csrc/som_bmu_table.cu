@@ -40,6 +40,10 @@
 namespace {
 
 constexpr int CHUNK = 128;  // samples a warp takes at a time ...
+// ... where the launch prunes: 64 (its test takes 32 samples at a time and the search rounds of a chunk are few either
+// way; measured 5 to 7 % faster than 128 at every map size, 32 slower again; the search that reads every row loses 1 %
+// with 64)
+constexpr int PRUNE_CHUNK = 64;
 constexpr int SMALL_CHUNK = 32;  // ... and near the end of a unit, so that its warps finish together
 constexpr int RING_STAGE = 224;  // bytes of one ring stage: 4 slots + 4 keys
 constexpr int SLOT_Q = SOM_SLOT_WORDS / 4;  // uint4 per slot
@@ -529,6 +533,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
     constexpr int R = L::R;
     constexpr int T = L::T;
     constexpr int ROWB = L::ROWB;
+    constexpr int CH = PRUNE ? PRUNE_CHUNK : CHUNK;  // samples a warp takes at a time
     // (pruning) the search rounds test again before their tail rows.  (With one bound per range instead of one per
     // 32-neuron group, as the wide fp16 layout first had it, this test lost 12 to 14 % at 64 x 64 and 128 x 128:
     // most samples passed it and their rows then started late.)
@@ -544,7 +549,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
     // of one round.  The bytes of round r+2 are in flight in registers, round r+1 is being
     // stored, round r is being read: slot and key latency never sits on the critical path.
     __shared__ __align__(16) unsigned char ring_sh[WARPS * 2 * RING_STAGE];
-    __shared__ unsigned char live_sh[PRUNE ? WARPS * CHUNK : 16];  // (pruning) a warp's surviving samples of a chunk
+    __shared__ unsigned char live_sh[PRUNE ? WARPS * CH : 16];  // (pruning) a warp's surviving samples of a chunk
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int q = lane & 7;
@@ -627,15 +632,15 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
         int64_t k_begin = (int64_t)part * part_len;
         int64_t k_end = min(n_pad, k_begin + part_len);  // a multiple of 4
         if (unit >= n_whole) {
-            const int64_t quarter = ((part_len >> 2) + CHUNK - 1) / CHUNK * CHUNK;
+            const int64_t quarter = ((part_len >> 2) + CH - 1) / CH * CH;
             k_begin += (int64_t)((unit - n_whole) & 3) * quarter;
             k_end = min(k_end, k_begin + quarter);
         }
         // full chunks first; the last 64 samples per warp of the unit go out in small chunks
         const int64_t unit_len = k_end > k_begin ? k_end - k_begin : 0;
         const int64_t tail_len = min(unit_len, (int64_t)WARPS * 2 * SMALL_CHUNK);
-        const int n_big = (int)((unit_len - tail_len) / CHUNK);
-        const int64_t small_begin = k_begin + (int64_t)n_big * CHUNK;
+        const int n_big = (int)((unit_len - tail_len) / CH);
+        const int64_t small_begin = k_begin + (int64_t)n_big * CH;
         const int n_chunks = n_big + (int)((k_end - small_begin + SMALL_CHUNK - 1) / SMALL_CHUNK);
 
         uint32_t curmask = 0;
@@ -649,9 +654,9 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             if (lane == 0) chunk = atomicAdd(&next_chunk, 1);
             chunk = __shfl_sync(0xffffffffu, chunk, 0);
             if (chunk >= n_chunks) break;
-            const int64_t w0 = chunk < n_big ? k_begin + (int64_t)chunk * CHUNK
+            const int64_t w0 = chunk < n_big ? k_begin + (int64_t)chunk * CH
                                               : small_begin + (int64_t)(chunk - n_big) * SMALL_CHUNK;
-            const int rounds = (int)(min(k_end, w0 + (chunk < n_big ? CHUNK : SMALL_CHUNK)) - w0) >> 2;
+            const int rounds = (int)(min(k_end, w0 + (chunk < n_big ? CH : SMALL_CHUNK)) - w0) >> 2;
 
             // Ring feed: lanes 0..11 carry the twelve 16-byte pieces of a round's four slots,
             // lanes 12..13 the two 16-byte pieces of its four keys.
@@ -663,7 +668,7 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
             const unsigned char* my_key = ring + 192 + sub * 8;
             int rounds_b = rounds;  // rounds of the search loop below
             int n_live = 0;         // (pruning) survivors of the chunk
-            unsigned char* live_list = live_sh + warp * CHUNK;  // (pruning) positions in the chunk of the samples to search
+            unsigned char* live_list = live_sh + warp * CH;  // (pruning) positions in the chunk of the samples to search
             if constexpr (PRUNE) {
                 // ---- pruning, before the search loop: find the samples of the chunk that this range can still
                 //      matter to.  A sample survives unless (smallest prefix score of the range for its mask) minus
@@ -708,12 +713,12 @@ k_bmu_table(const typename L::Store* __restrict__ W, const float* __restrict__ h
                 };
                 load_step(0);
 #pragma unroll
-                for (int p = 0; p < CHUNK / 32; ++p) {
+                for (int p = 0; p < CH / 32; ++p) {
                     if (32 * p >= n_chunk) break;  // (the same for every lane)
                     const int pos = lane + 32 * p;
                     const uint4 s0 = n0, s1 = n1, s2 = n2;
                     const u64 key0 = nkey;
-                    if (p + 1 < CHUNK / 32 && 32 * (p + 1) < n_chunk) load_step(p + 1);
+                    if (p + 1 < CH / 32 && 32 * (p + 1) < n_chunk) load_step(p + 1);
                     const uint32_t hdr = s0.x;
                     float lo[L::GROUPS];
                     // Step 1.  The samples are sorted by mask, so nearly always the 32 of this step share one: then
